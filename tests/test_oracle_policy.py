@@ -1,0 +1,219 @@
+"""Pins for oracle.policy: brute force, the paper's closed forms, bounds and ordering claims."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import bruteforce as BF
+from oracle import policy as P
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_policy_facts.txt")
+
+
+# ---------------------------------------------------------------- brute force
+@pytest.mark.parametrize("t", range(1, 9))
+def test_hsm_ism_match_unrestricted_search(t):
+    C, _ = P.hsm_tables(t, t + 2)
+    Ci, _ = P.ism_tables(t, t + 2)
+    for m in range(1, t + 3):
+        assert BF.hsm_unrestricted(t, m) == C[t, m], (t, m)
+        assert BF.ism_unrestricted(t, m) == Ci[t, m], (t, m)
+
+
+@pytest.mark.parametrize("alpha,beta", [(2, None), (3, None), (4, None), (5, None),
+                                        (4, 3), (3, 2), (2, 1), (4, 2)])
+def test_msm_matches_protocol_enumeration(alpha, beta):
+    for t in range(1, 8):
+        mm = alpha * t + 1
+        C = P.msm_tables(t, mm, alpha, beta)[0]
+        for m in range(1, mm + 1):
+            assert BF.msm_protocol(t, m, alpha, beta) == C[t, m], (t, m)
+
+
+def test_bruteforce_detects_planted_mistakes():
+    """A wrong index or a dropped term in the recursion must disagree with the search."""
+    def hsm_wrong(t_max, m_max, variant):
+        C = np.full((t_max + 1, m_max + 1), P.INF, dtype=np.int64)
+        C[1, 1:] = 1
+        for t in range(1, t_max + 1):
+            C[t, 1] = t * (t + 1) // 2
+        for m in range(2, m_max + 1):
+            for t in range(2, t_max + 1):
+                best = P.INF
+                for y in range(1, t):
+                    if variant == "no_y":
+                        q = C[t - y, m - 1] + C[y, m]
+                    elif variant == "swap_m":
+                        q = y + C[t - y, m] + C[y, m - 1]
+                    else:  # right part keeps the full budget
+                        q = y + C[t - y, m] + C[y, m] if t - y < t else P.INF
+                    best = min(best, q)
+                C[t, m] = best
+        return C
+    for variant in ("no_y", "swap_m"):
+        C = hsm_wrong(7, 5, variant)
+        bad = [(t, m) for t in range(2, 8) for m in range(2, 6)
+               if BF.hsm_unrestricted(t, m) != C[t, m]]
+        assert bad, variant
+
+
+# ---------------------------------------------------------------- closed forms
+def test_hsm_boundaries():
+    C, D = P.hsm_tables(120, 130)
+    for t in range(1, 121):
+        assert C[t, 1] == t * (t + 1) // 2                    # Section 3.1
+        for m in range(t, 131):
+            assert C[t, m] == 2 * t - 1                       # Section 3.1
+        assert all(C[1, 1:] == 1)
+    # Algorithm 1 sets D = 1 in the plentiful regime: it must be *an* argmin there
+    for t in range(2, 60):
+        for m in (t, t + 3):
+            assert 1 + C[t - 1, m - 1] + C[1, m] == C[t, m]
+
+
+def test_ism_boundaries():
+    C, _ = P.ism_tables(120, 130)
+    assert all(C[0, :] == 0)
+    for t in range(1, 121):
+        assert C[t, 1] == t * (t + 1) // 2                    # Section 3.2
+        assert C[t, 0] >= P.INF
+        for m in range(t, 131):
+            assert C[t, m] == t                               # Section 3.2
+        if t >= 2:
+            assert C[t, t - 1] > t
+
+
+@pytest.mark.parametrize("alpha", [2, 4, 5])
+def test_msm_boundaries(alpha):
+    t_max = 40
+    C, H, D1, D2 = P.msm_tables(t_max, alpha * t_max + 2, alpha)
+    for t in range(1, t_max + 1):
+        assert C[t, 1] == t * (t + 1) // 2                    # Section 3.3
+        for m in range(alpha * t, alpha * t_max + 3):
+            assert C[t, m] == t                               # Section 3.3
+        assert C[1, 1] == 1
+    # the smallest budget that reaches C = t
+    for t in range(2, t_max + 1):
+        sat = P.saturation_budget(P.MSM, t, alpha)
+        assert C[t, sat] == t and C[t, sat - 1] > t
+
+
+def test_golden_facts_from_the_paper():
+    cache = {}
+    n = 0
+    for line in open(GOLDEN):
+        line = line.split("#")[0].split()
+        if not line:
+            continue
+        mode, rel, t, m, val = line[0], line[1], int(line[2]), int(line[3]), int(line[4])
+        key = (mode, t, m)
+        if key not in cache:
+            if mode == "hsm":
+                cache[key] = int(P.hsm_tables(t, m)[0][t, m])
+            elif mode == "ism":
+                cache[key] = int(P.ism_tables(t, m)[0][t, m])
+            else:
+                cache[key] = int(P.msm_tables(t, m, int(mode[3:]))[0][t, m])
+        c = cache[key]
+        assert (c == val) if rel == "eq" else (c <= val), (mode, rel, t, m, val, c)
+        n += 1
+    assert n >= 10
+
+
+# ---------------------------------------------------------------- bounds of Section 3.5 / App. B
+def test_hsm_upper_bounds_and_monotonicity():
+    t_max, m_max = 400, 40
+    C, _ = P.hsm_tables(t_max, m_max)
+    for m in range(1, m_max + 1):
+        col = C[1:, m]
+        assert np.all(np.diff(col) > 0)                        # increasing in t (App. B.2)
+        for t in range(1, t_max + 1):
+            bound = t ** (1.0 + 1.0 / m)
+            assert C[t, m] <= m * bound + 1e-9                 # Proposition 1
+            if m >= 2 or t < 8:
+                assert C[t, m] < 4 * bound                     # numerical claim of Section 3.5
+    # more memory never hurts
+    assert np.all(np.diff(C[1:, 1:], axis=1) <= 0)
+    # short-sequence regime: C <= (a + 1) t whenever t <= m^a / a!
+    for m in range(2, m_max + 1):
+        for a in range(1, 5):
+            lim = m ** a / math.factorial(a)
+            for t in range(1, t_max + 1):
+                if t <= lim:
+                    assert C[t, m] <= (a + 1) * t, (t, m, a)
+
+
+def test_ism_short_sequence_bound():
+    t_max, m_max = 300, 30
+    C, _ = P.ism_tables(t_max, m_max)
+    for m in range(2, m_max + 1):
+        for a in range(1, 5):
+            lim = m ** a / math.factorial(a)
+            for t in range(1, t_max + 1):
+                if t <= lim:
+                    assert C[t, m] <= a * t, (t, m, a)         # App. B.3
+    assert np.all(np.diff(C[:, 1:], axis=0) > 0)
+    assert np.all(np.diff(C[1:, 1:], axis=1) <= 0)
+
+
+def test_ordering_of_the_three_schemes():
+    """Section 3.6 and the caption of the ISM/MSM cost figure, alpha = 5."""
+    alpha, t_max = 5, 300
+    m_hid = 50
+    Ch, _ = P.hsm_tables(t_max, m_hid)
+    Ci, _ = P.ism_tables(t_max, m_hid // alpha)
+    Cm = P.msm_tables(t_max, m_hid, alpha)[0]
+    for t in range(1, t_max + 1):
+        for m in (5, 10, 25, 50):
+            assert Cm[t, m] <= Ch[t, m]
+            assert Cm[t, m] <= Ci[t, m // alpha]
+    # hidden states win for long sequences, internal states for short ones
+    assert Ci[50, 10] < Ch[50, 50]
+    Ch1000 = P.hsm_tables(1000, 50)[0]
+    Ci1000 = P.ism_tables(1000, 10)[0]
+    assert Ch1000[1000, 50] < Ci1000[1000, 10]
+
+
+# ---------------------------------------------------------------- argmin validity, protocol simulation
+def test_tables_are_self_consistent():
+    t_max, m_max, alpha = 60, 40, 4
+    C, D = P.hsm_tables(t_max, m_max)
+    for t in range(2, t_max + 1):
+        for m in range(2, m_max + 1):
+            y = D[t, m]
+            assert 1 <= y < t and y + C[t - y, m - 1] + C[y, m] == C[t, m]
+    C, D = P.ism_tables(t_max, m_max)
+    for t in range(1, t_max + 1):
+        for m in range(1, m_max + 1):
+            y = D[t, m]
+            assert 1 <= y <= t and y + C[y - 1, m] + C[t - y, m - 1] == C[t, m]
+
+
+CASES = [(P.HSM, 1, 1), (P.HSM, 2, 1), (P.HSM, 7, 1), (P.HSM, 64, 8), (P.HSM, 50, 50),
+         (P.HSM, 33, 2), (P.HSM, 100, 5), (P.ISM, 1, 1), (P.ISM, 64, 8), (P.ISM, 40, 40),
+         (P.ISM, 40, 1), (P.ISM, 100, 3), (P.MSM, 1, 1), (P.MSM, 64, 8), (P.MSM, 64, 31),
+         (P.MSM, 30, 117), (P.MSM, 30, 1), (P.MSM, 100, 10)]
+
+
+@pytest.mark.parametrize("mode,t,m", CASES)
+def test_protocol_simulation_costs_exactly_C(mode, t, m):
+    tabs = P.plan_tables(mode, t, m, alpha=4)
+    sim = P.simulate(mode, t, m, tabs)
+    assert sim["forwards"] == int(tabs["C"][t, m])
+    assert sim["peak_units"] <= m
+    assert [op[1] for op in sim["ops"] if op[0] == "B"] == list(range(t, 0, -1))
+
+
+def test_protocol_simulation_with_beta():
+    for t, m in [(20, 7), (50, 12), (30, 90)]:
+        tabs = P.plan_tables(P.MSM, t, m, alpha=4, beta=3)
+        sim = P.simulate(P.MSM, t, m, tabs)
+        assert sim["forwards"] == int(tabs["C"][t, m])
+        assert sim["peak_units"] <= m
+        assert int(tabs["C"][t, m]) <= P.cost(P.MSM, t, m, alpha=4)
+
+
+def test_infeasible_budget_is_rejected():
+    with pytest.raises(P.ProtocolError):
+        P.simulate(P.ISM, 5, 0)
