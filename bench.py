@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark: LSTM BPTT sequence-steps/s under a memory budget m, on synthetic workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--mode msm] [--m 100]
+    python bench.py --impl reference ...      # times the fp64 CPU oracle instead
+
+A "step" is one whole training step: every forward, recomputed forward and backward operation
+the plan dictates over the workload's t time steps.  One JSON line is printed by rank 0.
+
+* value / ms_per_step: device-resident inputs, CUDA events around each step.
+* e2e: the same step through the host-buffer entry point, host<->device copies included.
+* roofline: the gate contraction of the forward operation, flops per operation over the
+  measured duration of one forward operation (see --help of the fields in the design doc).
+* cpu_baseline: the oracle on the host cores, on a truncated sequence.
+* budgets: the other budgets of the workload, with the time ratio against full-memory BPTT
+  beside the paper's model (C/t + 2) / 3.
+
+With several GPUs every rank runs an independent replica of the workload (the recurrence does
+not shard; no collective is on the data path) and the job's value is the sum.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOADS = {
+    # name: (mode, headline m, other budgets)
+    "c1": ("hsm", 8, []),
+    "c2": ("hsm", 64, [("hsm", 16), ("hsm", 256), ("ism", 16), ("ism", 64), ("ism", 256)]),
+    "c3": ("msm", 100, [("msm", 10), ("msm", 32), ("msm", 1000)]),
+    "c4": ("ism", 50, [("ism", 20), ("ism", 200), ("msm", 80), ("msm", 200), ("msm", 800)]),
+    "c5": ("msm", 341, [("msm", 1365), ("msm", 5461)]),
+    "p0": ("hsm", 100, [("hsm", 10), ("hsm", 50), ("hsm", 500), ("hsm", 1000)]),
+}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS))
+    ap.add_argument("--mode", default=None)
+    ap.add_argument("--m", type=int, default=None)
+    ap.add_argument("--t", type=int, default=None, help="override the sequence length")
+    ap.add_argument("--no-budgets", action="store_true", help="skip the other budgets")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thr = threading.Thread(target=self._read, daemon=True)
+            self.thr.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1]))
+                mx = float(r[2])
+                for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                                  ("sw_power_cap", 8)):
+                    if r[col].lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        busy = [v for v in sm if mx and v > 0.3 * mx] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(cfg, seconds: float):
+    """Time the oracle, as it stands, on a truncated copy of the workload."""
+    from oracle import lstm_bptt as O
+    from paper_1606_03401_b200 import synth
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count()
+    t_s, dt, tried = 2, 0.0, []
+    while True:
+        c = synth.with_overrides(cfg, t=t_s)
+        pr = synth.make_problem(c)
+        t0 = time.perf_counter()
+        O.lstm_bptt(pr["W"], pr["b"], pr["W_out"], pr["b_out"], pr["x"], pr["targets"], pr["h0"], pr["c0"])
+        dt = time.perf_counter() - t0
+        tried.append((t_s, dt))
+        if dt >= seconds / 3 or t_s >= cfg.t:
+            break
+        t_s = min(cfg.t, max(t_s * 2, int(t_s * seconds / max(dt, 1e-3) * 0.8)))
+    return {"value": t_s / dt, "unit": "seq-steps/s", "cores": cores, "kind": "oracle",
+            "sample": f"fp64 full-memory BPTT of the same layer sizes on the first {t_s} of {cfg.t} time steps "
+                      f"({dt:.1f} s; cost per step is constant in t)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1606_03401_b200 import synth
+    cfg = synth.CONFIGS[args.workload]
+    if args.t:
+        cfg = synth.with_overrides(cfg, t=args.t)
+    per = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals = []
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(cfg, per)
+        if i >= args.warmup:
+            vals.append(r)
+    v = statistics.mean(x["value"] for x in vals)
+    mode, m, _ = WORKLOADS[args.workload]
+    line = {"impl": "reference", "metric": "lstm_bptt_seq_steps_per_s", "value": v, "unit": "seq-steps/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.t / v,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: L{cfg.layers} I{cfg.input} H{cfg.hidden} B{cfg.batch} t{cfg.t}",
+                       "mode": "full-memory BPTT (oracle)", "m": None},
+            "cpu_baseline": {"value": v, "unit": "seq-steps/s", "cores": vals[-1]["cores"], "kind": "oracle",
+                             "sample": vals[-1]["sample"]},
+            "e2e": {"value": v, "unit": "seq-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1606_03401_b200 import binding as B
+    from paper_1606_03401_b200 import harness, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cfg = synth.CONFIGS[args.workload]
+    if args.t:
+        cfg = synth.with_overrides(cfg, t=args.t)
+    cfg = synth.with_overrides(cfg, seed=cfg.seed + 1000 * rank)   # independent replicas
+    mode0, m0, others = WORKLOADS[args.workload]
+    mode = args.mode or mode0
+    m = args.m or m0
+
+    dp = harness.DeviceProblem(cfg, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
+    stream = torch.cuda.current_stream()
+
+    def timed(plan, steps, warmup, sample_clocks=False):
+        for _ in range(warmup):
+            dp.enqueue(plan)
+        sampler = ClockSampler(local) if sample_clocks else None
+        barrier()
+        if sampler:
+            sampler.start()
+        evs = []
+        for _ in range(steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            dp.enqueue(plan)
+            e1.record(stream)
+            evs.append((e0, e1))
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        ms = [a.elapsed_time(b) for a, b in evs]
+        return sum(ms) / len(ms), clocks
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        tns = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(tns, op=dist.ReduceOp.MAX)
+        return float(tns.item())
+
+    plan = dp.plan(mode, m)
+    full = dp.full_memory_plan()
+    W = max(3, args.warmup)
+    ms, clocks = timed(plan, args.steps, W, sample_clocks=True)
+    ms = max_over_ranks(ms)
+    counters = dp.out["counters"].cpu().numpy()
+    assert int(counters[0]) == plan.cost and int(counters[3]) == 0, counters
+
+    # full-memory BPTT: the denominator of the time ratio, and (by difference) the duration of
+    # one forward operation
+    ms_full, _ = timed(full, max(2, args.steps // 2), 2)
+    ms_full = max_over_ranks(ms_full)
+    K = cfg.input + cfg.hidden
+    flops_fwd_op = 0
+    for l in range(cfg.layers):
+        K_l = (cfg.input if l == 0 else cfg.hidden) + cfg.hidden
+        flops_fwd_op += 2 * cfg.batch * K_l * 4 * cfg.hidden
+    pk = peaks()
+    extra_ops = plan.cost - cfg.t
+    if extra_ops > 0 and ms > ms_full:
+        fwd_op_ms = (ms - ms_full) / extra_ops
+    else:
+        fwd_op_ms = None
+    achieved = flops_fwd_op / (fwd_op_ms * 1e-3) / 1e12 if fwd_op_ms else None
+    peak_tf = pk["bf16_tflops_sustained"] if cfg.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2.0
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": (achieved / peak_tf) if achieved else None, "traffic": None,
+                "kernel": "forward operation (gate contraction + fused cell update)",
+                "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
+                       f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
+                       + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}
+
+    budgets = []
+    if not args.no_budgets and rank == 0 or (not args.no_budgets and world > 1):
+        for omode, om in others:
+            op = dp.plan(omode, om)
+            oms, _ = timed(op, max(2, args.steps // 2), 1)
+            oms = max_over_ranks(oms)
+            budgets.append({"mode": omode, "m": om, "C": op.cost, "ms_per_step": oms,
+                            "seq_steps_per_s": world * cfg.t / (oms * 1e-3),
+                            "ratio_vs_full": oms / ms_full, "paper_model_ratio": (op.cost / cfg.t + 2) / 3,
+                            "arena_bytes": op.arena_units * B.mebptt_lstm_unit_bytes(dp.desc)})
+
+    # end to end: host buffers in, host buffers out
+    e2e = None
+    if not args.no_e2e:
+        h = dp.host
+        pin = {k: torch.from_numpy(v.view(np.int16) if v.dtype == np.uint16 else v).pin_memory() for k, v in h.items()}
+        outs = {k: torch.empty(v.numel(), dtype=v.dtype).pin_memory() for k, v in dp.out.items() if v is not None}
+        hws = torch.empty(B.mebptt_lstm_host_workspace_bytes(dp.desc, plan), dtype=torch.uint8, device=dev)
+        h2d = sum(v.numel() * v.element_size() for v in pin.values())
+        d2h = sum(v.numel() * v.element_size() for v in outs.values())
+
+        def e2e_step():
+            B.mebptt_lstm_train_step_host(dp.desc, plan, pin["W"], pin["b"], pin["W_out"], pin["b_out"], pin["x"],
+                                          pin["targets"], pin["h0"], pin["c0"], hws, stream.cuda_stream,
+                                          outs["loss"], outs["dW"], outs["db"], outs["dW_out"], outs["db_out"],
+                                          None, outs["counters"])
+        e2e_step()
+        barrier()
+        n_e2e = max(2, args.steps // 2)
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()
+            torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / n_e2e
+        dt = max_over_ranks(dt)
+        e2e = {"value": world * cfg.t / dt, "unit": "seq-steps/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3}
+        del hws
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = oracle_sample(synth.with_overrides(cfg, seed=cfg.seed), args.cpu_seconds)
+
+    if rank == 0:
+        unit = B.mebptt_lstm_unit_bytes(dp.desc)
+        line = {
+            "metric": "lstm_bptt_seq_steps_per_s", "value": world * cfg.t / (ms * 1e-3), "unit": "seq-steps/s",
+            "n_gpus": world, "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: L{cfg.layers} I{cfg.input} H{cfg.hidden} B{cfg.batch} t{cfg.t} O{cfg.readout}",
+                       "mode": mode, "m": plan.m, "alpha": plan.alpha, "C": plan.cost,
+                       "train_steps_per_s": world / (ms * 1e-3),
+                       "ratio_vs_full": ms / ms_full, "paper_model_ratio": (plan.cost / cfg.t + 2) / 3,
+                       "full_memory_ms": ms_full,
+                       "arena_bytes": plan.arena_units * unit,
+                       "working_bytes_outside_budget": B.mebptt_lstm_working_bytes(dp.desc, plan),
+                       "full_memory_arena_bytes": full.arena_units * unit,
+                       "l2": "256 MiB buffer written between timed steps; x alone (131 MB at c3) exceeds L2",
+                       "replicas": world, "budgets": budgets},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * B.mebptt_lstm_launch_count(dp.desc, plan),
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

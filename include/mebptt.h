@@ -1,0 +1,273 @@
+/*
+ * mebptt.h -- memory-efficient backpropagation through time for LSTMs on one GPU.
+ *
+ * C interface of libmebptt.  Two groups of calls:
+ *
+ *   1. Planning (host only, no CUDA): solve the dynamic programs of the paper for a sequence
+ *      of length t and a memory budget m, in one of three schemes -- hidden-state
+ *      memorisation (BPTT-HSM, Section 3.1), internal-state memorisation (BPTT-ISM,
+ *      Section 3.2) or mixed memorisation (BPTT-MSM, Sections 3.3 and 3.4) -- and unroll the
+ *      execution protocol (Algorithm 2; Section 3.2 steps 1-4) into a linear tape.
+ *
+ *   2. Execution (device): one LSTM training step -- forward steps, recomputed forward
+ *      steps and backward steps in the order of the tape -- producing the loss and the
+ *      gradients of ordinary BPTT (Section 2.1) while holding no more than the budget.
+ *
+ * Conventions
+ *   - Every function returns an int status (MEBPTT_OK = 0, errors < 0) unless it returns a
+ *     value that cannot fail.  Nothing aborts, nothing throws.
+ *   - The library never allocates device memory.  The caller owns all device buffers and a
+ *     workspace whose size mebptt_lstm_workspace_bytes() reports.  Plans are host objects
+ *     owned by the library and released with mebptt_plan_free().
+ *   - Device work is enqueued on the caller's stream and the call returns without waiting.
+ *     Errors that only the device can see are written to counters[3].
+ *   - All matrices are dense and row-major.
+ *
+ * Units of the budget m (they differ by scheme, as in the paper)
+ *   - HSM, MSM: m counts hidden states.  The start state (h0, c0) is one of them; the single
+ *     working RNN core is not (Section 3.1: C(t, m) = 2t - 1 needs m >= t).
+ *   - ISM: m counts internal states, the one being worked on included; the initial hidden
+ *     state is free (Section 3.2: C(t, m) = t needs m >= t).
+ *   - An internal state takes alpha hidden-state units (beta when its input hidden state is
+ *     already stored and the Section 3.4 variant is on).  For the LSTM layouts of this
+ *     library alpha = 4 and beta = 3 (see mebptt_lstm_desc).
+ */
+#ifndef MEBPTT_H
+#define MEBPTT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- enumerations ------------------------------------------------------------------ */
+enum { MEBPTT_HSM = 0, MEBPTT_ISM = 1, MEBPTT_MSM = 2 };
+
+enum {
+  MEBPTT_OK = 0,
+  MEBPTT_ERR_ARG = -1,         /* null pointer, non-positive size, unknown enum value       */
+  MEBPTT_ERR_BUDGET = -2,      /* m < 1: no policy exists                                   */
+  MEBPTT_ERR_WORKSPACE = -3,   /* workspace missing, misaligned (256 B) or too small         */
+  MEBPTT_ERR_UNSUPPORTED = -4, /* shape / precision / plan this build cannot run             */
+  MEBPTT_ERR_CUDA = -5,        /* a CUDA runtime call failed                                 */
+  MEBPTT_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (reported in counters)  */
+  MEBPTT_ERR_OOM = -7,         /* host allocation failed                                     */
+  MEBPTT_ERR_PLAN = -8         /* tape failed validation                                     */
+};
+
+enum { MEBPTT_FP32 = 0, MEBPTT_TF32 = 1, MEBPTT_BF16 = 2 };
+
+/* ---- the tape ---------------------------------------------------------------------- */
+/*
+ * Algorithm 2 recurses on (t, m, s); its shape depends on the tables only, never on data, so
+ * it is unrolled once into a list of operations.  Two kinds exist:
+ *
+ *   MEBPTT_OP_FWD  one forward operation (the unit of cost, Section 3.1): reads the hidden
+ *                  state of step k-1 at location `src`, writes the state of step k at `dst`.
+ *                  dst_fmt tells what is written: MEBPTT_FMT_HIDDEN (h_k, c_k only),
+ *                  MEBPTT_FMT_INTERNAL (the whole internal state of Definition 3) or
+ *                  MEBPTT_FMT_INTERNAL_NOINPUT (the same without the copy of the input hidden
+ *                  state, Section 3.4).
+ *   MEBPTT_OP_BWD  one backward operation over step k: reads the internal state at `src`
+ *                  (and, for FMT_INTERNAL_NOINPUT, the hidden state of step k-1 at `aux`).
+ *
+ * Locations: >= 0 is an offset, in hidden-state units, into the slot arena (a stack: states are
+ * read in the reverse order of writing, Section 3.1); negative values name buffers outside the
+ * budget: the caller's initial state, the two scratch hidden states a forward sweep alternates
+ * between, and the working core (Section 3.1: "a single RNN core available for the purposes of
+ * intermediate calculations").  A memorisation is therefore not a copy: the forward operation
+ * that produces the state writes it where it will be kept (Push), and the next forward
+ * operation reads it from there (Peek).
+ */
+enum { MEBPTT_OP_FWD = 1, MEBPTT_OP_BWD = 2 };
+enum { MEBPTT_FMT_HIDDEN = 0, MEBPTT_FMT_INTERNAL = 1, MEBPTT_FMT_INTERNAL_NOINPUT = 2 };
+enum { MEBPTT_LOC_INIT = -1, MEBPTT_LOC_PING = -2, MEBPTT_LOC_PONG = -3, MEBPTT_LOC_CORE = -4 };
+
+typedef struct {
+  int32_t kind;     /* MEBPTT_OP_FWD or MEBPTT_OP_BWD                          */
+  int32_t k;        /* time step, 1 .. t                                       */
+  int32_t src;      /* location read                                           */
+  int32_t dst;      /* FWD: location written; BWD: unused (0)                  */
+  int32_t dst_fmt;  /* FWD: MEBPTT_FMT_*; BWD: format of the record at src     */
+  int32_t aux;      /* BWD with FMT_INTERNAL_NOINPUT: location of state k-1    */
+  int32_t units;    /* arena units in use (paper's accounting) after this op   */
+  int32_t reserved;
+} mebptt_op;
+
+/* ---- planning ---------------------------------------------------------------------- */
+typedef struct mebptt_plan mebptt_plan_t; /* opaque, host memory, library-owned */
+
+/*
+ * Solve the DP for (t, m, mode) and build the tape.
+ *   HSM: Eqs. (1)-(3) with C(t,1) = t(t+1)/2, C(1,m) = 1            (Section 3.1, Algorithm 1)
+ *   ISM: Eqs. (4)-(5) with C(0,m) = 0                               (Section 3.2)
+ *   MSM: Eqs. (6)-(9) with C(0,.) = 0, C(t>0, m<=0) = inf           (Section 3.3)
+ * alpha = 4, the Section 3.4 variant off.  argmin ties: smallest y (Algorithm 1 scans upward
+ * with a strict <); hidden state before internal state.
+ * t >= 1.  m < 1 gives MEBPTT_ERR_BUDGET.  m above the point where the cost stops falling
+ * (t for HSM/ISM, alpha (t-1) + 1 for MSM) is clamped to it: same policy, same cost.
+ * *out receives the plan; the caller releases it with mebptt_plan_free.
+ */
+int mebptt_plan(int64_t t, int64_t m, int mode, mebptt_plan_t **out);
+
+/*
+ * As above with explicit alpha >= 2 (Section 3.3) and beta: 0 switches the Section 3.4 variant
+ * off, 1 <= beta <= alpha switches it on (Eq. (10): an internal state pushed at y = 1 is charged
+ * beta units because its input hidden state is the stored start state).  Ignored for HSM; ISM
+ * uses alpha only to size its slots.
+ */
+int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_plan_t **out);
+
+void mebptt_plan_free(mebptt_plan_t *plan);
+
+/* C(t, m): the predicted number of forward operations (Section 3.1). */
+int64_t mebptt_plan_cost(const mebptt_plan_t *plan);
+/* Number of tape entries: C(t, m) forward + t backward operations. */
+int64_t mebptt_plan_num_ops(const mebptt_plan_t *plan);
+/* The tape (host memory, valid until mebptt_plan_free). */
+const mebptt_op *mebptt_plan_tape(const mebptt_plan_t *plan);
+/* Peak memory in the paper's units for this scheme (see "Units" above); <= m. */
+int64_t mebptt_plan_peak_units(const mebptt_plan_t *plan);
+/* Hidden-state units the slot arena must physically hold (the caller's start state is read in
+ * place, so this is peak - 1 for HSM/MSM and alpha * peak for ISM). */
+int64_t mebptt_plan_arena_units(const mebptt_plan_t *plan);
+/* Parameters after clamping. */
+int64_t mebptt_plan_t_len(const mebptt_plan_t *plan);
+int64_t mebptt_plan_m(const mebptt_plan_t *plan);
+int mebptt_plan_mode(const mebptt_plan_t *plan);
+int mebptt_plan_alpha(const mebptt_plan_t *plan);
+int mebptt_plan_beta(const mebptt_plan_t *plan);
+
+/*
+ * Borrowed pointers to the DP tables, row-major [t_dim][m_dim] with t_dim = t + 1 and
+ * m_dim = m + 1 (row / column 0 included).  C: costs, MEBPTT_INF where infeasible.
+ * D: position of the first push (HSM, ISM: Eq. (3), (5); MSM: D1 of Eq. (8)).
+ * D2, H: MSM only (Eq. (8), (9); H is 1 = hidden, 2 = internal), NULL otherwise.
+ * Any output pointer may be NULL.
+ */
+#define MEBPTT_INF ((int64_t)1 << 60)
+int mebptt_plan_tables(const mebptt_plan_t *plan, const int64_t **C, const int32_t **D,
+                       const int32_t **D2, const uint8_t **H, int64_t *t_dim, int64_t *m_dim);
+
+/*
+ * Replay the tape on the host with integer bookkeeping: every forward operation must find
+ * its input state, every backward operation its internal state, live states are never
+ * overwritten, backward operations come in the order t .. 1, the forward count equals
+ * C(t, m) and the units in use never exceed m.  MEBPTT_OK or MEBPTT_ERR_PLAN.
+ * mebptt_plan() already ran it; the call exists for tapes' users and tests.
+ */
+int mebptt_plan_validate(const mebptt_plan_t *plan);
+
+/* ---- execution --------------------------------------------------------------------- */
+/*
+ * A stack of `layers` LSTM cells without peepholes (the paper names the LSTM, Section 4,
+ * without printing it), gate order i, f, g, o:
+ *     z = W [in_t ; h_{t-1}] + b,  i,f,o = sigmoid, g = tanh,
+ *     c_t = f c_{t-1} + i g,  h_t = o tanh(c_t),
+ * in_t = x_t for layer 0 and the h_t of the layer below otherwise; the RNN core of
+ * Definition 1 is the whole stack at one time step and its hidden state (Definition 2) is
+ * (h, c) of every layer.  On top: y_t = W_out h_t + b_out (last layer) and the loss
+ *     L = sum_t 1/(batch*readout) sum (y_t - target_t)^2,
+ * a sum of per-step terms as Algorithm 2 requires (the output gradient is asked for at each
+ * step).
+ *
+ * dtype selects storage and arithmetic:
+ *   MEBPTT_FP32  everything float32, FMA arithmetic.
+ *   MEBPTT_TF32  everything stored as float32; contractions on tensor cores.
+ *   MEBPTT_BF16  operands (W, W_out, x, h0 and every stored h and gate) bfloat16; b, b_out,
+ *                targets, c0, every stored c, all accumulation and all gradients float32.
+ * With these layouts an internal state (h_t, c_t, the four gates, h_{t-1}, c_{t-1}) fits in
+ * alpha = 4 hidden-state units, beta = 3 without the input hidden state; plans made with a
+ * smaller alpha are refused (MEBPTT_ERR_UNSUPPORTED).
+ */
+typedef struct {
+  int32_t layers;   /* >= 1                                           */
+  int32_t input;    /* I: width of x_t                                */
+  int32_t hidden;   /* H: per layer                                   */
+  int32_t readout;  /* O: width of y_t and of the targets             */
+  int32_t batch;    /* B                                              */
+  int32_t dtype;    /* MEBPTT_FP32 | MEBPTT_TF32 | MEBPTT_BF16        */
+  int32_t want_dx;  /* 1: also return dL/dx                           */
+  int32_t reserved; /* 0                                              */
+  int64_t t;        /* sequence length; must equal the plan's         */
+} mebptt_lstm_desc;
+
+/* Bytes of one hidden-state unit (all layers) for this descriptor; 0 on a bad descriptor. */
+size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc *desc);
+
+/* Budget given in bytes -> hidden-state units (floor); the working memory outside the budget
+ * is not counted (Section 3.1 sets the working core apart). */
+int64_t mebptt_budget_bytes_to_units(const mebptt_lstm_desc *desc, size_t bytes);
+
+/* Size of the device workspace mebptt_lstm_train_step needs: the slot arena sized by the plan
+ * plus working memory outside the budget.  0 on error. */
+size_t mebptt_lstm_workspace_bytes(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);
+/* The part of that workspace that is not the slot arena. */
+size_t mebptt_lstm_working_bytes(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);
+
+/* Number of kernel launches one mebptt_lstm_train_step enqueues for this descriptor and plan
+ * (memsets not counted); -1 on error. */
+int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);
+
+/*
+ * One training step under the plan (Algorithm 2 for HSM; the four steps of Section 3.2 for
+ * ISM; Section 3.3 for MSM).  All pointers are DEVICE pointers unless said otherwise.
+ *
+ * Read-only inputs (never written):
+ *   W        layers concatenated; layer l is [4H][I_l + H] with I_0 = I, I_l = H; operand type
+ *   b        [layers][4H] float32
+ *   W_out    [O][H] operand type;  b_out [O] float32
+ *   x        [t][B][I] operand type;  targets [t][B][O] float32
+ *   h0       [layers][B][H] operand type;  c0 [layers][B][H] float32
+ * Workspace: caller-owned, 256-byte aligned, >= mebptt_lstm_workspace_bytes(); contents on
+ *   entry do not matter and are undefined on exit.
+ * stream: a cudaStream_t (NULL = the default stream).
+ * Outputs (overwritten, not accumulated; all float32):
+ *   loss [1]; dW like W; db like b; dW_out [O][H]; db_out [O]; dx [t][B][I] or NULL.
+ *   counters: int64[8] -- [0] forward operations executed, [1] backward operations executed,
+ *   [2] peak units (paper's accounting), [3] device status (MEBPTT_OK or an error code),
+ *   [4..7] reserved.  counters[0] equals mebptt_plan_cost(plan) after a successful step.
+ * Determinism: no atomics; for a fixed descriptor and inputs every plan yields bit-identical
+ *   outputs (each backward step sees bit-identical internal states whether they were stored
+ *   or recomputed, and all accumulations run in the order t .. 1).
+ * Returns MEBPTT_OK once everything is enqueued, or an error with nothing enqueued.
+ */
+int mebptt_lstm_train_step(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan,
+                           const void *W, const void *b, const void *W_out, const void *b_out,
+                           const void *x, const void *targets, const void *h0, const void *c0,
+                           void *workspace, size_t workspace_bytes, void *stream,
+                           float *loss, float *dW, float *db, float *dW_out, float *db_out,
+                           float *dx, int64_t *counters);
+
+/*
+ * The same step for callers whose data lives in HOST memory.  Inputs and outputs are host
+ * pointers (pinned memory makes the copies asynchronous); `workspace` is still a DEVICE buffer,
+ * of at least mebptt_lstm_host_workspace_bytes(), in which the call stages its copies of the
+ * inputs and outputs around the train step.  The call enqueues host-to-device copies, the step
+ * and device-to-host copies on `stream`; results are valid after the stream is synchronised.
+ */
+size_t mebptt_lstm_host_workspace_bytes(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);
+int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan,
+                                const void *W, const void *b, const void *W_out,
+                                const void *b_out, const void *x, const void *targets,
+                                const void *h0, const void *c0,
+                                void *workspace, size_t workspace_bytes, void *stream,
+                                float *loss, float *dW, float *db, float *dW_out, float *db_out,
+                                float *dx, int64_t *counters);
+
+/*
+ * Push / Pop of Algorithm 2 as an explicit copy, for callers that keep states in a pool of
+ * their own: copies `bytes` bytes from src to dst (device pointers, both 16-byte aligned,
+ * bytes a multiple of 16) on `stream`.  The train step itself writes memorised states in
+ * place and does not call this.
+ */
+int mebptt_slot_copy(void *dst, const void *src, size_t bytes, void *stream);
+
+const char *mebptt_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEBPTT_H */

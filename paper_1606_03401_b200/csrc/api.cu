@@ -1,0 +1,290 @@
+// C interface: execution.  Walks the tape of a plan and enqueues the device work of one
+// training step on the caller's stream; nothing here waits for the device.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+
+#include "kernels.hpp"
+#include "layout.hpp"
+#include "mebptt.h"
+#include "plan.hpp"
+
+using namespace mebptt;
+
+namespace {
+
+struct StepIO {
+  const char *W, *W_out, *x, *h0;
+  const float *b, *b_out, *targets, *c0;
+  char* ws;
+  float *loss, *dW, *db, *dW_out, *db_out, *dx;
+  int64_t* counters;
+};
+
+// Base address of the hidden block (or record) at a tape location; LOC_INIT has none.
+inline char* loc_base(const Layout& y, char* ws, int32_t loc) {
+  switch (loc) {
+    case MEBPTT_LOC_PING: return ws + y.off_ping;
+    case MEBPTT_LOC_PONG: return ws + y.off_pong;
+    case MEBPTT_LOC_CORE: return ws + y.off_core;
+    default: return ws + y.off_arena + (size_t)loc * y.unit;
+  }
+}
+
+inline void hidden_at(const Layout& y, const StepIO& io, int32_t loc, int l, const void** h, const float** c) {
+  const size_t bh = (size_t)y.B * y.H;
+  if (loc == MEBPTT_LOC_INIT) {
+    *h = io.h0 + (size_t)l * bh * y.esz;
+    *c = io.c0 + (size_t)l * bh;
+  } else {
+    char* base = loc_base(y, io.ws, loc);
+    *h = base + y.h_off(l);
+    *c = reinterpret_cast<const float*>(base + y.c_off(l));
+  }
+}
+
+int check_common(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  if (!valid_desc(desc) || !plan) return MEBPTT_ERR_ARG;
+  const Plan* p = reinterpret_cast<const Plan*>(plan);
+  if (p->t != desc->t) return MEBPTT_ERR_ARG;
+  // the LSTM's internal state needs 4 units (3 without its input hidden state)
+  if (p->mode != MEBPTT_HSM && p->alpha < 4) return MEBPTT_ERR_UNSUPPORTED;
+  if (p->mode == MEBPTT_MSM && p->beta != 0 && p->beta < 3) return MEBPTT_ERR_UNSUPPORTED;
+  return MEBPTT_OK;
+}
+
+int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const StepIO& io, cudaStream_t s) {
+  const size_t bh = (size_t)y.B * y.H;
+  const size_t plane_elems = y.plane / y.esz;
+  char* ws = io.ws;
+  float* dh_rec = reinterpret_cast<float*>(ws + y.off_dh);
+  float* dc_rec = reinterpret_cast<float*>(ws + y.off_dc);
+  float* dha = reinterpret_cast<float*>(ws + y.off_dha);
+  float* dz = reinterpret_cast<float*>(ws + y.off_dz);
+  float* dy = reinterpret_cast<float*>(ws + y.off_dy);
+  float* loss_part = reinterpret_cast<float*>(ws + y.off_loss_part);
+  float* loss_t = reinterpret_cast<float*>(ws + y.off_loss_t);
+
+  cudaMemsetAsync(dh_rec, 0, (size_t)y.L * bh * 4, s);
+  cudaMemsetAsync(dc_rec, 0, (size_t)y.L * bh * 4, s);
+  cudaMemsetAsync(io.dW, 0, y.w_total_elems() * 4, s);
+  cudaMemsetAsync(io.db, 0, (size_t)y.L * 4 * y.H * 4, s);
+  cudaMemsetAsync(io.dW_out, 0, (size_t)y.O * y.H * 4, s);
+  cudaMemsetAsync(io.db_out, 0, (size_t)y.O * 4, s);
+  cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
+
+  for (const mebptt_op& op : p->tape) {
+    const int64_t k = op.k;
+    const char* x_k = io.x + (size_t)(k - 1) * y.B * y.I * y.esz;
+    if (op.kind == MEBPTT_OP_FWD) {
+      char* dst = loc_base(y, ws, op.dst);
+      for (int l = 0; l < y.L; ++l) {
+        generic::FwdArgs a{};
+        hidden_at(y, io, op.src, l, &a.h_prev, &a.c_prev);
+        a.in = (l == 0) ? (const void*)x_k : (const void*)(dst + y.h_off(l - 1));
+        a.I = (l == 0) ? y.I : y.H;
+        a.W = io.W + y.w_layer_offset(l) * y.esz;
+        a.bias = io.b + (size_t)l * 4 * y.H;
+        a.h_out = dst + y.h_off(l);
+        a.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
+        if (op.dst_fmt != MEBPTT_FMT_HIDDEN) a.gates = dst + y.rec_gates + (size_t)l * y.gsz;
+        if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+          a.h_in_copy = dst + y.rec_in + y.h_off(l);
+          a.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
+        }
+        a.plane_elems = plane_elems;
+        a.B = y.B; a.H = y.H;
+        a.counters = (l == 0) ? io.counters : nullptr;
+        generic::forward_step(y.dtype, a, s);
+      }
+    } else {
+      char* rec = loc_base(y, ws, op.src);
+      // readout of the top layer, loss term, dy and the gradient entering the top layer
+      generic::ReadoutArgs r{};
+      r.h = rec + y.h_off(y.L - 1);
+      r.W_out = io.W_out; r.b_out = io.b_out;
+      r.target = io.targets + (size_t)(k - 1) * y.B * y.O;
+      r.dy = dy; r.loss_part = loss_part; r.n_loss_part = y.n_loss_part;
+      r.loss_k = loss_t + (k - 1);
+      r.dha = dha; r.dW_out = io.dW_out; r.db_out = io.db_out;
+      r.B = y.B; r.H = y.H; r.O = y.O;
+      generic::readout(y.dtype, r, s);
+      for (int l = y.L - 1; l >= 0; --l) {
+        generic::BwdArgs a{};
+        a.dha = dha;
+        a.dh_rec = dh_rec + (size_t)l * bh;
+        a.dc_rec = dc_rec + (size_t)l * bh;
+        a.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+        a.plane_elems = plane_elems;
+        a.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
+        if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+          a.h_prev = rec + y.rec_in + y.h_off(l);
+          a.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
+        } else {
+          hidden_at(y, io, op.aux, l, &a.h_prev, &a.c_prev);
+        }
+        a.in = (l == 0) ? (const void*)x_k : (const void*)(rec + y.h_off(l - 1));
+        a.I = (l == 0) ? y.I : y.H;
+        a.W = io.W + y.w_layer_offset(l) * y.esz;
+        a.dz = dz;
+        a.dW = io.dW + y.w_layer_offset(l);
+        a.db = io.db + (size_t)l * 4 * y.H;
+        a.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(k - 1) * y.B * y.I : nullptr);
+        a.B = y.B; a.H = y.H;
+        a.counters = (l == y.L - 1) ? io.counters : nullptr;
+        generic::backward_layer(y.dtype, a, s);
+      }
+    }
+  }
+  generic::finalize_step(loss_t, y.t, io.loss, io.counters, p->peak_units, s);
+  return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+}
+
+// staging area of the host-buffer variant, placed after the ordinary workspace
+struct Staging {
+  size_t W, b, W_out, b_out, x, targets, h0, c0, loss, dW, db, dW_out, db_out, dx, counters, total;
+  size_t nW, nb, nW_out, nb_out, nx, ntargets, nh0, nc0, ndx;  // bytes
+};
+
+void staging_layout(const Layout& y, bool want_dx, size_t base, Staging& g) {
+  size_t o = base;
+  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  const size_t bh = (size_t)y.B * y.H;
+  g.nW = y.w_total_elems() * y.esz; g.nb = (size_t)y.L * 4 * y.H * 4;
+  g.nW_out = (size_t)y.O * y.H * y.esz; g.nb_out = (size_t)y.O * 4;
+  g.nx = (size_t)y.t * y.B * y.I * y.esz; g.ntargets = (size_t)y.t * y.B * y.O * 4;
+  g.nh0 = (size_t)y.L * bh * y.esz; g.nc0 = (size_t)y.L * bh * 4;
+  g.ndx = want_dx ? (size_t)y.t * y.B * y.I * 4 : 0;
+  g.W = take(g.nW); g.b = take(g.nb); g.W_out = take(g.nW_out); g.b_out = take(g.nb_out);
+  g.x = take(g.nx); g.targets = take(g.ntargets); g.h0 = take(g.nh0); g.c0 = take(g.nc0);
+  g.loss = take(4); g.dW = take(y.w_total_elems() * 4); g.db = take(g.nb);
+  g.dW_out = take((size_t)y.O * y.H * 4); g.db_out = take(g.nb_out);
+  g.dx = take(g.ndx); g.counters = take(8 * sizeof(int64_t));
+  g.total = o;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc* desc) {
+  if (!valid_desc(desc)) return 0;
+  Layout y;
+  state_layout(desc, y);
+  return y.unit;
+}
+
+int64_t mebptt_budget_bytes_to_units(const mebptt_lstm_desc* desc, size_t bytes) {
+  const size_t u = mebptt_lstm_unit_bytes(desc);
+  return u ? (int64_t)(bytes / u) : -1;
+}
+
+size_t mebptt_lstm_workspace_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  if (check_common(desc, plan) != MEBPTT_OK) return 0;
+  Layout y;
+  workspace_layout(desc, reinterpret_cast<const Plan*>(plan), y);
+  return y.total;
+}
+
+size_t mebptt_lstm_working_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  if (check_common(desc, plan) != MEBPTT_OK) return 0;
+  Layout y;
+  workspace_layout(desc, reinterpret_cast<const Plan*>(plan), y);
+  return y.total - align_up((size_t)y.arena_units * y.unit, 256);
+}
+
+int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  if (check_common(desc, plan) != MEBPTT_OK) return -1;
+  const Plan* p = reinterpret_cast<const Plan*>(plan);
+  // forward operation: one kernel per layer; backward operation: 5 for the readout and
+  // 4 per layer; one to finalise
+  const int64_t L = desc->layers;
+  return p->cost * L + p->t * (5 + 4 * L) + 1;
+}
+
+int mebptt_lstm_train_step(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W,
+                           const void* b, const void* W_out, const void* b_out, const void* x,
+                           const void* targets, const void* h0, const void* c0, void* workspace,
+                           size_t workspace_bytes, void* stream, float* loss, float* dW, float* db,
+                           float* dW_out, float* db_out, float* dx, int64_t* counters) {
+  int rc = check_common(desc, plan);
+  if (rc != MEBPTT_OK) return rc;
+  if (!W || !b || !W_out || !b_out || !x || !targets || !h0 || !c0) return MEBPTT_ERR_ARG;
+  if (!loss || !dW || !db || !dW_out || !db_out || !counters) return MEBPTT_ERR_ARG;
+  if (desc->want_dx && !dx) return MEBPTT_ERR_ARG;
+  const Plan* p = reinterpret_cast<const Plan*>(plan);
+  Layout y;
+  workspace_layout(desc, p, y);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < y.total)
+    return MEBPTT_ERR_WORKSPACE;
+  StepIO io{(const char*)W, (const char*)W_out, (const char*)x, (const char*)h0,
+            (const float*)b, (const float*)b_out, (const float*)targets, (const float*)c0,
+            (char*)workspace, loss, dW, db, dW_out, db_out, dx, counters};
+  return run_step(desc, p, y, io, (cudaStream_t)stream);
+}
+
+size_t mebptt_lstm_host_workspace_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  if (check_common(desc, plan) != MEBPTT_OK) return 0;
+  Layout y;
+  workspace_layout(desc, reinterpret_cast<const Plan*>(plan), y);
+  Staging g;
+  staging_layout(y, desc->want_dx != 0, y.total, g);
+  return g.total;
+}
+
+int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W,
+                                const void* b, const void* W_out, const void* b_out, const void* x,
+                                const void* targets, const void* h0, const void* c0, void* workspace,
+                                size_t workspace_bytes, void* stream, float* loss, float* dW, float* db,
+                                float* dW_out, float* db_out, float* dx, int64_t* counters) {
+  int rc = check_common(desc, plan);
+  if (rc != MEBPTT_OK) return rc;
+  if (!W || !b || !W_out || !b_out || !x || !targets || !h0 || !c0) return MEBPTT_ERR_ARG;
+  if (!loss || !dW || !db || !dW_out || !db_out || !counters) return MEBPTT_ERR_ARG;
+  if (desc->want_dx && !dx) return MEBPTT_ERR_ARG;
+  const Plan* p = reinterpret_cast<const Plan*>(plan);
+  Layout y;
+  workspace_layout(desc, p, y);
+  Staging g;
+  staging_layout(y, desc->want_dx != 0, y.total, g);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < g.total)
+    return MEBPTT_ERR_WORKSPACE;
+  char* ws = (char*)workspace;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaMemcpyAsync(ws + g.W, W, g.nW, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.b, b, g.nb, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.W_out, W_out, g.nW_out, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.b_out, b_out, g.nb_out, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.x, x, g.nx, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.targets, targets, g.ntargets, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.h0, h0, g.nh0, cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(ws + g.c0, c0, g.nc0, cudaMemcpyHostToDevice, s);
+  if (cudaGetLastError() != cudaSuccess) return MEBPTT_ERR_CUDA;
+  StepIO io{ws + g.W, ws + g.W_out, ws + g.x, ws + g.h0,
+            (const float*)(ws + g.b), (const float*)(ws + g.b_out), (const float*)(ws + g.targets),
+            (const float*)(ws + g.c0), ws,
+            (float*)(ws + g.loss), (float*)(ws + g.dW), (float*)(ws + g.db), (float*)(ws + g.dW_out),
+            (float*)(ws + g.db_out), desc->want_dx ? (float*)(ws + g.dx) : nullptr,
+            (int64_t*)(ws + g.counters)};
+  rc = run_step(desc, p, y, io, s);
+  if (rc != MEBPTT_OK) return rc;
+  cudaMemcpyAsync(loss, ws + g.loss, 4, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(dW, ws + g.dW, y.w_total_elems() * 4, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(db, ws + g.db, g.nb, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(dW_out, ws + g.dW_out, (size_t)y.O * y.H * 4, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(db_out, ws + g.db_out, g.nb_out, cudaMemcpyDeviceToHost, s);
+  if (desc->want_dx) cudaMemcpyAsync(dx, ws + g.dx, g.ndx, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(counters, ws + g.counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost, s);
+  return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+}
+
+int mebptt_slot_copy(void* dst, const void* src, size_t bytes, void* stream) {
+  if (!dst || !src) return MEBPTT_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(dst) & 15) || (reinterpret_cast<uintptr_t>(src) & 15) || (bytes & 15))
+    return MEBPTT_ERR_ARG;
+  generic::copy_bytes(dst, src, bytes, (cudaStream_t)stream);
+  return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Host-callable launchers of the device kernels (declarations shared by the executor).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstddef>
+#include <cstdint>
+
+#include "mebptt.h"
+
+namespace mebptt {
+namespace generic {
+
+// One forward operation of one layer: state k-1 -> state k.
+struct FwdArgs {
+  const void* in;        // [B][I] operand type: x_k or the h_k of the layer below
+  const void* h_prev;    // [B][H] operand type
+  const float* c_prev;   // [B][H]
+  const void* W;         // [4H][I + H] operand type
+  const float* bias;     // [4H]
+  void* h_out;           // [B][H] operand type
+  float* c_out;          // [B][H]
+  void* gates;           // four planes [B][H] operand type, or NULL (hidden-state format)
+  void* h_in_copy;       // copy of h_prev for the internal state, or NULL
+  float* c_in_copy;      // copy of c_prev (non-NULL iff h_in_copy is)
+  size_t plane_elems;    // elements between gate planes
+  int B, I, H;
+  int64_t* counters;     // NULL for all but the first layer
+};
+
+// Readout, loss term and output gradient of step k, plus their parameter gradients.
+struct ReadoutArgs {
+  const void* h;         // [B][H] top layer h_k
+  const void* W_out;     // [O][H]
+  const float* b_out;    // [O]
+  const float* target;   // [B][O]
+  float* dy;             // [B][O] scratch
+  float* loss_part;      // scratch, n_loss_part values
+  int n_loss_part;
+  float* loss_k;         // loss term of this step
+  float* dha;            // [B][H]: dy W_out, the gradient entering the top layer
+  float* dW_out;         // [O][H] accumulated
+  float* db_out;         // [O] accumulated
+  int B, H, O;
+};
+
+// One backward operation of one layer.
+struct BwdArgs {
+  const float* dha;      // [B][H] gradient from above (readout or the layer above)
+  float* dh_rec;         // [B][H] in: gradient from step k+1; out: gradient for step k-1
+  float* dc_rec;         // [B][H] likewise for c
+  const void* gates;     // four planes
+  size_t plane_elems;
+  const float* c_t;      // [B][H]
+  const float* c_prev;   // [B][H]
+  const void* in;        // [B][I] input of this layer at step k
+  const void* h_prev;    // [B][H]
+  const void* W;         // [4H][I + H]
+  float* dz;             // [B][4H] scratch
+  float* dW;             // [4H][I + H] accumulated
+  float* db;             // [4H] accumulated
+  float* d_lo;           // [B][I]: gradient w.r.t. `in` (dx_k or the dha of the layer below), or NULL
+  int B, I, H;
+  int64_t* counters;     // NULL for all but the top layer
+};
+
+void forward_step(int dtype, const FwdArgs& a, cudaStream_t s);
+void readout(int dtype, const ReadoutArgs& a, cudaStream_t s);
+void backward_layer(int dtype, const BwdArgs& a, cudaStream_t s);
+void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
+                   cudaStream_t s);
+void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s);
+
+}  // namespace generic
+}  // namespace mebptt

@@ -1,0 +1,100 @@
+// Device memory layout of hidden states, internal states and the workspace.
+//
+// A hidden state (Definition 2) of the stack is, per layer, h (operand type) followed by c
+// (float32).  An internal state (Definition 3) is the output hidden state, the four gate
+// planes i, f, g, o of every layer (operand type, each [B][H]) and a copy of the input hidden
+// state.  The output hidden state comes first, so that a forward operation can read "the hidden
+// state at a location" without knowing which of the two formats the location holds.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+
+#include "mebptt.h"
+#include "plan.hpp"
+
+namespace mebptt {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  int L = 0, I = 0, H = 0, O = 0, B = 0;
+  int dtype = 0;
+  int64_t t = 0;
+  size_t esz = 0;        // bytes of one operand element
+  size_t hsz = 0;        // one layer's h, padded to 16 B
+  size_t csz = 0;        // one layer's c
+  size_t gsz = 0;        // one layer's four gate planes
+  size_t plane = 0;      // one gate plane, padded to 16 B
+  size_t unit = 0;       // one hidden state of the stack, padded to 256 B
+  size_t rec = 0;        // one internal state
+  // record-relative offsets
+  size_t rec_gates = 0;  // gates of layer 0
+  size_t rec_in = 0;     // input hidden state
+  // workspace offsets
+  size_t off_arena = 0, off_core = 0, off_ping = 0, off_pong = 0;
+  size_t off_dh = 0, off_dc = 0, off_dha = 0, off_dz = 0, off_dy = 0;
+  size_t off_loss_part = 0, off_loss_t = 0;
+  size_t total = 0;
+  int64_t arena_units = 0;
+  int n_loss_part = 0;
+
+  size_t w_layer_elems(int l) const { return (size_t)4 * H * ((l == 0 ? I : H) + H); }
+  size_t w_layer_offset(int l) const {  // elements before layer l
+    size_t o = 0;
+    for (int i = 0; i < l; ++i) o += w_layer_elems(i);
+    return o;
+  }
+  size_t w_total_elems() const { return w_layer_offset(L); }
+  // within a hidden block
+  size_t h_off(int l) const { return (size_t)l * (hsz + csz); }
+  size_t c_off(int l) const { return (size_t)l * (hsz + csz) + hsz; }
+};
+
+inline bool valid_desc(const mebptt_lstm_desc* d) {
+  if (!d) return false;
+  if (d->layers < 1 || d->layers > 16) return false;
+  if (d->input < 1 || d->hidden < 1 || d->readout < 1 || d->batch < 1 || d->t < 1) return false;
+  if (d->input > (1 << 16) || d->hidden > (1 << 16) || d->readout > (1 << 16) || d->batch > (1 << 16)) return false;
+  if (d->dtype != MEBPTT_FP32 && d->dtype != MEBPTT_TF32 && d->dtype != MEBPTT_BF16) return false;
+  if (d->want_dx != 0 && d->want_dx != 1) return false;
+  return true;
+}
+
+inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
+  y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
+  y.dtype = d->dtype; y.t = d->t;
+  y.esz = (d->dtype == MEBPTT_BF16) ? 2 : 4;
+  const size_t bh = (size_t)y.B * y.H;
+  y.hsz = align_up(bh * y.esz, 16);
+  y.csz = align_up(bh * 4, 16);
+  y.plane = align_up(bh * y.esz, 16);
+  y.gsz = 4 * y.plane;
+  y.unit = align_up((size_t)y.L * (y.hsz + y.csz), 256);
+  y.rec_gates = y.unit;
+  y.rec_in = y.unit + (size_t)y.L * y.gsz;
+  y.rec = y.rec_in + y.unit;
+}
+
+inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y) {
+  state_layout(d, y);
+  y.arena_units = p->arena_units;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  y.off_arena = take((size_t)y.arena_units * y.unit);
+  y.off_core = take(y.rec);
+  y.off_ping = take(y.unit);
+  y.off_pong = take(y.unit);
+  const size_t bh4 = (size_t)y.B * y.H * 4;
+  y.off_dh = take((size_t)y.L * bh4);
+  y.off_dc = take((size_t)y.L * bh4);
+  y.off_dha = take(bh4);
+  y.off_dz = take((size_t)y.B * 4 * y.H * 4);
+  y.off_dy = take((size_t)y.B * y.O * 4);
+  y.n_loss_part = ((y.B + 63) / 64) * ((y.O + 63) / 64);
+  y.off_loss_part = take((size_t)y.n_loss_part * 4);
+  y.off_loss_t = take((size_t)y.t * 4);
+  y.total = o;
+}
+
+}  // namespace mebptt

@@ -1,0 +1,488 @@
+// Host-side planner: the dynamic programs of Sections 3.1-3.4 and the unrolling of the
+// execution protocol (Algorithm 2; Section 3.2, steps 1-4) into a linear tape.
+//
+// Tables are kept column-major while they are filled (for a fixed budget m the scan over the
+// split point y walks one column forwards and one backwards), then transposed once into the
+// row-major layout the C interface documents.
+#include "plan.hpp"
+
+#include <algorithm>
+#include <cstring>
+#include <limits>
+#include <new>
+
+namespace mebptt {
+
+namespace {
+
+// ---------------------------------------------------------------------------------------
+// min / first-argmin of  base + i + a[i] + b[-i]  over i = 0 .. n-1  (a ascending, b descending)
+// Two passes: a vectorisable reduction, then a search for the first index that attains it.
+// ---------------------------------------------------------------------------------------
+template <class T>
+#if defined(__GNUC__) && defined(__x86_64__)
+__attribute__((target_clones("avx2", "default")))
+#endif
+T scan_min(const T* a, const T* b_last, int64_t n, T base) {
+  T best = std::numeric_limits<T>::max();
+  for (int64_t i = 0; i < n; ++i) {
+    T v = (T)(base + (T)i + a[i] + b_last[-i]);
+    best = v < best ? v : best;
+  }
+  return best;
+}
+
+template <class T>
+int64_t first_index(const T* a, const T* b_last, int64_t n, T base, T value) {
+  for (int64_t i = 0; i < n; ++i)
+    if ((T)(base + (T)i + a[i] + b_last[-i]) == value) return i;
+  return -1;
+}
+
+template <class T>
+struct Inf;
+template <>
+struct Inf<int32_t> {
+  static constexpr int32_t v = 1 << 29;  // three of them fit
+};
+template <>
+struct Inf<int64_t> {
+  static constexpr int64_t v = (int64_t)1 << 60;
+};
+
+// Column-major working tables: col(m)[t].
+template <class T>
+struct Cols {
+  int64_t t_dim, m_dim;
+  std::vector<T> v;
+  Cols(int64_t t, int64_t m, T fill) : t_dim(t + 1), m_dim(m + 1), v((size_t)(t + 1) * (m + 1), fill) {}
+  T* col(int64_t m) { return v.data() + (size_t)m * t_dim; }
+};
+
+template <class T>
+void solve_hsm(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
+  // Section 3.1: C(1, m) = 1, C(t, 1) = t (t + 1) / 2,
+  // C(t, m) = min_{1 <= y < t} y + C(t - y, m - 1) + C(y, m).
+  const T INF = Inf<T>::v;
+  for (int64_t m = 1; m <= m_max; ++m) {
+    T* c = C.col(m);
+    int32_t* d = D.col(m);
+    std::fill(d, d + t_max + 1, 0);
+    c[1] = 1;
+    if (m == 1) {
+      for (int64_t t = 1; t <= t_max; ++t) c[t] = (T)(t * (t + 1) / 2);
+      continue;
+    }
+    const T* cm1 = C.col(m - 1);
+    for (int64_t t = 2; t <= t_max; ++t) {
+      // y = 1 + i, i = 0 .. t-2 :  (1 + i) + c[1 + i] + cm1[t - 1 - i]
+      T best = scan_min<T>(c + 1, cm1 + (t - 1), t - 1, (T)1);
+      if (best >= INF) { c[t] = INF; continue; }
+      c[t] = best;
+      d[t] = (int32_t)(1 + first_index<T>(c + 1, cm1 + (t - 1), t - 1, (T)1, best));
+    }
+  }
+}
+
+template <class T>
+void solve_ism(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
+  // Section 3.2: C(0, m) = 0, C(t > 0, 0) = inf,
+  // C(t, m) = min_{1 <= y <= t} y + C(y - 1, m) + C(t - y, m - 1).
+  const T INF = Inf<T>::v;
+  for (int64_t m = 0; m <= m_max; ++m) {
+    C.col(m)[0] = 0;
+    std::fill(D.col(m), D.col(m) + t_max + 1, 0);
+  }
+  for (int64_t m = 1; m <= m_max; ++m) {
+    T* c = C.col(m);
+    int32_t* d = D.col(m);
+    const T* cm1 = C.col(m - 1);
+    for (int64_t t = 1; t <= t_max; ++t) {
+      // y = 1 + i, i = 0 .. t-1 :  (1 + i) + c[i] + cm1[t - 1 - i]
+      T best = scan_min<T>(c, cm1 + (t - 1), t, (T)1);
+      if (best >= INF) { c[t] = INF; continue; }
+      c[t] = best;
+      d[t] = (int32_t)(1 + first_index<T>(c, cm1 + (t - 1), t, (T)1, best));
+    }
+  }
+}
+
+template <class T>
+void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Cols<int32_t>& D1,
+               Cols<int32_t>& D2, Cols<uint8_t>& H) {
+  // Section 3.3 with the reading C(0, m) = 0 for every m (also m <= 0) and C(t > 0, m <= 0) = inf.
+  // Q1 = y + C(y, m) + C(t - y, m - 1), 1 <= y < t;  Q2 = y + C(y - 1, m) + C(t - y, m - a(y)),
+  // 1 <= y <= t, a(y) = alpha, or beta at y = 1 when the Section 3.4 variant is on.
+  const T INF = Inf<T>::v;
+  std::vector<T> nonpos((size_t)t_max + 1, INF);  // the column of any budget <= 0
+  nonpos[0] = 0;
+  for (int64_t m = 0; m <= m_max; ++m) {
+    C.col(m)[0] = 0;
+    std::fill(D1.col(m), D1.col(m) + t_max + 1, 0);
+    std::fill(D2.col(m), D2.col(m) + t_max + 1, 0);
+    std::fill(H.col(m), H.col(m) + t_max + 1, (uint8_t)0);
+  }
+  auto column = [&](int64_t m) -> const T* { return m <= 0 ? nonpos.data() : C.col(m); };
+  for (int64_t m = 1; m <= m_max; ++m) {
+    T* c = C.col(m);
+    const T* cm1 = column(m - 1);
+    const T* cma = column(m - alpha);
+    const T* cmb = beta > 0 ? column(m - beta) : nullptr;
+    for (int64_t t = 1; t <= t_max; ++t) {
+      T c1 = INF, c2 = INF;
+      int32_t y1 = 0, y2 = 0;
+      if (t >= 2) {
+        c1 = scan_min<T>(c + 1, cm1 + (t - 1), t - 1, (T)1);
+        if (c1 < INF) y1 = (int32_t)(1 + first_index<T>(c + 1, cm1 + (t - 1), t - 1, (T)1, c1));
+        else c1 = INF;
+      }
+      if (cmb) {
+        // y = 1 charged beta, y >= 2 charged alpha; keep the smallest y on ties
+        T q1 = (T)std::min<int64_t>((int64_t)1 + c[0] + cmb[t - 1], INF);
+        T rest = INF;
+        if (t >= 2) rest = scan_min<T>(c + 1, cma + (t - 2), t - 1, (T)2);
+        if (rest >= INF) rest = INF;
+        if (q1 <= rest) { c2 = q1; y2 = 1; }
+        else { c2 = rest; y2 = (int32_t)(2 + first_index<T>(c + 1, cma + (t - 2), t - 1, (T)2, rest)); }
+        if (c2 >= INF) { c2 = INF; y2 = 0; }
+      } else {
+        c2 = scan_min<T>(c, cma + (t - 1), t, (T)1);
+        if (c2 < INF) y2 = (int32_t)(1 + first_index<T>(c, cma + (t - 1), t, (T)1, c2));
+        else c2 = INF;
+      }
+      D1.col(m)[t] = y1;
+      D2.col(m)[t] = y2;
+      if (c1 >= INF && c2 >= INF) { c[t] = INF; continue; }
+      if (c1 <= c2) { c[t] = c1; H.col(m)[t] = 1; }   // ties: the hidden state (fewer units)
+      else          { c[t] = c2; H.col(m)[t] = 2; }
+    }
+  }
+}
+
+template <class S, class Dst>
+void transpose_into(Cols<S>& src, std::vector<Dst>& dst) {
+  dst.resize(src.v.size());
+  for (int64_t m = 0; m < src.m_dim; ++m) {
+    const S* c = src.col(m);
+    for (int64_t t = 0; t < src.t_dim; ++t) dst[(size_t)t * src.m_dim + m] = (Dst)c[t];
+  }
+}
+
+template <class S>
+void transpose_costs(Cols<S>& src, std::vector<int64_t>& dst) {
+  transpose_into(src, dst);
+  for (int64_t& v : dst)
+    if (v >= (int64_t)Inf<S>::v) v = Inf<int64_t>::v;
+}
+
+template <class T>
+void solve(Plan& p) {
+  const int64_t t = p.t, m = p.m;
+  Cols<T> C(t, m, Inf<T>::v);
+  Cols<int32_t> D(t, m, 0);
+  if (p.mode == MEBPTT_HSM) {
+    solve_hsm<T>(t, m, C, D);
+  } else if (p.mode == MEBPTT_ISM) {
+    solve_ism<T>(t, m, C, D);
+  } else {
+    Cols<int32_t> D2(t, m, 0);
+    Cols<uint8_t> H(t, m, 0);
+    solve_msm<T>(t, m, p.alpha, p.beta, C, D, D2, H);
+    transpose_into(D2, p.D2);
+    transpose_into(H, p.H);
+  }
+  transpose_costs(C, p.C);
+  transpose_into(D, p.D);
+}
+
+// ---------------------------------------------------------------------------------------
+// Unrolling the protocol
+// ---------------------------------------------------------------------------------------
+struct Emitter {
+  Plan& p;
+  int64_t units;      // paper's accounting
+  int64_t top = 0;    // physical arena top, hidden-state units
+  explicit Emitter(Plan& pl) : p(pl), units(pl.mode == MEBPTT_ISM ? 0 : 1) { p.peak_units = units; }
+
+  int64_t Cat(int64_t t, int64_t m) const { return p.C[(size_t)t * (p.m + 1) + m]; }
+  int32_t Dat(int64_t t, int64_t m) const { return p.D[(size_t)t * (p.m + 1) + m]; }
+  int32_t D2at(int64_t t, int64_t m) const { return p.D2[(size_t)t * (p.m + 1) + m]; }
+  int Hat(int64_t t, int64_t m) const { return p.H[(size_t)t * (p.m + 1) + m]; }
+
+  void fwd(int64_t k, int32_t src, int32_t dst, int fmt) {
+    mebptt_op op{};
+    op.kind = MEBPTT_OP_FWD; op.k = (int32_t)k; op.src = src; op.dst = dst; op.dst_fmt = fmt;
+    op.aux = 0; op.units = (int32_t)units;
+    p.tape.push_back(op);
+  }
+  void bwd(int64_t k, int32_t src, int fmt, int32_t aux) {
+    mebptt_op op{};
+    op.kind = MEBPTT_OP_BWD; op.k = (int32_t)k; op.src = src; op.dst = 0; op.dst_fmt = fmt;
+    op.aux = aux; op.units = (int32_t)units;
+    p.tape.push_back(op);
+  }
+  // n forward operations from the state of step s at `loc`; the last one writes `fmt` to
+  // `last_dst`, the others alternate between the two scratch states.  Returns nothing: the
+  // caller knows where the last state went.
+  void sweep(int64_t s, int64_t n, int32_t loc, int32_t last_dst, int last_fmt) {
+    int32_t cur = loc;
+    for (int64_t i = 1; i <= n; ++i) {
+      if (i == n) { fwd(s + i, cur, last_dst, last_fmt); return; }
+      int32_t dst = (cur == MEBPTT_LOC_PING) ? MEBPTT_LOC_PONG : MEBPTT_LOC_PING;
+      fwd(s + i, cur, dst, MEBPTT_FMT_HIDDEN);
+      cur = dst;
+    }
+  }
+  void grow(int64_t paper_units, int64_t phys_units) {
+    units += paper_units; top += phys_units;
+    p.peak_units = std::max(p.peak_units, units);
+    p.arena_units = std::max(p.arena_units, top);
+  }
+  void shrink(int64_t paper_units, int64_t phys_units) { units -= paper_units; top -= phys_units; }
+
+  // Algorithm 2.  `loc` holds the hidden state of step s (Peek).
+  void hsm(int64_t t, int64_t m, int64_t s, int32_t loc) {
+    for (;;) {
+      if (t == 0) return;
+      if (t == 1) {  // base case: forward and backward on the working core
+        fwd(s + 1, loc, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL);
+        bwd(s + 1, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL, 0);
+        return;
+      }
+      if (m == 1) {  // boundary C(t, 1): re-run from the start state before every backward step
+        for (int64_t k = t; k >= 1; --k) {
+          sweep(s, k, loc, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL);
+          bwd(s + k, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL, 0);
+        }
+        return;
+      }
+      const int64_t y = Dat(t, m);
+      const int32_t slot = (int32_t)top;
+      grow(1, 1);
+      // the sweep runs y operations (the printed bound t - 1 contradicts the cost y of
+      // Eq. (1)); its last one writes h_{s+y} straight into the slot: that is the Push
+      sweep(s, y, loc, slot, MEBPTT_FMT_HIDDEN);
+      hsm(t - y, m - 1, s + y, slot);
+      shrink(1, 1);  // Pop
+      t = y;         // left part, full budget
+    }
+  }
+
+  // Section 3.2, steps 1-4.
+  void ism(int64_t t, int64_t m, int64_t s, int32_t loc) {
+    const int a = p.alpha;
+    while (t > 0) {
+      const int64_t y = Dat(t, m);
+      const int32_t slot = (int32_t)top;
+      grow(1, a);
+      sweep(s, y, loc, slot, MEBPTT_FMT_INTERNAL);          // step 1
+      ism(t - y, m - 1, s + y, slot);                        // step 2
+      bwd(s + y, slot, MEBPTT_FMT_INTERNAL, 0);              // step 3
+      shrink(1, a);
+      t = y - 1;                                             // step 4
+    }
+  }
+
+  // Section 3.3 (and 3.4 when beta > 0).
+  void msm(int64_t t, int64_t m, int64_t s, int32_t loc) {
+    const int a = p.alpha, b = p.beta;
+    while (t > 0) {
+      if (Hat(t, m) == 1) {
+        const int64_t y = Dat(t, m);
+        const int32_t slot = (int32_t)top;
+        grow(1, 1);
+        sweep(s, y, loc, slot, MEBPTT_FMT_HIDDEN);
+        msm(t - y, m - 1, s + y, slot);
+        shrink(1, 1);
+        t = y;
+      } else {
+        const int64_t y = D2at(t, m);
+        if (y == t) {
+          // nothing to the right: the internal state never leaves the working core
+          sweep(s, y, loc, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL);
+          bwd(s + y, MEBPTT_LOC_CORE, MEBPTT_FMT_INTERNAL, 0);
+        } else {
+          const bool short_form = (b > 0 && y == 1);
+          const int u = short_form ? b : a;
+          const int fmt = short_form ? MEBPTT_FMT_INTERNAL_NOINPUT : MEBPTT_FMT_INTERNAL;
+          const int32_t slot = (int32_t)top;
+          grow(u, u);
+          sweep(s, y, loc, slot, fmt);
+          msm(t - y, m - u, s + y, slot);
+          bwd(s + y, slot, fmt, short_form ? loc : 0);
+          shrink(u, u);
+        }
+        t = y - 1;
+      }
+    }
+  }
+};
+
+}  // namespace
+
+int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out) {
+  if (!out) return MEBPTT_ERR_ARG;
+  *out = nullptr;
+  if (t < 1 || t > (int64_t)1 << 24) return MEBPTT_ERR_ARG;
+  if (mode != MEBPTT_HSM && mode != MEBPTT_ISM && mode != MEBPTT_MSM) return MEBPTT_ERR_ARG;
+  if (alpha < 2 || alpha > 64) return MEBPTT_ERR_ARG;
+  if (beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
+  if (m < 1) return MEBPTT_ERR_BUDGET;
+  if (mode != MEBPTT_MSM) beta = 0;
+  // beyond saturation more memory changes nothing
+  const int64_t sat = (mode == MEBPTT_MSM) ? std::max<int64_t>(1, (int64_t)alpha * (t - 1) + 1) : t;
+  m = std::min(m, sat);
+  Plan* p = new (std::nothrow) Plan();
+  if (!p) return MEBPTT_ERR_OOM;
+  p->t = t; p->m = m; p->mode = mode; p->alpha = alpha; p->beta = beta;
+  try {
+    if (t * (t + 1) / 2 + t < (int64_t)Inf<int32_t>::v) solve<int32_t>(*p);
+    else solve<int64_t>(*p);
+    p->cost = p->C[(size_t)t * (m + 1) + m];
+    if (p->cost >= MEBPTT_INF) { delete p; return MEBPTT_ERR_BUDGET; }
+    if (p->cost + t > (int64_t)1 << 28) { delete p; return MEBPTT_ERR_UNSUPPORTED; }  // tape too long
+    p->tape.reserve((size_t)(p->cost + t));
+    Emitter e(*p);
+    if (mode == MEBPTT_HSM) e.hsm(t, m, 0, MEBPTT_LOC_INIT);
+    else if (mode == MEBPTT_ISM) e.ism(t, m, 0, MEBPTT_LOC_INIT);
+    else e.msm(t, m, 0, MEBPTT_LOC_INIT);
+  } catch (const std::bad_alloc&) {
+    delete p;
+    return MEBPTT_ERR_OOM;
+  }
+  int rc = validate_plan(*p);
+  if (rc != MEBPTT_OK) { delete p; return rc; }
+  *out = p;
+  return MEBPTT_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Host replay of a tape with integer bookkeeping
+// ---------------------------------------------------------------------------------------
+int validate_plan(const Plan& p) {
+  struct Entry { int64_t off, units, pos; int fmt; };
+  std::vector<Entry> arena;            // live records, ascending offsets (a stack)
+  int64_t ping = -1, pong = -1;        // step whose hidden state sits there
+  int64_t core = -1;                   // step whose internal state the working core holds
+  int64_t next_bwd = p.t, forwards = 0, peak = 0;
+  const int a = p.alpha, b = p.beta;
+  auto rec_units = [&](int fmt) -> int64_t {
+    if (fmt == MEBPTT_FMT_HIDDEN) return 1;
+    if (fmt == MEBPTT_FMT_INTERNAL) return a;
+    return b;
+  };
+  auto hidden_at = [&](int32_t loc) -> int64_t {  // which step's hidden state is readable at loc
+    if (loc == MEBPTT_LOC_INIT) return 0;
+    if (loc == MEBPTT_LOC_PING) return ping;
+    if (loc == MEBPTT_LOC_PONG) return pong;
+    if (loc == MEBPTT_LOC_CORE) return core;
+    for (const Entry& e : arena) if (e.off == loc) return e.pos;
+    return -1;
+  };
+  for (const mebptt_op& op : p.tape) {
+    if (op.k < 1 || op.k > p.t) return MEBPTT_ERR_PLAN;
+    if (op.units < 0 || op.units > p.m) return MEBPTT_ERR_PLAN;
+    peak = std::max<int64_t>(peak, op.units);
+    if (op.kind == MEBPTT_OP_FWD) {
+      if (hidden_at(op.src) != op.k - 1) return MEBPTT_ERR_PLAN;
+      if (op.dst == op.src) return MEBPTT_ERR_PLAN;
+      ++forwards;
+      if (op.dst == MEBPTT_LOC_PING) { if (op.dst_fmt != MEBPTT_FMT_HIDDEN) return MEBPTT_ERR_PLAN; ping = op.k; }
+      else if (op.dst == MEBPTT_LOC_PONG) { if (op.dst_fmt != MEBPTT_FMT_HIDDEN) return MEBPTT_ERR_PLAN; pong = op.k; }
+      else if (op.dst == MEBPTT_LOC_CORE) { if (op.dst_fmt != MEBPTT_FMT_INTERNAL) return MEBPTT_ERR_PLAN; core = op.k; }
+      else if (op.dst >= 0) {
+        if (op.dst_fmt == MEBPTT_FMT_INTERNAL_NOINPUT && b <= 0) return MEBPTT_ERR_PLAN;
+        const int64_t u = rec_units(op.dst_fmt);
+        // writing at an offset retires everything at or above it (stack discipline) ...
+        while (!arena.empty() && arena.back().off >= op.dst) arena.pop_back();
+        // ... and must not run into what lies below
+        if (!arena.empty() && arena.back().off + arena.back().units > op.dst) return MEBPTT_ERR_PLAN;
+        if (op.dst + u > p.arena_units) return MEBPTT_ERR_PLAN;
+        arena.push_back(Entry{op.dst, u, op.k, op.dst_fmt});
+      } else return MEBPTT_ERR_PLAN;
+    } else if (op.kind == MEBPTT_OP_BWD) {
+      if (op.k != next_bwd) return MEBPTT_ERR_PLAN;
+      if (op.src == MEBPTT_LOC_CORE) {
+        if (core != op.k || op.dst_fmt != MEBPTT_FMT_INTERNAL) return MEBPTT_ERR_PLAN;
+        core = -1;
+      } else {
+        bool ok = false;
+        for (const Entry& e : arena)
+          if (e.off == op.src && e.pos == op.k && e.fmt == op.dst_fmt && e.fmt != MEBPTT_FMT_HIDDEN) ok = true;
+        if (!ok) return MEBPTT_ERR_PLAN;
+        if (op.dst_fmt == MEBPTT_FMT_INTERNAL_NOINPUT && hidden_at(op.aux) != op.k - 1) return MEBPTT_ERR_PLAN;
+      }
+      --next_bwd;
+    } else return MEBPTT_ERR_PLAN;
+  }
+  if (next_bwd != 0) return MEBPTT_ERR_PLAN;
+  if (forwards != p.cost) return MEBPTT_ERR_PLAN;
+  if (peak != p.peak_units || peak > p.m) return MEBPTT_ERR_PLAN;
+  return MEBPTT_OK;
+}
+
+}  // namespace mebptt
+
+// ---------------------------------------------------------------------------------------
+// C interface: planning
+// ---------------------------------------------------------------------------------------
+using mebptt::Plan;
+
+extern "C" {
+
+int mebptt_plan(int64_t t, int64_t m, int mode, mebptt_plan_t** out) {
+  return mebptt::build_plan(t, m, mode, 4, 0, reinterpret_cast<Plan**>(out));
+}
+
+int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_plan_t** out) {
+  return mebptt::build_plan(t, m, mode, alpha, beta, reinterpret_cast<Plan**>(out));
+}
+
+void mebptt_plan_free(mebptt_plan_t* plan) { delete reinterpret_cast<Plan*>(plan); }
+
+#define P_(x) (reinterpret_cast<const Plan*>(x))
+int64_t mebptt_plan_cost(const mebptt_plan_t* plan) { return plan ? P_(plan)->cost : -1; }
+int64_t mebptt_plan_num_ops(const mebptt_plan_t* plan) { return plan ? (int64_t)P_(plan)->tape.size() : -1; }
+const mebptt_op* mebptt_plan_tape(const mebptt_plan_t* plan) { return plan ? P_(plan)->tape.data() : nullptr; }
+int64_t mebptt_plan_peak_units(const mebptt_plan_t* plan) { return plan ? P_(plan)->peak_units : -1; }
+int64_t mebptt_plan_arena_units(const mebptt_plan_t* plan) { return plan ? P_(plan)->arena_units : -1; }
+int64_t mebptt_plan_t_len(const mebptt_plan_t* plan) { return plan ? P_(plan)->t : -1; }
+int64_t mebptt_plan_m(const mebptt_plan_t* plan) { return plan ? P_(plan)->m : -1; }
+int mebptt_plan_mode(const mebptt_plan_t* plan) { return plan ? P_(plan)->mode : -1; }
+int mebptt_plan_alpha(const mebptt_plan_t* plan) { return plan ? P_(plan)->alpha : -1; }
+int mebptt_plan_beta(const mebptt_plan_t* plan) { return plan ? P_(plan)->beta : -1; }
+
+int mebptt_plan_tables(const mebptt_plan_t* plan, const int64_t** C, const int32_t** D,
+                       const int32_t** D2, const uint8_t** H, int64_t* t_dim, int64_t* m_dim) {
+  if (!plan) return MEBPTT_ERR_ARG;
+  const Plan* p = P_(plan);
+  if (C) *C = p->C.data();
+  if (D) *D = p->D.data();
+  if (D2) *D2 = p->D2.empty() ? nullptr : p->D2.data();
+  if (H) *H = p->H.empty() ? nullptr : p->H.data();
+  if (t_dim) *t_dim = p->t + 1;
+  if (m_dim) *m_dim = p->m + 1;
+  return MEBPTT_OK;
+}
+
+int mebptt_plan_validate(const mebptt_plan_t* plan) {
+  if (!plan) return MEBPTT_ERR_ARG;
+  return mebptt::validate_plan(*P_(plan));
+}
+
+const char* mebptt_strerror(int status) {
+  switch (status) {
+    case MEBPTT_OK: return "ok";
+    case MEBPTT_ERR_ARG: return "invalid argument";
+    case MEBPTT_ERR_BUDGET: return "memory budget too small: no policy exists";
+    case MEBPTT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MEBPTT_ERR_UNSUPPORTED: return "unsupported shape, precision or plan";
+    case MEBPTT_ERR_CUDA: return "CUDA runtime error";
+    case MEBPTT_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case MEBPTT_ERR_OOM: return "out of host memory";
+    case MEBPTT_ERR_PLAN: return "tape failed validation";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

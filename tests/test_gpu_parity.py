@@ -1,0 +1,159 @@
+"""GPU parity: the CUDA path, called through the C interface, against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import policy as P
+from paper_1606_03401_b200 import synth
+from tests.util import assert_bit_identical, assert_close_to_oracle, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    from paper_1606_03401_b200 import harness
+    return harness
+
+
+def _cfg(base, **kw):
+    return synth.with_overrides(synth.CONFIGS[base], **kw)
+
+
+def test_c1_hsm_m8_matches_oracle(H):
+    """Config 1 in full: fp32, I32 H64 B4 t64, BPTT-HSM with m = 8."""
+    cfg = synth.CONFIGS["c1"]
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    plan = dp.plan("hsm", 8)
+    assert plan.cost == P.cost(P.HSM, 64, 8)
+    res = dp.run(plan)
+    ref = oracle_run(dp.prob)
+    assert_close_to_oracle(res, ref, "fp32", want_dx=True)
+    c = res["counters"]
+    assert c[0] == plan.cost and c[1] == cfg.t and c[2] == plan.peak_units and c[3] == 0
+
+
+POLICIES = [("hsm", 1), ("hsm", 2), ("hsm", 8), ("hsm", 64), ("ism", 1), ("ism", 3), ("ism", 8),
+            ("msm", 1), ("msm", 5), ("msm", 8), ("msm", 40), ("msm", 10 ** 6)]
+
+
+def test_c1_every_policy_is_bit_identical_to_full_memory(H):
+    cfg = synth.CONFIGS["c1"]
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][0] == cfg.t
+    for mode, m in POLICIES:
+        for beta in ((0, 3) if mode == "msm" else (0,)):
+            plan = dp.plan(mode, m, beta=beta)
+            res = dp.run(plan)
+            code = {"hsm": P.HSM, "ism": P.ISM, "msm": P.MSM}[mode]
+            assert res["counters"][0] == plan.cost == P.cost(code, cfg.t, plan.m, 4, beta or None)
+            assert res["counters"][1] == cfg.t and res["counters"][3] == 0
+            assert_bit_identical(res, full, want_dx=True)
+    # and twice the same plan gives the same bits
+    again = dp.run(dp.full_memory_plan())
+    assert_bit_identical(again, full, want_dx=True)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16", "tf32"])
+@pytest.mark.parametrize("shape", [dict(input=5, hidden=7, batch=3, t=11, readout=3),
+                                   dict(input=70, hidden=65, batch=67, t=9, readout=66),
+                                   dict(input=1, hidden=1, batch=1, t=1, readout=1)])
+def test_ragged_shapes_match_oracle(H, dtype, shape):
+    """Sizes that are no multiple of any tile, down to the degenerate 1 x 1 x 1 problem."""
+    cfg = _cfg("c1", dtype=dtype, **shape)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, dtype, want_dx=True)
+    for mode, m in [("hsm", 3), ("ism", 2), ("msm", 6)]:
+        res = dp.run(dp.plan(mode, m))
+        assert_bit_identical(res, full, want_dx=True)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_two_layers_match_oracle(H, dtype):
+    cfg = _cfg("c1", layers=2, dtype=dtype, input=24, hidden=40, batch=6, t=20, readout=10)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, dtype, want_dx=True)
+    for mode, m, beta in [("hsm", 4, 0), ("ism", 3, 0), ("msm", 9, 0), ("msm", 9, 3)]:
+        res = dp.run(dp.plan(mode, m, beta=beta))
+        assert_bit_identical(res, full, want_dx=True)
+
+
+def test_nonzero_initial_state_and_no_dx(H):
+    cfg = _cfg("c1", t=12)
+    prob = synth.make_problem(cfg)
+    r = np.random.default_rng(7)
+    prob["h0"] = synth.round_to_fp32(r.standard_normal(prob["h0"].shape) * 0.5)
+    prob["c0"] = synth.round_to_fp32(r.standard_normal(prob["c0"].shape) * 0.5)
+    dp = H.DeviceProblem(cfg, prob, want_dx=False)
+    res = dp.run(dp.plan("msm", 7, beta=3))
+    assert_close_to_oracle(res, oracle_run(prob), "fp32")
+
+
+def test_c2_shape_bf16_truncated(H):
+    """Config 2's layer sizes (I512 H512 B64, bf16) on a shortened sequence."""
+    cfg = _cfg("c2", t=24)
+    dp = H.DeviceProblem(cfg)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, "bf16")
+    for mode, m in [("hsm", 4), ("ism", 4)]:
+        plan = dp.plan(mode, m)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost
+        assert_bit_identical(res, full)
+
+
+def test_host_buffer_entry_point(H):
+    import torch
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg("c1", t=16)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    plan = dp.plan("hsm", 4)
+    dev = dp.run(plan)
+    h = dp.host
+    out = {k: np.zeros_like(v) for k, v in dev.items() if isinstance(v, np.ndarray)}
+    loss = np.zeros(1, np.float32)
+    ws = torch.empty(B.mebptt_lstm_host_workspace_bytes(dp.desc, plan), dtype=torch.uint8, device="cuda:0")
+    B.mebptt_lstm_train_step_host(dp.desc, plan, h["W"], h["b"], h["W_out"], h["b_out"], h["x"],
+                                  h["targets"], h["h0"], h["c0"], ws, None, loss, out["dW"], out["db"],
+                                  out["dW_out"], out["db_out"], out["dx"], out["counters"])
+    torch.cuda.synchronize()
+    out["loss"] = float(loss[0])
+    assert_bit_identical(out, dev, want_dx=True)
+    assert out["counters"][0] == plan.cost
+
+
+def test_workspace_errors(H):
+    import torch
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg("c1", t=8)
+    dp = H.DeviceProblem(cfg)
+    plan = dp.plan("hsm", 3)
+    need = B.mebptt_lstm_workspace_bytes(dp.desc, plan)
+    d, o = dp.dev, dp.out
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(B.MebpttError) as e:
+        B.mebptt_lstm_train_step(dp.desc, plan, d["W"], d["b"], d["W_out"], d["b_out"], d["x"], d["targets"],
+                                 d["h0"], d["c0"], small, None, o["loss"], o["dW"], o["db"], o["dW_out"],
+                                 o["db_out"], None, o["counters"])
+    assert e.value.status == B.MEBPTT_ERR_WORKSPACE
+    big = torch.empty(need + 512, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(B.MebpttError) as e:
+        B.mebptt_lstm_train_step(dp.desc, plan, d["W"], d["b"], d["W_out"], d["b_out"], d["x"], d["targets"],
+                                 d["h0"], d["c0"], big[16:], None, o["loss"], o["dW"], o["db"], o["dW_out"],
+                                 o["db_out"], None, o["counters"])
+    assert e.value.status == B.MEBPTT_ERR_WORKSPACE
+
+
+def test_slot_copy(H):
+    import torch
+    from paper_1606_03401_b200 import binding as B
+    src = torch.randint(0, 255, (1 << 20) + 48, dtype=torch.uint8, device="cuda:0")
+    dst = torch.zeros_like(src)
+    B.mebptt_slot_copy(dst, src, src.numel(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert torch.equal(src, dst)
