@@ -152,7 +152,7 @@ def test_workspace_errors(H):
 def test_slot_copy(H):
     import torch
     from paper_1606_03401_b200 import binding as B
-    src = torch.randint(0, 255, (1 << 20) + 48, dtype=torch.uint8, device="cuda:0")
+    src = torch.randint(0, 255, ((1 << 20) + 48,), dtype=torch.uint8, device="cuda:0")
     dst = torch.zeros_like(src)
     B.mebptt_slot_copy(dst, src, src.numel(), torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
