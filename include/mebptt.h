@@ -265,6 +265,21 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_
  */
 int mebptt_slot_copy(void *dst, const void *src, size_t bytes, void *stream);
 
+/*
+ * The batched contraction the training step uses for everything that is off the recurrence
+ * (input projections, readout, weight gradients), exposed for testing and reuse:
+ *     C[M][N] (+)= sum_k A(m,k) B(n,k)
+ * over bfloat16 operands with float32 accumulation on the tensor cores.  a_major / b_major:
+ * 0 = the operand is stored [m][k] (contraction index contiguous), 1 = stored [k][m].
+ * lda / ldb: row strides in elements, multiples of 8; A, B 16-byte aligned.  C is float32
+ * [M][ldc]; accumulate != 0 adds to it.  bias (nullable): float32 [N], added per column.
+ * status (nullable): device int, set to MEBPTT_ERR_TIMEOUT if a bounded wait expires.
+ * All pointers are device pointers.  No counterpart in the paper beyond "the RNN core".
+ */
+int mebptt_gemm_bf16(const void *A, int64_t lda, int a_major, const void *B, int64_t ldb, int b_major,
+                     float *C, int64_t ldc, int accumulate, const float *bias,
+                     int64_t M, int64_t N, int64_t K, int *status, void *stream);
+
 const char *mebptt_strerror(int status);
 
 #ifdef __cplusplus

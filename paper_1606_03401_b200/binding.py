@@ -80,6 +80,7 @@ _SIGS = {
     "mebptt_lstm_train_step": (_i32, _STEP_ARGS),
     "mebptt_lstm_train_step_host": (_i32, _STEP_ARGS),
     "mebptt_slot_copy": (_i32, [_vp, _vp, _sz, _vp]),
+    "mebptt_gemm_bf16": (_i32, [_vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "mebptt_strerror": (C.c_char_p, [_i32]),
 }
 for _name, (_res, _args) in _SIGS.items():
@@ -232,6 +233,12 @@ def mebptt_lstm_train_step_host(desc, plan, W, b, W_out, b_out, x, targets, h0, 
     is a device tensor of at least mebptt_lstm_host_workspace_bytes()."""
     _step(lib.mebptt_lstm_train_step_host, "mebptt_lstm_train_step_host", desc, plan, W, b, W_out,
           b_out, x, targets, h0, c0, workspace, stream, loss, dW, db, dW_out, db_out, dx, counters)
+
+
+def mebptt_gemm_bf16(A, lda, a_major, Bm, ldb, b_major, Cm, ldc, accumulate, bias, M, N, K, status=None,
+                     stream=None):
+    _check(lib.mebptt_gemm_bf16(_ptr(A), lda, a_major, _ptr(Bm), ldb, b_major, _ptr(Cm), ldc, int(accumulate),
+                                _ptr(bias), M, N, K, _ptr(status), stream), "mebptt_gemm_bf16")
 
 
 def mebptt_slot_copy(dst, src, nbytes: int, stream=None):

@@ -9,6 +9,7 @@
 #include "layout.hpp"
 #include "mebptt.h"
 #include "plan.hpp"
+#include "tc.hpp"
 
 using namespace mebptt;
 
@@ -277,6 +278,19 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
   if (desc->want_dx) cudaMemcpyAsync(dx, ws + g.dx, g.ndx, cudaMemcpyDeviceToHost, s);
   cudaMemcpyAsync(counters, ws + g.counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost, s);
   return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+}
+
+int mebptt_gemm_bf16(const void* A, int64_t lda, int a_major, const void* B, int64_t ldb, int b_major, float* C,
+                     int64_t ldc, int accumulate, const float* bias, int64_t M, int64_t N, int64_t K, int* status,
+                     void* stream) {
+  if (!A || !B || !C || M < 1 || N < 1 || K < 1 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30))
+    return MEBPTT_ERR_ARG;
+  if ((lda & 7) || (ldb & 7) || (reinterpret_cast<uintptr_t>(A) & 15) || (reinterpret_cast<uintptr_t>(B) & 15))
+    return MEBPTT_ERR_ARG;
+  if ((a_major != 0 && a_major != 1) || (b_major != 0 && b_major != 1)) return MEBPTT_ERR_ARG;
+  tc::GemmOut out{accumulate ? tc::GemmOut::ACCUM_F32 : tc::GemmOut::STORE_F32, C, ldc, bias};
+  return tc::gemm_bf16(A, lda, a_major == 1, B, ldb, b_major == 1, out, (int)M, (int)N, (int)K, status,
+                       (cudaStream_t)stream);
 }
 
 int mebptt_slot_copy(void* dst, const void* src, size_t bytes, void* stream) {

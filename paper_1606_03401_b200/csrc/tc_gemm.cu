@@ -1,0 +1,199 @@
+// Batched-over-time contractions on the tensor cores: C[M][N] (+)= sum_k A(m,k) B(n,k) with
+// bfloat16 operands and float32 accumulation in TMEM.
+//
+// These are the parts of the training step that do not sit on the recurrence and can therefore
+// be run for many time steps at once:
+//   input projection   Zx[(s,b)][g]  = sum_i x[(s,b)][i] W_ih[g][i] + bias[g]         (A, B K-major)
+//   readout            y[(s,b)][o]   = sum_j h[(s,b)][j] W_out[o][j]                 (A, B K-major)
+//   readout backward   dha[(s,b)][j] = sum_o dy[(s,b)][o] W_out^T[j][o]              (A, B K-major)
+//   weight gradients   dW[g][c]     += sum_(s,b) dz[(s,b)][g] in[(s,b)][c]           (A, B MN-major)
+// "K-major" means the operand is stored with the contraction index contiguous; "MN-major" that it
+// is stored [k][m] (rows are contraction indices), which is how dz and the layer inputs lie in
+// memory for the weight gradient, so no transposed copies are made.
+//
+// One CTA computes one 128 x 128 tile.  A single thread feeds a 3-stage ring of 128-byte
+// swizzled shared-memory tiles by TMA (64 contraction indices per stage); a single thread issues
+// tcgen05.mma (M = 128, N = 128, K = 16, four per stage) into a 128-column TMEM accumulator and
+// releases ring slots with tcgen05.commit; then all four warps read the accumulator with
+// tcgen05.ld (warp w owns TMEM lanes 32w .. 32w+31 = tile rows) and write the tile.
+// Out-of-range parts of a tile are zero-filled by TMA on the way in and masked on the way out.
+// The sum over k runs in one fixed order, so results do not depend on how callers batch steps.
+#include "sm100.cuh"
+#include "tc.hpp"
+#include "tmap.hpp"
+
+namespace mebptt {
+namespace tc {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;  // + slack to align the ring to 1024 B
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma,
+                                                        const __grid_constant__ CUtensorMap tmb, GemmOut out,
+                                                        int M, int N, int K, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full[STAGES], empty[STAGES], done;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int nk = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&done, 1);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tma);
+    tma_prefetch_desc(&tmb);
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 128);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer -----------------------------------------------------------------------
+    int armed = 0;  // stages whose full barrier still awaits bytes (for the failure path)
+    for (int kb = 0; kb < nk; ++kb) {
+      const int s = kb % STAGES;
+      if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { failed = 1; break; }
+      uint8_t* sA = ring + s * STAGE_BYTES;
+      uint8_t* sB = sA + A_BYTES;
+      mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
+      ++armed;
+      if (A_MN) {
+        tma_load_2d(sA, &tma, m0, kb * BK, &full[s]);
+        tma_load_2d(sA + 8192, &tma, m0 + 64, kb * BK, &full[s]);
+      } else {
+        tma_load_2d(sA, &tma, kb * BK, m0, &full[s]);
+      }
+      if (B_MN) {
+        tma_load_2d(sB, &tmb, n0, kb * BK, &full[s]);
+        tma_load_2d(sB + 8192, &tmb, n0 + 64, kb * BK, &full[s]);
+      } else {
+        tma_load_2d(sB, &tmb, kb * BK, n0, &full[s]);
+      }
+    }
+    (void)armed;
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer ---------------------------------------------------------------------
+    constexpr uint32_t idesc = make_idesc(1, BM, BN, A_MN, B_MN);
+    bool ok = true;
+    for (int kb = 0; kb < nk && ok; ++kb) {
+      const int s = kb % STAGES;
+      if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { failed = 1; ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t a0 = smem_u32(ring + s * STAGE_BYTES), b0 = a0 + A_BYTES;
+#pragma unroll
+      for (int k4 = 0; k4 < BK / 16; ++k4) {
+        // K-major: 16 contraction indices = 32 B along the row; MN-major: 16 rows of 128 B
+        const uint64_t da = A_MN ? make_desc_sw128(a0 + k4 * 2048, 8192, 1024) : make_desc_sw128(a0 + k4 * 32, 16, 1024);
+        const uint64_t db = B_MN ? make_desc_sw128(b0 + k4 * 2048, 8192, 1024) : make_desc_sw128(b0 + k4 * 32, 16, 1024);
+        mma_f16(tmem, da, db, idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+      }
+      mma_commit(&empty[s]);  // the slot may be refilled once these MMAs have read it
+    }
+    mma_commit(&done);
+  }
+
+  // ---- epilogue: all four warps ---------------------------------------------------------
+  __syncwarp();
+  bool ok = mbar_wait(&done, 0);
+  tc_fence_after_sync();
+  if (ok && !failed) {
+    const int row = m0 + warp * 32 + lane;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+      tmem_ld_wait();
+      const int col0 = n0 + c * 32;
+      if (row < M) {
+        if (out.kind == GemmOut::STORE_BF16) {
+          __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row * out.ld + col0;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < N) p[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
+        } else {
+          float* p = reinterpret_cast<float*>(out.ptr) + (size_t)row * out.ld + col0;
+          const bool vec = (col0 + 32 <= N) && ((reinterpret_cast<uintptr_t>(p) & 15) == 0);
+          if (vec) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                     __uint_as_float(r[j + 3]));
+              if (out.bias) {
+                v.x += out.bias[col0 + j]; v.y += out.bias[col0 + j + 1];
+                v.z += out.bias[col0 + j + 2]; v.w += out.bias[col0 + j + 3];
+              }
+              if (out.kind == GemmOut::ACCUM_F32) {
+                const float4 o = *reinterpret_cast<const float4*>(p + j);
+                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+              }
+              *reinterpret_cast<float4*>(p + j) = v;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < N) {
+                float v = __uint_as_float(r[j]);
+                if (out.bias) v += out.bias[col0 + j];
+                if (out.kind == GemmOut::ACCUM_F32) v += p[j];
+                p[j] = v;
+              }
+          }
+        }
+      }
+    }
+  } else if (status && threadIdx.x == 0) {
+    *status = MEBPTT_ERR_TIMEOUT;
+  }
+  // On the failure path the producer may still have loads in flight: give them a bounded
+  // chance to land before the shared memory goes away.
+  if (failed && warp == 0 && lane == 0)
+    for (int s = 0; s < STAGES; ++s) (void)mbar_wait(&full[s], 0);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 128);
+}
+
+}  // namespace
+
+int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
+              int M, int N, int K, int* status, cudaStream_t s) {
+  if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
+  CUtensorMap ta, tb;
+  // K-major: tensor is [M][K], box 64 (k) x 128 rows.  MN-major: tensor is [K][M], box 64 (m) x 64 rows.
+  bool ok = a_mn ? make_tmap_2d(&ta, A, 2, (uint64_t)M, (uint64_t)K, (uint64_t)lda * 2, 64, 64)
+                 : make_tmap_2d(&ta, A, 2, (uint64_t)K, (uint64_t)M, (uint64_t)lda * 2, 64, 128);
+  ok = ok && (b_mn ? make_tmap_2d(&tb, B, 2, (uint64_t)N, (uint64_t)K, (uint64_t)ldb * 2, 64, 64)
+                   : make_tmap_2d(&tb, B, 2, (uint64_t)K, (uint64_t)N, (uint64_t)ldb * 2, 64, 128));
+  if (!ok) return MEBPTT_ERR_UNSUPPORTED;
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  static const bool attrs = [] {
+    cudaFuncSetAttribute(gemm_bf16_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    cudaFuncSetAttribute(gemm_bf16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    cudaFuncSetAttribute(gemm_bf16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    cudaFuncSetAttribute(gemm_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    return true;
+  }();
+  (void)attrs;
+  if (a_mn && b_mn) gemm_bf16_kernel<true, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
+  else if (!a_mn && !b_mn) gemm_bf16_kernel<false, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
+  else if (a_mn) gemm_bf16_kernel<true, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
+  else gemm_bf16_kernel<false, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
+  return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+}
+
+}  // namespace tc
+}  // namespace mebptt
