@@ -190,9 +190,13 @@ typedef struct {
   int32_t batch;    /* B                                              */
   int32_t dtype;    /* MEBPTT_FP32 | MEBPTT_TF32 | MEBPTT_BF16        */
   int32_t want_dx;  /* 1: also return dL/dx                           */
-  int32_t reserved; /* 0                                              */
+  int32_t flags;    /* MEBPTT_FLAG_* or 0                             */
   int64_t t;        /* sequence length; must equal the plan's         */
 } mebptt_lstm_desc;
+
+/* Run on the CUDA-core kernels even where the tensor-core kernels cover the shape (the two
+ * paths round differently; results are deterministic within each). */
+enum { MEBPTT_FLAG_NO_TENSOR_CORES = 1 };
 
 /* Bytes of one hidden-state unit (all layers) for this descriptor; 0 on a bad descriptor. */
 size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc *desc);

@@ -46,7 +46,7 @@ OP_DTYPE = np.dtype([("kind", "<i4"), ("k", "<i4"), ("src", "<i4"), ("dst", "<i4
 class mebptt_lstm_desc(C.Structure):
     _fields_ = [("layers", C.c_int32), ("input", C.c_int32), ("hidden", C.c_int32),
                 ("readout", C.c_int32), ("batch", C.c_int32), ("dtype", C.c_int32),
-                ("want_dx", C.c_int32), ("reserved", C.c_int32), ("t", C.c_int64)]
+                ("want_dx", C.c_int32), ("flags", C.c_int32), ("t", C.c_int64)]
 
 
 _vp, _i64, _i32, _sz = C.c_void_p, C.c_int64, C.c_int, C.c_size_t
@@ -168,10 +168,13 @@ def mebptt_plan_ex(t: int, m: int, mode: int, alpha: int = 4, beta: int = 0) -> 
     return Plan(h)
 
 
-def make_desc(layers, input, hidden, readout, batch, t, dtype, want_dx=0) -> mebptt_lstm_desc:
+MEBPTT_FLAG_NO_TENSOR_CORES = 1
+
+
+def make_desc(layers, input, hidden, readout, batch, t, dtype, want_dx=0, flags=0) -> mebptt_lstm_desc:
     if isinstance(dtype, str):
         dtype = DTYPES[dtype]
-    return mebptt_lstm_desc(layers, input, hidden, readout, batch, dtype, int(want_dx), 0, t)
+    return mebptt_lstm_desc(layers, input, hidden, readout, batch, dtype, int(want_dx), int(flags), t)
 
 
 def mebptt_lstm_unit_bytes(desc) -> int:

@@ -15,13 +15,7 @@ using namespace mebptt;
 
 namespace {
 
-struct StepIO {
-  const char *W, *W_out, *x, *h0;
-  const float *b, *b_out, *targets, *c0;
-  char* ws;
-  float *loss, *dW, *db, *dW_out, *db_out, *dx;
-  int64_t* counters;
-};
+using StepIO = tc::StepPtrs;
 
 // Base address of the hidden block (or record) at a tape location; LOC_INIT has none.
 inline char* loc_base(const Layout& y, char* ws, int32_t loc) {
@@ -56,6 +50,7 @@ int check_common(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
 }
 
 int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const StepIO& io, cudaStream_t s) {
+  if (y.tensor_path) return (int)tc::run_step(y, p, io, desc->want_dx != 0, s, false);
   const size_t bh = (size_t)y.B * y.H;
   const size_t plane_elems = y.plane / y.esz;
   char* ws = io.ws;
@@ -192,12 +187,15 @@ size_t mebptt_lstm_working_bytes(const mebptt_lstm_desc* desc, const mebptt_plan
   if (check_common(desc, plan) != MEBPTT_OK) return 0;
   Layout y;
   workspace_layout(desc, reinterpret_cast<const Plan*>(plan), y);
-  return y.total - align_up((size_t)y.arena_units * y.unit, 256);
+  return y.total - y.off_core;
 }
 
 int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
   if (check_common(desc, plan) != MEBPTT_OK) return -1;
   const Plan* p = reinterpret_cast<const Plan*>(plan);
+  Layout y;
+  workspace_layout(desc, p, y);
+  if (y.tensor_path) return tc::run_step(y, p, StepIO{}, desc->want_dx != 0, nullptr, true);
   // forward operation: one kernel per layer; backward operation: 5 for the readout and
   // 4 per layer; one to finalise
   const int64_t L = desc->layers;
@@ -288,7 +286,7 @@ int mebptt_gemm_bf16(const void* A, int64_t lda, int a_major, const void* B, int
   if ((lda & 7) || (ldb & 7) || (reinterpret_cast<uintptr_t>(A) & 15) || (reinterpret_cast<uintptr_t>(B) & 15))
     return MEBPTT_ERR_ARG;
   if ((a_major != 0 && a_major != 1) || (b_major != 0 && b_major != 1)) return MEBPTT_ERR_ARG;
-  tc::GemmOut out{accumulate ? tc::GemmOut::ACCUM_F32 : tc::GemmOut::STORE_F32, C, ldc, bias};
+  tc::GemmOut out{accumulate ? tc::GemmOut::ACCUM_F32 : tc::GemmOut::STORE_F32, C, ldc, bias, 0};
   return tc::gemm_bf16(A, lda, a_major == 1, B, ldb, b_major == 1, out, (int)M, (int)N, (int)K, status,
                        (cudaStream_t)stream);
 }

@@ -5,6 +5,10 @@
 // planes i, f, g, o of every layer (operand type, each [B][H]) and a copy of the input hidden
 // state.  The output hidden state comes first, so that a forward operation can read "the hidden
 // state at a location" without knowing which of the two formats the location holds.
+//
+// Every block starts at a multiple of `granule` = lcm(256, H * element size) bytes from the
+// workspace base: the tensor-core path addresses h blocks through one TMA tensor map that views
+// the whole workspace as rows of H elements, so a block's offset must be a whole number of rows.
 #pragma once
 
 #include <cstddef>
@@ -16,25 +20,35 @@
 namespace mebptt {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t gcd_sz(size_t a, size_t b) { while (b) { size_t r = a % b; a = b; b = r; } return a; }
 
 struct Layout {
   int L = 0, I = 0, H = 0, O = 0, B = 0;
   int dtype = 0;
   int64_t t = 0;
+  bool tensor_path = false;
   size_t esz = 0;        // bytes of one operand element
-  size_t hsz = 0;        // one layer's h, padded to 16 B
+  size_t granule = 0;
+  size_t hsz = 0;        // one layer's h
   size_t csz = 0;        // one layer's c
   size_t gsz = 0;        // one layer's four gate planes
-  size_t plane = 0;      // one gate plane, padded to 16 B
-  size_t unit = 0;       // one hidden state of the stack, padded to 256 B
+  size_t plane = 0;      // one gate plane
+  size_t unit = 0;       // one hidden state of the stack
   size_t rec = 0;        // one internal state
   // record-relative offsets
   size_t rec_gates = 0;  // gates of layer 0
   size_t rec_in = 0;     // input hidden state
-  // workspace offsets
-  size_t off_arena = 0, off_core = 0, off_ping = 0, off_pong = 0;
+  // workspace offsets: states
+  size_t off_arena = 0, off_core = 0, off_ping = 0, off_pong = 0, off_init = 0;
+  // carried gradients and per-step scratch of the CUDA-core path
   size_t off_dh = 0, off_dc = 0, off_dha = 0, off_dz = 0, off_dy = 0;
   size_t off_loss_part = 0, off_loss_t = 0;
+  // tensor-core path: packed weights, staging of S consecutive time steps, control
+  int S = 0;             // time steps per staged chunk
+  size_t off_wp_ih = 0, off_wp_hh = 0, off_wpT_hh = 0, off_wpT_ih = 0, off_bias_p = 0, off_woutT = 0;
+  size_t off_zx = 0, off_hprev = 0, off_hk = 0, off_y = 0;
+  size_t off_sync = 0, off_tape = 0, off_status = 0;
+  size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
   int64_t arena_units = 0;
   int n_loss_part = 0;
@@ -58,19 +72,32 @@ inline bool valid_desc(const mebptt_lstm_desc* d) {
   if (d->input > (1 << 16) || d->hidden > (1 << 16) || d->readout > (1 << 16) || d->batch > (1 << 16)) return false;
   if (d->dtype != MEBPTT_FP32 && d->dtype != MEBPTT_TF32 && d->dtype != MEBPTT_BF16) return false;
   if (d->want_dx != 0 && d->want_dx != 1) return false;
+  if (d->flags & ~MEBPTT_FLAG_NO_TENSOR_CORES) return false;
   return true;
+}
+
+// Shapes the tensor-core kernels cover: one layer, bfloat16 operands, a batch that fits one MMA
+// tile, sizes that keep every TMA stride a multiple of 16 bytes, and a recurrent weight slice per
+// CTA (8 hidden units x 4 gates x H) that fits in shared memory with one CTA per SM.
+inline bool tensor_path_supported(const mebptt_lstm_desc* d) {
+  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && d->dtype == MEBPTT_BF16 && d->layers == 1 && d->batch <= 64 && d->hidden % 8 == 0 &&
+         d->input % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 && d->hidden / 8 <= 148 &&
+         d->hidden <= 1184;
 }
 
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
   y.dtype = d->dtype; y.t = d->t;
+  y.tensor_path = tensor_path_supported(d);
   y.esz = (d->dtype == MEBPTT_BF16) ? 2 : 4;
+  const size_t row = (size_t)y.H * y.esz;
+  y.granule = 256 / gcd_sz(256, row) * row;  // lcm(256, row bytes)
   const size_t bh = (size_t)y.B * y.H;
-  y.hsz = align_up(bh * y.esz, 16);
-  y.csz = align_up(bh * 4, 16);
-  y.plane = align_up(bh * y.esz, 16);
+  y.hsz = align_up(bh * y.esz, y.granule);
+  y.csz = align_up(bh * 4, y.granule);
+  y.plane = align_up(bh * y.esz, y.granule);
   y.gsz = 4 * y.plane;
-  y.unit = align_up((size_t)y.L * (y.hsz + y.csz), 256);
+  y.unit = (size_t)y.L * (y.hsz + y.csz);
   y.rec_gates = y.unit;
   y.rec_in = y.unit + (size_t)y.L * y.gsz;
   y.rec = y.rec_in + y.unit;
@@ -80,7 +107,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
   state_layout(d, y);
   y.arena_units = p->arena_units;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, y.granule); return r; };
   y.off_arena = take((size_t)y.arena_units * y.unit);
   y.off_core = take(y.rec);
   y.off_ping = take(y.unit);
@@ -88,12 +115,39 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
   const size_t bh4 = (size_t)y.B * y.H * 4;
   y.off_dh = take((size_t)y.L * bh4);
   y.off_dc = take((size_t)y.L * bh4);
-  y.off_dha = take(bh4);
-  y.off_dz = take((size_t)y.B * 4 * y.H * 4);
-  y.off_dy = take((size_t)y.B * y.O * 4);
-  y.n_loss_part = ((y.B + 63) / 64) * ((y.O + 63) / 64);
-  y.off_loss_part = take((size_t)y.n_loss_part * 4);
   y.off_loss_t = take((size_t)y.t * 4);
+  if (!y.tensor_path) {
+    y.off_dha = take(bh4);
+    y.off_dz = take((size_t)y.B * 4 * y.H * 4);
+    y.off_dy = take((size_t)y.B * y.O * 4);
+    y.n_loss_part = ((y.B + 63) / 64) * ((y.O + 63) / 64);
+    y.off_loss_part = take((size_t)y.n_loss_part * 4);
+  } else {
+    const size_t G = (size_t)4 * y.H;
+    y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
+    if (y.S > 64) y.S = 64;
+    const size_t SB = (size_t)y.S * y.B;
+    y.off_init = take(y.unit);
+    y.off_wp_ih = take(G * y.I * 2);
+    y.off_wp_hh = take(G * y.H * 2);
+    y.off_wpT_hh = take(G * y.H * 2);
+    y.off_wpT_ih = take(d->want_dx ? G * y.I * 2 : 0);
+    y.off_bias_p = take(G * 4);
+    y.off_woutT = take((size_t)y.O * y.H * 2);
+    y.off_zx = take(SB * G * 4);
+    y.off_dz = take(SB * G * 2);
+    y.off_hprev = take(SB * y.H * 2);
+    y.off_hk = take(SB * y.H * 2);
+    y.off_y = take(SB * y.O * 4);
+    y.off_dy = take(SB * y.O * 2);
+    y.off_dha = take(SB * y.H * 4);
+    y.off_loss_part = take((size_t)y.S * 16 * 4);
+    y.n_sync = (size_t)p->tape.size() + 8;
+    y.off_sync = take(y.n_sync * 4);
+    y.tape_bytes = (size_t)p->tape.size() * 32;
+    y.off_tape = take(y.tape_bytes);
+    y.off_status = take(256);
+  }
   y.total = o;
 }
 

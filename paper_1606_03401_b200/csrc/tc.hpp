@@ -18,6 +18,16 @@ struct GemmOut {
   void* ptr;          // [M][ld]
   int64_t ld;         // elements
   const float* bias;  // optional, per column, float32 outputs only
+  int perm_h;         // > 0: tile row 4 u + q is written to row q * perm_h + u (undoes the gate permutation)
+};
+
+// Caller buffers of one training step (device pointers).
+struct StepPtrs {
+  const char *W, *W_out, *x, *h0;
+  const float *b, *b_out, *targets, *c0;
+  char* ws;
+  float *loss, *dW, *db, *dW_out, *db_out, *dx;
+  int64_t* counters;
 };
 
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
@@ -26,5 +36,13 @@ struct GemmOut {
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
               int M, int N, int K, int* status, cudaStream_t s);
 
+}  // namespace tc
+
+struct Layout;
+struct Plan;
+namespace tc {
+// Enqueues one training step on the tensor-core path; returns a status.  With dry = true
+// nothing is enqueued and the number of kernel launches is returned instead.
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry);
 }  // namespace tc
 }  // namespace mebptt

@@ -112,6 +112,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   tc_fence_after_sync();
   if (ok && !failed) {
     const int row = m0 + warp * 32 + lane;
+    const int row_o = out.perm_h ? ((row & 3) * out.perm_h + (row >> 2)) : row;
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
       uint32_t r[32];
@@ -120,12 +121,12 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       const int col0 = n0 + c * 32;
       if (row < M) {
         if (out.kind == GemmOut::STORE_BF16) {
-          __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row * out.ld + col0;
+          __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row_o * out.ld + col0;
 #pragma unroll
           for (int j = 0; j < 32; ++j)
             if (col0 + j < N) p[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
         } else {
-          float* p = reinterpret_cast<float*>(out.ptr) + (size_t)row * out.ld + col0;
+          float* p = reinterpret_cast<float*>(out.ptr) + (size_t)row_o * out.ld + col0;
           const bool vec = (col0 + 32 <= N) && ((reinterpret_cast<uintptr_t>(p) & 15) == 0);
           if (vec) {
 #pragma unroll

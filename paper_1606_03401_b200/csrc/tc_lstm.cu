@@ -1,0 +1,847 @@
+// The LSTM recurrence on the tensor cores (bfloat16 operands, float32 accumulation and cell
+// state), one layer.
+//
+// What sits on the recurrence, and therefore cannot be batched over time, is only the
+// product with the recurrent weights: z_t = Zx_t + h_{t-1} W_hh^T going forward and
+// dh_{t-1} = dz_t W_hh going backward.  Both run in persistent kernels that walk a run of
+// consecutive tape operations with W_hh resident in shared memory:
+//
+//   fwd_run_kernel   CTA c owns hidden units 8c .. 8c+7, i.e. the 32 gate rows {i,f,g,o} x 8 of
+//                    W_hh, permuted so that the four gates of a unit are adjacent columns.  Per
+//                    step: TMA streams h_{t-1} ([B][H], 64 columns at a time) through a ring,
+//                    one thread issues tcgen05.mma (M = 64 or 128 batch rows, N = 32, K = 16)
+//                    into TMEM, then each thread owning a batch row reads its 32 accumulators,
+//                    adds the batched input projection Zx_t (bias included), applies the gates
+//                    and updates c_t, h_t for its 8 units -- c_t and h_t stay in registers from
+//                    step to step -- and writes the state where the tape says (scratch, a slot
+//                    of the arena, or a whole internal state).
+//   bwd_run_kernel   same ownership.  Per step each thread forms dz for its 8 units x 4 gates
+//                    from dh (read back from TMEM), dc (registers), the stored gates and cell
+//                    states, writes dz (bfloat16) to the staging chunk, and the CTA then
+//                    contracts the whole dz_t ([B][4H]) against its 8 rows of W_hh^T
+//                    (M = batch, N = 8, K = 16) to get its slice of dh_{t-1}.
+//
+// Between steps every CTA needs all of h_t (or dz_t): a grid-wide counter in global memory is
+// bumped by each CTA after its stores (release) and polled by the one thread that issues the
+// next step's TMA loads (acquire), with a proxy fence on both sides because the loads go
+// through the async proxy.  The kernels are launched cooperatively, so all CTAs are resident
+// and the wait cannot deadlock; it is bounded all the same.
+//
+// Everything off the recurrence is batched over S consecutive time steps and done by the
+// tensor-core GEMM: input projections before a forward run; readout, its gradient, and -- once
+// the backward pass has completed a chunk of S steps aligned to absolute time -- the weight
+// gradients.  Chunks are tied to time indices, not to run boundaries, and backward steps always
+// come in the order t .. 1, so every sum runs in the same order under every plan.
+#include <cstdio>
+#include <cstdlib>
+#include <vector>
+
+#include "layout.hpp"
+#include "sm100.cuh"
+#include "tc.hpp"
+#include "tmap.hpp"
+
+namespace mebptt {
+namespace tc {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int NU = 8;            // hidden units per CTA
+constexpr int NG = 4 * NU;       // gate columns per CTA
+constexpr int NST = 8;           // ring stages of 64 contraction indices
+constexpr int LOSS_PARTS = 16;   // partial sums per step of the loss
+
+// Tape entry as the kernels see it.  Offsets are in units of 16 bytes from the workspace base.
+struct DevOp {
+  int32_t k;
+  int32_t fmt;
+  uint32_t h_src, c_src;   // FWD: state k-1.            BWD: h_{k-1}, c_{k-1}
+  uint32_t h_dst, c_dst;   // FWD: where h_k, c_k go.    BWD: h_k, c_k of the stored internal state
+  uint32_t gates;          // FWD: gate planes to write, 0 = none.   BWD: gate planes to read
+  uint32_t in_copy;        // FWD: hidden block receiving the copy of state k-1, 0 = none
+};
+static_assert(sizeof(DevOp) == 32, "DevOp layout");
+
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ bool wait_or_fail(uint64_t* bar, uint32_t parity, volatile int* failed) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 256) {
+      if (*failed) return false;
+      __nanosleep(64);
+    }
+  }
+  *failed = 1;
+  return false;
+}
+__device__ __forceinline__ bool wait_counter(const uint32_t* ctr, uint32_t target, volatile int* failed) {
+  for (uint32_t i = 0; i < (kSpinLimit >> 1); ++i) {
+    if (ld_acquire(ctr) >= target) return true;
+    if (i > 4096 && *failed) return false;
+  }
+  *failed = 1;
+  return false;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+// ------------------------------------------------------------------------------------------
+// forward run
+// ------------------------------------------------------------------------------------------
+struct FwdRunArgs {
+  const DevOp* ops;      // this launch's operations (consecutive forward operations)
+  int n;
+  char* ws;              // workspace base
+  const float* zx;       // [n][B][4H]: input projection + bias, gate columns permuted (4 u + q)
+  uint32_t* sync;        // grid-wide step counter of this launch (zero on entry)
+  int* status;
+  int64_t* counters;
+  int B, H;
+  uint32_t plane16;      // distance between gate planes, in 16-byte units
+  uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
+};
+
+template <int BM>
+__global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__ CUtensorMap tm_h,
+                                                         const __grid_constant__ CUtensorMap tm_w,
+                                                         const FwdRunArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t wfull, full[NST], empty[NST], acc;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int KB = (a.H + 63) / 64;
+  uint8_t* sW = sm;                    // KB tiles of [32 rows][128 B]
+  uint8_t* ring = sm + KB * 4096;      // NST tiles of [BM rows][128 B]
+  constexpr uint32_t A_TILE = BM * 128;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, ncta = gridDim.x;
+  const bool is_p = (tid == 0), is_mma = (tid == 32);
+
+  if (tid == 0) {
+    mbar_init(&wfull, 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&acc, 1);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_h);
+    tma_prefetch_desc(&tm_w);
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 32);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  // the recurrent weights of this CTA's 8 units stay in shared memory for the whole run
+  if (is_p) {
+    mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 4096u);
+    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 4096, &tm_w, kb * 64, cta * NG, &wfull);
+  }
+
+  // ---- per-thread state: one batch row, the CTA's 8 hidden units ---------------------------
+  const int b = (BM == 64) ? (16 * warp + lane) : (32 * warp + lane);
+  const bool owner = ((BM == 64) ? (lane < 16) : true) && b < a.B;
+  const int j0 = cta * NU;
+  const size_t e0 = (size_t)b * a.H + j0;           // element index of (b, j0) in a [B][H] array
+  float c[NU];
+  uint4 hprev = make_uint4(0, 0, 0, 0);
+  float zx[NG];
+  {
+    const DevOp op0 = a.ops[0];
+    if (owner) {
+      const float* cp = reinterpret_cast<const float*>(a.ws + (size_t)op0.c_src * 16) + e0;
+      const float4 c0 = *reinterpret_cast<const float4*>(cp), c1 = *reinterpret_cast<const float4*>(cp + 4);
+      c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
+      hprev = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op0.h_src * 16) + e0);
+      const float4* zp = reinterpret_cast<const float4*>(a.zx + (size_t)b * 4 * a.H + (size_t)cta * NG);
+#pragma unroll
+      for (int v = 0; v < NG / 4; ++v) {
+        const float4 z = zp[v];
+        zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < NU; ++u) c[u] = 0.f;
+#pragma unroll
+      for (int v = 0; v < NG; ++v) zx[v] = 0.f;
+    }
+  }
+
+  uint32_t issued = 0;      // ring tiles requested so far (producer thread)
+  uint32_t consumed = 0;    // ring tiles multiplied so far (MMA thread)
+  constexpr uint32_t idesc = make_idesc(1, BM, NG, false, false);
+  const uint32_t row_bytes = (uint32_t)a.H * 2u;
+
+  for (int i = 0; i < a.n; ++i) {
+    const DevOp op = a.ops[i];
+    if (is_p) {
+      // ---- producer: h_{k-1} through the ring -------------------------------------------
+      bool ok = true;
+      if (i > 0) ok = wait_counter(a.sync, (uint32_t)i * (uint32_t)ncta, &failed);
+      if (ok) {
+        fence_proxy_async();
+        const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
+        for (int kb = 0; kb < KB && ok; ++kb, ++issued) {
+          const uint32_t s = issued % NST, it = issued / NST;
+          if (it > 0) ok = wait_or_fail(&empty[s], (it - 1) & 1, &failed);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full[s], A_TILE);
+          tma_load_2d(ring + s * A_TILE, &tm_h, kb * 64, row, &full[s]);
+        }
+      }
+    } else if (is_mma) {
+      // ---- MMA issuer -----------------------------------------------------------------------
+      bool ok = true;
+      if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
+      for (int kb = 0; kb < KB && ok; ++kb, ++consumed) {
+        const uint32_t s = consumed % NST, it = consumed / NST;
+        ok = wait_or_fail(&full[s], it & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a0 = smem_u32(ring + s * A_TILE), b0 = smem_u32(sW + kb * 4096);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          mma_f16(tmem, make_desc_sw128(a0 + k4 * 32, 16, 1024), make_desc_sw128(b0 + k4 * 32, 16, 1024), idesc,
+                  (kb > 0 || k4 > 0) ? 1u : 0u);
+        mma_commit(&empty[s]);
+      }
+      mma_commit(&acc);
+    }
+    __syncwarp();
+
+    // ---- gates and state update: every thread that owns a batch row ----------------------------
+    const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
+    tc_fence_after_sync();
+    uint32_t r[NG];
+    tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
+    tmem_ld_wait();
+    if (got && owner) {
+      uint32_t hq[4], gi[4], gf[4], gg[4], go[4];
+      float cin[NU];
+#pragma unroll
+      for (int u = 0; u < NU; u += 2) {
+        float hv[2], iv[2], fv[2], gv[2], ov[2];
+#pragma unroll
+        for (int d = 0; d < 2; ++d) {
+          const int q = 4 * (u + d);
+          iv[d] = sigmoid_fast(__uint_as_float(r[q + 0]) + zx[q + 0]);
+          fv[d] = sigmoid_fast(__uint_as_float(r[q + 1]) + zx[q + 1]);
+          gv[d] = tanh_fast(__uint_as_float(r[q + 2]) + zx[q + 2]);
+          ov[d] = sigmoid_fast(__uint_as_float(r[q + 3]) + zx[q + 3]);
+          cin[u + d] = c[u + d];
+          c[u + d] = fmaf(fv[d], c[u + d], iv[d] * gv[d]);
+          hv[d] = ov[d] * tanh_fast(c[u + d]);
+        }
+        hq[u / 2] = pack_bf16x2(hv[0], hv[1]);
+        gi[u / 2] = pack_bf16x2(iv[0], iv[1]);
+        gf[u / 2] = pack_bf16x2(fv[0], fv[1]);
+        gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
+        go[u / 2] = pack_bf16x2(ov[0], ov[1]);
+      }
+      char* ws = a.ws;
+      const uint4 hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.h_dst * 16) + e0) = hnew;
+      float* cd = reinterpret_cast<float*>(ws + (size_t)op.c_dst * 16) + e0;
+      *reinterpret_cast<float4*>(cd) = make_float4(c[0], c[1], c[2], c[3]);
+      *reinterpret_cast<float4*>(cd + 4) = make_float4(c[4], c[5], c[6], c[7]);
+      if (op.gates) {
+        __nv_bfloat16* g = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+        const size_t pl = (size_t)a.plane16 * 8;   // elements
+        *reinterpret_cast<uint4*>(g) = make_uint4(gi[0], gi[1], gi[2], gi[3]);
+        *reinterpret_cast<uint4*>(g + pl) = make_uint4(gf[0], gf[1], gf[2], gf[3]);
+        *reinterpret_cast<uint4*>(g + 2 * pl) = make_uint4(gg[0], gg[1], gg[2], gg[3]);
+        *reinterpret_cast<uint4*>(g + 3 * pl) = make_uint4(go[0], go[1], go[2], go[3]);
+      }
+      if (op.in_copy) {
+        char* blk = ws + (size_t)op.in_copy * 16;
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = hprev;
+        float* ci = reinterpret_cast<float*>(blk + (size_t)a.hsz16 * 16) + e0;
+        *reinterpret_cast<float4*>(ci) = make_float4(cin[0], cin[1], cin[2], cin[3]);
+        *reinterpret_cast<float4*>(ci + 4) = make_float4(cin[4], cin[5], cin[6], cin[7]);
+      }
+      hprev = hnew;
+      // the input projection of the next step does not depend on the recurrence: fetch it now
+      if (i + 1 < a.n) {
+        const float4* zp = reinterpret_cast<const float4*>(a.zx + ((size_t)(i + 1) * a.B + b) * 4 * a.H + (size_t)cta * NG);
+#pragma unroll
+        for (int v = 0; v < NG / 4; ++v) {
+          const float4 z = zp[v];
+          zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
+        }
+      }
+    }
+    fence_proxy_async();       // h_k will be read through TMA by every CTA
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      red_release_add(a.sync, 1u);
+    }
+    if (failed) break;         // uniform: written before the barrier or not at all
+  }
+
+  if (failed) {
+    if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
+    // loads that were requested may still be landing: give each ring slot a bounded chance
+    if (is_p)
+      for (uint32_t q = (issued > NST ? issued - NST : 0); q < issued; ++q)
+        (void)mbar_wait(&full[q % NST], (q / NST) & 1);
+    if (is_p) (void)mbar_wait(&wfull, 0);
+  } else if (cta == 0 && tid == 0) {
+    a.counters[0] += a.n;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 32);
+}
+
+// ------------------------------------------------------------------------------------------
+// backward run
+// ------------------------------------------------------------------------------------------
+struct BwdRunArgs {
+  const DevOp* ops;        // consecutive backward operations, k descending, all in one chunk
+  int n;
+  char* ws;
+  const float* dha;        // [S][B][H]: gradient entering h_k from the readout, row block (k-1) % S
+  __nv_bfloat16* dz;       // [S][B][4H] staging, row block (k-1) % S, gate columns permuted
+  float* dh;               // [B][H] carried dL/dh (in: from step k_hi + 1; out: for step k_lo - 1)
+  float* dc;               // [B][H] carried dL/dc
+  const float* loss_part;  // [S][LOSS_PARTS]
+  float* loss_t;           // [t]
+  uint32_t* sync;
+  int* status;
+  int64_t* counters;
+  int B, H, S;
+  uint32_t plane16, hsz16;
+};
+
+template <int BM>
+__global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__ CUtensorMap tm_dz,
+                                                         const __grid_constant__ CUtensorMap tm_wt,
+                                                         const BwdRunArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t wfull, full[NST], empty[NST], acc;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int KB = (4 * a.H + 63) / 64;
+  uint8_t* sW = sm;                    // KB tiles of [8 rows][128 B]: rows 8c .. 8c+7 of W_hh^T
+  uint8_t* ring = sm + KB * 1024;
+  constexpr uint32_t A_TILE = BM * 128;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, ncta = gridDim.x;
+  const bool is_p = (tid == 0), is_mma = (tid == 32);
+
+  if (tid == 0) {
+    mbar_init(&wfull, 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(&acc, 1);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_dz);
+    tma_prefetch_desc(&tm_wt);
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 32);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  if (is_p) {
+    mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 1024u);
+    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 1024, &tm_wt, kb * 64, cta * NU, &wfull);
+  }
+
+  const int b = (BM == 64) ? (16 * warp + lane) : (32 * warp + lane);
+  const bool owner = ((BM == 64) ? (lane < 16) : true) && b < a.B;
+  const int j0 = cta * NU;
+  const size_t e0 = (size_t)b * a.H + j0;
+  const size_t pl = (size_t)a.plane16 * 8;
+  float dh[NU], dc[NU];
+  if (owner) {
+    const float4 a0 = *reinterpret_cast<const float4*>(a.dh + e0), a1 = *reinterpret_cast<const float4*>(a.dh + e0 + 4);
+    const float4 c0 = *reinterpret_cast<const float4*>(a.dc + e0), c1 = *reinterpret_cast<const float4*>(a.dc + e0 + 4);
+    dh[0] = a0.x; dh[1] = a0.y; dh[2] = a0.z; dh[3] = a0.w; dh[4] = a1.x; dh[5] = a1.y; dh[6] = a1.z; dh[7] = a1.w;
+    dc[0] = c0.x; dc[1] = c0.y; dc[2] = c0.z; dc[3] = c0.w; dc[4] = c1.x; dc[5] = c1.y; dc[6] = c1.z; dc[7] = c1.w;
+  } else {
+#pragma unroll
+    for (int u = 0; u < NU; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
+  }
+
+  uint32_t issued = 0, consumed = 0;
+  constexpr uint32_t idesc = make_idesc(1, BM, NU, false, false);
+  const int G = 4 * a.H;
+
+  for (int i = 0; i < a.n; ++i) {
+    const DevOp op = a.ops[i];
+    const int sidx = (op.k - 1) % a.S;
+    if (i > 0) {
+      // dh for this step = the slice of dz_{k+1} W_hh this CTA computed in the previous iteration
+      const bool got = wait_or_fail(&acc, (uint32_t)(i - 1) & 1, &failed);
+      tc_fence_after_sync();
+      uint32_t r[NU];
+      tmem_ld_32x8(tmem + ((uint32_t)(32 * warp) << 16), r);
+      tmem_ld_wait();
+      if (got) {
+#pragma unroll
+        for (int u = 0; u < NU; ++u) dh[u] = __uint_as_float(r[u]);
+      }
+    }
+    if (owner && !failed) {
+      const char* ws = a.ws;
+      const float* dha = a.dha + ((size_t)sidx * a.B) * a.H + e0;
+      const float4 d0 = *reinterpret_cast<const float4*>(dha), d1 = *reinterpret_cast<const float4*>(dha + 4);
+      const float dhav[NU] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+      const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+      const uint4 qi = *reinterpret_cast<const uint4*>(g), qf = *reinterpret_cast<const uint4*>(g + pl);
+      const uint4 qg = *reinterpret_cast<const uint4*>(g + 2 * pl), qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
+      const uint32_t wi[4] = {qi.x, qi.y, qi.z, qi.w}, wf[4] = {qf.x, qf.y, qf.z, qf.w};
+      const uint32_t wg[4] = {qg.x, qg.y, qg.z, qg.w}, wo[4] = {qo.x, qo.y, qo.z, qo.w};
+      const float* ctp = reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0;
+      const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
+      const float4 t0 = *reinterpret_cast<const float4*>(ctp), t1 = *reinterpret_cast<const float4*>(ctp + 4);
+      const float4 p0 = *reinterpret_cast<const float4*>(cpp), p1 = *reinterpret_cast<const float4*>(cpp + 4);
+      const float ct[NU] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+      const float cp[NU] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+      uint32_t out[NG / 2];
+#pragma unroll
+      for (int u = 0; u < NU; ++u) {
+        const int w = u >> 1;
+        const bool hi = (u & 1) != 0;
+        const float gi = hi ? bf16_hi(wi[w]) : bf16_lo(wi[w]);
+        const float gf = hi ? bf16_hi(wf[w]) : bf16_lo(wf[w]);
+        const float gg = hi ? bf16_hi(wg[w]) : bf16_lo(wg[w]);
+        const float go = hi ? bf16_hi(wo[w]) : bf16_lo(wo[w]);
+        const float dht = dhav[u] + dh[u];
+        const float th = tanh_fast(ct[u]);
+        const float d_o = dht * th;
+        const float dct = fmaf(dht * go, 1.f - th * th, dc[u]);
+        const float zi = dct * gg * gi * (1.f - gi);
+        const float zf = dct * cp[u] * gf * (1.f - gf);
+        const float zg = dct * gi * (1.f - gg * gg);
+        const float zo = d_o * go * (1.f - go);
+        dc[u] = dct * gf;
+        out[2 * u] = pack_bf16x2(zi, zf);
+        out[2 * u + 1] = pack_bf16x2(zg, zo);
+      }
+      uint4* dzp = reinterpret_cast<uint4*>(a.dz + ((size_t)sidx * a.B + b) * G + (size_t)cta * NG);
+#pragma unroll
+      for (int v = 0; v < NG / 8; ++v) dzp[v] = make_uint4(out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
+    }
+    if (cta == 0 && tid == 0) {
+      // loss term of this step: its partial sums in a fixed order
+      float s = 0.f;
+      for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
+      a.loss_t[op.k - 1] = s;
+    }
+    fence_proxy_async();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      red_release_add(a.sync, 1u);
+    }
+    if (failed) break;
+
+    if (is_p) {
+      // ---- producer: all of dz_k through the ring -----------------------------------------
+      bool ok = wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed);
+      if (ok) {
+        fence_proxy_async();
+        const int32_t row = sidx * a.B;
+        for (int kb = 0; kb < KB && ok; ++kb, ++issued) {
+          const uint32_t s = issued % NST, it = issued / NST;
+          if (it > 0) ok = wait_or_fail(&empty[s], (it - 1) & 1, &failed);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full[s], A_TILE);
+          tma_load_2d(ring + s * A_TILE, &tm_dz, kb * 64, row, &full[s]);
+        }
+      }
+    } else if (is_mma) {
+      bool ok = true;
+      if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
+      for (int kb = 0; kb < KB && ok; ++kb, ++consumed) {
+        const uint32_t s = consumed % NST, it = consumed / NST;
+        ok = wait_or_fail(&full[s], it & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a0 = smem_u32(ring + s * A_TILE), b0 = smem_u32(sW + kb * 1024);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          mma_f16(tmem, make_desc_sw128(a0 + k4 * 32, 16, 1024), make_desc_sw128(b0 + k4 * 32, 16, 1024), idesc,
+                  (kb > 0 || k4 > 0) ? 1u : 0u);
+        mma_commit(&empty[s]);
+      }
+      mma_commit(&acc);
+    }
+    __syncwarp();
+  }
+
+  if (!failed) {
+    // the gradient that leaves the run: dh from the last product, dc from registers
+    const bool got = wait_or_fail(&acc, (uint32_t)(a.n - 1) & 1, &failed);
+    tc_fence_after_sync();
+    uint32_t r[NU];
+    tmem_ld_32x8(tmem + ((uint32_t)(32 * warp) << 16), r);
+    tmem_ld_wait();
+    if (got && owner) {
+      *reinterpret_cast<float4*>(a.dh + e0) = make_float4(__uint_as_float(r[0]), __uint_as_float(r[1]),
+                                                           __uint_as_float(r[2]), __uint_as_float(r[3]));
+      *reinterpret_cast<float4*>(a.dh + e0 + 4) = make_float4(__uint_as_float(r[4]), __uint_as_float(r[5]),
+                                                               __uint_as_float(r[6]), __uint_as_float(r[7]));
+      *reinterpret_cast<float4*>(a.dc + e0) = make_float4(dc[0], dc[1], dc[2], dc[3]);
+      *reinterpret_cast<float4*>(a.dc + e0 + 4) = make_float4(dc[4], dc[5], dc[6], dc[7]);
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (failed) {
+    if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
+    if (is_p) {
+      for (uint32_t q = (issued > NST ? issued - NST : 0); q < issued; ++q)
+        (void)mbar_wait(&full[q % NST], (q / NST) & 1);
+      (void)mbar_wait(&wfull, 0);
+    }
+    __syncthreads();
+  } else if (cta == 0 && tid == 0) {
+    a.counters[1] += a.n;
+  }
+  if (warp == 1) tmem_dealloc(tmem, 32);
+}
+
+// ------------------------------------------------------------------------------------------
+// small kernels off the recurrence
+// ------------------------------------------------------------------------------------------
+// Packs the weights once per training step: gate rows permuted to 4 u + q (the four gates of
+// hidden unit u adjacent), W_ih and W_hh split, their transposes for the backward products, the
+// transposed readout matrix, and the permuted bias.
+__global__ void pack_weights(const __nv_bfloat16* W, const float* bias, const __nv_bfloat16* W_out, int I, int H,
+                             int O, __nv_bfloat16* wp_ih, __nv_bfloat16* wp_hh, __nv_bfloat16* wpT_hh,
+                             __nv_bfloat16* wpT_ih, float* bias_p, __nv_bfloat16* woutT) {
+  const int G = 4 * H, K = I + H;
+  const size_t nW = (size_t)G * K;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < nW; e += stride) {
+    const int g = (int)(e / K), col = (int)(e % K);
+    const int q = g / H, u = g % H, gp = 4 * u + q;
+    const __nv_bfloat16 v = W[e];
+    if (col < I) {
+      wp_ih[(size_t)gp * I + col] = v;
+      if (wpT_ih) wpT_ih[(size_t)col * G + gp] = v;
+    } else {
+      wp_hh[(size_t)gp * H + (col - I)] = v;
+      wpT_hh[(size_t)(col - I) * G + gp] = v;
+    }
+  }
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < (size_t)G; e += stride) {
+    const int q = (int)e / H, u = (int)e % H;
+    bias_p[4 * u + q] = bias[e];
+  }
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < (size_t)O * H; e += stride) {
+    const int o = (int)(e / H), j = (int)(e % H);
+    woutT[(size_t)j * O + o] = W_out[e];
+  }
+}
+
+// Copies h_k and h_{k-1} of each step of a backward run from wherever the internal state lies
+// into the staging chunk (row block (k-1) % S), 16 bytes per thread per access.
+__global__ void gather_states(const DevOp* ops, int n, const char* ws, uint4* hk, uint4* hprev, int S,
+                              size_t block16) {  // block16: B*H*2/16
+  const DevOp op = ops[blockIdx.y];
+  const int sidx = (op.k - 1) % S;
+  const uint4* src_k = reinterpret_cast<const uint4*>(ws + (size_t)op.h_dst * 16);
+  const uint4* src_p = reinterpret_cast<const uint4*>(ws + (size_t)op.h_src * 16);
+  uint4* dk = hk + (size_t)sidx * block16;
+  uint4* dp = hprev + (size_t)sidx * block16;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < block16; e += (size_t)gridDim.x * blockDim.x) {
+    dk[e] = src_k[e];
+    dp[e] = src_p[e];
+  }
+}
+
+// y (float32, readout with bias) -> dy = 2 (y - target) / (B O) in bfloat16, and LOSS_PARTS
+// partial sums of the squared error per step (each a fixed-order sum over a fixed slice).
+__global__ void loss_dy(const DevOp* ops, const float* y, const float* targets, __nv_bfloat16* dy, float* loss_part,
+                        int S, int B, int O) {
+  __shared__ float red[256];
+  const DevOp op = ops[blockIdx.y];
+  const int sidx = (op.k - 1) % S;
+  const size_t n = (size_t)B * O;
+  const size_t per = (n + LOSS_PARTS - 1) / LOSS_PARTS;
+  const size_t lo = blockIdx.x * per, hi = (lo + per < n) ? lo + per : n;
+  const float* yp = y + (size_t)sidx * n;
+  const float* tp = targets + (size_t)(op.k - 1) * n;
+  __nv_bfloat16* dp = dy + (size_t)sidx * n;
+  const float inv = 1.f / ((float)B * (float)O);
+  float s = 0.f;
+  for (size_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
+    const float d = yp[e] - tp[e];
+    dp[e] = __float2bfloat16_rn(2.f * d * inv);
+    s = fmaf(d, d, s);
+  }
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) loss_part[sidx * LOSS_PARTS + blockIdx.x] = red[0] * inv;
+}
+
+// out[map(n)] += sum_r v[r][n], rows ascending; perm_h > 0 maps column 4 u + q to q perm_h + u.
+__global__ void colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out, int perm_h) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float s = 0.f;
+  for (int r = 0; r < rows; ++r) s += __bfloat162float(v[(size_t)r * N + n]);
+  const int o = perm_h ? ((n & 3) * perm_h + (n >> 2)) : n;
+  out[o] += s;
+}
+
+__global__ void finalize_tc(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
+                            const int* status) {
+  float s = 0.f;
+  for (int64_t i = threadIdx.x; i < t; i += 32) s += loss_t[i];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+  if (threadIdx.x == 0) {
+    *loss = s;
+    counters[2] = peak_units;
+    counters[3] = *status;
+  }
+}
+
+__global__ void copy16_tc(uint4* dst, const uint4* src, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+inline uint32_t off16(size_t byte_off) { return (uint32_t)(byte_off >> 4); }
+
+// With MEBPTT_DEBUG set in the environment, failed CUDA calls are named on stderr.
+inline bool cuda_ok(cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return true;
+  static const bool verbose = getenv("MEBPTT_DEBUG") != nullptr;
+  if (verbose) fprintf(stderr, "mebptt: %s failed: %s\n", what, cudaGetErrorString(e));
+  return false;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host: one training step
+// ------------------------------------------------------------------------------------------
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry) {
+  const int B = y.B, H = y.H, I = y.I, O = y.O, S = y.S, G = 4 * H, K = I + H;
+  const int BM = 64;  // batch rows per MMA tile (B <= 64)
+  const int ncta = H / NU;
+  int64_t launches = 0;
+  char* ws = io.ws;
+  auto at = [&](size_t off) { return ws + off; };
+
+  // ---- tape -> device operations -------------------------------------------------------------
+  auto block_off = [&](int32_t loc) -> size_t {
+    switch (loc) {
+      case MEBPTT_LOC_INIT: return y.off_init;
+      case MEBPTT_LOC_PING: return y.off_ping;
+      case MEBPTT_LOC_PONG: return y.off_pong;
+      case MEBPTT_LOC_CORE: return y.off_core;
+      default: return y.off_arena + (size_t)loc * y.unit;
+    }
+  };
+  const size_t nops = p->tape.size();
+  std::vector<DevOp> dev;
+  if (!dry) {
+    dev.resize(nops);
+    for (size_t i = 0; i < nops; ++i) {
+      const mebptt_op& op = p->tape[i];
+      DevOp d{};
+      d.k = op.k;
+      d.fmt = op.dst_fmt;
+      if (op.kind == MEBPTT_OP_FWD) {
+        const size_t src = block_off(op.src), dst = block_off(op.dst);
+        d.h_src = off16(src); d.c_src = off16(src + y.hsz);
+        d.h_dst = off16(dst); d.c_dst = off16(dst + y.hsz);
+        d.gates = (op.dst_fmt != MEBPTT_FMT_HIDDEN) ? off16(dst + y.rec_gates) : 0;
+        d.in_copy = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? off16(dst + y.rec_in) : 0;
+      } else {
+        const size_t rec = block_off(op.src);
+        const size_t prev = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? rec + y.rec_in : block_off(op.aux);
+        d.h_dst = off16(rec); d.c_dst = off16(rec + y.hsz);
+        d.h_src = off16(prev); d.c_src = off16(prev + y.hsz);
+        d.gates = off16(rec + y.rec_gates);
+      }
+      dev[i] = d;
+    }
+  }
+  const DevOp* dops = reinterpret_cast<const DevOp*>(at(y.off_tape));
+  uint32_t* sync = reinterpret_cast<uint32_t*>(at(y.off_sync));
+  int* status = reinterpret_cast<int*>(at(y.off_status));
+  float* loss_t = reinterpret_cast<float*>(at(y.off_loss_t));
+  float* dh = reinterpret_cast<float*>(at(y.off_dh));
+  float* dc = reinterpret_cast<float*>(at(y.off_dc));
+  float* zx = reinterpret_cast<float*>(at(y.off_zx));
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(at(y.off_dz));
+  __nv_bfloat16* hprev = reinterpret_cast<__nv_bfloat16*>(at(y.off_hprev));
+  __nv_bfloat16* hk = reinterpret_cast<__nv_bfloat16*>(at(y.off_hk));
+  float* yv = reinterpret_cast<float*>(at(y.off_y));
+  __nv_bfloat16* dyv = reinterpret_cast<__nv_bfloat16*>(at(y.off_dy));
+  float* dha = reinterpret_cast<float*>(at(y.off_dha));
+  float* loss_part = reinterpret_cast<float*>(at(y.off_loss_part));
+  __nv_bfloat16* wp_ih = reinterpret_cast<__nv_bfloat16*>(at(y.off_wp_ih));
+  __nv_bfloat16* wp_hh = reinterpret_cast<__nv_bfloat16*>(at(y.off_wp_hh));
+  __nv_bfloat16* wpT_hh = reinterpret_cast<__nv_bfloat16*>(at(y.off_wpT_hh));
+  __nv_bfloat16* wpT_ih = want_dx ? reinterpret_cast<__nv_bfloat16*>(at(y.off_wpT_ih)) : nullptr;
+  float* bias_p = reinterpret_cast<float*>(at(y.off_bias_p));
+  __nv_bfloat16* woutT = reinterpret_cast<__nv_bfloat16*>(at(y.off_woutT));
+
+  const int fwd_smem = ((H + 63) / 64) * 4096 + NST * BM * 128 + 1024;
+  const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
+  CUtensorMap tm_h, tm_w, tm_dz, tm_wt;
+  if (!dry) {
+    static const bool attrs = [] {
+      const int big = 220 * 1024;  // the kernels also hold a few static barriers
+      cudaFuncSetAttribute(fwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+      cudaFuncSetAttribute(bwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+      return true;
+    }();
+    (void)attrs;
+    // the whole workspace as rows of H bfloat16: any h block starts at a whole row
+    const uint64_t rows = y.total / ((size_t)H * 2);
+    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, (uint32_t)BM);
+    ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, NG);
+    ok = ok && make_tmap_2d(&tm_dz, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, (uint32_t)BM);
+    ok = ok && make_tmap_2d(&tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
+    if (!ok) return MEBPTT_ERR_UNSUPPORTED;
+
+    cudaMemsetAsync(dh, 0, (size_t)B * H * 4, s);
+    cudaMemsetAsync(dc, 0, (size_t)B * H * 4, s);
+    cudaMemsetAsync(io.dW, 0, (size_t)G * K * 4, s);
+    cudaMemsetAsync(io.db, 0, (size_t)G * 4, s);
+    cudaMemsetAsync(io.dW_out, 0, (size_t)O * H * 4, s);
+    cudaMemsetAsync(io.db_out, 0, (size_t)O * 4, s);
+    cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
+    cudaMemsetAsync(sync, 0, y.n_sync * 4, s);
+    cudaMemsetAsync(status, 0, 256, s);
+    cudaMemcpyAsync(at(y.off_tape), dev.data(), nops * sizeof(DevOp), cudaMemcpyHostToDevice, s);
+    pack_weights<<<592, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
+                                     reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh,
+                                     wpT_ih, bias_p, woutT);
+    // Peek of the initial state: the caller's (h0, c0) as a hidden block inside the workspace
+    copy16_tc<<<64, 256, 0, s>>>(reinterpret_cast<uint4*>(at(y.off_init)), reinterpret_cast<const uint4*>(io.h0),
+                                 (size_t)B * H * 2 / 16);
+    copy16_tc<<<64, 256, 0, s>>>(reinterpret_cast<uint4*>(at(y.off_init + y.hsz)),
+                                 reinterpret_cast<const uint4*>(io.c0), (size_t)B * H * 4 / 16);
+  }
+  launches += 3;
+
+  int launch_id = 0;
+  int rc = MEBPTT_OK;
+  if (!dry && !cuda_ok(cudaGetLastError(), "set-up (memsets, tape upload, weight packing)")) rc = MEBPTT_ERR_CUDA;
+  auto gemm = [&](const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn, GemmOut out, int M,
+                  int N, int Kc) {
+    ++launches;
+    if (dry || rc != MEBPTT_OK) return;
+    rc = gemm_bf16(A, lda, amn, Bm, ldb, bmn, out, M, N, Kc, status, s);
+    if (rc != MEBPTT_OK) cuda_ok(cudaErrorUnknown, "batched contraction");
+  };
+
+  size_t i = 0;
+  while (i < nops && rc == MEBPTT_OK) {
+    const mebptt_op& first = p->tape[i];
+    if (first.kind == MEBPTT_OP_FWD) {
+      // a forward run: consecutive operations k, k+1, ... each starting from the state the
+      // previous one wrote; at most S of them per launch
+      size_t j = i + 1;
+      while (j < nops && j - i < (size_t)S && p->tape[j].kind == MEBPTT_OP_FWD &&
+             p->tape[j].k == p->tape[j - 1].k + 1 && p->tape[j].src == p->tape[j - 1].dst)
+        ++j;
+      const int n = (int)(j - i);
+      const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(first.k - 1) * B * I;
+      gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, n * B, G, I);
+      ++launches;
+      if (!dry && rc == MEBPTT_OK) {
+        FwdRunArgs a{dops + i, n, ws, zx, sync + launch_id, status, io.counters, B, H, off16(y.plane), off16(y.hsz)};
+        void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
+        const void* fn = (const void*)fwd_run_kernel<64>;
+        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, fwd_smem, s), "forward run launch"))
+          rc = MEBPTT_ERR_CUDA;
+      }
+      ++launch_id;
+      i = j;
+    } else {
+      // a backward run: consecutive operations k, k-1, ... inside one chunk of S time steps
+      const int chunk = (first.k - 1) / S;
+      size_t j = i + 1;
+      while (j < nops && p->tape[j].kind == MEBPTT_OP_BWD && (p->tape[j].k - 1) / S == chunk) ++j;
+      const int n = (int)(j - i);
+      const int k_hi = first.k, k_lo = k_hi - n + 1;
+      const int s_lo = (k_lo - 1) % S;
+      launches += 3;
+      if (!dry && rc == MEBPTT_OK) {
+        const size_t block16 = (size_t)B * H * 2 / 16;
+        gather_states<<<dim3(16, n), 256, 0, s>>>(dops + i, n, ws, reinterpret_cast<uint4*>(hk),
+                                                  reinterpret_cast<uint4*>(hprev), S, block16);
+      }
+      // readout of the n steps at once, then loss terms and dy, then the gradient entering h_k
+      gemm(hk + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
+           GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
+      if (!dry && rc == MEBPTT_OK)
+        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(dops + i, yv, io.targets, dyv, loss_part, S, B, O);
+      gemm(dyv + (size_t)s_lo * B * O, O, false, woutT, O, false,
+           GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
+      if (!dry && rc == MEBPTT_OK) {
+        BwdRunArgs a{dops + i, n, ws, dha, dz, dh, dc, loss_part, loss_t, sync + launch_id, status, io.counters,
+                     B, H, S, off16(y.plane), off16(y.hsz)};
+        void* args[] = {(void*)&tm_dz, (void*)&tm_wt, (void*)&a};
+        const void* fn = (const void*)bwd_run_kernel<64>;
+        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, bwd_smem, s), "backward run launch"))
+          rc = MEBPTT_ERR_CUDA;
+      }
+      ++launch_id;
+      if (k_lo == chunk * S + 1) {
+        // the chunk is complete: its weight gradients, summed over (s, b) in ascending order
+        const int steps = (int)((int64_t)(chunk + 1) * S <= y.t ? S : y.t - (int64_t)chunk * S);
+        const int R = steps * B;
+        const __nv_bfloat16* xc = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)chunk * S * B * I;
+        gemm(dz, G, true, xc, I, true, GemmOut{GemmOut::ACCUM_F32, io.dW, K, nullptr, H}, G, I, R);
+        gemm(dz, G, true, hprev, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW + I, K, nullptr, H}, G, H, R);
+        gemm(dyv, O, true, hk, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
+        launches += 2;
+        if (!dry && rc == MEBPTT_OK) {
+          colsum_bf16<<<(G + 127) / 128, 128, 0, s>>>(dz, R, G, io.db, H);
+          colsum_bf16<<<(O + 127) / 128, 128, 0, s>>>(dyv, R, O, io.db_out, 0);
+        }
+        if (want_dx)
+          gemm(dz, G, false, wpT_ih, G, false,
+               GemmOut{GemmOut::STORE_F32, io.dx + (size_t)chunk * S * B * I, I, nullptr, 0}, R, I, G);
+      }
+      i = j;
+    }
+  }
+  ++launches;
+  if (!dry && rc == MEBPTT_OK) {
+    finalize_tc<<<1, 32, 0, s>>>(loss_t, y.t, io.loss, io.counters, p->peak_units, status);
+    if (!cuda_ok(cudaGetLastError(), "training step (last error)")) rc = MEBPTT_ERR_CUDA;
+  }
+  if (dry) return launches;
+  return rc;
+}
+
+}  // namespace tc
+}  // namespace mebptt

@@ -26,14 +26,15 @@ def _upload(arr: np.ndarray, device) -> torch.Tensor:
 class DeviceProblem:
     """One synthetic problem resident on a GPU, with output buffers and a workspace."""
 
-    def __init__(self, cfg: synth.LstmConfig, prob: dict | None = None, device="cuda:0", want_dx=False):
+    def __init__(self, cfg: synth.LstmConfig, prob: dict | None = None, device="cuda:0", want_dx=False,
+                 flags=0):
         self.cfg = cfg
         self.device = torch.device(device)
         self.prob = prob if prob is not None else synth.make_problem(cfg)
         self.host = synth.to_device_arrays(cfg, self.prob)
         self.want_dx = bool(want_dx)
         self.desc = B.make_desc(cfg.layers, cfg.input, cfg.hidden, cfg.readout, cfg.batch, cfg.t,
-                                cfg.dtype, want_dx=int(self.want_dx))
+                                cfg.dtype, want_dx=int(self.want_dx), flags=flags)
         self.dev = {k: _upload(v, self.device) for k, v in self.host.items()}
         f32 = dict(dtype=torch.float32, device=self.device)
         nW = self.host["W"].size

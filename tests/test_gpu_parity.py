@@ -157,3 +157,28 @@ def test_slot_copy(H):
     B.mebptt_slot_copy(dst, src, src.numel(), torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert torch.equal(src, dst)
+
+
+@pytest.mark.parametrize("shape", [dict(input=64, hidden=64, batch=64, t=40, readout=64),
+                                   dict(input=72, hidden=200, batch=24, t=37, readout=40),
+                                   dict(input=256, hidden=256, batch=64, t=50, readout=256)])
+def test_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
+    """bf16 shapes the tcgen05 kernels cover: oracle parity, bit identity across plans, and
+    agreement with the CUDA-core kernels (same roundings of stored values, other sum order)."""
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg("c2", **shape)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][3] == 0
+    assert_close_to_oracle(full, ref, "bf16", want_dx=True)
+    for mode, m, beta in [("hsm", 1, 0), ("hsm", 5, 0), ("ism", 1, 0), ("ism", 6, 0), ("msm", 9, 0), ("msm", 13, 3)]:
+        plan = dp.plan(mode, m, beta=beta)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+        assert_bit_identical(res, full, want_dx=True)
+    slow = H.DeviceProblem(cfg, dp.prob, want_dx=True, flags=B.MEBPTT_FLAG_NO_TENSOR_CORES)
+    other = slow.run(slow.full_memory_plan())
+    from tests.util import rel_l2
+    for k in ("dW", "db", "dW_out", "db_out", "dx"):
+        assert rel_l2(full[k], other[k]) < 1e-2, k
