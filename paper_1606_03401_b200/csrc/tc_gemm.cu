@@ -127,21 +127,28 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
             if (col0 + j < N) p[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
         } else {
           float* p = reinterpret_cast<float*>(out.ptr) + (size_t)row_o * out.ld + col0;
-          const bool vec = (col0 + 32 <= N) && ((reinterpret_cast<uintptr_t>(p) & 15) == 0);
+          const bool vec = (col0 + 32 <= N) && ((reinterpret_cast<uintptr_t>(p) & 15) == 0) &&
+                           ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0);
           if (vec) {
+            // all eight loads of the old values first, so that their latencies overlap
+            float4 o[8];
+            if (out.kind == GemmOut::ACCUM_F32) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                     __uint_as_float(r[j + 3]));
+              for (int j = 0; j < 8; ++j) o[j] = *reinterpret_cast<const float4*>(p + 4 * j);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
               if (out.bias) {
-                v.x += out.bias[col0 + j]; v.y += out.bias[col0 + j + 1];
-                v.z += out.bias[col0 + j + 2]; v.w += out.bias[col0 + j + 3];
+                const float4 bv = *reinterpret_cast<const float4*>(out.bias + col0 + 4 * j);
+                v.x += bv.x; v.y += bv.y; v.z += bv.z; v.w += bv.w;
               }
-              if (out.kind == GemmOut::ACCUM_F32) {
-                const float4 o = *reinterpret_cast<const float4*>(p + j);
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              *reinterpret_cast<float4*>(p + j) = v;
+              v.x += o[j].x; v.y += o[j].y; v.z += o[j].z; v.w += o[j].w;
+              *reinterpret_cast<float4*>(p + 4 * j) = v;
             }
           } else {
 #pragma unroll

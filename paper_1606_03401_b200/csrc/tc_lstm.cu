@@ -110,6 +110,7 @@ struct FwdRunArgs {
   int B, H;
   uint32_t plane16;      // distance between gate planes, in 16-byte units
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
+  uint32_t nst;          // ring stages (<= 16); H / 64 when all of h fits next to the weights
 };
 
 template <int BM>
@@ -117,7 +118,7 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
                                                          const __grid_constant__ CUtensorMap tm_w,
                                                          const FwdRunArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[NST], empty[NST], acc;
+  __shared__ uint64_t wfull, full[16], empty[16], acc;
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
 
@@ -130,10 +131,11 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
   const bool is_p = (tid == 0), is_mma = (tid == 32);
+  const uint32_t NSTr = a.nst;
 
   if (tid == 0) {
     mbar_init(&wfull, 1);
-    for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < 16; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(&acc, 1);
     failed = 0;
     mbar_fence_init();
@@ -196,7 +198,7 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
         fence_proxy_async();
         const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
         for (int kb = 0; kb < KB && ok; ++kb, ++issued) {
-          const uint32_t s = issued % NST, it = issued / NST;
+          const uint32_t s = issued % NSTr, it = issued / NSTr;
           if (it > 0) ok = wait_or_fail(&empty[s], (it - 1) & 1, &failed);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[s], A_TILE);
@@ -208,7 +210,7 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
       bool ok = true;
       if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
       for (int kb = 0; kb < KB && ok; ++kb, ++consumed) {
-        const uint32_t s = consumed % NST, it = consumed / NST;
+        const uint32_t s = consumed % NSTr, it = consumed / NSTr;
         ok = wait_or_fail(&full[s], it & 1, &failed);
         if (!ok) break;
         tc_fence_after_sync();
@@ -229,6 +231,9 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
     uint32_t r[NG];
     tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
     tmem_ld_wait();
+    uint4 hnew = make_uint4(0, 0, 0, 0);
+    uint32_t qi[4], qf[4], qg[4], qo[4];
+    float cold[NU];
     if (got && owner) {
       uint32_t hq[4], gi[4], gf[4], gg[4], go[4];
       float cin[NU];
@@ -252,26 +257,38 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
         gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
         go[u / 2] = pack_bf16x2(ov[0], ov[1]);
       }
+      // h_k first: it is what the other CTAs wait for
+      hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = hnew;
+#pragma unroll
+      for (int v = 0; v < 4; ++v) { qi[v] = gi[v]; qf[v] = gf[v]; qg[v] = gg[v]; qo[v] = go[v]; }
+#pragma unroll
+      for (int u = 0; u < NU; ++u) cold[u] = cin[u];
+    }
+    fence_proxy_async();       // h_k will be read through TMA by every CTA
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) red_release_add(a.sync, 1u);
+    if (got && owner) {
+      // the rest of the state is not on the critical path of the recurrence
       char* ws = a.ws;
-      const uint4 hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
-      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.h_dst * 16) + e0) = hnew;
       float* cd = reinterpret_cast<float*>(ws + (size_t)op.c_dst * 16) + e0;
       *reinterpret_cast<float4*>(cd) = make_float4(c[0], c[1], c[2], c[3]);
       *reinterpret_cast<float4*>(cd + 4) = make_float4(c[4], c[5], c[6], c[7]);
       if (op.gates) {
         __nv_bfloat16* g = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
         const size_t pl = (size_t)a.plane16 * 8;   // elements
-        *reinterpret_cast<uint4*>(g) = make_uint4(gi[0], gi[1], gi[2], gi[3]);
-        *reinterpret_cast<uint4*>(g + pl) = make_uint4(gf[0], gf[1], gf[2], gf[3]);
-        *reinterpret_cast<uint4*>(g + 2 * pl) = make_uint4(gg[0], gg[1], gg[2], gg[3]);
-        *reinterpret_cast<uint4*>(g + 3 * pl) = make_uint4(go[0], go[1], go[2], go[3]);
+        *reinterpret_cast<uint4*>(g) = make_uint4(qi[0], qi[1], qi[2], qi[3]);
+        *reinterpret_cast<uint4*>(g + pl) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+        *reinterpret_cast<uint4*>(g + 2 * pl) = make_uint4(qg[0], qg[1], qg[2], qg[3]);
+        *reinterpret_cast<uint4*>(g + 3 * pl) = make_uint4(qo[0], qo[1], qo[2], qo[3]);
       }
       if (op.in_copy) {
         char* blk = ws + (size_t)op.in_copy * 16;
         *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = hprev;
         float* ci = reinterpret_cast<float*>(blk + (size_t)a.hsz16 * 16) + e0;
-        *reinterpret_cast<float4*>(ci) = make_float4(cin[0], cin[1], cin[2], cin[3]);
-        *reinterpret_cast<float4*>(ci + 4) = make_float4(cin[4], cin[5], cin[6], cin[7]);
+        *reinterpret_cast<float4*>(ci) = make_float4(cold[0], cold[1], cold[2], cold[3]);
+        *reinterpret_cast<float4*>(ci + 4) = make_float4(cold[4], cold[5], cold[6], cold[7]);
       }
       hprev = hnew;
       // the input projection of the next step does not depend on the recurrence: fetch it now
@@ -284,13 +301,6 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
         }
       }
     }
-    fence_proxy_async();       // h_k will be read through TMA by every CTA
-    tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
-      __threadfence();
-      red_release_add(a.sync, 1u);
-    }
     if (failed) break;         // uniform: written before the barrier or not at all
   }
 
@@ -298,8 +308,8 @@ __global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__
     if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
     // loads that were requested may still be landing: give each ring slot a bounded chance
     if (is_p)
-      for (uint32_t q = (issued > NST ? issued - NST : 0); q < issued; ++q)
-        (void)mbar_wait(&full[q % NST], (q / NST) & 1);
+      for (uint32_t q = (issued > NSTr ? issued - NSTr : 0); q < issued; ++q)
+        (void)mbar_wait(&full[q % NSTr], (q / NSTr) & 1);
     if (is_p) (void)mbar_wait(&wfull, 0);
   } else if (cta == 0 && tid == 0) {
     a.counters[0] += a.n;
@@ -328,6 +338,53 @@ struct BwdRunArgs {
   int B, H, S;
   uint32_t plane16, hsz16;
 };
+
+// Gate derivatives of one batch row and the CTA's 8 hidden units at one step: reads the stored
+// gates and cell states, the readout gradient dha and the carried (dh, dc); writes dz (bfloat16,
+// columns 4 u + q) to the staging chunk and leaves dc = dc_t * f for the next (earlier) step.
+__device__ __forceinline__ void backward_gates(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int cta,
+                                               size_t e0, size_t pl, const float (&dh)[NU], float (&dc)[NU]) {
+  const int G = 4 * a.H;
+  const char* ws = a.ws;
+  const float* dha = a.dha + ((size_t)sidx * a.B) * a.H + e0;
+  const float4 d0 = *reinterpret_cast<const float4*>(dha), d1 = *reinterpret_cast<const float4*>(dha + 4);
+  const float dhav[NU] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+  const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+  const uint4 qi = *reinterpret_cast<const uint4*>(g), qf = *reinterpret_cast<const uint4*>(g + pl);
+  const uint4 qg = *reinterpret_cast<const uint4*>(g + 2 * pl), qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
+  const uint32_t wi[4] = {qi.x, qi.y, qi.z, qi.w}, wf[4] = {qf.x, qf.y, qf.z, qf.w};
+  const uint32_t wg[4] = {qg.x, qg.y, qg.z, qg.w}, wo[4] = {qo.x, qo.y, qo.z, qo.w};
+  const float* ctp = reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0;
+  const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
+  const float4 t0 = *reinterpret_cast<const float4*>(ctp), t1 = *reinterpret_cast<const float4*>(ctp + 4);
+  const float4 p0 = *reinterpret_cast<const float4*>(cpp), p1 = *reinterpret_cast<const float4*>(cpp + 4);
+  const float ct[NU] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+  const float cp[NU] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+  uint32_t out[NG / 2];
+#pragma unroll
+  for (int u = 0; u < NU; ++u) {
+    const int w = u >> 1;
+    const bool hi = (u & 1) != 0;
+    const float gi = hi ? bf16_hi(wi[w]) : bf16_lo(wi[w]);
+    const float gf = hi ? bf16_hi(wf[w]) : bf16_lo(wf[w]);
+    const float gg = hi ? bf16_hi(wg[w]) : bf16_lo(wg[w]);
+    const float go = hi ? bf16_hi(wo[w]) : bf16_lo(wo[w]);
+    const float dht = dhav[u] + dh[u];
+    const float th = tanh_fast(ct[u]);
+    const float d_o = dht * th;
+    const float dct = fmaf(dht * go, 1.f - th * th, dc[u]);
+    const float zi = dct * gg * gi * (1.f - gi);
+    const float zf = dct * cp[u] * gf * (1.f - gf);
+    const float zg = dct * gi * (1.f - gg * gg);
+    const float zo = d_o * go * (1.f - go);
+    dc[u] = dct * gf;
+    out[2 * u] = pack_bf16x2(zi, zf);
+    out[2 * u + 1] = pack_bf16x2(zg, zo);
+  }
+  uint4* dzp = reinterpret_cast<uint4*>(a.dz + ((size_t)sidx * a.B + b) * G + (size_t)cta * NG);
+#pragma unroll
+  for (int v = 0; v < NG / 8; ++v) dzp[v] = make_uint4(out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
+}
 
 template <int BM>
 __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__ CUtensorMap tm_dz,
@@ -403,47 +460,7 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
         for (int u = 0; u < NU; ++u) dh[u] = __uint_as_float(r[u]);
       }
     }
-    if (owner && !failed) {
-      const char* ws = a.ws;
-      const float* dha = a.dha + ((size_t)sidx * a.B) * a.H + e0;
-      const float4 d0 = *reinterpret_cast<const float4*>(dha), d1 = *reinterpret_cast<const float4*>(dha + 4);
-      const float dhav[NU] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-      const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
-      const uint4 qi = *reinterpret_cast<const uint4*>(g), qf = *reinterpret_cast<const uint4*>(g + pl);
-      const uint4 qg = *reinterpret_cast<const uint4*>(g + 2 * pl), qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
-      const uint32_t wi[4] = {qi.x, qi.y, qi.z, qi.w}, wf[4] = {qf.x, qf.y, qf.z, qf.w};
-      const uint32_t wg[4] = {qg.x, qg.y, qg.z, qg.w}, wo[4] = {qo.x, qo.y, qo.z, qo.w};
-      const float* ctp = reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0;
-      const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
-      const float4 t0 = *reinterpret_cast<const float4*>(ctp), t1 = *reinterpret_cast<const float4*>(ctp + 4);
-      const float4 p0 = *reinterpret_cast<const float4*>(cpp), p1 = *reinterpret_cast<const float4*>(cpp + 4);
-      const float ct[NU] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-      const float cp[NU] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
-      uint32_t out[NG / 2];
-#pragma unroll
-      for (int u = 0; u < NU; ++u) {
-        const int w = u >> 1;
-        const bool hi = (u & 1) != 0;
-        const float gi = hi ? bf16_hi(wi[w]) : bf16_lo(wi[w]);
-        const float gf = hi ? bf16_hi(wf[w]) : bf16_lo(wf[w]);
-        const float gg = hi ? bf16_hi(wg[w]) : bf16_lo(wg[w]);
-        const float go = hi ? bf16_hi(wo[w]) : bf16_lo(wo[w]);
-        const float dht = dhav[u] + dh[u];
-        const float th = tanh_fast(ct[u]);
-        const float d_o = dht * th;
-        const float dct = fmaf(dht * go, 1.f - th * th, dc[u]);
-        const float zi = dct * gg * gi * (1.f - gi);
-        const float zf = dct * cp[u] * gf * (1.f - gf);
-        const float zg = dct * gi * (1.f - gg * gg);
-        const float zo = d_o * go * (1.f - go);
-        dc[u] = dct * gf;
-        out[2 * u] = pack_bf16x2(zi, zf);
-        out[2 * u + 1] = pack_bf16x2(zg, zo);
-      }
-      uint4* dzp = reinterpret_cast<uint4*>(a.dz + ((size_t)sidx * a.B + b) * G + (size_t)cta * NG);
-#pragma unroll
-      for (int v = 0; v < NG / 8; ++v) dzp[v] = make_uint4(out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
-    }
+    if (owner && !failed) backward_gates(a, op, sidx, b, cta, e0, pl, dh, dc);
     if (cta == 0 && tid == 0) {
       // loss term of this step: its partial sums in a fixed order
       float s = 0.f;
@@ -453,10 +470,7 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
     fence_proxy_async();
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) {
-      __threadfence();
-      red_release_add(a.sync, 1u);
-    }
+    if (tid == 0) red_release_add(a.sync, 1u);
     if (failed) break;
 
     if (is_p) {
@@ -523,6 +537,183 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
     a.counters[1] += a.n;
   }
   if (warp == 1) tmem_dealloc(tmem, 32);
+}
+
+// ------------------------------------------------------------------------------------------
+// backward run, split over thread-block clusters
+// ------------------------------------------------------------------------------------------
+// The product dh_{k-1} = dz_k W_hh has K = 4H: a CTA that wants its 8 columns on its own must
+// pull all of dz_k (B x 4H) through shared memory every step.  Here CS neighbouring CTAs (one
+// cluster, 8 CS hidden units) share the work along K instead: CTA r multiplies the K-slice
+// [r G/CS, (r+1) G/CS) of dz_k by the matching [8 CS x G/CS] block of W_hh^T, resident in its
+// shared memory, into a partial [B x 8 CS] tile; the partial tiles go to shared memory, the
+// cluster synchronises, and each owner thread adds the CS partial values of its 8 columns in the
+// order r = 0 .. CS-1, reading its peers' tiles through distributed shared memory.
+template <int CS>
+__global__ void __launch_bounds__(128, 1) bwd_run_cluster_kernel(const __grid_constant__ CUtensorMap tm_dz,
+                                                                 const __grid_constant__ CUtensorMap tm_wt,
+                                                                 const BwdRunArgs a) {
+  constexpr int BM = 64;
+  constexpr int NC = NU * CS;              // columns of dh the cluster produces
+  constexpr int PLD = NC + 4;              // row pitch of a partial tile, floats
+  constexpr uint32_t A_TILE = BM * 128;
+  constexpr uint32_t W_TILE = NC * 128;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t wfull, full[16], acc;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int G = 4 * a.H;
+  const int KBS = (G / 64) / CS;           // 64-wide K blocks in this CTA's slice (<= 16)
+  uint8_t* sW = sm;                        // KBS tiles [NC rows][128 B]
+  uint8_t* ring = sW + KBS * W_TILE;       // KBS tiles [64 rows][128 B], all of the slice at once
+  float* part = reinterpret_cast<float*>(ring + KBS * A_TILE);  // 2 x [64][PLD]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, ncta = gridDim.x;
+  const uint32_t rank = cluster_ctarank();
+  const int cl = cta / CS;
+  const bool is_p = (tid == 0), is_mma = (tid == 32);
+
+  if (tid == 0) {
+    mbar_init(&wfull, 1);
+    for (int s = 0; s < 16; ++s) mbar_init(&full[s], 1);
+    mbar_init(&acc, 1);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_dz);
+    tma_prefetch_desc(&tm_wt);
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 64);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  if (is_p) {
+    mbar_arrive_expect_tx(&wfull, (uint32_t)KBS * W_TILE);
+    for (int kb = 0; kb < KBS; ++kb)
+      tma_load_2d(sW + kb * W_TILE, &tm_wt, ((int)rank * KBS + kb) * 64, cl * NC, &wfull);
+  }
+
+  const int b = 16 * warp + lane;
+  const bool row_thread = lane < 16;             // holds an accumulator row in TMEM
+  const bool owner = row_thread && b < a.B;
+  const int j0 = cta * NU;
+  const size_t e0 = (size_t)b * a.H + j0;
+  const size_t pl = (size_t)a.plane16 * 8;
+  float dh[NU], dc[NU];
+  if (owner) {
+    const float4 a0 = *reinterpret_cast<const float4*>(a.dh + e0), a1 = *reinterpret_cast<const float4*>(a.dh + e0 + 4);
+    const float4 c0 = *reinterpret_cast<const float4*>(a.dc + e0), c1 = *reinterpret_cast<const float4*>(a.dc + e0 + 4);
+    dh[0] = a0.x; dh[1] = a0.y; dh[2] = a0.z; dh[3] = a0.w; dh[4] = a1.x; dh[5] = a1.y; dh[6] = a1.z; dh[7] = a1.w;
+    dc[0] = c0.x; dc[1] = c0.y; dc[2] = c0.z; dc[3] = c0.w; dc[4] = c1.x; dc[5] = c1.y; dc[6] = c1.z; dc[7] = c1.w;
+  } else {
+#pragma unroll
+    for (int u = 0; u < NU; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
+  }
+  constexpr uint32_t idesc = make_idesc(1, BM, NC, false, false);
+
+  // Reduces the partial tiles of product number `it` into this thread's dh.  Every thread of every
+  // CTA of the cluster calls it (it contains the cluster barrier), whether or not anything failed.
+  auto reduce_partials = [&](int it) {
+    float* mine = part + (size_t)(it & 1) * BM * PLD;
+    const bool got = wait_or_fail(&acc, (uint32_t)it & 1, &failed);
+    tc_fence_after_sync();
+#pragma unroll
+    for (int c0 = 0; c0 < NC; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)c0, r);
+      tmem_ld_wait();
+      if (row_thread) {
+        float4* dst = reinterpret_cast<float4*>(mine + (size_t)b * PLD + c0);
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                               __uint_as_float(r[4 * v + 3]));
+      }
+    }
+    tc_fence_before_sync();
+    cluster_sync();
+    if (got && owner) {
+      float sum[NU];
+#pragma unroll
+      for (int u = 0; u < NU; ++u) sum[u] = 0.f;
+      const float* src = mine + (size_t)b * PLD + rank * NU;
+#pragma unroll
+      for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
+        const float4 v0 = ld_peer_f4(src, p), v1 = ld_peer_f4(src + 4, p);
+        sum[0] += v0.x; sum[1] += v0.y; sum[2] += v0.z; sum[3] += v0.w;
+        sum[4] += v1.x; sum[5] += v1.y; sum[6] += v1.z; sum[7] += v1.w;
+      }
+#pragma unroll
+      for (int u = 0; u < NU; ++u) dh[u] = sum[u];
+    }
+  };
+
+  for (int i = 0; i < a.n; ++i) {
+    const DevOp op = a.ops[i];
+    const int sidx = (op.k - 1) % a.S;
+    if (i > 0) reduce_partials(i - 1);
+    if (owner && !failed) backward_gates(a, op, sidx, b, cta, e0, pl, dh, dc);
+    if (cta == 0 && tid == 0) {
+      float s = 0.f;
+      for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
+      a.loss_t[op.k - 1] = s;
+    }
+    fence_proxy_async();
+    __syncthreads();
+    if (tid == 0) red_release_add(a.sync, 1u);
+
+    if (is_p) {
+      // this CTA's K-slice of dz_k, all of it in flight at once
+      if (wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed)) {
+        fence_proxy_async();
+        const int32_t row = sidx * a.B;
+        for (int kb = 0; kb < KBS; ++kb) {
+          mbar_arrive_expect_tx(&full[kb], A_TILE);
+          tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[kb]);
+        }
+      }
+    } else if (is_mma) {
+      bool ok = true;
+      if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
+      for (int kb = 0; kb < KBS && ok; ++kb) {
+        ok = wait_or_fail(&full[kb], (uint32_t)i & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a0 = smem_u32(ring + kb * A_TILE), b0 = smem_u32(sW + kb * W_TILE);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          mma_f16(tmem, make_desc_sw128(a0 + k4 * 32, 16, 1024), make_desc_sw128(b0 + k4 * 32, 16, 1024), idesc,
+                  (kb > 0 || k4 > 0) ? 1u : 0u);
+      }
+      mma_commit(&acc);
+    }
+    __syncwarp();
+  }
+
+  reduce_partials(a.n - 1);
+  if (owner && !failed) {
+    *reinterpret_cast<float4*>(a.dh + e0) = make_float4(dh[0], dh[1], dh[2], dh[3]);
+    *reinterpret_cast<float4*>(a.dh + e0 + 4) = make_float4(dh[4], dh[5], dh[6], dh[7]);
+    *reinterpret_cast<float4*>(a.dc + e0) = make_float4(dc[0], dc[1], dc[2], dc[3]);
+    *reinterpret_cast<float4*>(a.dc + e0 + 4) = make_float4(dc[4], dc[5], dc[6], dc[7]);
+  }
+  if (failed) {
+    if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
+    if (is_p) {
+      // loads that were requested may still be landing
+      for (int kb = 0; kb < KBS; ++kb) (void)mbar_wait(&full[kb], (uint32_t)(a.n - 1) & 1);
+      (void)mbar_wait(&wfull, 0);
+    }
+  } else if (cta == 0 && tid == 0) {
+    a.counters[1] += a.n;
+  }
+  tc_fence_before_sync();
+  cluster_sync();   // no CTA leaves while a peer may still read its partial tiles
+  if (warp == 1) tmem_dealloc(tmem, 64);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -604,14 +795,24 @@ __global__ void loss_dy(const DevOp* ops, const float* y, const float* targets, 
   if (threadIdx.x == 0) loss_part[sidx * LOSS_PARTS + blockIdx.x] = red[0] * inv;
 }
 
-// out[map(n)] += sum_r v[r][n], rows ascending; perm_h > 0 maps column 4 u + q to q perm_h + u.
+// out[map(n)] += sum_r v[r][n]; perm_h > 0 maps column 4 u + q to q perm_h + u.  A block of
+// 32 x 8 threads sums 32 columns: thread (x, g) takes rows g, g + 8, ... in ascending order, then
+// the eight partial sums are added in the order g = 0 .. 7.
 __global__ void colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out, int perm_h) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  if (n >= N) return;
+  __shared__ float part[8][33];
+  const int n = blockIdx.x * 32 + threadIdx.x, g = threadIdx.y;
   float s = 0.f;
-  for (int r = 0; r < rows; ++r) s += __bfloat162float(v[(size_t)r * N + n]);
-  const int o = perm_h ? ((n & 3) * perm_h + (n >> 2)) : n;
-  out[o] += s;
+  if (n < N)
+    for (int r = g; r < rows; r += 8) s += __bfloat162float(v[(size_t)r * N + n]);
+  part[g][threadIdx.x] = s;
+  __syncthreads();
+  if (g == 0 && n < N) {
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += part[i][threadIdx.x];
+    const int o = perm_h ? ((n & 3) * perm_h + (n >> 2)) : n;
+    out[o] += tot;
+  }
 }
 
 __global__ void finalize_tc(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
@@ -710,9 +911,12 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   float* bias_p = reinterpret_cast<float*>(at(y.off_bias_p));
   __nv_bfloat16* woutT = reinterpret_cast<__nv_bfloat16*>(at(y.off_woutT));
 
-  const int fwd_smem = ((H + 63) / 64) * 4096 + NST * BM * 128 + 1024;
+  const int KBh = (H + 63) / 64;
+  const int fwd_nst = (KBh <= 16 && KBh * 4096 + KBh * BM * 128 + 1024 <= 216 * 1024) ? KBh : NST;
+  const int fwd_smem = KBh * 4096 + fwd_nst * BM * 128 + 1024;
   const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
-  CUtensorMap tm_h, tm_w, tm_dz, tm_wt;
+  CUtensorMap tm_h, tm_w, tm_dz, tm_wt, tm_dz_b, tm_wt_c;
+  int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
   if (!dry) {
     static const bool attrs = [] {
       const int big = 220 * 1024;  // the kernels also hold a few static barriers
@@ -728,6 +932,34 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     ok = ok && make_tmap_2d(&tm_dz, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, (uint32_t)BM);
     ok = ok && make_tmap_2d(&tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
     if (!ok) return MEBPTT_ERR_UNSUPPORTED;
+    // the clustered backward kernel, if the device can keep enough clusters resident
+    // (MEBPTT_BWD_CLUSTER = 0, 4 or 8 in the environment overrides the choice)
+    const char* force = getenv("MEBPTT_BWD_CLUSTER");
+    for (int cs : {8, 4}) {
+      if (force && atoi(force) != cs) continue;
+      if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
+      const int kbs = (G / 64) / cs;
+      const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * BM * (NU * cs + 4) * 4 + 1024;
+      if (smem > 220 * 1024) continue;
+      const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
+      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem;
+      cudaLaunchAttribute at1[1];
+      at1[0].id = cudaLaunchAttributeClusterDimension;
+      at1[0].val.clusterDim.x = cs; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
+      cfg.attrs = at1; cfg.numAttrs = 1;
+      int nclusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+      if (nclusters * cs < ncta) continue;
+      bwd_cs = cs; bwdc_smem = smem;
+      break;
+    }
+    if (bwd_cs) {
+      ok = make_tmap_2d(&tm_dz_b, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, 64);
+      ok = ok && make_tmap_2d(&tm_wt_c, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, (uint32_t)(NU * bwd_cs));
+      if (!ok) return MEBPTT_ERR_UNSUPPORTED;
+    }
 
     cudaMemsetAsync(dh, 0, (size_t)B * H * 4, s);
     cudaMemsetAsync(dc, 0, (size_t)B * H * 4, s);
@@ -776,7 +1008,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, n * B, G, I);
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
-        FwdRunArgs a{dops + i, n, ws, zx, sync + launch_id, status, io.counters, B, H, off16(y.plane), off16(y.hsz)};
+        FwdRunArgs a{dops + i, n, ws, zx, sync + launch_id, status, io.counters, B, H, off16(y.plane), off16(y.hsz),
+                     (uint32_t)fwd_nst};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
         const void* fn = (const void*)fwd_run_kernel<64>;
         if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, fwd_smem, s), "forward run launch"))
@@ -808,10 +1041,23 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (!dry && rc == MEBPTT_OK) {
         BwdRunArgs a{dops + i, n, ws, dha, dz, dh, dc, loss_part, loss_t, sync + launch_id, status, io.counters,
                      B, H, S, off16(y.plane), off16(y.hsz)};
-        void* args[] = {(void*)&tm_dz, (void*)&tm_wt, (void*)&a};
-        const void* fn = (const void*)bwd_run_kernel<64>;
-        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, bwd_smem, s), "backward run launch"))
-          rc = MEBPTT_ERR_CUDA;
+        void* args[] = {(void*)(bwd_cs ? &tm_dz_b : &tm_dz), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
+        if (bwd_cs) {
+          cudaLaunchConfig_t cfg = {};
+          cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
+          cudaLaunchAttribute at2[2];
+          at2[0].id = cudaLaunchAttributeClusterDimension;
+          at2[0].val.clusterDim.x = bwd_cs; at2[0].val.clusterDim.y = 1; at2[0].val.clusterDim.z = 1;
+          at2[1].id = cudaLaunchAttributeCooperative;
+          at2[1].val.cooperative = 1;
+          cfg.attrs = at2; cfg.numAttrs = 2;
+          const void* fn = bwd_cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
+          if (!cuda_ok(cudaLaunchKernelExC(&cfg, fn, args), "backward run launch (clusters)")) rc = MEBPTT_ERR_CUDA;
+        } else {
+          const void* fn = (const void*)bwd_run_kernel<64>;
+          if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, bwd_smem, s), "backward run launch"))
+            rc = MEBPTT_ERR_CUDA;
+        }
       }
       ++launch_id;
       if (k_lo == chunk * S + 1) {
@@ -824,8 +1070,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         gemm(dyv, O, true, hk, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
         launches += 2;
         if (!dry && rc == MEBPTT_OK) {
-          colsum_bf16<<<(G + 127) / 128, 128, 0, s>>>(dz, R, G, io.db, H);
-          colsum_bf16<<<(O + 127) / 128, 128, 0, s>>>(dyv, R, O, io.db_out, 0);
+          colsum_bf16<<<(G + 31) / 32, dim3(32, 8), 0, s>>>(dz, R, G, io.db, H);
+          colsum_bf16<<<(O + 31) / 32, dim3(32, 8), 0, s>>>(dyv, R, O, io.db_out, 0);
         }
         if (want_dx)
           gemm(dz, G, false, wpT_ih, G, false,
