@@ -262,6 +262,37 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_
                                 float *dx, int64_t *counters);
 
 /*
+ * The training step for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: it never says where the working memory of an implementation comes from.)
+ *
+ * mebptt_lstm_train_step wants a workspace from its caller, and a caller normally gets one from
+ * cudaMalloc or from an allocator built on it.  That is not always possible where the step runs:
+ * a process that has already given all free device memory to something else, a plug-in whose host
+ * application hands it input and output buffers and nothing more, or a service in which an
+ * allocation would stall the other streams of the device.  This entry point takes the same inputs
+ * and outputs and no workspace; it uses a fixed array of MEBPTT_STATIC_WORKSPACE_BYTES that is part
+ * of the library image, so every GPU that loads the library holds that much memory until the
+ * process exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   - Problems whose workspace (mebptt_lstm_workspace_bytes) exceeds the array are refused with
+ *     MEBPTT_ERR_WORKSPACE and nothing is enqueued; use mebptt_lstm_train_step for those.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the parts that must start at
+ *     zero, so leftovers of the previous call do not matter, but two calls whose device work
+ *     overlaps (different streams, or the ordinary entry point given this memory) race: keep
+ *     calls on one stream or order them with events.
+ *   - Arguments, layouts, outputs, counters and determinism are those of mebptt_lstm_train_step.
+ */
+#define MEBPTT_STATIC_WORKSPACE_BYTES (32u << 20)
+int mebptt_lstm_train_step_static(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan,
+                                  const void *W, const void *b, const void *W_out, const void *b_out,
+                                  const void *x, const void *targets, const void *h0, const void *c0,
+                                  void *stream,
+                                  float *loss, float *dW, float *db, float *dW_out, float *db_out,
+                                  float *dx, int64_t *counters);
+
+/*
  * Push / Pop of Algorithm 2 as an explicit copy, for callers that keep states in a pool of
  * their own: copies `bytes` bytes from src to dst (device pointers, both 16-byte aligned,
  * bytes a multiple of 16) on `stream`.  The train step itself writes memorised states in

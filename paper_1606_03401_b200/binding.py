@@ -79,6 +79,7 @@ _SIGS = {
     "mebptt_lstm_launch_count": (_i64, [_descp, _vp]),
     "mebptt_lstm_train_step": (_i32, _STEP_ARGS),
     "mebptt_lstm_train_step_host": (_i32, _STEP_ARGS),
+    "mebptt_lstm_train_step_static": (_i32, [_descp, _vp] + [_vp] * 8 + [_vp] + [_vp] * 7),
     "mebptt_slot_copy": (_i32, [_vp, _vp, _sz, _vp]),
     "mebptt_gemm_bf16": (_i32, [_vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "mebptt_strerror": (C.c_char_p, [_i32]),
@@ -236,6 +237,22 @@ def mebptt_lstm_train_step_host(desc, plan, W, b, W_out, b_out, x, targets, h0, 
     is a device tensor of at least mebptt_lstm_host_workspace_bytes()."""
     _step(lib.mebptt_lstm_train_step_host, "mebptt_lstm_train_step_host", desc, plan, W, b, W_out,
           b_out, x, targets, h0, c0, workspace, stream, loss, dW, db, dW_out, db_out, dx, counters)
+
+
+MEBPTT_STATIC_WORKSPACE_BYTES = 32 << 20
+
+
+def mebptt_lstm_train_step_static(desc, plan, W, b, W_out, b_out, x, targets, h0, c0, stream,
+                                  loss, dW, db, dW_out, db_out, dx, counters):
+    """The training step without a caller-supplied workspace: for code that may not allocate
+    device memory.  Uses the library's built-in MEBPTT_STATIC_WORKSPACE_BYTES array; problems
+    that need more raise MebpttError(MEBPTT_ERR_WORKSPACE).  Calls share the array: keep them on
+    one stream."""
+    st = lib.mebptt_lstm_train_step_static(
+        C.byref(desc), plan.handle, _ptr(W), _ptr(b), _ptr(W_out), _ptr(b_out), _ptr(x), _ptr(targets),
+        _ptr(h0), _ptr(c0), stream, _ptr(loss), _ptr(dW), _ptr(db), _ptr(dW_out), _ptr(db_out), _ptr(dx),
+        _ptr(counters))
+    _check(st, "mebptt_lstm_train_step_static")
 
 
 def mebptt_gemm_bf16(A, lda, a_major, Bm, ldb, b_major, Cm, ldc, accumulate, bias, M, N, K, status=None,
