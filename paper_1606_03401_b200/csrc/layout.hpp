@@ -81,8 +81,8 @@ inline bool valid_desc(const mebptt_lstm_desc* d) {
 // CTA (8 hidden units x 4 gates x H) that fits in shared memory with one CTA per SM.
 inline bool tensor_path_supported(const mebptt_lstm_desc* d) {
   return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && d->dtype == MEBPTT_BF16 && d->layers == 1 && d->batch <= 64 && d->hidden % 8 == 0 &&
-         d->input % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 && d->hidden / 8 <= 148 &&
-         d->hidden <= 1184;
+         d->input % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
+         d->hidden <= 1024;
 }
 
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
@@ -101,6 +101,27 @@ inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.rec_gates = y.unit;
   y.rec_in = y.unit + (size_t)y.L * y.gsz;
   y.rec = y.rec_in + y.unit;
+}
+
+// Number of persistent-kernel launches the tensor-core executor makes for a plan: forward runs
+// are cut into pieces of at most S consecutive operations, backward runs at chunk boundaries.
+inline size_t count_runs(const Plan* p, int S) {
+  size_t runs = 0, i = 0;
+  const size_t n = p->tape.size();
+  while (i < n) {
+    size_t j = i + 1;
+    if (p->tape[i].kind == MEBPTT_OP_FWD) {
+      while (j < n && j - i < (size_t)S && p->tape[j].kind == MEBPTT_OP_FWD && p->tape[j].k == p->tape[j - 1].k + 1 &&
+             p->tape[j].src == p->tape[j - 1].dst)
+        ++j;
+    } else {
+      const int chunk = (p->tape[i].k - 1) / S;
+      while (j < n && p->tape[j].kind == MEBPTT_OP_BWD && (p->tape[j].k - 1) / S == chunk) ++j;
+    }
+    ++runs;
+    i = j;
+  }
+  return runs;
 }
 
 inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y) {
@@ -142,7 +163,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_dy = take(SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
     y.off_loss_part = take((size_t)y.S * 16 * 4);
-    y.n_sync = (size_t)p->tape.size() + 8;
+    y.n_sync = 32 * (count_runs(p, y.S) + 1);   // 32 words (one 128-byte line) per persistent launch
     y.off_sync = take(y.n_sync * 4);
     y.tape_bytes = (size_t)p->tape.size() * 32;
     y.off_tape = take(y.tape_bytes);

@@ -110,213 +110,231 @@ struct FwdRunArgs {
   int B, H;
   uint32_t plane16;      // distance between gate planes, in 16-byte units
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
-  uint32_t nst;          // ring stages (<= 16); H / 64 when all of h fits next to the weights
 };
 
-template <int BM>
-__global__ void __launch_bounds__(128, 1) fwd_run_kernel(const __grid_constant__ CUtensorMap tm_h,
+// Warps 0-3: epilogue (warp w owns rows 16w .. 16w+15 of the 64-row MMA tile, which are the
+// TMEM lanes it may read); warp 4: TMA producer; warp 5: MMA issuer.  All of h_{k-1} is resident
+// in shared memory for the step (H <= 1024), so the producer never waits for a free slot.
+// (Cutting the batch into groups with independent step counters was tried and does not help: a
+// step is bound by the latency of the exchange, which every group pays in full.)
+__global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__ CUtensorMap tm_h,
                                                          const __grid_constant__ CUtensorMap tm_w,
                                                          const FwdRunArgs a) {
+  constexpr int GR = 1;                    // batch groups (see above)
+  constexpr int RG = 64 / GR;              // tile rows per group
+  constexpr int TG = 128 / GR;             // epilogue threads per group
+  constexpr uint32_t A_TILE = 64 * 128;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[16], empty[16], acc;
+  __shared__ uint64_t wfull, full[GR][4], acc[GR];
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
 
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int KB = (a.H + 63) / 64;
-  uint8_t* sW = sm;                    // KB tiles of [32 rows][128 B]
-  uint8_t* ring = sm + KB * 4096;      // NST tiles of [BM rows][128 B]
-  constexpr uint32_t A_TILE = BM * 128;
+  const int KB = (a.H + 63) / 64;      // <= 16
+  uint8_t* sW = sm;                    // KB tiles of [32 rows][128 B]: this CTA's rows of W_hh
+  uint8_t* tiles = sm + KB * 4096;     // KB tiles of [64 rows][128 B]: all of h_{k-1}
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
-  const bool is_p = (tid == 0), is_mma = (tid == 32);
-  const uint32_t NSTr = a.nst;
+  const int Bg = (a.B + GR - 1) / GR;  // batch rows per group
+  const int NQ = (KB + 3) / 4;         // blocks of four K tiles, one barrier each
 
   if (tid == 0) {
     mbar_init(&wfull, 1);
-    for (int s = 0; s < 16; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(&acc, 1);
+    for (int g = 0; g < GR; ++g) {
+      for (int s = 0; s < 4; ++s) mbar_init(&full[g][s], 1);
+      mbar_init(&acc[g], 1);
+    }
     failed = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tm_h);
     tma_prefetch_desc(&tm_w);
   }
-  if (warp == 1) tmem_alloc(&tmem_slot, 32);
+  if (warp == 4) tmem_alloc(&tmem_slot, 32 * GR);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
-
-  // the recurrent weights of this CTA's 8 units stay in shared memory for the whole run
-  if (is_p) {
-    mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 4096u);
-    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 4096, &tm_w, kb * 64, cta * NG, &wfull);
-  }
-
-  // ---- per-thread state: one batch row, the CTA's 8 hidden units ---------------------------
-  const int b = (BM == 64) ? (16 * warp + lane) : (32 * warp + lane);
-  const bool owner = ((BM == 64) ? (lane < 16) : true) && b < a.B;
-  const int j0 = cta * NU;
-  const size_t e0 = (size_t)b * a.H + j0;           // element index of (b, j0) in a [B][H] array
-  float c[NU];
-  uint4 hprev = make_uint4(0, 0, 0, 0);
-  float zx[NG];
-  {
-    const DevOp op0 = a.ops[0];
-    if (owner) {
-      const float* cp = reinterpret_cast<const float*>(a.ws + (size_t)op0.c_src * 16) + e0;
-      const float4 c0 = *reinterpret_cast<const float4*>(cp), c1 = *reinterpret_cast<const float4*>(cp + 4);
-      c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
-      hprev = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op0.h_src * 16) + e0);
-      const float4* zp = reinterpret_cast<const float4*>(a.zx + (size_t)b * 4 * a.H + (size_t)cta * NG);
-#pragma unroll
-      for (int v = 0; v < NG / 4; ++v) {
-        const float4 z = zp[v];
-        zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
-      }
-    } else {
-#pragma unroll
-      for (int u = 0; u < NU; ++u) c[u] = 0.f;
-#pragma unroll
-      for (int v = 0; v < NG; ++v) zx[v] = 0.f;
-    }
-  }
-
-  uint32_t issued = 0;      // ring tiles requested so far (producer thread)
-  uint32_t consumed = 0;    // ring tiles multiplied so far (MMA thread)
-  constexpr uint32_t idesc = make_idesc(1, BM, NG, false, false);
   const uint32_t row_bytes = (uint32_t)a.H * 2u;
 
-  for (int i = 0; i < a.n; ++i) {
-    const DevOp op = a.ops[i];
-    if (is_p) {
-      // ---- producer: h_{k-1} through the ring -------------------------------------------
-      bool ok = true;
-      if (i > 0) ok = wait_counter(a.sync, (uint32_t)i * (uint32_t)ncta, &failed);
-      if (ok) {
-        fence_proxy_async();
+  if (warp == 4) {
+    // ---- producer ---------------------------------------------------------------------------
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 4096u);
+      for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 4096, &tm_w, kb * 64, cta * NG, &wfull);
+      int armed = -1;   // last step whose loads were requested (for the failure path)
+      for (int i = 0; i < a.n; ++i) {
+        const DevOp op = a.ops[i];
         const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
-        for (int kb = 0; kb < KB && ok; ++kb, ++issued) {
-          const uint32_t s = issued % NSTr, it = issued / NSTr;
-          if (it > 0) ok = wait_or_fail(&empty[s], (it - 1) & 1, &failed);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&full[s], A_TILE);
-          tma_load_2d(ring + s * A_TILE, &tm_h, kb * 64, row, &full[s]);
+        for (int g = 0; g < GR; ++g) {
+          if (i > 0 && !wait_counter(a.sync + g * 8, (uint32_t)i * (uint32_t)ncta, &failed)) continue;
+          if (failed) continue;
+          fence_proxy_async();
+          // one barrier per block of four K tiles
+          for (int q = 0; q < NQ; ++q) {
+            const int kb0 = 4 * q, kb1 = (kb0 + 4 < KB) ? kb0 + 4 : KB;
+            mbar_arrive_expect_tx(&full[g][q], (uint32_t)(kb1 - kb0) * RG * 128);
+            for (int kb = kb0; kb < kb1; ++kb)
+              tma_load_2d(tiles + kb * A_TILE + g * RG * 128, &tm_h, kb * 64, row + g * Bg, &full[g][q]);
+          }
+          if (g == GR - 1) armed = i;
         }
       }
-    } else if (is_mma) {
-      // ---- MMA issuer -----------------------------------------------------------------------
-      bool ok = true;
-      if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
-      for (int kb = 0; kb < KB && ok; ++kb, ++consumed) {
-        const uint32_t s = consumed % NSTr, it = consumed / NSTr;
-        ok = wait_or_fail(&full[s], it & 1, &failed);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t a0 = smem_u32(ring + s * A_TILE), b0 = smem_u32(sW + kb * 4096);
-#pragma unroll
-        for (int k4 = 0; k4 < 4; ++k4)
-          mma_f16(tmem, make_desc_sw128(a0 + k4 * 32, 16, 1024), make_desc_sw128(b0 + k4 * 32, 16, 1024), idesc,
-                  (kb > 0 || k4 > 0) ? 1u : 0u);
-        mma_commit(&empty[s]);
+      if (failed) {
+        // loads that were requested may still be landing: give them a bounded chance
+        (void)mbar_wait(&wfull, 0);
+        if (armed >= 0)
+          for (int g = 0; g < GR; ++g)
+            for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[g][q], (uint32_t)armed & 1);
       }
-      mma_commit(&acc);
     }
-    __syncwarp();
-
-    // ---- gates and state update: every thread that owns a batch row ----------------------------
-    const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
-    tc_fence_after_sync();
-    uint32_t r[NG];
-    tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
-    tmem_ld_wait();
-    uint4 hnew = make_uint4(0, 0, 0, 0);
-    uint32_t qi[4], qf[4], qg[4], qo[4];
-    float cold[NU];
-    if (got && owner) {
-      uint32_t hq[4], gi[4], gf[4], gg[4], go[4];
-      float cin[NU];
-#pragma unroll
-      for (int u = 0; u < NU; u += 2) {
-        float hv[2], iv[2], fv[2], gv[2], ov[2];
-#pragma unroll
-        for (int d = 0; d < 2; ++d) {
-          const int q = 4 * (u + d);
-          iv[d] = sigmoid_fast(__uint_as_float(r[q + 0]) + zx[q + 0]);
-          fv[d] = sigmoid_fast(__uint_as_float(r[q + 1]) + zx[q + 1]);
-          gv[d] = tanh_fast(__uint_as_float(r[q + 2]) + zx[q + 2]);
-          ov[d] = sigmoid_fast(__uint_as_float(r[q + 3]) + zx[q + 3]);
-          cin[u + d] = c[u + d];
-          c[u + d] = fmaf(fv[d], c[u + d], iv[d] * gv[d]);
-          hv[d] = ov[d] * tanh_fast(c[u + d]);
+  } else if (warp == 5) {
+    // ---- MMA issuer: the whole warp walks the loop (so that addresses and descriptors stay in
+    // uniform registers), one elected lane issues ------------------------------------------------
+    {
+      constexpr uint32_t idesc = make_idesc(1, 64, NG, false, false);
+      bool ok = wait_or_fail(&wfull, 0, &failed);
+      const uint64_t a_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
+      const uint64_t b_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
+      for (int i = 0; i < a.n; ++i) {
+        for (int g = 0; g < GR; ++g) {
+          const uint32_t d_tmem = tmem + (uint32_t)(g * NG);
+          // descriptors advance by plain additions to their address field: 2 (32 bytes) per K = 16
+          // inside a tile, one tile (8 KB of h, 4 KB of W) per 64 contraction indices
+          uint64_t da = a_desc0, db = b_desc0;
+          for (int q = 0; q < NQ && ok; ++q) {
+            ok = wait_or_fail(&full[g][q], (uint32_t)i & 1, &failed);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int nkb = (4 * q + 4 < KB) ? 4 : KB - 4 * q;
+            if (elect_one()) {
+              for (int kb = 0; kb < nkb; ++kb)
+                mma_f16_x4(d_tmem, da + (uint64_t)(kb * (A_TILE >> 4)), db + (uint64_t)(kb * (4096 >> 4)), idesc,
+                           (q > 0 || kb > 0) ? 1u : 0u);
+            }
+            __syncwarp();
+            da += 4 * (A_TILE >> 4);
+            db += 4 * (4096 >> 4);
+          }
+          if (elect_one()) mma_commit(&acc[g]);   // always: the epilogue counts on one arrival per (step, group)
+          __syncwarp();
         }
-        hq[u / 2] = pack_bf16x2(hv[0], hv[1]);
-        gi[u / 2] = pack_bf16x2(iv[0], iv[1]);
-        gf[u / 2] = pack_bf16x2(fv[0], fv[1]);
-        gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
-        go[u / 2] = pack_bf16x2(ov[0], ov[1]);
       }
-      // h_k first: it is what the other CTAs wait for
-      hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
-      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = hnew;
-#pragma unroll
-      for (int v = 0; v < 4; ++v) { qi[v] = gi[v]; qf[v] = gf[v]; qg[v] = gg[v]; qo[v] = go[v]; }
-#pragma unroll
-      for (int u = 0; u < NU; ++u) cold[u] = cin[u];
     }
-    fence_proxy_async();       // h_k will be read through TMA by every CTA
-    tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0) red_release_add(a.sync, 1u);
-    if (got && owner) {
-      // the rest of the state is not on the critical path of the recurrence
-      char* ws = a.ws;
-      float* cd = reinterpret_cast<float*>(ws + (size_t)op.c_dst * 16) + e0;
-      *reinterpret_cast<float4*>(cd) = make_float4(c[0], c[1], c[2], c[3]);
-      *reinterpret_cast<float4*>(cd + 4) = make_float4(c[4], c[5], c[6], c[7]);
-      if (op.gates) {
-        __nv_bfloat16* g = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
-        const size_t pl = (size_t)a.plane16 * 8;   // elements
-        *reinterpret_cast<uint4*>(g) = make_uint4(qi[0], qi[1], qi[2], qi[3]);
-        *reinterpret_cast<uint4*>(g + pl) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
-        *reinterpret_cast<uint4*>(g + 2 * pl) = make_uint4(qg[0], qg[1], qg[2], qg[3]);
-        *reinterpret_cast<uint4*>(g + 3 * pl) = make_uint4(qo[0], qo[1], qo[2], qo[3]);
-      }
-      if (op.in_copy) {
-        char* blk = ws + (size_t)op.in_copy * 16;
-        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = hprev;
-        float* ci = reinterpret_cast<float*>(blk + (size_t)a.hsz16 * 16) + e0;
-        *reinterpret_cast<float4*>(ci) = make_float4(cold[0], cold[1], cold[2], cold[3]);
-        *reinterpret_cast<float4*>(ci + 4) = make_float4(cold[4], cold[5], cold[6], cold[7]);
-      }
-      hprev = hnew;
-      // the input projection of the next step does not depend on the recurrence: fetch it now
-      if (i + 1 < a.n) {
-        const float4* zp = reinterpret_cast<const float4*>(a.zx + ((size_t)(i + 1) * a.B + b) * 4 * a.H + (size_t)cta * NG);
+  } else {
+    // ---- gates and state update: warp w owns tile rows 16w .. 16w+15 -------------------------
+    const int g = warp / (4 / GR);
+    const int rg = 16 * warp + lane - g * RG;          // row inside the group
+    const int b = g * Bg + rg;                          // batch row
+    const bool owner = lane < 16 && rg < Bg && b < a.B;
+    const int j0 = cta * NU;
+    const size_t e0 = (size_t)b * a.H + j0;             // element index of (b, j0) in a [B][H] array
+    const bool signaller = (warp % (4 / GR) == 0) && lane == 0;
+    float c[NU];
+    uint4 hprev = make_uint4(0, 0, 0, 0);
+    float zx[NG];
+    {
+      const DevOp op0 = a.ops[0];
+      if (owner) {
+        const float* cp = reinterpret_cast<const float*>(a.ws + (size_t)op0.c_src * 16) + e0;
+        const float4 c0 = *reinterpret_cast<const float4*>(cp), c1 = *reinterpret_cast<const float4*>(cp + 4);
+        c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
+        hprev = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op0.h_src * 16) + e0);
+        const float4* zp = reinterpret_cast<const float4*>(a.zx + (size_t)b * 4 * a.H + (size_t)cta * NG);
 #pragma unroll
         for (int v = 0; v < NG / 4; ++v) {
           const float4 z = zp[v];
           zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
         }
+      } else {
+#pragma unroll
+        for (int u = 0; u < NU; ++u) c[u] = 0.f;
+#pragma unroll
+        for (int v = 0; v < NG; ++v) zx[v] = 0.f;
       }
     }
-    if (failed) break;         // uniform: written before the barrier or not at all
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const bool got = wait_or_fail(&acc[g], (uint32_t)i & 1, &failed);
+      tc_fence_after_sync();
+      uint32_t r[NG];
+      tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)(g * NG), r);
+      tmem_ld_wait();
+      uint4 hnew = make_uint4(0, 0, 0, 0);
+      uint32_t gi[4], gf[4], gg[4], go[4];
+      float cin[NU];
+      if (got && owner) {
+        uint32_t hq[4];
+#pragma unroll
+        for (int u = 0; u < NU; u += 2) {
+          float hv[2], iv[2], fv[2], gv[2], ov[2];
+#pragma unroll
+          for (int d = 0; d < 2; ++d) {
+            const int q = 4 * (u + d);
+            iv[d] = sigmoid_fast(__uint_as_float(r[q + 0]) + zx[q + 0]);
+            fv[d] = sigmoid_fast(__uint_as_float(r[q + 1]) + zx[q + 1]);
+            gv[d] = tanh_fast(__uint_as_float(r[q + 2]) + zx[q + 2]);
+            ov[d] = sigmoid_fast(__uint_as_float(r[q + 3]) + zx[q + 3]);
+            cin[u + d] = c[u + d];
+            c[u + d] = fmaf(fv[d], c[u + d], iv[d] * gv[d]);
+            hv[d] = ov[d] * tanh_fast(c[u + d]);
+          }
+          hq[u / 2] = pack_bf16x2(hv[0], hv[1]);
+          gi[u / 2] = pack_bf16x2(iv[0], iv[1]);
+          gf[u / 2] = pack_bf16x2(fv[0], fv[1]);
+          gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
+          go[u / 2] = pack_bf16x2(ov[0], ov[1]);
+        }
+        // h_k first: it is what the other CTAs wait for
+        hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = hnew;
+      }
+      fence_proxy_async();       // h_k will be read through TMA by every CTA
+      tc_fence_before_sync();
+      named_barrier(1 + g, TG);
+      if (signaller) red_release_add(a.sync + g * 8, 1u);
+      if (got && owner) {
+        // the rest of the state is not on the critical path of the recurrence
+        char* ws = a.ws;
+        float* cd = reinterpret_cast<float*>(ws + (size_t)op.c_dst * 16) + e0;
+        *reinterpret_cast<float4*>(cd) = make_float4(c[0], c[1], c[2], c[3]);
+        *reinterpret_cast<float4*>(cd + 4) = make_float4(c[4], c[5], c[6], c[7]);
+        if (op.gates) {
+          __nv_bfloat16* gp = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+          const size_t pl = (size_t)a.plane16 * 8;   // elements
+          *reinterpret_cast<uint4*>(gp) = make_uint4(gi[0], gi[1], gi[2], gi[3]);
+          *reinterpret_cast<uint4*>(gp + pl) = make_uint4(gf[0], gf[1], gf[2], gf[3]);
+          *reinterpret_cast<uint4*>(gp + 2 * pl) = make_uint4(gg[0], gg[1], gg[2], gg[3]);
+          *reinterpret_cast<uint4*>(gp + 3 * pl) = make_uint4(go[0], go[1], go[2], go[3]);
+        }
+        if (op.in_copy) {
+          char* blk = ws + (size_t)op.in_copy * 16;
+          *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = hprev;
+          float* ci = reinterpret_cast<float*>(blk + (size_t)a.hsz16 * 16) + e0;
+          *reinterpret_cast<float4*>(ci) = make_float4(cin[0], cin[1], cin[2], cin[3]);
+          *reinterpret_cast<float4*>(ci + 4) = make_float4(cin[4], cin[5], cin[6], cin[7]);
+        }
+        hprev = hnew;
+        // the input projection of the next step does not depend on the recurrence: fetch it now
+        if (i + 1 < a.n) {
+          const float4* zp = reinterpret_cast<const float4*>(a.zx + ((size_t)(i + 1) * a.B + b) * 4 * a.H + (size_t)cta * NG);
+#pragma unroll
+          for (int v = 0; v < NG / 4; ++v) {
+            const float4 z = zp[v];
+            zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
+          }
+        }
+      }
+    }
   }
 
-  if (failed) {
-    if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
-    // loads that were requested may still be landing: give each ring slot a bounded chance
-    if (is_p)
-      for (uint32_t q = (issued > NSTr ? issued - NSTr : 0); q < issued; ++q)
-        (void)mbar_wait(&full[q % NSTr], (q / NSTr) & 1);
-    if (is_p) (void)mbar_wait(&wfull, 0);
-  } else if (cta == 0 && tid == 0) {
-    a.counters[0] += a.n;
-  }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 32);
+  if (tid == 0) {
+    if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
+    else if (cta == 0) a.counters[0] += a.n;
+  }
+  if (warp == 4) tmem_dealloc(tmem, 32 * GR);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -550,7 +568,7 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
 // cluster synchronises, and each owner thread adds the CS partial values of its 8 columns in the
 // order r = 0 .. CS-1, reading its peers' tiles through distributed shared memory.
 template <int CS>
-__global__ void __launch_bounds__(128, 1) bwd_run_cluster_kernel(const __grid_constant__ CUtensorMap tm_dz,
+__global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_constant__ CUtensorMap tm_dz,
                                                                  const __grid_constant__ CUtensorMap tm_wt,
                                                                  const BwdRunArgs a) {
   constexpr int BM = 64;
@@ -559,13 +577,14 @@ __global__ void __launch_bounds__(128, 1) bwd_run_cluster_kernel(const __grid_co
   constexpr uint32_t A_TILE = BM * 128;
   constexpr uint32_t W_TILE = NC * 128;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[16], acc;
+  __shared__ uint64_t wfull, full[4], acc, pready[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
 
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int G = 4 * a.H;
   const int KBS = (G / 64) / CS;           // 64-wide K blocks in this CTA's slice (<= 16)
+  const int NQ = (KBS + 3) / 4;            // blocks of four K tiles, one barrier each
   uint8_t* sW = sm;                        // KBS tiles [NC rows][128 B]
   uint8_t* ring = sW + KBS * W_TILE;       // KBS tiles [64 rows][128 B], all of the slice at once
   float* part = reinterpret_cast<float*>(ring + KBS * A_TILE);  // 2 x [64][PLD]
@@ -574,146 +593,172 @@ __global__ void __launch_bounds__(128, 1) bwd_run_cluster_kernel(const __grid_co
   const int cta = blockIdx.x, ncta = gridDim.x;
   const uint32_t rank = cluster_ctarank();
   const int cl = cta / CS;
-  const bool is_p = (tid == 0), is_mma = (tid == 32);
 
   if (tid == 0) {
     mbar_init(&wfull, 1);
-    for (int s = 0; s < 16; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s < 4; ++s) mbar_init(&full[s], 1);
     mbar_init(&acc, 1);
+    mbar_init(&pready[0], CS);
+    mbar_init(&pready[1], CS);
     failed = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tm_dz);
     tma_prefetch_desc(&tm_wt);
   }
-  if (warp == 1) tmem_alloc(&tmem_slot, 64);
+  if (warp == 4) tmem_alloc(&tmem_slot, 64);
   tc_fence_before_sync();
-  __syncthreads();
+  cluster_sync();                          // peers arrive on each other's barriers: all must be initialised
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
 
-  if (is_p) {
-    mbar_arrive_expect_tx(&wfull, (uint32_t)KBS * W_TILE);
-    for (int kb = 0; kb < KBS; ++kb)
-      tma_load_2d(sW + kb * W_TILE, &tm_wt, ((int)rank * KBS + kb) * 64, cl * NC, &wfull);
-  }
-
-  const int b = 16 * warp + lane;
-  const bool row_thread = lane < 16;             // holds an accumulator row in TMEM
-  const bool owner = row_thread && b < a.B;
-  const int j0 = cta * NU;
-  const size_t e0 = (size_t)b * a.H + j0;
-  const size_t pl = (size_t)a.plane16 * 8;
-  float dh[NU], dc[NU];
-  if (owner) {
-    const float4 a0 = *reinterpret_cast<const float4*>(a.dh + e0), a1 = *reinterpret_cast<const float4*>(a.dh + e0 + 4);
-    const float4 c0 = *reinterpret_cast<const float4*>(a.dc + e0), c1 = *reinterpret_cast<const float4*>(a.dc + e0 + 4);
-    dh[0] = a0.x; dh[1] = a0.y; dh[2] = a0.z; dh[3] = a0.w; dh[4] = a1.x; dh[5] = a1.y; dh[6] = a1.z; dh[7] = a1.w;
-    dc[0] = c0.x; dc[1] = c0.y; dc[2] = c0.z; dc[3] = c0.w; dc[4] = c1.x; dc[5] = c1.y; dc[6] = c1.z; dc[7] = c1.w;
-  } else {
-#pragma unroll
-    for (int u = 0; u < NU; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
-  }
-  constexpr uint32_t idesc = make_idesc(1, BM, NC, false, false);
-
-  // Reduces the partial tiles of product number `it` into this thread's dh.  Every thread of every
-  // CTA of the cluster calls it (it contains the cluster barrier), whether or not anything failed.
-  auto reduce_partials = [&](int it) {
-    float* mine = part + (size_t)(it & 1) * BM * PLD;
-    const bool got = wait_or_fail(&acc, (uint32_t)it & 1, &failed);
-    tc_fence_after_sync();
-#pragma unroll
-    for (int c0 = 0; c0 < NC; c0 += 32) {
-      uint32_t r[32];
-      tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)c0, r);
-      tmem_ld_wait();
-      if (row_thread) {
-        float4* dst = reinterpret_cast<float4*>(mine + (size_t)b * PLD + c0);
-#pragma unroll
-        for (int v = 0; v < 8; ++v)
-          dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                               __uint_as_float(r[4 * v + 3]));
-      }
-    }
-    tc_fence_before_sync();
-    cluster_sync();
-    if (got && owner) {
-      float sum[NU];
-#pragma unroll
-      for (int u = 0; u < NU; ++u) sum[u] = 0.f;
-      const float* src = mine + (size_t)b * PLD + rank * NU;
-#pragma unroll
-      for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
-        const float4 v0 = ld_peer_f4(src, p), v1 = ld_peer_f4(src + 4, p);
-        sum[0] += v0.x; sum[1] += v0.y; sum[2] += v0.z; sum[3] += v0.w;
-        sum[4] += v1.x; sum[5] += v1.y; sum[6] += v1.z; sum[7] += v1.w;
-      }
-#pragma unroll
-      for (int u = 0; u < NU; ++u) dh[u] = sum[u];
-    }
-  };
-
-  for (int i = 0; i < a.n; ++i) {
-    const DevOp op = a.ops[i];
-    const int sidx = (op.k - 1) % a.S;
-    if (i > 0) reduce_partials(i - 1);
-    if (owner && !failed) backward_gates(a, op, sidx, b, cta, e0, pl, dh, dc);
-    if (cta == 0 && tid == 0) {
-      float s = 0.f;
-      for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
-      a.loss_t[op.k - 1] = s;
-    }
-    fence_proxy_async();
-    __syncthreads();
-    if (tid == 0) red_release_add(a.sync, 1u);
-
-    if (is_p) {
-      // this CTA's K-slice of dz_k, all of it in flight at once
-      if (wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed)) {
+  if (warp == 4) {
+    // ---- producer: this CTA's K-slice of dz_k, all of it in flight at once ---------------------
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&wfull, (uint32_t)KBS * W_TILE);
+      for (int kb = 0; kb < KBS; ++kb)
+        tma_load_2d(sW + kb * W_TILE, &tm_wt, ((int)rank * KBS + kb) * 64, cl * NC, &wfull);
+      int armed = -1;
+      for (int i = 0; i < a.n; ++i) {
+        const int sidx = (a.ops[i].k - 1) % a.S;
+        if (!wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed)) continue;
         fence_proxy_async();
         const int32_t row = sidx * a.B;
-        for (int kb = 0; kb < KBS; ++kb) {
-          mbar_arrive_expect_tx(&full[kb], A_TILE);
-          tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[kb]);
+        for (int q = 0; q < NQ; ++q) {
+          const int kb0 = 4 * q, kb1 = (kb0 + 4 < KBS) ? kb0 + 4 : KBS;
+          mbar_arrive_expect_tx(&full[q], (uint32_t)(kb1 - kb0) * A_TILE);
+          for (int kb = kb0; kb < kb1; ++kb)
+            tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
         }
+        armed = i;
       }
-    } else if (is_mma) {
-      bool ok = true;
-      if (i == 0) ok = wait_or_fail(&wfull, 0, &failed);
-      for (int kb = 0; kb < KBS && ok; ++kb) {
-        ok = wait_or_fail(&full[kb], (uint32_t)i & 1, &failed);
+      if (failed) {
+        (void)mbar_wait(&wfull, 0);
+        if (armed >= 0)
+          for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
+      }
+    }
+  } else if (warp == 5) {
+    // ---- MMA issuer: the whole warp walks the loop, one elected lane issues --------------------
+    constexpr uint32_t idesc = make_idesc(1, BM, NC, false, false);
+    bool ok = wait_or_fail(&wfull, 0, &failed);
+    const uint64_t a_desc0 = make_desc_sw128(smem_u32(ring), 16, 1024);
+    const uint64_t b_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
+    for (int i = 0; i < a.n; ++i) {
+      uint64_t da = a_desc0, db = b_desc0;
+      for (int q = 0; q < NQ && ok; ++q) {
+        ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t a0 = smem_u32(ring + kb * A_TILE), b0 = smem_u32(sW + kb * W_TILE);
-#pragma unroll
-        for (int k4 = 0; k4 < 4; ++k4)
-          mma_f16(tmem, make_desc_sw128(a0 + k4 * 32, 16, 1024), make_desc_sw128(b0 + k4 * 32, 16, 1024), idesc,
-                  (kb > 0 || k4 > 0) ? 1u : 0u);
+        const int nkb = (4 * q + 4 < KBS) ? 4 : KBS - 4 * q;
+        if (elect_one()) {
+          for (int kb = 0; kb < nkb; ++kb)
+            mma_f16_x4(tmem, da + (uint64_t)(kb * (A_TILE >> 4)), db + (uint64_t)(kb * (W_TILE >> 4)), idesc,
+                       (q > 0 || kb > 0) ? 1u : 0u);
+        }
+        __syncwarp();
+        da += 4 * (A_TILE >> 4);
+        db += 4 * (W_TILE >> 4);
       }
-      mma_commit(&acc);
+      if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
+      __syncwarp();
     }
-    __syncwarp();
+  } else {
+    // ---- gate derivatives: warp w owns tile rows 16w .. 16w+15 ----------------------------------
+    const int b = 16 * warp + lane;
+    const bool row_thread = lane < 16;             // holds an accumulator row in TMEM
+    const bool owner = row_thread && b < a.B;
+    const int j0 = cta * NU;
+    const size_t e0 = (size_t)b * a.H + j0;
+    const size_t pl = (size_t)a.plane16 * 8;
+    float dh[NU], dc[NU];
+    if (owner) {
+      const float4 a0 = *reinterpret_cast<const float4*>(a.dh + e0), a1 = *reinterpret_cast<const float4*>(a.dh + e0 + 4);
+      const float4 c0 = *reinterpret_cast<const float4*>(a.dc + e0), c1 = *reinterpret_cast<const float4*>(a.dc + e0 + 4);
+      dh[0] = a0.x; dh[1] = a0.y; dh[2] = a0.z; dh[3] = a0.w; dh[4] = a1.x; dh[5] = a1.y; dh[6] = a1.z; dh[7] = a1.w;
+      dc[0] = c0.x; dc[1] = c0.y; dc[2] = c0.z; dc[3] = c0.w; dc[4] = c1.x; dc[5] = c1.y; dc[6] = c1.z; dc[7] = c1.w;
+    } else {
+#pragma unroll
+      for (int u = 0; u < NU; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
+    }
+
+    // Reduces the partial tiles of product number `it` into this thread's dh: own tile from TMEM
+    // to shared memory, tell every CTA of the cluster, wait until all of them have told us, then
+    // add the CS partial values of our columns in the order of the ranks.
+    auto reduce_partials = [&](int it) {
+      float* mine = part + (size_t)(it & 1) * BM * PLD;
+      const bool got = wait_or_fail(&acc, (uint32_t)it & 1, &failed);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c0 = 0; c0 < NC; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)c0, r);
+        tmem_ld_wait();
+        if (row_thread) {
+          float4* dst = reinterpret_cast<float4*>(mine + (size_t)b * PLD + c0);
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                 __uint_as_float(r[4 * v + 3]));
+        }
+      }
+      tc_fence_before_sync();
+      named_barrier(1, 128);
+      if (tid < CS) mbar_arrive_peer(&pready[it & 1], (uint32_t)tid);
+      bool all = false;
+      for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait_cluster(&pready[it & 1], (uint32_t)(it >> 1) & 1)) { all = true; break; }
+        if (spin > 256) {
+          if (failed) break;
+          __nanosleep(64);
+        }
+      }
+      if (!all) failed = 1;
+      if (got && all && owner) {
+        float sum[NU];
+#pragma unroll
+        for (int u = 0; u < NU; ++u) sum[u] = 0.f;
+        const float* src = mine + (size_t)b * PLD + rank * NU;
+#pragma unroll
+        for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
+          const float4 v0 = ld_peer_f4(src, p), v1 = ld_peer_f4(src + 4, p);
+          sum[0] += v0.x; sum[1] += v0.y; sum[2] += v0.z; sum[3] += v0.w;
+          sum[4] += v1.x; sum[5] += v1.y; sum[6] += v1.z; sum[7] += v1.w;
+        }
+#pragma unroll
+        for (int u = 0; u < NU; ++u) dh[u] = sum[u];
+      }
+    };
+
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const int sidx = (op.k - 1) % a.S;
+      if (i > 0) reduce_partials(i - 1);
+      if (owner && !failed) backward_gates(a, op, sidx, b, cta, e0, pl, dh, dc);
+      if (cta == 0 && tid == 0) {
+        float s = 0.f;
+        for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
+        a.loss_t[op.k - 1] = s;
+      }
+      fence_proxy_async();
+      named_barrier(1, 128);
+      if (tid == 0) red_release_add(a.sync, 1u);
+    }
+    reduce_partials(a.n - 1);
+    if (owner && !failed) {
+      *reinterpret_cast<float4*>(a.dh + e0) = make_float4(dh[0], dh[1], dh[2], dh[3]);
+      *reinterpret_cast<float4*>(a.dh + e0 + 4) = make_float4(dh[4], dh[5], dh[6], dh[7]);
+      *reinterpret_cast<float4*>(a.dc + e0) = make_float4(dc[0], dc[1], dc[2], dc[3]);
+      *reinterpret_cast<float4*>(a.dc + e0 + 4) = make_float4(dc[4], dc[5], dc[6], dc[7]);
+    }
   }
 
-  reduce_partials(a.n - 1);
-  if (owner && !failed) {
-    *reinterpret_cast<float4*>(a.dh + e0) = make_float4(dh[0], dh[1], dh[2], dh[3]);
-    *reinterpret_cast<float4*>(a.dh + e0 + 4) = make_float4(dh[4], dh[5], dh[6], dh[7]);
-    *reinterpret_cast<float4*>(a.dc + e0) = make_float4(dc[0], dc[1], dc[2], dc[3]);
-    *reinterpret_cast<float4*>(a.dc + e0 + 4) = make_float4(dc[4], dc[5], dc[6], dc[7]);
-  }
-  if (failed) {
-    if (tid == 0) *a.status = MEBPTT_ERR_TIMEOUT;
-    if (is_p) {
-      // loads that were requested may still be landing
-      for (int kb = 0; kb < KBS; ++kb) (void)mbar_wait(&full[kb], (uint32_t)(a.n - 1) & 1);
-      (void)mbar_wait(&wfull, 0);
-    }
-  } else if (cta == 0 && tid == 0) {
-    a.counters[1] += a.n;
-  }
   tc_fence_before_sync();
-  cluster_sync();   // no CTA leaves while a peer may still read its partial tiles
-  if (warp == 1) tmem_dealloc(tmem, 64);
+  cluster_sync();   // no CTA leaves while a peer may still read its partial tiles or signal it
+  if (tid == 0) {
+    if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
+    else if (cta == 0) a.counters[1] += a.n;
+  }
+  if (warp == 4) tmem_dealloc(tmem, 64);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -912,22 +957,22 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   __nv_bfloat16* woutT = reinterpret_cast<__nv_bfloat16*>(at(y.off_woutT));
 
   const int KBh = (H + 63) / 64;
-  const int fwd_nst = (KBh <= 16 && KBh * 4096 + KBh * BM * 128 + 1024 <= 216 * 1024) ? KBh : NST;
-  const int fwd_smem = KBh * 4096 + fwd_nst * BM * 128 + 1024;
+  const int fwd_smem = KBh * 4096 + KBh * 64 * 128 + 1024;
+  const int GRf = 1;
   const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
   CUtensorMap tm_h, tm_w, tm_dz, tm_wt, tm_dz_b, tm_wt_c;
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
   if (!dry) {
     static const bool attrs = [] {
       const int big = 220 * 1024;  // the kernels also hold a few static barriers
-      cudaFuncSetAttribute(fwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+      cudaFuncSetAttribute(fwd_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
       cudaFuncSetAttribute(bwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
       return true;
     }();
     (void)attrs;
     // the whole workspace as rows of H bfloat16: any h block starts at a whole row
     const uint64_t rows = y.total / ((size_t)H * 2);
-    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, (uint32_t)BM);
+    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, (uint32_t)(64 / GRf));
     ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, NG);
     ok = ok && make_tmap_2d(&tm_dz, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, (uint32_t)BM);
     ok = ok && make_tmap_2d(&tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
@@ -944,7 +989,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
       cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem;
+      cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
       cudaLaunchAttribute at1[1];
       at1[0].id = cudaLaunchAttributeClusterDimension;
       at1[0].val.clusterDim.x = cs; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
@@ -1008,11 +1053,11 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, n * B, G, I);
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
-        FwdRunArgs a{dops + i, n, ws, zx, sync + launch_id, status, io.counters, B, H, off16(y.plane), off16(y.hsz),
-                     (uint32_t)fwd_nst};
+        FwdRunArgs a{dops + i, n, ws, zx, sync + (size_t)launch_id * 32, status, io.counters, B, H, off16(y.plane),
+                     off16(y.hsz)};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
-        const void* fn = (const void*)fwd_run_kernel<64>;
-        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, fwd_smem, s), "forward run launch"))
+        const void* fn = (const void*)fwd_run_kernel;
+        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(192), args, fwd_smem, s), "forward run launch"))
           rc = MEBPTT_ERR_CUDA;
       }
       ++launch_id;
@@ -1039,12 +1084,12 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       gemm(dyv + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
-        BwdRunArgs a{dops + i, n, ws, dha, dz, dh, dc, loss_part, loss_t, sync + launch_id, status, io.counters,
+        BwdRunArgs a{dops + i, n, ws, dha, dz, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status, io.counters,
                      B, H, S, off16(y.plane), off16(y.hsz)};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b : &tm_dz), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         if (bwd_cs) {
           cudaLaunchConfig_t cfg = {};
-          cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
+          cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
           cudaLaunchAttribute at2[2];
           at2[0].id = cudaLaunchAttributeClusterDimension;
           at2[0].val.clusterDim.x = bwd_cs; at2[0].val.clusterDim.y = 1; at2[0].val.clusterDim.z = 1;
