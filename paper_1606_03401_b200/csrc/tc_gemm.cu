@@ -111,6 +111,70 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   bool ok = mbar_wait(&done, 0);
   tc_fence_after_sync();
   if (ok && !failed) {
+    // Float32 tiles whose rows can be written as aligned float4: each warp parks its 32 x 128
+    // block of the accumulator in the (now idle) operand ring, then writes -- or adds to -- one
+    // whole 512-byte row of C per instruction.  Everything else takes the per-thread path below.
+    const bool wide = out.kind != GemmOut::STORE_BF16 && (out.ld % 4 == 0) &&
+                      ((reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0) && (n0 % 4 == 0) &&
+                      ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0);
+    if (wide) {
+      constexpr int PITCH = BN + 4;   // floats; keeps both the parking and the row reads conflict-free
+      float* park = reinterpret_cast<float*>(ring) + (size_t)warp * 32 * PITCH;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+        tmem_ld_wait();
+        float4* dst = reinterpret_cast<float4*>(park + (size_t)lane * PITCH + c * 32);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                               __uint_as_float(r[4 * j + 3]));
+      }
+      __syncwarp();
+      const int col = n0 + lane * 4;
+      const bool col_ok = col + 3 < N;       // N % 4 == 0 is implied by ld % 4 == 0 only for ld == N: check
+      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (out.bias && col_ok) bv = *reinterpret_cast<const float4*>(out.bias + col);
+      float* base = reinterpret_cast<float*>(out.ptr);
+#pragma unroll 1
+      for (int r0 = 0; r0 < 32; r0 += 8) {
+        float4 old[8];
+        size_t off[8];
+        bool live[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int row = m0 + warp * 32 + r0 + j;
+          const int row_o = out.perm_h ? ((row & 3) * out.perm_h + (row >> 2)) : row;
+          live[j] = row < M && col_ok;
+          off[j] = (size_t)row_o * out.ld + col;
+          old[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (live[j] && out.kind == GemmOut::ACCUM_F32) old[j] = *reinterpret_cast<const float4*>(base + off[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (!live[j]) continue;
+          const float4 v = *reinterpret_cast<const float4*>(park + (size_t)(r0 + j) * PITCH + lane * 4);
+          *reinterpret_cast<float4*>(base + off[j]) =
+              make_float4(v.x + bv.x + old[j].x, v.y + bv.y + old[j].y, v.z + bv.z + old[j].z, v.w + bv.w + old[j].w);
+        }
+      }
+      // columns of a ragged right edge (N not a multiple of 4 inside this tile)
+      if (!col_ok && col < N) {
+        for (int r0 = 0; r0 < 32; ++r0) {
+          const int row = m0 + warp * 32 + r0;
+          if (row >= M) break;
+          const int row_o = out.perm_h ? ((row & 3) * out.perm_h + (row >> 2)) : row;
+          for (int j = 0; j < 4 && col + j < N; ++j) {
+            float v = park[(size_t)r0 * PITCH + lane * 4 + j];
+            if (out.bias) v += out.bias[col + j];
+            float* q = base + (size_t)row_o * out.ld + col + j;
+            if (out.kind == GemmOut::ACCUM_F32) v += *q;
+            *q = v;
+          }
+        }
+      }
+    } else {
     const int row = m0 + warp * 32 + lane;
     const int row_o = out.perm_h ? ((row & 3) * out.perm_h + (row >> 2)) : row;
 #pragma unroll 1
@@ -162,6 +226,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
           }
         }
       }
+    }
     }
   } else if (status && threadIdx.x == 0) {
     *status = MEBPTT_ERR_TIMEOUT;
