@@ -48,7 +48,7 @@ WORKLOADS = {
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS))
@@ -83,7 +83,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.thr = threading.Thread(target=self._read, daemon=True)
             self.thr.start()
         except Exception:
@@ -206,12 +206,15 @@ def main():
     stream = torch.cuda.current_stream()
 
     def timed(plan, steps, warmup, sample_clocks=False):
-        for _ in range(warmup):
-            dp.enqueue(plan)
+        # the sampler starts before the warm-up so that short timed regions still get samples;
+        # the warm-up runs the same kernels at the same load
         sampler = ClockSampler(local) if sample_clocks else None
-        barrier()
         if sampler:
             sampler.start()
+            time.sleep(0.3)
+        for _ in range(warmup):
+            dp.enqueue(plan)
+        barrier()
         evs = []
         for _ in range(steps):
             flush.fill_(1)

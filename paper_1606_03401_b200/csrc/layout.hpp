@@ -162,7 +162,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_y = take(SB * y.O * 4);
     y.off_dy = take(SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
-    y.off_loss_part = take((size_t)y.S * 16 * 4);
+    y.off_loss_part = take((size_t)y.S * 64 * 4);   // 64 partial sums per step
     y.n_sync = 32 * (count_runs(p, y.S) + 1);   // 32 words (one 128-byte line) per persistent launch
     y.off_sync = take(y.n_sync * 4);
     y.tape_bytes = (size_t)p->tape.size() * 32;

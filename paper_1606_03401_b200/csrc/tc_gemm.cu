@@ -11,7 +11,7 @@
 // is stored [k][m] (rows are contraction indices), which is how dz and the layer inputs lie in
 // memory for the weight gradient, so no transposed copies are made.
 //
-// One CTA computes one 128 x 128 tile.  A single thread feeds a 3-stage ring of 128-byte
+// One CTA computes one 128 x 128 tile.  A single thread feeds a 3- or 6-stage ring of 128-byte
 // swizzled shared-memory tiles by TMA (64 contraction indices per stage); a single thread issues
 // tcgen05.mma (M = 128, N = 128, K = 16, four per stage) into a 128-column TMEM accumulator and
 // releases ring slots with tcgen05.commit; then all four warps read the accumulator with
@@ -29,16 +29,16 @@ namespace {
 
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3;
+constexpr int BM = 128, BN = 128, BK = 64, MAX_STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;  // + slack to align the ring to 1024 B
+constexpr int gemm_smem(int stages) { return stages * STAGE_BYTES + 1024; }  // + slack to align the ring to 1024 B
 
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma,
                                                         const __grid_constant__ CUtensorMap tmb, GemmOut out,
-                                                        int M, int N, int K, int* status) {
+                                                        int M, int N, int K, int STAGES, int* status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full[STAGES], empty[STAGES], done;
+  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], done;
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
 
@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   const int nk = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(&done, 1);
     failed = 0;
     mbar_fence_init();
@@ -85,25 +85,31 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       }
     }
     (void)armed;
-  } else if (warp == 1 && lane == 0) {
-    // ---- MMA issuer ---------------------------------------------------------------------
+  } else if (warp == 1) {
+    // ---- MMA issuer: the whole warp walks the loop (descriptors stay in uniform registers), one
+    // elected lane issues --------------------------------------------------------------------------
     constexpr uint32_t idesc = make_idesc(1, BM, BN, A_MN, B_MN);
+    // K-major: 16 contraction indices = 32 B along the row; MN-major: 16 rows of 128 B
+    constexpr uint32_t A_STEP = A_MN ? (2048 >> 4) : (32 >> 4), B_STEP = B_MN ? (2048 >> 4) : (32 >> 4);
+    const uint32_t ring0 = smem_u32(ring);
+    const uint64_t a_desc0 = A_MN ? make_desc_sw128(ring0, 8192, 1024) : make_desc_sw128(ring0, 16, 1024);
+    const uint64_t b_desc0 = B_MN ? make_desc_sw128(ring0 + A_BYTES, 8192, 1024) : make_desc_sw128(ring0 + A_BYTES, 16, 1024);
     bool ok = true;
     for (int kb = 0; kb < nk && ok; ++kb) {
       const int s = kb % STAGES;
       if (!mbar_wait(&full[s], (kb / STAGES) & 1)) { failed = 1; ok = false; break; }
       tc_fence_after_sync();
-      const uint32_t a0 = smem_u32(ring + s * STAGE_BYTES), b0 = a0 + A_BYTES;
+      if (elect_one()) {
+        const uint64_t da = a_desc0 + (uint64_t)(s * (STAGE_BYTES >> 4)), db = b_desc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
-      for (int k4 = 0; k4 < BK / 16; ++k4) {
-        // K-major: 16 contraction indices = 32 B along the row; MN-major: 16 rows of 128 B
-        const uint64_t da = A_MN ? make_desc_sw128(a0 + k4 * 2048, 8192, 1024) : make_desc_sw128(a0 + k4 * 32, 16, 1024);
-        const uint64_t db = B_MN ? make_desc_sw128(b0 + k4 * 2048, 8192, 1024) : make_desc_sw128(b0 + k4 * 32, 16, 1024);
-        mma_f16(tmem, da, db, idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+        for (int k4 = 0; k4 < BK / 16; ++k4)
+          mma_f16(tmem, da + (uint64_t)(k4 * A_STEP), db + (uint64_t)(k4 * B_STEP), idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+        mma_commit(&empty[s]);  // the slot may be refilled once these MMAs have read it
       }
-      mma_commit(&empty[s]);  // the slot may be refilled once these MMAs have read it
+      __syncwarp();
     }
-    mma_commit(&done);
+    if (elect_one()) mma_commit(&done);
+    __syncwarp();
   }
 
   // ---- epilogue: all four warps ---------------------------------------------------------
@@ -254,17 +260,22 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   if (!ok) return MEBPTT_ERR_UNSUPPORTED;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
   static const bool attrs = [] {
-    cudaFuncSetAttribute(gemm_bf16_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
-    cudaFuncSetAttribute(gemm_bf16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
-    cudaFuncSetAttribute(gemm_bf16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
-    cudaFuncSetAttribute(gemm_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    const int most = gemm_smem(MAX_STAGES);
+    cudaFuncSetAttribute(gemm_bf16_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaFuncSetAttribute(gemm_bf16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaFuncSetAttribute(gemm_bf16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaFuncSetAttribute(gemm_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     return true;
   }();
   (void)attrs;
-  if (a_mn && b_mn) gemm_bf16_kernel<true, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
-  else if (!a_mn && !b_mn) gemm_bf16_kernel<false, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
-  else if (a_mn) gemm_bf16_kernel<true, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
-  else gemm_bf16_kernel<false, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, status);
+  // Large grids: 3 stages, two CTAs per SM, so that one CTA's epilogue overlaps the other's main
+  // loop.  Grids of at most one wave: 6 stages, more loads in flight per CTA to hide their latency.
+  const int stages = (grid.x * grid.y <= 148) ? MAX_STAGES : 3;
+  const int GEMM_SMEM = gemm_smem(stages);
+  if (a_mn && b_mn) gemm_bf16_kernel<true, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
+  else if (!a_mn && !b_mn) gemm_bf16_kernel<false, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
+  else if (a_mn) gemm_bf16_kernel<true, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
+  else gemm_bf16_kernel<false, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
   return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
 }
 

@@ -51,7 +51,7 @@ using namespace sm100;
 constexpr int NU = 8;            // hidden units per CTA
 constexpr int NG = 4 * NU;       // gate columns per CTA
 constexpr int NST = 8;           // ring stages of 64 contraction indices
-constexpr int LOSS_PARTS = 16;   // partial sums per step of the loss
+constexpr int LOSS_PARTS = 64;   // partial sums per step of the loss
 
 // Tape entry as the kernels see it.  Offsets are in units of 16 bytes from the workspace base.
 struct DevOp {
