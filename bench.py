@@ -59,6 +59,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--kernel-breakdown", action="store_true",
+                    help="also print device time per kernel for one step (CUPTI via torch.profiler) to stderr")
     return ap.parse_args()
 
 
@@ -115,6 +117,40 @@ class ClockSampler:
         busy = [v for v in sm if mx and v > 0.3 * mx] or sm
         return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def kernel_breakdown(dp, plans):
+    """Device time per kernel over one training step of each plan, measured with CUPTI
+    (kernels run back to back as in production, unlike under ncu)."""
+    import collections
+    import torch
+    from torch.profiler import ProfilerActivity, profile
+    for label, plan in plans:
+        for _ in range(2):
+            dp.enqueue(plan)
+        torch.cuda.synchronize()
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            dp.enqueue(plan)
+            torch.cuda.synchronize()
+        agg = collections.OrderedDict()
+        for ev in prof.events():
+            if ev.device_type == torch.autograd.DeviceType.CUDA:
+                name = ev.name.replace("mebptt::tc::(anonymous namespace)::", "").replace("void ", "")
+                name = name.split("(")[0][:48]
+                a = agg.setdefault(name, [0, 0.0])
+                a[0] += 1
+                a[1] += ev.device_time
+        tot = sum(a[1] for a in agg.values())
+        print(f"\n### {label}: C = {plan.cost}, t = {plan.t}; sum of device times {tot / 1e3:.2f} ms\n", file=sys.stderr)
+        print("| kernel | launches | total us | avg us | share |\n|---|---:|---:|---:|---:|", file=sys.stderr)
+        for k, (n, v) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
+            print(f"| {k} | {n} | {v:.1f} | {v / n:.2f} | {100 * v / tot:.1f}% |", file=sys.stderr)
+
+
+# DRAM traffic of the forward run kernel per forward operation, from the ncu capture summarised in
+# profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md (25.61 MB read + 0.03 MB written per launch
+# of 16 operations).  Valid for config 3's layer sizes and the kernel as profiled there.
+FWD_RUN_DRAM_BYTES_PER_OP_C3 = (25.610496e6 + 34.816e3) / 16
 
 
 def oracle_sample(cfg, seconds: float):
@@ -237,6 +273,8 @@ def main():
 
     plan = dp.plan(mode, m)
     full = dp.full_memory_plan()
+    if args.kernel_breakdown and rank == 0:
+        kernel_breakdown(dp, [(f"{mode} m={plan.m}", plan), ("full memory", full)])
     W = max(3, args.warmup)
     ms, clocks = timed(plan, args.steps, W, sample_clocks=True)
     ms = max_over_ranks(ms)
@@ -261,8 +299,11 @@ def main():
     achieved = flops_fwd_op / (fwd_op_ms * 1e-3) / 1e12 if fwd_op_ms else None
     peak_tf = pk["bf16_tflops_sustained"] if cfg.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2.0
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": (achieved / peak_tf) if achieved else None, "traffic": None,
+                "frac": (achieved / peak_tf) if achieved else None,
+                "traffic": FWD_RUN_DRAM_BYTES_PER_OP_C3 if (cfg.name == "c3" and cfg.input == 1024) else None,
                 "kernel": "forward operation (gate contraction + fused cell update)",
+                "traffic_note": "DRAM bytes per forward operation of fwd_run_kernel alone (ncu, 16-step launch); "
+                                "the batched input projection's traffic is not included",
                 "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
                        f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
                        + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}
