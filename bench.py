@@ -153,6 +153,22 @@ def kernel_breakdown(dp, plans):
 FWD_RUN_DRAM_BYTES_PER_OP_C3 = (25.610496e6 + 34.816e3) / 16
 
 
+def max_over_ranks(v: float, world: int, device) -> float:
+    """Slowest rank's time: the job is done when the last replica is."""
+    if world == 1:
+        return v
+    import torch
+    import torch.distributed as dist
+    tns = torch.tensor([v], dtype=torch.float64, device=device)
+    dist.all_reduce(tns, op=dist.ReduceOp.MAX)
+    return float(tns.item())
+
+
+def job_value(world: int, t: int, ms: float) -> float:
+    """Whole-job sequence-steps per second: every replica advances t steps in ms milliseconds."""
+    return world * t / (ms * 1e-3)
+
+
 def oracle_sample(cfg, seconds: float):
     """Time the oracle, as it stands, on a truncated copy of the workload."""
     from oracle import lstm_bptt as O
@@ -264,12 +280,8 @@ def main():
         ms = [a.elapsed_time(b) for a, b in evs]
         return sum(ms) / len(ms), clocks
 
-    def max_over_ranks(v):
-        if world == 1:
-            return v
-        tns = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(tns, op=dist.ReduceOp.MAX)
-        return float(tns.item())
+    def max_over(v):
+        return max_over_ranks(v, world, dev)
 
     plan = dp.plan(mode, m)
     full = dp.full_memory_plan()
@@ -277,14 +289,14 @@ def main():
         kernel_breakdown(dp, [(f"{mode} m={plan.m}", plan), ("full memory", full)])
     W = max(3, args.warmup)
     ms, clocks = timed(plan, args.steps, W, sample_clocks=True)
-    ms = max_over_ranks(ms)
+    ms = max_over(ms)
     counters = dp.out["counters"].cpu().numpy()
     assert int(counters[0]) == plan.cost and int(counters[3]) == 0, counters
 
     # full-memory BPTT: the denominator of the time ratio, and (by difference) the duration of
     # one forward operation
     ms_full, _ = timed(full, max(2, args.steps // 2), 2)
-    ms_full = max_over_ranks(ms_full)
+    ms_full = max_over(ms_full)
     K = cfg.input + cfg.hidden
     flops_fwd_op = 0
     for l in range(cfg.layers):
@@ -313,7 +325,7 @@ def main():
         for omode, om in others:
             op = dp.plan(omode, om)
             oms, _ = timed(op, max(2, args.steps // 2), 1)
-            oms = max_over_ranks(oms)
+            oms = max_over(oms)
             budgets.append({"mode": omode, "m": om, "C": op.cost, "ms_per_step": oms,
                             "seq_steps_per_s": world * cfg.t / (oms * 1e-3),
                             "ratio_vs_full": oms / ms_full, "paper_model_ratio": (op.cost / cfg.t + 2) / 3,
@@ -342,7 +354,7 @@ def main():
             e2e_step()
             torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / n_e2e
-        dt = max_over_ranks(dt)
+        dt = max_over(dt)
         e2e = {"value": world * cfg.t / dt, "unit": "seq-steps/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3}
         del hws
@@ -354,7 +366,7 @@ def main():
     if rank == 0:
         unit = B.mebptt_lstm_unit_bytes(dp.desc)
         line = {
-            "metric": "lstm_bptt_seq_steps_per_s", "value": world * cfg.t / (ms * 1e-3), "unit": "seq-steps/s",
+            "metric": "lstm_bptt_seq_steps_per_s", "value": job_value(world, cfg.t, ms), "unit": "seq-steps/s",
             "n_gpus": world, "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": f"{cfg.name}: L{cfg.layers} I{cfg.input} H{cfg.hidden} B{cfg.batch} t{cfg.t} O{cfg.readout}",

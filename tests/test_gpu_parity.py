@@ -182,3 +182,35 @@ def test_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
     from tests.util import rel_l2
     for k in ("dW", "db", "dW_out", "db_out", "dx"):
         assert rel_l2(full[k], other[k]) < 1e-2, k
+
+
+def test_c2_full_size_every_budget(H):
+    """Config 2 as timed: I512 H512 B64 t256 bf16, HSM and ISM at m = 16, 64, 256."""
+    cfg = synth.CONFIGS["c2"]
+    dp = H.DeviceProblem(cfg)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, "bf16")
+    for mode, code in (("hsm", P.HSM), ("ism", P.ISM)):
+        for m in (16, 64, 256):
+            plan = dp.plan(mode, m)
+            res = dp.run(plan)
+            assert res["counters"][0] == plan.cost == P.cost(code, cfg.t, plan.m)
+            assert res["counters"][2] == plan.peak_units <= m and res["counters"][3] == 0
+            assert_bit_identical(res, full)
+
+
+def test_c3_full_size_headline_budget(H):
+    """Config 3 as the benchmark times it: I1024 H1024 B64 t1000 bf16, MSM m = 100 (and m = 10),
+    against the fp64 oracle at full length and bit for bit against the full-memory run."""
+    cfg = synth.CONFIGS["c3"]
+    dp = H.DeviceProblem(cfg)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    errs = assert_close_to_oracle(full, ref, "bf16")
+    assert max(errs.values()) < 2e-2
+    for m in (100, 10):
+        plan = dp.plan("msm", m)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+        assert_bit_identical(res, full)
