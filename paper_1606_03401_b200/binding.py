@@ -12,7 +12,7 @@ import os
 import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmebptt.so")
+LIB_PATH = os.environ.get("MEBPTT_LIB") or os.path.join(_PKG, "libmebptt.so")   # MEBPTT_LIB: another build of the library
 
 MEBPTT_HSM, MEBPTT_ISM, MEBPTT_MSM = 0, 1, 2
 MEBPTT_FP32, MEBPTT_TF32, MEBPTT_BF16 = 0, 1, 2

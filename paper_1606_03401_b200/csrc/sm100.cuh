@@ -210,6 +210,14 @@ __device__ __forceinline__ float4 ld_peer_f4(const void* local_smem, uint32_t pe
   return v;
 }
 
+// Store into the shared memory of CTA `peer_rank` of this cluster, at the address that
+// `local_smem` has in this CTA.
+__device__ __forceinline__ void st_peer_f4(void* local_smem, uint32_t peer_rank, float4 v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem)), "r"(peer_rank));
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+               : "memory");
+}
 // Barrier among `count` threads (a multiple of 32) of this CTA; ids 1..15 (0 is __syncthreads).
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");

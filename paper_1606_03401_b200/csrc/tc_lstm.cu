@@ -158,35 +158,37 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   const uint32_t row_bytes = (uint32_t)a.H * 2u;
 
   if (warp == 4) {
-    // ---- producer ---------------------------------------------------------------------------
+    // ---- producer: lane 0 watches the step counter, then lanes 0 .. NQ-1 each request one block
+    // of four K tiles (issuing a TMA load costs ~80 ns; four lanes issue side by side) ------------
     if (lane == 0) {
       mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 4096u);
       for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 4096, &tm_w, kb * 64, cta * NG, &wfull);
-      int armed = -1;   // last step whose loads were requested (for the failure path)
-      for (int i = 0; i < a.n; ++i) {
-        const DevOp op = a.ops[i];
-        const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
-        for (int g = 0; g < GR; ++g) {
-          if (i > 0 && !wait_counter(a.sync + g * 8, (uint32_t)i * (uint32_t)ncta, &failed)) continue;
-          if (failed) continue;
-          fence_proxy_async();
-          // one barrier per block of four K tiles
-          for (int q = 0; q < NQ; ++q) {
-            const int kb0 = 4 * q, kb1 = (kb0 + 4 < KB) ? kb0 + 4 : KB;
-            mbar_arrive_expect_tx(&full[g][q], (uint32_t)(kb1 - kb0) * RG * 128);
-            for (int kb = kb0; kb < kb1; ++kb)
-              tma_load_2d(tiles + kb * A_TILE + g * RG * 128, &tm_h, kb * 64, row + g * Bg, &full[g][q]);
-          }
-          if (g == GR - 1) armed = i;
-        }
+    }
+    int armed = -1;   // last step whose loads were requested (for the failure path)
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
+      int go = 1;
+      if (lane == 0) go = (i == 0 || wait_counter(a.sync, (uint32_t)i * (uint32_t)ncta, &failed)) && !failed;
+      go = __shfl_sync(0xffffffffu, go, 0);
+      if (!go) continue;
+      if (lane < NQ) {
+        // the acquire of lane 0 reaches this lane through the shuffle; the proxy fence then orders
+        // this lane's TMA reads after the h_k written by the other CTAs
+        fence_proxy_async();
+        const int q = lane;
+        const int kb0 = 4 * q, kb1 = (kb0 + 4 < KB) ? kb0 + 4 : KB;
+        mbar_arrive_expect_tx(&full[0][q], (uint32_t)(kb1 - kb0) * A_TILE);
+        for (int kb = kb0; kb < kb1; ++kb) tma_load_2d(tiles + kb * A_TILE, &tm_h, kb * 64, row, &full[0][q]);
       }
-      if (failed) {
-        // loads that were requested may still be landing: give them a bounded chance
-        (void)mbar_wait(&wfull, 0);
-        if (armed >= 0)
-          for (int g = 0; g < GR; ++g)
-            for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[g][q], (uint32_t)armed & 1);
-      }
+      armed = i;
+      __syncwarp();
+    }
+    if (failed && lane == 0) {
+      // loads that were requested may still be landing: give them a bounded chance
+      (void)mbar_wait(&wfull, 0);
+      if (armed >= 0)
+        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[0][q], (uint32_t)armed & 1);
     }
   } else if (warp == 5) {
     // ---- MMA issuer: the whole warp walks the loop (so that addresses and descriptors stay in
@@ -289,9 +291,8 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
         hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
         *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = hnew;
       }
-      fence_proxy_async();       // h_k will be read through TMA by every CTA
       tc_fence_before_sync();
-      named_barrier(1 + g, TG);
+      named_barrier(1 + g, TG);   // all of this CTA's h_k stores precede the release below
       if (signaller) red_release_add(a.sync + g * 8, 1u);
       if (got && owner) {
         // the rest of the state is not on the critical path of the recurrence
@@ -357,27 +358,44 @@ struct BwdRunArgs {
   uint32_t plane16, hsz16;
 };
 
-// Gate derivatives of one batch row and the CTA's 8 hidden units at one step: reads the stored
-// gates and cell states, the readout gradient dha and the carried (dh, dc); writes dz (bfloat16,
-// columns 4 u + q) to the staging chunk and leaves dc = dc_t * f for the next (earlier) step.
-__device__ __forceinline__ void backward_gates(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int cta,
-                                               size_t e0, size_t pl, const float (&dh)[NU], float (&dc)[NU]) {
-  const int G = 4 * a.H;
+// What the gate derivatives of one batch row and 8 hidden units read from memory at one step: the
+// stored gates and cell states and the readout gradient.  None of it depends on the recurrence,
+// so it can be fetched while the exchange of the previous step is still in flight.
+struct GateInputs {
+  uint4 qi, qf, qg, qo;
+  float4 t0, t1, p0, p1, d0, d1;
+};
+__device__ __forceinline__ GateInputs load_gate_inputs(const BwdRunArgs& a, const DevOp& op, int sidx, size_t e0,
+                                                       size_t pl) {
+  GateInputs in;
   const char* ws = a.ws;
   const float* dha = a.dha + ((size_t)sidx * a.B) * a.H + e0;
-  const float4 d0 = *reinterpret_cast<const float4*>(dha), d1 = *reinterpret_cast<const float4*>(dha + 4);
-  const float dhav[NU] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+  in.d0 = *reinterpret_cast<const float4*>(dha);
+  in.d1 = *reinterpret_cast<const float4*>(dha + 4);
   const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
-  const uint4 qi = *reinterpret_cast<const uint4*>(g), qf = *reinterpret_cast<const uint4*>(g + pl);
-  const uint4 qg = *reinterpret_cast<const uint4*>(g + 2 * pl), qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
-  const uint32_t wi[4] = {qi.x, qi.y, qi.z, qi.w}, wf[4] = {qf.x, qf.y, qf.z, qf.w};
-  const uint32_t wg[4] = {qg.x, qg.y, qg.z, qg.w}, wo[4] = {qo.x, qo.y, qo.z, qo.w};
+  in.qi = *reinterpret_cast<const uint4*>(g);
+  in.qf = *reinterpret_cast<const uint4*>(g + pl);
+  in.qg = *reinterpret_cast<const uint4*>(g + 2 * pl);
+  in.qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
   const float* ctp = reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0;
   const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
-  const float4 t0 = *reinterpret_cast<const float4*>(ctp), t1 = *reinterpret_cast<const float4*>(ctp + 4);
-  const float4 p0 = *reinterpret_cast<const float4*>(cpp), p1 = *reinterpret_cast<const float4*>(cpp + 4);
-  const float ct[NU] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-  const float cp[NU] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+  in.t0 = *reinterpret_cast<const float4*>(ctp);
+  in.t1 = *reinterpret_cast<const float4*>(ctp + 4);
+  in.p0 = *reinterpret_cast<const float4*>(cpp);
+  in.p1 = *reinterpret_cast<const float4*>(cpp + 4);
+  return in;
+}
+
+// Gate derivatives from the fetched inputs and the carried (dh, dc); writes dz (bfloat16, columns
+// 4 u + q) to the staging chunk and leaves dc = dc_t * f for the next (earlier) step.
+__device__ __forceinline__ void compute_gates(const BwdRunArgs& a, const GateInputs& in, int sidx, int b, int cta,
+                                              const float (&dh)[NU], float (&dc)[NU]) {
+  const int G = 4 * a.H;
+  const float dhav[NU] = {in.d0.x, in.d0.y, in.d0.z, in.d0.w, in.d1.x, in.d1.y, in.d1.z, in.d1.w};
+  const uint32_t wi[4] = {in.qi.x, in.qi.y, in.qi.z, in.qi.w}, wf[4] = {in.qf.x, in.qf.y, in.qf.z, in.qf.w};
+  const uint32_t wg[4] = {in.qg.x, in.qg.y, in.qg.z, in.qg.w}, wo[4] = {in.qo.x, in.qo.y, in.qo.z, in.qo.w};
+  const float ct[NU] = {in.t0.x, in.t0.y, in.t0.z, in.t0.w, in.t1.x, in.t1.y, in.t1.z, in.t1.w};
+  const float cp[NU] = {in.p0.x, in.p0.y, in.p0.z, in.p0.w, in.p1.x, in.p1.y, in.p1.z, in.p1.w};
   uint32_t out[NG / 2];
 #pragma unroll
   for (int u = 0; u < NU; ++u) {
@@ -402,6 +420,12 @@ __device__ __forceinline__ void backward_gates(const BwdRunArgs& a, const DevOp&
   uint4* dzp = reinterpret_cast<uint4*>(a.dz + ((size_t)sidx * a.B + b) * G + (size_t)cta * NG);
 #pragma unroll
   for (int v = 0; v < NG / 8; ++v) dzp[v] = make_uint4(out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
+}
+
+__device__ __forceinline__ void backward_gates(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int cta,
+                                               size_t e0, size_t pl, const float (&dh)[NU], float (&dc)[NU]) {
+  const GateInputs in = load_gate_inputs(a, op, sidx, e0, pl);
+  compute_gates(a, in, sidx, b, cta, dh, dc);
 }
 
 template <int BM>
@@ -573,7 +597,6 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
                                                                  const BwdRunArgs a) {
   constexpr int BM = 64;
   constexpr int NC = NU * CS;              // columns of dh the cluster produces
-  constexpr int PLD = NC + 4;              // row pitch of a partial tile, floats
   constexpr uint32_t A_TILE = BM * 128;
   constexpr uint32_t W_TILE = NC * 128;
   extern __shared__ uint8_t smem_raw[];
@@ -587,7 +610,8 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
   const int NQ = (KBS + 3) / 4;            // blocks of four K tiles, one barrier each
   uint8_t* sW = sm;                        // KBS tiles [NC rows][128 B]
   uint8_t* ring = sW + KBS * W_TILE;       // KBS tiles [64 rows][128 B], all of the slice at once
-  float* part = reinterpret_cast<float*>(ring + KBS * A_TILE);  // 2 x [64][PLD]
+  // partial sums received from the cluster: [2 buffers][CS senders][64 rows][8 columns]
+  float* recv = reinterpret_cast<float*>(ring + KBS * A_TILE);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
@@ -612,30 +636,36 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
   const uint32_t tmem = tmem_slot;
 
   if (warp == 4) {
-    // ---- producer: this CTA's K-slice of dz_k, all of it in flight at once ---------------------
+    // ---- producer: this CTA's K-slice of dz_k, all of it in flight at once; lane 0 watches the
+    // step counter, lanes 0 .. NQ-1 each request one block of four K tiles -------------------------
     if (lane == 0) {
       mbar_arrive_expect_tx(&wfull, (uint32_t)KBS * W_TILE);
       for (int kb = 0; kb < KBS; ++kb)
         tma_load_2d(sW + kb * W_TILE, &tm_wt, ((int)rank * KBS + kb) * 64, cl * NC, &wfull);
-      int armed = -1;
-      for (int i = 0; i < a.n; ++i) {
-        const int sidx = (a.ops[i].k - 1) % a.S;
-        if (!wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed)) continue;
+    }
+    int armed = -1;
+    for (int i = 0; i < a.n; ++i) {
+      const int sidx = (a.ops[i].k - 1) % a.S;
+      int go = 1;
+      if (lane == 0) go = wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed) && !failed;
+      go = __shfl_sync(0xffffffffu, go, 0);
+      if (!go) continue;
+      if (lane < NQ) {
         fence_proxy_async();
         const int32_t row = sidx * a.B;
-        for (int q = 0; q < NQ; ++q) {
-          const int kb0 = 4 * q, kb1 = (kb0 + 4 < KBS) ? kb0 + 4 : KBS;
-          mbar_arrive_expect_tx(&full[q], (uint32_t)(kb1 - kb0) * A_TILE);
-          for (int kb = kb0; kb < kb1; ++kb)
-            tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
-        }
-        armed = i;
+        const int q = lane;
+        const int kb0 = 4 * q, kb1 = (kb0 + 4 < KBS) ? kb0 + 4 : KBS;
+        mbar_arrive_expect_tx(&full[q], (uint32_t)(kb1 - kb0) * A_TILE);
+        for (int kb = kb0; kb < kb1; ++kb)
+          tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
       }
-      if (failed) {
-        (void)mbar_wait(&wfull, 0);
-        if (armed >= 0)
-          for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
-      }
+      armed = i;
+      __syncwarp();
+    }
+    if (failed && lane == 0) {
+      (void)mbar_wait(&wfull, 0);
+      if (armed >= 0)
+        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
     }
   } else if (warp == 5) {
     // ---- MMA issuer: the whole warp walks the loop, one elected lane issues --------------------
@@ -681,11 +711,12 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
       for (int u = 0; u < NU; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
     }
 
-    // Reduces the partial tiles of product number `it` into this thread's dh: own tile from TMEM
-    // to shared memory, tell every CTA of the cluster, wait until all of them have told us, then
-    // add the CS partial values of our columns in the order of the ranks.
+    // Reduces the partial tiles of product number `it` into this thread's dh.  Each row thread
+    // reads its row of this CTA's partial tile from TMEM and sends the 8 columns that belong to
+    // CTA p straight into p's shared memory; once all CS senders have signalled, the owner adds
+    // the CS partial values of its columns in the order of the ranks.
     auto reduce_partials = [&](int it) {
-      float* mine = part + (size_t)(it & 1) * BM * PLD;
+      float* buf = recv + (size_t)(it & 1) * CS * BM * NU;
       const bool got = wait_or_fail(&acc, (uint32_t)it & 1, &failed);
       tc_fence_after_sync();
 #pragma unroll
@@ -694,16 +725,20 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
         tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)c0, r);
         tmem_ld_wait();
         if (row_thread) {
-          float4* dst = reinterpret_cast<float4*>(mine + (size_t)b * PLD + c0);
 #pragma unroll
-          for (int v = 0; v < 8; ++v)
-            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                                 __uint_as_float(r[4 * v + 3]));
+          for (int pp = 0; pp < 4; ++pp) {   // 32 columns = the columns of four CTAs
+            float* dst = buf + ((size_t)rank * BM + b) * NU;      // slot of sender `rank`, row b
+            const uint32_t peer = (uint32_t)(c0 / NU + pp);
+            st_peer_f4(dst, peer, make_float4(__uint_as_float(r[8 * pp]), __uint_as_float(r[8 * pp + 1]),
+                                              __uint_as_float(r[8 * pp + 2]), __uint_as_float(r[8 * pp + 3])));
+            st_peer_f4(dst + 4, peer, make_float4(__uint_as_float(r[8 * pp + 4]), __uint_as_float(r[8 * pp + 5]),
+                                                  __uint_as_float(r[8 * pp + 6]), __uint_as_float(r[8 * pp + 7])));
+          }
         }
       }
       tc_fence_before_sync();
       named_barrier(1, 128);
-      if (tid < CS) mbar_arrive_peer(&pready[it & 1], (uint32_t)tid);
+      if (tid < CS) mbar_arrive_peer(&pready[it & 1], (uint32_t)tid);   // release: the stores above are visible
       bool all = false;
       for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
         if (mbar_try_wait_cluster(&pready[it & 1], (uint32_t)(it >> 1) & 1)) { all = true; break; }
@@ -717,10 +752,10 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
         float sum[NU];
 #pragma unroll
         for (int u = 0; u < NU; ++u) sum[u] = 0.f;
-        const float* src = mine + (size_t)b * PLD + rank * NU;
 #pragma unroll
-        for (uint32_t p = 0; p < (uint32_t)CS; ++p) {
-          const float4 v0 = ld_peer_f4(src, p), v1 = ld_peer_f4(src + 4, p);
+        for (int p = 0; p < CS; ++p) {
+          const float4* src = reinterpret_cast<const float4*>(buf + ((size_t)p * BM + b) * NU);
+          const float4 v0 = src[0], v1 = src[1];
           sum[0] += v0.x; sum[1] += v0.y; sum[2] += v0.z; sum[3] += v0.w;
           sum[4] += v1.x; sum[5] += v1.y; sum[6] += v1.z; sum[7] += v1.w;
         }
@@ -729,19 +764,23 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
       }
     };
 
+    GateInputs gin;
+    if (owner) gin = load_gate_inputs(a, a.ops[0], (a.ops[0].k - 1) % a.S, e0, pl);
     for (int i = 0; i < a.n; ++i) {
       const DevOp op = a.ops[i];
       const int sidx = (op.k - 1) % a.S;
       if (i > 0) reduce_partials(i - 1);
-      if (owner && !failed) backward_gates(a, op, sidx, b, cta, e0, pl, dh, dc);
+      if (owner && !failed) compute_gates(a, gin, sidx, b, cta, dh, dc);
       if (cta == 0 && tid == 0) {
         float s = 0.f;
         for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
         a.loss_t[op.k - 1] = s;
       }
-      fence_proxy_async();
-      named_barrier(1, 128);
+      named_barrier(1, 128);   // all of this CTA's dz stores precede the release below
       if (tid == 0) red_release_add(a.sync, 1u);
+      // the inputs of the next (earlier) step do not depend on the recurrence: fetch them while the
+      // exchange of this step is in flight
+      if (owner && i + 1 < a.n) gin = load_gate_inputs(a, a.ops[i + 1], (a.ops[i + 1].k - 1) % a.S, e0, pl);
     }
     reduce_partials(a.n - 1);
     if (owner && !failed) {
@@ -984,7 +1023,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (force && atoi(force) != cs) continue;
       if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
       const int kbs = (G / 64) / cs;
-      const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * BM * (NU * cs + 4) * 4 + 1024;
+      const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * cs * BM * NU * 4 + 1024;
       if (smem > 220 * 1024) continue;
       const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
       cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
