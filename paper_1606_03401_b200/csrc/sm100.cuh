@@ -68,6 +68,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 // ---- proxies and fences ---------------------------------------------------------------
 // Orders generic-proxy accesses (ld/st) against async-proxy accesses (TMA, tcgen05 operands).
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// The same, restricted to global memory: what a thread needs between observing (acquire) data
+// that other CTAs wrote with ordinary stores and reading that data with TMA.
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 

@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
       if (lane < NQ) {
         // the acquire of lane 0 reaches this lane through the shuffle; the proxy fence then orders
         // this lane's TMA reads after the h_k written by the other CTAs
-        fence_proxy_async();
+        fence_proxy_async_global();
         const int q = lane;
         const int kb0 = 4 * q, kb1 = (kb0 + 4 < KB) ? kb0 + 4 : KB;
         mbar_arrive_expect_tx(&full[0][q], (uint32_t)(kb1 - kb0) * A_TILE);
@@ -646,12 +646,19 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
     int armed = -1;
     for (int i = 0; i < a.n; ++i) {
       const int sidx = (a.ops[i].k - 1) % a.S;
+      if (cta == 0 && lane == 31) {
+        // loss term of this step: its partial sums in a fixed order (on a lane that is off the
+        // critical path of the recurrence)
+        float sum = 0.f;
+        for (int p = 0; p < LOSS_PARTS; ++p) sum += a.loss_part[sidx * LOSS_PARTS + p];
+        a.loss_t[a.ops[i].k - 1] = sum;
+      }
       int go = 1;
       if (lane == 0) go = wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed) && !failed;
       go = __shfl_sync(0xffffffffu, go, 0);
       if (!go) continue;
       if (lane < NQ) {
-        fence_proxy_async();
+        fence_proxy_async_global();
         const int32_t row = sidx * a.B;
         const int q = lane;
         const int kb0 = 4 * q, kb1 = (kb0 + 4 < KBS) ? kb0 + 4 : KBS;
@@ -771,11 +778,6 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
       const int sidx = (op.k - 1) % a.S;
       if (i > 0) reduce_partials(i - 1);
       if (owner && !failed) compute_gates(a, gin, sidx, b, cta, dh, dc);
-      if (cta == 0 && tid == 0) {
-        float s = 0.f;
-        for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
-        a.loss_t[op.k - 1] = s;
-      }
       named_barrier(1, 128);   // all of this CTA's dz stores precede the release below
       if (tid == 0) red_release_add(a.sync, 1u);
       // the inputs of the next (earlier) step do not depend on the recurrence: fetch them while the
