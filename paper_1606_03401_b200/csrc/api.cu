@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
 
 #include "kernels.hpp"
@@ -49,8 +50,12 @@ int check_common(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
   return MEBPTT_OK;
 }
 
-int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const StepIO& io, cudaStream_t s) {
-  if (y.tensor_path) return (int)tc::run_step(y, p, io, desc->want_dx != 0, s, false);
+int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const StepIO& io, cudaStream_t s,
+             bool side_stream = true) {
+  if (y.tensor_path) {
+    static const bool no_overlap = getenv("MEBPTT_NO_OVERLAP") != nullptr;
+    return (int)tc::run_step(y, p, io, desc->want_dx != 0, s, false, side_stream && !no_overlap);
+  }
   const size_t bh = (size_t)y.B * y.H;
   const size_t plane_elems = y.plane / y.esz;
   char* ws = io.ws;
@@ -195,18 +200,20 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
   const Plan* p = reinterpret_cast<const Plan*>(plan);
   Layout y;
   workspace_layout(desc, p, y);
-  if (y.tensor_path) return tc::run_step(y, p, StepIO{}, desc->want_dx != 0, nullptr, true);
+  if (y.tensor_path) return tc::run_step(y, p, StepIO{}, desc->want_dx != 0, nullptr, true, false);
   // forward operation: one kernel per layer; backward operation: 5 for the readout and
   // 4 per layer; one to finalise
   const int64_t L = desc->layers;
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }
 
-int mebptt_lstm_train_step(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W,
-                           const void* b, const void* W_out, const void* b_out, const void* x,
-                           const void* targets, const void* h0, const void* c0, void* workspace,
-                           size_t workspace_bytes, void* stream, float* loss, float* dW, float* db,
-                           float* dW_out, float* db_out, float* dx, int64_t* counters) {
+}  // extern "C"
+
+namespace mebptt {
+int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W, const void* b,
+                    const void* W_out, const void* b_out, const void* x, const void* targets, const void* h0,
+                    const void* c0, void* workspace, size_t workspace_bytes, void* stream, float* loss, float* dW,
+                    float* db, float* dW_out, float* db_out, float* dx, int64_t* counters, bool side_stream) {
   int rc = check_common(desc, plan);
   if (rc != MEBPTT_OK) return rc;
   if (!W || !b || !W_out || !b_out || !x || !targets || !h0 || !c0) return MEBPTT_ERR_ARG;
@@ -220,7 +227,19 @@ int mebptt_lstm_train_step(const mebptt_lstm_desc* desc, const mebptt_plan_t* pl
   StepIO io{(const char*)W, (const char*)W_out, (const char*)x, (const char*)h0,
             (const float*)b, (const float*)b_out, (const float*)targets, (const float*)c0,
             (char*)workspace, loss, dW, db, dW_out, db_out, dx, counters};
-  return run_step(desc, p, y, io, (cudaStream_t)stream);
+  return run_step(desc, p, y, io, (cudaStream_t)stream, side_stream);
+}
+}  // namespace mebptt
+
+extern "C" {
+
+int mebptt_lstm_train_step(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W,
+                           const void* b, const void* W_out, const void* b_out, const void* x,
+                           const void* targets, const void* h0, const void* c0, void* workspace,
+                           size_t workspace_bytes, void* stream, float* loss, float* dW, float* db,
+                           float* dW_out, float* db_out, float* dx, int64_t* counters) {
+  return train_step_impl(desc, plan, W, b, W_out, b_out, x, targets, h0, c0, workspace, workspace_bytes, stream, loss,
+                         dW, db, dW_out, db_out, dx, counters, true);
 }
 
 size_t mebptt_lstm_host_workspace_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {

@@ -156,11 +156,13 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_bias_p = take(G * 4);
     y.off_woutT = take((size_t)y.O * y.H * 2);
     y.off_zx = take(SB * G * 4);
-    y.off_dz = take(SB * G * 2);
-    y.off_hprev = take(SB * y.H * 2);
-    y.off_hk = take(SB * y.H * 2);
+    // two copies of what the weight-gradient GEMMs read: they may still be running (on the
+    // library's side stream) while the backward pass fills the stages of the next chunk
+    y.off_dz = take(2 * SB * G * 2);
+    y.off_hprev = take(2 * SB * y.H * 2);
+    y.off_hk = take(2 * SB * y.H * 2);
     y.off_y = take(SB * y.O * 4);
-    y.off_dy = take(SB * y.O * 2);
+    y.off_dy = take(2 * SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
     y.off_loss_part = take((size_t)y.S * 64 * 4);   // 64 partial sums per step
     y.n_sync = 32 * (count_runs(p, y.S) + 1);   // 32 words (one 128-byte line) per persistent launch

@@ -14,6 +14,14 @@
 
 #include "mebptt.h"
 
+namespace mebptt {
+// The training step with a switch for the library-owned side stream (api.cu).
+int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, const void* W, const void* b,
+                    const void* W_out, const void* b_out, const void* x, const void* targets, const void* h0,
+                    const void* c0, void* workspace, size_t workspace_bytes, void* stream, float* loss, float* dW,
+                    float* db, float* dW_out, float* db_out, float* dx, int64_t* counters, bool side_stream);
+}
+
 namespace {
 
 // Every GPU that loads the library holds this array until the process exits.
@@ -56,7 +64,9 @@ extern "C" int mebptt_lstm_train_step_static(const mebptt_lstm_desc* desc, const
   if (rc != MEBPTT_OK) return rc;
   // The step itself clears everything in the workspace that has to start at zero (carried
   // gradients, step counters, status word), so what the previous call left behind is harmless.
-  return mebptt_lstm_train_step(desc, plan, W, b, W_out, b_out, x, targets, h0, c0, ws,
-                                (size_t)MEBPTT_STATIC_WORKSPACE_BYTES, stream, loss, dW, db, dW_out, db_out, dx,
-                                counters);
+  // Single-stream execution: the side stream of the ordinary entry point would have to be
+  // created on first use, and creating driver objects is a kind of allocation too.
+  return mebptt::train_step_impl(desc, plan, W, b, W_out, b_out, x, targets, h0, c0, ws,
+                                 (size_t)MEBPTT_STATIC_WORKSPACE_BYTES, stream, loss, dW, db, dW_out, db_out, dx,
+                                 counters, false);
 }

@@ -43,6 +43,9 @@ struct Plan;
 namespace tc {
 // Enqueues one training step on the tensor-core path; returns a status.  With dry = true
 // nothing is enqueued and the number of kernel launches is returned instead.
-int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry);
+// side_stream: run the weight-gradient GEMMs of a finished chunk on a stream owned by the library,
+// concurrently with the backward pass of the next chunk (joined back before the call's last kernel).
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
+                 bool side_stream);
 }  // namespace tc
 }  // namespace mebptt

@@ -34,6 +34,7 @@
 // come in the order t .. 1, so every sum runs in the same order under every plan.
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 #include <vector>
 
 #include "layout.hpp"
@@ -933,7 +934,40 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
 // ------------------------------------------------------------------------------------------
 // host: one training step
 // ------------------------------------------------------------------------------------------
-int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry) {
+// A second stream and four events per device, created on first use and kept for the life of the
+// process.  The side stream has lower priority than any stream a caller is likely to pass, so
+// that the cooperative kernels of the recurrence get their SMs first and the GEMMs fill the rest.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t ready[2] = {nullptr, nullptr};   // stages of parity p are complete (recorded on the caller's stream)
+  cudaEvent_t done[2] = {nullptr, nullptr};    // GEMMs reading parity p have finished (recorded on the side stream)
+  bool ok = false;
+};
+SideStream* side_stream_for_current_device() {
+  static std::mutex mu;
+  static SideStream table[64];
+  static bool tried[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  SideStream& t = table[dev];
+  if (!tried[dev]) {
+    tried[dev] = true;
+    int lo = 0, hi = 0;
+    cudaDeviceGetStreamPriorityRange(&lo, &hi);   // lo = numerically largest = least urgent
+    bool ok = cudaStreamCreateWithPriority(&t.stream, cudaStreamNonBlocking, lo) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i) {
+      ok = cudaEventCreateWithFlags(&t.ready[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&t.done[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) cudaGetLastError();
+    t.ok = ok;
+  }
+  return t.ok ? &t : nullptr;
+}
+
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
+                 bool side_stream) {
   const int B = y.B, H = y.H, I = y.I, O = y.O, S = y.S, G = 4 * H, K = I + H;
   const int BM = 64;  // batch rows per MMA tile (B <= 64)
   const int ncta = H / NU;
@@ -1001,7 +1035,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   const int fwd_smem = KBh * 4096 + KBh * 64 * 128 + 1024;
   const int GRf = 1;
   const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
-  CUtensorMap tm_h, tm_w, tm_dz, tm_wt, tm_dz_b, tm_wt_c;
+  CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
   if (!dry) {
     static const bool attrs = [] {
@@ -1015,7 +1049,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     const uint64_t rows = y.total / ((size_t)H * 2);
     bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, (uint32_t)(64 / GRf));
     ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, NG);
-    ok = ok && make_tmap_2d(&tm_dz, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, (uint32_t)BM);
+    for (int pb = 0; pb < 2; ++pb)
+      ok = ok && make_tmap_2d(&tm_dz[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64,
+                              (uint32_t)BM);
     ok = ok && make_tmap_2d(&tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
     if (!ok) return MEBPTT_ERR_UNSUPPORTED;
     // the clustered backward kernel, if the device can keep enough clusters resident
@@ -1042,7 +1078,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       break;
     }
     if (bwd_cs) {
-      ok = make_tmap_2d(&tm_dz_b, dz, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64, 64);
+      for (int pb = 0; pb < 2; ++pb)
+        ok = ok && make_tmap_2d(&tm_dz_b[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B,
+                                (uint64_t)G * 2, 64, 64);
       ok = ok && make_tmap_2d(&tm_wt_c, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, (uint32_t)(NU * bwd_cs));
       if (!ok) return MEBPTT_ERR_UNSUPPORTED;
     }
@@ -1071,13 +1109,17 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   int launch_id = 0;
   int rc = MEBPTT_OK;
   if (!dry && !cuda_ok(cudaGetLastError(), "set-up (memsets, tape upload, weight packing)")) rc = MEBPTT_ERR_CUDA;
-  auto gemm = [&](const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn, GemmOut out, int M,
-                  int N, int Kc) {
+  auto gemm_on = [&](cudaStream_t st, const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn,
+                     GemmOut out, int M, int N, int Kc) {
     ++launches;
     if (dry || rc != MEBPTT_OK) return;
-    rc = gemm_bf16(A, lda, amn, Bm, ldb, bmn, out, M, N, Kc, status, s);
+    rc = gemm_bf16(A, lda, amn, Bm, ldb, bmn, out, M, N, Kc, status, st);
     if (rc != MEBPTT_OK) cuda_ok(cudaErrorUnknown, "batched contraction");
   };
+  auto gemm = [&](const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn, GemmOut out, int M,
+                  int N, int Kc) { gemm_on(s, A, lda, amn, Bm, ldb, bmn, out, M, N, Kc); };
+  SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
+  bool side_busy[2] = {false, false};   // GEMMs reading the stages of this parity were put on the side stream
 
   size_t i = 0;
   while (i < nops && rc == MEBPTT_OK) {
@@ -1106,28 +1148,39 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     } else {
       // a backward run: consecutive operations k, k-1, ... inside one chunk of S time steps
       const int chunk = (first.k - 1) / S;
+      const int pb = chunk & 1;   // which copy of the stages this chunk uses
       size_t j = i + 1;
       while (j < nops && p->tape[j].kind == MEBPTT_OP_BWD && (p->tape[j].k - 1) / S == chunk) ++j;
       const int n = (int)(j - i);
       const int k_hi = first.k, k_lo = k_hi - n + 1;
       const int s_lo = (k_lo - 1) % S;
+      const size_t SB = (size_t)S * B;
+      __nv_bfloat16* dz_c = dz + (size_t)pb * SB * G;
+      __nv_bfloat16* hprev_c = hprev + (size_t)pb * SB * H;
+      __nv_bfloat16* hk_c = hk + (size_t)pb * SB * H;
+      __nv_bfloat16* dy_c = dyv + (size_t)pb * SB * O;
+      if (side && side_busy[pb]) {
+        // these stages were last read by GEMMs on the side stream (two chunks ago): wait for them
+        cudaStreamWaitEvent(s, side->done[pb], 0);
+        side_busy[pb] = false;
+      }
       launches += 3;
       if (!dry && rc == MEBPTT_OK) {
         const size_t block16 = (size_t)B * H * 2 / 16;
-        gather_states<<<dim3(16, n), 256, 0, s>>>(dops + i, n, ws, reinterpret_cast<uint4*>(hk),
-                                                  reinterpret_cast<uint4*>(hprev), S, block16);
+        gather_states<<<dim3(16, n), 256, 0, s>>>(dops + i, n, ws, reinterpret_cast<uint4*>(hk_c),
+                                                  reinterpret_cast<uint4*>(hprev_c), S, block16);
       }
       // readout of the n steps at once, then loss terms and dy, then the gradient entering h_k
-      gemm(hk + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
+      gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
            GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
       if (!dry && rc == MEBPTT_OK)
-        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(dops + i, yv, io.targets, dyv, loss_part, S, B, O);
-      gemm(dyv + (size_t)s_lo * B * O, O, false, woutT, O, false,
+        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(dops + i, yv, io.targets, dy_c, loss_part, S, B, O);
+      gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
-        BwdRunArgs a{dops + i, n, ws, dha, dz, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status, io.counters,
-                     B, H, S, off16(y.plane), off16(y.hsz)};
-        void* args[] = {(void*)(bwd_cs ? &tm_dz_b : &tm_dz), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
+        BwdRunArgs a{dops + i, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
+                     io.counters, B, H, S, off16(y.plane), off16(y.hsz)};
+        void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         if (bwd_cs) {
           cudaLaunchConfig_t cfg = {};
           cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
@@ -1147,25 +1200,41 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       }
       ++launch_id;
       if (k_lo == chunk * S + 1) {
-        // the chunk is complete: its weight gradients, summed over (s, b) in ascending order
+        // the chunk is complete: its weight gradients, summed over (s, b) in ascending order.
+        // They depend on nothing that follows, so they go to the side stream (in order: chunk c
+        // is accumulated before chunk c - 1) while the caller's stream moves on to the next chunk.
+        cudaStream_t gs = s;
+        if (side) {
+          cudaEventRecord(side->ready[pb], s);
+          cudaStreamWaitEvent(side->stream, side->ready[pb], 0);
+          gs = side->stream;
+        }
         const int steps = (int)((int64_t)(chunk + 1) * S <= y.t ? S : y.t - (int64_t)chunk * S);
         const int R = steps * B;
         const __nv_bfloat16* xc = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)chunk * S * B * I;
-        gemm(dz, G, true, xc, I, true, GemmOut{GemmOut::ACCUM_F32, io.dW, K, nullptr, H}, G, I, R);
-        gemm(dz, G, true, hprev, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW + I, K, nullptr, H}, G, H, R);
-        gemm(dyv, O, true, hk, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
+        gemm_on(gs, dz_c, G, true, xc, I, true, GemmOut{GemmOut::ACCUM_F32, io.dW, K, nullptr, H}, G, I, R);
+        gemm_on(gs, dz_c, G, true, hprev_c, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW + I, K, nullptr, H}, G, H, R);
+        gemm_on(gs, dy_c, O, true, hk_c, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
         launches += 2;
         if (!dry && rc == MEBPTT_OK) {
-          colsum_bf16<<<(G + 31) / 32, dim3(32, 8), 0, s>>>(dz, R, G, io.db, H);
-          colsum_bf16<<<(O + 31) / 32, dim3(32, 8), 0, s>>>(dyv, R, O, io.db_out, 0);
+          colsum_bf16<<<(G + 31) / 32, dim3(32, 8), 0, gs>>>(dz_c, R, G, io.db, H);
+          colsum_bf16<<<(O + 31) / 32, dim3(32, 8), 0, gs>>>(dy_c, R, O, io.db_out, 0);
         }
         if (want_dx)
-          gemm(dz, G, false, wpT_ih, G, false,
-               GemmOut{GemmOut::STORE_F32, io.dx + (size_t)chunk * S * B * I, I, nullptr, 0}, R, I, G);
+          gemm_on(gs, dz_c, G, false, wpT_ih, G, false,
+                  GemmOut{GemmOut::STORE_F32, io.dx + (size_t)chunk * S * B * I, I, nullptr, 0}, R, I, G);
+        if (side) {
+          cudaEventRecord(side->done[pb], side->stream);
+          side_busy[pb] = true;
+        }
       }
       i = j;
     }
   }
+  // everything the side stream did belongs to this call: join it before the last kernel
+  if (side)
+    for (int pb = 0; pb < 2; ++pb)
+      if (side_busy[pb]) cudaStreamWaitEvent(s, side->done[pb], 0);
   ++launches;
   if (!dry && rc == MEBPTT_OK) {
     finalize_tc<<<1, 32, 0, s>>>(loss_t, y.t, io.loss, io.counters, p->peak_units, status);
