@@ -1121,6 +1121,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
   bool side_busy[2] = {false, false};   // GEMMs reading the stages of this parity were put on the side stream
 
+  int zx_lo = 0, zx_hi = 0;   // time steps [zx_lo, zx_hi) whose input projections the Zx buffer holds
   size_t i = 0;
   while (i < nops && rc == MEBPTT_OK) {
     const mebptt_op& first = p->tape[i];
@@ -1132,12 +1133,20 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
              p->tape[j].k == p->tape[j - 1].k + 1 && p->tape[j].src == p->tape[j - 1].dst)
         ++j;
       const int n = (int)(j - i);
-      const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(first.k - 1) * B * I;
-      gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, n * B, G, I);
+      // Input projections Zx of the S steps from the start of the run on, unless the buffer already
+      // holds them: recomputation sweeps keep returning to the same stored state, so one
+      // projection serves many short runs.  (The values do not depend on how steps are batched.)
+      const int k0 = first.k;
+      if (!(k0 >= zx_lo && k0 + n <= zx_hi)) {
+        zx_lo = k0;
+        zx_hi = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
+        const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
+        gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
+      }
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
-        FwdRunArgs a{dops + i, n, ws, zx, sync + (size_t)launch_id * 32, status, io.counters, B, H, off16(y.plane),
-                     off16(y.hsz)};
+        FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 32, status,
+                     io.counters, B, H, off16(y.plane), off16(y.hsz)};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
         const void* fn = (const void*)fwd_run_kernel;
         if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(192), args, fwd_smem, s), "forward run launch"))
