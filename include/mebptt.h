@@ -43,7 +43,8 @@ extern "C" {
 #endif
 
 /* ---- enumerations ------------------------------------------------------------------ */
-enum { MEBPTT_HSM = 0, MEBPTT_ISM = 1, MEBPTT_MSM = 2 };
+enum { MEBPTT_HSM = 0, MEBPTT_ISM = 1, MEBPTT_MSM = 2,
+       MEBPTT_CHEN_SQRT = 3 /* reported by plans made with mebptt_plan_chen_sqrt; not accepted by mebptt_plan */ };
 
 enum {
   MEBPTT_OK = 0,
@@ -119,6 +120,17 @@ int mebptt_plan(int64_t t, int64_t m, int mode, mebptt_plan_t **out);
  * uses alpha only to size its slots.
  */
 int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_plan_t **out);
+
+/*
+ * Chen's sqrt(t) schedule (Section 2.2) as a plan for the same executor, for comparison with the
+ * DP policies (Sections 4.1, 4.2): segments of ceil(sqrt(t)) steps, hidden states memorised at the
+ * segment boundaries in one forward pass, then every internal state of one segment at a time.
+ * beta > 0: internal states are stored without their input hidden state (beta units each, the
+ * accounting of Section 4.2); beta = 0: with it (alpha units each).  The plan's m is set to the
+ * memory the schedule needs (mebptt_plan_peak_units); its cost is t plus the length of all
+ * segments but the last.  It carries no DP tables (mebptt_plan_tables returns NULL pointers).
+ */
+int mebptt_plan_chen_sqrt(int64_t t, int alpha, int beta, mebptt_plan_t **out);
 
 void mebptt_plan_free(mebptt_plan_t *plan);
 

@@ -136,6 +136,33 @@ def msm_tables(t_max: int, m_max: int, alpha: int, beta: int | None = None):
     return C, H, D1, D2
 
 
+# --------------------------------------------------------------------------------------
+# Section 2.2 / 4.2: Chen's sqrt(t) algorithm, for comparison
+# --------------------------------------------------------------------------------------
+def chen_sqrt(t: int, alpha: int, beta: int | None = None):
+    """Forward operations and memory units of Chen's sqrt(t) schedule.
+
+    The sequence is cut into segments of s = ceil(sqrt(t)) steps.  A first pass runs through all
+    segments but the last and keeps the hidden state at each boundary; then every segment, from
+    the last to the first, is run forward keeping all its internal states and backpropagated.
+    So every step is computed once, and every step outside the last segment a second time.
+    Memory (in hidden-state units, the start state included as in the mixed scheme): one unit per
+    kept boundary plus, at the worst moment, the internal states of one full segment (beta units
+    each when their input hidden states are left out as in Section 4.2, else alpha).
+    """
+    s = 1
+    while s * s < t:
+        s += 1
+    nseg = -(-t // s)
+    last = t - (nseg - 1) * s
+    forwards = t + (t - last)
+    per = beta if beta is not None else alpha
+    # while segment j is processed, the boundaries at its start and below are still kept
+    # (j of them, all nseg - 1 for the last segment) next to its internal states
+    peak = 1 + max(min(j, nseg - 1) + min(s, t - j * s) * per for j in range(nseg))
+    return {"forwards": forwards, "units": peak, "segment": s}
+
+
 def saturation_budget(mode: int, t: int, alpha: int = 4) -> int:
     """Smallest budget beyond which more memory cannot lower the cost (used to cap tables)."""
     if mode == MSM:

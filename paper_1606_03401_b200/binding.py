@@ -14,7 +14,7 @@ import numpy as np
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("MEBPTT_LIB") or os.path.join(_PKG, "libmebptt.so")   # MEBPTT_LIB: another build of the library
 
-MEBPTT_HSM, MEBPTT_ISM, MEBPTT_MSM = 0, 1, 2
+MEBPTT_HSM, MEBPTT_ISM, MEBPTT_MSM, MEBPTT_CHEN_SQRT = 0, 1, 2, 3
 MEBPTT_FP32, MEBPTT_TF32, MEBPTT_BF16 = 0, 1, 2
 MEBPTT_OK = 0
 MEBPTT_ERR_ARG, MEBPTT_ERR_BUDGET, MEBPTT_ERR_WORKSPACE, MEBPTT_ERR_UNSUPPORTED = -1, -2, -3, -4
@@ -56,6 +56,7 @@ _STEP_ARGS = [_descp, _vp] + [_vp] * 8 + [_vp, _sz, _vp] + [_vp] * 7
 _SIGS = {
     "mebptt_plan": (_i32, [_i64, _i64, _i32, C.POINTER(_vp)]),
     "mebptt_plan_ex": (_i32, [_i64, _i64, _i32, _i32, _i32, C.POINTER(_vp)]),
+    "mebptt_plan_chen_sqrt": (_i32, [_i64, _i32, _i32, C.POINTER(_vp)]),
     "mebptt_plan_free": (None, [_vp]),
     "mebptt_plan_cost": (_i64, [_vp]),
     "mebptt_plan_num_ops": (_i64, [_vp]),
@@ -145,8 +146,11 @@ class Plan:
                                       C.byref(td), C.byref(md)), "mebptt_plan_tables")
         shape = (td.value, md.value)
         n = shape[0] * shape[1]
-        out = {"C": np.ctypeslib.as_array(pc, shape=(n,)).reshape(shape).copy(),
-               "D": np.ctypeslib.as_array(pd, shape=(n,)).reshape(shape).copy()}
+        out = {}
+        if pc:
+            out["C"] = np.ctypeslib.as_array(pc, shape=(n,)).reshape(shape).copy()
+        if pd:
+            out["D"] = np.ctypeslib.as_array(pd, shape=(n,)).reshape(shape).copy()
         if pd2:
             out["D2"] = np.ctypeslib.as_array(pd2, shape=(n,)).reshape(shape).copy()
         if ph:
@@ -170,6 +174,12 @@ def mebptt_plan_ex(t: int, m: int, mode: int, alpha: int = 4, beta: int = 0) -> 
 
 
 MEBPTT_FLAG_NO_TENSOR_CORES = 1
+
+
+def mebptt_plan_chen_sqrt(t: int, alpha: int = 4, beta: int = 3) -> Plan:
+    h = _vp()
+    _check(lib.mebptt_plan_chen_sqrt(t, alpha, beta, C.byref(h)), "mebptt_plan_chen_sqrt")
+    return Plan(h)
 
 
 def make_desc(layers, input, hidden, readout, batch, t, dtype, want_dx=0, flags=0) -> mebptt_lstm_desc:

@@ -320,6 +320,67 @@ struct Emitter {
 
 }  // namespace
 
+// Chen's sqrt(t) schedule (Section 2.2) as a tape for the same executor: cut the sequence into
+// segments of s = ceil(sqrt(t)) steps; one forward pass memorises the hidden state at every
+// segment boundary; then, from the last segment to the first, run forward through the segment
+// memorising every internal state (the last segment does this on its first visit) and
+// backpropagate through them.  Section 4.1 notes that this is one (suboptimal) policy of the
+// mixed scheme; Section 4.2 counts its memory with the input hidden states left out (beta units
+// per internal state), which is what beta > 0 selects here.
+int build_chen_plan(int64_t t, int alpha, int beta, Plan** out) {
+  if (!out) return MEBPTT_ERR_ARG;
+  *out = nullptr;
+  if (t < 1 || t > (int64_t)1 << 24) return MEBPTT_ERR_ARG;
+  if (alpha < 2 || alpha > 64 || beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
+  Plan* p = new (std::nothrow) Plan();
+  if (!p) return MEBPTT_ERR_OOM;
+  p->t = t; p->mode = MEBPTT_CHEN_SQRT; p->alpha = alpha; p->beta = beta;
+  try {
+    int64_t s = 1;
+    while (s * s < t) ++s;
+    const int64_t nseg = (t + s - 1) / s;
+    const int u = beta > 0 ? beta : alpha;
+    const int fmt = beta > 0 ? MEBPTT_FMT_INTERNAL_NOINPUT : MEBPTT_FMT_INTERNAL;
+    p->m = (int64_t)1 << 40;  // no budget while emitting; set to the peak below
+    Emitter e(*p);
+    int32_t loc = MEBPTT_LOC_INIT;
+    for (int64_t j = 0; j + 1 < nseg; ++j) {
+      const int32_t slot = (int32_t)e.top;
+      e.grow(1, 1);
+      e.sweep(j * s, s, loc, slot, MEBPTT_FMT_HIDDEN);
+      loc = slot;
+    }
+    std::vector<int32_t> slots, prevs;
+    for (int64_t j = nseg - 1; j >= 0; --j) {
+      const int64_t start = j * s, len = std::min<int64_t>(s, t - start);
+      int32_t prev = (j == 0) ? (int32_t)MEBPTT_LOC_INIT : (int32_t)(j - 1);
+      slots.clear(); prevs.clear();
+      for (int64_t i = 1; i <= len; ++i) {
+        const int32_t slot = (int32_t)e.top;
+        e.grow(u, u);
+        e.fwd(start + i, prev, slot, fmt);
+        slots.push_back(slot); prevs.push_back(prev);
+        prev = slot;
+      }
+      for (int64_t i = len; i >= 1; --i) {
+        e.bwd(start + i, slots[(size_t)i - 1], fmt, beta > 0 ? prevs[(size_t)i - 1] : 0);
+        e.shrink(u, u);
+      }
+      if (j > 0) e.shrink(1, 1);
+    }
+    p->cost = 0;
+    for (const mebptt_op& op : p->tape) p->cost += (op.kind == MEBPTT_OP_FWD);
+    p->m = p->peak_units;
+  } catch (const std::bad_alloc&) {
+    delete p;
+    return MEBPTT_ERR_OOM;
+  }
+  int rc = validate_plan(*p);
+  if (rc != MEBPTT_OK) { delete p; return rc; }
+  *out = p;
+  return MEBPTT_OK;
+}
+
 int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out) {
   if (!out) return MEBPTT_ERR_ARG;
   *out = nullptr;
@@ -434,6 +495,10 @@ int mebptt_plan(int64_t t, int64_t m, int mode, mebptt_plan_t** out) {
   return mebptt::build_plan(t, m, mode, 4, 0, reinterpret_cast<Plan**>(out));
 }
 
+int mebptt_plan_chen_sqrt(int64_t t, int alpha, int beta, mebptt_plan_t** out) {
+  return mebptt::build_chen_plan(t, alpha, beta, reinterpret_cast<Plan**>(out));
+}
+
 int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_plan_t** out) {
   return mebptt::build_plan(t, m, mode, alpha, beta, reinterpret_cast<Plan**>(out));
 }
@@ -456,8 +521,8 @@ int mebptt_plan_tables(const mebptt_plan_t* plan, const int64_t** C, const int32
                        const int32_t** D2, const uint8_t** H, int64_t* t_dim, int64_t* m_dim) {
   if (!plan) return MEBPTT_ERR_ARG;
   const Plan* p = P_(plan);
-  if (C) *C = p->C.data();
-  if (D) *D = p->D.data();
+  if (C) *C = p->C.empty() ? nullptr : p->C.data();
+  if (D) *D = p->D.empty() ? nullptr : p->D.data();
   if (D2) *D2 = p->D2.empty() ? nullptr : p->D2.data();
   if (H) *H = p->H.empty() ? nullptr : p->H.data();
   if (t_dim) *t_dim = p->t + 1;

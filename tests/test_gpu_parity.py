@@ -214,3 +214,16 @@ def test_c3_full_size_headline_budget(H):
         res = dp.run(plan)
         assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
         assert_bit_identical(res, full)
+
+
+@pytest.mark.parametrize("base,kw", [("c1", dict()), ("c2", dict(t=70))])
+def test_chen_sqrt_plan_gives_the_same_gradients(H, base, kw):
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg(base, **kw)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    full = dp.run(dp.full_memory_plan())
+    for beta in (0, 3):
+        plan = B.mebptt_plan_chen_sqrt(cfg.t, 4, beta)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][2] == plan.peak_units and res["counters"][3] == 0
+        assert_bit_identical(res, full, want_dx=True)

@@ -178,3 +178,20 @@ def test_train_step_argument_errors_need_no_gpu():
     st = B.lib.mebptt_slot_copy(None, None, 16, None)
     assert st == B.MEBPTT_ERR_ARG
     assert B.mebptt_strerror(B.MEBPTT_ERR_BUDGET).startswith("memory budget")
+
+
+@pytest.mark.parametrize("beta", [0, 3])
+def test_chen_sqrt_schedule(beta):
+    """Chen's sqrt(t) schedule as a tape: cost and memory as the oracle derives them from the
+    description of Section 2.2, and never cheaper than the DP at the same memory (Section 4.1)."""
+    for t in (1, 2, 3, 7, 10, 17, 64, 100, 256, 1000):
+        plan = B.mebptt_plan_chen_sqrt(t, 4, beta)
+        ref = P.chen_sqrt(t, 4, beta or None)
+        assert plan.mode == B.MEBPTT_CHEN_SQRT
+        assert plan.cost == ref["forwards"] and plan.peak_units == ref["units"] == plan.m
+        assert plan.validate() == B.MEBPTT_OK
+        assert _replay(plan) == plan.cost
+        assert P.cost(P.MSM, t, plan.peak_units, 4, beta or None) <= plan.cost
+        assert "C" not in plan.tables()
+    # two forward operations per step on average, at most (Section 2.2)
+    assert B.mebptt_plan_chen_sqrt(1000, 4, 3).cost <= 2 * 1000
