@@ -227,3 +227,38 @@ def test_chen_sqrt_plan_gives_the_same_gradients(H, base, kw):
         res = dp.run(plan)
         assert res["counters"][0] == plan.cost and res["counters"][2] == plan.peak_units and res["counters"][3] == 0
         assert_bit_identical(res, full, want_dx=True)
+
+
+def test_c4_shape_truncated_ism_versus_msm(H):
+    """Config 4's layer sizes (I256 H1024 B32, float32 storage) on a shortened sequence: ISM with
+    m internal states against MSM with alpha * m hidden-state units, as the paper compares them."""
+    cfg = _cfg("c4", t=48)
+    dp = H.DeviceProblem(cfg)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, "tf32")
+    for mode, m in [("ism", 5), ("msm", 20)]:
+        plan = dp.plan(mode, m)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][3] == 0
+        assert_bit_identical(res, full)
+    assert dp.plan("msm", 20).cost <= dp.plan("ism", 5).cost      # Section 3.6
+
+
+def test_c5_shape_truncated_two_layers_byte_budget(H):
+    """Config 5's layer sizes (two layers, I1024 H2048 B128, bf16) on a very short sequence, with
+    the budget given in bytes and converted to hidden-state units."""
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg("c5", t=6)
+    dp = H.DeviceProblem(cfg)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert_close_to_oracle(full, ref, "bf16")
+    unit = B.mebptt_lstm_unit_bytes(dp.desc)
+    assert unit == 2 * 128 * 2048 * 6
+    m = B.mebptt_budget_bytes_to_units(dp.desc, 16 << 20)         # 16 MiB -> 5 units
+    assert m == (16 << 20) // unit == 5
+    plan = dp.plan("msm", m)
+    res = dp.run(plan)
+    assert res["counters"][0] == plan.cost and res["counters"][2] <= m
+    assert_bit_identical(res, full)
