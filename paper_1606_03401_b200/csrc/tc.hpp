@@ -28,6 +28,11 @@ struct StepPtrs {
   char* ws;
   float *loss, *dW, *db, *dW_out, *db_out, *dx;
   int64_t* counters;
+  // optional: the targets still lie in host memory at `targets_host`; the step copies them to
+  // `targets` on a copy stream while the forward pass runs and waits for them before the first
+  // backward run
+  const void* targets_host = nullptr;
+  size_t targets_bytes = 0;
 };
 
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
@@ -47,5 +52,10 @@ namespace tc {
 // concurrently with the backward pass of the next chunk (joined back before the call's last kernel).
 int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
                  bool side_stream);
+
+// Enqueues the host-to-device copy of the targets on the library's copy stream, ordered after
+// everything already in `s`, and returns the event that marks its completion (nullptr if the
+// side streams are unavailable: the caller then copies on `s`).
+cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s);
 }  // namespace tc
 }  // namespace mebptt

@@ -941,6 +941,8 @@ struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t ready[2] = {nullptr, nullptr};   // stages of parity p are complete (recorded on the caller's stream)
   cudaEvent_t done[2] = {nullptr, nullptr};    // GEMMs reading parity p have finished (recorded on the side stream)
+  cudaStream_t copy = nullptr;                 // host-to-device copies that overlap the forward pass
+  cudaEvent_t copy_from = nullptr, copy_done = nullptr;
   bool ok = false;
 };
 SideStream* side_stream_for_current_device() {
@@ -960,10 +962,23 @@ SideStream* side_stream_for_current_device() {
       ok = cudaEventCreateWithFlags(&t.ready[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&t.done[i], cudaEventDisableTiming) == cudaSuccess;
     }
+    ok = ok && cudaStreamCreateWithFlags(&t.copy, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&t.copy_from, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&t.copy_done, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) cudaGetLastError();
     t.ok = ok;
   }
   return t.ok ? &t : nullptr;
+}
+
+cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s) {
+  SideStream* side = side_stream_for_current_device();
+  if (!side) return nullptr;
+  cudaEventRecord(side->copy_from, s);            // the previous step on `s` may still read dst
+  cudaStreamWaitEvent(side->copy, side->copy_from, 0);
+  cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, side->copy);
+  cudaEventRecord(side->copy_done, side->copy);
+  return side->copy_done;
 }
 
 int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
@@ -1105,6 +1120,14 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
                                  reinterpret_cast<const uint4*>(io.c0), (size_t)B * H * 4 / 16);
   }
   launches += 3;
+  // The targets, if they are still on the host: requested after every other host-to-device copy of
+  // this step (the copy engine serves requests in order), on a stream of their own.
+  cudaEvent_t targets_ready = nullptr;
+  if (!dry && io.targets_host) {
+    targets_ready = copy_targets_async(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, s);
+    if (!targets_ready)
+      cudaMemcpyAsync(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, cudaMemcpyHostToDevice, s);
+  }
 
   int launch_id = 0;
   int rc = MEBPTT_OK;
@@ -1121,6 +1144,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
   bool side_busy[2] = {false, false};   // GEMMs reading the stages of this parity were put on the side stream
 
+  bool targets_waited = false;
   int zx_lo = 0, zx_hi = 0;   // time steps [zx_lo, zx_hi) whose input projections the Zx buffer holds
   size_t i = 0;
   while (i < nops && rc == MEBPTT_OK) {
@@ -1156,6 +1180,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       i = j;
     } else {
       // a backward run: consecutive operations k, k-1, ... inside one chunk of S time steps
+      if (targets_ready && !targets_waited) {
+        cudaStreamWaitEvent(s, targets_ready, 0);   // the targets were copied beside the forward pass
+        targets_waited = true;
+      }
       const int chunk = (first.k - 1) / S;
       const int pb = chunk & 1;   // which copy of the stages this chunk uses
       size_t j = i + 1;
