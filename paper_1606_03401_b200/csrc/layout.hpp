@@ -13,6 +13,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <vector>
 
 #include "mebptt.h"
 #include "plan.hpp"
@@ -46,7 +47,7 @@ struct Layout {
   // tensor-core path: packed weights, staging of S consecutive time steps, control
   int S = 0;             // time steps per staged chunk
   size_t off_wp_ih = 0, off_wp_hh = 0, off_wpT_hh = 0, off_wpT_ih = 0, off_bias_p = 0, off_woutT = 0;
-  size_t off_zx = 0, off_hprev = 0, off_hk = 0, off_y = 0;
+  size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
@@ -103,25 +104,63 @@ inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.rec = y.rec_in + y.unit;
 }
 
-// Number of persistent-kernel launches the tensor-core executor makes for a plan: forward runs
-// are cut into pieces of at most S consecutive operations, backward runs at chunk boundaries.
-inline size_t count_runs(const Plan* p, int S) {
-  size_t runs = 0, i = 0;
+// The tensor-core executor cuts the tape into work items:
+//   FWD   a run of consecutive forward operations, each starting from the state the previous one
+//         wrote, at most S of them (one persistent launch);
+//   BWD   a run of consecutive backward operations inside one chunk of S time steps;
+//   LEAF  n >= 2 consecutive leaves of the recursion -- FWD(k -> working core), BWD(k),
+//         FWD(k-1 -> working core), BWD(k-1), ... -- whose forward operations each start from a
+//         memorised state, inside one chunk.  Their forward operations do not depend on one another,
+//         so they are computed together by batched GEMMs instead of step by step.
+struct WorkItem {
+  enum Kind { FWD, BWD, LEAF } kind;
+  size_t i;   // first tape entry
+  int n;      // operations (FWD, BWD) or leaves (LEAF: 2 n tape entries)
+};
+inline bool is_leaf_at(const Plan* p, size_t i) {
   const size_t n = p->tape.size();
+  if (i + 1 >= n) return false;
+  const mebptt_op& f = p->tape[i];
+  const mebptt_op& b = p->tape[i + 1];
+  if (f.kind != MEBPTT_OP_FWD || b.kind != MEBPTT_OP_BWD) return false;
+  if (f.dst != MEBPTT_LOC_CORE || b.src != MEBPTT_LOC_CORE || f.k != b.k) return false;
+  if (f.src == MEBPTT_LOC_CORE) return false;
+  // a leaf proper: not the last step of a longer sweep
+  if (i > 0 && p->tape[i - 1].kind == MEBPTT_OP_FWD && p->tape[i - 1].dst == f.src && p->tape[i - 1].k == f.k - 1)
+    return false;
+  return true;
+}
+inline std::vector<WorkItem> work_items(const Plan* p, int S) {
+  std::vector<WorkItem> items;
+  const size_t n = p->tape.size();
+  size_t i = 0;
   while (i < n) {
+    if (is_leaf_at(p, i)) {
+      const int chunk = (p->tape[i].k - 1) / S;
+      int leaves = 1;
+      while (is_leaf_at(p, i + 2 * (size_t)leaves) && p->tape[i + 2 * (size_t)leaves].k == p->tape[i].k - leaves &&
+             (p->tape[i + 2 * (size_t)leaves].k - 1) / S == chunk)
+        ++leaves;
+      if (leaves >= 2) {
+        items.push_back(WorkItem{WorkItem::LEAF, i, leaves});
+        i += 2 * (size_t)leaves;
+        continue;
+      }
+    }
     size_t j = i + 1;
     if (p->tape[i].kind == MEBPTT_OP_FWD) {
       while (j < n && j - i < (size_t)S && p->tape[j].kind == MEBPTT_OP_FWD && p->tape[j].k == p->tape[j - 1].k + 1 &&
              p->tape[j].src == p->tape[j - 1].dst)
         ++j;
+      items.push_back(WorkItem{WorkItem::FWD, i, (int)(j - i)});
     } else {
       const int chunk = (p->tape[i].k - 1) / S;
       while (j < n && p->tape[j].kind == MEBPTT_OP_BWD && (p->tape[j].k - 1) / S == chunk) ++j;
+      items.push_back(WorkItem{WorkItem::BWD, i, (int)(j - i)});
     }
-    ++runs;
     i = j;
   }
-  return runs;
+  return items;
 }
 
 inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y) {
@@ -164,10 +203,11 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_y = take(SB * y.O * 4);
     y.off_dy = take(2 * SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
+    y.off_zleaf = take(SB * G * 4);   // pre-activations of a batch of leaves
     y.off_loss_part = take((size_t)y.S * 64 * 4);   // 64 partial sums per step
-    y.n_sync = 32 * (count_runs(p, y.S) + 1);   // 32 words (one 128-byte line) per persistent launch
+    y.n_sync = 32 * (work_items(p, y.S).size() + 1);   // 32 words (one 128-byte line) per persistent launch
     y.off_sync = take(y.n_sync * 4);
-    y.tape_bytes = (size_t)p->tape.size() * 32;
+    y.tape_bytes = (size_t)p->tape.size() * 32 * 2;   // the tape, and the compacted entries of leaf batches
     y.off_tape = take(y.tape_bytes);
     y.off_status = take(256);
   }

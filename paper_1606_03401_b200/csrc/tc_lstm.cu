@@ -357,6 +357,7 @@ struct BwdRunArgs {
   int64_t* counters;
   int B, H, S;
   uint32_t plane16, hsz16;
+  const float* zleaf;      // leaf batch: [S][B][4H] pre-activations z_k (gate columns permuted); NULL otherwise
 };
 
 // What the gate derivatives of one batch row and 8 hidden units read from memory at one step: the
@@ -366,24 +367,57 @@ struct GateInputs {
   uint4 qi, qf, qg, qo;
   float4 t0, t1, p0, p1, d0, d1;
 };
-__device__ __forceinline__ GateInputs load_gate_inputs(const BwdRunArgs& a, const DevOp& op, int sidx, size_t e0,
-                                                       size_t pl) {
+__device__ __forceinline__ GateInputs load_gate_inputs(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int cta,
+                                                       size_t e0, size_t pl) {
   GateInputs in;
   const char* ws = a.ws;
   const float* dha = a.dha + ((size_t)sidx * a.B) * a.H + e0;
   in.d0 = *reinterpret_cast<const float4*>(dha);
   in.d1 = *reinterpret_cast<const float4*>(dha + 4);
+  const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
+  in.p0 = *reinterpret_cast<const float4*>(cpp);
+  in.p1 = *reinterpret_cast<const float4*>(cpp + 4);
+  if (a.zleaf) {
+    // A leaf of the recursion: no internal state was stored.  Its forward operation is redone
+    // here from the pre-activations, with exactly the arithmetic of the forward kernel (gates
+    // rounded to bfloat16 as they would have been stored, c_k from the unrounded gates).
+    const float4* zp = reinterpret_cast<const float4*>(a.zleaf + ((size_t)sidx * a.B + b) * 4 * a.H + (size_t)cta * NG);
+    const float cp[NU] = {in.p0.x, in.p0.y, in.p0.z, in.p0.w, in.p1.x, in.p1.y, in.p1.z, in.p1.w};
+    float ct[NU];
+    uint32_t gi[4], gf[4], gg[4], go[4];
+#pragma unroll
+    for (int u = 0; u < NU; u += 2) {
+      float iv[2], fv[2], gv[2], ov[2];
+#pragma unroll
+      for (int d = 0; d < 2; ++d) {
+        const float4 z = zp[u + d];
+        iv[d] = sigmoid_fast(z.x);
+        fv[d] = sigmoid_fast(z.y);
+        gv[d] = tanh_fast(z.z);
+        ov[d] = sigmoid_fast(z.w);
+        ct[u + d] = fmaf(fv[d], cp[u + d], iv[d] * gv[d]);
+      }
+      gi[u / 2] = pack_bf16x2(iv[0], iv[1]);
+      gf[u / 2] = pack_bf16x2(fv[0], fv[1]);
+      gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
+      go[u / 2] = pack_bf16x2(ov[0], ov[1]);
+    }
+    in.qi = make_uint4(gi[0], gi[1], gi[2], gi[3]);
+    in.qf = make_uint4(gf[0], gf[1], gf[2], gf[3]);
+    in.qg = make_uint4(gg[0], gg[1], gg[2], gg[3]);
+    in.qo = make_uint4(go[0], go[1], go[2], go[3]);
+    in.t0 = make_float4(ct[0], ct[1], ct[2], ct[3]);
+    in.t1 = make_float4(ct[4], ct[5], ct[6], ct[7]);
+    return in;
+  }
   const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
   in.qi = *reinterpret_cast<const uint4*>(g);
   in.qf = *reinterpret_cast<const uint4*>(g + pl);
   in.qg = *reinterpret_cast<const uint4*>(g + 2 * pl);
   in.qo = *reinterpret_cast<const uint4*>(g + 3 * pl);
   const float* ctp = reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0;
-  const float* cpp = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0;
   in.t0 = *reinterpret_cast<const float4*>(ctp);
   in.t1 = *reinterpret_cast<const float4*>(ctp + 4);
-  in.p0 = *reinterpret_cast<const float4*>(cpp);
-  in.p1 = *reinterpret_cast<const float4*>(cpp + 4);
   return in;
 }
 
@@ -425,7 +459,7 @@ __device__ __forceinline__ void compute_gates(const BwdRunArgs& a, const GateInp
 
 __device__ __forceinline__ void backward_gates(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int cta,
                                                size_t e0, size_t pl, const float (&dh)[NU], float (&dc)[NU]) {
-  const GateInputs in = load_gate_inputs(a, op, sidx, e0, pl);
+  const GateInputs in = load_gate_inputs(a, op, sidx, b, cta, e0, pl);
   compute_gates(a, in, sidx, b, cta, dh, dc);
 }
 
@@ -773,7 +807,7 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
     };
 
     GateInputs gin;
-    if (owner) gin = load_gate_inputs(a, a.ops[0], (a.ops[0].k - 1) % a.S, e0, pl);
+    if (owner) gin = load_gate_inputs(a, a.ops[0], (a.ops[0].k - 1) % a.S, b, cta, e0, pl);
     for (int i = 0; i < a.n; ++i) {
       const DevOp op = a.ops[i];
       const int sidx = (op.k - 1) % a.S;
@@ -783,7 +817,7 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
       if (tid == 0) red_release_add(a.sync, 1u);
       // the inputs of the next (earlier) step do not depend on the recurrence: fetch them while the
       // exchange of this step is in flight
-      if (owner && i + 1 < a.n) gin = load_gate_inputs(a, a.ops[i + 1], (a.ops[i + 1].k - 1) % a.S, e0, pl);
+      if (owner && i + 1 < a.n) gin = load_gate_inputs(a, a.ops[i + 1], (a.ops[i + 1].k - 1) % a.S, b, cta, e0, pl);
     }
     reduce_partials(a.n - 1);
     if (owner && !failed) {
@@ -848,9 +882,30 @@ __global__ void gather_states(const DevOp* ops, int n, const char* ws, uint4* hk
   uint4* dk = hk + (size_t)sidx * block16;
   uint4* dp = hprev + (size_t)sidx * block16;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < block16; e += (size_t)gridDim.x * blockDim.x) {
-    dk[e] = src_k[e];
+    if (hk) dk[e] = src_k[e];   // leaf batches have no stored h_k: leaf_forward writes it
     dp[e] = src_p[e];
   }
+}
+
+// The forward operations of a batch of leaves, after the batched GEMMs have produced their
+// pre-activations z (row block (k-1) % S, gate columns 4 u + q): h_k = o tanh(f c_{k-1} + i g),
+// written to the staging chunk for the readout and the weight gradients.  Same arithmetic as the
+// epilogue of the forward run kernel; the gates themselves are redone by the backward kernel.
+__global__ void leaf_forward(const DevOp* ops, int n, const char* ws, const float* z, __nv_bfloat16* hk, int S, int B,
+                             int H, int64_t* counters) {
+  const DevOp op = ops[blockIdx.y];
+  const int sidx = (op.k - 1) % S;
+  const size_t bh = (size_t)B * H;
+  const float* cprev = reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16);
+  const float4* zs = reinterpret_cast<const float4*>(z + (size_t)sidx * bh * 4);
+  __nv_bfloat16* out = hk + (size_t)sidx * bh;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < bh; e += (size_t)gridDim.x * blockDim.x) {
+    const float4 zz = zs[e];   // (b, u): columns 4 u .. 4 u + 3 of row b
+    const float iv = sigmoid_fast(zz.x), fv = sigmoid_fast(zz.y), gv = tanh_fast(zz.z), ov = sigmoid_fast(zz.w);
+    const float c = fmaf(fv, cprev[e], iv * gv);
+    out[e] = __float2bfloat16_rn(ov * tanh_fast(c));
+  }
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) counters[0] += n;
 }
 
 // y (float32, readout with bias) -> dy = 2 (y - target) / (B O) in bfloat16, and LOSS_PARTS
@@ -1001,9 +1056,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     }
   };
   const size_t nops = p->tape.size();
+  const std::vector<WorkItem> items = work_items(p, S);
   std::vector<DevOp> dev;
   if (!dry) {
-    dev.resize(nops);
+    dev.resize(2 * nops);   // [0, nops): the tape; [nops, 2 nops): the compacted leaves of leaf batches
     for (size_t i = 0; i < nops; ++i) {
       const mebptt_op& op = p->tape[i];
       DevOp d{};
@@ -1023,6 +1079,17 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         d.gates = off16(rec + y.rec_gates);
       }
       dev[i] = d;
+    }
+    for (const WorkItem& it : items) {
+      if (it.kind != WorkItem::LEAF) continue;
+      for (int j = 0; j < it.n; ++j) {
+        const mebptt_op& f = p->tape[it.i + 2 * (size_t)j];   // the leaf's forward operation
+        const size_t src = block_off(f.src);
+        DevOp d{};
+        d.k = f.k;
+        d.h_src = off16(src); d.c_src = off16(src + y.hsz);   // state k-1, memorised
+        dev[nops + it.i + (size_t)j] = d;
+      }
     }
   }
   const DevOp* dops = reinterpret_cast<const DevOp*>(at(y.off_tape));
@@ -1109,7 +1176,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
     cudaMemsetAsync(sync, 0, y.n_sync * 4, s);
     cudaMemsetAsync(status, 0, 256, s);
-    cudaMemcpyAsync(at(y.off_tape), dev.data(), nops * sizeof(DevOp), cudaMemcpyHostToDevice, s);
+    cudaMemcpyAsync(at(y.off_tape), dev.data(), 2 * nops * sizeof(DevOp), cudaMemcpyHostToDevice, s);
     pack_weights<<<592, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
                                      reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh,
                                      wpT_ih, bias_p, woutT);
@@ -1146,17 +1213,15 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
 
   bool targets_waited = false;
   int zx_lo = 0, zx_hi = 0;   // time steps [zx_lo, zx_hi) whose input projections the Zx buffer holds
-  size_t i = 0;
-  while (i < nops && rc == MEBPTT_OK) {
+  float* zleaf = reinterpret_cast<float*>(at(y.off_zleaf));
+  for (size_t item = 0; item < items.size() && rc == MEBPTT_OK; ++item) {
+    const WorkItem& wi = items[item];
+    const size_t i = wi.i;
     const mebptt_op& first = p->tape[i];
-    if (first.kind == MEBPTT_OP_FWD) {
+    if (wi.kind == WorkItem::FWD) {
       // a forward run: consecutive operations k, k+1, ... each starting from the state the
       // previous one wrote; at most S of them per launch
-      size_t j = i + 1;
-      while (j < nops && j - i < (size_t)S && p->tape[j].kind == MEBPTT_OP_FWD &&
-             p->tape[j].k == p->tape[j - 1].k + 1 && p->tape[j].src == p->tape[j - 1].dst)
-        ++j;
-      const int n = (int)(j - i);
+      const int n = wi.n;
       // Input projections Zx of the S steps from the start of the run on, unless the buffer already
       // holds them: recomputation sweeps keep returning to the same stored state, so one
       // projection serves many short runs.  (The values do not depend on how steps are batched.)
@@ -1177,18 +1242,18 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
           rc = MEBPTT_ERR_CUDA;
       }
       ++launch_id;
-      i = j;
     } else {
-      // a backward run: consecutive operations k, k-1, ... inside one chunk of S time steps
+      // a backward run: consecutive operations k, k-1, ... inside one chunk of S time steps --
+      // or a batch of leaves, whose forward operations are done here as well, all at once
+      const bool leaf = wi.kind == WorkItem::LEAF;
+      const DevOp* bops = leaf ? dops + nops + i : dops + i;
       if (targets_ready && !targets_waited) {
         cudaStreamWaitEvent(s, targets_ready, 0);   // the targets were copied beside the forward pass
         targets_waited = true;
       }
       const int chunk = (first.k - 1) / S;
       const int pb = chunk & 1;   // which copy of the stages this chunk uses
-      size_t j = i + 1;
-      while (j < nops && p->tape[j].kind == MEBPTT_OP_BWD && (p->tape[j].k - 1) / S == chunk) ++j;
-      const int n = (int)(j - i);
+      const int n = wi.n;
       const int k_hi = first.k, k_lo = k_hi - n + 1;
       const int s_lo = (k_lo - 1) % S;
       const size_t SB = (size_t)S * B;
@@ -1204,19 +1269,31 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       launches += 3;
       if (!dry && rc == MEBPTT_OK) {
         const size_t block16 = (size_t)B * H * 2 / 16;
-        gather_states<<<dim3(16, n), 256, 0, s>>>(dops + i, n, ws, reinterpret_cast<uint4*>(hk_c),
+        gather_states<<<dim3(16, n), 256, 0, s>>>(bops, n, ws, leaf ? nullptr : reinterpret_cast<uint4*>(hk_c),
                                                   reinterpret_cast<uint4*>(hprev_c), S, block16);
+      }
+      if (leaf) {
+        // z_k = W_ih x_k + b + W_hh h_{k-1} for the n leaves at once (their h_{k-1} are all
+        // memorised), then h_k; the gates are redone inside the backward kernel
+        const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k_lo - 1) * B * I;
+        gemm(xk, I, false, wp_ih, I, false,
+             GemmOut{GemmOut::STORE_F32, zleaf + (size_t)s_lo * B * G, G, bias_p, 0}, n * B, G, I);
+        gemm(hprev_c + (size_t)s_lo * B * H, H, false, wp_hh, H, false,
+             GemmOut{GemmOut::ACCUM_F32, zleaf + (size_t)s_lo * B * G, G, nullptr, 0}, n * B, G, H);
+        ++launches;
+        if (!dry && rc == MEBPTT_OK)
+          leaf_forward<<<dim3(32, n), 256, 0, s>>>(bops, n, ws, zleaf, hk_c, S, B, H, io.counters);
       }
       // readout of the n steps at once, then loss terms and dy, then the gradient entering h_k
       gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
            GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
       if (!dry && rc == MEBPTT_OK)
-        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(dops + i, yv, io.targets, dy_c, loss_part, S, B, O);
+        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(bops, yv, io.targets, dy_c, loss_part, S, B, O);
       gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
-        BwdRunArgs a{dops + i, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
-                     io.counters, B, H, S, off16(y.plane), off16(y.hsz)};
+        BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
+                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         if (bwd_cs) {
           cudaLaunchConfig_t cfg = {};
@@ -1265,7 +1342,6 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
           side_busy[pb] = true;
         }
       }
-      i = j;
     }
   }
   // everything the side stream did belongs to this call: join it before the last kernel
