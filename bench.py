@@ -9,8 +9,9 @@ the plan dictates over the workload's t time steps.  One JSON line is printed by
 
 * value / ms_per_step: device-resident inputs, CUDA events around each step.
 * e2e: the same step through the host-buffer entry point, host<->device copies included.
-* roofline: the gate contraction of the forward operation, flops per operation over the
-  measured duration of one forward operation (see --help of the fields in the design doc).
+* roofline: the dominant kernel (a run of forward operations), timed launch by launch with CUDA
+  events on the launching stream in three extra steps: flops of the recurrent gate contraction
+  per launch over the mean launch duration, against the measured bf16 peak.
 * cpu_baseline: the oracle on the host cores, on a truncated sequence.
 * budgets: the other budgets of the workload, with the time ratio against full-memory BPTT
   beside the paper's model (C/t + 2) / 3.
@@ -306,21 +307,50 @@ def main():
         flops_fwd_op += 2 * cfg.batch * K_l * 4 * cfg.hidden
     pk = peaks()
     extra_ops = plan.cost - cfg.t
-    if extra_ops > 0 and ms > ms_full:
-        fwd_op_ms = (ms - ms_full) / extra_ops
-    else:
-        fwd_op_ms = None
-    achieved = flops_fwd_op / (fwd_op_ms * 1e-3) / 1e12 if fwd_op_ms else None
     peak_tf = pk["bf16_tflops_sustained"] if cfg.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2.0
-    roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": (achieved / peak_tf) if achieved else None,
-                "traffic": FWD_RUN_DRAM_BYTES_PER_OP_C3 if (cfg.name == "c3" and cfg.input == 1024) else None,
-                "kernel": "forward operation (gate contraction + fused cell update)",
-                "traffic_note": "DRAM bytes per forward operation of fwd_run_kernel alone (ncu, 16-step launch); "
-                                "the batched input projection's traffic is not included",
-                "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
-                       f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
-                       + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}
+    runs = None
+    if B.mebptt_lstm_launch_count(dp.desc, plan) and cfg.dtype == "bf16":
+        # the dominant kernel, timed launch by launch with CUDA events on the launching stream
+        # (separate steps: the event pairs cost stream time, so the whole-step figure above has none)
+        B.mebptt_lstm_run_times()
+        dp.desc.flags |= B.MEBPTT_FLAG_TIME_RUNS
+        for _ in range(3):
+            flush.fill_(1)
+            dp.enqueue(plan)
+        torch.cuda.synchronize()
+        dp.desc.flags &= ~B.MEBPTT_FLAG_TIME_RUNS
+        runs = B.mebptt_lstm_run_times()
+        if runs["forward"][1] == 0:
+            runs = None     # the shape runs on the CUDA-core path
+    if runs:
+        f_ms, f_n, f_ops = runs["forward"]
+        b_ms, b_n, b_ops = runs["backward"]
+        flops_rec = 2 * cfg.batch * cfg.hidden * 4 * cfg.hidden      # the recurrent contraction of one operation
+        achieved = f_ops * flops_rec / (f_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": achieved / peak_tf,
+                    "traffic": FWD_RUN_DRAM_BYTES_PER_OP_C3 * (f_ops / f_n) if (cfg.name == "c3" and cfg.input == 1024) else None,
+                    "kernel": "fwd_run_kernel (a run of forward operations: recurrent gate contraction + cell update)",
+                    "launches": f_n // 3, "ops_per_launch": f_ops / f_n, "us_per_launch": f_ms * 1e3 / f_n,
+                    "us_per_op": f_ms * 1e3 / f_ops,
+                    "share_of_step": (f_ms / 3) / ms,
+                    "backward_runs": {"kernel": "bwd_run_cluster_kernel", "launches": b_n // 3,
+                                      "us_per_op": b_ms * 1e3 / max(1, b_ops), "share_of_step": (b_ms / 3) / ms},
+                    "traffic_note": "DRAM bytes per launch = bytes per operation (ncu, 16-operation launch) x mean operations per launch",
+                    "how": f"CUDA events around each launch, 3 steps; {flops_rec} flops per operation x operations per launch / mean "
+                           f"launch duration; peak = bf16 sustained ({pk['source']})"}
+    else:
+        if extra_ops > 0 and ms > ms_full:
+            fwd_op_ms = (ms - ms_full) / extra_ops
+        else:
+            fwd_op_ms = None
+        achieved = flops_fwd_op / (fwd_op_ms * 1e-3) / 1e12 if fwd_op_ms else None
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": (achieved / peak_tf) if achieved else None, "traffic": None,
+                    "kernel": "forward operation on the CUDA-core path (gate contraction + cell update, several launches)",
+                    "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
+                           f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
+                           + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}
 
     budgets = []
     if not args.no_budgets and rank == 0 or (not args.no_budgets and world > 1):

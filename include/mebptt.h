@@ -209,6 +209,11 @@ typedef struct {
 /* Run on the CUDA-core kernels even where the tensor-core kernels cover the shape (the two
  * paths round differently; results are deterministic within each). */
 enum { MEBPTT_FLAG_NO_TENSOR_CORES = 1 };
+/* Measurement aid: bracket every launch of the two persistent kernels of the tensor-core path
+ * (forward runs, backward runs) with a pair of CUDA events on the caller's stream, to be
+ * collected by mebptt_lstm_run_times.  Each pair costs a few microseconds of stream time, so a
+ * step that is timed as a whole should not set it.  Ignored by the CUDA-core path. */
+enum { MEBPTT_FLAG_TIME_RUNS = 2 };
 
 /* Bytes of one hidden-state unit (all layers) for this descriptor; 0 on a bad descriptor. */
 size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc *desc);
@@ -311,6 +316,18 @@ int mebptt_lstm_train_step_static(const mebptt_lstm_desc *desc, const mebptt_pla
  * place and does not call this.
  */
 int mebptt_slot_copy(void *dst, const void *src, size_t bytes, void *stream);
+
+/*
+ * Collects the event pairs recorded on the current device by steps whose descriptor carried
+ * MEBPTT_FLAG_TIME_RUNS since the last call: waits for each pair, and returns per class
+ * (index 0: forward runs, one launch executes a run of consecutive forward operations of
+ * Algorithm 1-3's "execute" steps; index 1: backward runs) the summed elapsed milliseconds,
+ * the number of launches and the number of operations they executed.  ms, launches and ops are
+ * host arrays of 2 elements.  Returns MEBPTT_OK, MEBPTT_ERR_ARG on a null pointer, or
+ * MEBPTT_ERR_CUDA if an event could not be read (the other pairs are still returned).  The
+ * paper has no counterpart; it serves the per-kernel figures of a benchmark.
+ */
+int mebptt_lstm_run_times(double *ms, int64_t *launches, int64_t *ops);
 
 /*
  * The batched contraction the training step uses for everything that is off the recurrence

@@ -81,6 +81,7 @@ _SIGS = {
     "mebptt_lstm_train_step": (_i32, _STEP_ARGS),
     "mebptt_lstm_train_step_host": (_i32, _STEP_ARGS),
     "mebptt_lstm_train_step_static": (_i32, [_descp, _vp] + [_vp] * 8 + [_vp] + [_vp] * 7),
+    "mebptt_lstm_run_times": (_i32, [C.POINTER(C.c_double), C.POINTER(_i64), C.POINTER(_i64)]),
     "mebptt_slot_copy": (_i32, [_vp, _vp, _sz, _vp]),
     "mebptt_gemm_bf16": (_i32, [_vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "mebptt_strerror": (C.c_char_p, [_i32]),
@@ -174,6 +175,7 @@ def mebptt_plan_ex(t: int, m: int, mode: int, alpha: int = 4, beta: int = 0) -> 
 
 
 MEBPTT_FLAG_NO_TENSOR_CORES = 1
+MEBPTT_FLAG_TIME_RUNS = 2
 
 
 def mebptt_plan_chen_sqrt(t: int, alpha: int = 4, beta: int = 3) -> Plan:
@@ -263,6 +265,13 @@ def mebptt_lstm_train_step_static(desc, plan, W, b, W_out, b_out, x, targets, h0
         _ptr(h0), _ptr(c0), stream, _ptr(loss), _ptr(dW), _ptr(db), _ptr(dW_out), _ptr(db_out), _ptr(dx),
         _ptr(counters))
     _check(st, "mebptt_lstm_train_step_static")
+
+
+def mebptt_lstm_run_times() -> dict:
+    """{"forward": (ms, launches, ops), "backward": (...)} of the steps run with MEBPTT_FLAG_TIME_RUNS."""
+    ms, n, ops = (C.c_double * 2)(), (_i64 * 2)(), (_i64 * 2)()
+    _check(lib.mebptt_lstm_run_times(ms, n, ops), "mebptt_lstm_run_times")
+    return {"forward": (ms[0], n[0], ops[0]), "backward": (ms[1], n[1], ops[1])}
 
 
 def mebptt_gemm_bf16(A, lda, a_major, Bm, ldb, b_major, Cm, ldc, accumulate, bias, M, N, K, status=None,

@@ -227,6 +227,7 @@ int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, con
   StepIO io{(const char*)W, (const char*)W_out, (const char*)x, (const char*)h0,
             (const float*)b, (const float*)b_out, (const float*)targets, (const float*)c0,
             (char*)workspace, loss, dW, db, dW_out, db_out, dx, counters};
+  io.time_runs = (desc->flags & MEBPTT_FLAG_TIME_RUNS) != 0;
   return run_step(desc, p, y, io, (cudaStream_t)stream, side_stream);
 }
 }  // namespace mebptt
@@ -290,6 +291,7 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
             (float*)(ws + g.db_out), desc->want_dx ? (float*)(ws + g.dx) : nullptr,
             (int64_t*)(ws + g.counters)};
   if (late_targets) { io.targets_host = targets; io.targets_bytes = g.ntargets; }
+  io.time_runs = (desc->flags & MEBPTT_FLAG_TIME_RUNS) != 0;
   rc = run_step(desc, p, y, io, s);
   if (rc != MEBPTT_OK) return rc;
   cudaMemcpyAsync(loss, ws + g.loss, 4, cudaMemcpyDeviceToHost, s);
@@ -301,6 +303,8 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
   cudaMemcpyAsync(counters, ws + g.counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost, s);
   return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
 }
+
+int mebptt_lstm_run_times(double* ms, int64_t* launches, int64_t* ops) { return tc::run_times(ms, launches, ops); }
 
 int mebptt_gemm_bf16(const void* A, int64_t lda, int a_major, const void* B, int64_t ldb, int b_major, float* C,
                      int64_t ldc, int accumulate, const float* bias, int64_t M, int64_t N, int64_t K, int* status,

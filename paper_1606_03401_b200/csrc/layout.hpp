@@ -73,7 +73,7 @@ inline bool valid_desc(const mebptt_lstm_desc* d) {
   if (d->input > (1 << 16) || d->hidden > (1 << 16) || d->readout > (1 << 16) || d->batch > (1 << 16)) return false;
   if (d->dtype != MEBPTT_FP32 && d->dtype != MEBPTT_TF32 && d->dtype != MEBPTT_BF16) return false;
   if (d->want_dx != 0 && d->want_dx != 1) return false;
-  if (d->flags & ~MEBPTT_FLAG_NO_TENSOR_CORES) return false;
+  if (d->flags & ~(MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_TIME_RUNS)) return false;
   return true;
 }
 

@@ -33,6 +33,8 @@ struct StepPtrs {
   // backward run
   const void* targets_host = nullptr;
   size_t targets_bytes = 0;
+  // bracket every launch of the two persistent kernels with CUDA events (collected by run_times)
+  bool time_runs = false;
 };
 
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
@@ -57,5 +59,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
 // everything already in `s`, and returns the event that marks its completion (nullptr if the
 // side streams are unavailable: the caller then copies on `s`).
 cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s);
+
+// Waits for the event pairs recorded on the current device by steps run with time_runs, adds up
+// elapsed milliseconds, launches and operations per class (0: forward runs, 1: backward runs)
+// and forgets them.
+int run_times(double* ms, int64_t* launches, int64_t* ops);
 }  // namespace tc
 }  // namespace mebptt

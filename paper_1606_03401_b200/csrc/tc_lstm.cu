@@ -1026,6 +1026,63 @@ SideStream* side_stream_for_current_device() {
   return t.ok ? &t : nullptr;
 }
 
+// Event pairs around the launches of the persistent kernels, per device; filled only by steps
+// that ask for it.
+struct RunTimer {
+  struct Span { cudaEvent_t e0, e1; int cls; int ops; };
+  std::mutex mu;
+  std::vector<Span> spans;
+  std::vector<cudaEvent_t> pool;
+  cudaEvent_t get() {
+    if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return e;
+  }
+};
+RunTimer* run_timer_for_current_device() {
+  static RunTimer table[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  return &table[dev];
+}
+// Records the start of a span on `s`; the returned index is closed by span_end.
+int span_begin(RunTimer* rt, int cls, int ops, cudaStream_t s) {
+  if (!rt) return -1;
+  std::lock_guard<std::mutex> lock(rt->mu);
+  RunTimer::Span sp{rt->get(), rt->get(), cls, ops};
+  if (!sp.e0 || !sp.e1) return -1;
+  cudaEventRecord(sp.e0, s);
+  rt->spans.push_back(sp);
+  return (int)rt->spans.size() - 1;
+}
+void span_end(RunTimer* rt, int idx, cudaStream_t s) {
+  if (!rt || idx < 0) return;
+  std::lock_guard<std::mutex> lock(rt->mu);
+  cudaEventRecord(rt->spans[idx].e1, s);
+}
+
+int run_times(double* ms, int64_t* launches, int64_t* ops) {
+  RunTimer* rt = run_timer_for_current_device();
+  if (!rt || !ms || !launches || !ops) return MEBPTT_ERR_ARG;
+  for (int c = 0; c < 2; ++c) { ms[c] = 0.0; launches[c] = 0; ops[c] = 0; }
+  std::lock_guard<std::mutex> lock(rt->mu);
+  int rc = MEBPTT_OK;
+  for (const RunTimer::Span& sp : rt->spans) {
+    float t = 0.f;
+    if (cudaEventSynchronize(sp.e1) != cudaSuccess || cudaEventElapsedTime(&t, sp.e0, sp.e1) != cudaSuccess) {
+      cudaGetLastError();
+      rc = MEBPTT_ERR_CUDA;
+    } else {
+      ms[sp.cls] += t; launches[sp.cls] += 1; ops[sp.cls] += sp.ops;
+    }
+    rt->pool.push_back(sp.e0);
+    rt->pool.push_back(sp.e1);
+  }
+  rt->spans.clear();
+  return rc;
+}
+
 cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s) {
   SideStream* side = side_stream_for_current_device();
   if (!side) return nullptr;
@@ -1211,6 +1268,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
   bool side_busy[2] = {false, false};   // GEMMs reading the stages of this parity were put on the side stream
 
+  RunTimer* timer = (!dry && io.time_runs) ? run_timer_for_current_device() : nullptr;
   bool targets_waited = false;
   int zx_lo = 0, zx_hi = 0;   // time steps [zx_lo, zx_hi) whose input projections the Zx buffer holds
   float* zleaf = reinterpret_cast<float*>(at(y.off_zleaf));
@@ -1238,8 +1296,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
                      io.counters, B, H, off16(y.plane), off16(y.hsz)};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
         const void* fn = (const void*)fwd_run_kernel;
+        const int span = span_begin(timer, 0, n, s);
         if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(192), args, fwd_smem, s), "forward run launch"))
           rc = MEBPTT_ERR_CUDA;
+        span_end(timer, span, s);
       }
       ++launch_id;
     } else {
@@ -1295,6 +1355,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
                      io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
+        const int span = span_begin(timer, 1, n, s);
         if (bwd_cs) {
           cudaLaunchConfig_t cfg = {};
           cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
@@ -1311,6 +1372,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
           if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, bwd_smem, s), "backward run launch"))
             rc = MEBPTT_ERR_CUDA;
         }
+        span_end(timer, span, s);
       }
       ++launch_id;
       if (k_lo == chunk * S + 1) {

@@ -184,6 +184,29 @@ def test_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
         assert rel_l2(full[k], other[k]) < 1e-2, k
 
 
+def test_run_times_count_every_backward_operation_and_change_no_result(H):
+    """The per-launch event timing: results stay bit-identical, every backward operation is inside
+    a timed backward run, forward runs hold at most C(t, m) operations (leaves of the recursion
+    are computed in batches outside them), and the collection clears itself."""
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg("c2", input=128, hidden=128, batch=32, t=45, readout=64)
+    dp = H.DeviceProblem(cfg)
+    plan = dp.plan("hsm", 4)
+    plain = dp.run(plan)
+    B.mebptt_lstm_run_times()
+    dp.desc.flags |= B.MEBPTT_FLAG_TIME_RUNS
+    timed = dp.run(plan)
+    dp.desc.flags &= ~B.MEBPTT_FLAG_TIME_RUNS
+    assert_bit_identical(timed, plain)
+    r = B.mebptt_lstm_run_times()
+    f_ms, f_n, f_ops = r["forward"]
+    b_ms, b_n, b_ops = r["backward"]
+    assert b_ops == cfg.t and 0 < b_n <= cfg.t and b_ms > 0
+    assert 0 < f_ops <= plan.cost and 0 < f_n <= f_ops and f_ms > 0
+    again = B.mebptt_lstm_run_times()
+    assert again["forward"][1] == 0 and again["backward"][1] == 0
+
+
 def test_c2_full_size_every_budget(H):
     """Config 2 as timed: I512 H512 B64 t256 bf16, HSM and ISM at m = 16, 64, 256."""
     cfg = synth.CONFIGS["c2"]
