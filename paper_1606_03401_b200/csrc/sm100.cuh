@@ -17,6 +17,14 @@ namespace sm100 {
 
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls; with back-off this is on the order of a second
 
+// Programmatic dependent launch.  A kernel launched with the stream-serialization attribute may
+// become resident while its predecessor in the stream still runs; grid_dep_wait returns once the
+// predecessor has completed and its writes are visible, so no global memory is touched before
+// it.  grid_dep_launch lets the successor become resident once every CTA of this grid has
+// called it (or exited).  Both are no-ops for kernels launched without the attribute.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

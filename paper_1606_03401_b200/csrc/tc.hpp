@@ -39,9 +39,11 @@ struct StepPtrs {
 
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
 // [m][k]; lda / ldb are row strides in elements (multiples of 8).  `status` (device, nullable)
-// receives MEBPTT_ERR_TIMEOUT if a bounded wait expires.
+// receives MEBPTT_ERR_TIMEOUT if a bounded wait expires.  early: the kernel may become resident
+// before the previous kernel of the stream has finished (it still waits for it before touching
+// memory).
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s);
+              int M, int N, int K, int* status, cudaStream_t s, bool early = true);
 
 }  // namespace tc
 

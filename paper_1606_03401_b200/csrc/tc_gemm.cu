@@ -18,6 +18,7 @@
 // tcgen05.ld (warp w owns TMEM lanes 32w .. 32w+31 = tile rows) and write the tile.
 // Out-of-range parts of a tile are zero-filled by TMA on the way in and masked on the way out.
 // The sum over k runs in one fixed order, so results do not depend on how callers batch steps.
+#include "launch.hpp"
 #include "sm100.cuh"
 #include "tc.hpp"
 #include "tmap.hpp"
@@ -60,6 +61,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
+  grid_dep_wait();     // operands (and, when accumulating, C) come from the kernels before this one
+  grid_dep_launch();
 
   if (warp == 0 && lane == 0) {
     // ---- producer -----------------------------------------------------------------------
@@ -249,7 +252,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
 }  // namespace
 
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s) {
+              int M, int N, int K, int* status, cudaStream_t s, bool early) {
   if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
   CUtensorMap ta, tb;
   // K-major: tensor is [M][K], box 64 (k) x 128 rows.  MN-major: tensor is [K][M], box 64 (m) x 64 rows.
@@ -272,11 +275,11 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   // loop.  Grids of at most one wave: 6 stages, more loads in flight per CTA to hide their latency.
   const int stages = (grid.x * grid.y <= 148) ? MAX_STAGES : 3;
   const int GEMM_SMEM = gemm_smem(stages);
-  if (a_mn && b_mn) gemm_bf16_kernel<true, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
-  else if (!a_mn && !b_mn) gemm_bf16_kernel<false, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
-  else if (a_mn) gemm_bf16_kernel<true, false><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
-  else gemm_bf16_kernel<false, true><<<grid, 128, GEMM_SMEM, s>>>(ta, tb, out, M, N, K, stages, status);
-  return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+  auto* fn = a_mn ? (b_mn ? gemm_bf16_kernel<true, true> : gemm_bf16_kernel<true, false>)
+                  : (b_mn ? gemm_bf16_kernel<false, true> : gemm_bf16_kernel<false, false>);
+  const cudaError_t e = launch_on(early, fn, grid, dim3(128), (size_t)GEMM_SMEM, s, ta, tb, out, M, N, K, stages, status);
+  if (e != cudaSuccess) cudaGetLastError();
+  return e == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
 }
 
 }  // namespace tc

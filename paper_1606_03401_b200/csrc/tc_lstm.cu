@@ -37,6 +37,7 @@
 #include <mutex>
 #include <vector>
 
+#include "launch.hpp"
 #include "layout.hpp"
 #include "sm100.cuh"
 #include "tc.hpp"
@@ -157,6 +158,7 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
   const uint32_t row_bytes = (uint32_t)a.H * 2u;
+  grid_dep_wait();   // everything above touched no global memory; everything below may
 
   if (warp == 4) {
     // ---- producer: lane 0 watches the step counter, then lanes 0 .. NQ-1 each request one block
@@ -183,6 +185,7 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
         for (int kb = kb0; kb < kb1; ++kb) tma_load_2d(tiles + kb * A_TILE, &tm_h, kb * 64, row, &full[0][q]);
       }
       armed = i;
+      if (i == a.n - 1 && lane == 0) grid_dep_launch();   // last step under way: the next kernel may set itself up
       __syncwarp();
     }
     if (failed && lane == 0) {
@@ -496,6 +499,8 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
+  grid_dep_wait();
+  if (tid == 0) grid_dep_launch();
 
   if (is_p) {
     mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 1024u);
@@ -669,6 +674,7 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
   cluster_sync();                          // peers arrive on each other's barriers: all must be initialised
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
+  grid_dep_wait();
 
   if (warp == 4) {
     // ---- producer: this CTA's K-slice of dz_k, all of it in flight at once; lane 0 watches the
@@ -702,6 +708,7 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
           tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
       }
       armed = i;
+      if (i == a.n - 1 && lane == 0) grid_dep_launch();
       __syncwarp();
     }
     if (failed && lane == 0) {
@@ -846,6 +853,8 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
 __global__ void pack_weights(const __nv_bfloat16* W, const float* bias, const __nv_bfloat16* W_out, int I, int H,
                              int O, __nv_bfloat16* wp_ih, __nv_bfloat16* wp_hh, __nv_bfloat16* wpT_hh,
                              __nv_bfloat16* wpT_ih, float* bias_p, __nv_bfloat16* woutT) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int G = 4 * H, K = I + H;
   const size_t nW = (size_t)G * K;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -875,6 +884,8 @@ __global__ void pack_weights(const __nv_bfloat16* W, const float* bias, const __
 // into the staging chunk (row block (k-1) % S), 16 bytes per thread per access.
 __global__ void gather_states(const DevOp* ops, int n, const char* ws, uint4* hk, uint4* hprev, int S,
                               size_t block16) {  // block16: B*H*2/16
+  grid_dep_wait();
+  grid_dep_launch();
   const DevOp op = ops[blockIdx.y];
   const int sidx = (op.k - 1) % S;
   const uint4* src_k = reinterpret_cast<const uint4*>(ws + (size_t)op.h_dst * 16);
@@ -893,6 +904,8 @@ __global__ void gather_states(const DevOp* ops, int n, const char* ws, uint4* hk
 // epilogue of the forward run kernel; the gates themselves are redone by the backward kernel.
 __global__ void leaf_forward(const DevOp* ops, int n, const char* ws, const float* z, __nv_bfloat16* hk, int S, int B,
                              int H, int64_t* counters) {
+  grid_dep_wait();
+  grid_dep_launch();
   const DevOp op = ops[blockIdx.y];
   const int sidx = (op.k - 1) % S;
   const size_t bh = (size_t)B * H;
@@ -913,6 +926,8 @@ __global__ void leaf_forward(const DevOp* ops, int n, const char* ws, const floa
 __global__ void loss_dy(const DevOp* ops, const float* y, const float* targets, __nv_bfloat16* dy, float* loss_part,
                         int S, int B, int O) {
   __shared__ float red[256];
+  grid_dep_wait();
+  grid_dep_launch();
   const DevOp op = ops[blockIdx.y];
   const int sidx = (op.k - 1) % S;
   const size_t n = (size_t)B * O;
@@ -942,6 +957,8 @@ __global__ void loss_dy(const DevOp* ops, const float* y, const float* targets, 
 // the eight partial sums are added in the order g = 0 .. 7.
 __global__ void colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out, int perm_h) {
   __shared__ float part[8][33];
+  grid_dep_wait();
+  grid_dep_launch();
   const int n = blockIdx.x * 32 + threadIdx.x, g = threadIdx.y;
   float s = 0.f;
   if (n < N)
@@ -959,6 +976,8 @@ __global__ void colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out,
 
 __global__ void finalize_tc(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
                             const int* status) {
+  grid_dep_wait();
+  grid_dep_launch();
   float s = 0.f;
   for (int64_t i = threadIdx.x; i < t; i += 32) s += loss_t[i];
   for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
@@ -970,6 +989,8 @@ __global__ void finalize_tc(const float* loss_t, int64_t t, float* loss, int64_t
 }
 
 __global__ void copy16_tc(uint4* dst, const uint4* src, size_t n) {
+  grid_dep_wait();
+  grid_dep_launch();
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = src[i];
 }
@@ -1234,14 +1255,13 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     cudaMemsetAsync(sync, 0, y.n_sync * 4, s);
     cudaMemsetAsync(status, 0, 256, s);
     cudaMemcpyAsync(at(y.off_tape), dev.data(), 2 * nops * sizeof(DevOp), cudaMemcpyHostToDevice, s);
-    pack_weights<<<592, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
-                                     reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh,
-                                     wpT_ih, bias_p, woutT);
+    launch_pdl(pack_weights, dim3(592), dim3(256), 0, s, reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
+               reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh, wpT_ih, bias_p, woutT);
     // Peek of the initial state: the caller's (h0, c0) as a hidden block inside the workspace
-    copy16_tc<<<64, 256, 0, s>>>(reinterpret_cast<uint4*>(at(y.off_init)), reinterpret_cast<const uint4*>(io.h0),
-                                 (size_t)B * H * 2 / 16);
-    copy16_tc<<<64, 256, 0, s>>>(reinterpret_cast<uint4*>(at(y.off_init + y.hsz)),
-                                 reinterpret_cast<const uint4*>(io.c0), (size_t)B * H * 4 / 16);
+    launch_pdl(copy16_tc, dim3(64), dim3(256), 0, s, reinterpret_cast<uint4*>(at(y.off_init)),
+               reinterpret_cast<const uint4*>(io.h0), (size_t)B * H * 2 / 16);
+    launch_pdl(copy16_tc, dim3(64), dim3(256), 0, s, reinterpret_cast<uint4*>(at(y.off_init + y.hsz)),
+               reinterpret_cast<const uint4*>(io.c0), (size_t)B * H * 4 / 16);
   }
   launches += 3;
   // The targets, if they are still on the host: requested after every other host-to-device copy of
@@ -1260,7 +1280,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
                      GemmOut out, int M, int N, int Kc) {
     ++launches;
     if (dry || rc != MEBPTT_OK) return;
-    rc = gemm_bf16(A, lda, amn, Bm, ldb, bmn, out, M, N, Kc, status, st);
+    // on the side stream a kernel that is resident early only takes room from the one that runs
+    rc = gemm_bf16(A, lda, amn, Bm, ldb, bmn, out, M, N, Kc, status, st, st == s);
     if (rc != MEBPTT_OK) cuda_ok(cudaErrorUnknown, "batched contraction");
   };
   auto gemm = [&](const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn, GemmOut out, int M,
@@ -1297,7 +1318,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
         const void* fn = (const void*)fwd_run_kernel;
         const int span = span_begin(timer, 0, n, s);
-        if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(192), args, fwd_smem, s), "forward run launch"))
+        if (!cuda_ok(launch_coop(fn, ncta, 192, fwd_smem, s, args, 1), "forward run launch"))
           rc = MEBPTT_ERR_CUDA;
         span_end(timer, span, s);
       }
@@ -1329,8 +1350,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       launches += 3;
       if (!dry && rc == MEBPTT_OK) {
         const size_t block16 = (size_t)B * H * 2 / 16;
-        gather_states<<<dim3(16, n), 256, 0, s>>>(bops, n, ws, leaf ? nullptr : reinterpret_cast<uint4*>(hk_c),
-                                                  reinterpret_cast<uint4*>(hprev_c), S, block16);
+        launch_pdl(gather_states, dim3(16, n), dim3(256), 0, s, bops, n, ws,
+                   leaf ? nullptr : reinterpret_cast<uint4*>(hk_c), reinterpret_cast<uint4*>(hprev_c), S, block16);
       }
       if (leaf) {
         // z_k = W_ih x_k + b + W_hh h_{k-1} for the n leaves at once (their h_{k-1} are all
@@ -1342,13 +1363,13 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
              GemmOut{GemmOut::ACCUM_F32, zleaf + (size_t)s_lo * B * G, G, nullptr, 0}, n * B, G, H);
         ++launches;
         if (!dry && rc == MEBPTT_OK)
-          leaf_forward<<<dim3(32, n), 256, 0, s>>>(bops, n, ws, zleaf, hk_c, S, B, H, io.counters);
+          launch_pdl(leaf_forward, dim3(32, n), dim3(256), 0, s, bops, n, ws, zleaf, hk_c, S, B, H, io.counters);
       }
       // readout of the n steps at once, then loss terms and dy, then the gradient entering h_k
       gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
            GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
       if (!dry && rc == MEBPTT_OK)
-        loss_dy<<<dim3(LOSS_PARTS, n), 256, 0, s>>>(bops, yv, io.targets, dy_c, loss_part, S, B, O);
+        launch_pdl(loss_dy, dim3(LOSS_PARTS, n), dim3(256), 0, s, bops, yv, io.targets, dy_c, loss_part, S, B, O);
       gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
@@ -1357,20 +1378,13 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         const int span = span_begin(timer, 1, n, s);
         if (bwd_cs) {
-          cudaLaunchConfig_t cfg = {};
-          cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = bwdc_smem; cfg.stream = s;
-          cudaLaunchAttribute at2[2];
-          at2[0].id = cudaLaunchAttributeClusterDimension;
-          at2[0].val.clusterDim.x = bwd_cs; at2[0].val.clusterDim.y = 1; at2[0].val.clusterDim.z = 1;
-          at2[1].id = cudaLaunchAttributeCooperative;
-          at2[1].val.cooperative = 1;
-          cfg.attrs = at2; cfg.numAttrs = 2;
           const void* fn = bwd_cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
-          if (!cuda_ok(cudaLaunchKernelExC(&cfg, fn, args), "backward run launch (clusters)")) rc = MEBPTT_ERR_CUDA;
+          // launched in plain stream order: early residency of a clustered grid measured no gain
+          if (!cuda_ok(launch_coop(fn, ncta, 192, bwdc_smem, s, args, bwd_cs, false), "backward run launch (clusters)"))
+            rc = MEBPTT_ERR_CUDA;
         } else {
           const void* fn = (const void*)bwd_run_kernel<64>;
-          if (!cuda_ok(cudaLaunchCooperativeKernel(fn, dim3(ncta), dim3(128), args, bwd_smem, s), "backward run launch"))
-            rc = MEBPTT_ERR_CUDA;
+          if (!cuda_ok(launch_coop(fn, ncta, 128, bwd_smem, s, args, 1), "backward run launch")) rc = MEBPTT_ERR_CUDA;
         }
         span_end(timer, span, s);
       }
@@ -1393,8 +1407,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         gemm_on(gs, dy_c, O, true, hk_c, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
         launches += 2;
         if (!dry && rc == MEBPTT_OK) {
-          colsum_bf16<<<(G + 31) / 32, dim3(32, 8), 0, gs>>>(dz_c, R, G, io.db, H);
-          colsum_bf16<<<(O + 31) / 32, dim3(32, 8), 0, gs>>>(dy_c, R, O, io.db_out, 0);
+          launch_on(gs == s, colsum_bf16, dim3((G + 31) / 32), dim3(32, 8), 0, gs, dz_c, R, G, io.db, H);
+          launch_on(gs == s, colsum_bf16, dim3((O + 31) / 32), dim3(32, 8), 0, gs, dy_c, R, O, io.db_out, 0);
         }
         if (want_dx)
           gemm_on(gs, dz_c, G, false, wpT_ih, G, false,
@@ -1412,7 +1426,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (side_busy[pb]) cudaStreamWaitEvent(s, side->done[pb], 0);
   ++launches;
   if (!dry && rc == MEBPTT_OK) {
-    finalize_tc<<<1, 32, 0, s>>>(loss_t, y.t, io.loss, io.counters, p->peak_units, status);
+    launch_pdl(finalize_tc, dim3(1), dim3(32), 0, s, loss_t, (int64_t)y.t, io.loss, io.counters, (int64_t)p->peak_units, status);
     if (!cuda_ok(cudaGetLastError(), "training step (last error)")) rc = MEBPTT_ERR_CUDA;
   }
   if (dry) return launches;
