@@ -11,7 +11,7 @@
 // is stored [k][m] (rows are contraction indices), which is how dz and the layer inputs lie in
 // memory for the weight gradient, so no transposed copies are made.
 //
-// One CTA computes one 128 x 128 tile.  A single thread feeds a 3- or 6-stage ring of 128-byte
+// One CTA computes one 128 x 128 tile (128 x 32 where C is short and wide: see gemm_bf16).  A single thread feeds a 3- or 6-stage ring of 128-byte
 // swizzled shared-memory tiles by TMA (64 contraction indices per stage); a single thread issues
 // tcgen05.mma (M = 128, N = 128, K = 16, four per stage) into a 128-column TMEM accumulator and
 // releases ring slots with tcgen05.commit; then all four warps read the accumulator with
@@ -30,14 +30,17 @@ namespace {
 
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128, BK = 64, MAX_STAGES = 6;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int gemm_smem(int stages) { return stages * STAGE_BYTES + 1024; }  // + slack to align the ring to 1024 B
+constexpr int BM = 128, BK = 64, MAX_STAGES = 6;
+constexpr int BN_WIDE = 128, BN_NARROW = 32;   // tile widths; narrow tiles spread a short-and-wide C over more SMs
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int gemm_smem(int stages, int bn) { return stages * (A_BYTES + bn * BK * 2) + 1024; }  // + slack to align the ring to 1024 B
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int BN = BN_WIDE>
 __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma,
                                                         const __grid_constant__ CUtensorMap tmb, GemmOut out,
                                                         int M, int N, int K, int STAGES, int* status) {
+  constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  static_assert(BN == BN_WIDE || (!A_MN && !B_MN), "narrow tiles exist for K-major operands only");
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], done;
   __shared__ uint32_t tmem_slot;
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
     tma_prefetch_desc(&tma);
     tma_prefetch_desc(&tmb);
   }
-  if (warp == 1) tmem_alloc(&tmem_slot, 128);
+  if (warp == 1) tmem_alloc(&tmem_slot, BN);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -123,7 +126,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
     // Float32 tiles whose rows can be written as aligned float4: each warp parks its 32 x 128
     // block of the accumulator in the (now idle) operand ring, then writes -- or adds to -- one
     // whole 512-byte row of C per instruction.  Everything else takes the per-thread path below.
-    const bool wide = out.kind != GemmOut::STORE_BF16 && (out.ld % 4 == 0) &&
+    const bool wide = BN == BN_WIDE && out.kind != GemmOut::STORE_BF16 && (out.ld % 4 == 0) &&
                       ((reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0) && (n0 % 4 == 0) &&
                       ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0);
     if (wide) {
@@ -246,7 +249,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
     for (int s = 0; s < STAGES; ++s) (void)mbar_wait(&full[s], 0);
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 128);
+  if (warp == 1) tmem_dealloc(tmem, BN);
 }
 
 }  // namespace
@@ -254,29 +257,38 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
               int M, int N, int K, int* status, cudaStream_t s, bool early) {
   if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
+  // A short-and-wide product over K-major operands (a few steps' worth of rows against a whole
+  // weight matrix) gives few 128-wide tiles, each streaming all of K through one SM: 32-wide tiles
+  // put four times as many SMs to work on the same bytes.
+  const int wide_tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
+  const bool narrow = !a_mn && !b_mn && wide_tiles <= 37 && N >= 2 * BN_NARROW;
+  const int BN = narrow ? BN_NARROW : BN_WIDE;
   CUtensorMap ta, tb;
-  // K-major: tensor is [M][K], box 64 (k) x 128 rows.  MN-major: tensor is [K][M], box 64 (m) x 64 rows.
+  // K-major: tensor is [M][K], box 64 (k) x tile rows.  MN-major: tensor is [K][M], box 64 (m) x 64 rows.
   bool ok = a_mn ? make_tmap_2d(&ta, A, 2, (uint64_t)M, (uint64_t)K, (uint64_t)lda * 2, 64, 64)
                  : make_tmap_2d(&ta, A, 2, (uint64_t)K, (uint64_t)M, (uint64_t)lda * 2, 64, 128);
   ok = ok && (b_mn ? make_tmap_2d(&tb, B, 2, (uint64_t)N, (uint64_t)K, (uint64_t)ldb * 2, 64, 64)
-                   : make_tmap_2d(&tb, B, 2, (uint64_t)K, (uint64_t)N, (uint64_t)ldb * 2, 64, 128));
+                   : make_tmap_2d(&tb, B, 2, (uint64_t)K, (uint64_t)N, (uint64_t)ldb * 2, 64, (uint32_t)BN));
   if (!ok) return MEBPTT_ERR_UNSUPPORTED;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
   static const bool attrs = [] {
-    const int most = gemm_smem(MAX_STAGES);
+    const int most = gemm_smem(MAX_STAGES, BN_WIDE);
     cudaFuncSetAttribute(gemm_bf16_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     cudaFuncSetAttribute(gemm_bf16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     cudaFuncSetAttribute(gemm_bf16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
     cudaFuncSetAttribute(gemm_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaFuncSetAttribute(gemm_bf16_kernel<false, false, BN_NARROW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         gemm_smem(MAX_STAGES, BN_NARROW));
     return true;
   }();
   (void)attrs;
   // Large grids: 3 stages, two CTAs per SM, so that one CTA's epilogue overlaps the other's main
   // loop.  Grids of at most one wave: 6 stages, more loads in flight per CTA to hide their latency.
   const int stages = (grid.x * grid.y <= 148) ? MAX_STAGES : 3;
-  const int GEMM_SMEM = gemm_smem(stages);
-  auto* fn = a_mn ? (b_mn ? gemm_bf16_kernel<true, true> : gemm_bf16_kernel<true, false>)
-                  : (b_mn ? gemm_bf16_kernel<false, true> : gemm_bf16_kernel<false, false>);
+  const int GEMM_SMEM = gemm_smem(stages, BN);
+  auto* fn = narrow ? gemm_bf16_kernel<false, false, BN_NARROW>
+             : a_mn ? (b_mn ? gemm_bf16_kernel<true, true> : gemm_bf16_kernel<true, false>)
+                    : (b_mn ? gemm_bf16_kernel<false, true> : gemm_bf16_kernel<false, false>);
   const cudaError_t e = launch_on(early, fn, grid, dim3(128), (size_t)GEMM_SMEM, s, ta, tb, out, M, N, K, stages, status);
   if (e != cudaSuccess) cudaGetLastError();
   return e == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;

@@ -59,3 +59,12 @@ def test_gemm_training_shapes():
     # input projection of 16 steps at config 3, and a weight-gradient chunk
     assert _run(1024, 4096, 1024, False, False, bias=True) < 1e-4
     assert _run(4096, 2048, 1024, True, True, accumulate=True) < 1e-4
+
+
+def test_gemm_short_and_wide_shapes():
+    # a short backward run at config 3: readout of one and two steps, pre-activations of two leaves
+    # (these take the 32-wide tiles)
+    assert _run(64, 1024, 1024, False, False, bias=True) < 1e-4
+    assert _run(128, 1024, 1024, False, False) < 1e-4
+    assert _run(128, 4096, 1024, False, False, accumulate=True) < 1e-4
+    assert _run(40, 264, 200, False, False, accumulate=True, bias=True, pad=8) < 1e-4
