@@ -86,6 +86,12 @@ inline bool tensor_path_supported(const mebptt_lstm_desc* d) {
          d->hidden <= 1024;
 }
 
+// Partial sums of the squared error per time step on the tensor-core path.  Where 32-row groups
+// of the readout tile stay inside one step (B % 32 == 0) the readout GEMM's epilogue forms them:
+// one per (32 batch rows, 32 readout columns).  Otherwise a separate kernel forms 64 per step.
+inline bool loss_fused(int B, int O) { return B % 32 == 0 && (B / 32) * ((O + 31) / 32) <= 256; }
+inline int loss_parts_per_step(int B, int O) { return loss_fused(B, O) ? (B / 32) * ((O + 31) / 32) : 64; }
+
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
   y.dtype = d->dtype; y.t = d->t;
@@ -204,7 +210,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_dy = take(2 * SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
     y.off_zleaf = take(SB * G * 4);   // pre-activations of a batch of leaves
-    y.off_loss_part = take((size_t)y.S * 64 * 4);   // 64 partial sums per step
+    y.off_loss_part = take((size_t)y.S * loss_parts_per_step(y.B, y.O) * 4);
     y.n_sync = 32 * (work_items(p, y.S).size() + 1);   // 32 words (one 128-byte line) per persistent launch
     y.off_sync = take(y.n_sync * 4);
     y.tape_bytes = (size_t)p->tape.size() * 32 * 2;   // the tape, and the compacted entries of leaf batches

@@ -13,12 +13,19 @@ namespace tc {
 
 // Where a GEMM tile goes.
 struct GemmOut {
-  enum Kind : int { STORE_F32 = 0, ACCUM_F32 = 1, STORE_BF16 = 2 };
+  enum Kind : int { STORE_F32 = 0, ACCUM_F32 = 1, STORE_BF16 = 2, LOSS_DY = 3 };
   int kind;
   void* ptr;          // [M][ld]
   int64_t ld;         // elements
   const float* bias;  // optional, per column, float32 outputs only
   int perm_h;         // > 0: tile row 4 u + q is written to row q * perm_h + u (undoes the gate permutation)
+  // LOSS_DY: the product (plus bias) is the readout y and is not stored.  With d = y - target[m][n],
+  // ptr receives dy = 2 d scale in bfloat16 and loss_part[(m / 32) * parts + n / 32] the sum of
+  // d * d * scale over that 32 x 32 block, in a fixed order (rows of M in groups of 32).
+  const float* target = nullptr;   // [M][ld]
+  float* loss_part = nullptr;
+  int parts = 0;                   // ceil(N / 32)
+  float scale = 0.f;
 };
 
 // Caller buffers of one training step (device pointers).

@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
     // Float32 tiles whose rows can be written as aligned float4: each warp parks its 32 x 128
     // block of the accumulator in the (now idle) operand ring, then writes -- or adds to -- one
     // whole 512-byte row of C per instruction.  Everything else takes the per-thread path below.
-    const bool wide = BN == BN_WIDE && out.kind != GemmOut::STORE_BF16 && (out.ld % 4 == 0) &&
+    const bool wide = BN == BN_WIDE && out.kind != GemmOut::STORE_BF16 && out.kind != GemmOut::LOSS_DY && (out.ld % 4 == 0) &&
                       ((reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0) && (n0 % 4 == 0) &&
                       ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0);
     if (wide) {
@@ -195,7 +195,50 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
       tmem_ld_wait();
       const int col0 = n0 + c * 32;
-      if (row < M) {
+      if (out.kind == GemmOut::LOSS_DY) {
+        // squared-error loss fused into the readout: this lane's row against its targets, columns in
+        // ascending order, then the 32 rows of the warp in a fixed butterfly order
+        float sq = 0.f;
+        if (row < M) {
+          const float* tp = out.target + (size_t)row * out.ld + col0;
+          __nv_bfloat16* dp = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row * out.ld + col0;
+          const float two = 2.f * out.scale;
+          if (col0 + 32 <= N && ((reinterpret_cast<uintptr_t>(tp) & 15) == 0) && ((reinterpret_cast<uintptr_t>(dp) & 15) == 0) &&
+              ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0)) {
+            float4 t4[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t4[j] = *reinterpret_cast<const float4*>(tp + 4 * j);
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (out.bias) bv = *reinterpret_cast<const float4*>(out.bias + col0 + 4 * j);
+              const float d0 = (__uint_as_float(r[4 * j]) + bv.x) - t4[j].x;
+              const float d1 = (__uint_as_float(r[4 * j + 1]) + bv.y) - t4[j].y;
+              const float d2 = (__uint_as_float(r[4 * j + 2]) + bv.z) - t4[j].z;
+              const float d3 = (__uint_as_float(r[4 * j + 3]) + bv.w) - t4[j].w;
+              sq = fmaf(d0, d0, sq); sq = fmaf(d1, d1, sq); sq = fmaf(d2, d2, sq); sq = fmaf(d3, d3, sq);
+              packed[2 * j] = pack_bf16x2(d0 * two, d1 * two);
+              packed[2 * j + 1] = pack_bf16x2(d2 * two, d3 * two);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              *reinterpret_cast<uint4*>(dp + 8 * j) = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < N) {
+                const float d = (__uint_as_float(r[j]) + (out.bias ? out.bias[col0 + j] : 0.f)) - tp[j];
+                sq = fmaf(d, d, sq);
+                dp[j] = __float2bfloat16_rn(d * two);
+              }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (lane == 0 && m0 + warp * 32 < M && col0 < N)
+          out.loss_part[(size_t)((m0 + warp * 32) / 32) * out.parts + col0 / 32] = sq * out.scale;
+      } else if (row < M) {
         if (out.kind == GemmOut::STORE_BF16) {
           __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row_o * out.ld + col0;
 #pragma unroll

@@ -91,10 +91,6 @@ __device__ __forceinline__ bool wait_counter(const uint32_t* ctr, uint32_t targe
   *failed = 1;
   return false;
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
 
@@ -353,7 +349,7 @@ struct BwdRunArgs {
   __nv_bfloat16* dz;       // [S][B][4H] staging, row block (k-1) % S, gate columns permuted
   float* dh;               // [B][H] carried dL/dh (in: from step k_hi + 1; out: for step k_lo - 1)
   float* dc;               // [B][H] carried dL/dc
-  const float* loss_part;  // [S][LOSS_PARTS]
+  const float* loss_part;  // [S][loss_parts]
   float* loss_t;           // [t]
   uint32_t* sync;
   int* status;
@@ -361,6 +357,7 @@ struct BwdRunArgs {
   int B, H, S;
   uint32_t plane16, hsz16;
   const float* zleaf;      // leaf batch: [S][B][4H] pre-activations z_k (gate columns permuted); NULL otherwise
+  int loss_parts;          // partial sums of the loss per step
 };
 
 // What the gate derivatives of one batch row and 8 hidden units read from memory at one step: the
@@ -546,7 +543,7 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
     if (cta == 0 && tid == 0) {
       // loss term of this step: its partial sums in a fixed order
       float s = 0.f;
-      for (int p = 0; p < LOSS_PARTS; ++p) s += a.loss_part[sidx * LOSS_PARTS + p];
+      for (int p = 0; p < a.loss_parts; ++p) s += a.loss_part[sidx * a.loss_parts + p];
       a.loss_t[op.k - 1] = s;
     }
     fence_proxy_async();
@@ -691,7 +688,7 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
         // loss term of this step: its partial sums in a fixed order (on a lane that is off the
         // critical path of the recurrence)
         float sum = 0.f;
-        for (int p = 0; p < LOSS_PARTS; ++p) sum += a.loss_part[sidx * LOSS_PARTS + p];
+        for (int p = 0; p < a.loss_parts; ++p) sum += a.loss_part[sidx * a.loss_parts + p];
         a.loss_t[a.ops[i].k - 1] = sum;
       }
       int go = 1;
@@ -1347,7 +1344,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         cudaStreamWaitEvent(s, side->done[pb], 0);
         side_busy[pb] = false;
       }
-      launches += 3;
+      launches += 2;   // gather_states and the backward run itself
       if (!dry && rc == MEBPTT_OK) {
         const size_t block16 = (size_t)B * H * 2 / 16;
         launch_pdl(gather_states, dim3(16, n), dim3(256), 0, s, bops, n, ws,
@@ -1365,16 +1362,28 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         if (!dry && rc == MEBPTT_OK)
           launch_pdl(leaf_forward, dim3(32, n), dim3(256), 0, s, bops, n, ws, zleaf, hk_c, S, B, H, io.counters);
       }
-      // readout of the n steps at once, then loss terms and dy, then the gradient entering h_k
-      gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
-           GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
-      if (!dry && rc == MEBPTT_OK)
-        launch_pdl(loss_dy, dim3(LOSS_PARTS, n), dim3(256), 0, s, bops, yv, io.targets, dy_c, loss_part, S, B, O);
+      // readout of the n steps at once, loss terms and dy, then the gradient entering h_k
+      const bool fused_loss = loss_fused(B, O);
+      const int parts = loss_parts_per_step(B, O);
+      if (fused_loss) {
+        GemmOut o{GemmOut::LOSS_DY, dy_c + (size_t)s_lo * B * O, O, io.b_out, 0};
+        o.target = io.targets + (size_t)(k_lo - 1) * B * O;
+        o.loss_part = loss_part + (size_t)s_lo * parts;
+        o.parts = (O + 31) / 32;
+        o.scale = 1.f / ((float)B * (float)O);
+        gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false, o, n * B, O, H);
+      } else {
+        gemm(hk_c + (size_t)s_lo * B * H, H, false, io.W_out, H, false,
+             GemmOut{GemmOut::STORE_F32, yv + (size_t)s_lo * B * O, O, io.b_out, 0}, n * B, O, H);
+        ++launches;
+        if (!dry && rc == MEBPTT_OK)
+          launch_pdl(loss_dy, dim3(LOSS_PARTS, n), dim3(256), 0, s, bops, yv, io.targets, dy_c, loss_part, S, B, O);
+      }
       gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
         BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
-                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr};
+                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         const int span = span_begin(timer, 1, n, s);
         if (bwd_cs) {
