@@ -275,14 +275,16 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
   cudaMemcpyAsync(ws + g.b, b, g.nb, cudaMemcpyHostToDevice, s);
   cudaMemcpyAsync(ws + g.W_out, W_out, g.nW_out, cudaMemcpyHostToDevice, s);
   cudaMemcpyAsync(ws + g.b_out, b_out, g.nb_out, cudaMemcpyHostToDevice, s);
-  cudaMemcpyAsync(ws + g.x, x, g.nx, cudaMemcpyHostToDevice, s);
   cudaMemcpyAsync(ws + g.h0, h0, g.nh0, cudaMemcpyHostToDevice, s);
   cudaMemcpyAsync(ws + g.c0, c0, g.nc0, cudaMemcpyHostToDevice, s);
-  // the targets are not needed before the first backward operation: the tensor-core path copies
-  // them beside the forward pass
+  // x is read progressively by the forward pass and the targets not before the first backward
+  // operation: the tensor-core path copies both beside the forward pass
   static const bool no_overlap = getenv("MEBPTT_NO_OVERLAP") != nullptr;
   const bool late_targets = y.tensor_path && !no_overlap;
-  if (!late_targets) cudaMemcpyAsync(ws + g.targets, targets, g.ntargets, cudaMemcpyHostToDevice, s);
+  if (!late_targets) {
+    cudaMemcpyAsync(ws + g.x, x, g.nx, cudaMemcpyHostToDevice, s);
+    cudaMemcpyAsync(ws + g.targets, targets, g.ntargets, cudaMemcpyHostToDevice, s);
+  }
   if (cudaGetLastError() != cudaSuccess) return MEBPTT_ERR_CUDA;
   StepIO io{ws + g.W, ws + g.W_out, ws + g.x, ws + g.h0,
             (const float*)(ws + g.b), (const float*)(ws + g.b_out), (const float*)(ws + g.targets),
@@ -290,7 +292,10 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
             (float*)(ws + g.loss), (float*)(ws + g.dW), (float*)(ws + g.db), (float*)(ws + g.dW_out),
             (float*)(ws + g.db_out), desc->want_dx ? (float*)(ws + g.dx) : nullptr,
             (int64_t*)(ws + g.counters)};
-  if (late_targets) { io.targets_host = targets; io.targets_bytes = g.ntargets; }
+  if (late_targets) {
+    io.targets_host = targets; io.targets_bytes = g.ntargets;
+    io.x_host = x; io.x_bytes = g.nx;
+  }
   io.time_runs = (desc->flags & MEBPTT_FLAG_TIME_RUNS) != 0;
   rc = run_step(desc, p, y, io, s);
   if (rc != MEBPTT_OK) return rc;

@@ -40,6 +40,10 @@ struct StepPtrs {
   // backward run
   const void* targets_host = nullptr;
   size_t targets_bytes = 0;
+  // optional, likewise: x still lies in host memory; it is copied to `x` in pieces along the time
+  // axis on the copy stream, and each forward run waits only for the pieces it reads
+  const void* x_host = nullptr;
+  size_t x_bytes = 0;
   // bracket every launch of the two persistent kernels with CUDA events (collected by run_times)
   bool time_runs = false;
 };
@@ -64,10 +68,6 @@ namespace tc {
 int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
                  bool side_stream);
 
-// Enqueues the host-to-device copy of the targets on the library's copy stream, ordered after
-// everything already in `s`, and returns the event that marks its completion (nullptr if the
-// side streams are unavailable: the caller then copies on `s`).
-cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s);
 
 // Waits for the event pairs recorded on the current device by steps run with time_runs, adds up
 // elapsed milliseconds, launches and operations per class (0: forward runs, 1: backward runs)

@@ -1010,12 +1010,14 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
 // A second stream and four events per device, created on first use and kept for the life of the
 // process.  The side stream has lower priority than any stream a caller is likely to pass, so
 // that the cooperative kernels of the recurrence get their SMs first and the GEMMs fill the rest.
+constexpr int X_PIECES = 8;
 struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t ready[2] = {nullptr, nullptr};   // stages of parity p are complete (recorded on the caller's stream)
   cudaEvent_t done[2] = {nullptr, nullptr};    // GEMMs reading parity p have finished (recorded on the side stream)
   cudaStream_t copy = nullptr;                 // host-to-device copies that overlap the forward pass
   cudaEvent_t copy_from = nullptr, copy_done = nullptr;
+  cudaEvent_t x_ready[X_PIECES] = {};          // pieces of x (along time) have arrived
   bool ok = false;
 };
 SideStream* side_stream_for_current_device() {
@@ -1038,6 +1040,8 @@ SideStream* side_stream_for_current_device() {
     ok = ok && cudaStreamCreateWithFlags(&t.copy, cudaStreamNonBlocking) == cudaSuccess &&
          cudaEventCreateWithFlags(&t.copy_from, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&t.copy_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < X_PIECES && ok; ++i)
+      ok = cudaEventCreateWithFlags(&t.x_ready[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) cudaGetLastError();
     t.ok = ok;
   }
@@ -1101,14 +1105,40 @@ int run_times(double* ms, int64_t* launches, int64_t* ops) {
   return rc;
 }
 
-cudaEvent_t copy_targets_async(void* dst, const void* src, size_t bytes, cudaStream_t s) {
+// Inputs that are still in host memory, copied on the library's copy stream beside the forward
+// pass: x in X_PIECES pieces along the time axis (event x_ready[p] marks piece p), then the
+// targets (event copy_done).  Ordered after everything already in `s`: the previous step on `s`
+// may still read the destinations.
+struct LateCopies {
+  SideStream* side = nullptr;
+  int x_pieces = 0;            // 0: x was not copied here
+  int64_t steps_per_piece = 0;
+  bool targets = false;
+};
+LateCopies start_late_copies(const StepPtrs& io, int64_t t, cudaStream_t s) {
+  LateCopies lc;
   SideStream* side = side_stream_for_current_device();
-  if (!side) return nullptr;
-  cudaEventRecord(side->copy_from, s);            // the previous step on `s` may still read dst
+  if (!side || (!io.x_host && !io.targets_host)) return lc;
+  lc.side = side;
+  cudaEventRecord(side->copy_from, s);
   cudaStreamWaitEvent(side->copy, side->copy_from, 0);
-  cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, side->copy);
-  cudaEventRecord(side->copy_done, side->copy);
-  return side->copy_done;
+  if (io.x_host) {
+    const size_t per_step = io.x_bytes / (size_t)t;
+    lc.steps_per_piece = (t + X_PIECES - 1) / X_PIECES;
+    lc.x_pieces = (int)((t + lc.steps_per_piece - 1) / lc.steps_per_piece);
+    for (int p = 0; p < lc.x_pieces; ++p) {
+      const int64_t lo = p * lc.steps_per_piece, hi = (lo + lc.steps_per_piece < t) ? lo + lc.steps_per_piece : t;
+      cudaMemcpyAsync(const_cast<char*>(io.x) + (size_t)lo * per_step, (const char*)io.x_host + (size_t)lo * per_step,
+                      (size_t)(hi - lo) * per_step, cudaMemcpyHostToDevice, side->copy);
+      cudaEventRecord(side->x_ready[p], side->copy);
+    }
+  }
+  if (io.targets_host) {
+    cudaMemcpyAsync(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, cudaMemcpyHostToDevice, side->copy);
+    cudaEventRecord(side->copy_done, side->copy);
+    lc.targets = true;
+  }
+  return lc;
 }
 
 int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
@@ -1263,12 +1293,19 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   launches += 3;
   // The targets, if they are still on the host: requested after every other host-to-device copy of
   // this step (the copy engine serves requests in order), on a stream of their own.
-  cudaEvent_t targets_ready = nullptr;
-  if (!dry && io.targets_host) {
-    targets_ready = copy_targets_async(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, s);
-    if (!targets_ready)
+  LateCopies late;
+  if (!dry && (io.targets_host || io.x_host)) {
+    late = start_late_copies(io, y.t, s);
+    if (io.x_host && !late.x_pieces)
+      cudaMemcpyAsync(const_cast<char*>(io.x), io.x_host, io.x_bytes, cudaMemcpyHostToDevice, s);
+    if (io.targets_host && !late.targets)
       cudaMemcpyAsync(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, cudaMemcpyHostToDevice, s);
   }
+  int x_waited = 0;   // pieces of x the caller's stream has already waited for
+  auto need_x = [&](int64_t steps) {   // time steps [0, steps) of x are about to be read on `s`
+    while (x_waited < late.x_pieces && (int64_t)x_waited * late.steps_per_piece < steps)
+      cudaStreamWaitEvent(s, late.side->x_ready[x_waited++], 0);
+  };
 
   int launch_id = 0;
   int rc = MEBPTT_OK;
@@ -1306,6 +1343,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         zx_lo = k0;
         zx_hi = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
         const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
+        need_x(zx_hi - 1);
         gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
       }
       ++launches;
@@ -1325,8 +1363,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       // or a batch of leaves, whose forward operations are done here as well, all at once
       const bool leaf = wi.kind == WorkItem::LEAF;
       const DevOp* bops = leaf ? dops + nops + i : dops + i;
-      if (targets_ready && !targets_waited) {
-        cudaStreamWaitEvent(s, targets_ready, 0);   // the targets were copied beside the forward pass
+      if (!targets_waited) {
+        need_x(y.t);                                  // leaves and weight gradients read x anywhere
+        if (late.targets) cudaStreamWaitEvent(s, late.side->copy_done, 0);   // copied beside the forward pass
         targets_waited = true;
       }
       const int chunk = (first.k - 1) / S;
