@@ -153,7 +153,7 @@ def kernel_breakdown(dp, plans):
 # DRAM traffic of the forward run kernel per forward operation, from the ncu capture summarised in
 # profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md (25.61 MB read, nothing written to DRAM, per
 # launch of 16 operations).  Valid for config 3's layer sizes and the kernel as profiled there.
-FWD_RUN_DRAM_BYTES_PER_OP_C3 = 25.611776e6 / 16
+FWD_RUN_DRAM_BYTES_PER_OP_C3 = 25.612032e6 / 16
 
 
 def max_over_ranks(v: float, world: int, device) -> float:
