@@ -347,7 +347,9 @@ def main():
         achieved = flops_fwd_op / (fwd_op_ms * 1e-3) / 1e12 if fwd_op_ms else None
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": (achieved / peak_tf) if achieved else None, "traffic": None,
-                    "kernel": "forward operation on the CUDA-core path (gate contraction + cell update, several launches)",
+                    "kernel": ("forward operation, step by step (per layer: two tensor-core GEMMs and a cell kernel)"
+                               if cfg.dtype == "bf16" and not (cfg.batch % 32) else
+                               "forward operation on the CUDA-core path (gate contraction + cell update in one launch per layer)"),
                     "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
                            f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
                            + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}

@@ -66,7 +66,17 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   float* dy = reinterpret_cast<float*>(ws + y.off_dy);
   float* loss_part = reinterpret_cast<float*>(ws + y.off_loss_part);
   float* loss_t = reinterpret_cast<float*>(ws + y.off_loss_t);
+  int* status = reinterpret_cast<int*>(ws + y.off_status);
+  stepwise::Scratch tcw{};
+  if (y.stepwise_tc) {
+    tcw.z = reinterpret_cast<float*>(ws + y.off_z);
+    tcw.dz16 = reinterpret_cast<__nv_bfloat16*>(ws + y.off_dz16);
+    tcw.dy16 = reinterpret_cast<__nv_bfloat16*>(dy);
+    tcw.status = status;
+  }
+  int rc = MEBPTT_OK;
 
+  cudaMemsetAsync(status, 0, 256, s);
   cudaMemsetAsync(dh_rec, 0, (size_t)y.L * bh * 4, s);
   cudaMemsetAsync(dc_rec, 0, (size_t)y.L * bh * 4, s);
   cudaMemsetAsync(io.dW, 0, y.w_total_elems() * 4, s);
@@ -76,6 +86,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
 
   for (const mebptt_op& op : p->tape) {
+    if (rc != MEBPTT_OK) break;
     const int64_t k = op.k;
     const char* x_k = io.x + (size_t)(k - 1) * y.B * y.I * y.esz;
     if (op.kind == MEBPTT_OP_FWD) {
@@ -97,7 +108,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.plane_elems = plane_elems;
         a.B = y.B; a.H = y.H;
         a.counters = (l == 0) ? io.counters : nullptr;
-        generic::forward_step(y.dtype, a, s);
+        if (y.stepwise_tc) rc = stepwise::forward_step(a, tcw, s);
+        else generic::forward_step(y.dtype, a, s);
+        if (rc != MEBPTT_OK) break;
       }
     } else {
       char* rec = loc_base(y, ws, op.src);
@@ -110,7 +123,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
       r.loss_k = loss_t + (k - 1);
       r.dha = dha; r.dW_out = io.dW_out; r.db_out = io.db_out;
       r.B = y.B; r.H = y.H; r.O = y.O;
-      generic::readout(y.dtype, r, s);
+      if (y.stepwise_tc) rc = stepwise::readout(r, tcw, s);
+      else generic::readout(y.dtype, r, s);
+      if (rc != MEBPTT_OK) break;
       for (int l = y.L - 1; l >= 0; --l) {
         generic::BwdArgs a{};
         a.dha = dha;
@@ -134,11 +149,14 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(k - 1) * y.B * y.I : nullptr);
         a.B = y.B; a.H = y.H;
         a.counters = (l == y.L - 1) ? io.counters : nullptr;
-        generic::backward_layer(y.dtype, a, s);
+        if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, s);
+        else generic::backward_layer(y.dtype, a, s);
+        if (rc != MEBPTT_OK) break;
       }
     }
   }
-  generic::finalize_step(loss_t, y.t, io.loss, io.counters, p->peak_units, s);
+  if (rc != MEBPTT_OK) return rc;
+  generic::finalize_step(loss_t, y.t, io.loss, io.counters, p->peak_units, status, s);
   return cudaGetLastError() == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
 }
 
@@ -204,6 +222,12 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
   // forward operation: one kernel per layer; backward operation: 5 for the readout and
   // 4 per layer; one to finalise
   const int64_t L = desc->layers;
+  if (y.stepwise_tc) {
+    // forward operation: two GEMMs and the cell kernel per layer; readout: 5; backward operation
+    // per layer: gate kernel, two dW GEMMs, db, and one or two d_in GEMMs
+    const int64_t bwd = 4 * L + 2 * (L - 1) + (desc->want_dx ? 2 : 1);
+    return p->cost * 3 * L + p->t * (5 + bwd) + 1;
+  }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }
 

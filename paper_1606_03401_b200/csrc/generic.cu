@@ -283,13 +283,15 @@ __global__ void sum_partials(const float* part, int n, float scale, float* out) 
 }
 
 // loss = sum_t loss_t in ascending t by one warp (lane-strided partials, then a fixed tree)
-__global__ void finalize(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units) {
+__global__ void finalize(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
+                         const int* status) {
   float s = 0.f;
   for (int64_t i = threadIdx.x; i < t; i += 32) s += loss_t[i];
   for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
   if (threadIdx.x == 0) {
     *loss = s;
     counters[2] = peak_units;
+    counters[3] = *status;
   }
 }
 
@@ -367,8 +369,8 @@ void backward_layer(int dtype, const BwdArgs& a, cudaStream_t s) {
   else backward_layer_t<float>(a, s);
 }
 void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
-                   cudaStream_t s) {
-  finalize<<<1, 32, 0, s>>>(loss_t, t, loss, counters, peak_units);
+                   const int* status, cudaStream_t s) {
+  finalize<<<1, 32, 0, s>>>(loss_t, t, loss, counters, peak_units, status);
 }
 void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s) {
   const size_t n = bytes / 16;

@@ -1,6 +1,7 @@
 // Host-callable launchers of the device kernels (declarations shared by the executor).
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <cstddef>
@@ -67,9 +68,24 @@ struct BwdArgs {
 void forward_step(int dtype, const FwdArgs& a, cudaStream_t s);
 void readout(int dtype, const ReadoutArgs& a, cudaStream_t s);
 void backward_layer(int dtype, const BwdArgs& a, cudaStream_t s);
+// status: device word whose value goes to counters[3]
 void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
-                   cudaStream_t s);
+                   const int* status, cudaStream_t s);
 void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s);
 
 }  // namespace generic
+
+// The same three operations with their contractions on the tensor cores (bfloat16 storage,
+// dimensions that are multiples of 8, B a multiple of 32).  Each returns a status.
+namespace stepwise {
+struct Scratch {
+  float* z;                 // [B][4H] pre-activations of the forward operation in flight
+  __nv_bfloat16* dz16;      // [B][4H] dz rounded for the contractions
+  __nv_bfloat16* dy16;      // [B][O]
+  int* status;              // device word that receives MEBPTT_ERR_TIMEOUT from a bounded wait
+};
+int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s);
+int readout(const generic::ReadoutArgs& a, const Scratch& w, cudaStream_t s);
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, cudaStream_t s);
+}  // namespace stepwise
 }  // namespace mebptt

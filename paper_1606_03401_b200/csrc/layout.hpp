@@ -28,6 +28,7 @@ struct Layout {
   int dtype = 0;
   int64_t t = 0;
   bool tensor_path = false;
+  bool stepwise_tc = false;   // step-by-step operations with their contractions on the tensor cores
   size_t esz = 0;        // bytes of one operand element
   size_t granule = 0;
   size_t hsz = 0;        // one layer's h
@@ -47,6 +48,7 @@ struct Layout {
   // tensor-core path: packed weights, staging of S consecutive time steps, control
   int S = 0;             // time steps per staged chunk
   size_t off_wp_ih = 0, off_wp_hh = 0, off_wpT_hh = 0, off_wpT_ih = 0, off_bias_p = 0, off_woutT = 0;
+  size_t off_z = 0, off_dz16 = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
   size_t n_sync = 0, tape_bytes = 0;
@@ -92,10 +94,20 @@ inline bool tensor_path_supported(const mebptt_lstm_desc* d) {
 inline bool loss_fused(int B, int O) { return B % 32 == 0 && (B / 32) * ((O + 31) / 32) <= 256; }
 inline int loss_parts_per_step(int B, int O) { return loss_fused(B, O) ? (B / 32) * ((O + 31) / 32) : 64; }
 
+// Shapes outside the persistent kernels' range whose step-by-step operations can still give
+// their contractions to the tensor-core GEMM: bfloat16 storage, TMA-friendly strides, and whole
+// 32-row groups per step for the loss epilogue.
+inline bool stepwise_tc_supported(const mebptt_lstm_desc* d) {
+  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && !tensor_path_supported(d) && d->dtype == MEBPTT_BF16 &&
+         d->batch % 32 == 0 && d->input % 8 == 0 && d->hidden % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
+         (d->batch / 32) * ((d->readout + 31) / 32) <= 4096;
+}
+
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
   y.dtype = d->dtype; y.t = d->t;
   y.tensor_path = tensor_path_supported(d);
+  y.stepwise_tc = stepwise_tc_supported(d);
   y.esz = (d->dtype == MEBPTT_BF16) ? 2 : 4;
   const size_t row = (size_t)y.H * y.esz;
   y.granule = 256 / gcd_sz(256, row) * row;  // lcm(256, row bytes)
@@ -187,7 +199,13 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_dz = take((size_t)y.B * 4 * y.H * 4);
     y.off_dy = take((size_t)y.B * y.O * 4);
     y.n_loss_part = ((y.B + 63) / 64) * ((y.O + 63) / 64);
+    if (y.stepwise_tc) {
+      y.n_loss_part = (y.B / 32) * ((y.O + 31) / 32);
+      y.off_z = take((size_t)y.B * 4 * y.H * 4);
+      y.off_dz16 = take((size_t)y.B * 4 * y.H * 2);
+    }
     y.off_loss_part = take((size_t)y.n_loss_part * 4);
+    y.off_status = take(256);
   } else {
     const size_t G = (size_t)4 * y.H;
     y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;

@@ -1,0 +1,170 @@
+// Step-by-step LSTM operations with every contraction on the tensor cores.
+//
+// The persistent kernels keep W_hh in shared memory and cover one layer, a batch of at most 64
+// and H <= 1024.  Outside that range (several layers, H = 2048, B = 128) a forward or backward
+// operation is carried out layer by layer as a short sequence of launches, like the CUDA-core
+// path does, but with its contractions given to the tcgen05 GEMM (bfloat16 operands, float32
+// accumulation in a fixed order) and the gate arithmetic in small element-wise kernels:
+//   forward    z  = in W[:, :I]^T + b ;  z += h_prev W[:, I:]^T ;  gates, c, h from z
+//   readout    y  = h W_out^T + b_out, loss term and dy in the GEMM's epilogue ; dha = dy W_out ;
+//              dW_out += dy^T h ; db_out += sum_b dy
+//   backward   dz from the stored gates ; dW += dz^T [in ; h_prev] ; db += sum_b dz ;
+//              d_in = dz W[:, :I] ; dh = dz W[:, I:]
+// dz and dy are rounded to bfloat16 before they enter a contraction (as on the persistent path);
+// db is summed from the unrounded dz.  Every sum has a fixed order, and an operation's launches
+// do not depend on the plan, so results are bit-identical across plans.
+#include "kernels.hpp"
+#include "tc.hpp"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace mebptt {
+namespace stepwise {
+
+namespace {
+
+using tc::GemmOut;
+using tc::gemm_bf16;
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf(-a)); }
+
+// z [B][4H] (column q H + j: gate q of unit j, bias included) -> gates, c_k, h_k and, for an
+// internal state, the copies of h_{k-1}, c_{k-1}.
+__global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
+                         bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H,
+                         int64_t* counters) {
+  const size_t n = (size_t)B * H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / H), j = (int)(e % H);
+    const float* row = z + (size_t)b * 4 * H;
+    const float gi = sigmoidf_(row[j]), gf = sigmoidf_(row[H + j]);
+    const float gg = tanhf(row[2 * H + j]), go = sigmoidf_(row[3 * H + j]);
+    const float cp = c_prev[e];
+    const float c = fmaf(gf, cp, gi * gg);
+    c_out[e] = c;
+    h_out[e] = __float2bfloat16_rn(go * tanhf(c));
+    if (gates) {
+      gates[e] = __float2bfloat16_rn(gi);
+      gates[plane + e] = __float2bfloat16_rn(gf);
+      gates[2 * plane + e] = __float2bfloat16_rn(gg);
+      gates[3 * plane + e] = __float2bfloat16_rn(go);
+    }
+    if (h_in_copy) { h_in_copy[e] = h_prev[e]; c_in_copy[e] = cp; }
+  }
+  if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[0] += 1;
+}
+
+// Gate derivatives: dh = dha + dh_rec; dz [B][4H] in float32 (for db) and bfloat16 (for the
+// contractions); dc_rec = dc * f.
+__global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const bf16* gates, size_t plane,
+                         const float* c_t, const float* c_prev, float* dz, bf16* dz16, int B, int H,
+                         int64_t* counters) {
+  const size_t n = (size_t)B * H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / H), j = (int)(e % H);
+    const float gi = __bfloat162float(gates[e]), gf = __bfloat162float(gates[plane + e]);
+    const float gg = __bfloat162float(gates[2 * plane + e]), go = __bfloat162float(gates[3 * plane + e]);
+    const float dh = dha[e] + dh_rec[e];
+    const float th = tanhf(c_t[e]);
+    const float d_o = dh * th;
+    const float dc = fmaf(dh * go, 1.f - th * th, dc_rec[e]);
+    const float v0 = dc * gg * gi * (1.f - gi);
+    const float v1 = dc * c_prev[e] * gf * (1.f - gf);
+    const float v2 = dc * gi * (1.f - gg * gg);
+    const float v3 = d_o * go * (1.f - go);
+    const size_t r = (size_t)b * 4 * H + j;
+    dz[r] = v0; dz[r + H] = v1; dz[r + 2 * (size_t)H] = v2; dz[r + 3 * (size_t)H] = v3;
+    dz16[r] = __float2bfloat16_rn(v0); dz16[r + H] = __float2bfloat16_rn(v1);
+    dz16[r + 2 * (size_t)H] = __float2bfloat16_rn(v2); dz16[r + 3 * (size_t)H] = __float2bfloat16_rn(v3);
+    dc_rec[e] = dc * gf;
+  }
+  if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
+}
+
+// out[n] += sum_b v[b][n], b ascending
+template <class T>
+__global__ void colsum_accum(const T* v, int B, int N, float* out) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += (float)v[(size_t)b * N + n];
+  out[n] += s;
+}
+
+__global__ void sum_parts(const float* part, int n, float* out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < n; ++i) s += part[i];
+    *out = s;
+  }
+}
+
+inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
+
+}  // namespace
+
+int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
+  const int K = a.I + a.H, G = 4 * a.H;
+  const bf16* W = (const bf16*)a.W;
+  int rc = gemm_bf16(a.in, a.I, false, W, K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0}, a.B, G, a.I,
+                     w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  rc = gemm_bf16(a.h_prev, a.H, false, W + a.I, K, false, GemmOut{GemmOut::ACCUM_F32, w.z, G, nullptr, 0}, a.B, G,
+                 a.H, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  const size_t n = (size_t)a.B * a.H;
+  cell_fwd<<<ew_blocks(n), 256, 0, s>>>(w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
+                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
+  return MEBPTT_OK;
+}
+
+int readout(const generic::ReadoutArgs& a, const Scratch& w, cudaStream_t s) {
+  const bf16* W_out = (const bf16*)a.W_out;
+  GemmOut o{GemmOut::LOSS_DY, w.dy16, a.O, a.b_out, 0};
+  o.target = a.target;
+  o.loss_part = a.loss_part;
+  o.parts = (a.O + 31) / 32;
+  o.scale = 1.f / ((float)a.B * (float)a.O);
+  int rc = gemm_bf16(a.h, a.H, false, W_out, a.H, false, o, a.B, a.O, a.H, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  sum_parts<<<1, 32, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k);
+  // dha[b][j] = sum_o dy[b][o] W_out[o][j]: W_out read as the [k][n] operand
+  rc = gemm_bf16(w.dy16, a.O, false, W_out, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B, a.H,
+                 a.O, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  // dW_out[o][j] += sum_b dy[b][o] h[b][j]: both operands stored [k = b][.]
+  rc = gemm_bf16(w.dy16, a.O, true, a.h, a.H, true, GemmOut{GemmOut::ACCUM_F32, a.dW_out, a.H, nullptr, 0}, a.O, a.H,
+                 a.B, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  colsum_accum<bf16><<<(a.O + 127) / 128, 128, 0, s>>>(w.dy16, a.B, a.O, a.db_out);
+  return MEBPTT_OK;
+}
+
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, cudaStream_t s) {
+  const int K = a.I + a.H, G = 4 * a.H;
+  const size_t n = (size_t)a.B * a.H;
+  const bf16* W = (const bf16*)a.W;
+  gate_bwd<<<ew_blocks(n), 256, 0, s>>>(a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
+                                        a.dz, w.dz16, a.B, a.H, a.counters);
+  // dW[g][c] += sum_b dz[b][g] [in ; h_prev][b][c]   (h_prev is read before dh_rec is replaced)
+  int rc = gemm_bf16(w.dz16, G, true, a.in, a.I, true, GemmOut{GemmOut::ACCUM_F32, a.dW, K, nullptr, 0}, G, a.I, a.B,
+                     w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  rc = gemm_bf16(w.dz16, G, true, a.h_prev, a.H, true, GemmOut{GemmOut::ACCUM_F32, a.dW + a.I, K, nullptr, 0}, G, a.H,
+                 a.B, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  colsum_accum<float><<<(G + 127) / 128, 128, 0, s>>>(a.dz, a.B, G, a.db);
+  // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
+  if (a.d_lo) {
+    rc = gemm_bf16(w.dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
+                   w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+  }
+  return gemm_bf16(w.dz16, G, false, W + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B, a.H,
+                   G, w.status, s);
+}
+
+}  // namespace stepwise
+}  // namespace mebptt

@@ -207,6 +207,38 @@ def test_run_times_count_every_backward_operation_and_change_no_result(H):
     assert again["forward"][1] == 0 and again["backward"][1] == 0
 
 
+@pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=21, readout=40),
+                                   dict(layers=3, input=24, hidden=64, batch=96, t=13, readout=8),
+                                   dict(layers=1, input=128, hidden=1152, batch=64, t=9, readout=64),
+                                   dict(layers=1, input=64, hidden=128, batch=128, t=17, readout=72)])
+def test_stepwise_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
+    """bf16 shapes outside the persistent kernels' range (several layers, H > 1024, B > 64): every
+    operation is a sequence of launches whose contractions run on the tensor cores.  Oracle
+    parity, bit identity across plans, agreement with the CUDA-core kernels."""
+    from paper_1606_03401_b200 import binding as B
+    from tests.util import rel_l2
+    cfg = _cfg("c2", **shape)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][3] == 0
+    assert_close_to_oracle(full, ref, "bf16", want_dx=True)
+    for mode, m, beta in [("hsm", 1, 0), ("hsm", 4, 0), ("ism", 2, 0), ("msm", 9, 0), ("msm", 13, 3)]:
+        plan = dp.plan(mode, m, beta=beta)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+        assert_bit_identical(res, full, want_dx=True)
+    slow = H.DeviceProblem(cfg, dp.prob, want_dx=True, flags=B.MEBPTT_FLAG_NO_TENSOR_CORES)
+    other = slow.run(slow.full_memory_plan())
+    assert abs(other["loss"] - full["loss"]) < 1e-3 * abs(other["loss"])
+    for k in ("dW", "db", "dW_out", "db_out", "dx"):
+        assert rel_l2(full[k], other[k]) < 1e-2, k
+    # without dx the first layer skips its input-gradient contraction; nothing else may change
+    nodx = H.DeviceProblem(cfg, dp.prob, want_dx=False)
+    res = nodx.run(nodx.plan("msm", 9))
+    assert_bit_identical(res, full)
+
+
 def test_c2_full_size_every_budget(H):
     """Config 2 as timed: I512 H512 B64 t256 bf16, HSM and ISM at m = 16, 64, 256."""
     cfg = synth.CONFIGS["c2"]
