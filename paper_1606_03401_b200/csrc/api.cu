@@ -70,9 +70,14 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   stepwise::Scratch tcw{};
   if (y.stepwise_tc) {
     tcw.z = reinterpret_cast<float*>(ws + y.off_z);
-    tcw.dz16 = reinterpret_cast<__nv_bfloat16*>(ws + y.off_dz16);
-    tcw.dy16 = reinterpret_cast<__nv_bfloat16*>(dy);
     tcw.status = status;
+    tcw.S = y.S; tcw.I0 = y.I;
+    tcw.st_dz = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_dz);
+    tcw.st_in = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_in);
+    tcw.st_hp = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_hp);
+    tcw.st_dy = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_dy);
+    tcw.st_h = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_h);
+    tcw.split = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), (size_t)148 * 128 * 128};
   }
   int rc = MEBPTT_OK;
 
@@ -123,7 +128,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
       r.loss_k = loss_t + (k - 1);
       r.dha = dha; r.dW_out = io.dW_out; r.db_out = io.db_out;
       r.B = y.B; r.H = y.H; r.O = y.O;
-      if (y.stepwise_tc) rc = stepwise::readout(r, tcw, s);
+      const int sidx = y.stepwise_tc ? (int)((k - 1) % y.S) : 0;
+      if (y.stepwise_tc) rc = stepwise::readout(r, tcw, sidx, s);
       else generic::readout(y.dtype, r, s);
       if (rc != MEBPTT_OK) break;
       for (int l = y.L - 1; l >= 0; --l) {
@@ -149,9 +155,17 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(k - 1) * y.B * y.I : nullptr);
         a.B = y.B; a.H = y.H;
         a.counters = (l == y.L - 1) ? io.counters : nullptr;
-        if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, s);
+        if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, l, sidx, s);
         else generic::backward_layer(y.dtype, a, s);
         if (rc != MEBPTT_OK) break;
+      }
+      if (y.stepwise_tc && sidx == 0 && rc == MEBPTT_OK) {
+        // the chunk's first step has been backpropagated: its weight gradients in one go
+        const int64_t chunk = (k - 1) / y.S;
+        const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
+        size_t w_off[16];
+        for (int l = 0; l < y.L; ++l) w_off[l] = y.w_layer_offset(l);
+        rc = stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
       }
     }
   }
@@ -223,10 +237,17 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
   // 4 per layer; one to finalise
   const int64_t L = desc->layers;
   if (y.stepwise_tc) {
-    // forward operation: two GEMMs and the cell kernel per layer; readout: 5; backward operation
-    // per layer: gate kernel, two dW GEMMs, db, and one or two d_in GEMMs
-    const int64_t bwd = 4 * L + 2 * (L - 1) + (desc->want_dx ? 2 : 1);
-    return p->cost * 3 * L + p->t * (5 + bwd) + 1;
+    // forward operation: two GEMMs and the cell kernel per layer; readout: 3 and the dha GEMM;
+    // backward operation per layer: gate kernel, db, and one or two d_in GEMMs
+    // (a contraction that is split along K takes a second launch to add its parts)
+    const size_t pf = (size_t)148 * 128 * 128;
+    const int G = 4 * y.H;
+    const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, G, pf) > 1 ? 2 : 1;   // dz W -> [B][H]
+    const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, G, pf) > 1 ? 2 : 1;   // dz W -> [B][I]
+    const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, y.O, pf) > 1 ? 2 : 1;
+    const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs
+    return p->cost * 3 * L + p->t * (3 + dha + bwd) + chunks * (2 * L + 1) + 1;
   }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }

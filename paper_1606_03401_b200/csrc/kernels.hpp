@@ -8,6 +8,7 @@
 #include <cstdint>
 
 #include "mebptt.h"
+#include "tc.hpp"
 
 namespace mebptt {
 namespace generic {
@@ -80,12 +81,22 @@ void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s);
 namespace stepwise {
 struct Scratch {
   float* z;                 // [B][4H] pre-activations of the forward operation in flight
-  __nv_bfloat16* dz16;      // [B][4H] dz rounded for the contractions
-  __nv_bfloat16* dy16;      // [B][O]
   int* status;              // device word that receives MEBPTT_ERR_TIMEOUT from a bounded wait
+  tc::SplitWs split;        // scratch of the contractions that are split along K
+  // stages of one chunk of S time steps, row block (k - 1) % S of B rows per step
+  int S, I0;                // I0: input width of the first layer
+  __nv_bfloat16* st_dz;     // [L][S B][4H]
+  __nv_bfloat16* st_in;     // layer 0: [S B][I0]; layers l > 0: [S B][H] each, after it
+  __nv_bfloat16* st_hp;     // [L][S B][H]  h_{k-1}
+  __nv_bfloat16* st_dy;     // [S B][O]
+  __nv_bfloat16* st_h;      // [S B][H]  top layer h_k
 };
 int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s);
-int readout(const generic::ReadoutArgs& a, const Scratch& w, cudaStream_t s);
-int backward_layer(const generic::BwdArgs& a, const Scratch& w, cudaStream_t s);
+// sidx: row block of this step in the stages; l: layer
+int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s);
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx, cudaStream_t s);
+// dW (w_off[l]: element offset of layer l) and dW_out from the first `steps` row blocks of the stages
+int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
+                float* dW_out, cudaStream_t s);
 }  // namespace stepwise
 }  // namespace mebptt

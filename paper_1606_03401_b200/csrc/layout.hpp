@@ -48,7 +48,7 @@ struct Layout {
   // tensor-core path: packed weights, staging of S consecutive time steps, control
   int S = 0;             // time steps per staged chunk
   size_t off_wp_ih = 0, off_wp_hh = 0, off_wpT_hh = 0, off_wpT_ih = 0, off_bias_p = 0, off_woutT = 0;
-  size_t off_z = 0, off_dz16 = 0;
+  size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
   size_t n_sync = 0, tape_bytes = 0;
@@ -202,7 +202,16 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     if (y.stepwise_tc) {
       y.n_loss_part = (y.B / 32) * ((y.O + 31) / 32);
       y.off_z = take((size_t)y.B * 4 * y.H * 4);
-      y.off_dz16 = take((size_t)y.B * 4 * y.H * 2);
+      // stages of one chunk of S steps for the weight-gradient contractions
+      y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
+      const size_t rows = (size_t)y.S * y.B;
+      y.off_st_dz = take((size_t)y.L * rows * 4 * y.H * 2);
+      y.off_st_in = take(rows * y.I * 2 + (size_t)(y.L - 1) * rows * y.H * 2);
+      y.off_st_hp = take((size_t)y.L * rows * y.H * 2);
+      y.off_st_dy = take(rows * y.O * 2);
+      y.off_st_h = take(rows * y.H * 2);
+      // split-K scratch: at most a wave of 128 x 128 float32 tiles
+      y.off_split = take((size_t)148 * 128 * 128 * 4);
     }
     y.off_loss_part = take((size_t)y.n_loss_part * 4);
     y.off_status = take(256);

@@ -8,8 +8,11 @@
 //   forward    z  = in W[:, :I]^T + b ;  z += h_prev W[:, I:]^T ;  gates, c, h from z
 //   readout    y  = h W_out^T + b_out, loss term and dy in the GEMM's epilogue ; dha = dy W_out ;
 //              dW_out += dy^T h ; db_out += sum_b dy
-//   backward   dz from the stored gates ; dW += dz^T [in ; h_prev] ; db += sum_b dz ;
-//              d_in = dz W[:, :I] ; dh = dz W[:, I:]
+//   backward   dz from the stored gates ; db += sum_b dz ; d_in = dz W[:, :I] ; dh = dz W[:, I:]
+//   per chunk  dW += dz^T [in ; h_prev] and dW_out += dy^T h over the S steps of a chunk at once:
+//              dz, dy and the operands they meet are staged per step (row block (k - 1) % S), and
+//              the chunk is flushed when its first step has been backpropagated.  Chunks are
+//              tied to absolute time, so the order of every sum is the same for every plan.
 // dz and dy are rounded to bfloat16 before they enter a contraction (as on the persistent path);
 // db is summed from the unrounded dz.  Every sum has a fixed order, and an operation's launches
 // do not depend on the plan, so results are bit-identical across plans.
@@ -58,10 +61,16 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev
 
 // Gate derivatives: dh = dha + dh_rec; dz [B][4H] in float32 (for db) and bfloat16 (for the
 // contractions); dc_rec = dc * f.
+// Also copies this step's layer input and h_{k-1} to their stages (n_in16, n_hp16: 16-byte words).
 __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const bf16* gates, size_t plane,
                          const float* c_t, const float* c_prev, float* dz, bf16* dz16, int B, int H,
-                         int64_t* counters) {
+                         int64_t* counters, const uint4* in, uint4* st_in, size_t n_in16, const uint4* hp,
+                         uint4* st_hp, size_t n_hp16) {
   const size_t n = (size_t)B * H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_in16; e += (size_t)gridDim.x * blockDim.x)
+    st_in[e] = in[e];
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_hp16; e += (size_t)gridDim.x * blockDim.x)
+    st_hp[e] = hp[e];
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
     const float gi = __bfloat162float(gates[e]), gf = __bfloat162float(gates[plane + e]);
@@ -93,7 +102,11 @@ __global__ void colsum_accum(const T* v, int B, int N, float* out) {
   out[n] += s;
 }
 
-__global__ void sum_parts(const float* part, int n, float* out) {
+// Loss term of one step from its partial sums (block 0, one thread); every block helps copy the
+// top layer's h_k to its stage.
+__global__ void sum_parts_stage_h(const float* part, int n, float* out, const uint4* h, uint4* st_h, size_t n_h16) {
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_h16; e += (size_t)gridDim.x * blockDim.x)
+    st_h[e] = h[e];
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     float s = 0.f;
     for (int i = 0; i < n; ++i) s += part[i];
@@ -109,10 +122,10 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
   const int K = a.I + a.H, G = 4 * a.H;
   const bf16* W = (const bf16*)a.W;
   int rc = gemm_bf16(a.in, a.I, false, W, K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0}, a.B, G, a.I,
-                     w.status, s);
+                     w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
   rc = gemm_bf16(a.h_prev, a.H, false, W + a.I, K, false, GemmOut{GemmOut::ACCUM_F32, w.z, G, nullptr, 0}, a.B, G,
-                 a.H, w.status, s);
+                 a.H, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
   cell_fwd<<<ew_blocks(n), 256, 0, s>>>(w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
@@ -120,50 +133,69 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
   return MEBPTT_OK;
 }
 
-int readout(const generic::ReadoutArgs& a, const Scratch& w, cudaStream_t s) {
+int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s) {
   const bf16* W_out = (const bf16*)a.W_out;
-  GemmOut o{GemmOut::LOSS_DY, w.dy16, a.O, a.b_out, 0};
+  bf16* dy16 = w.st_dy + (size_t)sidx * a.B * a.O;
+  GemmOut o{GemmOut::LOSS_DY, dy16, a.O, a.b_out, 0};
   o.target = a.target;
   o.loss_part = a.loss_part;
   o.parts = (a.O + 31) / 32;
   o.scale = 1.f / ((float)a.B * (float)a.O);
-  int rc = gemm_bf16(a.h, a.H, false, W_out, a.H, false, o, a.B, a.O, a.H, w.status, s);
+  int rc = gemm_bf16(a.h, a.H, false, W_out, a.H, false, o, a.B, a.O, a.H, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
-  sum_parts<<<1, 32, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k);
+  const size_t n_h16 = (size_t)a.B * a.H * 2 / 16;
+  sum_parts_stage_h<<<ew_blocks(n_h16 * 8), 256, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k, (const uint4*)a.h,
+                                                          (uint4*)(w.st_h + (size_t)sidx * a.B * a.H), n_h16);
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]: W_out read as the [k][n] operand
-  rc = gemm_bf16(w.dy16, a.O, false, W_out, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B, a.H,
-                 a.O, w.status, s);
+  rc = gemm_bf16(dy16, a.O, false, W_out, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B, a.H,
+                 a.O, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
-  // dW_out[o][j] += sum_b dy[b][o] h[b][j]: both operands stored [k = b][.]
-  rc = gemm_bf16(w.dy16, a.O, true, a.h, a.H, true, GemmOut{GemmOut::ACCUM_F32, a.dW_out, a.H, nullptr, 0}, a.O, a.H,
-                 a.B, w.status, s);
-  if (rc != MEBPTT_OK) return rc;
-  colsum_accum<bf16><<<(a.O + 127) / 128, 128, 0, s>>>(w.dy16, a.B, a.O, a.db_out);
+  colsum_accum<bf16><<<(a.O + 127) / 128, 128, 0, s>>>(dy16, a.B, a.O, a.db_out);
   return MEBPTT_OK;
 }
 
-int backward_layer(const generic::BwdArgs& a, const Scratch& w, cudaStream_t s) {
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx, cudaStream_t s) {
   const int K = a.I + a.H, G = 4 * a.H;
   const size_t n = (size_t)a.B * a.H;
   const bf16* W = (const bf16*)a.W;
+  const size_t rows = (size_t)w.S * a.B;   // rows of one layer's stages
+  bf16* dz16 = w.st_dz + ((size_t)l * rows + (size_t)sidx * a.B) * G;
+  bf16* st_in = w.st_in + (l == 0 ? 0 : rows * w.I0 + (size_t)(l - 1) * rows * a.H) + (size_t)sidx * a.B * a.I;
+  bf16* st_hp = w.st_hp + ((size_t)l * rows + (size_t)sidx * a.B) * a.H;
   gate_bwd<<<ew_blocks(n), 256, 0, s>>>(a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
-                                        a.dz, w.dz16, a.B, a.H, a.counters);
-  // dW[g][c] += sum_b dz[b][g] [in ; h_prev][b][c]   (h_prev is read before dh_rec is replaced)
-  int rc = gemm_bf16(w.dz16, G, true, a.in, a.I, true, GemmOut{GemmOut::ACCUM_F32, a.dW, K, nullptr, 0}, G, a.I, a.B,
-                     w.status, s);
-  if (rc != MEBPTT_OK) return rc;
-  rc = gemm_bf16(w.dz16, G, true, a.h_prev, a.H, true, GemmOut{GemmOut::ACCUM_F32, a.dW + a.I, K, nullptr, 0}, G, a.H,
-                 a.B, w.status, s);
-  if (rc != MEBPTT_OK) return rc;
+                                        a.dz, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
+                                        (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
+                                        (size_t)a.B * a.H * 2 / 16);
   colsum_accum<float><<<(G + 127) / 128, 128, 0, s>>>(a.dz, a.B, G, a.db);
   // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
   if (a.d_lo) {
-    rc = gemm_bf16(w.dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
-                   w.status, s);
+    int rc = gemm_bf16(dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
+                       w.status, s, true, &w.split);
     if (rc != MEBPTT_OK) return rc;
   }
-  return gemm_bf16(w.dz16, G, false, W + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B, a.H,
-                   G, w.status, s);
+  return gemm_bf16(dz16, G, false, W + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B, a.H,
+                   G, w.status, s, true, &w.split);
+}
+
+// Weight gradients of a finished chunk: `steps` row blocks of B rows, from block 0 on.
+int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
+                float* dW_out, cudaStream_t s) {
+  const int G = 4 * H, R = steps * B;
+  const size_t rows = (size_t)w.S * B;
+  for (int l = 0; l < L; ++l) {
+    const int I = l == 0 ? I0 : H, K = I + H;
+    const bf16* dz = w.st_dz + (size_t)l * rows * G;
+    const bf16* in = w.st_in + (l == 0 ? 0 : rows * I0 + (size_t)(l - 1) * rows * H);
+    const bf16* hp = w.st_hp + (size_t)l * rows * H;
+    float* dWl = dW + w_off[l];
+    // dW[g][c] += sum over (step, b) of dz[.][g] [in ; h_prev][.][c]: both operands stored [k][.]
+    int rc = gemm_bf16(dz, G, true, in, I, true, GemmOut{GemmOut::ACCUM_F32, dWl, K, nullptr, 0}, G, I, R, w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+    rc = gemm_bf16(dz, G, true, hp, H, true, GemmOut{GemmOut::ACCUM_F32, dWl + I, K, nullptr, 0}, G, H, R, w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+  }
+  return gemm_bf16(w.st_dy, O, true, w.st_h, H, true, GemmOut{GemmOut::ACCUM_F32, dW_out, H, nullptr, 0}, O, H, R,
+                   w.status, s);
 }
 
 }  // namespace stepwise

@@ -48,13 +48,26 @@ struct StepPtrs {
   bool time_runs = false;
 };
 
+// Scratch for contractions that are split along K: a product with few output tiles and a long
+// contraction index would otherwise stream all of K through a handful of SMs.  Each part writes
+// its float32 tile here and a second kernel adds the parts in index order.
+struct SplitWs {
+  float* partial;        // device, partial_floats floats
+  size_t partial_floats;
+};
+
+// Parts gemm_bf16 splits the contraction index into, given scratch for partial_floats floats and
+// an output it can split for (a plain float32 store, no bias, rows that take float4); 1 = no
+// split, otherwise a second launch adds the parts.
+int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_floats);
+
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
 // [m][k]; lda / ldb are row strides in elements (multiples of 8).  `status` (device, nullable)
 // receives MEBPTT_ERR_TIMEOUT if a bounded wait expires.  early: the kernel may become resident
 // before the previous kernel of the stream has finished (it still waits for it before touching
 // memory).
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s, bool early = true);
+              int M, int N, int K, int* status, cudaStream_t s, bool early = true, const SplitWs* split = nullptr);
 
 }  // namespace tc
 

@@ -18,6 +18,8 @@
 // tcgen05.ld (warp w owns TMEM lanes 32w .. 32w+31 = tile rows) and write the tile.
 // Out-of-range parts of a tile are zero-filled by TMA on the way in and masked on the way out.
 // The sum over k runs in one fixed order, so results do not depend on how callers batch steps.
+#include <cstdlib>
+
 #include "launch.hpp"
 #include "sm100.cuh"
 #include "tc.hpp"
@@ -38,7 +40,8 @@ constexpr int gemm_smem(int stages, int bn) { return stages * (A_BYTES + bn * BK
 template <bool A_MN, bool B_MN, int BN = BN_WIDE>
 __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma,
                                                         const __grid_constant__ CUtensorMap tmb, GemmOut out,
-                                                        int M, int N, int K, int STAGES, int* status) {
+                                                        int M, int N, int K, int STAGES, int* status,
+                                                        float* partial) {
   constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
   static_assert(BN == BN_WIDE || (!A_MN && !B_MN), "narrow tiles exist for K-major operands only");
   extern __shared__ uint8_t smem_raw[];
@@ -49,7 +52,12 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int nk = (K + BK - 1) / BK;
+  // this CTA's part of the contraction index: blocks [kb_lo, kb_lo + nk) of 64
+  const int splits = gridDim.z;
+  const int nk_all = (K + BK - 1) / BK;
+  const int kb_lo = (int)((int64_t)nk_all * blockIdx.z / splits);
+  const int nk = (int)((int64_t)nk_all * (blockIdx.z + 1) / splits) - kb_lo;
+  const int tile = blockIdx.y * gridDim.x + blockIdx.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -78,16 +86,16 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
       ++armed;
       if (A_MN) {
-        tma_load_2d(sA, &tma, m0, kb * BK, &full[s]);
-        tma_load_2d(sA + 8192, &tma, m0 + 64, kb * BK, &full[s]);
+        tma_load_2d(sA, &tma, m0, (kb_lo + kb) * BK, &full[s]);
+        tma_load_2d(sA + 8192, &tma, m0 + 64, (kb_lo + kb) * BK, &full[s]);
       } else {
-        tma_load_2d(sA, &tma, kb * BK, m0, &full[s]);
+        tma_load_2d(sA, &tma, (kb_lo + kb) * BK, m0, &full[s]);
       }
       if (B_MN) {
-        tma_load_2d(sB, &tmb, n0, kb * BK, &full[s]);
-        tma_load_2d(sB + 8192, &tmb, n0 + 64, kb * BK, &full[s]);
+        tma_load_2d(sB, &tmb, n0, (kb_lo + kb) * BK, &full[s]);
+        tma_load_2d(sB + 8192, &tmb, n0 + 64, (kb_lo + kb) * BK, &full[s]);
       } else {
-        tma_load_2d(sB, &tmb, kb * BK, n0, &full[s]);
+        tma_load_2d(sB, &tmb, (kb_lo + kb) * BK, n0, &full[s]);
       }
     }
     (void)armed;
@@ -122,7 +130,29 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   __syncwarp();
   bool ok = mbar_wait(&done, 0);
   tc_fence_after_sync();
-  if (ok && !failed) {
+  bool finish = ok && !failed;
+  if (finish && splits > 1) {
+    // a part of a contraction split along K: the raw float32 tile goes to the scratch, and a
+    // second kernel adds the parts in index order
+    float* mine = partial + (((size_t)tile * splits + blockIdx.z) * BM + (size_t)(warp * 32 + lane)) * BN;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *(reinterpret_cast<float4*>(mine + c * 32) + j) =
+            make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                        __uint_as_float(r[4 * j + 3]));
+    }
+    finish = false;
+  }
+  auto load_acc = [&](int c, uint32_t (&r)[32]) {
+    tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+    tmem_ld_wait();
+  };
+  if (finish) {
     // Float32 tiles whose rows can be written as aligned float4: each warp parks its 32 x 128
     // block of the accumulator in the (now idle) operand ring, then writes -- or adds to -- one
     // whole 512-byte row of C per instruction.  Everything else takes the per-thread path below.
@@ -135,8 +165,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
-        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
-        tmem_ld_wait();
+        load_acc(c, r);
         float4* dst = reinterpret_cast<float4*>(park + (size_t)lane * PITCH + c * 32);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -192,8 +221,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
       uint32_t r[32];
-      tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
-      tmem_ld_wait();
+      load_acc(c, r);
       const int col0 = n0 + c * 32;
       if (out.kind == GemmOut::LOSS_DY) {
         // squared-error loss fused into the readout: this lane's row against its targets, columns in
@@ -283,7 +311,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       }
     }
     }
-  } else if (status && threadIdx.x == 0) {
+  } else if ((!ok || failed) && status && threadIdx.x == 0) {
     *status = MEBPTT_ERR_TIMEOUT;
   }
   // On the failure path the producer may still have loads in flight: give them a bounded
@@ -295,10 +323,54 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
   if (warp == 1) tmem_dealloc(tmem, BN);
 }
 
+// C[m][n] = sum over the parts, in index order, of a contraction that was split along K.
+// partial: [tile][part][128][bn] with tile = (m / 128) * tiles_x + n / bn.  One thread per four
+// adjacent columns.
+__global__ void splitk_reduce(const float* partial, int splits, int M, int N, int tiles_x, int bn, float* out, int64_t ld) {
+  grid_dep_wait();
+  grid_dep_launch();
+  const int n4 = (N + 3) / 4;
+  const size_t total = (size_t)M * n4;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const int m = (int)(e / n4), n = (int)(e % n4) * 4;
+    const int tile = (m / BM) * tiles_x + n / bn;
+    const float* p = partial + (((size_t)tile * splits) * BM + (size_t)(m % BM)) * bn + (n % bn);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int z = 0; z < splits; ++z) {
+      const float4 v = *reinterpret_cast<const float4*>(p + (size_t)z * BM * bn);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    float* q = out + (size_t)m * ld + n;
+    if (n + 3 < N) *reinterpret_cast<float4*>(q) = acc;
+    else {
+      const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+      for (int j = 0; j < 4 && n + j < N; ++j) q[j] = a[j];
+    }
+  }
+}
+
 }  // namespace
 
+// Few tiles and a long contraction index: split K so that about a wave of CTAs streams the
+// operands, each part at least 8 blocks of 64 long; a second kernel adds the parts.  Only where at
+// least four parts come out of it: below that the extra pass costs more than it saves.
+int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_floats) {
+  static const bool no_split = getenv("MEBPTT_NO_SPLITK") != nullptr;
+  if (no_split) return 1;
+  const int wide_tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
+  const bool narrow = !a_mn && !b_mn && wide_tiles <= 37 && N >= 2 * BN_NARROW;
+  const int BN = narrow ? BN_NARROW : BN_WIDE;
+  const int tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
+  const int nk = (K + BK - 1) / BK;
+  int want = 148 / tiles;
+  if (want > nk / 8) want = nk / 8;
+  if (want > 16) want = 16;
+  while (want > 1 && (size_t)tiles * want * BM * BN > partial_floats) --want;
+  return want >= 4 ? want : 1;
+}
+
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s, bool early) {
+              int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split) {
   if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
   // A short-and-wide product over K-major operands (a few steps' worth of rows against a whole
   // weight matrix) gives few 128-wide tiles, each streaming all of K through one SM: 32-wide tiles
@@ -314,6 +386,11 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
                    : make_tmap_2d(&tb, B, 2, (uint64_t)K, (uint64_t)N, (uint64_t)ldb * 2, 64, (uint32_t)BN));
   if (!ok) return MEBPTT_ERR_UNSUPPORTED;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  int splits = 1;
+  if (split && split->partial && out.kind == GemmOut::STORE_F32 && !out.bias && !out.perm_h && out.ld % 4 == 0 &&
+      (reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0)
+    splits = gemm_split_count(a_mn, b_mn, M, N, K, split->partial_floats);
+  grid.z = splits;
   static const bool attrs = [] {
     const int most = gemm_smem(MAX_STAGES, BN_WIDE);
     cudaFuncSetAttribute(gemm_bf16_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
@@ -327,14 +404,28 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   (void)attrs;
   // Large grids: 3 stages, two CTAs per SM, so that one CTA's epilogue overlaps the other's main
   // loop.  Grids of at most one wave: 6 stages, more loads in flight per CTA to hide their latency.
-  const int stages = (grid.x * grid.y <= 148) ? MAX_STAGES : 3;
+  const int stages = (grid.x * grid.y * grid.z <= 148) ? MAX_STAGES : 3;
   const int GEMM_SMEM = gemm_smem(stages, BN);
   auto* fn = narrow ? gemm_bf16_kernel<false, false, BN_NARROW>
              : a_mn ? (b_mn ? gemm_bf16_kernel<true, true> : gemm_bf16_kernel<true, false>)
                     : (b_mn ? gemm_bf16_kernel<false, true> : gemm_bf16_kernel<false, false>);
-  const cudaError_t e = launch_on(early, fn, grid, dim3(128), (size_t)GEMM_SMEM, s, ta, tb, out, M, N, K, stages, status);
-  if (e != cudaSuccess) cudaGetLastError();
-  return e == cudaSuccess ? MEBPTT_OK : MEBPTT_ERR_CUDA;
+  const cudaError_t e = launch_on(early, fn, grid, dim3(128), (size_t)GEMM_SMEM, s, ta, tb, out, M, N, K, stages, status,
+                                  splits > 1 ? split->partial : nullptr);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return MEBPTT_ERR_CUDA;
+  }
+  if (splits > 1) {
+    const size_t quads = (size_t)M * ((N + 3) / 4);
+    const int blocks = (int)((quads + 255) / 256 > 1184 ? 1184 : (quads + 255) / 256);
+    const cudaError_t e2 = launch_on(early, splitk_reduce, dim3(blocks), dim3(256), 0, s, (const float*)split->partial,
+                                     splits, M, N, (int)grid.x, BN, reinterpret_cast<float*>(out.ptr), out.ld);
+    if (e2 != cudaSuccess) {
+      cudaGetLastError();
+      return MEBPTT_ERR_CUDA;
+    }
+  }
+  return MEBPTT_OK;
 }
 
 }  // namespace tc
