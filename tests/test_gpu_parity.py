@@ -317,3 +317,35 @@ def test_c5_shape_truncated_two_layers_byte_budget(H):
     res = dp.run(plan)
     assert res["counters"][0] == plan.cost and res["counters"][2] <= m
     assert_bit_identical(res, full)
+
+
+def test_c4_full_size_properties(H):
+    """Config 4 as specified (I256 H1024 B32 t4000, float32 storage), where the oracle is out of
+    reach: ISM m = 50 against the full-memory run of the same problem, bit for bit, and the
+    executed forward count against the oracle's cost table."""
+    cfg = synth.CONFIGS["c4"]
+    dp = H.DeviceProblem(cfg)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][0] == cfg.t and full["counters"][3] == 0 and np.isfinite(full["loss"])
+    plan = dp.plan("ism", 50)
+    res = dp.run(plan)
+    assert res["counters"][0] == plan.cost == P.cost(P.ISM, cfg.t, 50)
+    assert res["counters"][1] == cfg.t and res["counters"][2] <= 50 and res["counters"][3] == 0
+    assert_bit_identical(res, full)
+
+
+def test_c5_full_size_properties(H):
+    """Config 5 as specified (two layers, I1024 H2048 B128 t1000, bf16) with the 1 GiB budget:
+    bit identity with the full-memory run, forward count equal to C(t, m), peak within budget."""
+    from paper_1606_03401_b200 import binding as B
+    cfg = synth.CONFIGS["c5"]
+    dp = H.DeviceProblem(cfg)
+    m = B.mebptt_budget_bytes_to_units(dp.desc, 1 << 30)
+    assert m == 341
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][0] == cfg.t and full["counters"][3] == 0 and np.isfinite(full["loss"])
+    plan = dp.plan("msm", m)
+    res = dp.run(plan)
+    assert res["counters"][0] == plan.cost == P.cost(P.MSM, cfg.t, m, alpha=4)
+    assert res["counters"][1] == cfg.t and res["counters"][2] <= m and res["counters"][3] == 0
+    assert_bit_identical(res, full)
