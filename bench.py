@@ -394,6 +394,33 @@ def main():
                "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3}
         del hws
 
+    # slot save / restore as an explicit copy: one internal state of this workload, and a large
+    # block, against the measured HBM copy rate (bytes read + bytes written)
+    slot_io = None
+    if rank == 0:
+        unit_b = B.mebptt_lstm_unit_bytes(dp.desc)
+        slot_io = []
+        for label, nbytes in (("one internal state (4 units)", 4 * unit_b), ("1 GiB", 1 << 30)):
+            a = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+            b_ = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+            reps = 20 if nbytes < (64 << 20) else 5
+            for _ in range(3):
+                B.mebptt_slot_copy(b_, a, nbytes, stream.cuda_stream)
+            ms_c = []
+            for _ in range(reps):
+                flush.fill_(1)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                B.mebptt_slot_copy(b_, a, nbytes, stream.cuda_stream)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ms_c.append(e0.elapsed_time(e1))
+            med = statistics.median(ms_c)
+            gbs = 2 * nbytes / (med * 1e-3) / 1e9
+            slot_io.append({"what": label, "bytes": nbytes, "us": med * 1e3, "GB_s": gbs,
+                            "frac_of_hbm_peak": gbs / pk["hbm_gbs"], "peak_GB_s": pk["hbm_gbs"]})
+            del a, b_
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = oracle_sample(synth.with_overrides(cfg, seed=cfg.seed), args.cpu_seconds)
@@ -413,7 +440,7 @@ def main():
                        "working_bytes_outside_budget": B.mebptt_lstm_working_bytes(dp.desc, plan),
                        "full_memory_arena_bytes": full.arena_units * unit,
                        "l2": "256 MiB buffer written between timed steps; x alone (131 MB at c3) exceeds L2",
-                       "replicas": world, "budgets": budgets},
+                       "replicas": world, "budgets": budgets, "slot_io": slot_io},
             "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * B.mebptt_lstm_launch_count(dp.desc, plan),
             "roofline": roofline, "cpu_baseline": cpu,
         }

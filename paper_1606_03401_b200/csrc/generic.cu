@@ -295,11 +295,6 @@ __global__ void finalize(const float* loss_t, int64_t t, float* loss, int64_t* c
   }
 }
 
-__global__ void copy16(uint4* dst, const uint4* src, size_t n) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-    dst[i] = src[i];
-}
-
 inline dim3 tiles(int M, int N) { return dim3((N + TN - 1) / TN, (M + TM - 1) / TM); }
 
 template <class T>
@@ -372,13 +367,5 @@ void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counter
                    const int* status, cudaStream_t s) {
   finalize<<<1, 32, 0, s>>>(loss_t, t, loss, counters, peak_units, status);
 }
-void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s) {
-  const size_t n = bytes / 16;
-  if (n == 0) return;
-  size_t blocks = (n + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  copy16<<<(unsigned)blocks, 256, 0, s>>>((uint4*)dst, (const uint4*)src, n);
-}
-
 }  // namespace generic
 }  // namespace mebptt

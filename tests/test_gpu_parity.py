@@ -149,14 +149,20 @@ def test_workspace_errors(H):
     assert e.value.status == B.MEBPTT_ERR_WORKSPACE
 
 
-def test_slot_copy(H):
+@pytest.mark.parametrize("nbytes", [16, 4096 + 16, (256 << 10) - 16, 256 << 10, (1 << 20) + 48, 393216 * 4,
+                                    (32 << 10) * 148 * 3 + 16, (200 << 20) + 32])
+def test_slot_copy(H, nbytes):
+    """Byte-exact copies: below and above the switch to bulk asynchronous copies, a ragged last
+    chunk, fewer chunks than SMs, several rounds per CTA; the bytes around the destination stay."""
     import torch
     from paper_1606_03401_b200 import binding as B
-    src = torch.randint(0, 255, ((1 << 20) + 48,), dtype=torch.uint8, device="cuda:0")
-    dst = torch.zeros_like(src)
-    B.mebptt_slot_copy(dst, src, src.numel(), torch.cuda.current_stream().cuda_stream)
+    g = torch.Generator(device="cuda:0").manual_seed(nbytes % 1000)
+    src = torch.randint(0, 255, (nbytes,), dtype=torch.uint8, device="cuda:0", generator=g)
+    dst = torch.full((nbytes + 512,), 7, dtype=torch.uint8, device="cuda:0")
+    B.mebptt_slot_copy(dst[256:256 + nbytes], src, nbytes, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
-    assert torch.equal(src, dst)
+    assert torch.equal(src, dst[256:256 + nbytes])
+    assert bool((dst[:256] == 7).all()) and bool((dst[256 + nbytes:] == 7).all())
 
 
 @pytest.mark.parametrize("shape", [dict(input=64, hidden=64, batch=64, t=40, readout=64),
