@@ -187,7 +187,10 @@ int mebptt_plan_validate(const mebptt_plan_t *plan);
  *
  * dtype selects storage and arithmetic:
  *   MEBPTT_FP32  everything float32, FMA arithmetic.
- *   MEBPTT_TF32  everything stored as float32; contractions on tensor cores.
+ *   MEBPTT_TF32  everything stored as float32; contractions on tensor cores (each float32
+ *                product as three bfloat16 products of 16-bit-mantissa halves, float32
+ *                accumulation: at least tf32 accuracy) where the widths are multiples of 8
+ *                and the batch a multiple of 32, in float32 FMA arithmetic elsewhere.
  *   MEBPTT_BF16  operands (W, W_out, x, h0 and every stored h and gate) bfloat16; b, b_out,
  *                targets, c0, every stored c, all accumulation and all gradients float32.
  * With these layouts an internal state (h_t, c_t, the four gates, h_{t-1}, c_{t-1}) fits in

@@ -79,6 +79,21 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     tcw.st_h = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_h);
     tcw.split = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), (size_t)148 * 128 * 128};
   }
+  stepwise3::Scratch x3{};
+  size_t w_off[16];
+  for (int l = 0; l < y.L; ++l) w_off[l] = y.w_layer_offset(l);
+  auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
+  if (y.stepwise_x3) {
+    x3.z = reinterpret_cast<float*>(ws + y.off_z);
+    x3.status = status;
+    x3.split = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), (size_t)148 * 128 * 128};
+    x3.S = y.S; x3.I0 = y.I;
+    x3.a3 = bf(y.off_a3); x3.w3 = bf(y.off_w3); x3.wmn3 = bf(y.off_wmn3);
+    x3.wout3 = bf(y.off_wout3); x3.woutmn3 = bf(y.off_woutmn3);
+    x3.st_dz3 = bf(y.off_st_dz); x3.st_in2 = bf(y.off_st_in); x3.st_hp2 = bf(y.off_st_hp);
+    x3.st_dy3 = bf(y.off_st_dy); x3.st_h3 = bf(y.off_st_h);
+  }
+  const bool staged = y.stepwise_tc || y.stepwise_x3;   // weight gradients per chunk of S steps
   int rc = MEBPTT_OK;
 
   cudaMemsetAsync(status, 0, 256, s);
@@ -90,6 +105,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   cudaMemsetAsync(io.db_out, 0, (size_t)y.O * 4, s);
   cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
 
+  if (y.stepwise_x3)
+    stepwise3::pack_weights(x3, y.L, y.I, y.H, y.O, reinterpret_cast<const float*>(io.W), w_off,
+                            reinterpret_cast<const float*>(io.W_out), s);
   for (const mebptt_op& op : p->tape) {
     if (rc != MEBPTT_OK) break;
     const int64_t k = op.k;
@@ -113,7 +131,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.plane_elems = plane_elems;
         a.B = y.B; a.H = y.H;
         a.counters = (l == 0) ? io.counters : nullptr;
-        if (y.stepwise_tc) rc = stepwise::forward_step(a, tcw, s);
+        if (y.stepwise_x3) rc = stepwise3::forward_step(a, x3, l, w_off[l], s);
+        else if (y.stepwise_tc) rc = stepwise::forward_step(a, tcw, s);
         else generic::forward_step(y.dtype, a, s);
         if (rc != MEBPTT_OK) break;
       }
@@ -128,8 +147,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
       r.loss_k = loss_t + (k - 1);
       r.dha = dha; r.dW_out = io.dW_out; r.db_out = io.db_out;
       r.B = y.B; r.H = y.H; r.O = y.O;
-      const int sidx = y.stepwise_tc ? (int)((k - 1) % y.S) : 0;
-      if (y.stepwise_tc) rc = stepwise::readout(r, tcw, sidx, s);
+      const int sidx = staged ? (int)((k - 1) % y.S) : 0;
+      if (y.stepwise_x3) rc = stepwise3::readout(r, x3, sidx, s);
+      else if (y.stepwise_tc) rc = stepwise::readout(r, tcw, sidx, s);
       else generic::readout(y.dtype, r, s);
       if (rc != MEBPTT_OK) break;
       for (int l = y.L - 1; l >= 0; --l) {
@@ -155,17 +175,17 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(k - 1) * y.B * y.I : nullptr);
         a.B = y.B; a.H = y.H;
         a.counters = (l == y.L - 1) ? io.counters : nullptr;
-        if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, l, sidx, s);
+        if (y.stepwise_x3) rc = stepwise3::backward_layer(a, x3, l, w_off[l], sidx, s);
+        else if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, l, sidx, s);
         else generic::backward_layer(y.dtype, a, s);
         if (rc != MEBPTT_OK) break;
       }
-      if (y.stepwise_tc && sidx == 0 && rc == MEBPTT_OK) {
+      if (staged && sidx == 0 && rc == MEBPTT_OK) {
         // the chunk's first step has been backpropagated: its weight gradients in one go
         const int64_t chunk = (k - 1) / y.S;
         const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
-        size_t w_off[16];
-        for (int l = 0; l < y.L; ++l) w_off[l] = y.w_layer_offset(l);
-        rc = stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+        rc = y.stepwise_x3 ? stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s)
+                           : stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
       }
     }
   }
@@ -248,6 +268,19 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
     const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs
     return p->cost * 3 * L + p->t * (3 + dha + bwd) + chunks * (2 * L + 1) + 1;
+  }
+  if (y.stepwise_x3) {
+    // weights: 2 packing kernels per layer and 2 for the readout; forward operation: split, GEMM,
+    // cell per layer; readout: split, GEMM, loss sum, split, db_out, dha GEMM; backward operation
+    // per layer: gate kernel, db, one or two d_in GEMMs; a chunk: 3 GEMMs per product
+    const size_t pf = (size_t)148 * 128 * 128;
+    const int G = 4 * y.H;
+    const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, 3 * G, pf) > 1 ? 2 : 1;
+    const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, 3 * G, pf) > 1 ? 2 : 1;
+    const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, 3 * y.O, pf) > 1 ? 2 : 1;
+    const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    const int64_t chunks = (p->t + y.S - 1) / y.S;
+    return 2 * L + 2 + p->cost * 3 * L + p->t * (5 + dha + bwd) + chunks * 3 * (2 * L + 1) + 1;
   }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }

@@ -99,4 +99,34 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
                 float* dW_out, cudaStream_t s);
 }  // namespace stepwise
+
+// The same for float32 storage (MEBPTT_TF32): operands split into two bfloat16 halves, three
+// bfloat16 products per float32 product.
+namespace stepwise3 {
+struct Scratch {
+  float* z;                  // [B][4H]
+  int* status;
+  tc::SplitWs split;
+  int S, I0;
+  __nv_bfloat16* a3;         // [B][3 (I + H)]: the forward operation's left operand
+  __nv_bfloat16* w3;         // per layer at 3 * (element offset of the layer): [4H][3K], [hi | mid | hi]
+  __nv_bfloat16* wmn3;       // likewise [3 * 4H][K], [hi ; mid ; hi]
+  __nv_bfloat16* wout3;      // [O][3H]
+  __nv_bfloat16* woutmn3;    // [3 O][H]
+  // stages of one chunk of S steps, row block (k - 1) % S of B rows per step
+  __nv_bfloat16* st_dz3;     // [L][S B][3 * 4H]  [hi | hi | mid]
+  __nv_bfloat16* st_in2;     // layer 0: [S B][2 I0]; layers l > 0: [S B][2H] each, after it; [hi | mid]
+  __nv_bfloat16* st_hp2;     // [L][S B][2H]
+  __nv_bfloat16* st_dy3;     // [S B][3 O]
+  __nv_bfloat16* st_h3;      // [S B][3 H]  top layer h_k
+};
+// W: all layers' weights (float32), w_off[l] the element offset of layer l
+void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W, const size_t* w_off,
+                  const float* W_out, cudaStream_t s);
+int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_off, cudaStream_t s);
+int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s);
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_off, int sidx, cudaStream_t s);
+int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
+                float* dW_out, cudaStream_t s);
+}  // namespace stepwise3
 }  // namespace mebptt

@@ -29,6 +29,7 @@ struct Layout {
   int64_t t = 0;
   bool tensor_path = false;
   bool stepwise_tc = false;   // step-by-step operations with their contractions on the tensor cores
+  bool stepwise_x3 = false;   // likewise for float32 storage, operands split into bfloat16 halves
   size_t esz = 0;        // bytes of one operand element
   size_t granule = 0;
   size_t hsz = 0;        // one layer's h
@@ -48,6 +49,7 @@ struct Layout {
   // tensor-core path: packed weights, staging of S consecutive time steps, control
   int S = 0;             // time steps per staged chunk
   size_t off_wp_ih = 0, off_wp_hh = 0, off_wpT_hh = 0, off_wpT_ih = 0, off_bias_p = 0, off_woutT = 0;
+  size_t off_a3 = 0, off_w3 = 0, off_wmn3 = 0, off_wout3 = 0, off_woutmn3 = 0;
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
@@ -103,11 +105,20 @@ inline bool stepwise_tc_supported(const mebptt_lstm_desc* d) {
          (d->batch / 32) * ((d->readout + 31) / 32) <= 4096;
 }
 
+// Float32 storage with tensor-core contractions (MEBPTT_TF32): the same step-by-step scheme over
+// operands split into bfloat16 halves.
+inline bool stepwise_x3_supported(const mebptt_lstm_desc* d) {
+  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && d->dtype == MEBPTT_TF32 && d->batch % 32 == 0 &&
+         d->input % 8 == 0 && d->hidden % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
+         (d->batch / 32) * ((d->readout + 31) / 32) <= 4096;
+}
+
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
   y.dtype = d->dtype; y.t = d->t;
   y.tensor_path = tensor_path_supported(d);
   y.stepwise_tc = stepwise_tc_supported(d);
+  y.stepwise_x3 = stepwise_x3_supported(d);
   y.esz = (d->dtype == MEBPTT_BF16) ? 2 : 4;
   const size_t row = (size_t)y.H * y.esz;
   y.granule = 256 / gcd_sz(256, row) * row;  // lcm(256, row bytes)
@@ -212,6 +223,24 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_st_h = take(rows * y.H * 2);
       // split-K scratch: at most a wave of 128 x 128 float32 tiles
       y.off_split = take((size_t)148 * 128 * 128 * 4);
+    }
+    if (y.stepwise_x3) {
+      const size_t G = 4 * (size_t)y.H, Kmax = (size_t)(y.I > y.H ? y.I : y.H) + y.H;
+      y.n_loss_part = (y.B / 32) * ((y.O + 31) / 32);
+      y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
+      const size_t rows = (size_t)y.S * y.B;
+      y.off_z = take((size_t)y.B * G * 4);
+      y.off_split = take((size_t)148 * 128 * 128 * 4);
+      y.off_a3 = take((size_t)y.B * 3 * Kmax * 2);
+      y.off_w3 = take(3 * y.w_total_elems() * 2);
+      y.off_wmn3 = take(3 * y.w_total_elems() * 2);
+      y.off_wout3 = take((size_t)3 * y.O * y.H * 2);
+      y.off_woutmn3 = take((size_t)3 * y.O * y.H * 2);
+      y.off_st_dz = take((size_t)y.L * rows * 3 * G * 2);
+      y.off_st_in = take(rows * 2 * y.I * 2 + (size_t)(y.L - 1) * rows * 2 * y.H * 2);
+      y.off_st_hp = take((size_t)y.L * rows * 2 * y.H * 2);
+      y.off_st_dy = take(rows * 3 * y.O * 2);
+      y.off_st_h = take(rows * 3 * y.H * 2);
     }
     y.off_loss_part = take((size_t)y.n_loss_part * 4);
     y.off_status = take(256);

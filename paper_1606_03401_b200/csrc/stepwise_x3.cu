@@ -1,0 +1,270 @@
+// Step-by-step LSTM operations for float32 storage with every contraction on the tensor cores
+// (MEBPTT_TF32).
+//
+// A float32 value v is split into two bfloat16 numbers, hi = bf16(v) and mid = bf16(v - hi), which
+// together carry 16 bits of mantissa.  A product of two such values is taken as
+//     a b  ~=  a_hi b_hi + a_hi b_mid + a_mid b_hi
+// (the dropped term is 2^-18 relative), accumulated in float32: better than a tf32 product, at
+// three bfloat16 MMAs.  The three terms are one contraction over a tripled index: the left
+// operand is laid out [hi | hi | mid] along K and the right operand [hi | mid | hi], so the
+// bfloat16 GEMM is used as it is.  Weights are split once per training step, activations and
+// gradients where they are produced.
+//
+// Operations (per layer), with K = I + H, G = 4H:
+//   forward    a3 = split([in ; h_prev]) ; z = a3 W3^T + b ; gates, c, h from z
+//   readout    h3 = split(h) ; y = h3 Wout3^T + b_out with loss and dy (float32) in the epilogue ;
+//              dy3 = split(dy) ; db_out += sum_b dy ; dha = dy3 WoutMN3
+//   backward   dz (float32) and dz3 from the stored gates ; db += sum_b dz ; d_in = dz3 WMN3
+//   per chunk  dW += dz^T [in ; h_prev], dW_out += dy^T h from the staged halves: three GEMMs per
+//              product (hi hi, hi mid, mid hi)
+// All sums run in a fixed order and nothing depends on the plan: results are bit-identical across
+// plans.
+#include "kernels.hpp"
+#include "tc.hpp"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace mebptt {
+namespace stepwise3 {
+
+namespace {
+
+using tc::GemmOut;
+using tc::gemm_bf16;
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf(-a)); }
+__device__ __forceinline__ void split2(float v, bf16& hi, bf16& mid) {
+  hi = __float2bfloat16_rn(v);
+  mid = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
+
+// out [R][3C] = [hi | mid | hi] of W [R][C]: the right operand of a contraction over columns.
+__global__ void pack3_cols(const float* W, int R, int C, bf16* out) {
+  const size_t n = (size_t)R * C;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = e / C, c = e % C;
+    bf16 hi, mid;
+    split2(W[e], hi, mid);
+    bf16* o = out + r * 3 * (size_t)C + c;
+    o[0] = hi; o[C] = mid; o[2 * (size_t)C] = hi;
+  }
+}
+// out [3R][C] = [hi ; mid ; hi] of W [R][C]: the right operand of a contraction over rows.
+__global__ void pack3_rows(const float* W, int R, int C, bf16* out) {
+  const size_t n = (size_t)R * C;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    bf16 hi, mid;
+    split2(W[e], hi, mid);
+    out[e] = hi; out[n + e] = mid; out[2 * n + e] = hi;
+  }
+}
+// out [B][3 (Ca + Cb)] = [hi | hi | mid] of the rows [a[b] ; b_[b]] (b_ may be NULL with Cb = 0):
+// the left operand of a contraction over columns.
+__global__ void split_a3(const float* a, int Ca, const float* b_, int Cb, int B, bf16* out) {
+  const int C = Ca + Cb;
+  const size_t n = (size_t)B * C;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = e / C;
+    const int c = (int)(e % C);
+    const float v = c < Ca ? a[r * Ca + c] : b_[r * Cb + (c - Ca)];
+    bf16 hi, mid;
+    split2(v, hi, mid);
+    bf16* o = out + r * 3 * (size_t)C + c;
+    o[0] = hi; o[C] = hi; o[2 * (size_t)C] = mid;
+  }
+}
+
+__global__ void cell_fwd(const float* z, const float* c_prev, const float* h_prev, float* h_out, float* c_out,
+                         float* gates, size_t plane, float* h_in_copy, float* c_in_copy, int B, int H,
+                         int64_t* counters) {
+  const size_t n = (size_t)B * H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / H), j = (int)(e % H);
+    const float* row = z + (size_t)b * 4 * H;
+    const float gi = sigmoidf_(row[j]), gf = sigmoidf_(row[H + j]);
+    const float gg = tanhf(row[2 * H + j]), go = sigmoidf_(row[3 * H + j]);
+    const float cp = c_prev[e];
+    const float c = fmaf(gf, cp, gi * gg);
+    c_out[e] = c;
+    h_out[e] = go * tanhf(c);
+    if (gates) { gates[e] = gi; gates[plane + e] = gf; gates[2 * plane + e] = gg; gates[3 * plane + e] = go; }
+    if (h_in_copy) { h_in_copy[e] = h_prev[e]; c_in_copy[e] = cp; }
+  }
+  if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[0] += 1;
+}
+
+// Gate derivatives: dz [B][4H] float32 (for db), dz3 rows [hi | hi | mid] in the stage (left operand
+// of dz W and of the chunk's dW), and the halves [hi | mid] of this step's layer input and h_{k-1}.
+__global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const float* gates, size_t plane,
+                         const float* c_t, const float* c_prev, float* dz, bf16* dz3, int B, int H, int64_t* counters,
+                         const float* in, int I, bf16* st_in2, const float* hp, bf16* st_hp2) {
+  const size_t n = (size_t)B * H;
+  const size_t G = 4 * (size_t)H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / H), j = (int)(e % H);
+    const float gi = gates[e], gf = gates[plane + e], gg = gates[2 * plane + e], go = gates[3 * plane + e];
+    const float dh = dha[e] + dh_rec[e];
+    const float th = tanhf(c_t[e]);
+    const float d_o = dh * th;
+    const float dc = fmaf(dh * go, 1.f - th * th, dc_rec[e]);
+    const float v[4] = {dc * gg * gi * (1.f - gi), dc * c_prev[e] * gf * (1.f - gf), dc * gi * (1.f - gg * gg),
+                        d_o * go * (1.f - go)};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const size_t col = (size_t)q * H + j;
+      dz[(size_t)b * G + col] = v[q];
+      bf16 hi, mid;
+      split2(v[q], hi, mid);
+      bf16* o = dz3 + (size_t)b * 3 * G + col;
+      o[0] = hi; o[G] = hi; o[2 * G] = mid;
+    }
+    dc_rec[e] = dc * gf;
+    // h_{k-1}: same index space
+    bf16 hi, mid;
+    split2(hp[e], hi, mid);
+    st_hp2[(size_t)b * 2 * H + j] = hi;
+    st_hp2[(size_t)b * 2 * H + H + j] = mid;
+  }
+  const size_t ni = (size_t)B * I;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < ni; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t b = e / I, c = e % I;
+    bf16 hi, mid;
+    split2(in[e], hi, mid);
+    st_in2[b * 2 * I + c] = hi;
+    st_in2[b * 2 * I + I + c] = mid;
+  }
+  if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
+}
+
+template <class T>
+__global__ void colsum_accum(const T* v, int B, int N, float* out) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += (float)v[(size_t)b * N + n];
+  out[n] += s;
+}
+
+__global__ void sum_parts(const float* part, int n, float* out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < n; ++i) s += part[i];
+    *out = s;
+  }
+}
+
+}  // namespace
+
+void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W, const size_t* w_off,
+                  const float* W_out, cudaStream_t s) {
+  const int G = 4 * H;
+  for (int l = 0; l < L; ++l) {
+    const int K = (l == 0 ? I0 : H) + H;
+    const size_t n = (size_t)G * K;
+    pack3_cols<<<ew_blocks(n), 256, 0, s>>>(W + w_off[l], G, K, w.w3 + 3 * w_off[l]);
+    pack3_rows<<<ew_blocks(n), 256, 0, s>>>(W + w_off[l], G, K, w.wmn3 + 3 * w_off[l]);
+  }
+  const size_t no = (size_t)O * H;
+  pack3_cols<<<ew_blocks(no), 256, 0, s>>>(W_out, O, H, w.wout3);
+  pack3_rows<<<ew_blocks(no), 256, 0, s>>>(W_out, O, H, w.woutmn3);
+}
+
+int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_off, cudaStream_t s) {
+  const int K = a.I + a.H, G = 4 * a.H;
+  const size_t nk = (size_t)a.B * K;
+  split_a3<<<ew_blocks(nk), 256, 0, s>>>((const float*)a.in, a.I, (const float*)a.h_prev, a.H, a.B, w.a3);
+  int rc = gemm_bf16(w.a3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0},
+                     a.B, G, 3 * K, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  const size_t n = (size_t)a.B * a.H;
+  cell_fwd<<<ew_blocks(n), 256, 0, s>>>(w.z, a.c_prev, (const float*)a.h_prev, (float*)a.h_out, a.c_out, (float*)a.gates,
+                                        a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
+  (void)l;
+  return MEBPTT_OK;
+}
+
+int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s) {
+  bf16* h3 = w.st_h3 + (size_t)sidx * a.B * 3 * a.H;
+  bf16* dy3 = w.st_dy3 + (size_t)sidx * a.B * 3 * a.O;
+  const size_t nh = (size_t)a.B * a.H, no = (size_t)a.B * a.O;
+  split_a3<<<ew_blocks(nh), 256, 0, s>>>((const float*)a.h, a.H, nullptr, 0, a.B, h3);
+  GemmOut o{GemmOut::LOSS_DY, nullptr, a.O, a.b_out, 0};
+  o.target = a.target;
+  o.dy32 = a.dy;
+  o.loss_part = a.loss_part;
+  o.parts = (a.O + 31) / 32;
+  o.scale = 1.f / ((float)a.B * (float)a.O);
+  int rc = gemm_bf16(h3, 3 * a.H, false, w.wout3, 3 * a.H, false, o, a.B, a.O, 3 * a.H, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  sum_parts<<<1, 32, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k);
+  split_a3<<<ew_blocks(no), 256, 0, s>>>(a.dy, a.O, nullptr, 0, a.B, dy3);
+  colsum_accum<float><<<(a.O + 127) / 128, 128, 0, s>>>(a.dy, a.B, a.O, a.db_out);
+  // dha[b][j] = sum_o dy[b][o] W_out[o][j]
+  return gemm_bf16(dy3, 3 * a.O, false, w.woutmn3, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B,
+                   a.H, 3 * a.O, w.status, s, true, &w.split);
+}
+
+int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_off, int sidx, cudaStream_t s) {
+  const int K = a.I + a.H, G = 4 * a.H;
+  const size_t n = (size_t)a.B * a.H;
+  const size_t rows = (size_t)w.S * a.B;
+  bf16* dz3 = w.st_dz3 + ((size_t)l * rows + (size_t)sidx * a.B) * 3 * G;
+  bf16* in2 = w.st_in2 + (l == 0 ? 0 : rows * 2 * w.I0 + (size_t)(l - 1) * rows * 2 * a.H) + (size_t)sidx * a.B * 2 * a.I;
+  bf16* hp2 = w.st_hp2 + ((size_t)l * rows + (size_t)sidx * a.B) * 2 * a.H;
+  gate_bwd<<<ew_blocks(n), 256, 0, s>>>(a.dha, a.dh_rec, a.dc_rec, (const float*)a.gates, a.plane_elems, a.c_t, a.c_prev,
+                                        a.dz, dz3, a.B, a.H, a.counters, (const float*)a.in, a.I, in2,
+                                        (const float*)a.h_prev, hp2);
+  colsum_accum<float><<<(G + 127) / 128, 128, 0, s>>>(a.dz, a.B, G, a.db);
+  const bf16* WMN = w.wmn3 + 3 * w_off;   // [3G][K]
+  if (a.d_lo) {
+    int rc = gemm_bf16(dz3, 3 * G, false, WMN, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I,
+                       3 * G, w.status, s, true, &w.split);
+    if (rc != MEBPTT_OK) return rc;
+  }
+  return gemm_bf16(dz3, 3 * G, false, WMN + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B,
+                   a.H, 3 * G, w.status, s, true, &w.split);
+}
+
+namespace {
+// C[m][n] += sum_r (a_hi a_mid)[r][m] (b_hi b_mid)[r][n] as hi hi + hi mid + mid hi; a3 rows are
+// [hi | hi | mid] of width Ma, b2 rows [hi | mid] of width Nb.
+int accum3(const bf16* a3, int Ma, const bf16* b2, int Nb, bool b_is_a3, float* C, int64_t ldc, int R, int* status,
+           cudaStream_t s) {
+  const int64_t lda = 3 * (int64_t)Ma, ldb = (b_is_a3 ? 3 : 2) * (int64_t)Nb;
+  const bf16* a_hi = a3;
+  const bf16* a_mid = a3 + 2 * (size_t)Ma;
+  const bf16* b_hi = b2;
+  const bf16* b_mid = b2 + (b_is_a3 ? 2 : 1) * (size_t)Nb;
+  const GemmOut o{GemmOut::ACCUM_F32, C, ldc, nullptr, 0};
+  int rc = gemm_bf16(a_hi, lda, true, b_hi, ldb, true, o, Ma, Nb, R, status, s);
+  if (rc != MEBPTT_OK) return rc;
+  rc = gemm_bf16(a_hi, lda, true, b_mid, ldb, true, o, Ma, Nb, R, status, s);
+  if (rc != MEBPTT_OK) return rc;
+  return gemm_bf16(a_mid, lda, true, b_hi, ldb, true, o, Ma, Nb, R, status, s);
+}
+}  // namespace
+
+int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
+                float* dW_out, cudaStream_t s) {
+  const int G = 4 * H, R = steps * B;
+  const size_t rows = (size_t)w.S * B;
+  for (int l = 0; l < L; ++l) {
+    const int I = l == 0 ? I0 : H, K = I + H;
+    const bf16* dz3 = w.st_dz3 + (size_t)l * rows * 3 * G;
+    const bf16* in2 = w.st_in2 + (l == 0 ? 0 : rows * 2 * I0 + (size_t)(l - 1) * rows * 2 * H);
+    const bf16* hp2 = w.st_hp2 + (size_t)l * rows * 2 * H;
+    float* dWl = dW + w_off[l];
+    int rc = accum3(dz3, G, in2, I, false, dWl, K, R, w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+    rc = accum3(dz3, G, hp2, H, false, dWl + I, K, R, w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+  }
+  return accum3(w.st_dy3, O, w.st_h3, H, true, dW_out, H, R, w.status, s);
+}
+
+}  // namespace stepwise3
+}  // namespace mebptt

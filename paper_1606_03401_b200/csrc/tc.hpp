@@ -23,6 +23,7 @@ struct GemmOut {
   // ptr receives dy = 2 d scale in bfloat16 and loss_part[(m / 32) * parts + n / 32] the sum of
   // d * d * scale over that 32 x 32 block, in a fixed order (rows of M in groups of 32).
   const float* target = nullptr;   // [M][ld]
+  float* dy32 = nullptr;           // optional: dy in float32 as well, [M][ld] (ptr may then be NULL)
   float* loss_part = nullptr;
   int parts = 0;                   // ceil(N / 32)
   float scale = 0.f;

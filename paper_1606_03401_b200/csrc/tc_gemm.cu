@@ -231,8 +231,9 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
           const float* tp = out.target + (size_t)row * out.ld + col0;
           __nv_bfloat16* dp = reinterpret_cast<__nv_bfloat16*>(out.ptr) + (size_t)row * out.ld + col0;
           const float two = 2.f * out.scale;
+          float* d32 = out.dy32 ? out.dy32 + (size_t)row * out.ld + col0 : nullptr;
           if (col0 + 32 <= N && ((reinterpret_cast<uintptr_t>(tp) & 15) == 0) && ((reinterpret_cast<uintptr_t>(dp) & 15) == 0) &&
-              ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0)) {
+              ((reinterpret_cast<uintptr_t>(out.bias) & 15) == 0) && ((reinterpret_cast<uintptr_t>(d32) & 15) == 0)) {
             float4 t4[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) t4[j] = *reinterpret_cast<const float4*>(tp + 4 * j);
@@ -248,17 +249,21 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
               sq = fmaf(d0, d0, sq); sq = fmaf(d1, d1, sq); sq = fmaf(d2, d2, sq); sq = fmaf(d3, d3, sq);
               packed[2 * j] = pack_bf16x2(d0 * two, d1 * two);
               packed[2 * j + 1] = pack_bf16x2(d2 * two, d3 * two);
+              if (d32) *reinterpret_cast<float4*>(d32 + 4 * j) = make_float4(d0 * two, d1 * two, d2 * two, d3 * two);
             }
+            if (out.ptr) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              *reinterpret_cast<uint4*>(dp + 8 * j) = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+              for (int j = 0; j < 4; ++j)
+                *reinterpret_cast<uint4*>(dp + 8 * j) = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+            }
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (col0 + j < N) {
                 const float d = (__uint_as_float(r[j]) + (out.bias ? out.bias[col0 + j] : 0.f)) - tp[j];
                 sq = fmaf(d, d, sq);
-                dp[j] = __float2bfloat16_rn(d * two);
+                if (out.ptr) dp[j] = __float2bfloat16_rn(d * two);
+                if (d32) d32[j] = d * two;
               }
           }
         }

@@ -245,6 +245,33 @@ def test_stepwise_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
     assert_bit_identical(res, full)
 
 
+@pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=21, readout=40),
+                                   dict(layers=1, input=24, hidden=256, batch=96, t=13, readout=8),
+                                   dict(layers=1, input=128, hidden=1152, batch=32, t=9, readout=64)])
+def test_float32_storage_on_tensor_cores_matches_oracle_within_1e_4(H, shape):
+    """The tf32 data type: float32 storage, contractions on the tensor cores as three bfloat16
+    products per float32 product.  Oracle parity at the float32 tolerance, bit identity across
+    plans, agreement with the float32 FMA kernels."""
+    from paper_1606_03401_b200 import binding as B
+    from tests.util import rel_l2
+    cfg = _cfg("c4", **shape)
+    assert cfg.dtype == "tf32"
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    ref = oracle_run(dp.prob)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][3] == 0
+    assert_close_to_oracle(full, ref, "tf32", want_dx=True)
+    for mode, m, beta in [("hsm", 1, 0), ("hsm", 4, 0), ("ism", 2, 0), ("msm", 9, 0), ("msm", 13, 3)]:
+        plan = dp.plan(mode, m, beta=beta)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+        assert_bit_identical(res, full, want_dx=True)
+    slow = H.DeviceProblem(cfg, dp.prob, want_dx=True, flags=B.MEBPTT_FLAG_NO_TENSOR_CORES)
+    other = slow.run(slow.full_memory_plan())
+    for k in ("dW", "db", "dW_out", "db_out", "dx"):
+        assert rel_l2(full[k], other[k]) < 1e-4, k
+
+
 def test_c2_full_size_every_budget(H):
     """Config 2 as timed: I512 H512 B64 t256 bf16, HSM and ISM at m = 16, 64, 256."""
     cfg = synth.CONFIGS["c2"]
