@@ -17,6 +17,8 @@
 // db is summed from the unrounded dz.  Every sum has a fixed order, and an operation's launches
 // do not depend on the plan, so results are bit-identical across plans.
 #include "kernels.hpp"
+#include "launch.hpp"
+#include "sm100.cuh"
 #include "tc.hpp"
 
 #include <cuda_bf16.h>
@@ -38,6 +40,8 @@ __device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf
 __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
                          bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H,
                          int64_t* counters) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
@@ -66,6 +70,8 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
                          const float* c_t, const float* c_prev, float* dz, bf16* dz16, int B, int H,
                          int64_t* counters, const uint4* in, uint4* st_in, size_t n_in16, const uint4* hp,
                          uint4* st_hp, size_t n_hp16) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_in16; e += (size_t)gridDim.x * blockDim.x)
     st_in[e] = in[e];
@@ -95,6 +101,8 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
 // out[n] += sum_b v[b][n], b ascending
 template <class T>
 __global__ void colsum_accum(const T* v, int B, int N, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= N) return;
   float s = 0.f;
@@ -105,6 +113,8 @@ __global__ void colsum_accum(const T* v, int B, int N, float* out) {
 // Loss term of one step from its partial sums (block 0, one thread); every block helps copy the
 // top layer's h_k to its stage.
 __global__ void sum_parts_stage_h(const float* part, int n, float* out, const uint4* h, uint4* st_h, size_t n_h16) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_h16; e += (size_t)gridDim.x * blockDim.x)
     st_h[e] = h[e];
   if (threadIdx.x == 0 && blockIdx.x == 0) {
@@ -128,7 +138,7 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
                  a.H, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
-  cell_fwd<<<ew_blocks(n), 256, 0, s>>>(w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
+  launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
                                         a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
   return MEBPTT_OK;
 }
@@ -144,13 +154,13 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   int rc = gemm_bf16(a.h, a.H, false, W_out, a.H, false, o, a.B, a.O, a.H, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
   const size_t n_h16 = (size_t)a.B * a.H * 2 / 16;
-  sum_parts_stage_h<<<ew_blocks(n_h16 * 8), 256, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k, (const uint4*)a.h,
+  launch_pdl(sum_parts_stage_h, dim3(ew_blocks(n_h16 * 8)), dim3(256), 0, s, a.loss_part, (a.B / 32) * o.parts, a.loss_k, (const uint4*)a.h,
                                                           (uint4*)(w.st_h + (size_t)sidx * a.B * a.H), n_h16);
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]: W_out read as the [k][n] operand
   rc = gemm_bf16(dy16, a.O, false, W_out, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B, a.H,
                  a.O, w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
-  colsum_accum<bf16><<<(a.O + 127) / 128, 128, 0, s>>>(dy16, a.B, a.O, a.db_out);
+  launch_pdl(colsum_accum<bf16>, dim3((a.O + 127) / 128), dim3(128), 0, s, dy16, a.B, a.O, a.db_out);
   return MEBPTT_OK;
 }
 
@@ -162,11 +172,11 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
   bf16* dz16 = w.st_dz + ((size_t)l * rows + (size_t)sidx * a.B) * G;
   bf16* st_in = w.st_in + (l == 0 ? 0 : rows * w.I0 + (size_t)(l - 1) * rows * a.H) + (size_t)sidx * a.B * a.I;
   bf16* st_hp = w.st_hp + ((size_t)l * rows + (size_t)sidx * a.B) * a.H;
-  gate_bwd<<<ew_blocks(n), 256, 0, s>>>(a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
+  launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
                                         a.dz, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
                                         (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
                                         (size_t)a.B * a.H * 2 / 16);
-  colsum_accum<float><<<(G + 127) / 128, 128, 0, s>>>(a.dz, a.B, G, a.db);
+  launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, a.dz, a.B, G, a.db);
   // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
   if (a.d_lo) {
     int rc = gemm_bf16(dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,

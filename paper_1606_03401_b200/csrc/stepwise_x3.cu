@@ -20,6 +20,8 @@
 // All sums run in a fixed order and nothing depends on the plan: results are bit-identical across
 // plans.
 #include "kernels.hpp"
+#include "launch.hpp"
+#include "sm100.cuh"
 #include "tc.hpp"
 
 #include <cuda_bf16.h>
@@ -44,6 +46,8 @@ inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n
 
 // out [R][3C] = [hi | mid | hi] of W [R][C]: the right operand of a contraction over columns.
 __global__ void pack3_cols(const float* W, int R, int C, bf16* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)R * C;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const size_t r = e / C, c = e % C;
@@ -55,6 +59,8 @@ __global__ void pack3_cols(const float* W, int R, int C, bf16* out) {
 }
 // out [3R][C] = [hi ; mid ; hi] of W [R][C]: the right operand of a contraction over rows.
 __global__ void pack3_rows(const float* W, int R, int C, bf16* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)R * C;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     bf16 hi, mid;
@@ -65,6 +71,8 @@ __global__ void pack3_rows(const float* W, int R, int C, bf16* out) {
 // out [B][3 (Ca + Cb)] = [hi | hi | mid] of the rows [a[b] ; b_[b]] (b_ may be NULL with Cb = 0):
 // the left operand of a contraction over columns.
 __global__ void split_a3(const float* a, int Ca, const float* b_, int Cb, int B, bf16* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const int C = Ca + Cb;
   const size_t n = (size_t)B * C;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
@@ -81,6 +89,8 @@ __global__ void split_a3(const float* a, int Ca, const float* b_, int Cb, int B,
 __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_prev, float* h_out, float* c_out,
                          float* gates, size_t plane, float* h_in_copy, float* c_in_copy, int B, int H,
                          int64_t* counters) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
@@ -102,6 +112,8 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_pre
 __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const float* gates, size_t plane,
                          const float* c_t, const float* c_prev, float* dz, bf16* dz3, int B, int H, int64_t* counters,
                          const float* in, int I, bf16* st_in2, const float* hp, bf16* st_hp2) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   const size_t G = 4 * (size_t)H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
@@ -142,6 +154,8 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
 
 template <class T>
 __global__ void colsum_accum(const T* v, int B, int N, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= N) return;
   float s = 0.f;
@@ -150,6 +164,8 @@ __global__ void colsum_accum(const T* v, int B, int N, float* out) {
 }
 
 __global__ void sum_parts(const float* part, int n, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     float s = 0.f;
     for (int i = 0; i < n; ++i) s += part[i];
@@ -165,23 +181,23 @@ void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W,
   for (int l = 0; l < L; ++l) {
     const int K = (l == 0 ? I0 : H) + H;
     const size_t n = (size_t)G * K;
-    pack3_cols<<<ew_blocks(n), 256, 0, s>>>(W + w_off[l], G, K, w.w3 + 3 * w_off[l]);
-    pack3_rows<<<ew_blocks(n), 256, 0, s>>>(W + w_off[l], G, K, w.wmn3 + 3 * w_off[l]);
+    launch_pdl(pack3_cols, dim3(ew_blocks(n)), dim3(256), 0, s, W + w_off[l], G, K, w.w3 + 3 * w_off[l]);
+    launch_pdl(pack3_rows, dim3(ew_blocks(n)), dim3(256), 0, s, W + w_off[l], G, K, w.wmn3 + 3 * w_off[l]);
   }
   const size_t no = (size_t)O * H;
-  pack3_cols<<<ew_blocks(no), 256, 0, s>>>(W_out, O, H, w.wout3);
-  pack3_rows<<<ew_blocks(no), 256, 0, s>>>(W_out, O, H, w.woutmn3);
+  launch_pdl(pack3_cols, dim3(ew_blocks(no)), dim3(256), 0, s, W_out, O, H, w.wout3);
+  launch_pdl(pack3_rows, dim3(ew_blocks(no)), dim3(256), 0, s, W_out, O, H, w.woutmn3);
 }
 
 int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_off, cudaStream_t s) {
   const int K = a.I + a.H, G = 4 * a.H;
   const size_t nk = (size_t)a.B * K;
-  split_a3<<<ew_blocks(nk), 256, 0, s>>>((const float*)a.in, a.I, (const float*)a.h_prev, a.H, a.B, w.a3);
+  launch_pdl(split_a3, dim3(ew_blocks(nk)), dim3(256), 0, s, (const float*)a.in, a.I, (const float*)a.h_prev, a.H, a.B, w.a3);
   int rc = gemm_bf16(w.a3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0},
                      a.B, G, 3 * K, w.status, s);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
-  cell_fwd<<<ew_blocks(n), 256, 0, s>>>(w.z, a.c_prev, (const float*)a.h_prev, (float*)a.h_out, a.c_out, (float*)a.gates,
+  launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const float*)a.h_prev, (float*)a.h_out, a.c_out, (float*)a.gates,
                                         a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
   (void)l;
   return MEBPTT_OK;
@@ -191,7 +207,7 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   bf16* h3 = w.st_h3 + (size_t)sidx * a.B * 3 * a.H;
   bf16* dy3 = w.st_dy3 + (size_t)sidx * a.B * 3 * a.O;
   const size_t nh = (size_t)a.B * a.H, no = (size_t)a.B * a.O;
-  split_a3<<<ew_blocks(nh), 256, 0, s>>>((const float*)a.h, a.H, nullptr, 0, a.B, h3);
+  launch_pdl(split_a3, dim3(ew_blocks(nh)), dim3(256), 0, s, (const float*)a.h, a.H, nullptr, 0, a.B, h3);
   GemmOut o{GemmOut::LOSS_DY, nullptr, a.O, a.b_out, 0};
   o.target = a.target;
   o.dy32 = a.dy;
@@ -200,9 +216,9 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   o.scale = 1.f / ((float)a.B * (float)a.O);
   int rc = gemm_bf16(h3, 3 * a.H, false, w.wout3, 3 * a.H, false, o, a.B, a.O, 3 * a.H, w.status, s);
   if (rc != MEBPTT_OK) return rc;
-  sum_parts<<<1, 32, 0, s>>>(a.loss_part, (a.B / 32) * o.parts, a.loss_k);
-  split_a3<<<ew_blocks(no), 256, 0, s>>>(a.dy, a.O, nullptr, 0, a.B, dy3);
-  colsum_accum<float><<<(a.O + 127) / 128, 128, 0, s>>>(a.dy, a.B, a.O, a.db_out);
+  launch_pdl(sum_parts, dim3(1), dim3(32), 0, s, a.loss_part, (a.B / 32) * o.parts, a.loss_k);
+  launch_pdl(split_a3, dim3(ew_blocks(no)), dim3(256), 0, s, a.dy, a.O, nullptr, 0, a.B, dy3);
+  launch_pdl(colsum_accum<float>, dim3((a.O + 127) / 128), dim3(128), 0, s, a.dy, a.B, a.O, a.db_out);
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]
   return gemm_bf16(dy3, 3 * a.O, false, w.woutmn3, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B,
                    a.H, 3 * a.O, w.status, s, true, &w.split);
@@ -215,10 +231,10 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_
   bf16* dz3 = w.st_dz3 + ((size_t)l * rows + (size_t)sidx * a.B) * 3 * G;
   bf16* in2 = w.st_in2 + (l == 0 ? 0 : rows * 2 * w.I0 + (size_t)(l - 1) * rows * 2 * a.H) + (size_t)sidx * a.B * 2 * a.I;
   bf16* hp2 = w.st_hp2 + ((size_t)l * rows + (size_t)sidx * a.B) * 2 * a.H;
-  gate_bwd<<<ew_blocks(n), 256, 0, s>>>(a.dha, a.dh_rec, a.dc_rec, (const float*)a.gates, a.plane_elems, a.c_t, a.c_prev,
+  launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const float*)a.gates, a.plane_elems, a.c_t, a.c_prev,
                                         a.dz, dz3, a.B, a.H, a.counters, (const float*)a.in, a.I, in2,
                                         (const float*)a.h_prev, hp2);
-  colsum_accum<float><<<(G + 127) / 128, 128, 0, s>>>(a.dz, a.B, G, a.db);
+  launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, a.dz, a.B, G, a.db);
   const bf16* WMN = w.wmn3 + 3 * w_off;   // [3G][K]
   if (a.d_lo) {
     int rc = gemm_bf16(dz3, 3 * G, false, WMN, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I,
