@@ -7,6 +7,7 @@
 #include "plan.hpp"
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <limits>
 #include <new>
@@ -39,6 +40,59 @@ int64_t first_index(const T* a, const T* b_last, int64_t n, T base, T value) {
   return -1;
 }
 
+// First argmin of  i + a[i] + b[-i]  over i = 0 .. n-1 when that sequence is convex in i: a local
+// minimum is then the global one, and walking from a nearby guess (the answer for the previous
+// t) costs O(1) on average instead of a scan.  Left first, through ties, so that the smallest
+// index wins exactly as in the scan.
+template <class T>
+int64_t convex_first_argmin(const T* a, const T* b_last, int64_t n, int64_t guess) {
+  auto f = [&](int64_t j) { return (T)((T)j + a[j] + b_last[-j]); };
+  int64_t i = guess < 0 ? 0 : (guess > n - 1 ? n - 1 : guess);
+  T v = f(i);
+  bool moved = false;
+  while (i > 0) {
+    const T w = f(i - 1);
+    if (w > v) break;
+    v = w; --i; moved = true;
+  }
+  if (!moved) {
+    while (i < n - 1) {
+      const T w = f(i + 1);
+      if (w >= v) break;
+      v = w; ++i;
+    }
+  }
+  return i;
+}
+
+// A column of costs seen as a sequence in t: the longest prefix lo .. hi of it that is finite and
+// convex (second differences >= 0), extended one element at a time.  Appendix A remarks that the
+// O(t^2 m) scan can be brought down to O(t m) "by exploiting convexity in t"; the paper does not
+// prove convexity, so it is checked on the numbers before it is used, and wherever it fails the
+// scan is kept.
+template <class T>
+struct ConvexPrefix {
+  const T* c;
+  int64_t lo, hi;   // c[lo .. hi] is finite and convex; hi = lo - 1 while empty
+  ConvexPrefix(const T* col, int64_t first) : c(col), lo(first), hi(first - 1) {}
+  // c[t] has just been written (or is being read in order); returns whether the prefix now reaches t
+  bool extend(int64_t t, T inf) {
+    if (hi != t - 1 || c[t] >= inf) return false;
+    if (t - lo >= 2 && (int64_t)c[t] - c[t - 1] < (int64_t)c[t - 1] - c[t - 2]) return false;
+    hi = t;
+    return true;
+  }
+  void extend_to(int64_t t_max, T inf) {
+    for (int64_t t = hi + 1; t <= t_max && extend(t, inf); ++t) {}
+  }
+};
+
+inline bool plan_scan_only() {
+  // verification aid: MEBPTT_PLAN_SCAN=1 keeps the plain scan everywhere (the tests compare the two)
+  const char* e = getenv("MEBPTT_PLAN_SCAN");
+  return e && e[0] == '1';
+}
+
 template <class T>
 struct Inf;
 template <>
@@ -64,6 +118,7 @@ void solve_hsm(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
   // Section 3.1: C(1, m) = 1, C(t, 1) = t (t + 1) / 2,
   // C(t, m) = min_{1 <= y < t} y + C(t - y, m - 1) + C(y, m).
   const T INF = Inf<T>::v;
+  const bool scan_only = plan_scan_only();
   for (int64_t m = 1; m <= m_max; ++m) {
     T* c = C.col(m);
     int32_t* d = D.col(m);
@@ -74,12 +129,25 @@ void solve_hsm(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
       continue;
     }
     const T* cm1 = C.col(m - 1);
+    ConvexPrefix<T> cur(c, 1), prev(cm1, 1);
+    if (!scan_only) prev.extend_to(t_max, INF);
+    cur.extend(1, INF);
+    int64_t guess = 0;
     for (int64_t t = 2; t <= t_max; ++t) {
       // y = 1 + i, i = 0 .. t-2 :  (1 + i) + c[1 + i] + cm1[t - 1 - i]
-      T best = scan_min<T>(c + 1, cm1 + (t - 1), t - 1, (T)1);
-      if (best >= INF) { c[t] = INF; continue; }
-      c[t] = best;
-      d[t] = (int32_t)(1 + first_index<T>(c + 1, cm1 + (t - 1), t - 1, (T)1, best));
+      if (!scan_only && cur.hi >= t - 1 && prev.hi >= t - 1) {
+        // c on [1, t-1] and cm1 on [1, t-1] are convex, hence so is the sum over the split point
+        guess = convex_first_argmin<T>(c + 1, cm1 + (t - 1), t - 1, guess);
+        c[t] = (T)((T)1 + (T)guess + c[1 + guess] + cm1[t - 1 - guess]);
+        d[t] = (int32_t)(1 + guess);
+      } else {
+        T best = scan_min<T>(c + 1, cm1 + (t - 1), t - 1, (T)1);
+        if (best >= INF) { c[t] = INF; continue; }
+        c[t] = best;
+        guess = first_index<T>(c + 1, cm1 + (t - 1), t - 1, (T)1, best);
+        d[t] = (int32_t)(1 + guess);
+      }
+      cur.extend(t, INF);
     }
   }
 }
@@ -89,6 +157,7 @@ void solve_ism(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
   // Section 3.2: C(0, m) = 0, C(t > 0, 0) = inf,
   // C(t, m) = min_{1 <= y <= t} y + C(y - 1, m) + C(t - y, m - 1).
   const T INF = Inf<T>::v;
+  const bool scan_only = plan_scan_only();
   for (int64_t m = 0; m <= m_max; ++m) {
     C.col(m)[0] = 0;
     std::fill(D.col(m), D.col(m) + t_max + 1, 0);
@@ -97,12 +166,24 @@ void solve_ism(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
     T* c = C.col(m);
     int32_t* d = D.col(m);
     const T* cm1 = C.col(m - 1);
+    ConvexPrefix<T> cur(c, 0), prev(cm1, 0);
+    if (!scan_only) prev.extend_to(t_max, INF);
+    cur.extend(0, INF);
+    int64_t guess = 0;
     for (int64_t t = 1; t <= t_max; ++t) {
       // y = 1 + i, i = 0 .. t-1 :  (1 + i) + c[i] + cm1[t - 1 - i]
-      T best = scan_min<T>(c, cm1 + (t - 1), t, (T)1);
-      if (best >= INF) { c[t] = INF; continue; }
-      c[t] = best;
-      d[t] = (int32_t)(1 + first_index<T>(c, cm1 + (t - 1), t, (T)1, best));
+      if (!scan_only && cur.hi >= t - 1 && prev.hi >= t - 1) {
+        guess = convex_first_argmin<T>(c, cm1 + (t - 1), t, guess);
+        c[t] = (T)((T)1 + (T)guess + c[guess] + cm1[t - 1 - guess]);
+        d[t] = (int32_t)(1 + guess);
+      } else {
+        T best = scan_min<T>(c, cm1 + (t - 1), t, (T)1);
+        if (best >= INF) { c[t] = INF; continue; }
+        c[t] = best;
+        guess = first_index<T>(c, cm1 + (t - 1), t, (T)1, best);
+        d[t] = (int32_t)(1 + guess);
+      }
+      cur.extend(t, INF);
     }
   }
 }

@@ -57,6 +57,28 @@ def test_whole_cost_tables_match_oracle():
     assert np.array_equal(tabs["D2"][itl], ref["D2"][itl])
 
 
+@pytest.mark.parametrize("mode", [P.HSM, P.ISM, P.MSM])
+def test_convexity_shortcut_changes_no_table_entry(mode, monkeypatch):
+    """Where a cost column is convex in t the planner walks from the previous split point instead
+    of scanning every y (Appendix A's remark); with MEBPTT_PLAN_SCAN=1 it scans everywhere.  Both
+    must give the same C and the same D (smallest y on ties) in every cell."""
+    for t, m in [(150, 150), (257, 31), (64, 200), (2, 1), (1, 5)]:
+        fast = B.mebptt_plan_ex(t, m, mode, 4, 0).tables()
+        monkeypatch.setenv("MEBPTT_PLAN_SCAN", "1")
+        slow = B.mebptt_plan_ex(t, m, mode, 4, 0).tables()
+        monkeypatch.delenv("MEBPTT_PLAN_SCAN")
+        for k in fast:
+            assert np.array_equal(fast[k], slow[k]), (mode, t, m, k)
+
+
+def test_long_sequence_plans_match_oracle_columns():
+    """t = 4000 (config 4): the fast path's costs against the oracle's own DP at a few budgets."""
+    for mode, m in [(P.ISM, 20), (P.ISM, 50), (P.HSM, 12)]:
+        plan = B.mebptt_plan_ex(4000, m, mode, 4, 0)
+        assert plan.cost == _oracle_cost(mode, 4000, m)
+        assert plan.validate() == B.MEBPTT_OK
+
+
 def test_benchmark_budgets_match_oracle():
     """The (t, m) points of the timed workloads; the oracle runs its own DP for each."""
     for mode, t, m, alpha, beta in [(P.HSM, 64, 8, 4, 0), (P.HSM, 256, 16, 4, 0), (P.ISM, 256, 64, 4, 0),
