@@ -5,6 +5,7 @@
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
+#include <vector>
 
 #include "kernels.hpp"
 #include "layout.hpp"
@@ -78,6 +79,12 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     tcw.st_dy = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_dy);
     tcw.st_h = reinterpret_cast<__nv_bfloat16*>(ws + y.off_st_h);
     tcw.split = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), (size_t)148 * 128 * 128};
+    tcw.split_run = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), y.split_floats};
+    tcw.zrun = reinterpret_cast<float*>(ws + y.off_zrun);
+    tcw.hrun = reinterpret_cast<__nv_bfloat16*>(ws + y.off_hrun);
+    tcw.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
+    tcw.loss_part = loss_part;
+    tcw.colsum_part = reinterpret_cast<float*>(ws + y.off_colsum);
   }
   stepwise3::Scratch x3{};
   size_t w_off[16];
@@ -108,8 +115,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   if (y.stepwise_x3)
     stepwise3::pack_weights(x3, y.L, y.I, y.H, y.O, reinterpret_cast<const float*>(io.W), w_off,
                             reinterpret_cast<const float*>(io.W_out), s);
-  for (const mebptt_op& op : p->tape) {
-    if (rc != MEBPTT_OK) break;
+  auto run_op = [&](const mebptt_op& op) {
     const int64_t k = op.k;
     const char* x_k = io.x + (size_t)(k - 1) * y.B * y.I * y.esz;
     if (op.kind == MEBPTT_OP_FWD) {
@@ -151,7 +157,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
       if (y.stepwise_x3) rc = stepwise3::readout(r, x3, sidx, s);
       else if (y.stepwise_tc) rc = stepwise::readout(r, tcw, sidx, s);
       else generic::readout(y.dtype, r, s);
-      if (rc != MEBPTT_OK) break;
+      if (rc != MEBPTT_OK) return;
       for (int l = y.L - 1; l >= 0; --l) {
         generic::BwdArgs a{};
         a.dha = dha;
@@ -186,6 +192,88 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
         rc = y.stepwise_x3 ? stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s)
                            : stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+      }
+    }
+  };
+
+  // The bfloat16 step-by-step path takes runs of consecutive operations one layer at a time (the
+  // input products, the readout and the gradients handed down are then batched over the run);
+  // everything else, and the leaves of the recursion, go operation by operation.  Both give the
+  // same bits; MEBPTT_STEPWISE_PER_OP=1 keeps to single operations (the tests compare the two).
+  const bool per_op_only = getenv("MEBPTT_STEPWISE_PER_OP") != nullptr;
+  if (!y.stepwise_tc || per_op_only) {
+    for (const mebptt_op& op : p->tape) {
+      if (rc != MEBPTT_OK) break;
+      run_op(op);
+    }
+  } else {
+    const std::vector<WorkItem> items = work_items(p, y.S);
+    std::vector<stepwise::FwdRunStep> fst((size_t)y.S);
+    std::vector<stepwise::BwdRunStep> bst((size_t)y.S);
+    std::vector<const void*> h_top((size_t)y.S);
+    for (const WorkItem& wi : items) {
+      if (rc != MEBPTT_OK) break;
+      const mebptt_op* ops = p->tape.data() + wi.i;
+      if (wi.kind == WorkItem::LEAF || wi.n == 1) {
+        const size_t cnt = wi.kind == WorkItem::LEAF ? 2 * (size_t)wi.n : 1;
+        for (size_t j = 0; j < cnt && rc == MEBPTT_OK; ++j) run_op(ops[j]);
+      } else if (wi.kind == WorkItem::FWD) {
+        const int n = wi.n;
+        const int64_t k0 = ops[0].k;
+        for (int l = 0; l < y.L && rc == MEBPTT_OK; ++l) {
+          for (int j = 0; j < n; ++j) {
+            const mebptt_op& op = ops[j];
+            char* dst = loc_base(y, ws, op.dst);
+            stepwise::FwdRunStep& f = fst[j];
+            f = stepwise::FwdRunStep{};
+            hidden_at(y, io, op.src, l, &f.h_prev, &f.c_prev);
+            f.h_out = dst + y.h_off(l);
+            f.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
+            if (op.dst_fmt != MEBPTT_FMT_HIDDEN) f.gates = dst + y.rec_gates + (size_t)l * y.gsz;
+            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+              f.h_in_copy = dst + y.rec_in + y.h_off(l);
+              f.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
+            }
+          }
+          const void* in = (l == 0) ? (const void*)(io.x + (size_t)(k0 - 1) * y.B * y.I * y.esz) : (const void*)tcw.hrun;
+          rc = stepwise::forward_run_layer(fst.data(), n, in, l == 0 ? y.I : y.H, io.W + y.w_layer_offset(l) * y.esz,
+                                           io.b + (size_t)l * 4 * y.H, l + 1 < y.L, y.B, y.H, plane_elems,
+                                           l == 0 ? io.counters : nullptr, tcw, s);
+        }
+      } else {
+        // n backward operations, time descending, inside one chunk: index a = step - first step
+        const int n = wi.n;
+        const int64_t k_hi = ops[0].k, k_lo = k_hi - n + 1;
+        const int s_lo = (int)((k_lo - 1) % y.S);
+        auto op_at = [&](int a) -> const mebptt_op& { return ops[n - 1 - a]; };
+        for (int a = 0; a < n; ++a) h_top[a] = loc_base(y, ws, op_at(a).src) + y.h_off(y.L - 1);
+        rc = stepwise::readout_run(h_top.data(), n, s_lo, io.W_out, io.b_out, io.targets + (size_t)(k_lo - 1) * y.B * y.O,
+                                   loss_t + (k_lo - 1), io.db_out, y.B, y.H, y.O, tcw, s);
+        for (int l = y.L - 1; l >= 0 && rc == MEBPTT_OK; --l) {
+          for (int a = 0; a < n; ++a) {
+            const mebptt_op& op = op_at(a);
+            char* rec = loc_base(y, ws, op.src);
+            stepwise::BwdRunStep& b = bst[a];
+            b.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+            b.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
+            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+              b.h_prev = rec + y.rec_in + y.h_off(l);
+              b.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
+            } else {
+              hidden_at(y, io, op.aux, l, &b.h_prev, &b.c_prev);
+            }
+            b.in = (l == 0) ? (const void*)(io.x + (size_t)(op.k - 1) * y.B * y.I * y.esz) : (const void*)(rec + y.h_off(l - 1));
+          }
+          float* d_lo = (l > 0) ? tcw.dha_run : (desc->want_dx ? io.dx + (size_t)(k_lo - 1) * y.B * y.I : nullptr);
+          rc = stepwise::backward_run_layer(bst.data(), n, s_lo, l, l == 0 ? y.I : y.H, io.W + y.w_layer_offset(l) * y.esz,
+                                            dh_rec + (size_t)l * bh, dc_rec + (size_t)l * bh, dz, io.db + (size_t)l * 4 * y.H,
+                                            d_lo, y.B, y.H, plane_elems, l == y.L - 1 ? io.counters : nullptr, tcw, s);
+        }
+        if (s_lo == 0 && rc == MEBPTT_OK) {
+          const int64_t chunk = (k_lo - 1) / y.S;
+          const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
+          rc = stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+        }
       }
     }
   }
@@ -267,7 +355,17 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, y.O, pf) > 1 ? 2 : 1;
     const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
     const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs
-    return p->cost * 3 * L + p->t * (3 + dha + bwd) + chunks * (2 * L + 1) + 1;
+    // runs of n >= 2 operations go layer by layer: one input product per layer and run, the
+    // readout once per run (stage, GEMM with loss, loss terms, dha, two for db_out), the gradient handed
+    // down once per layer and run
+    int64_t n_launch = chunks * (2 * L + 1) + 1;
+    for (const WorkItem& wi : work_items(p, y.S)) {
+      if (wi.kind == WorkItem::LEAF) n_launch += wi.n * (3 * L + 3 + dha + bwd);
+      else if (wi.kind == WorkItem::FWD) n_launch += wi.n == 1 ? 3 * L : L * (1 + 2 * (int64_t)wi.n);
+      else if (wi.n == 1) n_launch += 3 + dha + bwd;
+      else n_launch += 5 + dha + L * wi.n * (2 + to_h) + (L - 1) * to_h + (desc->want_dx ? to_x : 0);
+    }
+    return n_launch;
   }
   if (y.stepwise_x3) {
     // weights: 2 packing kernels per layer and 2 for the readout; forward operation: split, GEMM,

@@ -90,6 +90,13 @@ struct Scratch {
   __nv_bfloat16* st_hp;     // [L][S B][H]  h_{k-1}
   __nv_bfloat16* st_dy;     // [S B][O]
   __nv_bfloat16* st_h;      // [S B][H]  top layer h_k
+  // a run of up to S operations, one layer at a time
+  float* zrun;              // [S B][4H] pre-activations of the run's steps
+  __nv_bfloat16* hrun;      // [S B][H]  the layer's h_k, read by the layer above
+  float* dha_run;           // [S B][H]  gradient entering the layer at each step (row block: step - first step)
+  float* loss_part;         // partial sums of the loss terms, per step
+  float* colsum_part;       // [S][O] per-step column sums of dy
+  tc::SplitWs split_run;    // split-K scratch for a product over all rows of a run
 };
 int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s);
 // sidx: row block of this step in the stages; l: layer
@@ -98,6 +105,30 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
 // dW (w_off[l]: element offset of layer l) and dW_out from the first `steps` row blocks of the stages
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
                 float* dW_out, cudaStream_t s);
+
+// One step of a run, as one layer sees it.
+struct FwdRunStep {
+  const void* h_prev; const float* c_prev;     // state k-1 of the layer
+  void* h_out; float* c_out;                   // where state k goes
+  void* gates; void* h_in_copy; float* c_in_copy;   // as in FwdArgs
+};
+struct BwdRunStep {
+  const void* gates; const float* c_t; const float* c_prev; const void* in; const void* h_prev;   // as in BwdArgs
+};
+// n consecutive forward operations of one layer.  in: the layer's inputs of all n steps, [n B][I]
+// (x, or w.hrun as the layer below left it); stage_h: leave the layer's h_k in w.hrun.
+int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const void* W, const float* bias, bool stage_h,
+                      int B, int H, size_t plane_elems, int64_t* counters, const Scratch& w, cudaStream_t s);
+// Readout, loss terms, dy and the gradient entering the top layer (-> w.dha_run) for the n steps
+// whose stages are the row blocks s_lo .. s_lo + n - 1; h_top[a]: the top layer's h of step s_lo + a;
+// target, loss_t: those of the first of the steps.
+int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out, const float* b_out, const float* target,
+                float* loss_t, float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s);
+// The n backward operations of layer l, time descending (st[a]: step s_lo + a), reading w.dha_run;
+// d_lo (nullable): [n B][I] gradient w.r.t. the layer's inputs, written once for the whole run.
+int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, const void* W, float* dh_rec, float* dc_rec,
+                       float* dz, float* db, float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
+                       const Scratch& w, cudaStream_t s);
 }  // namespace stepwise
 
 // The same for float32 storage (MEBPTT_TF32): operands split into two bfloat16 halves, three

@@ -53,6 +53,7 @@ struct Layout {
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
+  size_t off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_colsum = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
   int64_t arena_units = 0;
@@ -221,8 +222,16 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_st_hp = take((size_t)y.L * rows * y.H * 2);
       y.off_st_dy = take(rows * y.O * 2);
       y.off_st_h = take(rows * y.H * 2);
-      // split-K scratch: at most a wave of 128 x 128 float32 tiles
-      y.off_split = take((size_t)148 * 128 * 128 * 4);
+      // a run of up to S consecutive operations, one layer at a time: pre-activations of the run,
+      // the layer's h_k (the next layer's input), the gradient entering the layer at every step
+      y.off_zrun = take(rows * 4 * y.H * 4);
+      y.off_hrun = take(rows * y.H * 2);
+      y.off_dha_run = take(rows * y.H * 4);
+      y.off_colsum = take((size_t)y.S * y.O * 4);
+      // split-K scratch: a wave of 128 x 128 float32 tiles for one step, times the 8 row tiles of
+      // a whole run (its products are split like a single step's, to sum in the same order)
+      y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
+      y.off_split = take(y.split_floats * 4);
     }
     if (y.stepwise_x3) {
       const size_t G = 4 * (size_t)y.H, Kmax = (size_t)(y.I > y.H ? y.I : y.H) + y.H;
@@ -242,7 +251,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_st_dy = take(rows * 3 * y.O * 2);
       y.off_st_h = take(rows * 3 * y.H * 2);
     }
-    y.off_loss_part = take((size_t)y.n_loss_part * 4);
+    y.off_loss_part = take((size_t)y.n_loss_part * 4 * (y.stepwise_tc ? y.S : 1));
     y.off_status = take(256);
   } else {
     const size_t G = (size_t)4 * y.H;

@@ -39,7 +39,7 @@ __device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf
 // internal state, the copies of h_{k-1}, c_{k-1}.
 __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
                          bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H,
-                         int64_t* counters) {
+                         int64_t* counters, bf16* h_stage) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
@@ -51,7 +51,9 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev
     const float cp = c_prev[e];
     const float c = fmaf(gf, cp, gi * gg);
     c_out[e] = c;
-    h_out[e] = __float2bfloat16_rn(go * tanhf(c));
+    const bf16 hv = __float2bfloat16_rn(go * tanhf(c));
+    h_out[e] = hv;
+    if (h_stage) h_stage[e] = hv;   // a second copy, where the layer above reads its inputs of a whole run
     if (gates) {
       gates[e] = __float2bfloat16_rn(gi);
       gates[plane + e] = __float2bfloat16_rn(gf);
@@ -124,6 +126,53 @@ __global__ void sum_parts_stage_h(const float* part, int n, float* out, const ui
   }
 }
 
+// Up to 32 device pointers passed by value (a run has at most S = 1024 / B <= 32 steps).
+struct RunPtrs { const void* p[32]; };
+
+// Row block a of `dst` (n16 16-byte words each) <- src.p[a]; blockIdx.y = a.
+__global__ void stage_blocks(RunPtrs src, uint4* dst, size_t n16) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const uint4* from = reinterpret_cast<const uint4*>(src.p[blockIdx.y]);
+  uint4* to = dst + (size_t)blockIdx.y * n16;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n16; e += (size_t)gridDim.x * blockDim.x) to[e] = from[e];
+}
+
+// Loss terms of n steps from their partial sums, each summed in index order.
+__global__ void sum_parts_steps(const float* part, int per_step, int n, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int a = blockIdx.x * blockDim.x + threadIdx.x;
+  if (a >= n) return;
+  float s = 0.f;
+  for (int i = 0; i < per_step; ++i) s += part[(size_t)a * per_step + i];
+  out[a] = s;
+}
+
+// Column sums of n row blocks at once: part[a][c] = sum_b v[a][b][c], b ascending (blockIdx.y = a),
+// then out[c] += part[a][c] for a = n-1 .. 0 (time descending): the sums and the order of n
+// single-step calls of colsum_accum.
+template <class T>
+__global__ void colsum_steps(const T* v, int B, int N, float* part) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= N) return;
+  const T* blk = v + (size_t)blockIdx.y * B * N;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += (float)blk[(size_t)b * N + c];
+  part[(size_t)blockIdx.y * N + c] = s;
+}
+__global__ void add_steps_descending(const float* part, int n, int N, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= N) return;
+  float acc = out[c];
+  for (int a = n - 1; a >= 0; --a) acc += part[(size_t)a * N + c];
+  out[c] = acc;
+}
+
 inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
 
 }  // namespace
@@ -139,7 +188,7 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
   launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
-                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
+                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr);
   return MEBPTT_OK;
 }
 
@@ -206,6 +255,91 @@ int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O,
   }
   return gemm_bf16(w.st_dy, O, true, w.st_h, H, true, GemmOut{GemmOut::ACCUM_F32, dW_out, H, nullptr, 0}, O, H, R,
                    w.status, s);
+}
+
+// ---- runs of consecutive operations, one layer at a time -----------------------------------------
+// What depends on the previous step is only the product with the recurrent weights; the product
+// with the layer's input, the readout and the gradient handed to the layer below are taken for
+// all steps of the run at once.  Every element is computed by the same sums in the same order as
+// in the single-step functions above (a contraction that those split along K is split into the
+// same parts here), so a plan's results do not depend on how its tape falls into runs.
+
+int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const void* Wl, const float* bias,
+                      bool stage_h, int B, int H, size_t plane_elems, int64_t* counters, const Scratch& w,
+                      cudaStream_t s) {
+  const int K = I + H, G = 4 * H;
+  const bf16* W = (const bf16*)Wl;
+  int rc = gemm_bf16(in, I, false, W, K, false, GemmOut{GemmOut::STORE_F32, w.zrun, G, bias, 0}, n * B, G, I, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  const size_t bh = (size_t)B * H;
+  for (int j = 0; j < n; ++j) {
+    float* z = w.zrun + (size_t)j * B * G;
+    rc = gemm_bf16(st[j].h_prev, H, false, W + I, K, false, GemmOut{GemmOut::ACCUM_F32, z, G, nullptr, 0}, B, G, H,
+                   w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+    launch_pdl(cell_fwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)z, st[j].c_prev, (const bf16*)st[j].h_prev,
+               (bf16*)st[j].h_out, st[j].c_out, (bf16*)st[j].gates, plane_elems, (bf16*)st[j].h_in_copy, st[j].c_in_copy, B,
+               H, counters, stage_h ? w.hrun + (size_t)j * bh : (bf16*)nullptr);
+  }
+  return MEBPTT_OK;
+}
+
+int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out_, const float* b_out, const float* target,
+                float* loss_t, float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s) {
+  const bf16* W_out = (const bf16*)W_out_;
+  const size_t n_h16 = (size_t)B * H * 2 / 16;
+  RunPtrs ptrs{};
+  for (int a = 0; a < n; ++a) ptrs.p[a] = h_top[a];
+  bf16* st_h = w.st_h + (size_t)s_lo * B * H;
+  bf16* dy16 = w.st_dy + (size_t)s_lo * B * O;
+  launch_pdl(stage_blocks, dim3(ew_blocks(n_h16 * 8) > 64 ? 64 : ew_blocks(n_h16 * 8), n), dim3(256), 0, s, ptrs,
+             (uint4*)st_h, n_h16);
+  const int parts = (O + 31) / 32, per_step = (B / 32) * parts;
+  GemmOut o{GemmOut::LOSS_DY, dy16, O, b_out, 0};
+  o.target = target;
+  o.loss_part = w.loss_part;
+  o.parts = parts;
+  o.scale = 1.f / ((float)B * (float)O);
+  int rc = gemm_bf16(st_h, H, false, W_out, H, false, o, n * B, O, H, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  launch_pdl(sum_parts_steps, dim3(1), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
+  // the gradient entering the top layer at every step of the run, split along K like a single step's
+  const int splits = tc::gemm_split_count(false, true, B, H, O, w.split.partial_floats);
+  rc = gemm_bf16(dy16, O, false, W_out, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H, O,
+                 w.status, s, true, &w.split_run, splits);
+  if (rc != MEBPTT_OK) return rc;
+  launch_pdl(colsum_steps<bf16>, dim3((O + 127) / 128, n), dim3(128), 0, s, (const bf16*)dy16, B, O, w.colsum_part);
+  launch_pdl(add_steps_descending, dim3((O + 127) / 128), dim3(128), 0, s, (const float*)w.colsum_part, n, O, db_out);
+  return MEBPTT_OK;
+}
+
+int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, const void* Wl, float* dh_rec, float* dc_rec,
+                       float* dz, float* db, float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
+                       const Scratch& w, cudaStream_t s) {
+  const int K = I + H, G = 4 * H;
+  const size_t bh = (size_t)B * H;
+  const bf16* W = (const bf16*)Wl;
+  const size_t rows = (size_t)w.S * B;
+  bf16* dz_l = w.st_dz + (size_t)l * rows * G;
+  bf16* in_l = w.st_in + (l == 0 ? 0 : rows * w.I0 + (size_t)(l - 1) * rows * H);
+  bf16* hp_l = w.st_hp + (size_t)l * rows * H;
+  for (int a = n - 1; a >= 0; --a) {   // time descending
+    const size_t row0 = (size_t)(s_lo + a) * B;
+    bf16* dz16 = dz_l + row0 * G;
+    launch_pdl(gate_bwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)(w.dha_run + (size_t)a * bh), (const float*)dh_rec,
+               dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t, st[a].c_prev, dz, dz16, B, H, counters,
+               (const uint4*)st[a].in, (uint4*)(in_l + row0 * I), (size_t)B * I * 2 / 16, (const uint4*)st[a].h_prev,
+               (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16);
+    launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, (const float*)dz, B, G, db);
+    const int rc = gemm_bf16(dz16, G, false, W + I, K, true, GemmOut{GemmOut::STORE_F32, dh_rec, H, nullptr, 0}, B, H, G,
+                             w.status, s, true, &w.split);
+    if (rc != MEBPTT_OK) return rc;
+  }
+  if (!d_lo) return MEBPTT_OK;
+  // the gradient w.r.t. the layer's inputs (dx, or what enters the layer below) for the whole run
+  const int splits = tc::gemm_split_count(false, true, B, I, G, w.split.partial_floats);
+  return gemm_bf16(dz_l + (size_t)s_lo * B * G, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, d_lo, I, nullptr, 0},
+                   n * B, I, G, w.status, s, true, &w.split_run, splits);
 }
 
 }  // namespace stepwise

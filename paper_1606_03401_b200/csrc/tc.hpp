@@ -67,8 +67,11 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 // receives MEBPTT_ERR_TIMEOUT if a bounded wait expires.  early: the kernel may become resident
 // before the previous kernel of the stream has finished (it still waits for it before touching
 // memory).
+// force_splits > 0: split the contraction index into exactly that many parts (the caller took the
+// count from gemm_split_count for a product of another height, so that both sum in the same order).
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s, bool early = true, const SplitWs* split = nullptr);
+              int M, int N, int K, int* status, cudaStream_t s, bool early = true, const SplitWs* split = nullptr,
+              int force_splits = 0);
 
 }  // namespace tc
 

@@ -375,7 +375,7 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 }
 
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split) {
+              int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split, int force_splits) {
   if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
   // A short-and-wide product over K-major operands (a few steps' worth of rows against a whole
   // weight matrix) gives few 128-wide tiles, each streaming all of K through one SM: 32-wide tiles
@@ -394,7 +394,10 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   int splits = 1;
   if (split && split->partial && out.kind == GemmOut::STORE_F32 && !out.bias && !out.perm_h && out.ld % 4 == 0 &&
       (reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0)
-    splits = gemm_split_count(a_mn, b_mn, M, N, K, split->partial_floats);
+    splits = force_splits > 0 ? force_splits : gemm_split_count(a_mn, b_mn, M, N, K, split->partial_floats);
+  else if (force_splits > 1)
+    return MEBPTT_ERR_ARG;
+  if (splits > 1 && (size_t)grid.x * grid.y * splits * BM * BN > split->partial_floats) return MEBPTT_ERR_WORKSPACE;
   grid.z = splits;
   static const bool attrs = [] {
     const int most = gemm_smem(MAX_STAGES, BN_WIDE);

@@ -245,6 +245,28 @@ def test_stepwise_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
     assert_bit_identical(res, full)
 
 
+@pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=45, readout=40),
+                                   dict(layers=3, input=24, hidden=64, batch=96, t=23, readout=8),
+                                   dict(layers=2, input=128, hidden=2048, batch=128, t=19, readout=128)])
+def test_stepwise_runs_give_the_bits_of_single_operations(H, shape, monkeypatch):
+    """The step-by-step tensor-core path takes runs of consecutive operations one layer at a time,
+    with the input products, the readout and the gradients handed down batched over the run (at
+    config 5's widths some of those contractions are split along K).  Operation by operation
+    (MEBPTT_STEPWISE_PER_OP=1) every sum must come out the same, bit for bit, under long runs and
+    short ones, with and without dx."""
+    cfg = _cfg("c5", **shape)
+    for want_dx in (True, False):
+        dp = H.DeviceProblem(cfg, want_dx=want_dx)
+        plans = [dp.full_memory_plan(), dp.plan("msm", 11), dp.plan("hsm", 3), dp.plan("ism", 2)]
+        runs = [dp.run(p) for p in plans]
+        monkeypatch.setenv("MEBPTT_STEPWISE_PER_OP", "1")
+        single = dp.run(plans[0])
+        monkeypatch.delenv("MEBPTT_STEPWISE_PER_OP")
+        for p, r in zip(plans, runs):
+            assert r["counters"][0] == p.cost and r["counters"][1] == cfg.t and r["counters"][3] == 0
+            assert_bit_identical(r, single, want_dx=want_dx)
+
+
 @pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=21, readout=40),
                                    dict(layers=1, input=24, hidden=256, batch=96, t=13, readout=8),
                                    dict(layers=1, input=128, hidden=1152, batch=32, t=9, readout=64)])
