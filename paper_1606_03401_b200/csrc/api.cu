@@ -99,6 +99,11 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     x3.wout3 = bf(y.off_wout3); x3.woutmn3 = bf(y.off_woutmn3);
     x3.st_dz3 = bf(y.off_st_dz); x3.st_in2 = bf(y.off_st_in); x3.st_hp2 = bf(y.off_st_hp);
     x3.st_dy3 = bf(y.off_st_dy); x3.st_h3 = bf(y.off_st_h);
+    x3.split_run = tc::SplitWs{reinterpret_cast<float*>(ws + y.off_split), y.split_floats};
+    x3.dy_run = reinterpret_cast<float*>(ws + y.off_dy_run);
+    x3.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
+    x3.loss_part = loss_part;
+    x3.colsum_part = reinterpret_cast<float*>(ws + y.off_colsum);
   }
   const bool staged = y.stepwise_tc || y.stepwise_x3;   // weight gradients per chunk of S steps
   int rc = MEBPTT_OK;
@@ -201,7 +206,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   // everything else, and the leaves of the recursion, go operation by operation.  Both give the
   // same bits; MEBPTT_STEPWISE_PER_OP=1 keeps to single operations (the tests compare the two).
   const bool per_op_only = getenv("MEBPTT_STEPWISE_PER_OP") != nullptr;
-  if (!y.stepwise_tc || per_op_only) {
+  if (!(y.stepwise_tc || y.stepwise_x3) || per_op_only) {
     for (const mebptt_op& op : p->tape) {
       if (rc != MEBPTT_OK) break;
       run_op(op);
@@ -214,9 +219,56 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     for (const WorkItem& wi : items) {
       if (rc != MEBPTT_OK) break;
       const mebptt_op* ops = p->tape.data() + wi.i;
-      if (wi.kind == WorkItem::LEAF || wi.n == 1) {
-        const size_t cnt = wi.kind == WorkItem::LEAF ? 2 * (size_t)wi.n : 1;
+      if (wi.kind == WorkItem::LEAF || wi.n == 1 || (y.stepwise_x3 && wi.kind == WorkItem::FWD)) {
+        // (with float32 storage a forward operation is one contraction over [input ; h], so there is
+        // nothing of it to take out of the recurrence)
+        const size_t cnt = wi.kind == WorkItem::LEAF ? 2 * (size_t)wi.n : (size_t)wi.n;
         for (size_t j = 0; j < cnt && rc == MEBPTT_OK; ++j) run_op(ops[j]);
+      } else if (y.stepwise_x3) {
+        // float32 storage: the readout of the run at once, then its backward operations one by one
+        const int n = wi.n;
+        const int64_t k_hi = ops[0].k, k_lo = k_hi - n + 1;
+        const int s_lo = (int)((k_lo - 1) % y.S);
+        auto op_at = [&](int a) -> const mebptt_op& { return ops[n - 1 - a]; };
+        for (int a = 0; a < n; ++a) h_top[a] = loc_base(y, ws, op_at(a).src) + y.h_off(y.L - 1);
+        rc = stepwise3::readout_run(reinterpret_cast<const float* const*>(h_top.data()), n, s_lo, io.b_out,
+                                    io.targets + (size_t)(k_lo - 1) * y.B * y.O, loss_t + (k_lo - 1), io.db_out, y.B, y.H,
+                                    y.O, x3, s);
+        for (int a = n - 1; a >= 0 && rc == MEBPTT_OK; --a) {
+          const mebptt_op& op = op_at(a);
+          char* rec = loc_base(y, ws, op.src);
+          const char* x_k = io.x + (size_t)(op.k - 1) * y.B * y.I * y.esz;
+          for (int l = y.L - 1; l >= 0 && rc == MEBPTT_OK; --l) {
+            generic::BwdArgs b{};
+            b.dha = (l == y.L - 1) ? x3.dha_run + (size_t)a * bh : dha;
+            b.dh_rec = dh_rec + (size_t)l * bh;
+            b.dc_rec = dc_rec + (size_t)l * bh;
+            b.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+            b.plane_elems = plane_elems;
+            b.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
+            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+              b.h_prev = rec + y.rec_in + y.h_off(l);
+              b.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
+            } else {
+              hidden_at(y, io, op.aux, l, &b.h_prev, &b.c_prev);
+            }
+            b.in = (l == 0) ? (const void*)x_k : (const void*)(rec + y.h_off(l - 1));
+            b.I = (l == 0) ? y.I : y.H;
+            b.W = io.W + y.w_layer_offset(l) * y.esz;
+            b.dz = dz;
+            b.dW = io.dW + y.w_layer_offset(l);
+            b.db = io.db + (size_t)l * 4 * y.H;
+            b.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(op.k - 1) * y.B * y.I : nullptr);
+            b.B = y.B; b.H = y.H;
+            b.counters = (l == y.L - 1) ? io.counters : nullptr;
+            rc = stepwise3::backward_layer(b, x3, l, w_off[l], s_lo + a, s);
+          }
+        }
+        if (s_lo == 0 && rc == MEBPTT_OK) {
+          const int64_t chunk = (k_lo - 1) / y.S;
+          const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
+          rc = stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+        }
       } else if (wi.kind == WorkItem::FWD) {
         const int n = wi.n;
         const int64_t k0 = ops[0].k;
@@ -378,7 +430,14 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, 3 * y.O, pf) > 1 ? 2 : 1;
     const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
     const int64_t chunks = (p->t + y.S - 1) / y.S;
-    return 2 * L + 2 + p->cost * 3 * L + p->t * (5 + dha + bwd) + chunks * 3 * (2 * L + 1) + 1;
+    // the readout of a run of n >= 2 backward operations is taken once for the run (split, GEMM with
+    // loss, loss terms, split, two for db_out, dha)
+    int64_t readouts = 0;
+    for (const WorkItem& wi : work_items(p, y.S)) {
+      if (wi.kind == WorkItem::LEAF) readouts += wi.n * (5 + dha);
+      else if (wi.kind == WorkItem::BWD) readouts += wi.n == 1 ? 5 + dha : 6 + dha;
+    }
+    return 2 * L + 2 + p->cost * 3 * L + readouts + p->t * bwd + chunks * 3 * (2 * L + 1) + 1;
   }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }

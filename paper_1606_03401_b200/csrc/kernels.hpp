@@ -150,6 +150,12 @@ struct Scratch {
   __nv_bfloat16* st_hp2;     // [L][S B][2H]
   __nv_bfloat16* st_dy3;     // [S B][3 O]
   __nv_bfloat16* st_h3;      // [S B][3 H]  top layer h_k
+  // the readout of a run of up to S backward operations at once
+  float* dy_run;             // [S B][O]
+  float* dha_run;            // [S B][H]  gradient entering the top layer at each step of the run
+  float* loss_part;          // partial sums of the loss terms, per step
+  float* colsum_part;        // [S][O]
+  tc::SplitWs split_run;     // split-K scratch for a product over all rows of a run
 };
 // W: all layers' weights (float32), w_off[l] the element offset of layer l
 void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W, const size_t* w_off,
@@ -157,6 +163,11 @@ void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W,
 int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_off, cudaStream_t s);
 int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s);
 int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_off, int sidx, cudaStream_t s);
+// Readout, loss terms, dy and the gradient entering the top layer (-> w.dha_run, row block a for
+// step s_lo + a) of n steps at once; h_top[a]: the top layer's h of step s_lo + a; target, loss_t:
+// those of the first of the steps.
+int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, const float* target, float* loss_t,
+                float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s);
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
                 float* dW_out, cudaStream_t s);
 }  // namespace stepwise3

@@ -53,7 +53,7 @@ struct Layout {
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
-  size_t off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_colsum = 0, split_floats = 0;
+  size_t off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, off_colsum = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
   int64_t arena_units = 0;
@@ -239,7 +239,12 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
       const size_t rows = (size_t)y.S * y.B;
       y.off_z = take((size_t)y.B * G * 4);
-      y.off_split = take((size_t)148 * 128 * 128 * 4);
+      // the readout of a run of up to S steps at once; its split-K scratch as on the bfloat16 path
+      y.off_dy_run = take(rows * y.O * 4);
+      y.off_dha_run = take(rows * y.H * 4);
+      y.off_colsum = take((size_t)y.S * y.O * 4);
+      y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
+      y.off_split = take(y.split_floats * 4);
       y.off_a3 = take((size_t)y.B * 3 * Kmax * 2);
       y.off_w3 = take(3 * y.w_total_elems() * 2);
       y.off_wmn3 = take(3 * y.w_total_elems() * 2);
@@ -251,7 +256,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_st_dy = take(rows * 3 * y.O * 2);
       y.off_st_h = take(rows * 3 * y.H * 2);
     }
-    y.off_loss_part = take((size_t)y.n_loss_part * 4 * (y.stepwise_tc ? y.S : 1));
+    y.off_loss_part = take((size_t)y.n_loss_part * 4 * ((y.stepwise_tc || y.stepwise_x3) ? y.S : 1));
     y.off_status = take(256);
   } else {
     const size_t G = (size_t)4 * y.H;

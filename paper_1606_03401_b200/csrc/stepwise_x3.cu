@@ -86,6 +86,25 @@ __global__ void split_a3(const float* a, int Ca, const float* b_, int Cb, int B,
   }
 }
 
+// The same split for up to 32 row blocks of [B][C] that lie apart (blockIdx.y picks the block);
+// block a goes to rows a B .. of `out`.
+struct RunPtrs { const float* p[32]; };
+__global__ void split_blocks3(RunPtrs src, int C, int B, bf16* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const float* a = src.p[blockIdx.y];
+  bf16* dst = out + (size_t)blockIdx.y * B * 3 * C;
+  const size_t n = (size_t)B * C;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = e / C;
+    const int c = (int)(e % C);
+    bf16 hi, mid;
+    split2(a[e], hi, mid);
+    bf16* o = dst + r * 3 * (size_t)C + c;
+    o[0] = hi; o[C] = hi; o[2 * (size_t)C] = mid;
+  }
+}
+
 __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_prev, float* h_out, float* c_out,
                          float* gates, size_t plane, float* h_in_copy, float* c_in_copy, int B, int H,
                          int64_t* counters) {
@@ -163,6 +182,38 @@ __global__ void colsum_accum(const T* v, int B, int N, float* out) {
   out[n] += s;
 }
 
+// Loss terms of n steps from their partial sums, each summed in index order.
+__global__ void sum_parts_steps(const float* part, int per_step, int n, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int a = blockIdx.x * blockDim.x + threadIdx.x;
+  if (a >= n) return;
+  float s = 0.f;
+  for (int i = 0; i < per_step; ++i) s += part[(size_t)a * per_step + i];
+  out[a] = s;
+}
+// part[a][c] = sum_b v[a][b][c], b ascending (blockIdx.y = a); then out[c] += part[a][c] for
+// a = n-1 .. 0 (time descending): the sums and the order of n single-step calls of colsum_accum.
+__global__ void colsum_steps(const float* v, int B, int N, float* part) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= N) return;
+  const float* blk = v + (size_t)blockIdx.y * B * N;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += blk[(size_t)b * N + c];
+  part[(size_t)blockIdx.y * N + c] = s;
+}
+__global__ void add_steps_descending(const float* part, int n, int N, float* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= N) return;
+  float acc = out[c];
+  for (int a = n - 1; a >= 0; --a) acc += part[(size_t)a * N + c];
+  out[c] = acc;
+}
+
 __global__ void sum_parts(const float* part, int n, float* out) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
@@ -222,6 +273,35 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]
   return gemm_bf16(dy3, 3 * a.O, false, w.woutmn3, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B,
                    a.H, 3 * a.O, w.status, s, true, &w.split);
+}
+
+// The readout of n steps at once (a run of backward operations inside one chunk): every element
+// by the sums of the single-step function, the contraction for dha split along K into the parts a
+// single step would take.
+int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, const float* target, float* loss_t,
+                float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s) {
+  bf16* h3 = w.st_h3 + (size_t)s_lo * B * 3 * H;
+  bf16* dy3 = w.st_dy3 + (size_t)s_lo * B * 3 * O;
+  const size_t nh = (size_t)B * H, no = (size_t)n * B * O;
+  RunPtrs ptrs{};
+  for (int a = 0; a < n; ++a) ptrs.p[a] = h_top[a];
+  launch_pdl(split_blocks3, dim3(ew_blocks(nh) > 64 ? 64 : ew_blocks(nh), n), dim3(256), 0, s, ptrs, H, B, h3);
+  const int parts = (O + 31) / 32, per_step = (B / 32) * parts;
+  GemmOut o{GemmOut::LOSS_DY, nullptr, O, b_out, 0};
+  o.target = target;
+  o.dy32 = w.dy_run;
+  o.loss_part = w.loss_part;
+  o.parts = parts;
+  o.scale = 1.f / ((float)B * (float)O);
+  int rc = gemm_bf16(h3, 3 * H, false, w.wout3, 3 * H, false, o, n * B, O, 3 * H, w.status, s);
+  if (rc != MEBPTT_OK) return rc;
+  launch_pdl(sum_parts_steps, dim3(1), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
+  launch_pdl(split_a3, dim3(ew_blocks(no)), dim3(256), 0, s, (const float*)w.dy_run, O, (const float*)nullptr, 0, n * B, dy3);
+  launch_pdl(colsum_steps, dim3((O + 127) / 128, n), dim3(128), 0, s, (const float*)w.dy_run, B, O, w.colsum_part);
+  launch_pdl(add_steps_descending, dim3((O + 127) / 128), dim3(128), 0, s, (const float*)w.colsum_part, n, O, db_out);
+  const int splits = tc::gemm_split_count(false, true, B, H, 3 * O, w.split.partial_floats);
+  return gemm_bf16(dy3, 3 * O, false, w.woutmn3, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H,
+                   3 * O, w.status, s, true, &w.split_run, splits);
 }
 
 int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_off, int sidx, cudaStream_t s) {

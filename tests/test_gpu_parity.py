@@ -267,6 +267,23 @@ def test_stepwise_runs_give_the_bits_of_single_operations(H, shape, monkeypatch)
             assert_bit_identical(r, single, want_dx=want_dx)
 
 
+@pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=45, readout=40),
+                                   dict(layers=1, input=256, hidden=1024, batch=32, t=70, readout=256)])
+def test_float32_storage_run_readout_gives_the_bits_of_single_operations(H, shape, monkeypatch):
+    """With float32 storage the readout of a run of backward operations is taken for the whole run
+    at once; operation by operation (MEBPTT_STEPWISE_PER_OP=1) the bits must be the same."""
+    cfg = _cfg("c4", **shape)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    plans = [dp.full_memory_plan(), dp.plan("msm", 11), dp.plan("ism", 3), dp.plan("hsm", 2)]
+    runs = [dp.run(p) for p in plans]
+    monkeypatch.setenv("MEBPTT_STEPWISE_PER_OP", "1")
+    single = dp.run(plans[0])
+    monkeypatch.delenv("MEBPTT_STEPWISE_PER_OP")
+    for p, r in zip(plans, runs):
+        assert r["counters"][0] == p.cost and r["counters"][1] == cfg.t and r["counters"][3] == 0
+        assert_bit_identical(r, single, want_dx=True)
+
+
 @pytest.mark.parametrize("shape", [dict(layers=2, input=64, hidden=72, batch=32, t=21, readout=40),
                                    dict(layers=1, input=24, hidden=256, batch=96, t=13, readout=8),
                                    dict(layers=1, input=128, hidden=1152, batch=32, t=9, readout=64)])
