@@ -225,6 +225,22 @@ size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc *desc);
  * is not counted (Section 3.1 sets the working core apart). */
 int64_t mebptt_budget_bytes_to_units(const mebptt_lstm_desc *desc, size_t bytes);
 
+/*
+ * Plan from a budget given in bytes (config 5 of the benchmark states its budgets that way).
+ * The bytes are turned into the mode's own unit -- hidden-state units for HSM and MSM, internal
+ * states (alpha = 4 units each) for ISM -- and the policy is that of mebptt_plan for that m.
+ *   include_working = 0: the budget is what the paper budgets, the memorised states only
+ *                        (Section 3 keeps the working core outside m).
+ *   include_working = 1: the budget is the whole device workspace of a training step: the largest
+ *                        m is taken for which mebptt_lstm_workspace_bytes of the resulting plan
+ *                        still fits.  (Appendix C notes that the working memory has to be part
+ *                        of the allowance once it is not negligible; here it is not: staging for
+ *                        a chunk of time steps, packed weights.)
+ * MEBPTT_ERR_BUDGET if not even m = 1 fits.  *out as for mebptt_plan.
+ */
+int mebptt_plan_for_bytes(const mebptt_lstm_desc *desc, size_t budget_bytes, int mode, int include_working,
+                          mebptt_plan_t **out);
+
 /* Size of the device workspace mebptt_lstm_train_step needs: the slot arena sized by the plan
  * plus working memory outside the budget.  0 on error. */
 size_t mebptt_lstm_workspace_bytes(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);

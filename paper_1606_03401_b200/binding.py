@@ -74,6 +74,7 @@ _SIGS = {
     "mebptt_plan_validate": (_i32, [_vp]),
     "mebptt_lstm_unit_bytes": (_sz, [_descp]),
     "mebptt_budget_bytes_to_units": (_i64, [_descp, _sz]),
+    "mebptt_plan_for_bytes": (_i32, [_descp, _sz, _i32, _i32, C.POINTER(_vp)]),
     "mebptt_lstm_workspace_bytes": (_sz, [_descp, _vp]),
     "mebptt_lstm_working_bytes": (_sz, [_descp, _vp]),
     "mebptt_lstm_host_workspace_bytes": (_sz, [_descp, _vp]),
@@ -196,6 +197,13 @@ def mebptt_lstm_unit_bytes(desc) -> int:
 
 def mebptt_budget_bytes_to_units(desc, nbytes: int) -> int:
     return lib.mebptt_budget_bytes_to_units(C.byref(desc), nbytes)
+
+
+def mebptt_plan_for_bytes(desc, nbytes: int, mode: int, include_working: bool = False) -> Plan:
+    h = _vp()
+    _check(lib.mebptt_plan_for_bytes(C.byref(desc), nbytes, mode, int(include_working), C.byref(h)),
+           "mebptt_plan_for_bytes")
+    return Plan(h)
 
 
 def mebptt_lstm_workspace_bytes(desc, plan: Plan) -> int:

@@ -373,6 +373,33 @@ int64_t mebptt_budget_bytes_to_units(const mebptt_lstm_desc* desc, size_t bytes)
   return u ? (int64_t)(bytes / u) : -1;
 }
 
+int mebptt_plan_for_bytes(const mebptt_lstm_desc* desc, size_t budget_bytes, int mode, int include_working,
+                          mebptt_plan_t** out) {
+  if (!out || !valid_desc(desc) || mode < MEBPTT_HSM || mode > MEBPTT_MSM) return MEBPTT_ERR_ARG;
+  *out = nullptr;
+  const size_t unit = mebptt_lstm_unit_bytes(desc);
+  if (!unit) return MEBPTT_ERR_ARG;
+  const size_t per_m = (mode == MEBPTT_ISM) ? 4 * unit : unit;   // what one more of the mode's units costs
+  int64_t m = (int64_t)(budget_bytes / per_m);
+  for (int round = 0; round < 64 && m >= 1; ++round) {
+    mebptt_plan_t* plan = nullptr;
+    const int rc = mebptt_plan(desc->t, m, mode, &plan);
+    if (rc != MEBPTT_OK) return rc;
+    if (!include_working) { *out = plan; return MEBPTT_OK; }
+    const size_t need = mebptt_lstm_workspace_bytes(desc, plan);
+    if (need == 0) { mebptt_plan_free(plan); return MEBPTT_ERR_UNSUPPORTED; }
+    if (need <= budget_bytes) { *out = plan; return MEBPTT_OK; }
+    // too large by `need - budget_bytes`: give up that many units (the working memory changes
+    // little with m, so this lands on or just above the answer; the loop settles the rest).
+    // A budget above the mode's saturation point was clamped by the planner: go on from there.
+    const int64_t m_used = mebptt_plan_m(plan);
+    mebptt_plan_free(plan);
+    const int64_t drop = (int64_t)((need - budget_bytes + per_m - 1) / per_m);
+    m = (m_used < m ? m_used : m) - (drop > 0 ? drop : 1);
+  }
+  return MEBPTT_ERR_BUDGET;
+}
+
 size_t mebptt_lstm_workspace_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
   if (check_common(desc, plan) != MEBPTT_OK) return 0;
   Layout y;

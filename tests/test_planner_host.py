@@ -158,6 +158,38 @@ def test_budget_clamping_and_errors():
         B.mebptt_plan_ex(10, 4, B.MEBPTT_MSM, 4, 5)
 
 
+def test_plan_from_a_byte_budget():
+    """Budgets in bytes (config 5's way of stating them): the mode's own unit, and, when the
+    working memory is to be counted, the largest m whose whole workspace fits."""
+    desc = B.make_desc(2, 1024, 2048, 1024, 128, 1000, "bf16")
+    unit = B.mebptt_lstm_unit_bytes(desc)
+    assert unit == 2 * 128 * 2048 * 6
+    plan = B.mebptt_plan_for_bytes(desc, 1 << 30, B.MEBPTT_MSM)
+    assert plan.m == 341 and plan.cost == _oracle_cost(P.MSM, 1000, 341)
+    assert B.mebptt_plan_for_bytes(desc, 4 << 30, B.MEBPTT_MSM).m == 1365
+    # 16 GiB is past the point where the cost stops falling: clamped, full memory
+    assert B.mebptt_plan_for_bytes(desc, 16 << 30, B.MEBPTT_MSM).cost == 1000
+    # internal states cost four units each
+    assert B.mebptt_plan_for_bytes(desc, 1 << 30, B.MEBPTT_ISM).m == (1 << 30) // (4 * unit)
+    # counting the working memory: the workspace fits, and one more unit would not
+    small = B.make_desc(1, 256, 256, 256, 64, 300, "bf16")
+    u = B.mebptt_lstm_unit_bytes(small)
+    for mode in (B.MEBPTT_HSM, B.MEBPTT_ISM, B.MEBPTT_MSM):
+        free = B.mebptt_plan_for_bytes(small, 64 << 20, mode)
+        budget = B.mebptt_lstm_working_bytes(small, free) + 37 * u + 1000
+        plan = B.mebptt_plan_for_bytes(small, budget, mode, include_working=True)
+        assert B.mebptt_lstm_workspace_bytes(small, plan) <= budget
+        nxt = B.mebptt_plan_ex(300, plan.m + 1, mode, 4, 0)
+        assert nxt.m == plan.m or B.mebptt_lstm_workspace_bytes(small, nxt) > budget
+        assert 1 <= plan.m <= 37
+    with pytest.raises(B.MebpttError) as e:
+        B.mebptt_plan_for_bytes(small, 4096, B.MEBPTT_MSM, include_working=True)
+    assert e.value.status == B.MEBPTT_ERR_BUDGET
+    with pytest.raises(B.MebpttError) as e:
+        B.mebptt_plan_for_bytes(small, u - 1, B.MEBPTT_HSM)
+    assert e.value.status == B.MEBPTT_ERR_BUDGET
+
+
 def test_descriptor_queries():
     d = B.make_desc(1, 1024, 1024, 1024, 64, 1000, "bf16")
     unit = B.mebptt_lstm_unit_bytes(d)
