@@ -41,7 +41,9 @@ WORKLOADS = {
     "c2": ("hsm", 64, [("hsm", 16), ("hsm", 256), ("ism", 16), ("ism", 64), ("ism", 256)]),
     # "chen": Chen's sqrt(t) schedule (Section 2.2) on the same executor; it needs 127 units at
     # t = 1000 (alpha = 4, beta = 3), so MSM at m = 127 is the like-for-like DP policy
-    "c3": ("msm", 100, [("msm", 10), ("msm", 32), ("msm", 127), ("chen", 0), ("msm", 1000)]),
+    # "chenrec": Chen's recursive schedule with k = 3 cuts per level (22 units at t = 1000), beside
+    # MSM at the same 22 units
+    "c3": ("msm", 100, [("msm", 10), ("msm", 22), ("chenrec", 3), ("msm", 32), ("msm", 127), ("chen", 0), ("msm", 1000)]),
     "c4": ("ism", 50, [("ism", 20), ("ism", 200), ("msm", 80), ("msm", 200), ("msm", 800)]),
     "c5": ("msm", 341, [("msm", 1365), ("msm", 5461)]),
     "p0": ("hsm", 100, [("hsm", 10), ("hsm", 50), ("hsm", 500), ("hsm", 1000)]),
@@ -357,7 +359,8 @@ def main():
     budgets = []
     if not args.no_budgets and rank == 0 or (not args.no_budgets and world > 1):
         for omode, om in others:
-            op = B.mebptt_plan_chen_sqrt(cfg.t, 4, 3) if omode == "chen" else dp.plan(omode, om)
+            op = (B.mebptt_plan_chen_sqrt(cfg.t, 4, 3) if omode == "chen" else
+                  B.mebptt_plan_chen_recursive(cfg.t, om, 4, 3) if omode == "chenrec" else dp.plan(omode, om))
             om = op.m
             oms, _ = timed(op, max(2, args.steps // 2), 1)
             oms = max_over(oms)

@@ -44,7 +44,8 @@ extern "C" {
 
 /* ---- enumerations ------------------------------------------------------------------ */
 enum { MEBPTT_HSM = 0, MEBPTT_ISM = 1, MEBPTT_MSM = 2,
-       MEBPTT_CHEN_SQRT = 3 /* reported by plans made with mebptt_plan_chen_sqrt; not accepted by mebptt_plan */ };
+       MEBPTT_CHEN_SQRT = 3,      /* reported by plans made with mebptt_plan_chen_sqrt; not accepted by mebptt_plan */
+       MEBPTT_CHEN_RECURSIVE = 4  /* likewise for mebptt_plan_chen_recursive */ };
 
 enum {
   MEBPTT_OK = 0,
@@ -131,6 +132,18 @@ int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_p
  * segments but the last.  It carries no DP tables (mebptt_plan_tables returns NULL pointers).
  */
 int mebptt_plan_chen_sqrt(int64_t t, int alpha, int beta, mebptt_plan_t **out);
+
+/*
+ * Chen's recursive schedule (Section 2.2), likewise: a sequence of more than k steps is cut into
+ * k + 1 parts as equal as they come (the first ones a step longer), one forward pass memorises the
+ * hidden states at the k cuts, and the parts are treated the same way from the last to the first;
+ * a sequence of at most k steps is run forward keeping every internal state and backpropagated.
+ * k = 1 is bisection, the least memory the scheme can do with (about log2 t hidden states).
+ * Reading of the paper's one-paragraph summary: "k" counts the states memorised per level, which
+ * is what its memory figure O(k log_{k+1} t) and its minimum log2 t at k = 1 need.
+ * alpha, beta, m, cost and tables as for mebptt_plan_chen_sqrt.  1 <= k <= 4096.
+ */
+int mebptt_plan_chen_recursive(int64_t t, int k, int alpha, int beta, mebptt_plan_t **out);
 
 void mebptt_plan_free(mebptt_plan_t *plan);
 

@@ -163,6 +163,44 @@ def chen_sqrt(t: int, alpha: int, beta: int | None = None):
     return {"forwards": forwards, "units": peak, "segment": s}
 
 
+def chen_recursive(t: int, k: int, alpha: int, beta: int | None = None):
+    """Forward operations and memory units of Chen's recursive schedule (Section 2.2).
+
+    A sequence of more than k steps is cut into k + 1 parts as equal as they come (the first ones
+    one step longer); one pass runs through all parts but the last and keeps the hidden state at
+    each of the k cuts; the parts are then treated the same way, last to first, each cut being
+    dropped once the part that starts there is done.  A sequence of at most k steps is run forward
+    keeping every internal state (beta units each when their input hidden states are left out,
+    else alpha) and backpropagated.  Units count the start state, as in the mixed scheme.
+    Reading: the paper's summary says "k equal parts"; k memorised states per level (k + 1
+    parts) is what its figures need -- memory O(k log_{k+1} t) and a minimum of log2 t at k = 1.
+    """
+    per = beta if beta is not None else alpha
+    memo = {}
+
+    def rec(n):
+        if n in memo:
+            return memo[n]
+        if n <= k:
+            memo[n] = (n, n * per)
+            return memo[n]
+        base, rem = divmod(n, k + 1)
+        sizes = [base + (1 if i < rem else 0) for i in range(k + 1)]
+        forwards = sum(sizes[:k])
+        peak = k
+        for j in range(k, -1, -1):          # while part j is treated, the cuts 1 .. j are still kept
+            f, pk = rec(sizes[j])
+            forwards += f
+            peak = max(peak, j + pk)
+        memo[n] = (forwards, peak)
+        return memo[n]
+
+    import sys
+    sys.setrecursionlimit(max(sys.getrecursionlimit(), 10000))
+    f, pk = rec(t)
+    return {"forwards": f, "units": 1 + pk}
+
+
 def saturation_budget(mode: int, t: int, alpha: int = 4) -> int:
     """Smallest budget beyond which more memory cannot lower the cost (used to cap tables)."""
     if mode == MSM:

@@ -14,7 +14,7 @@ import numpy as np
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("MEBPTT_LIB") or os.path.join(_PKG, "libmebptt.so")   # MEBPTT_LIB: another build of the library
 
-MEBPTT_HSM, MEBPTT_ISM, MEBPTT_MSM, MEBPTT_CHEN_SQRT = 0, 1, 2, 3
+MEBPTT_HSM, MEBPTT_ISM, MEBPTT_MSM, MEBPTT_CHEN_SQRT, MEBPTT_CHEN_RECURSIVE = 0, 1, 2, 3, 4
 MEBPTT_FP32, MEBPTT_TF32, MEBPTT_BF16 = 0, 1, 2
 MEBPTT_OK = 0
 MEBPTT_ERR_ARG, MEBPTT_ERR_BUDGET, MEBPTT_ERR_WORKSPACE, MEBPTT_ERR_UNSUPPORTED = -1, -2, -3, -4
@@ -57,6 +57,7 @@ _SIGS = {
     "mebptt_plan": (_i32, [_i64, _i64, _i32, C.POINTER(_vp)]),
     "mebptt_plan_ex": (_i32, [_i64, _i64, _i32, _i32, _i32, C.POINTER(_vp)]),
     "mebptt_plan_chen_sqrt": (_i32, [_i64, _i32, _i32, C.POINTER(_vp)]),
+    "mebptt_plan_chen_recursive": (_i32, [_i64, _i32, _i32, _i32, C.POINTER(_vp)]),
     "mebptt_plan_free": (None, [_vp]),
     "mebptt_plan_cost": (_i64, [_vp]),
     "mebptt_plan_num_ops": (_i64, [_vp]),
@@ -182,6 +183,12 @@ MEBPTT_FLAG_TIME_RUNS = 2
 def mebptt_plan_chen_sqrt(t: int, alpha: int = 4, beta: int = 3) -> Plan:
     h = _vp()
     _check(lib.mebptt_plan_chen_sqrt(t, alpha, beta, C.byref(h)), "mebptt_plan_chen_sqrt")
+    return Plan(h)
+
+
+def mebptt_plan_chen_recursive(t: int, k: int, alpha: int = 4, beta: int = 3) -> Plan:
+    h = _vp()
+    _check(lib.mebptt_plan_chen_recursive(t, k, alpha, beta, C.byref(h)), "mebptt_plan_chen_recursive")
     return Plan(h)
 
 

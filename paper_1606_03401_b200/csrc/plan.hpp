@@ -23,6 +23,7 @@ struct Plan {
 
 int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out);
 int build_chen_plan(int64_t t, int alpha, int beta, Plan** out);
+int build_chen_recursive_plan(int64_t t, int k, int alpha, int beta, Plan** out);
 int validate_plan(const Plan& p);
 
 }  // namespace mebptt

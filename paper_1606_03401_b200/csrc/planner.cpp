@@ -462,6 +462,95 @@ int build_chen_plan(int64_t t, int alpha, int beta, Plan** out) {
   return MEBPTT_OK;
 }
 
+// Chen's recursive schedule (Section 2.2) as a tape: a sequence of more than k steps is cut into
+// k + 1 parts as equal as they come, one forward pass memorises the hidden state at the k cuts,
+// and the parts are then treated the same way from the last to the first; a sequence of at most
+// k steps is run forward with every internal state kept and backpropagated.  (The paper's
+// summary speaks of "k equal parts" and of stopping "once the subsequence length becomes less than
+// k"; k memorised states per level, hence k + 1 parts, is the reading under which its figures --
+// memory O(k log_{k+1} t), at least log_2 t for k = 1 -- come out.)
+int build_chen_recursive_plan(int64_t t, int k, int alpha, int beta, Plan** out) {
+  if (!out) return MEBPTT_ERR_ARG;
+  *out = nullptr;
+  if (t < 1 || t > (int64_t)1 << 24 || k < 1 || k > 4096) return MEBPTT_ERR_ARG;
+  if (alpha < 2 || alpha > 64 || beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
+  Plan* p = new (std::nothrow) Plan();
+  if (!p) return MEBPTT_ERR_OOM;
+  p->t = t; p->mode = MEBPTT_CHEN_RECURSIVE; p->alpha = alpha; p->beta = beta;
+  try {
+    const int u = beta > 0 ? beta : alpha;
+    const int fmt = beta > 0 ? MEBPTT_FMT_INTERNAL_NOINPUT : MEBPTT_FMT_INTERNAL;
+    p->m = (int64_t)1 << 40;  // no budget while emitting; set to the peak below
+    Emitter e(*p);
+    struct Frame { int64_t start, len; int32_t loc; int stage; std::vector<int64_t> cut; std::vector<int32_t> locs; int j; };
+    std::vector<Frame> stack;
+    stack.push_back(Frame{0, t, MEBPTT_LOC_INIT, 0, {}, {}, 0});
+    std::vector<int32_t> slots, prevs;
+    while (!stack.empty()) {
+      Frame& f = stack.back();
+      if (f.len <= k) {
+        // every internal state of the segment, then back through them
+        int32_t prev = f.loc;
+        slots.clear(); prevs.clear();
+        for (int64_t i = 1; i <= f.len; ++i) {
+          const int32_t slot = (int32_t)e.top;
+          e.grow(u, u);
+          e.fwd(f.start + i, prev, slot, fmt);
+          slots.push_back(slot); prevs.push_back(prev);
+          prev = slot;
+        }
+        for (int64_t i = f.len; i >= 1; --i) {
+          e.bwd(f.start + i, slots[(size_t)i - 1], fmt, beta > 0 ? prevs[(size_t)i - 1] : 0);
+          e.shrink(u, u);
+        }
+        stack.pop_back();
+        continue;
+      }
+      if (f.stage == 0) {
+        // cuts[0] = start, cuts[k + 1] = end; the first len mod (k + 1) parts are one step longer
+        const int64_t parts = k + 1, base = f.len / parts, rem = f.len % parts;
+        f.cut.assign(1, f.start);
+        for (int64_t i = 0; i < parts; ++i) f.cut.push_back(f.cut.back() + base + (i < rem ? 1 : 0));
+        f.locs.assign(1, f.loc);
+        int32_t cur = f.loc;
+        for (int64_t i = 1; i <= k; ++i) {
+          const int32_t slot = (int32_t)e.top;
+          e.grow(1, 1);
+          e.sweep(f.cut[(size_t)i - 1], f.cut[(size_t)i] - f.cut[(size_t)i - 1], cur, slot, MEBPTT_FMT_HIDDEN);
+          f.locs.push_back(slot);
+          cur = slot;
+        }
+        f.stage = 1;
+        f.j = k;
+      } else {
+        // part j + 1 has just been backpropagated: the state at its start is no longer needed
+        e.shrink(1, 1);
+        --f.j;
+      }
+      if (f.j < 0) { stack.pop_back(); continue; }
+      if (f.j == 0) {
+        // the first part starts at the state the caller holds: nothing of ours to release after it
+        const Frame child{f.cut[0], f.cut[1] - f.cut[0], f.locs[0], 0, {}, {}, 0};
+        stack.pop_back();
+        stack.push_back(child);
+        continue;
+      }
+      const Frame child{f.cut[(size_t)f.j], f.cut[(size_t)f.j + 1] - f.cut[(size_t)f.j], f.locs[(size_t)f.j], 0, {}, {}, 0};
+      stack.push_back(child);
+    }
+    p->cost = 0;
+    for (const mebptt_op& op : p->tape) p->cost += (op.kind == MEBPTT_OP_FWD);
+    p->m = p->peak_units;
+  } catch (const std::bad_alloc&) {
+    delete p;
+    return MEBPTT_ERR_OOM;
+  }
+  int rc = validate_plan(*p);
+  if (rc != MEBPTT_OK) { delete p; return rc; }
+  *out = p;
+  return MEBPTT_OK;
+}
+
 int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out) {
   if (!out) return MEBPTT_ERR_ARG;
   *out = nullptr;
@@ -576,6 +665,9 @@ int mebptt_plan(int64_t t, int64_t m, int mode, mebptt_plan_t** out) {
   return mebptt::build_plan(t, m, mode, 4, 0, reinterpret_cast<Plan**>(out));
 }
 
+int mebptt_plan_chen_recursive(int64_t t, int k, int alpha, int beta, mebptt_plan_t** out) {
+  return mebptt::build_chen_recursive_plan(t, k, alpha, beta, reinterpret_cast<Plan**>(out));
+}
 int mebptt_plan_chen_sqrt(int64_t t, int alpha, int beta, mebptt_plan_t** out) {
   return mebptt::build_chen_plan(t, alpha, beta, reinterpret_cast<Plan**>(out));
 }

@@ -344,7 +344,8 @@ def test_c3_full_size_headline_budget(H):
 
 
 @pytest.mark.parametrize("base,kw", [("c1", dict()), ("c2", dict(t=70))])
-def test_chen_sqrt_plan_gives_the_same_gradients(H, base, kw):
+def test_chen_plans_give_the_same_gradients(H, base, kw):
+    """Chen's sqrt(t) and recursive schedules run on the same executor as the DP policies."""
     from paper_1606_03401_b200 import binding as B
     cfg = _cfg(base, **kw)
     dp = H.DeviceProblem(cfg, want_dx=True)
@@ -354,6 +355,11 @@ def test_chen_sqrt_plan_gives_the_same_gradients(H, base, kw):
         res = dp.run(plan)
         assert res["counters"][0] == plan.cost and res["counters"][2] == plan.peak_units and res["counters"][3] == 0
         assert_bit_identical(res, full, want_dx=True)
+        for k in (1, 3):
+            plan = B.mebptt_plan_chen_recursive(cfg.t, k, 4, beta)
+            res = dp.run(plan)
+            assert res["counters"][0] == plan.cost and res["counters"][2] == plan.peak_units and res["counters"][3] == 0
+            assert_bit_identical(res, full, want_dx=True)
 
 
 def test_c4_shape_truncated_ism_versus_msm(H):

@@ -249,3 +249,30 @@ def test_chen_sqrt_schedule(beta):
         assert "C" not in plan.tables()
     # two forward operations per step on average, at most (Section 2.2)
     assert B.mebptt_plan_chen_sqrt(1000, 4, 3).cost <= 2 * 1000
+
+
+@pytest.mark.parametrize("beta", [0, 3])
+def test_chen_recursive_schedule(beta):
+    """Chen's recursive schedule as a tape: cost and memory as the oracle derives them from the
+    description of Section 2.2; never cheaper than the DP at the same memory (Section 4.1); for
+    k = 1 (bisection) the memory is about log2 t hidden states, and the cost grows like
+    t log t (Section 2.2's figures)."""
+    import math
+    for t in (1, 2, 3, 7, 10, 17, 64, 100, 257, 1000):
+        for k in (1, 2, 3, 8, 31):
+            plan = B.mebptt_plan_chen_recursive(t, k, 4, beta)
+            ref = P.chen_recursive(t, k, 4, beta or None)
+            assert plan.mode == B.MEBPTT_CHEN_RECURSIVE
+            assert plan.cost == ref["forwards"] and plan.peak_units == ref["units"] == plan.m, (t, k)
+            assert plan.validate() == B.MEBPTT_OK
+            assert _replay(plan) == plan.cost
+            assert P.cost(P.MSM, t, plan.peak_units, 4, beta or None) <= plan.cost
+    per = 3
+    bis = B.mebptt_plan_chen_recursive(1024, 1, 4, per)
+    # ten levels of one cut each, the start state, and one internal state at the bottom
+    assert bis.peak_units == 1 + 10 + per
+    assert bis.cost == 1024 + 10 * 512
+    # with t <= k there is nothing to cut: standard BPTT
+    assert B.mebptt_plan_chen_recursive(20, 20, 4, 0).cost == 20
+    with pytest.raises(B.MebpttError):
+        B.mebptt_plan_chen_recursive(10, 0, 4, 3)
