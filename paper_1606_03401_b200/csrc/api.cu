@@ -104,6 +104,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     x3.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
     x3.loss_part = loss_part;
     x3.colsum_part = reinterpret_cast<float*>(ws + y.off_colsum);
+    x3.a3_run = bf(y.off_a3_run);
+    x3.h_run = reinterpret_cast<float*>(ws + y.off_hrun);
   }
   const bool staged = y.stepwise_tc || y.stepwise_x3;   // weight gradients per chunk of S steps
   int rc = MEBPTT_OK;
@@ -219,11 +221,36 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     for (const WorkItem& wi : items) {
       if (rc != MEBPTT_OK) break;
       const mebptt_op* ops = p->tape.data() + wi.i;
-      if (wi.kind == WorkItem::LEAF || wi.n == 1 || (y.stepwise_x3 && wi.kind == WorkItem::FWD)) {
-        // (with float32 storage a forward operation is one contraction over [input ; h], so there is
-        // nothing of it to take out of the recurrence)
-        const size_t cnt = wi.kind == WorkItem::LEAF ? 2 * (size_t)wi.n : (size_t)wi.n;
+      if (wi.kind == WorkItem::LEAF || wi.n == 1) {
+        const size_t cnt = wi.kind == WorkItem::LEAF ? 2 * (size_t)wi.n : 1;
         for (size_t j = 0; j < cnt && rc == MEBPTT_OK; ++j) run_op(ops[j]);
+      } else if (y.stepwise_x3 && wi.kind == WorkItem::FWD) {
+        // float32 storage: a forward operation is one contraction over [input ; h], so nothing of
+        // it can be taken out of the recurrence; what a run saves is the splitting of the operands
+        // (once for all inputs of the run; h_k by the cell kernel that produces it)
+        const int n = wi.n;
+        const int64_t k0 = ops[0].k;
+        for (int l = 0; l < y.L && rc == MEBPTT_OK; ++l) {
+          for (int j = 0; j < n; ++j) {
+            const mebptt_op& op = ops[j];
+            char* dst = loc_base(y, ws, op.dst);
+            stepwise::FwdRunStep& f = fst[j];
+            f = stepwise::FwdRunStep{};
+            hidden_at(y, io, op.src, l, &f.h_prev, &f.c_prev);
+            f.h_out = dst + y.h_off(l);
+            f.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
+            if (op.dst_fmt != MEBPTT_FMT_HIDDEN) f.gates = dst + y.rec_gates + (size_t)l * y.gsz;
+            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+              f.h_in_copy = dst + y.rec_in + y.h_off(l);
+              f.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
+            }
+          }
+          const int I_l = l == 0 ? y.I : y.H;
+          const float* in = (l == 0) ? reinterpret_cast<const float*>(io.x) + (size_t)(k0 - 1) * y.B * y.I : x3.h_run;
+          rc = stepwise3::forward_run_layer(fst.data(), n, in, (int64_t)y.B * I_l, I_l, io.b + (size_t)l * 4 * y.H, y.B,
+                                            y.H, plane_elems, l == 0 ? io.counters : nullptr, x3, w_off[l],
+                                            l + 1 < y.L ? x3.h_run : nullptr, s);
+        }
       } else if (y.stepwise_x3) {
         // float32 storage: the readout of the run at once, then its backward operations one by one
         const int n = wi.n;
@@ -459,12 +486,15 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t chunks = (p->t + y.S - 1) / y.S;
     // the readout of a run of n >= 2 backward operations is taken once for the run (split, GEMM with
     // loss, loss terms, split, two for db_out, dha)
-    int64_t readouts = 0;
+    // and a run of n >= 2 forward operations splits its operands once per layer (then GEMM and cell
+    // kernel per step)
+    int64_t readouts = 0, forwards = 0;
     for (const WorkItem& wi : work_items(p, y.S)) {
-      if (wi.kind == WorkItem::LEAF) readouts += wi.n * (5 + dha);
+      if (wi.kind == WorkItem::LEAF) { readouts += wi.n * (5 + dha); forwards += wi.n * 3 * L; }
       else if (wi.kind == WorkItem::BWD) readouts += wi.n == 1 ? 5 + dha : 6 + dha;
+      else forwards += wi.n == 1 ? 3 * L : L * (1 + 2 * (int64_t)wi.n);
     }
-    return 2 * L + 2 + p->cost * 3 * L + readouts + p->t * bwd + chunks * 3 * (2 * L + 1) + 1;
+    return 2 * L + 2 + forwards + readouts + p->t * bwd + chunks * 3 * (2 * L + 1) + 1;
   }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }

@@ -156,6 +156,8 @@ struct Scratch {
   float* loss_part;          // partial sums of the loss terms, per step
   float* colsum_part;        // [S][O]
   tc::SplitWs split_run;     // split-K scratch for a product over all rows of a run
+  __nv_bfloat16* a3_run;     // [S][B][3 (I + H)]: left operands of a run of forward operations
+  float* h_run;              // [S][B][H]: a layer's h_k of a run, the inputs of the layer above
 };
 // W: all layers' weights (float32), w_off[l] the element offset of layer l
 void pack_weights(const Scratch& w, int L, int I0, int H, int O, const float* W, const size_t* w_off,
@@ -170,5 +172,11 @@ int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, 
                 float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s);
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
                 float* dW_out, cudaStream_t s);
+// n consecutive forward operations of one layer (st as on the bfloat16 path).  in: the layer's input
+// of the first step, the others in_step_stride floats apart; h_stage (nullable): [n][B][H] copy of
+// the layer's h_k for the layer above.
+int forward_run_layer(const stepwise::FwdRunStep* st, int n, const float* in, int64_t in_step_stride, int I,
+                      const float* bias, int B, int H, size_t plane_elems, int64_t* counters, const Scratch& w,
+                      size_t w_off, float* h_stage, cudaStream_t s);
 }  // namespace stepwise3
 }  // namespace mebptt

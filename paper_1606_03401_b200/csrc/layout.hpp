@@ -53,7 +53,7 @@ struct Layout {
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
-  size_t off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, off_colsum = 0, split_floats = 0;
+  size_t off_a3_run = 0, off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, off_colsum = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
   int64_t arena_units = 0;
@@ -240,6 +240,8 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       const size_t rows = (size_t)y.S * y.B;
       y.off_z = take((size_t)y.B * G * 4);
       // the readout of a run of up to S steps at once; its split-K scratch as on the bfloat16 path
+      y.off_a3_run = take(rows * 3 * Kmax * 2);
+      y.off_hrun = take(y.L > 1 ? rows * y.H * 4 : 0);
       y.off_dy_run = take(rows * y.O * 4);
       y.off_dha_run = take(rows * y.H * 4);
       y.off_colsum = take((size_t)y.S * y.O * 4);

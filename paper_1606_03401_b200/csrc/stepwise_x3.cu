@@ -105,9 +105,35 @@ __global__ void split_blocks3(RunPtrs src, int C, int B, bf16* out) {
   }
 }
 
+// a3_next (optional): the left operand [B][3K] of the next step of a run, whose h columns
+// (I .. I + H - 1 of each third) receive the halves of h_k here instead of from a split kernel.
+// Left operands of a run of n forward operations: out[j] = [B][3 (I + H)] (blockIdx.y = j) gets the
+// halves of the layer input of step j in its input columns, and out[0] those of h0 (the h of the
+// state the run starts from) in its h columns; the h columns of the later steps are filled by the
+// cell kernel of the step before.
+__global__ void split_run_inputs(const float* in, int64_t in_step_stride, int I, const float* h0, int H, int B, bf16* out) {
+  sm100::grid_dep_wait();
+  sm100::grid_dep_launch();
+  const int j = blockIdx.y;
+  const size_t K = (size_t)I + H;
+  bf16* dst = out + (size_t)j * B * 3 * K;
+  const float* src = in + (size_t)j * in_step_stride;
+  const size_t n = (size_t)B * (j == 0 ? K : (size_t)I);
+  const size_t C = j == 0 ? K : (size_t)I;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = e / C;
+    const size_t c = e % C;
+    const float v = c < (size_t)I ? src[r * I + c] : h0[r * H + (c - I)];
+    bf16 hi, mid;
+    split2(v, hi, mid);
+    bf16* o = dst + r * 3 * K + c;
+    o[0] = hi; o[K] = hi; o[2 * K] = mid;
+  }
+}
+
 __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_prev, float* h_out, float* c_out,
                          float* gates, size_t plane, float* h_in_copy, float* c_in_copy, int B, int H,
-                         int64_t* counters) {
+                         int64_t* counters, bf16* a3_next, int I) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
@@ -119,7 +145,15 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_pre
     const float cp = c_prev[e];
     const float c = fmaf(gf, cp, gi * gg);
     c_out[e] = c;
-    h_out[e] = go * tanhf(c);
+    const float hv = go * tanhf(c);
+    h_out[e] = hv;
+    if (a3_next) {
+      const size_t K = (size_t)I + H;
+      bf16 hi, mid;
+      split2(hv, hi, mid);
+      bf16* o = a3_next + (size_t)b * 3 * K + I + j;
+      o[0] = hi; o[K] = hi; o[2 * K] = mid;
+    }
     if (gates) { gates[e] = gi; gates[plane + e] = gf; gates[2 * plane + e] = gg; gates[3 * plane + e] = go; }
     if (h_in_copy) { h_in_copy[e] = h_prev[e]; c_in_copy[e] = cp; }
   }
@@ -249,8 +283,37 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_of
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
   launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const float*)a.h_prev, (float*)a.h_out, a.c_out, (float*)a.gates,
-                                        a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters);
+                                        a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, 0);
   (void)l;
+  return MEBPTT_OK;
+}
+
+// n consecutive forward operations of one layer.  One launch splits the layer's inputs of all n
+// steps and the h of the state the run starts from into the left operands a3_run[j] = [B][3K];
+// every step is then the single-step contraction over its operand and the cell kernel, which also
+// writes the halves of h_k into the operand of the next step.  The operands hold what the
+// single-step function would have put there, so every sum is the same.
+int forward_run_layer(const stepwise::FwdRunStep* st, int n, const float* in, int64_t in_step_stride, int I, const float* bias,
+                      int B, int H, size_t plane_elems, int64_t* counters, const Scratch& w, size_t w_off,
+                      float* h_stage, cudaStream_t s) {
+  const int K = I + H, G = 4 * H;
+  const size_t row3 = (size_t)B * 3 * K;
+  launch_pdl(split_run_inputs, dim3(ew_blocks((size_t)B * K) > 128 ? 128 : ew_blocks((size_t)B * K), n), dim3(256), 0, s, in,
+             in_step_stride, I, (const float*)st[0].h_prev, H, B, w.a3_run);
+  const size_t nbh = (size_t)B * H;
+  for (int j = 0; j < n; ++j) {
+    const int rc = gemm_bf16(w.a3_run + (size_t)j * row3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false,
+                             GemmOut{GemmOut::STORE_F32, w.z, G, bias, 0}, B, G, 3 * K, w.status, s);
+    if (rc != MEBPTT_OK) return rc;
+    float* h_out = (float*)st[j].h_out;
+    launch_pdl(cell_fwd, dim3(ew_blocks(nbh)), dim3(256), 0, s, (const float*)w.z, st[j].c_prev, (const float*)st[j].h_prev, h_out,
+               st[j].c_out, (float*)st[j].gates, plane_elems, (float*)st[j].h_in_copy, st[j].c_in_copy, B, H, counters,
+               j + 1 < n ? w.a3_run + (size_t)(j + 1) * row3 : (bf16*)nullptr, I);
+    if (h_stage) {
+      // the layer above reads the h_k of the run from one block: a copy beside the tape's place
+      cudaMemcpyAsync(h_stage + (size_t)j * nbh, h_out, nbh * 4, cudaMemcpyDeviceToDevice, s);
+    }
+  }
   return MEBPTT_OK;
 }
 
