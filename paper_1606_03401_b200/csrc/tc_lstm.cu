@@ -1018,6 +1018,7 @@ struct SideStream {
   cudaStream_t copy = nullptr;                 // host-to-device copies that overlap the forward pass
   cudaEvent_t copy_from = nullptr, copy_done = nullptr;
   cudaEvent_t x_ready[X_PIECES] = {};          // pieces of x (along time) have arrived
+  cudaEvent_t t_ready[X_PIECES] = {};          // pieces of the targets have arrived (copied last piece first)
   bool ok = false;
 };
 SideStream* side_stream_for_current_device() {
@@ -1041,7 +1042,8 @@ SideStream* side_stream_for_current_device() {
          cudaEventCreateWithFlags(&t.copy_from, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&t.copy_done, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < X_PIECES && ok; ++i)
-      ok = cudaEventCreateWithFlags(&t.x_ready[i], cudaEventDisableTiming) == cudaSuccess;
+      ok = cudaEventCreateWithFlags(&t.x_ready[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&t.t_ready[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) cudaGetLastError();
     t.ok = ok;
   }
@@ -1107,12 +1109,15 @@ int run_times(double* ms, int64_t* launches, int64_t* ops) {
 
 // Inputs that are still in host memory, copied on the library's copy stream beside the forward
 // pass: x in X_PIECES pieces along the time axis (event x_ready[p] marks piece p), then the
-// targets (event copy_done).  Ordered after everything already in `s`: the previous step on `s`
-// may still read the destinations.
+// targets, likewise in pieces but from the last one to the first (event t_ready[p]): the backward
+// pass starts at the end of the sequence and reaches the early targets long after they arrive.
+// Ordered after everything already in `s`: the previous step on `s` may still read the destinations.
 struct LateCopies {
   SideStream* side = nullptr;
   int x_pieces = 0;            // 0: x was not copied here
   int64_t steps_per_piece = 0;
+  int t_pieces = 0;            // 0: the targets were not copied here
+  int64_t t_steps_per_piece = 0;
   bool targets = false;
 };
 LateCopies start_late_copies(const StepPtrs& io, int64_t t, cudaStream_t s) {
@@ -1134,7 +1139,16 @@ LateCopies start_late_copies(const StepPtrs& io, int64_t t, cudaStream_t s) {
     }
   }
   if (io.targets_host) {
-    cudaMemcpyAsync(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, cudaMemcpyHostToDevice, side->copy);
+    const size_t per_step = io.targets_bytes / (size_t)t;
+    lc.t_steps_per_piece = (t + X_PIECES - 1) / X_PIECES;
+    lc.t_pieces = (int)((t + lc.t_steps_per_piece - 1) / lc.t_steps_per_piece);
+    for (int p = lc.t_pieces - 1; p >= 0; --p) {
+      const int64_t lo = p * lc.t_steps_per_piece, hi = (lo + lc.t_steps_per_piece < t) ? lo + lc.t_steps_per_piece : t;
+      cudaMemcpyAsync(reinterpret_cast<char*>(const_cast<float*>(io.targets)) + (size_t)lo * per_step,
+                      (const char*)io.targets_host + (size_t)lo * per_step, (size_t)(hi - lo) * per_step,
+                      cudaMemcpyHostToDevice, side->copy);
+      cudaEventRecord(side->t_ready[p], side->copy);
+    }
     cudaEventRecord(side->copy_done, side->copy);
     lc.targets = true;
   }
@@ -1307,6 +1321,16 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       cudaStreamWaitEvent(s, late.side->x_ready[x_waited++], 0);
   };
 
+  int t_waited = 0;   // pieces of the targets, counted from the last, the caller's stream has waited for
+  auto need_targets = [&](int64_t k_lo) {   // the targets of time steps k_lo .. t are about to be read on `s`
+    if (!late.t_pieces) return;
+    const int first_piece = (int)((k_lo - 1) / late.t_steps_per_piece);
+    while (t_waited < late.t_pieces - first_piece) {
+      cudaStreamWaitEvent(s, late.side->t_ready[late.t_pieces - 1 - t_waited], 0);
+      ++t_waited;
+    }
+  };
+
   int launch_id = 0;
   int rc = MEBPTT_OK;
   if (!dry && !cuda_ok(cudaGetLastError(), "set-up (memsets, tape upload, weight packing)")) rc = MEBPTT_ERR_CUDA;
@@ -1365,7 +1389,6 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       const DevOp* bops = leaf ? dops + nops + i : dops + i;
       if (!targets_waited) {
         need_x(y.t);                                  // leaves and weight gradients read x anywhere
-        if (late.targets) cudaStreamWaitEvent(s, late.side->copy_done, 0);   // copied beside the forward pass
         targets_waited = true;
       }
       const int chunk = (first.k - 1) / S;
@@ -1373,6 +1396,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       const int n = wi.n;
       const int k_hi = first.k, k_lo = k_hi - n + 1;
       const int s_lo = (k_lo - 1) % S;
+      need_targets(k_lo);   // the targets of steps k_lo .. t (backward steps come in descending order)
       const size_t SB = (size_t)S * B;
       __nv_bfloat16* dz_c = dz + (size_t)pb * SB * G;
       __nv_bfloat16* hprev_c = hprev + (size_t)pb * SB * H;

@@ -107,12 +107,18 @@ def test_c2_shape_bf16_truncated(H):
         assert_bit_identical(res, full)
 
 
-def test_host_buffer_entry_point(H):
+@pytest.mark.parametrize("base,kw,mode,m", [("c1", dict(t=16), "hsm", 4),
+                                            ("c2", dict(input=128, hidden=256, batch=64, t=150, readout=128), "msm", 9),
+                                            ("c5", dict(layers=2, input=64, hidden=72, batch=32, t=21, readout=40), "msm", 9)])
+def test_host_buffer_entry_point(H, base, kw, mode, m):
+    """Host buffers in, host buffers out, on each of the paths (on the persistent tensor path x and
+    the targets are copied in pieces beside the forward pass, the targets last piece first): the
+    bits of the device-resident call."""
     import torch
     from paper_1606_03401_b200 import binding as B
-    cfg = _cfg("c1", t=16)
+    cfg = _cfg(base, **kw)
     dp = H.DeviceProblem(cfg, want_dx=True)
-    plan = dp.plan("hsm", 4)
+    plan = dp.plan(mode, m)
     dev = dp.run(plan)
     h = dp.host
     out = {k: np.zeros_like(v) for k, v in dev.items() if isinstance(v, np.ndarray)}
