@@ -433,3 +433,28 @@ def test_c5_full_size_properties(H):
     assert res["counters"][0] == plan.cost == P.cost(P.MSM, cfg.t, m, alpha=4)
     assert res["counters"][1] == cfg.t and res["counters"][2] <= m and res["counters"][3] == 0
     assert_bit_identical(res, full)
+
+
+@pytest.mark.parametrize("base,kw,plans", [
+    ("c1", dict(t=20), [("hsm", 4), ("msm", 9)]),                                                   # CUDA-core path
+    ("c2", dict(input=128, hidden=256, batch=64, t=70, readout=128), [("hsm", 5), ("msm", 13), ("ism", 70)]),  # persistent tensor path
+    ("c5", dict(layers=2, input=64, hidden=72, batch=32, t=45, readout=40), [("msm", 11), ("ism", 45)]),      # step by step, bf16
+    ("c4", dict(layers=1, input=64, hidden=128, batch=32, t=45, readout=40), [("msm", 11), ("ism", 45)]),     # step by step, float32 storage
+])
+def test_launch_count_is_what_the_profiler_sees(H, base, kw, plans):
+    """mebptt_lstm_launch_count (the benchmark's gpu_launches) against the kernels CUPTI records for
+    one training step (memsets and copies are not kernels and are not counted by either)."""
+    import torch
+    from torch.profiler import ProfilerActivity, profile
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg(base, **kw)
+    dp = H.DeviceProblem(cfg)
+    for mode, m in plans:
+        plan = dp.plan(mode, m)
+        dp.run(plan)
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            dp.enqueue(plan)
+            torch.cuda.synchronize()
+        seen = sum(1 for ev in prof.events()
+                   if ev.device_type == torch.autograd.DeviceType.CUDA and not ev.name.startswith(("Memset", "Memcpy")))
+        assert seen == B.mebptt_lstm_launch_count(dp.desc, plan), (base, mode, m, seen)
