@@ -84,7 +84,6 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     tcw.hrun = reinterpret_cast<__nv_bfloat16*>(ws + y.off_hrun);
     tcw.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
     tcw.loss_part = loss_part;
-    tcw.colsum_part = reinterpret_cast<float*>(ws + y.off_colsum);
   }
   stepwise3::Scratch x3{};
   size_t w_off[16];
@@ -103,7 +102,6 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     x3.dy_run = reinterpret_cast<float*>(ws + y.off_dy_run);
     x3.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
     x3.loss_part = loss_part;
-    x3.colsum_part = reinterpret_cast<float*>(ws + y.off_colsum);
     x3.a3_run = bf(y.off_a3_run);
     x3.h_run = reinterpret_cast<float*>(ws + y.off_hrun);
   }
@@ -197,8 +195,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         // the chunk's first step has been backpropagated: its weight gradients in one go
         const int64_t chunk = (k - 1) / y.S;
         const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
-        rc = y.stepwise_x3 ? stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s)
-                           : stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+        rc = y.stepwise_x3 ? stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, io.db, io.db_out, s)
+                           : stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, io.db, io.db_out, s);
       }
     }
   };
@@ -259,8 +257,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         auto op_at = [&](int a) -> const mebptt_op& { return ops[n - 1 - a]; };
         for (int a = 0; a < n; ++a) h_top[a] = loc_base(y, ws, op_at(a).src) + y.h_off(y.L - 1);
         rc = stepwise3::readout_run(reinterpret_cast<const float* const*>(h_top.data()), n, s_lo, io.b_out,
-                                    io.targets + (size_t)(k_lo - 1) * y.B * y.O, loss_t + (k_lo - 1), io.db_out, y.B, y.H,
-                                    y.O, x3, s);
+                                    io.targets + (size_t)(k_lo - 1) * y.B * y.O, loss_t + (k_lo - 1), y.B, y.H, y.O, x3, s);
         for (int a = n - 1; a >= 0 && rc == MEBPTT_OK; --a) {
           const mebptt_op& op = op_at(a);
           char* rec = loc_base(y, ws, op.src);
@@ -294,7 +291,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         if (s_lo == 0 && rc == MEBPTT_OK) {
           const int64_t chunk = (k_lo - 1) / y.S;
           const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
-          rc = stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+          rc = stepwise3::flush_chunk(x3, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, io.db, io.db_out, s);
         }
       } else if (wi.kind == WorkItem::FWD) {
         const int n = wi.n;
@@ -327,7 +324,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         auto op_at = [&](int a) -> const mebptt_op& { return ops[n - 1 - a]; };
         for (int a = 0; a < n; ++a) h_top[a] = loc_base(y, ws, op_at(a).src) + y.h_off(y.L - 1);
         rc = stepwise::readout_run(h_top.data(), n, s_lo, io.W_out, io.b_out, io.targets + (size_t)(k_lo - 1) * y.B * y.O,
-                                   loss_t + (k_lo - 1), io.db_out, y.B, y.H, y.O, tcw, s);
+                                   loss_t + (k_lo - 1), y.B, y.H, y.O, tcw, s);
         for (int l = y.L - 1; l >= 0 && rc == MEBPTT_OK; --l) {
           for (int a = 0; a < n; ++a) {
             const mebptt_op& op = op_at(a);
@@ -345,13 +342,12 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
           }
           float* d_lo = (l > 0) ? tcw.dha_run : (desc->want_dx ? io.dx + (size_t)(k_lo - 1) * y.B * y.I : nullptr);
           rc = stepwise::backward_run_layer(bst.data(), n, s_lo, l, l == 0 ? y.I : y.H, io.W + y.w_layer_offset(l) * y.esz,
-                                            dh_rec + (size_t)l * bh, dc_rec + (size_t)l * bh, dz, io.db + (size_t)l * 4 * y.H,
-                                            d_lo, y.B, y.H, plane_elems, l == y.L - 1 ? io.counters : nullptr, tcw, s);
+                                            dh_rec + (size_t)l * bh, dc_rec + (size_t)l * bh, d_lo, y.B, y.H, plane_elems, l == y.L - 1 ? io.counters : nullptr, tcw, s);
         }
         if (s_lo == 0 && rc == MEBPTT_OK) {
           const int64_t chunk = (k_lo - 1) / y.S;
           const int steps = (int)((chunk + 1) * y.S <= y.t ? y.S : y.t - chunk * y.S);
-          rc = stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, s);
+          rc = stepwise::flush_chunk(tcw, steps, y.L, y.B, y.I, y.H, y.O, w_off, io.dW, io.dW_out, io.db, io.db_out, s);
         }
       }
     }
@@ -451,50 +447,49 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
   // 4 per layer; one to finalise
   const int64_t L = desc->layers;
   if (y.stepwise_tc) {
-    // forward operation: two GEMMs and the cell kernel per layer; readout: 3 and the dha GEMM;
-    // backward operation per layer: gate kernel, db, and one or two d_in GEMMs
+    // forward operation: two GEMMs and the cell kernel per layer; readout: GEMM with loss, loss
+    // term and stage, dha GEMM; backward operation per layer: gate kernel and one or two d_in GEMMs
     // (a contraction that is split along K takes a second launch to add its parts)
     const size_t pf = (size_t)148 * 128 * 128;
     const int G = 4 * y.H;
     const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, G, pf) > 1 ? 2 : 1;   // dz W -> [B][H]
     const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, G, pf) > 1 ? 2 : 1;   // dz W -> [B][I]
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, y.O, pf) > 1 ? 2 : 1;
-    const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
-    const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs
+    const int64_t bwd = L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs and L + 1 bias sums
     // runs of n >= 2 operations go layer by layer: one input product per layer and run, the
-    // readout once per run (stage, GEMM with loss, loss terms, dha, two for db_out), the gradient handed
-    // down once per layer and run
-    int64_t n_launch = chunks * (2 * L + 1) + 1;
+    // readout once per run (stage, GEMM with loss, loss terms, dha), the gradient handed down
+    // once per layer and run
+    int64_t n_launch = chunks * (3 * L + 2) + 1;
     for (const WorkItem& wi : work_items(p, y.S)) {
-      if (wi.kind == WorkItem::LEAF) n_launch += wi.n * (3 * L + 3 + dha + bwd);
+      if (wi.kind == WorkItem::LEAF) n_launch += wi.n * (3 * L + 2 + dha + bwd);
       else if (wi.kind == WorkItem::FWD) n_launch += wi.n == 1 ? 3 * L : L * (1 + 2 * (int64_t)wi.n);
-      else if (wi.n == 1) n_launch += 3 + dha + bwd;
-      else n_launch += 5 + dha + L * wi.n * (2 + to_h) + (L - 1) * to_h + (desc->want_dx ? to_x : 0);
+      else if (wi.n == 1) n_launch += 2 + dha + bwd;
+      else n_launch += 3 + dha + L * wi.n * (1 + to_h) + (L - 1) * to_h + (desc->want_dx ? to_x : 0);
     }
     return n_launch;
   }
   if (y.stepwise_x3) {
     // weights: 2 packing kernels per layer and 2 for the readout; forward operation: split, GEMM,
-    // cell per layer; readout: split, GEMM, loss sum, split, db_out, dha GEMM; backward operation
-    // per layer: gate kernel, db, one or two d_in GEMMs; a chunk: 3 GEMMs per product
+    // cell per layer; readout: split, GEMM, loss sum, split, dha GEMM; backward operation per
+    // layer: gate kernel, one or two d_in GEMMs; a chunk: 3 GEMMs per product and L + 1 bias sums
     const size_t pf = (size_t)148 * 128 * 128;
     const int G = 4 * y.H;
     const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, 3 * G, pf) > 1 ? 2 : 1;
     const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, 3 * G, pf) > 1 ? 2 : 1;
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, 3 * y.O, pf) > 1 ? 2 : 1;
-    const int64_t bwd = 2 * L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    const int64_t bwd = L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
     const int64_t chunks = (p->t + y.S - 1) / y.S;
-    // the readout of a run of n >= 2 backward operations is taken once for the run (split, GEMM with
-    // loss, loss terms, split, two for db_out, dha)
-    // and a run of n >= 2 forward operations splits its operands once per layer (then GEMM and cell
-    // kernel per step)
+    // the readout of a run of n >= 2 backward operations is taken once for the run (the same
+    // launches), and a run of n >= 2 forward operations splits its operands once per layer (then
+    // GEMM and cell kernel per step)
     int64_t readouts = 0, forwards = 0;
     for (const WorkItem& wi : work_items(p, y.S)) {
-      if (wi.kind == WorkItem::LEAF) { readouts += wi.n * (5 + dha); forwards += wi.n * 3 * L; }
-      else if (wi.kind == WorkItem::BWD) readouts += wi.n == 1 ? 5 + dha : 6 + dha;
+      if (wi.kind == WorkItem::LEAF) { readouts += wi.n * (4 + dha); forwards += wi.n * 3 * L; }
+      else if (wi.kind == WorkItem::BWD) readouts += 4 + dha;
       else forwards += wi.n == 1 ? 3 * L : L * (1 + 2 * (int64_t)wi.n);
     }
-    return 2 * L + 2 + forwards + readouts + p->t * bwd + chunks * 3 * (2 * L + 1) + 1;
+    return 2 * L + 2 + forwards + readouts + p->t * bwd + chunks * (3 * (2 * L + 1) + L + 1) + 1;
   }
   return p->cost * L + p->t * (5 + 4 * L) + 1;
 }

@@ -95,16 +95,15 @@ struct Scratch {
   __nv_bfloat16* hrun;      // [S B][H]  the layer's h_k, read by the layer above
   float* dha_run;           // [S B][H]  gradient entering the layer at each step (row block: step - first step)
   float* loss_part;         // partial sums of the loss terms, per step
-  float* colsum_part;       // [S][O] per-step column sums of dy
   tc::SplitWs split_run;    // split-K scratch for a product over all rows of a run
 };
 int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s);
 // sidx: row block of this step in the stages; l: layer
 int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStream_t s);
 int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx, cudaStream_t s);
-// dW (w_off[l]: element offset of layer l) and dW_out from the first `steps` row blocks of the stages
+// dW (w_off[l]: element offset of layer l), db ([L][4H]), dW_out and db_out from the first `steps` row blocks of the stages
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
-                float* dW_out, cudaStream_t s);
+                float* dW_out, float* db, float* db_out, cudaStream_t s);
 
 // One step of a run, as one layer sees it.
 struct FwdRunStep {
@@ -123,11 +122,11 @@ int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const 
 // whose stages are the row blocks s_lo .. s_lo + n - 1; h_top[a]: the top layer's h of step s_lo + a;
 // target, loss_t: those of the first of the steps.
 int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out, const float* b_out, const float* target,
-                float* loss_t, float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s);
+                float* loss_t, int B, int H, int O, const Scratch& w, cudaStream_t s);
 // The n backward operations of layer l, time descending (st[a]: step s_lo + a), reading w.dha_run;
 // d_lo (nullable): [n B][I] gradient w.r.t. the layer's inputs, written once for the whole run.
 int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, const void* W, float* dh_rec, float* dc_rec,
-                       float* dz, float* db, float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
+                       float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
                        const Scratch& w, cudaStream_t s);
 }  // namespace stepwise
 
@@ -154,7 +153,6 @@ struct Scratch {
   float* dy_run;             // [S B][O]
   float* dha_run;            // [S B][H]  gradient entering the top layer at each step of the run
   float* loss_part;          // partial sums of the loss terms, per step
-  float* colsum_part;        // [S][O]
   tc::SplitWs split_run;     // split-K scratch for a product over all rows of a run
   __nv_bfloat16* a3_run;     // [S][B][3 (I + H)]: left operands of a run of forward operations
   float* h_run;              // [S][B][H]: a layer's h_k of a run, the inputs of the layer above
@@ -169,9 +167,9 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_
 // step s_lo + a) of n steps at once; h_top[a]: the top layer's h of step s_lo + a; target, loss_t:
 // those of the first of the steps.
 int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, const float* target, float* loss_t,
-                float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s);
+                int B, int H, int O, const Scratch& w, cudaStream_t s);
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
-                float* dW_out, cudaStream_t s);
+                float* dW_out, float* db, float* db_out, cudaStream_t s);
 // n consecutive forward operations of one layer (st as on the bfloat16 path).  in: the layer's input
 // of the first step, the others in_step_stride floats apart; h_stage (nullable): [n][B][H] copy of
 // the layer's h_k for the layer above.

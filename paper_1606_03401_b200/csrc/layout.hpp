@@ -53,7 +53,7 @@ struct Layout {
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
   size_t off_sync = 0, off_tape = 0, off_status = 0;
-  size_t off_a3_run = 0, off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, off_colsum = 0, split_floats = 0;
+  size_t off_a3_run = 0, off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
   int64_t arena_units = 0;
@@ -227,7 +227,6 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_zrun = take(rows * 4 * y.H * 4);
       y.off_hrun = take(rows * y.H * 2);
       y.off_dha_run = take(rows * y.H * 4);
-      y.off_colsum = take((size_t)y.S * y.O * 4);
       // split-K scratch: a wave of 128 x 128 float32 tiles for one step, times the 8 row tiles of
       // a whole run (its products are split like a single step's, to sum in the same order)
       y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
@@ -244,7 +243,6 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_hrun = take(y.L > 1 ? rows * y.H * 4 : 0);
       y.off_dy_run = take(rows * y.O * 4);
       y.off_dha_run = take(rows * y.H * 4);
-      y.off_colsum = take((size_t)y.S * y.O * 4);
       y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
       y.off_split = take(y.split_floats * 4);
       y.off_a3 = take((size_t)y.B * 3 * Kmax * 2);

@@ -6,15 +6,15 @@
 // path does, but with its contractions given to the tcgen05 GEMM (bfloat16 operands, float32
 // accumulation in a fixed order) and the gate arithmetic in small element-wise kernels:
 //   forward    z  = in W[:, :I]^T + b ;  z += h_prev W[:, I:]^T ;  gates, c, h from z
-//   readout    y  = h W_out^T + b_out, loss term and dy in the GEMM's epilogue ; dha = dy W_out ;
-//              dW_out += dy^T h ; db_out += sum_b dy
-//   backward   dz from the stored gates ; db += sum_b dz ; d_in = dz W[:, :I] ; dh = dz W[:, I:]
-//   per chunk  dW += dz^T [in ; h_prev] and dW_out += dy^T h over the S steps of a chunk at once:
-//              dz, dy and the operands they meet are staged per step (row block (k - 1) % S), and
-//              the chunk is flushed when its first step has been backpropagated.  Chunks are
-//              tied to absolute time, so the order of every sum is the same for every plan.
-// dz and dy are rounded to bfloat16 before they enter a contraction (as on the persistent path);
-// db is summed from the unrounded dz.  Every sum has a fixed order, and an operation's launches
+//   readout    y  = h W_out^T + b_out, loss term and dy in the GEMM's epilogue ; dha = dy W_out
+//   backward   dz from the stored gates ; d_in = dz W[:, :I] ; dh = dz W[:, I:]
+//   per chunk  dW += dz^T [in ; h_prev], db += sum of dz, dW_out += dy^T h and db_out += sum of dy
+//              over the S steps of a chunk at once: dz, dy and the operands they meet are staged
+//              per step (row block (k - 1) % S), and the chunk is flushed when its first step has
+//              been backpropagated.  Chunks are tied to absolute time, so the order of every sum
+//              is the same for every plan.
+// dz and dy are rounded to bfloat16 before they enter a contraction or a bias gradient (as on the
+// persistent path).  Every sum has a fixed order, and an operation's launches
 // do not depend on the plan, so results are bit-identical across plans.
 #include "kernels.hpp"
 #include "launch.hpp"
@@ -92,7 +92,7 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
     const float v2 = dc * gi * (1.f - gg * gg);
     const float v3 = d_o * go * (1.f - go);
     const size_t r = (size_t)b * 4 * H + j;
-    dz[r] = v0; dz[r + H] = v1; dz[r + 2 * (size_t)H] = v2; dz[r + 3 * (size_t)H] = v3;
+    if (dz) { dz[r] = v0; dz[r + H] = v1; dz[r + 2 * (size_t)H] = v2; dz[r + 3 * (size_t)H] = v3; }
     dz16[r] = __float2bfloat16_rn(v0); dz16[r + H] = __float2bfloat16_rn(v1);
     dz16[r + 2 * (size_t)H] = __float2bfloat16_rn(v2); dz16[r + 3 * (size_t)H] = __float2bfloat16_rn(v3);
     dc_rec[e] = dc * gf;
@@ -100,16 +100,40 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
   if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
 }
 
-// out[n] += sum_b v[b][n], b ascending
-template <class T>
-__global__ void colsum_accum(const T* v, int B, int N, float* out) {
+// out[c] += sum over the rows r = 0 .. R-1 of v[r][c]: the bias gradients of a chunk from its
+// staged rows (row = step within the chunk, then batch index).  Sixteen partial sums per column
+// (rows r = y, y + 16, ... ascending for y = 0 .. 15), added in the order of y: fixed, and the
+// same whatever the plan.  One block per 64 columns (N is a multiple of 8).
+__global__ void __launch_bounds__(512) colsum_rows(const bf16* v, int R, int N, float* out) {
+  __shared__ float part[16][64];
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  if (n >= N) return;
-  float s = 0.f;
-  for (int b = 0; b < B; ++b) s += (float)v[(size_t)b * N + n];
-  out[n] += s;
+  const int c = blockIdx.x * 64 + 2 * threadIdx.x, y = threadIdx.y;
+  float a0 = 0.f, a1 = 0.f;
+  if (c < N) {
+    int r = y;
+    for (; r + 48 < R; r += 64) {
+      __nv_bfloat162 x[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) x[u] = *reinterpret_cast<const __nv_bfloat162*>(v + (size_t)(r + 16 * u) * N + c);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { a0 += __low2float(x[u]); a1 += __high2float(x[u]); }
+    }
+    for (; r < R; r += 16) {
+      const __nv_bfloat162 x = *reinterpret_cast<const __nv_bfloat162*>(v + (size_t)r * N + c);
+      a0 += __low2float(x); a1 += __high2float(x);
+    }
+  }
+  part[y][2 * threadIdx.x] = a0;
+  part[y][2 * threadIdx.x + 1] = a1;
+  __syncthreads();
+  const int t = y * 32 + threadIdx.x;
+  if (t < 64 && blockIdx.x * 64 + t < N) {
+    float acc = 0.f;
+#pragma unroll
+    for (int g = 0; g < 16; ++g) acc += part[g][t];
+    out[blockIdx.x * 64 + t] += acc;
+  }
 }
 
 // Loss term of one step from its partial sums (block 0, one thread); every block helps copy the
@@ -149,30 +173,6 @@ __global__ void sum_parts_steps(const float* part, int per_step, int n, float* o
   out[a] = s;
 }
 
-// Column sums of n row blocks at once: part[a][c] = sum_b v[a][b][c], b ascending (blockIdx.y = a),
-// then out[c] += part[a][c] for a = n-1 .. 0 (time descending): the sums and the order of n
-// single-step calls of colsum_accum.
-template <class T>
-__global__ void colsum_steps(const T* v, int B, int N, float* part) {
-  sm100::grid_dep_wait();
-  sm100::grid_dep_launch();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= N) return;
-  const T* blk = v + (size_t)blockIdx.y * B * N;
-  float s = 0.f;
-  for (int b = 0; b < B; ++b) s += (float)blk[(size_t)b * N + c];
-  part[(size_t)blockIdx.y * N + c] = s;
-}
-__global__ void add_steps_descending(const float* part, int n, int N, float* out) {
-  sm100::grid_dep_wait();
-  sm100::grid_dep_launch();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= N) return;
-  float acc = out[c];
-  for (int a = n - 1; a >= 0; --a) acc += part[(size_t)a * N + c];
-  out[c] = acc;
-}
-
 inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
 
 }  // namespace
@@ -208,9 +208,7 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]: W_out read as the [k][n] operand
   rc = gemm_bf16(dy16, a.O, false, W_out, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B, a.H,
                  a.O, w.status, s, true, &w.split);
-  if (rc != MEBPTT_OK) return rc;
-  launch_pdl(colsum_accum<bf16>, dim3((a.O + 127) / 128), dim3(128), 0, s, dy16, a.B, a.O, a.db_out);
-  return MEBPTT_OK;
+  return rc;   // db_out is summed from the staged dy when the chunk is flushed
 }
 
 int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx, cudaStream_t s) {
@@ -222,10 +220,9 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
   bf16* st_in = w.st_in + (l == 0 ? 0 : rows * w.I0 + (size_t)(l - 1) * rows * a.H) + (size_t)sidx * a.B * a.I;
   bf16* st_hp = w.st_hp + ((size_t)l * rows + (size_t)sidx * a.B) * a.H;
   launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
-                                        a.dz, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
+                                        (float*)nullptr, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
                                         (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
                                         (size_t)a.B * a.H * 2 / 16);
-  launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, a.dz, a.B, G, a.db);
   // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
   if (a.d_lo) {
     int rc = gemm_bf16(dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
@@ -238,12 +235,14 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
 
 // Weight gradients of a finished chunk: `steps` row blocks of B rows, from block 0 on.
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
-                float* dW_out, cudaStream_t s) {
+                float* dW_out, float* db, float* db_out, cudaStream_t s) {
   const int G = 4 * H, R = steps * B;
   const size_t rows = (size_t)w.S * B;
   for (int l = 0; l < L; ++l) {
     const int I = l == 0 ? I0 : H, K = I + H;
     const bf16* dz = w.st_dz + (size_t)l * rows * G;
+    // db[g] += sum over (step, b) of the staged dz (as the contractions below see it)
+    launch_pdl(colsum_rows, dim3((G + 63) / 64), dim3(32, 16), 0, s, dz, R, G, db + (size_t)l * G);
     const bf16* in = w.st_in + (l == 0 ? 0 : rows * I0 + (size_t)(l - 1) * rows * H);
     const bf16* hp = w.st_hp + (size_t)l * rows * H;
     float* dWl = dW + w_off[l];
@@ -253,6 +252,7 @@ int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O,
     rc = gemm_bf16(dz, G, true, hp, H, true, GemmOut{GemmOut::ACCUM_F32, dWl + I, K, nullptr, 0}, G, H, R, w.status, s);
     if (rc != MEBPTT_OK) return rc;
   }
+  launch_pdl(colsum_rows, dim3((O + 63) / 64), dim3(32, 16), 0, s, (const bf16*)w.st_dy, R, O, db_out);
   return gemm_bf16(w.st_dy, O, true, w.st_h, H, true, GemmOut{GemmOut::ACCUM_F32, dW_out, H, nullptr, 0}, O, H, R,
                    w.status, s);
 }
@@ -285,7 +285,7 @@ int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const 
 }
 
 int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out_, const float* b_out, const float* target,
-                float* loss_t, float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s) {
+                float* loss_t, int B, int H, int O, const Scratch& w, cudaStream_t s) {
   const bf16* W_out = (const bf16*)W_out_;
   const size_t n_h16 = (size_t)B * H * 2 / 16;
   RunPtrs ptrs{};
@@ -307,14 +307,11 @@ int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out_, c
   const int splits = tc::gemm_split_count(false, true, B, H, O, w.split.partial_floats);
   rc = gemm_bf16(dy16, O, false, W_out, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H, O,
                  w.status, s, true, &w.split_run, splits);
-  if (rc != MEBPTT_OK) return rc;
-  launch_pdl(colsum_steps<bf16>, dim3((O + 127) / 128, n), dim3(128), 0, s, (const bf16*)dy16, B, O, w.colsum_part);
-  launch_pdl(add_steps_descending, dim3((O + 127) / 128), dim3(128), 0, s, (const float*)w.colsum_part, n, O, db_out);
-  return MEBPTT_OK;
+  return rc;
 }
 
 int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, const void* Wl, float* dh_rec, float* dc_rec,
-                       float* dz, float* db, float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
+                       float* d_lo, int B, int H, size_t plane_elems, int64_t* counters,
                        const Scratch& w, cudaStream_t s) {
   const int K = I + H, G = 4 * H;
   const size_t bh = (size_t)B * H;
@@ -327,10 +324,9 @@ int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, cons
     const size_t row0 = (size_t)(s_lo + a) * B;
     bf16* dz16 = dz_l + row0 * G;
     launch_pdl(gate_bwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)(w.dha_run + (size_t)a * bh), (const float*)dh_rec,
-               dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t, st[a].c_prev, dz, dz16, B, H, counters,
+               dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t, st[a].c_prev, (float*)nullptr, dz16, B, H, counters,
                (const uint4*)st[a].in, (uint4*)(in_l + row0 * I), (size_t)B * I * 2 / 16, (const uint4*)st[a].h_prev,
                (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16);
-    launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, (const float*)dz, B, G, db);
     const int rc = gemm_bf16(dz16, G, false, W + I, K, true, GemmOut{GemmOut::STORE_F32, dh_rec, H, nullptr, 0}, B, H, G,
                              w.status, s, true, &w.split);
     if (rc != MEBPTT_OK) return rc;

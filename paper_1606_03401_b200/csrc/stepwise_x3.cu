@@ -13,10 +13,10 @@
 // Operations (per layer), with K = I + H, G = 4H:
 //   forward    a3 = split([in ; h_prev]) ; z = a3 W3^T + b ; gates, c, h from z
 //   readout    h3 = split(h) ; y = h3 Wout3^T + b_out with loss and dy (float32) in the epilogue ;
-//              dy3 = split(dy) ; db_out += sum_b dy ; dha = dy3 WoutMN3
-//   backward   dz (float32) and dz3 from the stored gates ; db += sum_b dz ; d_in = dz3 WMN3
+//              dy3 = split(dy) ; dha = dy3 WoutMN3
+//   backward   dz3 from the stored gates ; d_in = dz3 WMN3
 //   per chunk  dW += dz^T [in ; h_prev], dW_out += dy^T h from the staged halves: three GEMMs per
-//              product (hi hi, hi mid, mid hi)
+//              product (hi hi, hi mid, mid hi); db += sum of dz, db_out += sum of dy, as hi + mid
 // All sums run in a fixed order and nothing depends on the plan: results are bit-identical across
 // plans.
 #include "kernels.hpp"
@@ -181,7 +181,7 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const size_t col = (size_t)q * H + j;
-      dz[(size_t)b * G + col] = v[q];
+      if (dz) dz[(size_t)b * G + col] = v[q];
       bf16 hi, mid;
       split2(v[q], hi, mid);
       bf16* o = dz3 + (size_t)b * 3 * G + col;
@@ -205,15 +205,36 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
   if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
 }
 
-template <class T>
-__global__ void colsum_accum(const T* v, int B, int N, float* out) {
+// out[c] += sum over the rows r = 0 .. R-1 of hi + mid, for rows [hi | hi | mid] of width 3 N as
+// the stages hold them: the bias gradients of a chunk (row = step within the chunk, then batch
+// index).  Sixteen partial sums per column (rows r = y, y + 16, ... ascending for y = 0 .. 15),
+// added in the order of y: fixed, and the same whatever the plan.  One block per 64 columns (N is
+// a multiple of 8).
+__global__ void __launch_bounds__(512) colsum_rows3(const bf16* v3, int R, int N, float* out) {
+  __shared__ float part[16][64];
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  if (n >= N) return;
-  float s = 0.f;
-  for (int b = 0; b < B; ++b) s += (float)v[(size_t)b * N + n];
-  out[n] += s;
+  const int c = blockIdx.x * 64 + 2 * threadIdx.x, y = threadIdx.y;
+  float a0 = 0.f, a1 = 0.f;
+  if (c < N) {
+    for (int r = y; r < R; r += 16) {
+      const bf16* row = v3 + (size_t)r * 3 * N + c;
+      const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(row);
+      const __nv_bfloat162 mid = *reinterpret_cast<const __nv_bfloat162*>(row + 2 * (size_t)N);
+      a0 += __low2float(hi) + __low2float(mid);
+      a1 += __high2float(hi) + __high2float(mid);
+    }
+  }
+  part[y][2 * threadIdx.x] = a0;
+  part[y][2 * threadIdx.x + 1] = a1;
+  __syncthreads();
+  const int t = y * 32 + threadIdx.x;
+  if (t < 64 && blockIdx.x * 64 + t < N) {
+    float acc = 0.f;
+#pragma unroll
+    for (int g = 0; g < 16; ++g) acc += part[g][t];
+    out[blockIdx.x * 64 + t] += acc;
+  }
 }
 
 // Loss terms of n steps from their partial sums, each summed in index order.
@@ -226,28 +247,6 @@ __global__ void sum_parts_steps(const float* part, int per_step, int n, float* o
   for (int i = 0; i < per_step; ++i) s += part[(size_t)a * per_step + i];
   out[a] = s;
 }
-// part[a][c] = sum_b v[a][b][c], b ascending (blockIdx.y = a); then out[c] += part[a][c] for
-// a = n-1 .. 0 (time descending): the sums and the order of n single-step calls of colsum_accum.
-__global__ void colsum_steps(const float* v, int B, int N, float* part) {
-  sm100::grid_dep_wait();
-  sm100::grid_dep_launch();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= N) return;
-  const float* blk = v + (size_t)blockIdx.y * B * N;
-  float s = 0.f;
-  for (int b = 0; b < B; ++b) s += blk[(size_t)b * N + c];
-  part[(size_t)blockIdx.y * N + c] = s;
-}
-__global__ void add_steps_descending(const float* part, int n, int N, float* out) {
-  sm100::grid_dep_wait();
-  sm100::grid_dep_launch();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= N) return;
-  float acc = out[c];
-  for (int a = n - 1; a >= 0; --a) acc += part[(size_t)a * N + c];
-  out[c] = acc;
-}
-
 __global__ void sum_parts(const float* part, int n, float* out) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
@@ -332,7 +331,6 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
   if (rc != MEBPTT_OK) return rc;
   launch_pdl(sum_parts, dim3(1), dim3(32), 0, s, a.loss_part, (a.B / 32) * o.parts, a.loss_k);
   launch_pdl(split_a3, dim3(ew_blocks(no)), dim3(256), 0, s, a.dy, a.O, nullptr, 0, a.B, dy3);
-  launch_pdl(colsum_accum<float>, dim3((a.O + 127) / 128), dim3(128), 0, s, a.dy, a.B, a.O, a.db_out);
   // dha[b][j] = sum_o dy[b][o] W_out[o][j]
   return gemm_bf16(dy3, 3 * a.O, false, w.woutmn3, a.H, true, GemmOut{GemmOut::STORE_F32, a.dha, a.H, nullptr, 0}, a.B,
                    a.H, 3 * a.O, w.status, s, true, &w.split);
@@ -342,7 +340,7 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
 // by the sums of the single-step function, the contraction for dha split along K into the parts a
 // single step would take.
 int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, const float* target, float* loss_t,
-                float* db_out, int B, int H, int O, const Scratch& w, cudaStream_t s) {
+                int B, int H, int O, const Scratch& w, cudaStream_t s) {
   bf16* h3 = w.st_h3 + (size_t)s_lo * B * 3 * H;
   bf16* dy3 = w.st_dy3 + (size_t)s_lo * B * 3 * O;
   const size_t nh = (size_t)B * H, no = (size_t)n * B * O;
@@ -360,8 +358,6 @@ int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, 
   if (rc != MEBPTT_OK) return rc;
   launch_pdl(sum_parts_steps, dim3(1), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
   launch_pdl(split_a3, dim3(ew_blocks(no)), dim3(256), 0, s, (const float*)w.dy_run, O, (const float*)nullptr, 0, n * B, dy3);
-  launch_pdl(colsum_steps, dim3((O + 127) / 128, n), dim3(128), 0, s, (const float*)w.dy_run, B, O, w.colsum_part);
-  launch_pdl(add_steps_descending, dim3((O + 127) / 128), dim3(128), 0, s, (const float*)w.colsum_part, n, O, db_out);
   const int splits = tc::gemm_split_count(false, true, B, H, 3 * O, w.split.partial_floats);
   return gemm_bf16(dy3, 3 * O, false, w.woutmn3, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H,
                    3 * O, w.status, s, true, &w.split_run, splits);
@@ -375,9 +371,8 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_
   bf16* in2 = w.st_in2 + (l == 0 ? 0 : rows * 2 * w.I0 + (size_t)(l - 1) * rows * 2 * a.H) + (size_t)sidx * a.B * 2 * a.I;
   bf16* hp2 = w.st_hp2 + ((size_t)l * rows + (size_t)sidx * a.B) * 2 * a.H;
   launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const float*)a.gates, a.plane_elems, a.c_t, a.c_prev,
-                                        a.dz, dz3, a.B, a.H, a.counters, (const float*)a.in, a.I, in2,
+                                        (float*)nullptr, dz3, a.B, a.H, a.counters, (const float*)a.in, a.I, in2,
                                         (const float*)a.h_prev, hp2);
-  launch_pdl(colsum_accum<float>, dim3((G + 127) / 128), dim3(128), 0, s, a.dz, a.B, G, a.db);
   const bf16* WMN = w.wmn3 + 3 * w_off;   // [3G][K]
   if (a.d_lo) {
     int rc = gemm_bf16(dz3, 3 * G, false, WMN, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I,
@@ -408,12 +403,13 @@ int accum3(const bf16* a3, int Ma, const bf16* b2, int Nb, bool b_is_a3, float* 
 }  // namespace
 
 int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O, const size_t* w_off, float* dW,
-                float* dW_out, cudaStream_t s) {
+                float* dW_out, float* db, float* db_out, cudaStream_t s) {
   const int G = 4 * H, R = steps * B;
   const size_t rows = (size_t)w.S * B;
   for (int l = 0; l < L; ++l) {
     const int I = l == 0 ? I0 : H, K = I + H;
     const bf16* dz3 = w.st_dz3 + (size_t)l * rows * 3 * G;
+    launch_pdl(colsum_rows3, dim3((G + 63) / 64), dim3(32, 16), 0, s, dz3, R, G, db + (size_t)l * G);
     const bf16* in2 = w.st_in2 + (l == 0 ? 0 : rows * 2 * I0 + (size_t)(l - 1) * rows * 2 * H);
     const bf16* hp2 = w.st_hp2 + (size_t)l * rows * 2 * H;
     float* dWl = dW + w_off[l];
@@ -422,6 +418,7 @@ int flush_chunk(const Scratch& w, int steps, int L, int B, int I0, int H, int O,
     rc = accum3(dz3, G, hp2, H, false, dWl + I, K, R, w.status, s);
     if (rc != MEBPTT_OK) return rc;
   }
+  launch_pdl(colsum_rows3, dim3((O + 63) / 64), dim3(32, 16), 0, s, (const bf16*)w.st_dy3, R, O, db_out);
   return accum3(w.st_dy3, O, w.st_h3, H, true, dW_out, H, R, w.status, s);
 }
 
