@@ -68,6 +68,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   float* loss_part = reinterpret_cast<float*>(ws + y.off_loss_part);
   float* loss_t = reinterpret_cast<float*>(ws + y.off_loss_t);
   int* status = reinterpret_cast<int*>(ws + y.off_status);
+  // where each layer's dh of the latest backward operation lies: in its buffer (zero at first), or
+  // in the parts of a contraction split along K
+  std::vector<tc::SplitParts> dh_parts((size_t)y.L);
   stepwise::Scratch tcw{};
   if (y.stepwise_tc) {
     tcw.z = reinterpret_cast<float*>(ws + y.off_z);
@@ -84,6 +87,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     tcw.hrun = reinterpret_cast<__nv_bfloat16*>(ws + y.off_hrun);
     tcw.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
     tcw.loss_part = loss_part;
+    tcw.split_dh = reinterpret_cast<float*>(ws + y.off_split_dh);
+    tcw.dh_parts = dh_parts.data();
   }
   stepwise3::Scratch x3{};
   size_t w_off[16];
@@ -102,6 +107,8 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
     x3.dy_run = reinterpret_cast<float*>(ws + y.off_dy_run);
     x3.dha_run = reinterpret_cast<float*>(ws + y.off_dha_run);
     x3.loss_part = loss_part;
+    x3.split_dh = reinterpret_cast<float*>(ws + y.off_split_dh);
+    x3.dh_parts = dh_parts.data();
     x3.a3_run = bf(y.off_a3_run);
     x3.h_run = reinterpret_cast<float*>(ws + y.off_hrun);
   }
@@ -455,7 +462,8 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, G, pf) > 1 ? 2 : 1;   // dz W -> [B][H]
     const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, G, pf) > 1 ? 2 : 1;   // dz W -> [B][I]
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, y.O, pf) > 1 ? 2 : 1;
-    const int64_t bwd = L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    // (the recurrent dh = dz W_hh is one launch in any case: its parts are added by the next gate kernel)
+    const int64_t bwd = L + L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
     const int64_t chunks = (p->t + y.S - 1) / y.S;   // each flushed by 2 L + 1 GEMMs and L + 1 bias sums
     // runs of n >= 2 operations go layer by layer: one input product per layer and run, the
     // readout once per run (stage, GEMM with loss, loss terms, dha), the gradient handed down
@@ -465,7 +473,7 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
       if (wi.kind == WorkItem::LEAF) n_launch += wi.n * (3 * L + 2 + dha + bwd);
       else if (wi.kind == WorkItem::FWD) n_launch += wi.n == 1 ? 3 * L : L * (1 + 2 * (int64_t)wi.n);
       else if (wi.n == 1) n_launch += 2 + dha + bwd;
-      else n_launch += 3 + dha + L * wi.n * (1 + to_h) + (L - 1) * to_h + (desc->want_dx ? to_x : 0);
+      else n_launch += 3 + dha + L * wi.n * 2 + (L - 1) * to_h + (desc->want_dx ? to_x : 0);
     }
     return n_launch;
   }
@@ -478,7 +486,7 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     const int64_t to_h = tc::gemm_split_count(false, true, y.B, y.H, 3 * G, pf) > 1 ? 2 : 1;
     const int64_t to_x = tc::gemm_split_count(false, true, y.B, y.I, 3 * G, pf) > 1 ? 2 : 1;
     const int64_t dha = tc::gemm_split_count(false, true, y.B, y.H, 3 * y.O, pf) > 1 ? 2 : 1;
-    const int64_t bwd = L + to_h * L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);
+    const int64_t bwd = L + L + to_h * (L - 1) + (desc->want_dx ? to_x : 0);   // dh = dz W_hh: one launch in any case
     const int64_t chunks = (p->t + y.S - 1) / y.S;
     // the readout of a run of n >= 2 backward operations is taken once for the run (the same
     // launches), and a run of n >= 2 forward operations splits its operands once per layer (then

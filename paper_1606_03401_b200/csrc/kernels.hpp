@@ -78,6 +78,9 @@ void copy_bytes(void* dst, const void* src, size_t bytes, cudaStream_t s);
 
 // The same three operations with their contractions on the tensor cores (bfloat16 storage,
 // dimensions that are multiples of 8, B a multiple of 32).  Each returns a status.
+// Floats of split-K scratch for one step's dh = dz W_hh of one layer: a wave of 128 x 128 tiles.
+constexpr size_t DH_PART_FLOATS = (size_t)148 * 128 * 128;
+
 namespace stepwise {
 struct Scratch {
   float* z;                 // [B][4H] pre-activations of the forward operation in flight
@@ -95,6 +98,10 @@ struct Scratch {
   __nv_bfloat16* hrun;      // [S B][H]  the layer's h_k, read by the layer above
   float* dha_run;           // [S B][H]  gradient entering the layer at each step (row block: step - first step)
   float* loss_part;         // partial sums of the loss terms, per step
+  // the recurrent gradient dh = dz W_hh of a layer is consumed only by the layer's next gate
+  // kernel: where that contraction is split along K, the gate kernel adds the parts itself
+  float* split_dh;          // [L][DH_PART_FLOATS] split-K scratch of that product, one per layer
+  tc::SplitParts* dh_parts; // host, [L]: where each layer's latest dh lies (updated by every backward operation)
   tc::SplitWs split_run;    // split-K scratch for a product over all rows of a run
 };
 int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s);
@@ -153,6 +160,8 @@ struct Scratch {
   float* dy_run;             // [S B][O]
   float* dha_run;            // [S B][H]  gradient entering the top layer at each step of the run
   float* loss_part;          // partial sums of the loss terms, per step
+  float* split_dh;           // as on the bfloat16 path: per-layer split-K scratch of dh = dz W_hh,
+  tc::SplitParts* dh_parts;  // and where each layer's latest dh lies (host, [L])
   tc::SplitWs split_run;     // split-K scratch for a product over all rows of a run
   __nv_bfloat16* a3_run;     // [S][B][3 (I + H)]: left operands of a run of forward operations
   float* h_run;              // [S][B][H]: a layer's h_k of a run, the inputs of the layer above

@@ -52,7 +52,7 @@ struct Layout {
   size_t off_a3 = 0, off_w3 = 0, off_wmn3 = 0, off_wout3 = 0, off_woutmn3 = 0;
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
-  size_t off_sync = 0, off_tape = 0, off_status = 0;
+  size_t off_sync = 0, off_tape = 0, off_status = 0, off_split_dh = 0;
   size_t off_a3_run = 0, off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
@@ -231,6 +231,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       // a whole run (its products are split like a single step's, to sum in the same order)
       y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
       y.off_split = take(y.split_floats * 4);
+      y.off_split_dh = take((size_t)y.L * 148 * 128 * 128 * 4);   // per layer: the parts of dh = dz W_hh
     }
     if (y.stepwise_x3) {
       const size_t G = 4 * (size_t)y.H, Kmax = (size_t)(y.I > y.H ? y.I : y.H) + y.H;
@@ -245,6 +246,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.off_dha_run = take(rows * y.H * 4);
       y.split_floats = (size_t)148 * 128 * 128 * ((rows + 127) / 128);
       y.off_split = take(y.split_floats * 4);
+      y.off_split_dh = take((size_t)y.L * 148 * 128 * 128 * 4);
       y.off_a3 = take((size_t)y.B * 3 * Kmax * 2);
       y.off_w3 = take(3 * y.w_total_elems() * 2);
       y.off_wmn3 = take(3 * y.w_total_elems() * 2);

@@ -71,7 +71,7 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev
 __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const bf16* gates, size_t plane,
                          const float* c_t, const float* c_prev, float* dz, bf16* dz16, int B, int H,
                          int64_t* counters, const uint4* in, uint4* st_in, size_t n_in16, const uint4* hp,
-                         uint4* st_hp, size_t n_hp16) {
+                         uint4* st_hp, size_t n_hp16, const tc::SplitParts dh_parts) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
@@ -83,7 +83,8 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
     const int b = (int)(e / H), j = (int)(e % H);
     const float gi = __bfloat162float(gates[e]), gf = __bfloat162float(gates[plane + e]);
     const float gg = __bfloat162float(gates[2 * plane + e]), go = __bfloat162float(gates[3 * plane + e]);
-    const float dh = dha[e] + dh_rec[e];
+    // the gradient from step k + 1: stored, or still in the parts of the contraction that made it
+    const float dh = dha[e] + (dh_parts.splits ? tc::split_parts_sum(dh_parts, b, j) : dh_rec[e]);
     const float th = tanhf(c_t[e]);
     const float d_o = dh * th;
     const float dc = fmaf(dh * go, 1.f - th * th, dc_rec[e]);
@@ -222,15 +223,16 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
   launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
                                         (float*)nullptr, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
                                         (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
-                                        (size_t)a.B * a.H * 2 / 16);
+                                        (size_t)a.B * a.H * 2 / 16, w.dh_parts[l]);
   // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
   if (a.d_lo) {
     int rc = gemm_bf16(dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
                        w.status, s, true, &w.split);
     if (rc != MEBPTT_OK) return rc;
   }
+  const tc::SplitWs own{w.split_dh + (size_t)l * DH_PART_FLOATS, DH_PART_FLOATS};
   return gemm_bf16(dz16, G, false, W + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B, a.H,
-                   G, w.status, s, true, &w.split);
+                   G, w.status, s, true, &own, 0, &w.dh_parts[l]);
 }
 
 // Weight gradients of a finished chunk: `steps` row blocks of B rows, from block 0 on.
@@ -326,9 +328,10 @@ int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, cons
     launch_pdl(gate_bwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)(w.dha_run + (size_t)a * bh), (const float*)dh_rec,
                dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t, st[a].c_prev, (float*)nullptr, dz16, B, H, counters,
                (const uint4*)st[a].in, (uint4*)(in_l + row0 * I), (size_t)B * I * 2 / 16, (const uint4*)st[a].h_prev,
-               (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16);
+               (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16, w.dh_parts[l]);
+    const tc::SplitWs own{w.split_dh + (size_t)l * DH_PART_FLOATS, DH_PART_FLOATS};
     const int rc = gemm_bf16(dz16, G, false, W + I, K, true, GemmOut{GemmOut::STORE_F32, dh_rec, H, nullptr, 0}, B, H, G,
-                             w.status, s, true, &w.split);
+                             w.status, s, true, &own, 0, &w.dh_parts[l]);
     if (rc != MEBPTT_OK) return rc;
   }
   if (!d_lo) return MEBPTT_OK;

@@ -164,7 +164,8 @@ __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_pre
 // of dz W and of the chunk's dW), and the halves [hi | mid] of this step's layer input and h_{k-1}.
 __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const float* gates, size_t plane,
                          const float* c_t, const float* c_prev, float* dz, bf16* dz3, int B, int H, int64_t* counters,
-                         const float* in, int I, bf16* st_in2, const float* hp, bf16* st_hp2) {
+                         const float* in, int I, bf16* st_in2, const float* hp, bf16* st_hp2,
+                         const tc::SplitParts dh_parts) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
@@ -172,7 +173,8 @@ __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, c
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
     const float gi = gates[e], gf = gates[plane + e], gg = gates[2 * plane + e], go = gates[3 * plane + e];
-    const float dh = dha[e] + dh_rec[e];
+    // the gradient from step k + 1: stored, or still in the parts of the contraction that made it
+    const float dh = dha[e] + (dh_parts.splits ? tc::split_parts_sum(dh_parts, b, j) : dh_rec[e]);
     const float th = tanhf(c_t[e]);
     const float d_o = dh * th;
     const float dc = fmaf(dh * go, 1.f - th * th, dc_rec[e]);
@@ -372,15 +374,16 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, size_t w_
   bf16* hp2 = w.st_hp2 + ((size_t)l * rows + (size_t)sidx * a.B) * 2 * a.H;
   launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const float*)a.gates, a.plane_elems, a.c_t, a.c_prev,
                                         (float*)nullptr, dz3, a.B, a.H, a.counters, (const float*)a.in, a.I, in2,
-                                        (const float*)a.h_prev, hp2);
+                                        (const float*)a.h_prev, hp2, w.dh_parts[l]);
   const bf16* WMN = w.wmn3 + 3 * w_off;   // [3G][K]
   if (a.d_lo) {
     int rc = gemm_bf16(dz3, 3 * G, false, WMN, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I,
                        3 * G, w.status, s, true, &w.split);
     if (rc != MEBPTT_OK) return rc;
   }
+  const tc::SplitWs own{w.split_dh + (size_t)l * DH_PART_FLOATS, DH_PART_FLOATS};
   return gemm_bf16(dz3, 3 * G, false, WMN + a.I, K, true, GemmOut{GemmOut::STORE_F32, a.dh_rec, a.H, nullptr, 0}, a.B,
-                   a.H, 3 * G, w.status, s, true, &w.split);
+                   a.H, 3 * G, w.status, s, true, &own, 0, &w.dh_parts[l]);
 }
 
 namespace {

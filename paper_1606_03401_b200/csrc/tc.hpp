@@ -57,6 +57,23 @@ struct SplitWs {
   size_t partial_floats;
 };
 
+// Where a contraction that was split along K left its parts, for a consumer that adds them itself
+// (in index order, starting from zero: the sum the library's own second pass would have stored).
+// splits == 0: the product was not split and lies where GemmOut says.
+struct SplitParts {
+  const float* partial = nullptr;   // [tile][part][128][bn], tile = (m / 128) * tiles_x + n / bn
+  int splits = 0, tiles_x = 0, bn = 0;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ float split_parts_sum(const SplitParts& sp, int m, int n) {
+  const int tile = (m >> 7) * sp.tiles_x + n / sp.bn;
+  const float* p = sp.partial + (((size_t)tile * sp.splits) * 128 + (size_t)(m & 127)) * sp.bn + (n % sp.bn);
+  float acc = 0.f;
+  for (int z = 0; z < sp.splits; ++z) acc += p[(size_t)z * 128 * sp.bn];
+  return acc;
+}
+#endif
+
 // Parts gemm_bf16 splits the contraction index into, given scratch for partial_floats floats and
 // an output it can split for (a plain float32 store, no bias, rows that take float4); 1 = no
 // split, otherwise a second launch adds the parts.
@@ -69,9 +86,11 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 // memory).
 // force_splits > 0: split the contraction index into exactly that many parts (the caller took the
 // count from gemm_split_count for a product of another height, so that both sum in the same order).
+// defer (optional): if the product is split, the pass that adds the parts is left to the caller's
+// next kernel and *defer says where they are; if it is not, *defer says so (splits = 0).
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
               int M, int N, int K, int* status, cudaStream_t s, bool early = true, const SplitWs* split = nullptr,
-              int force_splits = 0);
+              int force_splits = 0, SplitParts* defer = nullptr);
 
 }  // namespace tc
 

@@ -375,7 +375,8 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 }
 
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
-              int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split, int force_splits) {
+              int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split, int force_splits,
+              SplitParts* defer) {
   if (M <= 0 || N <= 0 || K <= 0) return MEBPTT_ERR_ARG;
   // A short-and-wide product over K-major operands (a few steps' worth of rows against a whole
   // weight matrix) gives few 128-wide tiles, each streaming all of K through one SM: 32-wide tiles
@@ -423,7 +424,8 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
     cudaGetLastError();
     return MEBPTT_ERR_CUDA;
   }
-  if (splits > 1) {
+  if (defer) *defer = splits > 1 ? SplitParts{split->partial, splits, (int)grid.x, BN} : SplitParts{};
+  if (splits > 1 && !defer) {
     const size_t quads = (size_t)M * ((N + 3) / 4);
     const int blocks = (int)((quads + 255) / 256 > 1184 ? 1184 : (quads + 255) / 256);
     const cudaError_t e2 = launch_on(early, splitk_reduce, dim3(blocks), dim3(256), 0, s, (const float*)split->partial,
