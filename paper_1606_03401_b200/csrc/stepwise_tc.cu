@@ -37,17 +37,23 @@ __device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf
 
 // z [B][4H] (column q H + j: gate q of unit j, bias included) -> gates, c_k, h_k and, for an
 // internal state, the copies of h_{k-1}, c_{k-1}.
+// zp: where the recurrent product lies if it was split along K (its parts are then added to z here).
 __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
                          bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H,
-                         int64_t* counters, bf16* h_stage) {
+                         int64_t* counters, bf16* h_stage, const tc::SplitParts zp) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
     const float* row = z + (size_t)b * 4 * H;
-    const float gi = sigmoidf_(row[j]), gf = sigmoidf_(row[H + j]);
-    const float gg = tanhf(row[2 * H + j]), go = sigmoidf_(row[3 * H + j]);
+    float zi = row[j], zf = row[H + j], zg = row[2 * H + j], zo = row[3 * H + j];
+    if (zp.splits) {
+      zi += tc::split_parts_sum(zp, b, j);         zf += tc::split_parts_sum(zp, b, H + j);
+      zg += tc::split_parts_sum(zp, b, 2 * H + j); zo += tc::split_parts_sum(zp, b, 3 * H + j);
+    }
+    const float gi = sigmoidf_(zi), gf = sigmoidf_(zf);
+    const float gg = tanhf(zg), go = sigmoidf_(zo);
     const float cp = c_prev[e];
     const float c = fmaf(gf, cp, gi * gg);
     c_out[e] = c;
@@ -184,12 +190,14 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
   int rc = gemm_bf16(a.in, a.I, false, W, K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0}, a.B, G, a.I,
                      w.status, s, true, &w.split);
   if (rc != MEBPTT_OK) return rc;
+  // the recurrent part: split along K where that puts more SMs to work, its parts added by the cell kernel
+  tc::SplitParts zp;
   rc = gemm_bf16(a.h_prev, a.H, false, W + a.I, K, false, GemmOut{GemmOut::ACCUM_F32, w.z, G, nullptr, 0}, a.B, G,
-                 a.H, w.status, s, true, &w.split);
+                 a.H, w.status, s, true, &w.split, tc::gemm_split_count_deferred(a.B, G, a.H), &zp);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
   launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
-                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr);
+                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, zp);
   return MEBPTT_OK;
 }
 
@@ -276,12 +284,13 @@ int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const 
   const size_t bh = (size_t)B * H;
   for (int j = 0; j < n; ++j) {
     float* z = w.zrun + (size_t)j * B * G;
+    tc::SplitParts zp;
     rc = gemm_bf16(st[j].h_prev, H, false, W + I, K, false, GemmOut{GemmOut::ACCUM_F32, z, G, nullptr, 0}, B, G, H,
-                   w.status, s);
+                   w.status, s, true, &w.split, tc::gemm_split_count_deferred(B, G, H), &zp);
     if (rc != MEBPTT_OK) return rc;
     launch_pdl(cell_fwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)z, st[j].c_prev, (const bf16*)st[j].h_prev,
                (bf16*)st[j].h_out, st[j].c_out, (bf16*)st[j].gates, plane_elems, (bf16*)st[j].h_in_copy, st[j].c_in_copy, B,
-               H, counters, stage_h ? w.hrun + (size_t)j * bh : (bf16*)nullptr);
+               H, counters, stage_h ? w.hrun + (size_t)j * bh : (bf16*)nullptr, zp);
   }
   return MEBPTT_OK;
 }

@@ -131,17 +131,26 @@ __global__ void split_run_inputs(const float* in, int64_t in_step_stride, int I,
   }
 }
 
+// z holds the contraction without the bias, or, if it was split along K, zp says where its parts
+// lie (they are added here); bias [4H] is added last.
 __global__ void cell_fwd(const float* z, const float* c_prev, const float* h_prev, float* h_out, float* c_out,
                          float* gates, size_t plane, float* h_in_copy, float* c_in_copy, int B, int H,
-                         int64_t* counters, bf16* a3_next, int I) {
+                         int64_t* counters, bf16* a3_next, int I, const float* bias, const tc::SplitParts zp) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
   const size_t n = (size_t)B * H;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
     const int b = (int)(e / H), j = (int)(e % H);
-    const float* row = z + (size_t)b * 4 * H;
-    const float gi = sigmoidf_(row[j]), gf = sigmoidf_(row[H + j]);
-    const float gg = tanhf(row[2 * H + j]), go = sigmoidf_(row[3 * H + j]);
+    float zi, zf, zg, zo;
+    if (zp.splits) {
+      zi = tc::split_parts_sum(zp, b, j);         zf = tc::split_parts_sum(zp, b, H + j);
+      zg = tc::split_parts_sum(zp, b, 2 * H + j); zo = tc::split_parts_sum(zp, b, 3 * H + j);
+    } else {
+      const float* row = z + (size_t)b * 4 * H;
+      zi = row[j]; zf = row[H + j]; zg = row[2 * H + j]; zo = row[3 * H + j];
+    }
+    const float gi = sigmoidf_(zi + bias[j]), gf = sigmoidf_(zf + bias[H + j]);
+    const float gg = tanhf(zg + bias[2 * H + j]), go = sigmoidf_(zo + bias[3 * H + j]);
     const float cp = c_prev[e];
     const float c = fmaf(gf, cp, gi * gg);
     c_out[e] = c;
@@ -279,12 +288,14 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, int l, size_t w_of
   const int K = a.I + a.H, G = 4 * a.H;
   const size_t nk = (size_t)a.B * K;
   launch_pdl(split_a3, dim3(ew_blocks(nk)), dim3(256), 0, s, (const float*)a.in, a.I, (const float*)a.h_prev, a.H, a.B, w.a3);
-  int rc = gemm_bf16(w.a3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false, GemmOut{GemmOut::STORE_F32, w.z, G, a.bias, 0},
-                     a.B, G, 3 * K, w.status, s);
+  // split along K where that puts more SMs to work; the cell kernel adds the parts, and the bias
+  tc::SplitParts zp;
+  int rc = gemm_bf16(w.a3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false, GemmOut{GemmOut::STORE_F32, w.z, G, nullptr, 0},
+                     a.B, G, 3 * K, w.status, s, true, &w.split, tc::gemm_split_count_deferred(a.B, G, 3 * K), &zp);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
   launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const float*)a.h_prev, (float*)a.h_out, a.c_out, (float*)a.gates,
-                                        a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, 0);
+                                        a.plane_elems, (float*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, 0, a.bias, zp);
   (void)l;
   return MEBPTT_OK;
 }
@@ -303,13 +314,15 @@ int forward_run_layer(const stepwise::FwdRunStep* st, int n, const float* in, in
              in_step_stride, I, (const float*)st[0].h_prev, H, B, w.a3_run);
   const size_t nbh = (size_t)B * H;
   for (int j = 0; j < n; ++j) {
+    tc::SplitParts zp;
     const int rc = gemm_bf16(w.a3_run + (size_t)j * row3, 3 * K, false, w.w3 + 3 * w_off, 3 * K, false,
-                             GemmOut{GemmOut::STORE_F32, w.z, G, bias, 0}, B, G, 3 * K, w.status, s);
+                             GemmOut{GemmOut::STORE_F32, w.z, G, nullptr, 0}, B, G, 3 * K, w.status, s, true, &w.split,
+                             tc::gemm_split_count_deferred(B, G, 3 * K), &zp);
     if (rc != MEBPTT_OK) return rc;
     float* h_out = (float*)st[j].h_out;
     launch_pdl(cell_fwd, dim3(ew_blocks(nbh)), dim3(256), 0, s, (const float*)w.z, st[j].c_prev, (const float*)st[j].h_prev, h_out,
                st[j].c_out, (float*)st[j].gates, plane_elems, (float*)st[j].h_in_copy, st[j].c_in_copy, B, H, counters,
-               j + 1 < n ? w.a3_run + (size_t)(j + 1) * row3 : (bf16*)nullptr, I);
+               j + 1 < n ? w.a3_run + (size_t)(j + 1) * row3 : (bf16*)nullptr, I, bias, zp);
     if (h_stage) {
       // the layer above reads the h_k of the run from one block: a copy beside the tape's place
       cudaMemcpyAsync(h_stage + (size_t)j * nbh, h_out, nbh * 4, cudaMemcpyDeviceToDevice, s);

@@ -79,6 +79,11 @@ __device__ __forceinline__ float split_parts_sum(const SplitParts& sp, int m, in
 // split, otherwise a second launch adds the parts.
 int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_floats);
 
+// Parts for a contraction whose adding-up is left to its consumer (gemm_bf16's `defer`): no pass
+// of its own has to pay off, so two parts are worth having; always over 128-wide tiles, about a
+// wave of CTAs, each part at least 8 blocks of 64 long.
+int gemm_split_count_deferred(int M, int N, int K);
+
 // C (+)= A B^T over bfloat16 operands.  a_mn / b_mn: the operand is stored [k][m] instead of
 // [m][k]; lda / ldb are row strides in elements (multiples of 8).  `status` (device, nullable)
 // receives MEBPTT_ERR_TIMEOUT if a bounded wait expires.  early: the kernel may become resident
@@ -87,7 +92,9 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 // force_splits > 0: split the contraction index into exactly that many parts (the caller took the
 // count from gemm_split_count for a product of another height, so that both sum in the same order).
 // defer (optional): if the product is split, the pass that adds the parts is left to the caller's
-// next kernel and *defer says where they are; if it is not, *defer says so (splits = 0).
+// next kernel and *defer says where they are (C is then not touched, not even when accumulating:
+// the consumer adds the parts to it); if it is not, *defer says so (splits = 0).  With defer and
+// force_splits > 1 the tiles are 128 wide whatever the shape.
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
               int M, int N, int K, int* status, cudaStream_t s, bool early = true, const SplitWs* split = nullptr,
               int force_splits = 0, SplitParts* defer = nullptr);

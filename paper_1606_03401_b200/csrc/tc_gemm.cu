@@ -374,6 +374,17 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
   return want >= 4 ? want : 1;
 }
 
+int gemm_split_count_deferred(int M, int N, int K) {
+  static const bool no_split = getenv("MEBPTT_NO_SPLITK") != nullptr;
+  if (no_split) return 1;
+  const int tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
+  const int nk = (K + BK - 1) / BK;
+  int want = 148 / tiles;
+  if (want > nk / 8) want = nk / 8;
+  if (want > 16) want = 16;
+  return want >= 2 ? want : 1;
+}
+
 int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, const GemmOut& out,
               int M, int N, int K, int* status, cudaStream_t s, bool early, const SplitWs* split, int force_splits,
               SplitParts* defer) {
@@ -382,7 +393,7 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   // weight matrix) gives few 128-wide tiles, each streaming all of K through one SM: 32-wide tiles
   // put four times as many SMs to work on the same bytes.
   const int wide_tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
-  const bool narrow = !a_mn && !b_mn && wide_tiles <= 37 && N >= 2 * BN_NARROW;
+  const bool narrow = !a_mn && !b_mn && wide_tiles <= 37 && N >= 2 * BN_NARROW && !(defer && force_splits > 1);
   const int BN = narrow ? BN_NARROW : BN_WIDE;
   CUtensorMap ta, tb;
   // K-major: tensor is [M][K], box 64 (k) x tile rows.  MN-major: tensor is [K][M], box 64 (m) x 64 rows.
@@ -393,8 +404,8 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
   if (!ok) return MEBPTT_ERR_UNSUPPORTED;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
   int splits = 1;
-  if (split && split->partial && out.kind == GemmOut::STORE_F32 && !out.bias && !out.perm_h && out.ld % 4 == 0 &&
-      (reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0)
+  if (split && split->partial && (out.kind == GemmOut::STORE_F32 || (defer && out.kind == GemmOut::ACCUM_F32)) &&
+      !out.bias && !out.perm_h && out.ld % 4 == 0 && (reinterpret_cast<uintptr_t>(out.ptr) & 15) == 0)
     splits = force_splits > 0 ? force_splits : gemm_split_count(a_mn, b_mn, M, N, K, split->partial_floats);
   else if (force_splits > 1)
     return MEBPTT_ERR_ARG;
