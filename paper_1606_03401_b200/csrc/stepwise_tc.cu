@@ -35,76 +35,173 @@ typedef __nv_bfloat16 bf16;
 
 __device__ __forceinline__ float sigmoidf_(float a) { return 1.0f / (1.0f + expf(-a)); }
 
+// V consecutive elements at once (V = 4 where every array involved is 16-byte aligned, else 1).
+template <int V> __device__ __forceinline__ void ld(const float* p, float (&v)[V]) {
+  if constexpr (V == 4) { const float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+  else v[0] = *p;
+}
+template <int V> __device__ __forceinline__ void st(float* p, const float (&v)[V]) {
+  if constexpr (V == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  else *p = v[0];
+}
+template <int V> __device__ __forceinline__ void ld(const bf16* p, float (&v)[V]) {
+  if constexpr (V == 4) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xFFFF0000u);
+  } else v[0] = __bfloat162float(*p);
+}
+template <int V> __device__ __forceinline__ void st(bf16* p, const float (&v)[V]) {   // rounds to nearest even
+  if constexpr (V == 4) *reinterpret_cast<uint2*>(p) = make_uint2(sm100::pack_bf16x2(v[0], v[1]), sm100::pack_bf16x2(v[2], v[3]));
+  else *p = __float2bfloat16_rn(v[0]);
+}
+template <int V> __device__ __forceinline__ void cp(bf16* dst, const bf16* src) {
+  if constexpr (V == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(src);
+  else *dst = *src;
+}
+// v[i] += the sum of the parts at (m, n + i); the V columns lie in one tile (n is a multiple of V)
+template <int V> __device__ __forceinline__ void add_parts(const tc::SplitParts& sp, int m, int n, float (&v)[V]) {
+  const int tile = (m >> 7) * sp.tiles_x + n / sp.bn;
+  const float* p = sp.partial + (((size_t)tile * sp.splits) * 128 + (size_t)(m & 127)) * sp.bn + (n % sp.bn);
+  float acc[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] = 0.f;
+  for (int z = 0; z < sp.splits; ++z) {
+    float t[V];
+    ld<V>(p + (size_t)z * 128 * sp.bn, t);
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] += t[i];
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) v[i] += acc[i];
+}
+
 // z [B][4H] (column q H + j: gate q of unit j, bias included) -> gates, c_k, h_k and, for an
 // internal state, the copies of h_{k-1}, c_{k-1}.
 // zp: where the recurrent product lies if it was split along K (its parts are then added to z here).
+template <int V>
 __global__ void cell_fwd(const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
                          bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H,
                          int64_t* counters, bf16* h_stage, const tc::SplitParts zp) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
-  const size_t n = (size_t)B * H;
-  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+  const size_t n = (size_t)B * H / V;
+  for (size_t g = blockIdx.x * (size_t)blockDim.x + threadIdx.x; g < n; g += (size_t)gridDim.x * blockDim.x) {
+    const size_t e = g * V;
     const int b = (int)(e / H), j = (int)(e % H);
     const float* row = z + (size_t)b * 4 * H;
-    float zi = row[j], zf = row[H + j], zg = row[2 * H + j], zo = row[3 * H + j];
-    if (zp.splits) {
-      zi += tc::split_parts_sum(zp, b, j);         zf += tc::split_parts_sum(zp, b, H + j);
-      zg += tc::split_parts_sum(zp, b, 2 * H + j); zo += tc::split_parts_sum(zp, b, 3 * H + j);
+    float zq[4][V];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      ld<V>(row + (size_t)q * H + j, zq[q]);
+      if (zp.splits) add_parts<V>(zp, b, q * H + j, zq[q]);
     }
-    const float gi = sigmoidf_(zi), gf = sigmoidf_(zf);
-    const float gg = tanhf(zg), go = sigmoidf_(zo);
-    const float cp = c_prev[e];
-    const float c = fmaf(gf, cp, gi * gg);
-    c_out[e] = c;
-    const bf16 hv = __float2bfloat16_rn(go * tanhf(c));
-    h_out[e] = hv;
-    if (h_stage) h_stage[e] = hv;   // a second copy, where the layer above reads its inputs of a whole run
+    float cp_[V], c[V], hv[V], gi[V], gf[V], gg[V], go[V];
+    ld<V>(c_prev + e, cp_);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      gi[i] = sigmoidf_(zq[0][i]); gf[i] = sigmoidf_(zq[1][i]);
+      gg[i] = tanhf(zq[2][i]);     go[i] = sigmoidf_(zq[3][i]);
+      c[i] = fmaf(gf[i], cp_[i], gi[i] * gg[i]);
+      hv[i] = go[i] * tanhf(c[i]);
+    }
+    st<V>(c_out + e, c);
+    st<V>(h_out + e, hv);
+    if (h_stage) st<V>(h_stage + e, hv);   // a second copy, where the layer above reads its inputs of a whole run
     if (gates) {
-      gates[e] = __float2bfloat16_rn(gi);
-      gates[plane + e] = __float2bfloat16_rn(gf);
-      gates[2 * plane + e] = __float2bfloat16_rn(gg);
-      gates[3 * plane + e] = __float2bfloat16_rn(go);
+      st<V>(gates + e, gi); st<V>(gates + plane + e, gf);
+      st<V>(gates + 2 * plane + e, gg); st<V>(gates + 3 * plane + e, go);
     }
-    if (h_in_copy) { h_in_copy[e] = h_prev[e]; c_in_copy[e] = cp; }
+    if (h_in_copy) { cp<V>(h_in_copy + e, h_prev + e); st<V>(c_in_copy + e, cp_); }
   }
   if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[0] += 1;
 }
 
-// Gate derivatives: dh = dha + dh_rec; dz [B][4H] in float32 (for db) and bfloat16 (for the
-// contractions); dc_rec = dc * f.
+// Gate derivatives: dh = dha + dh_rec; dz [B][4H] rounded to bfloat16 (for the contractions and the
+// bias gradient), and in float32 as well if dz is given; dc_rec = dc * f.
 // Also copies this step's layer input and h_{k-1} to their stages (n_in16, n_hp16: 16-byte words).
+template <int V>
 __global__ void gate_bwd(const float* dha, const float* dh_rec, float* dc_rec, const bf16* gates, size_t plane,
                          const float* c_t, const float* c_prev, float* dz, bf16* dz16, int B, int H,
                          int64_t* counters, const uint4* in, uint4* st_in, size_t n_in16, const uint4* hp,
                          uint4* st_hp, size_t n_hp16, const tc::SplitParts dh_parts) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
-  const size_t n = (size_t)B * H;
+  const size_t n = (size_t)B * H / V;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_in16; e += (size_t)gridDim.x * blockDim.x)
     st_in[e] = in[e];
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n_hp16; e += (size_t)gridDim.x * blockDim.x)
     st_hp[e] = hp[e];
-  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+  for (size_t g = blockIdx.x * (size_t)blockDim.x + threadIdx.x; g < n; g += (size_t)gridDim.x * blockDim.x) {
+    const size_t e = g * V;
     const int b = (int)(e / H), j = (int)(e % H);
-    const float gi = __bfloat162float(gates[e]), gf = __bfloat162float(gates[plane + e]);
-    const float gg = __bfloat162float(gates[2 * plane + e]), go = __bfloat162float(gates[3 * plane + e]);
+    float gi[V], gf[V], gg[V], go[V], dh[V], rec[V], ct[V], cpv[V], dcr[V];
+    ld<V>(gates + e, gi); ld<V>(gates + plane + e, gf); ld<V>(gates + 2 * plane + e, gg); ld<V>(gates + 3 * plane + e, go);
+    ld<V>(dha + e, dh);
     // the gradient from step k + 1: stored, or still in the parts of the contraction that made it
-    const float dh = dha[e] + (dh_parts.splits ? tc::split_parts_sum(dh_parts, b, j) : dh_rec[e]);
-    const float th = tanhf(c_t[e]);
-    const float d_o = dh * th;
-    const float dc = fmaf(dh * go, 1.f - th * th, dc_rec[e]);
-    const float v0 = dc * gg * gi * (1.f - gi);
-    const float v1 = dc * c_prev[e] * gf * (1.f - gf);
-    const float v2 = dc * gi * (1.f - gg * gg);
-    const float v3 = d_o * go * (1.f - go);
+    if (dh_parts.splits) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) rec[i] = 0.f;
+      add_parts<V>(dh_parts, b, j, rec);
+    } else {
+      ld<V>(dh_rec + e, rec);
+    }
+    ld<V>(c_t + e, ct); ld<V>(c_prev + e, cpv); ld<V>(dc_rec + e, dcr);
+    float v[4][V], dcn[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const float d = dh[i] + rec[i];
+      const float th = tanhf(ct[i]);
+      const float d_o = d * th;
+      const float dc = fmaf(d * go[i], 1.f - th * th, dcr[i]);
+      v[0][i] = dc * gg[i] * gi[i] * (1.f - gi[i]);
+      v[1][i] = dc * cpv[i] * gf[i] * (1.f - gf[i]);
+      v[2][i] = dc * gi[i] * (1.f - gg[i] * gg[i]);
+      v[3][i] = d_o * go[i] * (1.f - go[i]);
+      dcn[i] = dc * gf[i];
+    }
     const size_t r = (size_t)b * 4 * H + j;
-    if (dz) { dz[r] = v0; dz[r + H] = v1; dz[r + 2 * (size_t)H] = v2; dz[r + 3 * (size_t)H] = v3; }
-    dz16[r] = __float2bfloat16_rn(v0); dz16[r + H] = __float2bfloat16_rn(v1);
-    dz16[r + 2 * (size_t)H] = __float2bfloat16_rn(v2); dz16[r + 3 * (size_t)H] = __float2bfloat16_rn(v3);
-    dc_rec[e] = dc * gf;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (dz) st<V>(dz + r + (size_t)q * H, v[q]);
+      st<V>(dz16 + r + (size_t)q * H, v[q]);
+    }
+    st<V>(dc_rec + e, dcn);
   }
   if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
+}
+
+// every pointer a multiple of 16 bytes?
+template <class... P>
+inline bool aligned16(P... p) { return ((... | reinterpret_cast<uintptr_t>(p)) & 15) == 0; }
+
+inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
+
+// The two element-wise kernels, four elements per thread where the addresses allow (same results).
+void run_cell_fwd(cudaStream_t s, const float* z, const float* c_prev, const bf16* h_prev, bf16* h_out, float* c_out,
+                  bf16* gates, size_t plane, bf16* h_in_copy, float* c_in_copy, int B, int H, int64_t* counters,
+                  bf16* h_stage, const tc::SplitParts& zp) {
+  const size_t n = (size_t)B * H;
+  const bool vec = H % 4 == 0 && plane % 8 == 0 &&
+                   aligned16(z, c_prev, h_prev, h_out, c_out, gates, h_in_copy, c_in_copy, h_stage, zp.partial);
+  if (vec)
+    launch_pdl(cell_fwd<4>, dim3(ew_blocks(n / 4)), dim3(256), 0, s, z, c_prev, h_prev, h_out, c_out, gates, plane, h_in_copy,
+               c_in_copy, B, H, counters, h_stage, zp);
+  else
+    launch_pdl(cell_fwd<1>, dim3(ew_blocks(n)), dim3(256), 0, s, z, c_prev, h_prev, h_out, c_out, gates, plane, h_in_copy,
+               c_in_copy, B, H, counters, h_stage, zp);
+}
+void run_gate_bwd(cudaStream_t s, const float* dha, const float* dh_rec, float* dc_rec, const bf16* gates, size_t plane,
+                  const float* c_t, const float* c_prev, bf16* dz16, int B, int H, int64_t* counters, const uint4* in,
+                  uint4* st_in, size_t n_in16, const uint4* hp, uint4* st_hp, size_t n_hp16, const tc::SplitParts& parts) {
+  const size_t n = (size_t)B * H;
+  const bool vec = H % 4 == 0 && plane % 8 == 0 && aligned16(dha, dh_rec, dc_rec, gates, c_t, c_prev, dz16, parts.partial);
+  if (vec)
+    launch_pdl(gate_bwd<4>, dim3(ew_blocks(n / 4)), dim3(256), 0, s, dha, dh_rec, dc_rec, gates, plane, c_t, c_prev,
+               (float*)nullptr, dz16, B, H, counters, in, st_in, n_in16, hp, st_hp, n_hp16, parts);
+  else
+    launch_pdl(gate_bwd<1>, dim3(ew_blocks(n)), dim3(256), 0, s, dha, dh_rec, dc_rec, gates, plane, c_t, c_prev,
+               (float*)nullptr, dz16, B, H, counters, in, st_in, n_in16, hp, st_hp, n_hp16, parts);
 }
 
 // out[c] += sum over the rows r = 0 .. R-1 of v[r][c]: the bias gradients of a chunk from its
@@ -180,7 +277,6 @@ __global__ void sum_parts_steps(const float* part, int per_step, int n, float* o
   out[a] = s;
 }
 
-inline int ew_blocks(size_t n) { return (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256); }
 
 }  // namespace
 
@@ -196,8 +292,8 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
                  a.H, w.status, s, true, &w.split, tc::gemm_split_count_deferred(a.B, G, a.H), &zp);
   if (rc != MEBPTT_OK) return rc;
   const size_t n = (size_t)a.B * a.H;
-  launch_pdl(cell_fwd, dim3(ew_blocks(n)), dim3(256), 0, s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates,
-                                        a.plane_elems, (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, zp);
+  run_cell_fwd(s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates, a.plane_elems,
+               (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, zp);
   return MEBPTT_OK;
 }
 
@@ -228,10 +324,9 @@ int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx,
   bf16* dz16 = w.st_dz + ((size_t)l * rows + (size_t)sidx * a.B) * G;
   bf16* st_in = w.st_in + (l == 0 ? 0 : rows * w.I0 + (size_t)(l - 1) * rows * a.H) + (size_t)sidx * a.B * a.I;
   bf16* st_hp = w.st_hp + ((size_t)l * rows + (size_t)sidx * a.B) * a.H;
-  launch_pdl(gate_bwd, dim3(ew_blocks(n)), dim3(256), 0, s, a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev,
-                                        (float*)nullptr, dz16, a.B, a.H, a.counters, (const uint4*)a.in, (uint4*)st_in,
-                                        (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
-                                        (size_t)a.B * a.H * 2 / 16, w.dh_parts[l]);
+  run_gate_bwd(s, a.dha, a.dh_rec, a.dc_rec, (const bf16*)a.gates, a.plane_elems, a.c_t, a.c_prev, dz16, a.B, a.H, a.counters,
+               (const uint4*)a.in, (uint4*)st_in, (size_t)a.B * a.I * 2 / 16, (const uint4*)a.h_prev, (uint4*)st_hp,
+               (size_t)a.B * a.H * 2 / 16, w.dh_parts[l]);
   // d_in = dz W: columns < I feed dx or the layer below, the rest is the new dh_rec
   if (a.d_lo) {
     int rc = gemm_bf16(dz16, G, false, W, K, true, GemmOut{GemmOut::STORE_F32, a.d_lo, a.I, nullptr, 0}, a.B, a.I, G,
@@ -288,9 +383,9 @@ int forward_run_layer(const FwdRunStep* st, int n, const void* in, int I, const 
     rc = gemm_bf16(st[j].h_prev, H, false, W + I, K, false, GemmOut{GemmOut::ACCUM_F32, z, G, nullptr, 0}, B, G, H,
                    w.status, s, true, &w.split, tc::gemm_split_count_deferred(B, G, H), &zp);
     if (rc != MEBPTT_OK) return rc;
-    launch_pdl(cell_fwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)z, st[j].c_prev, (const bf16*)st[j].h_prev,
-               (bf16*)st[j].h_out, st[j].c_out, (bf16*)st[j].gates, plane_elems, (bf16*)st[j].h_in_copy, st[j].c_in_copy, B,
-               H, counters, stage_h ? w.hrun + (size_t)j * bh : (bf16*)nullptr, zp);
+    run_cell_fwd(s, z, st[j].c_prev, (const bf16*)st[j].h_prev, (bf16*)st[j].h_out, st[j].c_out, (bf16*)st[j].gates,
+                 plane_elems, (bf16*)st[j].h_in_copy, st[j].c_in_copy, B, H, counters,
+                 stage_h ? w.hrun + (size_t)j * bh : (bf16*)nullptr, zp);
   }
   return MEBPTT_OK;
 }
@@ -334,10 +429,10 @@ int backward_run_layer(const BwdRunStep* st, int n, int s_lo, int l, int I, cons
   for (int a = n - 1; a >= 0; --a) {   // time descending
     const size_t row0 = (size_t)(s_lo + a) * B;
     bf16* dz16 = dz_l + row0 * G;
-    launch_pdl(gate_bwd, dim3(ew_blocks(bh)), dim3(256), 0, s, (const float*)(w.dha_run + (size_t)a * bh), (const float*)dh_rec,
-               dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t, st[a].c_prev, (float*)nullptr, dz16, B, H, counters,
-               (const uint4*)st[a].in, (uint4*)(in_l + row0 * I), (size_t)B * I * 2 / 16, (const uint4*)st[a].h_prev,
-               (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16, w.dh_parts[l]);
+    run_gate_bwd(s, w.dha_run + (size_t)a * bh, dh_rec, dc_rec, (const bf16*)st[a].gates, plane_elems, st[a].c_t,
+                 st[a].c_prev, dz16, B, H, counters, (const uint4*)st[a].in, (uint4*)(in_l + row0 * I),
+                 (size_t)B * I * 2 / 16, (const uint4*)st[a].h_prev, (uint4*)(hp_l + row0 * H), (size_t)B * H * 2 / 16,
+                 w.dh_parts[l]);
     const tc::SplitWs own{w.split_dh + (size_t)l * DH_PART_FLOATS, DH_PART_FLOATS};
     const int rc = gemm_bf16(dz16, G, false, W + I, K, true, GemmOut{GemmOut::STORE_F32, dh_rec, H, nullptr, 0}, B, H, G,
                              w.status, s, true, &own, 0, &w.dh_parts[l]);
