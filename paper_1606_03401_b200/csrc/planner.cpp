@@ -7,10 +7,13 @@
 #include "plan.hpp"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <limits>
 #include <new>
+#include <system_error>
+#include <thread>
 
 namespace mebptt {
 
@@ -204,12 +207,33 @@ void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Co
     std::fill(H.col(m), H.col(m) + t_max + 1, (uint8_t)0);
   }
   auto column = [&](int64_t m) -> const T* { return m <= 0 ? nonpos.data() : C.col(m); };
-  for (int64_t m = 1; m <= m_max; ++m) {
+  // The columns of this mode are not convex in t, so every cell is a scan; what is left to gain is
+  // that cell (t, m) needs the columns m - 1, m - alpha, m - beta only up to row t - 1.  Several
+  // threads therefore fill consecutive columns at once, each a few rows behind the columns it
+  // reads (rows[m]: how far column m has got).  The values are those of the plain loop.
+  std::vector<std::atomic<int64_t>> rows((size_t)m_max + 1);
+  for (auto& r : rows) r.store(0, std::memory_order_relaxed);
+  auto wait_for = [&](int64_t m, int64_t upto) -> int64_t {   // until column m is filled up to row `upto`; how far it is
+    if (m <= 0) return t_max;
+    int64_t got;
+    while ((got = rows[(size_t)m].load(std::memory_order_acquire)) < upto) std::this_thread::yield();
+    return got;
+  };
+  std::atomic<int64_t> next_column{1};
+  auto worker = [&]() {
+   for (;;) {
+    const int64_t m = next_column.fetch_add(1, std::memory_order_relaxed);
+    if (m > m_max) return;
     T* c = C.col(m);
     const T* cm1 = column(m - 1);
     const T* cma = column(m - alpha);
     const T* cmb = beta > 0 ? column(m - beta) : nullptr;
+    int64_t sure = 0;   // rows of the columns read that are known to be there
     for (int64_t t = 1; t <= t_max; ++t) {
+      if (sure < t - 1) {
+        sure = std::min(wait_for(m - 1, t - 1), wait_for(m - alpha, t - 1));
+        if (cmb) sure = std::min(sure, wait_for(m - beta, t - 1));
+      }
       T c1 = INF, c2 = INF;
       int32_t y1 = 0, y2 = 0;
       if (t >= 2) {
@@ -233,11 +257,26 @@ void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Co
       }
       D1.col(m)[t] = y1;
       D2.col(m)[t] = y2;
-      if (c1 >= INF && c2 >= INF) { c[t] = INF; continue; }
-      if (c1 <= c2) { c[t] = c1; H.col(m)[t] = 1; }   // ties: the hidden state (fewer units)
-      else          { c[t] = c2; H.col(m)[t] = 2; }
+      if (c1 >= INF && c2 >= INF) c[t] = INF;
+      else if (c1 <= c2) { c[t] = c1; H.col(m)[t] = 1; }   // ties: the hidden state (fewer units)
+      else               { c[t] = c2; H.col(m)[t] = 2; }
+      if ((t & 7) == 0 || t == t_max) rows[(size_t)m].store(t, std::memory_order_release);
     }
+   }
+  };
+  // few, short columns are not worth a thread
+  unsigned n_threads = std::thread::hardware_concurrency();
+  if (n_threads > 16) n_threads = 16;
+  if (n_threads < 1 || plan_scan_only() || t_max * m_max < 200000) n_threads = 1;
+  if ((int64_t)n_threads > m_max) n_threads = (unsigned)m_max;
+  std::vector<std::thread> pool;
+  try {
+    for (unsigned i = 1; i < n_threads; ++i) pool.emplace_back(worker);
+  } catch (const std::system_error&) {
+    // fewer threads than hoped for: the ones that started, and this one, do all the columns
   }
+  worker();
+  for (std::thread& th : pool) th.join();
 }
 
 template <class S, class Dst>

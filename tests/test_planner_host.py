@@ -60,9 +60,12 @@ def test_whole_cost_tables_match_oracle():
 @pytest.mark.parametrize("mode", [P.HSM, P.ISM, P.MSM])
 def test_convexity_shortcut_changes_no_table_entry(mode, monkeypatch):
     """Where a cost column is convex in t the planner walks from the previous split point instead
-    of scanning every y (Appendix A's remark); with MEBPTT_PLAN_SCAN=1 it scans everywhere.  Both
-    must give the same C and the same D (smallest y on ties) in every cell."""
-    for t, m in [(150, 150), (257, 31), (64, 200), (2, 1), (1, 5)]:
+    of scanning every y (Appendix A's remark), and the mixed mode's columns are filled by several
+    threads; with MEBPTT_PLAN_SCAN=1 one thread scans everywhere.  Both must give the same C and
+    the same D (smallest y on ties) in every cell."""
+    # (the last size is large enough for the mixed mode's columns to be filled by several threads,
+    # which MEBPTT_PLAN_SCAN=1 also turns off)
+    for t, m in [(150, 150), (257, 31), (64, 200), (2, 1), (1, 5)] + ([(300, 800)] if mode == P.MSM else []):
         fast = B.mebptt_plan_ex(t, m, mode, 4, 0).tables()
         monkeypatch.setenv("MEBPTT_PLAN_SCAN", "1")
         slow = B.mebptt_plan_ex(t, m, mode, 4, 0).tables()
