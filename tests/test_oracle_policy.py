@@ -217,3 +217,33 @@ def test_protocol_simulation_with_beta():
 def test_infeasible_budget_is_rejected():
     with pytest.raises(P.ProtocolError):
         P.simulate(P.ISM, 5, 0)
+
+
+def test_chen_schedules_against_closed_forms():
+    """Chen's schedules (Section 2.2) where their cost and memory can be written down by hand.
+
+    sqrt(t) on a perfect square t = s^2: s - 1 segments are run twice, so t + (t - s) forward
+    operations, and at the worst moment s - 1 boundaries plus s internal states are kept (plus the
+    start state).  Recursive with k = 1 on t = 2^d: every level reruns the first half of each
+    piece, t / 2 operations per level over d levels, and keeps one state per level; the last piece
+    of one step keeps one internal state.  With k >= t nothing is cut: standard BPTT."""
+    for s in (2, 3, 8, 31):
+        r = P.chen_sqrt(s * s, 4, 3)
+        assert r["forwards"] == 2 * s * s - s and r["units"] == 1 + (s - 1) + 3 * s
+        r = P.chen_sqrt(s * s, 4)
+        assert r["units"] == 1 + (s - 1) + 4 * s
+    for d in (1, 2, 5, 10):
+        t = 1 << d
+        r = P.chen_recursive(t, 1, 4, 3)
+        assert r["forwards"] == t + d * (t // 2) and r["units"] == 1 + d + 3
+    for t, k in [(5, 5), (7, 30)]:
+        r = P.chen_recursive(t, k, 4)
+        assert r["forwards"] == t and r["units"] == 1 + 4 * t
+    # k cuts per level: a three-way cut of 9 steps with k = 2 ends in pieces of one step after two
+    # levels: passes of 6 and 3 x 2 steps, 9 single steps at the bottom
+    r = P.chen_recursive(9, 2, 4, 3)
+    assert r["forwards"] == 6 + 3 * 2 + 9 and r["units"] == 1 + 2 + 2 + 3
+    # the paper's figures: memory grows like k log_{k+1} t, at least log2 t hidden states at k = 1
+    assert P.chen_recursive(1000, 1, 4, 3)["units"] >= 10
+    for t in (100, 1000):
+        assert P.chen_recursive(t, 3, 4, 3)["forwards"] >= P.cost(P.MSM, t, P.chen_recursive(t, 3, 4, 3)["units"], 4, 3)
