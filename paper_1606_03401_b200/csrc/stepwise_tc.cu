@@ -291,7 +291,6 @@ int forward_step(const generic::FwdArgs& a, const Scratch& w, cudaStream_t s) {
   rc = gemm_bf16(a.h_prev, a.H, false, W + a.I, K, false, GemmOut{GemmOut::ACCUM_F32, w.z, G, nullptr, 0}, a.B, G,
                  a.H, w.status, s, true, &w.split, tc::gemm_split_count_deferred(a.B, G, a.H), &zp);
   if (rc != MEBPTT_OK) return rc;
-  const size_t n = (size_t)a.B * a.H;
   run_cell_fwd(s, w.z, a.c_prev, (const bf16*)a.h_prev, (bf16*)a.h_out, a.c_out, (bf16*)a.gates, a.plane_elems,
                (bf16*)a.h_in_copy, a.c_in_copy, a.B, a.H, a.counters, (bf16*)nullptr, zp);
   return MEBPTT_OK;
@@ -318,7 +317,6 @@ int readout(const generic::ReadoutArgs& a, const Scratch& w, int sidx, cudaStrea
 
 int backward_layer(const generic::BwdArgs& a, const Scratch& w, int l, int sidx, cudaStream_t s) {
   const int K = a.I + a.H, G = 4 * a.H;
-  const size_t n = (size_t)a.B * a.H;
   const bf16* W = (const bf16*)a.W;
   const size_t rows = (size_t)w.S * a.B;   // rows of one layer's stages
   bf16* dz16 = w.st_dz + ((size_t)l * rows + (size_t)sidx * a.B) * G;

@@ -522,7 +522,6 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
 
   uint32_t issued = 0, consumed = 0;
   constexpr uint32_t idesc = make_idesc(1, BM, NU, false, false);
-  const int G = 4 * a.H;
 
   for (int i = 0; i < a.n; ++i) {
     const DevOp op = a.ops[i];
