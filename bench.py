@@ -153,9 +153,9 @@ def kernel_breakdown(dp, plans):
 
 
 # DRAM traffic of the forward run kernel per forward operation, from the ncu capture summarised in
-# profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md (25.61 MB read, nothing written to DRAM, per
-# launch of 16 operations).  Valid for config 3's layer sizes and the kernel as profiled there.
-FWD_RUN_DRAM_BYTES_PER_OP_C3 = 25.612032e6 / 16
+# profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md (42.39 MB read, 0.29 MB written, per launch of
+# 32 operations).  Valid for config 3's layer sizes and the kernel as profiled there.
+FWD_RUN_DRAM_BYTES_PER_OP_C3 = (42.389248e6 + 0.290816e6) / 32
 
 
 def max_over_ranks(v: float, world: int, device) -> float:
@@ -338,7 +338,7 @@ def main():
                     "share_of_step": (f_ms / 3) / ms,
                     "backward_runs": {"kernel": "bwd_run_cluster_kernel", "launches": b_n // 3,
                                       "us_per_op": b_ms * 1e3 / max(1, b_ops), "share_of_step": (b_ms / 3) / ms},
-                    "traffic_note": "DRAM bytes per launch = bytes per operation (ncu, 16-operation launch) x mean operations per launch",
+                    "traffic_note": "DRAM bytes per launch = bytes per operation (ncu, 32-operation launch) x mean operations per launch",
                     "how": f"CUDA events around each launch, 3 steps; {flops_rec} flops per operation x operations per launch / mean "
                            f"launch duration; peak = bf16 sustained ({pk['source']})"}
     else:
