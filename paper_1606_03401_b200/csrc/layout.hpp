@@ -134,6 +134,14 @@ inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.rec = y.rec_in + y.unit;
 }
 
+// Steps per chunk on the step-by-step paths: 2048 rows of the batched GEMMs, at most 32 steps (a
+// run's per-step pointers are passed to kernels by value).  At config 5 (B = 128): 1024 rows
+// 31.1 ms per step at t = 256 and 229 MB of working memory, 2048 rows 28.0 ms and 407 MB.
+inline int stepwise_chunk_steps(int B) {
+  const int s = 2048 / B > 0 ? 2048 / B : 1;
+  return s > 32 ? 32 : s;
+}
+
 // The tensor-core executor cuts the tape into work items:
 //   FWD   a run of consecutive forward operations, each starting from the state the previous one
 //         wrote, at most S of them (one persistent launch);
@@ -215,7 +223,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
       y.n_loss_part = (y.B / 32) * ((y.O + 31) / 32);
       y.off_z = take((size_t)y.B * 4 * y.H * 4);
       // stages of one chunk of S steps for the weight-gradient contractions
-      y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
+      y.S = stepwise_chunk_steps(y.B);
       const size_t rows = (size_t)y.S * y.B;
       y.off_st_dz = take((size_t)y.L * rows * 4 * y.H * 2);
       y.off_st_in = take(rows * y.I * 2 + (size_t)(y.L - 1) * rows * y.H * 2);
@@ -236,7 +244,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     if (y.stepwise_x3) {
       const size_t G = 4 * (size_t)y.H, Kmax = (size_t)(y.I > y.H ? y.I : y.H) + y.H;
       y.n_loss_part = (y.B / 32) * ((y.O + 31) / 32);
-      y.S = 1024 / y.B > 0 ? 1024 / y.B : 1;
+      y.S = stepwise_chunk_steps(y.B);
       const size_t rows = (size_t)y.S * y.B;
       y.off_z = take((size_t)y.B * G * 4);
       // the readout of a run of up to S steps at once; its split-K scratch as on the bfloat16 path

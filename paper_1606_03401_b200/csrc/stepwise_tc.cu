@@ -254,7 +254,7 @@ __global__ void sum_parts_stage_h(const float* part, int n, float* out, const ui
   }
 }
 
-// Up to 32 device pointers passed by value (a run has at most S = 1024 / B <= 32 steps).
+// Up to 32 device pointers passed by value (a run has at most 32 steps).
 struct RunPtrs { const void* p[32]; };
 
 // Row block a of `dst` (n16 16-byte words each) <- src.p[a]; blockIdx.y = a.
