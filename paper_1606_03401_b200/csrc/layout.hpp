@@ -134,8 +134,9 @@ inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.rec = y.rec_in + y.unit;
 }
 
-// Steps per chunk on the step-by-step paths: 2048 rows of the batched GEMMs, at most 32 steps (a
-// run's per-step pointers are passed to kernels by value).  At config 5 (B = 128): 1024 rows
+// Steps per chunk on the step-by-step paths: 2048 rows of the batched GEMMs, at most 32 steps (at
+// batch 32, 64 steps were measured: config 4 at full memory 134 -> 128 ms per step for 134 MB more
+// working memory, not taken).  At config 5 (B = 128): 1024 rows
 // 31.1 ms per step at t = 256 and 229 MB of working memory, 2048 rows 28.0 ms and 407 MB.
 inline int stepwise_chunk_steps(int B) {
   const int s = 2048 / B > 0 ? 2048 / B : 1;

@@ -254,8 +254,8 @@ __global__ void sum_parts_stage_h(const float* part, int n, float* out, const ui
   }
 }
 
-// Up to 32 device pointers passed by value (a run has at most 32 steps).
-struct RunPtrs { const void* p[32]; };
+// Up to 64 device pointers passed by value (a run has at most 64 steps).
+struct RunPtrs { const void* p[64]; };
 
 // Row block a of `dst` (n16 16-byte words each) <- src.p[a]; blockIdx.y = a.
 __global__ void stage_blocks(RunPtrs src, uint4* dst, size_t n16) {
@@ -406,7 +406,7 @@ int readout_run(const void* const* h_top, int n, int s_lo, const void* W_out_, c
   o.scale = 1.f / ((float)B * (float)O);
   int rc = gemm_bf16(st_h, H, false, W_out, H, false, o, n * B, O, H, w.status, s);
   if (rc != MEBPTT_OK) return rc;
-  launch_pdl(sum_parts_steps, dim3(1), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
+  launch_pdl(sum_parts_steps, dim3((n + 31) / 32), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
   // the gradient entering the top layer at every step of the run, split along K like a single step's
   const int splits = tc::gemm_split_count(false, true, B, H, O, w.split.partial_floats);
   rc = gemm_bf16(dy16, O, false, W_out, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H, O,

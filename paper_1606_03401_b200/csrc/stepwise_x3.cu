@@ -86,9 +86,9 @@ __global__ void split_a3(const float* a, int Ca, const float* b_, int Cb, int B,
   }
 }
 
-// The same split for up to 32 row blocks of [B][C] that lie apart (blockIdx.y picks the block);
+// The same split for up to 64 row blocks of [B][C] that lie apart (blockIdx.y picks the block);
 // block a goes to rows a B .. of `out`.
-struct RunPtrs { const float* p[32]; };
+struct RunPtrs { const float* p[64]; };
 __global__ void split_blocks3(RunPtrs src, int C, int B, bf16* out) {
   sm100::grid_dep_wait();
   sm100::grid_dep_launch();
@@ -371,7 +371,7 @@ int readout_run(const float* const* h_top, int n, int s_lo, const float* b_out, 
   o.scale = 1.f / ((float)B * (float)O);
   int rc = gemm_bf16(h3, 3 * H, false, w.wout3, 3 * H, false, o, n * B, O, 3 * H, w.status, s);
   if (rc != MEBPTT_OK) return rc;
-  launch_pdl(sum_parts_steps, dim3(1), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
+  launch_pdl(sum_parts_steps, dim3((n + 31) / 32), dim3(32), 0, s, (const float*)w.loss_part, per_step, n, loss_t);
   launch_pdl(split_a3, dim3(ew_blocks(no)), dim3(256), 0, s, (const float*)w.dy_run, O, (const float*)nullptr, 0, n * B, dy3);
   const int splits = tc::gemm_split_count(false, true, B, H, 3 * O, w.split.partial_floats);
   return gemm_bf16(dy3, 3 * O, false, w.woutmn3, H, true, GemmOut{GemmOut::STORE_F32, w.dha_run, H, nullptr, 0}, n * B, H,
