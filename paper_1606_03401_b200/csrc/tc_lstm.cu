@@ -1364,7 +1364,16 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       const int k0 = first.k;
       if (!(k0 >= zx_lo && k0 + n <= zx_hi)) {
         zx_lo = k0;
-        zx_hi = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
+        // as far as the runs that will still find their steps in this window reach (the first
+        // forward run that does not fit in the S steps from k0 on replaces the window)
+        const int cap = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
+        zx_hi = k0 + n;
+        for (size_t j = item + 1; j < items.size(); ++j) {
+          if (items[j].kind != WorkItem::FWD) continue;
+          const int kj = p->tape[items[j].i].k, ej = kj + items[j].n;
+          if (kj < k0 || ej > cap) break;
+          if (ej > zx_hi) zx_hi = ej;
+        }
         const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
         need_x(zx_hi - 1);
         gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
