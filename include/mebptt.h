@@ -78,8 +78,8 @@ enum { MEBPTT_FP32 = 0, MEBPTT_TF32 = 1, MEBPTT_BF16 = 2 };
  * Locations: >= 0 is an offset, in hidden-state units, into the slot arena (a stack: states are
  * read in the reverse order of writing, Section 3.1); negative values name buffers outside the
  * budget: the caller's initial state, the two scratch hidden states a forward sweep alternates
- * between, and the working core (Section 3.1: "a single RNN core available for the purposes of
- * intermediate calculations").  A memorisation is therefore not a copy: the forward operation
+ * between, and the working core (the one RNN core that Section 3.1 keeps for intermediate calculations,
+ * outside the budget m).  A memorisation is therefore not a copy: the forward operation
  * that produces the state writes it where it will be kept (Push), and the next forward
  * operation reads it from there (Peek).
  */
@@ -320,13 +320,21 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_
  * application hands it input and output buffers and nothing more, or a service in which an
  * allocation would stall the other streams of the device.  This entry point takes the same inputs
  * and outputs and no workspace; it uses a fixed array of MEBPTT_STATIC_WORKSPACE_BYTES that is part
- * of the library image, so every GPU that loads the library holds that much memory until the
- * process exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ * of the library image.  It calls no cudaMalloc, cudaFree or other allocating routine, and creates
+ * no stream or event.
  *
  *   - Problems whose workspace (mebptt_lstm_workspace_bytes) exceeds the array are refused with
  *     MEBPTT_ERR_WORKSPACE and nothing is enqueued; use mebptt_lstm_train_step for those.
- *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before starting any stream capture.
+ *   - The first call on each device is a set-up call: it looks up the array's device address
+ *     (with that device current).  With CUDA's default lazy module loading that look-up is also
+ *     the moment the driver places the array -- and, at their first launch, the code of the
+ *     kernels -- in device memory; only with CUDA_MODULE_LOADING=EAGER does this happen when the
+ *     library is loaded.  So make one call (any small problem will do) per device while device
+ *     memory is still to be had, and before starting any stream capture; it fails with
+ *     MEBPTT_ERR_CUDA if the array cannot be placed.  From then on the GPU holds the array until
+ *     the process exits, and later calls reserve nothing.
+ *   - A descriptor with MEBPTT_FLAG_TIME_RUNS is refused with MEBPTT_ERR_ARG: per-launch timing
+ *     creates CUDA events, which this entry point promises not to do.
  *   - All calls on a device share the one array.  Each call clears the parts that must start at
  *     zero, so leftovers of the previous call do not matter, but two calls whose device work
  *     overlaps (different streams, or the ordinary entry point given this memory) race: keep

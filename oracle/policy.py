@@ -172,7 +172,7 @@ def chen_recursive(t: int, k: int, alpha: int, beta: int | None = None):
     dropped once the part that starts there is done.  A sequence of at most k steps is run forward
     keeping every internal state (beta units each when their input hidden states are left out,
     else alpha) and backpropagated.  Units count the start state, as in the mixed scheme.
-    Reading: the paper's summary says "k equal parts"; k memorised states per level (k + 1
+    Reading: Section 2.2 summarises the scheme as a split into k parts; k memorised states per level (k + 1
     parts) is what its figures need -- memory O(k log_{k+1} t) and a minimum of log2 t at k = 1.
     """
     per = beta if beta is not None else alpha

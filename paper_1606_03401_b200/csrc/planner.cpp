@@ -70,7 +70,7 @@ int64_t convex_first_argmin(const T* a, const T* b_last, int64_t n, int64_t gues
 
 // A column of costs seen as a sequence in t: the longest prefix lo .. hi of it that is finite and
 // convex (second differences >= 0), extended one element at a time.  Appendix A remarks that the
-// O(t^2 m) scan can be brought down to O(t m) "by exploiting convexity in t"; the paper does not
+// O(t^2 m) scan can be brought down to O(t m) through convexity in t; the paper does not
 // prove convexity, so it is checked on the numbers before it is used, and wherever it fails the
 // scan is kept.
 template <class T>
@@ -504,9 +504,9 @@ int build_chen_plan(int64_t t, int alpha, int beta, Plan** out) {
 // Chen's recursive schedule (Section 2.2) as a tape: a sequence of more than k steps is cut into
 // k + 1 parts as equal as they come, one forward pass memorises the hidden state at the k cuts,
 // and the parts are then treated the same way from the last to the first; a sequence of at most
-// k steps is run forward with every internal state kept and backpropagated.  (The paper's
-// summary speaks of "k equal parts" and of stopping "once the subsequence length becomes less than
-// k"; k memorised states per level, hence k + 1 parts, is the reading under which its figures --
+// k steps is run forward with every internal state kept and backpropagated.  (Section 2.2
+// summarises the scheme as a split into k parts that stops when a part is shorter than k;
+// k memorised states per level, hence k + 1 parts, is the reading under which its figures --
 // memory O(k log_{k+1} t), at least log_2 t for k = 1 -- come out.)
 int build_chen_recursive_plan(int64_t t, int k, int alpha, int beta, Plan** out) {
   if (!out) return MEBPTT_ERR_ARG;

@@ -6,7 +6,13 @@
 // Some callers cannot do that at the point where they train: code that runs after the process
 // has handed all free device memory to another component, plug-ins that are only given input
 // and output buffers by their host application, and set-ups where any allocation would stall
-// other streams on the device.  For them the scratch is reserved when the library is loaded.
+// other streams on the device.  For them the scratch is a fixed array in the library image.
+//
+// When the array takes up device memory: this file is a module of its own, and with CUDA's
+// default lazy module loading a module is placed on a device when something of it is first
+// asked for -- here the symbol look-up of the first call on that device (at load time only with
+// CUDA_MODULE_LOADING=EAGER).  That first call is therefore a set-up call, to be made while
+// device memory is still available; afterwards the array stays until the process exits.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -24,7 +30,7 @@ int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, con
 
 namespace {
 
-// Every GPU that loads the library holds this array until the process exits.
+// Every GPU on which the entry point below has been called holds this array until the process exits.
 static __device__ __align__(256) unsigned char g_static_workspace[MEBPTT_STATIC_WORKSPACE_BYTES];
 
 constexpr int kMaxDevices = 64;
@@ -56,6 +62,8 @@ extern "C" int mebptt_lstm_train_step_static(const mebptt_lstm_desc* desc, const
                                              const void* x, const void* targets, const void* h0, const void* c0,
                                              void* stream, float* loss, float* dW, float* db, float* dW_out,
                                              float* db_out, float* dx, int64_t* counters) {
+  // per-launch timing records CUDA events, created on demand: not here
+  if (desc && (desc->flags & MEBPTT_FLAG_TIME_RUNS)) return MEBPTT_ERR_ARG;
   const size_t need = mebptt_lstm_workspace_bytes(desc, plan);
   if (need == 0) return MEBPTT_ERR_ARG;                                   // bad descriptor or plan
   if (need > (size_t)MEBPTT_STATIC_WORKSPACE_BYTES) return MEBPTT_ERR_WORKSPACE;  // does not fit the fixed array

@@ -8,6 +8,11 @@ of the chosen precision, so every consumer sees exactly the same numbers:
 * x, targets ~ N(0, 1) i.i.d.
 * W (all layers), W_out ~ U(-1/sqrt(H), 1/sqrt(H)); biases 0 except the forget-gate block,
   which is 1; h0 = c0 = 0.
+* ``make_problem(cfg, general=True)`` keeps x, targets and the weights and draws what the
+  benchmark recipe leaves at a constant: every bias entry of every layer and of the readout
+  ~ U(-0.3, 0.3) (the forget-gate block keeps its offset of 1), h0, c0 ~ 0.5 N(0, 1).  A
+  consumer that mislaid a bias entry, dropped the readout bias or mishandled the caller's
+  initial state cannot pass on such a problem.
 
 Arrays are returned as float64 holding values that are exactly representable in the storage
 type ("bf16": x, W, W_out, h0 in bfloat16 and the rest in float32; "fp32"/"tf32": float32).
@@ -73,8 +78,12 @@ def round_to_fp32(a: np.ndarray) -> np.ndarray:
     return np.asarray(a, np.float64).astype(np.float32).astype(np.float64)
 
 
-def make_problem(cfg: LstmConfig) -> dict:
-    """Draw one problem.  Keys: W (list per layer), b (list), W_out, b_out, x, targets, h0, c0."""
+def make_problem(cfg: LstmConfig, general: bool = False) -> dict:
+    """Draw one problem.  Keys: W (list per layer), b (list), W_out, b_out, x, targets, h0, c0.
+
+    general: also draw the biases, the readout bias and the initial state (after everything else,
+    so that x, targets and the weights are those of the plain problem with the same seed).
+    """
     rng = np.random.Generator(np.random.Philox(key=cfg.seed))
     L, I, H, B, t, O = cfg.layers, cfg.input, cfg.hidden, cfg.batch, cfg.t, cfg.readout
     lim = 1.0 / np.sqrt(H)
@@ -92,6 +101,11 @@ def make_problem(cfg: LstmConfig) -> dict:
     targets = round_to_fp32(rng.standard_normal(size=(t, B, O)))
     h0 = np.zeros((L, B, H))
     c0 = np.zeros((L, B, H))
+    if general:
+        b = [round_to_fp32(v + rng.uniform(-0.3, 0.3, size=4 * H)) for v in b]
+        b_out = round_to_fp32(rng.uniform(-0.3, 0.3, size=O))
+        h0 = opnd(0.5 * rng.standard_normal(size=(L, B, H)))
+        c0 = round_to_fp32(0.5 * rng.standard_normal(size=(L, B, H)))
     return {"W": W, "b": b, "W_out": W_out, "b_out": b_out, "x": x, "targets": targets,
             "h0": h0, "c0": c0}
 

@@ -138,3 +138,55 @@ def test_synthetic_problem_is_seeded_and_representable():
     assert synth.round_to_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
     d = synth.to_device_arrays(cfg, a)
     assert d["W"].dtype == np.uint16 and d["targets"].dtype == np.float32
+
+
+def test_general_problem_keeps_the_plain_draws_and_adds_distinguishing_values():
+    from paper_1606_03401_b200 import synth
+    cfg = synth.with_overrides(synth.CONFIGS["c2"], t=3, batch=2, hidden=8, input=8, readout=8, layers=2)
+    a, g = synth.make_problem(cfg), synth.make_problem(cfg, general=True)
+    for k in ("W_out", "x", "targets"):
+        assert np.array_equal(a[k], g[k])
+    assert all(np.array_equal(u, v) for u, v in zip(a["W"], g["W"]))
+    for l in range(2):
+        d = g["b"][l] - a["b"][l]
+        assert np.all(np.abs(d) <= 0.3 + 1e-6) and len(np.unique(g["b"][l])) == 32
+    assert len(np.unique(g["b_out"])) == 8 and np.all(np.abs(g["b_out"]) <= 0.3 + 1e-6)
+    assert np.array_equal(synth.round_to_bf16(g["h0"]), g["h0"]) and np.abs(g["h0"]).max() > 0
+    assert np.array_equal(synth.round_to_fp32(g["c0"]), g["c0"]) and np.abs(g["c0"]).max() > 0
+
+
+def test_block_check_catches_what_the_whole_tensor_norm_lets_through():
+    """The parity helper compares block by block: one wrong 128 x 128 tile, one wrong gate row
+    block entry or one wrong group of bias entries, planted in a copy of the oracle's result, stays
+    far below the whole-tensor tolerance and must still be refused."""
+    import pytest
+    from tests.util import assert_close_to_oracle, flat_oracle
+    r = np.random.default_rng(5)
+    H, K, O, t, B, I = 256, 768, 128, 6, 4, 128
+    ref = {"loss": 1.0, "dW": [r.standard_normal((4 * H, K))], "db": [r.standard_normal(4 * H)],
+           "dW_out": r.standard_normal((O, H)), "db_out": r.standard_normal(O), "dx": r.standard_normal((t, B, I))}
+
+    def result():
+        fo = flat_oracle(ref)
+        return {"loss": 1.0, **{k: v.copy() for k, v in fo.items()}}
+
+    assert_close_to_oracle(result(), ref, "bf16", want_dx=True)
+    for key, plant in [
+        ("dW", lambda a: a.reshape(4 * H, K).__setitem__((slice(128, 256), slice(256, 384)), 0.0)),       # a lost tile
+        ("db", lambda a: a.__setitem__(slice(512, 544), a[512:544] * 1.5)),                              # 32 entries off
+        ("dW_out", lambda a: a.reshape(O, H).__setitem__((slice(0, 128), slice(128, 256)),
+                                                         a.reshape(O, H)[0:128, 0:128])),                # a misplaced tile
+        ("db_out", lambda a: a.__setitem__(slice(96, 128), 0.0)),                                        # dropped entries
+        ("dx", lambda a: a.reshape(t, B, I).__setitem__(0, 0.0)),                                        # a missing step
+    ]:
+        res = result()
+        plant(res[key])
+        with pytest.raises(AssertionError):
+            assert_close_to_oracle(res, ref, "bf16", want_dx=True)
+    # a dW tile that is 12 % off is under the whole-tensor tolerance at this size: only the block check sees it
+    res = result()
+    res["dW"].reshape(4 * H, K)[128:256, 256:384] *= 0.88
+    from tests.util import rel_l2
+    assert rel_l2(res["dW"], flat_oracle(ref)["dW"]) < 2e-2
+    with pytest.raises(AssertionError):
+        assert_close_to_oracle(res, ref, "bf16", want_dx=True)

@@ -44,9 +44,16 @@ def test_static_workspace_step_matches_ordinary_step_twice(base, kw, mode, m):
     dp = harness.DeviceProblem(cfg, want_dx=True)
     plan = dp.plan(mode, m)
     assert B.mebptt_lstm_workspace_bytes(dp.desc, plan) <= B.MEBPTT_STATIC_WORKSPACE_BYTES
+    import torch
     want = dp.run(plan)                      # ordinary entry point, caller-owned workspace
-    first = _static_run(dp, plan)
+    first = _static_run(dp, plan)            # the set-up call of this device, if no earlier test made it
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     second = _static_run(dp, plan)           # same array, previous contents still in it
+    torch.cuda.synchronize()
+    # nothing was reserved by the later call: the driver reports the same free memory (torch's own
+    # caching allocator serves the result copies from host memory and blocks it already holds)
+    assert torch.cuda.mem_get_info()[0] >= free_before
     for got in (first, second):
         assert got["counters"][0] == plan.cost and got["counters"][1] == cfg.t and got["counters"][3] == 0
         assert_bit_identical(got, want, want_dx=True)
@@ -54,6 +61,18 @@ def test_static_workspace_step_matches_ordinary_step_twice(base, kw, mode, m):
     other = dp.full_memory_plan()
     if B.mebptt_lstm_workspace_bytes(dp.desc, other) <= B.MEBPTT_STATIC_WORKSPACE_BYTES:
         assert_bit_identical(_static_run(dp, other), want, want_dx=True)
+
+
+def test_static_workspace_step_refuses_per_launch_timing():
+    """Timing every launch creates CUDA events on demand, which the allocation-free call must not."""
+    from paper_1606_03401_b200 import binding as B
+    desc = B.make_desc(1, 64, 128, 64, 32, 40, "bf16", flags=B.MEBPTT_FLAG_TIME_RUNS)
+    plan = B.mebptt_plan(40, 9, B.MEBPTT_MSM)
+    dummy = np.zeros(8, np.float32)
+    with pytest.raises(B.MebpttError) as e:
+        B.mebptt_lstm_train_step_static(desc, plan, dummy, dummy, dummy, dummy, dummy, dummy, dummy, dummy, None,
+                                        dummy, dummy, dummy, dummy, dummy, None, dummy)
+    assert e.value.status == B.MEBPTT_ERR_ARG
 
 
 def test_static_workspace_step_refuses_what_does_not_fit():
