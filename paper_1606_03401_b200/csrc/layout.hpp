@@ -296,7 +296,7 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_dha = take(SB * y.H * 4);
     y.off_zleaf = take(SB * G * 4);   // pre-activations of a batch of leaves
     y.off_loss_part = take((size_t)y.S * loss_parts_per_step(y.B, y.O) * 4);
-    y.n_sync = 32 * (work_items(p, y.S).size() + 1);   // 32 words (one 128-byte line) per persistent launch
+    y.n_sync = 64 * (work_items(p, y.S).size() + 1);   // two 128-byte lines per persistent launch (one per group of CTAs)
     y.off_sync = take(y.n_sync * 4);
     y.tape_bytes = (size_t)p->tape.size() * 32 * 2;   // the tape, and the compacted entries of leaf batches
     y.off_tape = take(y.tape_bytes);

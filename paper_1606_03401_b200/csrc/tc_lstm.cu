@@ -97,58 +97,178 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 // ------------------------------------------------------------------------------------------
 // forward run
 // ------------------------------------------------------------------------------------------
+// What bounds a step of the recurrence is the time h_{k-1} takes to reach every SM that holds a
+// part of W_hh (the bytes all SMs pull through the L2 together, and the bytes each takes in) and
+// the number of MMA instructions one thread must issue for a tile (one per 16 contraction
+// indices, whatever the tile's size).  Three things cut both:
+//
+//   * The batch rows of an LSTM never mix, so the grid is cut into groups of CTAs that each own
+//     FB = 32 batch rows: a CTA pulls only its group's rows of h_{k-1} and groups synchronise
+//     among themselves only (a step counter per group).
+//   * The product is taken transposed: gate rows of W_hh (resident in shared memory, rows permuted
+//     to 4 u + q) are the M side of the MMA and the 32 batch rows the N side, so that a tile of
+//     full height serves a batch slice of 32.
+//   * Two neighbouring CTAs (a cluster of two) share 32 hidden units and split the contraction
+//     index: CTA r keeps the block [128 gate rows][K half r] of W_hh, pulls only that half of the
+//     columns of h_{k-1}, and issues half the MMAs.  The partial tile [128][32] leaves TMEM one
+//     gate row per thread and goes, 64 rows each, to the CTA that owns those rows -- into its
+//     shared memory, its own or the neighbour's (distributed shared memory).
+//
+// Each of the 128 epilogue threads then owns four hidden units of one batch row: it adds, in a
+// fixed order, z = (Zx + part 0) + part 1 -- Zx being the batched input projection, bias included
+// -- applies the gates and updates c_t, h_t (which stay in registers from step to step), and
+// writes the state where the tape says (scratch, a slot of the arena, or a whole internal state).
+// fwd_run_kernel is the same computation without clusters: one CTA per 16 hidden units takes both
+// halves of the contraction into two accumulators.  Both give the same bits, and so do the
+// batched GEMMs of a leaf batch, which accumulate Zx, the first and the second half in that order.
+//
+// Warps 0-3: epilogue; warp 4: TMA producer; warp 5: MMA issuer.  All of h_{k-1} a CTA needs is
+// resident in shared memory for the step (H <= 1024), so the producer never waits for a free slot.
+constexpr int FU = 16;          // hidden units per CTA
+constexpr int FG = 4 * FU;      // gate rows per CTA
+constexpr int FB = 32;          // batch rows per group of CTAs: the N of the MMA
+constexpr int PART_LD = FB + 4; // row stride of a partial tile in shared memory (floats)
+constexpr int SYNC_STRIDE = 32; // words between the step counters of two groups (one 128-byte line each)
+
 struct FwdRunArgs {
   const DevOp* ops;      // this launch's operations (consecutive forward operations)
   int n;
   char* ws;              // workspace base
   const float* zx;       // [n][B][4H]: input projection + bias, gate columns permuted (4 u + q)
-  uint32_t* sync;        // grid-wide step counter of this launch (zero on entry)
+  uint32_t* sync;        // step counters of this launch, one per group (zero on entry)
   int* status;
   int64_t* counters;
   int B, H;
+  int ncg;               // CTAs per group
+  int bb;                // K tiles (64 contraction indices each) per barrier and, in slab mode, per copy
+  int slab;              // 1: tm_h is a blocked 3-D map and one copy brings bb tiles; 0: one 2-D copy per tile
   uint32_t plane16;      // distance between gate planes, in 16-byte units
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
 };
 
-// Warps 0-3: epilogue (warp w owns rows 16w .. 16w+15 of the 64-row MMA tile, which are the
-// TMEM lanes it may read); warp 4: TMA producer; warp 5: MMA issuer.  All of h_{k-1} is resident
-// in shared memory for the step (H <= 1024), so the producer never waits for a free slot.
-// (Cutting the batch into groups with independent step counters was tried and does not help: a
-// step is bound by the latency of the exchange, which every group pays in full.)
+// 64-wide blocks of the contraction index in the first part of the split (all of them if there is one)
+__host__ __device__ inline int fwd_first_part_blocks(int H) {
+  const int KB = (H + 63) / 64;
+  return KB >= 2 ? (KB + 1) / 2 : KB;
+}
+
+// State update of one thread: batch row b, hidden units j0 .. j0 + 3.  z[u] holds the four
+// pre-activations (i, f, g, o) of unit j0 + u; writes h_k at once and the rest of the state after
+// `signal` has told the other CTAs that h_k is there.
+struct FwdCell {
+  float c[4];
+  uint2 hprev;
+  float4 zx[4];
+};
+__device__ __forceinline__ void fwd_cell_init(FwdCell& st, const FwdRunArgs& a, bool owner, int b, int j0, size_t e0) {
+#pragma unroll
+  for (int u = 0; u < 4; ++u) { st.c[u] = 0.f; st.zx[u] = make_float4(0.f, 0.f, 0.f, 0.f); }
+  st.hprev = make_uint2(0, 0);
+  if (!owner) return;
+  const DevOp op0 = a.ops[0];
+  const float4 c0 = *(reinterpret_cast<const float4*>(a.ws + (size_t)op0.c_src * 16) + e0 / 4);
+  st.c[0] = c0.x; st.c[1] = c0.y; st.c[2] = c0.z; st.c[3] = c0.w;
+  st.hprev = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op0.h_src * 16) + e0);
+  const float4* zp = reinterpret_cast<const float4*>(a.zx + (size_t)b * 4 * a.H + (size_t)4 * j0);
+#pragma unroll
+  for (int v = 0; v < 4; ++v) st.zx[v] = zp[v];
+}
+struct FwdCellOut {
+  uint2 hnew, gi, gf, gg, go;
+  float cin[4];
+};
+__device__ __forceinline__ void fwd_cell_gates(FwdCell& st, const float4 (&z)[4], FwdCellOut& o) {
+  float hv[4], iv[4], fv[4], gv[4], ov[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    iv[u] = sigmoid_fast(z[u].x);
+    fv[u] = sigmoid_fast(z[u].y);
+    gv[u] = tanh_fast(z[u].z);
+    ov[u] = sigmoid_fast(z[u].w);
+    o.cin[u] = st.c[u];
+    st.c[u] = fmaf(fv[u], st.c[u], iv[u] * gv[u]);
+    hv[u] = ov[u] * tanh_fast(st.c[u]);
+  }
+  o.hnew = make_uint2(pack_bf16x2(hv[0], hv[1]), pack_bf16x2(hv[2], hv[3]));
+  o.gi = make_uint2(pack_bf16x2(iv[0], iv[1]), pack_bf16x2(iv[2], iv[3]));
+  o.gf = make_uint2(pack_bf16x2(fv[0], fv[1]), pack_bf16x2(fv[2], fv[3]));
+  o.gg = make_uint2(pack_bf16x2(gv[0], gv[1]), pack_bf16x2(gv[2], gv[3]));
+  o.go = make_uint2(pack_bf16x2(ov[0], ov[1]), pack_bf16x2(ov[2], ov[3]));
+}
+// The part of the state that is not on the critical path of the recurrence, and the input
+// projection of the next step (which does not depend on the recurrence either).
+__device__ __forceinline__ void fwd_cell_rest(FwdCell& st, const FwdRunArgs& a, const DevOp& op, const FwdCellOut& o,
+                                              int i, int b, int j0, size_t e0) {
+  char* ws = a.ws;
+  *(reinterpret_cast<float4*>(ws + (size_t)op.c_dst * 16) + e0 / 4) = make_float4(st.c[0], st.c[1], st.c[2], st.c[3]);
+  if (op.gates) {
+    __nv_bfloat16* gp = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+    const size_t pl = (size_t)a.plane16 * 8;   // elements
+    *reinterpret_cast<uint2*>(gp) = o.gi;
+    *reinterpret_cast<uint2*>(gp + pl) = o.gf;
+    *reinterpret_cast<uint2*>(gp + 2 * pl) = o.gg;
+    *reinterpret_cast<uint2*>(gp + 3 * pl) = o.go;
+  }
+  if (op.in_copy) {
+    char* blk = ws + (size_t)op.in_copy * 16;
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = st.hprev;
+    *(reinterpret_cast<float4*>(blk + (size_t)a.hsz16 * 16) + e0 / 4) = make_float4(o.cin[0], o.cin[1], o.cin[2], o.cin[3]);
+  }
+  st.hprev = o.hnew;
+  if (i + 1 < a.n) {
+    const float4* zp = reinterpret_cast<const float4*>(a.zx + ((size_t)(i + 1) * a.B + b) * 4 * a.H + (size_t)4 * j0);
+#pragma unroll
+    for (int v = 0; v < 4; ++v) st.zx[v] = zp[v];
+  }
+}
+// z = (Zx + part 0) + part 1 for the 16 gate rows of this thread; a part is [64 gate rows][PART_LD]
+// with the batch row as the column.
+__device__ __forceinline__ void fwd_cell_sum(const FwdCell& st, const float* part0, const float* part1, int row0, int col,
+                                             float4 (&z)[4]) {
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const float* p = part0 + (size_t)(row0 + 4 * u) * PART_LD + col;
+    z[u] = make_float4(st.zx[u].x + p[0], st.zx[u].y + p[PART_LD], st.zx[u].z + p[2 * PART_LD], st.zx[u].w + p[3 * PART_LD]);
+    if (part1) {
+      const float* q = part1 + (size_t)(row0 + 4 * u) * PART_LD + col;
+      z[u].x += q[0]; z[u].y += q[PART_LD]; z[u].z += q[2 * PART_LD]; z[u].w += q[3 * PART_LD];
+    }
+  }
+}
+
+// One CTA per 16 hidden units and group; both halves of the contraction, into two accumulators.
 __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__ CUtensorMap tm_h,
                                                          const __grid_constant__ CUtensorMap tm_w,
                                                          const FwdRunArgs a) {
-  constexpr int GR = 1;                    // batch groups (see above)
-  constexpr int RG = 64 / GR;              // tile rows per group
-  constexpr int TG = 128 / GR;             // epilogue threads per group
-  constexpr uint32_t A_TILE = 64 * 128;
+  constexpr uint32_t W_TILE = FG * 128;   // [64 gate rows][64 contraction indices]
+  constexpr uint32_t H_TILE = FB * 128;   // [32 batch rows][64 contraction indices]
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[GR][4], acc[GR];
+  __shared__ uint64_t wfull, full[4], acc;
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
 
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int KB = (a.H + 63) / 64;      // <= 16
-  uint8_t* sW = sm;                    // KB tiles of [32 rows][128 B]: this CTA's rows of W_hh
-  uint8_t* tiles = sm + KB * 4096;     // KB tiles of [64 rows][128 B]: all of h_{k-1}
+  const int KB0 = fwd_first_part_blocks(a.H);
+  uint8_t* sW = sm;                    // KB tiles: this CTA's rows of W_hh
+  uint8_t* tiles = sm + KB * W_TILE;   // KB tiles: the group's rows of h_{k-1}
+  const int NQ = KB0 < KB ? 2 : 1;     // parts of the contraction: one barrier, one copy (slab mode), one accumulator each
+  float* part = reinterpret_cast<float*>(tiles + NQ * KB0 * H_TILE);   // [2][FG][PART_LD]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int cta = blockIdx.x, ncta = gridDim.x;
-  const int Bg = (a.B + GR - 1) / GR;  // batch rows per group
-  const int NQ = (KB + 3) / 4;         // blocks of four K tiles, one barrier each
+  const int grp = blockIdx.x / a.ncg, cta = blockIdx.x % a.ncg;
+  uint32_t* const sync = a.sync + grp * SYNC_STRIDE;
 
   if (tid == 0) {
     mbar_init(&wfull, 1);
-    for (int g = 0; g < GR; ++g) {
-      for (int s = 0; s < 4; ++s) mbar_init(&full[g][s], 1);
-      mbar_init(&acc[g], 1);
-    }
+    for (int s = 0; s < 4; ++s) mbar_init(&full[s], 1);
+    mbar_init(&acc, 1);
     failed = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tm_h);
     tma_prefetch_desc(&tm_w);
   }
-  if (warp == 4) tmem_alloc(&tmem_slot, 32 * GR);
+  if (warp == 4) tmem_alloc(&tmem_slot, 64);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -157,28 +277,37 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   grid_dep_wait();   // everything above touched no global memory; everything below may
 
   if (warp == 4) {
-    // ---- producer: lane 0 watches the step counter, then lanes 0 .. NQ-1 each request one block
-    // of four K tiles (issuing a TMA load costs ~80 ns; four lanes issue side by side) ------------
+    // ---- producer: lane 0 watches the group's step counter, then h_{k-1} is requested.  A copy
+    // instruction takes the TMA unit ~80-120 ns to accept whatever its size, and the unit takes one
+    // at a time: 16 tiles requested one by one are a microsecond.  In slab mode one copy (a 3-D box
+    // over a map that sees the row as blocks of 64 columns) brings a whole part of the split. ------
     if (lane == 0) {
-      mbar_arrive_expect_tx(&wfull, (uint32_t)KB * 4096u);
-      for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * 4096, &tm_w, kb * 64, cta * NG, &wfull);
+      mbar_arrive_expect_tx(&wfull, (uint32_t)KB * W_TILE);
+      for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + kb * W_TILE, &tm_w, kb * 64, cta * FG, &wfull);
     }
     int armed = -1;   // last step whose loads were requested (for the failure path)
     for (int i = 0; i < a.n; ++i) {
       const DevOp op = a.ops[i];
-      const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes);
+      // rows of the group inside the block of h_{k-1}; rows past the batch are never used (they
+      // only reach accumulator columns that no thread reads)
+      const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes) + grp * FB;
       int go = 1;
-      if (lane == 0) go = (i == 0 || wait_counter(a.sync, (uint32_t)i * (uint32_t)ncta, &failed)) && !failed;
+      if (lane == 0) go = (i == 0 || wait_counter(sync, (uint32_t)i * (uint32_t)a.ncg, &failed)) && !failed;
       go = __shfl_sync(0xffffffffu, go, 0);
       if (!go) continue;
-      if (lane < NQ) {
-        // the acquire of lane 0 reaches this lane through the shuffle; the proxy fence then orders
-        // this lane's TMA reads after the h_k written by the other CTAs
+      // the acquire of lane 0 reaches the other lanes through the shuffle; the proxy fence then orders
+      // a lane's TMA read after the h_k written by the other CTAs
+      if (a.slab) {
+        if (lane < NQ) {
+          fence_proxy_async_global();
+          mbar_arrive_expect_tx(&full[lane], (uint32_t)KB0 * H_TILE);   // a box counts in full, also where it is filled with zeros
+          tma_load_3d(tiles + lane * KB0 * H_TILE, &tm_h, 0, row, lane * KB0, &full[lane]);
+        }
+      } else if (lane < KB) {
         fence_proxy_async_global();
-        const int q = lane;
-        const int kb0 = 4 * q, kb1 = (kb0 + 4 < KB) ? kb0 + 4 : KB;
-        mbar_arrive_expect_tx(&full[0][q], (uint32_t)(kb1 - kb0) * A_TILE);
-        for (int kb = kb0; kb < kb1; ++kb) tma_load_2d(tiles + kb * A_TILE, &tm_h, kb * 64, row, &full[0][q]);
+        const int q = lane >= KB0 ? 1 : 0;
+        if (lane == q * KB0) mbar_arrive_expect_tx(&full[q], (uint32_t)(q ? KB - KB0 : KB0) * H_TILE);
+        tma_load_2d(tiles + lane * H_TILE, &tm_h, lane * 64, row, &full[q]);
       }
       armed = i;
       if (i == a.n - 1 && lane == 0) grid_dep_launch();   // last step under way: the next kernel may set itself up
@@ -188,144 +317,77 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
       // loads that were requested may still be landing: give them a bounded chance
       (void)mbar_wait(&wfull, 0);
       if (armed >= 0)
-        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[0][q], (uint32_t)armed & 1);
+        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
     }
   } else if (warp == 5) {
     // ---- MMA issuer: the whole warp walks the loop (so that addresses and descriptors stay in
     // uniform registers), one elected lane issues ------------------------------------------------
-    {
-      constexpr uint32_t idesc = make_idesc(1, 64, NG, false, false);
-      bool ok = wait_or_fail(&wfull, 0, &failed);
-      const uint64_t a_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
-      const uint64_t b_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
-      for (int i = 0; i < a.n; ++i) {
-        for (int g = 0; g < GR; ++g) {
-          const uint32_t d_tmem = tmem + (uint32_t)(g * NG);
-          // descriptors advance by plain additions to their address field: 2 (32 bytes) per K = 16
-          // inside a tile, one tile (8 KB of h, 4 KB of W) per 64 contraction indices
-          uint64_t da = a_desc0, db = b_desc0;
-          for (int q = 0; q < NQ && ok; ++q) {
-            ok = wait_or_fail(&full[g][q], (uint32_t)i & 1, &failed);
-            if (!ok) break;
-            tc_fence_after_sync();
-            const int nkb = (4 * q + 4 < KB) ? 4 : KB - 4 * q;
-            if (elect_one()) {
-              for (int kb = 0; kb < nkb; ++kb)
-                mma_f16_x4(d_tmem, da + (uint64_t)(kb * (A_TILE >> 4)), db + (uint64_t)(kb * (4096 >> 4)), idesc,
-                           (q > 0 || kb > 0) ? 1u : 0u);
-            }
-            __syncwarp();
-            da += 4 * (A_TILE >> 4);
-            db += 4 * (4096 >> 4);
-          }
-          if (elect_one()) mma_commit(&acc[g]);   // always: the epilogue counts on one arrival per (step, group)
-          __syncwarp();
+    constexpr uint32_t idesc = make_idesc(1, FG, FB, false, false);
+    bool ok = wait_or_fail(&wfull, 0, &failed);
+    const uint64_t w_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
+    const uint64_t h_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
+    for (int i = 0; i < a.n; ++i) {
+      // descriptors advance by plain additions to their address field: 2 (32 bytes) per K = 16
+      // inside a tile, one tile (8 KB of W, 4 KB of h) per 64 contraction indices
+      uint64_t dw = w_desc0, dh = h_desc0;
+      for (int q = 0; q < NQ && ok; ++q) {
+        ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int nkb = q ? KB - KB0 : KB0;   // part q of the split, into accumulator q
+        if (elect_one()) {
+          for (int kb = 0; kb < nkb; ++kb)
+            mma_f16_x4(tmem + (uint32_t)(q * FB), dw + (uint64_t)(kb * (W_TILE >> 4)), dh + (uint64_t)(kb * (H_TILE >> 4)),
+                       idesc, kb ? 1u : 0u);
         }
+        __syncwarp();
+        dw += (uint64_t)KB0 * (W_TILE >> 4);
+        dh += (uint64_t)KB0 * (H_TILE >> 4);
       }
+      if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
+      __syncwarp();
     }
   } else {
-    // ---- gates and state update: warp w owns tile rows 16w .. 16w+15 -------------------------
-    const int g = warp / (4 / GR);
-    const int rg = 16 * warp + lane - g * RG;          // row inside the group
-    const int b = g * Bg + rg;                          // batch row
-    const bool owner = lane < 16 && rg < Bg && b < a.B;
-    const int j0 = cta * NU;
+    // ---- gates and state update ------------------------------------------------------------------
+    // as a reader of TMEM: warp w, lanes 0 .. 15 hold accumulator rows (gate rows) 16 w .. 16 w + 15;
+    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of the CTA
+    const int zrow = 16 * warp + lane;
+    const int b = grp * FB + lane;                      // batch row
+    const int j0 = cta * FU + 4 * warp;                 // first hidden unit
+    const bool owner = b < a.B && j0 < a.H;
     const size_t e0 = (size_t)b * a.H + j0;             // element index of (b, j0) in a [B][H] array
-    const bool signaller = (warp % (4 / GR) == 0) && lane == 0;
-    float c[NU];
-    uint4 hprev = make_uint4(0, 0, 0, 0);
-    float zx[NG];
-    {
-      const DevOp op0 = a.ops[0];
-      if (owner) {
-        const float* cp = reinterpret_cast<const float*>(a.ws + (size_t)op0.c_src * 16) + e0;
-        const float4 c0 = *reinterpret_cast<const float4*>(cp), c1 = *reinterpret_cast<const float4*>(cp + 4);
-        c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
-        hprev = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op0.h_src * 16) + e0);
-        const float4* zp = reinterpret_cast<const float4*>(a.zx + (size_t)b * 4 * a.H + (size_t)cta * NG);
-#pragma unroll
-        for (int v = 0; v < NG / 4; ++v) {
-          const float4 z = zp[v];
-          zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
-        }
-      } else {
-#pragma unroll
-        for (int u = 0; u < NU; ++u) c[u] = 0.f;
-#pragma unroll
-        for (int v = 0; v < NG; ++v) zx[v] = 0.f;
-      }
-    }
+    const bool two = KB0 < KB;
+    FwdCell st;
+    fwd_cell_init(st, a, owner, b, j0, e0);
     for (int i = 0; i < a.n; ++i) {
       const DevOp op = a.ops[i];
-      const bool got = wait_or_fail(&acc[g], (uint32_t)i & 1, &failed);
+      const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
       tc_fence_after_sync();
-      uint32_t r[NG];
-      tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)(g * NG), r);
-      tmem_ld_wait();
-      uint4 hnew = make_uint4(0, 0, 0, 0);
-      uint32_t gi[4], gf[4], gg[4], go[4];
-      float cin[NU];
-      if (got && owner) {
-        uint32_t hq[4];
+      for (int h = 0; h < (two ? 2 : 1); ++h) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)(h * FB), r);
+        tmem_ld_wait();
+        if (lane < 16) {
+          float4* dst = reinterpret_cast<float4*>(part + ((size_t)h * FG + zrow) * PART_LD);
 #pragma unroll
-        for (int u = 0; u < NU; u += 2) {
-          float hv[2], iv[2], fv[2], gv[2], ov[2];
-#pragma unroll
-          for (int d = 0; d < 2; ++d) {
-            const int q = 4 * (u + d);
-            iv[d] = sigmoid_fast(__uint_as_float(r[q + 0]) + zx[q + 0]);
-            fv[d] = sigmoid_fast(__uint_as_float(r[q + 1]) + zx[q + 1]);
-            gv[d] = tanh_fast(__uint_as_float(r[q + 2]) + zx[q + 2]);
-            ov[d] = sigmoid_fast(__uint_as_float(r[q + 3]) + zx[q + 3]);
-            cin[u + d] = c[u + d];
-            c[u + d] = fmaf(fv[d], c[u + d], iv[d] * gv[d]);
-            hv[d] = ov[d] * tanh_fast(c[u + d]);
-          }
-          hq[u / 2] = pack_bf16x2(hv[0], hv[1]);
-          gi[u / 2] = pack_bf16x2(iv[0], iv[1]);
-          gf[u / 2] = pack_bf16x2(fv[0], fv[1]);
-          gg[u / 2] = pack_bf16x2(gv[0], gv[1]);
-          go[u / 2] = pack_bf16x2(ov[0], ov[1]);
+          for (int v = 0; v < FB / 4; ++v)
+            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                 __uint_as_float(r[4 * v + 3]));
         }
-        // h_k first: it is what the other CTAs wait for
-        hnew = make_uint4(hq[0], hq[1], hq[2], hq[3]);
-        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = hnew;
       }
       tc_fence_before_sync();
-      named_barrier(1 + g, TG);   // all of this CTA's h_k stores precede the release below
-      if (signaller) red_release_add(a.sync + g * 8, 1u);
+      named_barrier(1, 128);   // the accumulators of every gate row are in shared memory
+      FwdCellOut out;
       if (got && owner) {
-        // the rest of the state is not on the critical path of the recurrence
-        char* ws = a.ws;
-        float* cd = reinterpret_cast<float*>(ws + (size_t)op.c_dst * 16) + e0;
-        *reinterpret_cast<float4*>(cd) = make_float4(c[0], c[1], c[2], c[3]);
-        *reinterpret_cast<float4*>(cd + 4) = make_float4(c[4], c[5], c[6], c[7]);
-        if (op.gates) {
-          __nv_bfloat16* gp = reinterpret_cast<__nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
-          const size_t pl = (size_t)a.plane16 * 8;   // elements
-          *reinterpret_cast<uint4*>(gp) = make_uint4(gi[0], gi[1], gi[2], gi[3]);
-          *reinterpret_cast<uint4*>(gp + pl) = make_uint4(gf[0], gf[1], gf[2], gf[3]);
-          *reinterpret_cast<uint4*>(gp + 2 * pl) = make_uint4(gg[0], gg[1], gg[2], gg[3]);
-          *reinterpret_cast<uint4*>(gp + 3 * pl) = make_uint4(go[0], go[1], go[2], go[3]);
-        }
-        if (op.in_copy) {
-          char* blk = ws + (size_t)op.in_copy * 16;
-          *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(blk) + e0) = hprev;
-          float* ci = reinterpret_cast<float*>(blk + (size_t)a.hsz16 * 16) + e0;
-          *reinterpret_cast<float4*>(ci) = make_float4(cin[0], cin[1], cin[2], cin[3]);
-          *reinterpret_cast<float4*>(ci + 4) = make_float4(cin[4], cin[5], cin[6], cin[7]);
-        }
-        hprev = hnew;
-        // the input projection of the next step does not depend on the recurrence: fetch it now
-        if (i + 1 < a.n) {
-          const float4* zp = reinterpret_cast<const float4*>(a.zx + ((size_t)(i + 1) * a.B + b) * 4 * a.H + (size_t)cta * NG);
-#pragma unroll
-          for (int v = 0; v < NG / 4; ++v) {
-            const float4 z = zp[v];
-            zx[4 * v] = z.x; zx[4 * v + 1] = z.y; zx[4 * v + 2] = z.z; zx[4 * v + 3] = z.w;
-          }
-        }
+        float4 z[4];
+        fwd_cell_sum(st, part, two ? part + FG * PART_LD : nullptr, 16 * warp, lane, z);
+        fwd_cell_gates(st, z, out);
+        // h_k first: it is what the other CTAs wait for
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = out.hnew;
       }
+      named_barrier(1, 128);   // all of this CTA's h_k stores precede the release below; the parts are free again
+      if (tid == 0) red_release_add(sync, 1u);
+      if (got && owner) fwd_cell_rest(st, a, op, out, i, b, j0, e0);
     }
   }
 
@@ -333,9 +395,177 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   __syncthreads();
   if (tid == 0) {
     if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
-    else if (cta == 0) a.counters[0] += a.n;
+    else if (blockIdx.x == 0) a.counters[0] += a.n;
   }
-  if (warp == 4) tmem_dealloc(tmem, 32 * GR);
+  if (warp == 4) tmem_dealloc(tmem, 64);
+}
+
+// Clusters of two CTAs per 32 hidden units and group, each taking one half of the contraction.
+__global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_constant__ CUtensorMap tm_h,
+                                                              const __grid_constant__ CUtensorMap tm_w,
+                                                              const FwdRunArgs a) {
+  constexpr int PG = 2 * FG;              // gate rows of the pair: the M of the MMA
+  constexpr uint32_t W_TILE = PG * 128;   // [128 gate rows][64 contraction indices]
+  constexpr uint32_t H_TILE = FB * 128;   // [32 batch rows][64 contraction indices]
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t wfull, full[4], acc, pready;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int KB = (a.H + 63) / 64;          // 2 .. 16
+  const int KB0 = fwd_first_part_blocks(a.H);
+  const uint32_t rank = cluster_ctarank();
+  const int kb_lo = rank ? KB0 : 0;        // this CTA's blocks of the contraction index
+  const int nkb = rank ? KB - KB0 : KB0;   // 1 .. 8
+  uint8_t* sW = sm;                        // KB0 tiles: the pair's gate rows, this CTA's K blocks
+  uint8_t* tiles = sm + KB0 * W_TILE;      // KB0 tiles: the group's rows of h_{k-1}, this CTA's K blocks
+  const int NQ = (nkb + a.bb - 1) / a.bb;  // blocks of bb K tiles: one barrier and (slab mode) one copy each
+  float* part = reinterpret_cast<float*>(tiles + ((KB0 + a.bb - 1) / a.bb) * a.bb * H_TILE);   // [2 senders][FG][PART_LD]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int grp = blockIdx.x / a.ncg, pair = (blockIdx.x % a.ncg) >> 1;
+  uint32_t* const sync = a.sync + grp * SYNC_STRIDE;
+
+  if (tid == 0) {
+    mbar_init(&wfull, 1);
+    for (int s = 0; s < 4; ++s) mbar_init(&full[s], 1);
+    mbar_init(&acc, 1);
+    mbar_init(&pready, 2);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_h);
+    tma_prefetch_desc(&tm_w);
+  }
+  if (warp == 4) tmem_alloc(&tmem_slot, 32);
+  tc_fence_before_sync();
+  cluster_sync();                          // the neighbour arrives on this CTA's barrier: it must be initialised
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  const uint32_t row_bytes = (uint32_t)a.H * 2u;
+  grid_dep_wait();
+
+  if (warp == 4) {
+    // ---- producer ----------------------------------------------------------------------------
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&wfull, (uint32_t)nkb * W_TILE);
+      for (int kb = 0; kb < nkb; ++kb) tma_load_2d(sW + kb * W_TILE, &tm_w, (kb_lo + kb) * 64, pair * PG, &wfull);
+    }
+    int armed = -1;
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes) + grp * FB;
+      int go = 1;
+      if (lane == 0) go = (i == 0 || wait_counter(sync, (uint32_t)i * (uint32_t)a.ncg, &failed)) && !failed;
+      go = __shfl_sync(0xffffffffu, go, 0);
+      if (!go) continue;
+      if (a.slab) {
+        if (lane < NQ) {
+          fence_proxy_async_global();
+          mbar_arrive_expect_tx(&full[lane], (uint32_t)a.bb * H_TILE);   // a box counts in full
+          tma_load_3d(tiles + lane * a.bb * H_TILE, &tm_h, 0, row, kb_lo + lane * a.bb, &full[lane]);
+        }
+      } else if (lane < nkb) {
+        fence_proxy_async_global();
+        const int q = lane / a.bb;
+        if (lane == q * a.bb) mbar_arrive_expect_tx(&full[q], (uint32_t)((nkb - lane < a.bb) ? nkb - lane : a.bb) * H_TILE);
+        tma_load_2d(tiles + lane * H_TILE, &tm_h, (kb_lo + lane) * 64, row, &full[q]);
+      }
+      armed = i;
+      if (i == a.n - 1 && lane == 0) grid_dep_launch();
+      __syncwarp();
+    }
+    if (failed && lane == 0) {
+      (void)mbar_wait(&wfull, 0);
+      if (armed >= 0)
+        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
+    }
+  } else if (warp == 5) {
+    // ---- MMA issuer ----------------------------------------------------------------------------
+    constexpr uint32_t idesc = make_idesc(1, PG, FB, false, false);
+    bool ok = wait_or_fail(&wfull, 0, &failed);
+    const uint64_t w_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
+    const uint64_t h_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
+    for (int i = 0; i < a.n; ++i) {
+      uint64_t dw = w_desc0, dh = h_desc0;
+      for (int q = 0; q < NQ && ok; ++q) {
+        ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int cnt = ((q + 1) * a.bb <= nkb) ? a.bb : nkb - q * a.bb;
+        if (elect_one()) {
+          for (int kb = 0; kb < cnt; ++kb)
+            mma_f16_x4(tmem, dw + (uint64_t)(kb * (W_TILE >> 4)), dh + (uint64_t)(kb * (H_TILE >> 4)), idesc,
+                       (q > 0 || kb > 0) ? 1u : 0u);
+        }
+        __syncwarp();
+        dw += (uint64_t)a.bb * (W_TILE >> 4);
+        dh += (uint64_t)a.bb * (H_TILE >> 4);
+      }
+      if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
+      __syncwarp();
+    }
+  } else {
+    // ---- gates and state update ------------------------------------------------------------------
+    // as a reader of TMEM: thread (w, lane) holds gate row 32 w + lane of the pair's partial tile; rows
+    // 0 .. 63 belong to the units of CTA 0 of the pair, rows 64 .. 127 to those of CTA 1;
+    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of this CTA
+    const int prow = 32 * warp + lane;
+    const uint32_t row_owner = (uint32_t)(prow >> 6);
+    float* const send_to = part + ((size_t)rank * FG + (prow & 63)) * PART_LD;   // my slot as a sender, at the owner
+    const int b = grp * FB + lane;
+    const int j0 = pair * 2 * FU + (int)rank * FU + 4 * warp;
+    const bool owner = b < a.B && j0 < a.H;
+    const size_t e0 = (size_t)b * a.H + j0;
+    FwdCell st;
+    fwd_cell_init(st, a, owner, b, j0, e0);
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
+      tc_fence_after_sync();
+      {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int v = 0; v < FB / 4; ++v)
+          st_peer_f4(send_to + 4 * v, row_owner,
+                     make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                 __uint_as_float(r[4 * v + 3])));
+      }
+      tc_fence_before_sync();
+      named_barrier(1, 128);
+      if (tid < 2) mbar_arrive_peer(&pready, (uint32_t)tid);   // release: the stores above are visible to both CTAs
+      bool all = false;
+      for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait_cluster(&pready, (uint32_t)i & 1)) { all = true; break; }
+        if (spin > 256) {
+          if (failed) break;
+          __nanosleep(64);
+        }
+      }
+      if (!all) failed = 1;
+      FwdCellOut out;
+      const bool good = got && all && owner;
+      if (good) {
+        float4 z[4];
+        fwd_cell_sum(st, part, part + FG * PART_LD, 16 * warp, lane, z);
+        fwd_cell_gates(st, z, out);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = out.hnew;
+      }
+      named_barrier(1, 128);   // all of this CTA's h_k stores precede the release below; the parts are free again
+      if (tid == 0) red_release_add(sync, 1u);
+      if (good) fwd_cell_rest(st, a, op, out, i, b, j0, e0);
+    }
+  }
+
+  tc_fence_before_sync();
+  cluster_sync();   // no CTA leaves while its neighbour may still write into its shared memory or signal it
+  if (tid == 0) {
+    if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
+    else if (blockIdx.x == 0) a.counters[0] += a.n;
+  }
+  if (warp == 4) tmem_dealloc(tmem, 32);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1232,8 +1462,14 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   __nv_bfloat16* woutT = reinterpret_cast<__nv_bfloat16*>(at(y.off_woutT));
 
   const int KBh = (H + 63) / 64;
-  const int fwd_smem = KBh * 4096 + KBh * 64 * 128 + 1024;
-  const int GRf = 1;
+  const int KB0 = fwd_first_part_blocks(H);       // 64-wide blocks of the recurrent contraction in its first part
+  const int fwd_groups = B > FB ? 2 : 1;          // groups of CTAs that each own FB batch rows
+  int fwd_ncg = (H + FU - 1) / FU;                // CTAs per group
+  const int fwd_parts = KB0 < KBh ? 2 : 1;
+  int fwd_smem = (KBh * FG + fwd_parts * KB0 * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
+  bool fwd_pair = false;                          // clusters of two CTAs that split the contraction
+  bool fwd_slab = false;                          // h_{k-1} by one copy per part instead of one per K tile
+  int fwd_bb = KB0;                               // K tiles per barrier
   const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
   CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
@@ -1247,8 +1483,41 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     (void)attrs;
     // the whole workspace as rows of H bfloat16: any h block starts at a whole row
     const uint64_t rows = y.total / ((size_t)H * 2);
-    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, (uint32_t)(64 / GRf));
-    ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, NG);
+    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, FB);
+    ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, FG);
+    if (ok && KB0 < KBh) {
+      // the paired forward kernel, if the device can keep its clusters resident and
+      // MEBPTT_FWD_PAIR=1 in the environment asks for it (measured slower so far: the hand-over of
+      // the partial tiles between the two CTAs costs more than the halved contraction saves)
+      const char* force = getenv("MEBPTT_FWD_PAIR");
+      const int pairs = (H + 2 * FU - 1) / (2 * FU);
+      const int grid = fwd_groups * 2 * pairs;
+      const int bb = KB0 >= 4 ? (KB0 + 1) / 2 : KB0;   // two barriers per step where a half is long enough
+      const int smem = (KB0 * 2 * FG + ((KB0 + bb - 1) / bb) * bb * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
+      if (force && atoi(force) == 1) {
+        const void* fn = (const void*)fwd_run_pair_kernel;
+        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute at1[1];
+        at1[0].id = cudaLaunchAttributeClusterDimension;
+        at1[0].val.clusterDim.x = 2; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
+        cfg.attrs = at1; cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) cudaGetLastError();
+        else if (nclusters * 2 >= grid &&
+                 make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, 2 * FG)) {
+          fwd_pair = true; fwd_ncg = 2 * pairs; fwd_smem = smem; fwd_bb = bb;
+        }
+      }
+    }
+    if (ok && H % 64 == 0) {
+      CUtensorMap blocked;
+      if (make_tmap_blocks64(&blocked, ws, (uint64_t)H, rows, (uint64_t)H * 2, FB, (uint32_t)fwd_bb)) {
+        tm_h = blocked;
+        fwd_slab = true;
+      }
+    }
     for (int pb = 0; pb < 2; ++pb)
       ok = ok && make_tmap_2d(&tm_dz[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64,
                               (uint32_t)BM);
@@ -1380,12 +1649,12 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       }
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
-        FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 32, status,
-                     io.counters, B, H, off16(y.plane), off16(y.hsz)};
+        FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
+                     io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0, off16(y.plane), off16(y.hsz)};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
-        const void* fn = (const void*)fwd_run_kernel;
+        const void* fn = fwd_pair ? (const void*)fwd_run_pair_kernel : (const void*)fwd_run_kernel;
         const int span = span_begin(timer, 0, n, s);
-        if (!cuda_ok(launch_coop(fn, ncta, 192, fwd_smem, s, args, 1), "forward run launch"))
+        if (!cuda_ok(launch_coop(fn, fwd_groups * fwd_ncg, 192, fwd_smem, s, args, fwd_pair ? 2 : 1), "forward run launch"))
           rc = MEBPTT_ERR_CUDA;
         span_end(timer, span, s);
       }
@@ -1427,8 +1696,13 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k_lo - 1) * B * I;
         gemm(xk, I, false, wp_ih, I, false,
              GemmOut{GemmOut::STORE_F32, zleaf + (size_t)s_lo * B * G, G, bias_p, 0}, n * B, G, I);
+        // the recurrent part in the two parts the forward kernels sum it in, in their order
+        const int k_first = KB0 < KBh ? 64 * KB0 : H;
         gemm(hprev_c + (size_t)s_lo * B * H, H, false, wp_hh, H, false,
-             GemmOut{GemmOut::ACCUM_F32, zleaf + (size_t)s_lo * B * G, G, nullptr, 0}, n * B, G, H);
+             GemmOut{GemmOut::ACCUM_F32, zleaf + (size_t)s_lo * B * G, G, nullptr, 0}, n * B, G, k_first);
+        if (k_first < H)
+          gemm(hprev_c + (size_t)s_lo * B * H + k_first, H, false, wp_hh + k_first, H, false,
+               GemmOut{GemmOut::ACCUM_F32, zleaf + (size_t)s_lo * B * G, G, nullptr, 0}, n * B, G, H - k_first);
         ++launches;
         if (!dry && rc == MEBPTT_OK)
           launch_pdl(leaf_forward, dim3(32, n), dim3(256), 0, s, bops, n, ws, zleaf, hk_c, S, B, H, io.counters);
@@ -1453,7 +1727,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
-        BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 32, status,
+        BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
                      io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         const int span = span_begin(timer, 1, n, s);

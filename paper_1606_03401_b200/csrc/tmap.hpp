@@ -43,4 +43,24 @@ inline bool make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, uin
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same 2-D array of 2-byte elements seen as [cols / 64][rows][64]: coordinate 0 runs inside a
+// block of 64 columns (128 bytes), coordinate 1 over the rows, coordinate 2 over the blocks.  One
+// box of (64, box_rows, box_blocks) then lands in shared memory as box_blocks consecutive tiles
+// of [box_rows][128 B], 128-byte swizzled -- the layout a K-major MMA operand wants -- with a
+// single copy instruction.  cols must be a multiple of 64 (a partial last block would read on into
+// the next row instead of being zero-filled).
+inline bool make_tmap_blocks64(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows,
+                               uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_blocks) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || cols % 64 != 0 || box_blocks > 256 || box_rows > 256) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride_bytes & 15)) return false;
+  cuuint64_t gdim[3] = {64, rows, cols / 64};
+  cuuint64_t gstr[2] = {row_stride_bytes, 128};
+  cuuint32_t box[3] = {64, box_rows, box_blocks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace mebptt
