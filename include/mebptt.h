@@ -311,6 +311,24 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_
                                 float *dx, int64_t *counters);
 
 /*
+ * What a training step derives from (descriptor, plan, workspace address, device) alone -- the
+ * runs the tape of Algorithm 2 is cut into, the tape in the form the kernels read, the kernel
+ * variants the device can keep resident, the TMA tensor maps -- is prepared once and kept in a
+ * small cache inside the library (eight sets, least recently used out first); mebptt_plan_free
+ * drops the sets of its plan.  The first mebptt_lstm_train_step of a combination therefore costs
+ * some host time (page-locked memory is allocated for the tape); later ones only look the set up,
+ * copy the tape asynchronously and enqueue.  (The paper has no counterpart: its Algorithm 2
+ * walks the policy tables on the host at every step.)
+ *
+ * mebptt_lstm_prepare makes the host part of a set ahead of time, or finds it; it needs no GPU
+ * and returns a status.  mebptt_lstm_prepare_stats fills out[0..3] (host array) with: sets built
+ * since the library was loaded, look-ups served from the cache, sets whose tape lies in
+ * page-locked memory, sets held now.
+ */
+int mebptt_lstm_prepare(const mebptt_lstm_desc *desc, const mebptt_plan_t *plan);
+int mebptt_lstm_prepare_stats(int64_t *out);
+
+/*
  * The training step for callers that cannot allocate device memory.  (The paper has no
  * counterpart: it never says where the working memory of an implementation comes from.)
  *

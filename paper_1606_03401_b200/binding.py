@@ -84,6 +84,8 @@ _SIGS = {
     "mebptt_lstm_train_step_host": (_i32, _STEP_ARGS),
     "mebptt_lstm_train_step_static": (_i32, [_descp, _vp] + [_vp] * 8 + [_vp] + [_vp] * 7),
     "mebptt_lstm_run_times": (_i32, [C.POINTER(C.c_double), C.POINTER(_i64), C.POINTER(_i64)]),
+    "mebptt_lstm_prepare": (_i32, [_descp, _vp]),
+    "mebptt_lstm_prepare_stats": (_i32, [C.POINTER(_i64)]),
     "mebptt_slot_copy": (_i32, [_vp, _vp, _sz, _vp]),
     "mebptt_gemm_bf16": (_i32, [_vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "mebptt_strerror": (C.c_char_p, [_i32]),
@@ -280,6 +282,16 @@ def mebptt_lstm_train_step_static(desc, plan, W, b, W_out, b_out, x, targets, h0
         _ptr(h0), _ptr(c0), stream, _ptr(loss), _ptr(dW), _ptr(db), _ptr(dW_out), _ptr(db_out), _ptr(dx),
         _ptr(counters))
     _check(st, "mebptt_lstm_train_step_static")
+
+
+def mebptt_lstm_prepare(desc, plan) -> None:
+    _check(lib.mebptt_lstm_prepare(C.byref(desc), plan._h), "mebptt_lstm_prepare")
+
+
+def mebptt_lstm_prepare_stats() -> dict:
+    out = (_i64 * 4)()
+    _check(lib.mebptt_lstm_prepare_stats(out), "mebptt_lstm_prepare_stats")
+    return {"built": out[0], "reused": out[1], "page_locked": out[2], "held": out[3]}
 
 
 def mebptt_lstm_run_times() -> dict:

@@ -523,6 +523,7 @@ int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, con
             (const float*)b, (const float*)b_out, (const float*)targets, (const float*)c0,
             (char*)workspace, loss, dW, db, dW_out, db_out, dx, counters};
   io.time_runs = (desc->flags & MEBPTT_FLAG_TIME_RUNS) != 0;
+  io.pageable_tape = !side_stream;   // the allocation-free entry point (the only caller without side stream) locks no pages
   return run_step(desc, p, y, io, (cudaStream_t)stream, side_stream);
 }
 }  // namespace mebptt
@@ -605,6 +606,22 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
 }
 
 int mebptt_lstm_run_times(double* ms, int64_t* launches, int64_t* ops) { return tc::run_times(ms, launches, ops); }
+
+int mebptt_lstm_prepare(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
+  const int rc = check_common(desc, plan);
+  if (rc != MEBPTT_OK) return rc;
+  const Plan* p = reinterpret_cast<const Plan*>(plan);
+  Layout y;
+  workspace_layout(desc, p, y);
+  if (!y.tensor_path) return MEBPTT_OK;   // the other paths walk the plan's tape as it is
+  return tc::prepare_host(y, p, desc->want_dx != 0);
+}
+
+int mebptt_lstm_prepare_stats(int64_t* out) {
+  if (!out) return MEBPTT_ERR_ARG;
+  tc::prepare_stats(out);
+  return MEBPTT_OK;
+}
 
 int mebptt_gemm_bf16(const void* A, int64_t lda, int a_major, const void* B, int64_t ldb, int b_major, float* C,
                      int64_t ldc, int accumulate, const float* bias, int64_t M, int64_t N, int64_t K, int* status,

@@ -9,6 +9,7 @@
 namespace mebptt {
 
 struct Plan {
+  uint64_t id = 0;          // unique per plan object of the process (what cached per-plan data is keyed by)
   int64_t t = 0, m = 0;
   int mode = 0, alpha = 4, beta = 0;
   int64_t cost = 0;         // C(t, m)

@@ -16,6 +16,18 @@
 #include <thread>
 
 namespace mebptt {
+namespace tc { void forget_plan(uint64_t plan_id); }
+namespace {
+Plan* new_plan() {
+  static std::atomic<uint64_t> next_id{1};
+  Plan* p = new (std::nothrow) Plan();
+  if (p) p->id = next_id.fetch_add(1);
+  return p;
+}
+}  // namespace
+}  // namespace mebptt
+
+namespace mebptt {
 
 namespace {
 
@@ -452,7 +464,7 @@ int build_chen_plan(int64_t t, int alpha, int beta, Plan** out) {
   *out = nullptr;
   if (t < 1 || t > (int64_t)1 << 24) return MEBPTT_ERR_ARG;
   if (alpha < 2 || alpha > 64 || beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
-  Plan* p = new (std::nothrow) Plan();
+  Plan* p = new_plan();
   if (!p) return MEBPTT_ERR_OOM;
   p->t = t; p->mode = MEBPTT_CHEN_SQRT; p->alpha = alpha; p->beta = beta;
   try {
@@ -513,7 +525,7 @@ int build_chen_recursive_plan(int64_t t, int k, int alpha, int beta, Plan** out)
   *out = nullptr;
   if (t < 1 || t > (int64_t)1 << 24 || k < 1 || k > 4096) return MEBPTT_ERR_ARG;
   if (alpha < 2 || alpha > 64 || beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
-  Plan* p = new (std::nothrow) Plan();
+  Plan* p = new_plan();
   if (!p) return MEBPTT_ERR_OOM;
   p->t = t; p->mode = MEBPTT_CHEN_RECURSIVE; p->alpha = alpha; p->beta = beta;
   try {
@@ -602,7 +614,7 @@ int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out) 
   // beyond saturation more memory changes nothing
   const int64_t sat = (mode == MEBPTT_MSM) ? std::max<int64_t>(1, (int64_t)alpha * (t - 1) + 1) : t;
   m = std::min(m, sat);
-  Plan* p = new (std::nothrow) Plan();
+  Plan* p = new_plan();
   if (!p) return MEBPTT_ERR_OOM;
   p->t = t; p->m = m; p->mode = mode; p->alpha = alpha; p->beta = beta;
   try {
@@ -715,7 +727,11 @@ int mebptt_plan_ex(int64_t t, int64_t m, int mode, int alpha, int beta, mebptt_p
   return mebptt::build_plan(t, m, mode, alpha, beta, reinterpret_cast<Plan**>(out));
 }
 
-void mebptt_plan_free(mebptt_plan_t* plan) { delete reinterpret_cast<Plan*>(plan); }
+void mebptt_plan_free(mebptt_plan_t* plan) {
+  if (!plan) return;
+  mebptt::tc::forget_plan(reinterpret_cast<Plan*>(plan)->id);   // what the executor prepared for this plan goes with it
+  delete reinterpret_cast<Plan*>(plan);
+}
 
 #define P_(x) (reinterpret_cast<const Plan*>(x))
 int64_t mebptt_plan_cost(const mebptt_plan_t* plan) { return plan ? P_(plan)->cost : -1; }

@@ -47,6 +47,9 @@ struct StepPtrs {
   size_t x_bytes = 0;
   // bracket every launch of the two persistent kernels with CUDA events (collected by run_times)
   bool time_runs = false;
+  // keep the host copy of the tape in pageable memory (the allocation-free entry point: page-locking
+  // memory is an allocation too); its upload may then hold up the calling thread
+  bool pageable_tape = false;
 };
 
 // Scratch for contractions that are split along K: a product with few output tiles and a long
@@ -111,6 +114,14 @@ namespace tc {
 int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
                  bool side_stream);
 
+
+// The prepared sets (work items, device tape, kernel variants, tensor maps) that run_step keeps per
+// (problem, plan, workspace, device).  forget_plan drops those of a plan that is being freed;
+// prepare_host makes (or finds) the host part only and returns its status; prepare_stats fills
+// out[0..3] with sets built, sets reused, sets with a page-locked tape, sets held.
+void forget_plan(uint64_t plan_id);
+int prepare_host(const Layout& y, const Plan* p, bool want_dx);
+void prepare_stats(int64_t* out);
 
 // Waits for the event pairs recorded on the current device by steps run with time_runs, adds up
 // elapsed milliseconds, launches and operations per class (0: forward runs, 1: backward runs)

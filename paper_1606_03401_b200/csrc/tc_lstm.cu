@@ -32,8 +32,11 @@
 // the backward pass has completed a chunk of S steps aligned to absolute time -- the weight
 // gradients.  Chunks are tied to time indices, not to run boundaries, and backward steps always
 // come in the order t .. 1, so every sum runs in the same order under every plan.
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
+#include <memory>
 #include <mutex>
 #include <vector>
 
@@ -146,6 +149,12 @@ struct FwdRunArgs {
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
 };
 
+// The exchange ring of the paired kernel (described there): value of an empty word, slots, rows per slot.
+constexpr uint32_t XR_EMPTY = 0xffffffffu;
+constexpr int XR_SLOTS = 4;
+constexpr int XR_ROWS = 2 * FB;
+__device__ __forceinline__ uint32_t xr_word(uint32_t w) { return w == XR_EMPTY ? 0x7fff7fffu : w; }
+
 // 64-wide blocks of the contraction index in the first part of the split (all of them if there is one)
 __host__ __device__ inline int fwd_first_part_blocks(int H) {
   const int KB = (H + 63) / 64;
@@ -189,7 +198,9 @@ __device__ __forceinline__ void fwd_cell_gates(FwdCell& st, const float4 (&z)[4]
     st.c[u] = fmaf(fv[u], st.c[u], iv[u] * gv[u]);
     hv[u] = ov[u] * tanh_fast(st.c[u]);
   }
-  o.hnew = make_uint2(pack_bf16x2(hv[0], hv[1]), pack_bf16x2(hv[2], hv[3]));
+  // (a pair of NaNs with every payload bit set is what an empty word of the exchange ring of the
+  // paired kernel holds: such a result is written as the canonical NaN pair by both kernels)
+  o.hnew = make_uint2(xr_word(pack_bf16x2(hv[0], hv[1])), xr_word(pack_bf16x2(hv[2], hv[3])));
   o.gi = make_uint2(pack_bf16x2(iv[0], iv[1]), pack_bf16x2(iv[2], iv[3]));
   o.gf = make_uint2(pack_bf16x2(fv[0], fv[1]), pack_bf16x2(fv[2], fv[3]));
   o.gg = make_uint2(pack_bf16x2(gv[0], gv[1]), pack_bf16x2(gv[2], gv[3]));
@@ -401,16 +412,45 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
 }
 
 // Clusters of two CTAs per 32 hidden units and group, each taking one half of the contraction.
-__global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_constant__ CUtensorMap tm_h,
-                                                              const __grid_constant__ CUtensorMap tm_w,
-                                                              const FwdRunArgs a) {
+//
+// How h_k travels.  A grid-wide counter (stores, release, poll with acquire, then a TMA fetch) puts
+// four dependent trips through the L2 on every step: measured 1.5 us for the signalling round of 128
+// CTAs alone.  Here h_k is its own signal.  Besides writing h_k where the tape says, every thread
+// writes it (strong, relaxed stores) into a ring of four exchange slots, [64 batch rows][H] each,
+// whose words hold an impossible value until then -- 0xffffffff, two bfloat16 NaNs with all payload
+// bits set; a value the arithmetic produces is rewritten if it collides.  The consumers read their
+// rows and columns of the slot with strong loads straight into registers, take every 16-byte piece
+// that holds no such word, put it into shared memory in the 128-byte swizzled tile layout, and ask
+// again only for what was not there yet.  One trip of the data through the L2 instead of four.
+//   Slot (i mod 4) is written at step i, read at step i + 1 and put back to the impossible value by
+// its writers at step i + 2, which is safe (who produces at step i + 2 has read all of h_{i+1}, so
+// everybody has finished reading h_i) and two steps ahead of the next writing.  That a reader of
+// step i + 5 cannot meet the words of step i any more is not left to the two steps in between: the
+// grid-wide counter is kept, off the critical path -- a spare warp signals (release) after the
+// stores of each step and acquires, for a step s, the signals of step s - 3 before the readers of
+// step s start.  Only the first exchange of a launch, which follows the initial clearing of the
+// ring, waits for the counter on the critical path.
+//
+// The partial tiles change hands between the two CTAs by asynchronous stores into (distributed)
+// shared memory that count their bytes on a barrier of the receiver.
+
+struct FwdPairArgs {
+  FwdRunArgs r;
+  __nv_bfloat16* xring;  // [XR_SLOTS][XR_ROWS][H]
+};
+
+__global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_constant__ CUtensorMap tm_w,
+                                                              const FwdPairArgs pa) {
+  const FwdRunArgs& a = pa.r;
   constexpr int PG = 2 * FG;              // gate rows of the pair: the M of the MMA
   constexpr uint32_t W_TILE = PG * 128;   // [128 gate rows][64 contraction indices]
   constexpr uint32_t H_TILE = FB * 128;   // [32 batch rows][64 contraction indices]
+  constexpr int MAXLD = 16;               // 16-byte pieces of h_{k-1} per thread and step: 8 rows x 2 (8 K tiles of 8 pieces / 32 lanes)
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[4], acc, pready;
+  __shared__ uint64_t wfull, full[2], acc, pready;
   __shared__ uint32_t tmem_slot;
   __shared__ int failed;
+  __shared__ volatile int lag_ok;          // readers of local step s may start once lag_ok >= s
 
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int KB = (a.H + 63) / 64;          // 2 .. 16
@@ -418,68 +458,61 @@ __global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_const
   const uint32_t rank = cluster_ctarank();
   const int kb_lo = rank ? KB0 : 0;        // this CTA's blocks of the contraction index
   const int nkb = rank ? KB - KB0 : KB0;   // 1 .. 8
+  const int nkb_a = (nkb + 1) / 2;         // K tiles behind the first of the two barriers
   uint8_t* sW = sm;                        // KB0 tiles: the pair's gate rows, this CTA's K blocks
   uint8_t* tiles = sm + KB0 * W_TILE;      // KB0 tiles: the group's rows of h_{k-1}, this CTA's K blocks
-  const int NQ = (nkb + a.bb - 1) / a.bb;  // blocks of bb K tiles: one barrier and (slab mode) one copy each
-  float* part = reinterpret_cast<float*>(tiles + ((KB0 + a.bb - 1) / a.bb) * a.bb * H_TILE);   // [2 senders][FG][PART_LD]
+  float* part = reinterpret_cast<float*>(tiles + KB0 * H_TILE);   // [2 senders][FG][PART_LD]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int grp = blockIdx.x / a.ncg, pair = (blockIdx.x % a.ncg) >> 1;
   uint32_t* const sync = a.sync + grp * SYNC_STRIDE;
+  const int rows_g = (a.B - grp * FB < FB) ? a.B - grp * FB : FB;   // batch rows of this group
 
   if (tid == 0) {
     mbar_init(&wfull, 1);
-    for (int s = 0; s < 4; ++s) mbar_init(&full[s], 1);
+    mbar_init(&full[0], 4);                // one arrival per epilogue warp
+    mbar_init(&full[1], 4);
     mbar_init(&acc, 1);
-    mbar_init(&pready, 2);
+    mbar_init(&pready, 1);
     failed = 0;
+    lag_ok = 0;
     mbar_fence_init();
-    tma_prefetch_desc(&tm_h);
     tma_prefetch_desc(&tm_w);
   }
+  // rows past the batch and columns past H are never fetched: they stay zero
+  for (int e = tid; e < KB0 * (int)H_TILE / 16; e += 192) reinterpret_cast<uint4*>(tiles)[e] = make_uint4(0, 0, 0, 0);
   if (warp == 4) tmem_alloc(&tmem_slot, 32);
+  fence_proxy_async();
   tc_fence_before_sync();
-  cluster_sync();                          // the neighbour arrives on this CTA's barrier: it must be initialised
+  cluster_sync();                          // the neighbour signals this CTA's barrier: it must be initialised
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
-  const uint32_t row_bytes = (uint32_t)a.H * 2u;
   grid_dep_wait();
 
   if (warp == 4) {
-    // ---- producer ----------------------------------------------------------------------------
+    // ---- W_hh, then the counter: signal each step once its stores are out, and keep the readers'
+    // licence (lag_ok) ahead of them ---------------------------------------------------------------
     if (lane == 0) {
       mbar_arrive_expect_tx(&wfull, (uint32_t)nkb * W_TILE);
       for (int kb = 0; kb < nkb; ++kb) tma_load_2d(sW + kb * W_TILE, &tm_w, (kb_lo + kb) * 64, pair * PG, &wfull);
     }
-    int armed = -1;
     for (int i = 0; i < a.n; ++i) {
-      const DevOp op = a.ops[i];
-      const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes) + grp * FB;
-      int go = 1;
-      if (lane == 0) go = (i == 0 || wait_counter(sync, (uint32_t)i * (uint32_t)a.ncg, &failed)) && !failed;
-      go = __shfl_sync(0xffffffffu, go, 0);
-      if (!go) continue;
-      if (a.slab) {
-        if (lane < NQ) {
-          fence_proxy_async_global();
-          mbar_arrive_expect_tx(&full[lane], (uint32_t)a.bb * H_TILE);   // a box counts in full
-          tma_load_3d(tiles + lane * a.bb * H_TILE, &tm_h, 0, row, kb_lo + lane * a.bb, &full[lane]);
+      named_barrier(2, 160);               // the epilogue threads' stores of step i (arrive) precede the release
+      if (lane == 0) {
+        red_release_add(sync, 1u);
+        if (i + 1 < a.n) {
+          // the readers of local step s want the signals of step max(0, s - 3): once those of step
+          // max(0, i - 1) are in, the readers of steps up to i + 2 may go -- long before they get there,
+          // except for the first exchange of the launch
+          const uint32_t need = (uint32_t)(i > 1 ? i : 1) * (uint32_t)a.ncg;
+          if (wait_counter(sync, need, &failed) && !failed)
+            asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32((const void*)&lag_ok)), "r"(i + 2) : "memory");
         }
-      } else if (lane < nkb) {
-        fence_proxy_async_global();
-        const int q = lane / a.bb;
-        if (lane == q * a.bb) mbar_arrive_expect_tx(&full[q], (uint32_t)((nkb - lane < a.bb) ? nkb - lane : a.bb) * H_TILE);
-        tma_load_2d(tiles + lane * H_TILE, &tm_h, (kb_lo + lane) * 64, row, &full[q]);
+        if (i + 2 == a.n || a.n == 1) grid_dep_launch();   // last step under way: the next kernel may set itself up
       }
-      armed = i;
-      if (i == a.n - 1 && lane == 0) grid_dep_launch();
       __syncwarp();
     }
-    if (failed && lane == 0) {
-      (void)mbar_wait(&wfull, 0);
-      if (armed >= 0)
-        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
-    }
+    if (failed && lane == 0) (void)mbar_wait(&wfull, 0);
   } else if (warp == 5) {
     // ---- MMA issuer ----------------------------------------------------------------------------
     constexpr uint32_t idesc = make_idesc(1, PG, FB, false, false);
@@ -488,60 +521,126 @@ __global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_const
     const uint64_t h_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
     for (int i = 0; i < a.n; ++i) {
       uint64_t dw = w_desc0, dh = h_desc0;
-      for (int q = 0; q < NQ && ok; ++q) {
+      for (int q = 0; q < 2 && ok; ++q) {
         ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
         if (!ok) break;
         tc_fence_after_sync();
-        const int cnt = ((q + 1) * a.bb <= nkb) ? a.bb : nkb - q * a.bb;
+        const int cnt = q ? nkb - nkb_a : nkb_a;
         if (elect_one()) {
           for (int kb = 0; kb < cnt; ++kb)
             mma_f16_x4(tmem, dw + (uint64_t)(kb * (W_TILE >> 4)), dh + (uint64_t)(kb * (H_TILE >> 4)), idesc,
                        (q > 0 || kb > 0) ? 1u : 0u);
         }
         __syncwarp();
-        dw += (uint64_t)a.bb * (W_TILE >> 4);
-        dh += (uint64_t)a.bb * (H_TILE >> 4);
+        dw += (uint64_t)nkb_a * (W_TILE >> 4);
+        dh += (uint64_t)nkb_a * (H_TILE >> 4);
       }
       if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
       __syncwarp();
     }
   } else {
-    // ---- gates and state update ------------------------------------------------------------------
+    // ---- epilogue warps: fetch h_{k-1}, then gates and state update ------------------------------
     // as a reader of TMEM: thread (w, lane) holds gate row 32 w + lane of the pair's partial tile; rows
     // 0 .. 63 belong to the units of CTA 0 of the pair, rows 64 .. 127 to those of CTA 1;
-    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of this CTA
+    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of this CTA;
+    // as a reader of h_{k-1}: batch rows 8 w .. 8 w + 7 of the group, 16-byte piece `lane` of every
+    // run of four K tiles (512 bytes of a row)
     const int prow = 32 * warp + lane;
     const uint32_t row_owner = (uint32_t)(prow >> 6);
-    float* const send_to = part + ((size_t)rank * FG + (prow & 63)) * PART_LD;   // my slot as a sender, at the owner
+    const uint32_t send_addr = peer_smem_u32(part + ((size_t)rank * FG + (prow & 63)) * PART_LD, row_owner);
+    const uint32_t send_bar = peer_smem_u32(&pready, row_owner);
     const int b = grp * FB + lane;
     const int j0 = pair * 2 * FU + (int)rank * FU + 4 * warp;
     const bool owner = b < a.B && j0 < a.H;
     const size_t e0 = (size_t)b * a.H + j0;
+    const size_t xr_slot = (size_t)XR_ROWS * a.H;          // elements per exchange slot
     FwdCell st;
     fwd_cell_init(st, a, owner, b, j0, e0);
+    if (owner) {
+      // the ring starts empty (the first signal of every CTA, which the readers of step 1 wait for,
+      // comes after these stores)
+#pragma unroll
+      for (int sl = 0; sl < XR_SLOTS; ++sl) st_relaxed_u2(pa.xring + sl * xr_slot + e0, make_uint2(XR_EMPTY, XR_EMPTY));
+    }
+    // what this thread fetches: piece p (0 .. 8 lpr - 1) is row 8 w + p / lpr, K tile 4 (p % lpr) + lane / 8,
+    // 16-byte column lane % 8 of that tile; lpr = loads per row = 1 or 2 (up to 8 K tiles of 8 pieces
+    // for 32 lanes).  Which pieces exist, and which lie behind the first barrier, never changes.
+    const int ls = nkb > 4 ? 1 : 0;                          // log2(lpr)
+    const int c8 = lane & 7, kq = lane >> 3;
+    uint32_t pieces = 0, first_half = 0;
+    for (int p = 0; p < (8 << ls); ++p) {
+      const int row = 8 * warp + (p >> ls), kb = 4 * (p & ls) + kq;
+      if (row < rows_g && kb < nkb && (kb_lo + kb) * 64 + c8 * 8 < a.H) {
+        pieces |= 1u << p;
+        if (kb < nkb_a) first_half |= 1u << p;
+      }
+    }
+    const size_t g_off0 = (size_t)(grp * FB + 8 * warp) * a.H + (size_t)(kb_lo + kq) * 64 + c8 * 8;   // piece 0, in elements
     for (int i = 0; i < a.n; ++i) {
       const DevOp op = a.ops[i];
+      // ---- h_{k-1}: from where the tape says at the first step (written before this launch), from
+      // the ring afterwards -------------------------------------------------------------------------
+      {
+        const __nv_bfloat16* src = ((i == 0) ? reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op.h_src * 16)
+                                             : pa.xring + (size_t)((i - 1) % XR_SLOTS) * xr_slot) + g_off0;
+        if (i > 0) {
+          bool lic = false;
+          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+            int seen;
+            asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(seen) : "r"(smem_u32((const void*)&lag_ok)) : "memory");
+            if (seen >= i) { lic = true; break; }
+            if (spin > 64 && failed) break;
+          }
+          if (!lic) failed = 1;
+        }
+        for (int half = 0; half < 2; ++half) {
+          // first the pieces of the K tiles behind the first barrier, then the rest
+          uint32_t want = half ? (pieces & ~first_half) : first_half;
+          for (uint32_t round = 0; want != 0 && !failed; ++round) {
+            if (round >= (kSpinLimit >> 4)) { failed = 1; break; }
+            if (round > 0) __nanosleep(100);   // what was not there yet: ask again, but leave the L2 to the writers
+            uint4 v[MAXLD];
+#pragma unroll
+            for (int p = 0; p < MAXLD; ++p)
+              if (want >> p & 1u) v[p] = ld_relaxed_u4(src + (size_t)(p >> ls) * a.H + (p & ls) * 256);
+#pragma unroll
+            for (int p = 0; p < MAXLD; ++p) {
+              if (want >> p & 1u) {
+                const uint4 w = v[p];
+                if (i == 0 || (w.x != XR_EMPTY && w.y != XR_EMPTY && w.z != XR_EMPTY && w.w != XR_EMPTY)) {
+                  const int row = 8 * warp + (p >> ls), kb = 4 * (p & ls) + kq;
+                  *reinterpret_cast<uint4*>(tiles + kb * H_TILE + row * 128 + ((c8 ^ (row & 7)) << 4)) = w;
+                  want &= ~(1u << p);
+                }
+              }
+            }
+          }
+          fence_proxy_async_smem();        // the tiles are read by the tensor core through the async proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full[half]);
+        }
+      }
+      // ---- the pair's partial tile: every gate row to the CTA that owns its unit -------------------
       const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
       tc_fence_after_sync();
+      if (tid == 0) mbar_arrive_expect_tx(&pready, 2u * FG * FB * 4u);   // 64 rows of 32 floats from each of the two CTAs
       {
         uint32_t r[32];
         tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
         tmem_ld_wait();
 #pragma unroll
         for (int v = 0; v < FB / 4; ++v)
-          st_peer_f4(send_to + 4 * v, row_owner,
-                     make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                                 __uint_as_float(r[4 * v + 3])));
+          st_async_f4(send_addr + 16u * v, send_bar,
+                      make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                  __uint_as_float(r[4 * v + 3])));
       }
       tc_fence_before_sync();
-      named_barrier(1, 128);
-      if (tid < 2) mbar_arrive_peer(&pready, (uint32_t)tid);   // release: the stores above are visible to both CTAs
       bool all = false;
       for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
         if (mbar_try_wait_cluster(&pready, (uint32_t)i & 1)) { all = true; break; }
         if (spin > 256) {
           if (failed) break;
-          __nanosleep(64);
+          __nanosleep(32);
         }
       }
       if (!all) failed = 1;
@@ -551,11 +650,13 @@ __global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_const
         float4 z[4];
         fwd_cell_sum(st, part, part + FG * PART_LD, 16 * warp, lane, z);
         fwd_cell_gates(st, z, out);
+        // h_k into the ring first: it is what the other CTAs wait for
+        if (i + 1 < a.n) st_relaxed_u2(pa.xring + (size_t)(i % XR_SLOTS) * xr_slot + e0, out.hnew);
         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = out.hnew;
+        if (i + 2 < a.n) st_relaxed_u2(pa.xring + (size_t)((i + 2) % XR_SLOTS) * xr_slot + e0, make_uint2(XR_EMPTY, XR_EMPTY));
+        fwd_cell_rest(st, a, op, out, i, b, j0, e0);
       }
-      named_barrier(1, 128);   // all of this CTA's h_k stores precede the release below; the parts are free again
-      if (tid == 0) red_release_add(sync, 1u);
-      if (good) fwd_cell_rest(st, a, op, out, i, b, j0, e0);
+      named_barrier_arrive(2, 160);        // the spare warp signals once every epilogue thread is here
     }
   }
 
@@ -1384,16 +1485,52 @@ LateCopies start_late_copies(const StepPtrs& io, int64_t t, cudaStream_t s) {
   return lc;
 }
 
-int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
-                 bool side_stream) {
-  const int B = y.B, H = y.H, I = y.I, O = y.O, S = y.S, G = 4 * H, K = I + H;
-  const int BM = 64;  // batch rows per MMA tile (B <= 64)
-  const int ncta = H / NU;
-  int64_t launches = 0;
-  char* ws = io.ws;
-  auto at = [&](size_t off) { return ws + off; };
+// ------------------------------------------------------------------------------------------
+// What a step needs besides the caller's pointers, prepared once and kept
+// ------------------------------------------------------------------------------------------
+// Everything here follows from the descriptor, the plan and the workspace address alone: the work
+// items the tape is cut into, where each forward run finds its input projections, the tape as the
+// kernels read it (in page-locked host memory, so that its upload is an asynchronous copy that
+// does not hold up the calling thread), the kernel variants the device can keep resident and the
+// tensor maps.  A step looks its set up in a small cache, most recently used first; freeing a
+// plan drops the entries made for it.
+struct Prepared {
+  // key
+  uint64_t plan_id = 0;
+  int I = 0, H = 0, O = 0, B = 0;
+  int64_t t = 0;
+  bool want_dx = false;
+  char* ws = nullptr;      // nullptr: host part only (no tensor maps)
+  int device = -1;
+  // host part
+  std::vector<WorkItem> items;
+  std::vector<int> zx_hi;  // per item: a forward run that projects its inputs anew does so up to this step (exclusive); 0: the window in place serves it
+  DevOp* tape = nullptr;   // [2 nops]: the tape, then the compacted leaves of leaf batches
+  size_t tape_entries = 0;
+  bool pinned = false;
+  // device part
+  CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
+  int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
+  int fwd_ncg = 0, fwd_smem = 0, fwd_bb = 0;
+  bool fwd_pair = false, fwd_slab = false;
+  int rc = MEBPTT_OK;
 
-  // ---- tape -> device operations -------------------------------------------------------------
+  Prepared() = default;
+  Prepared(const Prepared&) = delete;
+  Prepared& operator=(const Prepared&) = delete;
+  ~Prepared() {
+    if (tape && pinned) cudaFreeHost(tape);
+    else if (tape) free(tape);
+  }
+};
+
+namespace {
+std::mutex g_prep_mu;
+std::vector<std::shared_ptr<Prepared>> g_prep;     // most recently used first
+constexpr size_t kPrepCapacity = 8;
+std::atomic<int64_t> g_prep_stats[3];               // sets built, sets reused, sets whose tape lies in page-locked memory
+
+void build_host_part(Prepared& P, const Layout& y, const Plan* p, bool allow_pinned) {
   auto block_off = [&](int32_t loc) -> size_t {
     switch (loc) {
       case MEBPTT_LOC_INIT: return y.off_init;
@@ -1403,43 +1540,241 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       default: return y.off_arena + (size_t)loc * y.unit;
     }
   };
+  const int S = y.S;
   const size_t nops = p->tape.size();
-  const std::vector<WorkItem> items = work_items(p, S);
-  std::vector<DevOp> dev;
-  if (!dry) {
-    dev.resize(2 * nops);   // [0, nops): the tape; [nops, 2 nops): the compacted leaves of leaf batches
-    for (size_t i = 0; i < nops; ++i) {
-      const mebptt_op& op = p->tape[i];
-      DevOp d{};
-      d.k = op.k;
-      d.fmt = op.dst_fmt;
-      if (op.kind == MEBPTT_OP_FWD) {
-        const size_t src = block_off(op.src), dst = block_off(op.dst);
-        d.h_src = off16(src); d.c_src = off16(src + y.hsz);
-        d.h_dst = off16(dst); d.c_dst = off16(dst + y.hsz);
-        d.gates = (op.dst_fmt != MEBPTT_FMT_HIDDEN) ? off16(dst + y.rec_gates) : 0;
-        d.in_copy = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? off16(dst + y.rec_in) : 0;
-      } else {
-        const size_t rec = block_off(op.src);
-        const size_t prev = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? rec + y.rec_in : block_off(op.aux);
-        d.h_dst = off16(rec); d.c_dst = off16(rec + y.hsz);
-        d.h_src = off16(prev); d.c_src = off16(prev + y.hsz);
-        d.gates = off16(rec + y.rec_gates);
-      }
-      dev[i] = d;
+  P.items = work_items(p, S);
+  // Input projections Zx: computed for the S steps from the start of a forward run on, unless the
+  // buffer already holds them: recomputation sweeps keep returning to the same stored state, so one
+  // projection serves many short runs.  (The values do not depend on how steps are batched.)  The
+  // tape is known, so the window ends where the last run that will still find its steps in it ends
+  // (the first forward run that does not fit in the S steps from the window's start on replaces it).
+  P.zx_hi.assign(P.items.size(), 0);
+  int zx_lo = 0, zx_hi = 0;
+  for (size_t item = 0; item < P.items.size(); ++item) {
+    const WorkItem& wi = P.items[item];
+    if (wi.kind != WorkItem::FWD) continue;
+    const int k0 = p->tape[wi.i].k, n = wi.n;
+    if (k0 >= zx_lo && k0 + n <= zx_hi) continue;
+    zx_lo = k0;
+    const int cap = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
+    zx_hi = k0 + n;
+    for (size_t j = item + 1; j < P.items.size(); ++j) {
+      if (P.items[j].kind != WorkItem::FWD) continue;
+      const int kj = p->tape[P.items[j].i].k, ej = kj + P.items[j].n;
+      if (kj < k0 || ej > cap) break;
+      if (ej > zx_hi) zx_hi = ej;
     }
-    for (const WorkItem& it : items) {
-      if (it.kind != WorkItem::LEAF) continue;
-      for (int j = 0; j < it.n; ++j) {
-        const mebptt_op& f = p->tape[it.i + 2 * (size_t)j];   // the leaf's forward operation
-        const size_t src = block_off(f.src);
-        DevOp d{};
-        d.k = f.k;
-        d.h_src = off16(src); d.c_src = off16(src + y.hsz);   // state k-1, memorised
-        dev[nops + it.i + (size_t)j] = d;
+    P.zx_hi[item] = zx_hi;
+  }
+  // the tape as the kernels read it
+  P.tape_entries = 2 * nops;
+  const size_t bytes = (P.tape_entries ? P.tape_entries : 1) * sizeof(DevOp);
+  void* mem = nullptr;
+  if (allow_pinned && cudaHostAlloc(&mem, bytes, cudaHostAllocDefault) == cudaSuccess) {
+    P.pinned = true;
+  } else {
+    if (allow_pinned) cudaGetLastError();
+    mem = malloc(bytes);
+  }
+  P.tape = static_cast<DevOp*>(mem);
+  if (!P.tape) { P.rc = MEBPTT_ERR_OOM; return; }
+  memset(P.tape, 0, bytes);
+  for (size_t i = 0; i < nops; ++i) {
+    const mebptt_op& op = p->tape[i];
+    DevOp d{};
+    d.k = op.k;
+    d.fmt = op.dst_fmt;
+    if (op.kind == MEBPTT_OP_FWD) {
+      const size_t src = block_off(op.src), dst = block_off(op.dst);
+      d.h_src = off16(src); d.c_src = off16(src + y.hsz);
+      d.h_dst = off16(dst); d.c_dst = off16(dst + y.hsz);
+      d.gates = (op.dst_fmt != MEBPTT_FMT_HIDDEN) ? off16(dst + y.rec_gates) : 0;
+      d.in_copy = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? off16(dst + y.rec_in) : 0;
+    } else {
+      const size_t rec = block_off(op.src);
+      const size_t prev = (op.dst_fmt == MEBPTT_FMT_INTERNAL) ? rec + y.rec_in : block_off(op.aux);
+      d.h_dst = off16(rec); d.c_dst = off16(rec + y.hsz);
+      d.h_src = off16(prev); d.c_src = off16(prev + y.hsz);
+      d.gates = off16(rec + y.rec_gates);
+    }
+    P.tape[i] = d;
+  }
+  for (const WorkItem& it : P.items) {
+    if (it.kind != WorkItem::LEAF) continue;
+    for (int j = 0; j < it.n; ++j) {
+      const mebptt_op& f = p->tape[it.i + 2 * (size_t)j];   // the leaf's forward operation
+      const size_t src = block_off(f.src);
+      DevOp d{};
+      d.k = f.k;
+      d.h_src = off16(src); d.c_src = off16(src + y.hsz);   // state k-1, memorised
+      P.tape[nops + it.i + (size_t)j] = d;
+    }
+  }
+}
+
+// Kernel variants and tensor maps for the workspace at `ws` on the current device.
+void build_device_part(Prepared& P, const Layout& y, char* ws) {
+  const int B = y.B, H = y.H, S = y.S, G = 4 * H;
+  const int BM = 64;  // batch rows per MMA tile (B <= 64)
+  const int ncta = H / NU;
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + y.off_dz);
+  __nv_bfloat16* wp_hh = reinterpret_cast<__nv_bfloat16*>(ws + y.off_wp_hh);
+  __nv_bfloat16* wpT_hh = reinterpret_cast<__nv_bfloat16*>(ws + y.off_wpT_hh);
+  const int KBh = (H + 63) / 64;
+  const int KB0 = fwd_first_part_blocks(H);       // 64-wide blocks of the recurrent contraction in its first part
+  const int fwd_groups = B > FB ? 2 : 1;          // groups of CTAs that each own FB batch rows
+  const int fwd_parts = KB0 < KBh ? 2 : 1;
+  P.fwd_ncg = (H + FU - 1) / FU;                  // CTAs per group
+  P.fwd_smem = (KBh * FG + fwd_parts * KB0 * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
+  P.fwd_pair = false;                             // clusters of two CTAs that split the contraction
+  P.fwd_slab = false;                             // h_{k-1} by one copy per part instead of one per K tile
+  P.fwd_bb = KB0;                                 // K tiles per barrier
+  P.bwd_cs = 0; P.bwdc_smem = 0;
+  {
+    // function attributes belong to the device that is current
+    const int big = 220 * 1024;  // the kernels also hold a few static barriers
+    cudaFuncSetAttribute(fwd_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(bwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  }
+  // the whole workspace as rows of H bfloat16: any h block starts at a whole row
+  const uint64_t rows = y.total / ((size_t)H * 2);
+  bool ok = make_tmap_2d(&P.tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, FB);
+  ok = ok && make_tmap_2d(&P.tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, FG);
+  if (ok && KB0 < KBh) {
+    // the paired forward kernel, if the device can keep its clusters resident and
+    // MEBPTT_FWD_PAIR=1 in the environment asks for it (measured slower so far: the hand-over of
+    // the partial tiles between the two CTAs costs more than the halved contraction saves)
+    const char* force = getenv("MEBPTT_FWD_PAIR");
+    const int pairs = (H + 2 * FU - 1) / (2 * FU);
+    const int grid = fwd_groups * 2 * pairs;
+    const int smem = KB0 * (2 * FG + FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
+    if (force && atoi(force) == 1) {
+      const void* fn = (const void*)fwd_run_pair_kernel;
+      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
+      cudaLaunchAttribute at1[1];
+      at1[0].id = cudaLaunchAttributeClusterDimension;
+      at1[0].val.clusterDim.x = 2; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
+      cfg.attrs = at1; cfg.numAttrs = 1;
+      int nclusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) cudaGetLastError();
+      else if (nclusters * 2 >= grid &&
+               make_tmap_2d(&P.tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, 2 * FG)) {
+        P.fwd_pair = true; P.fwd_ncg = 2 * pairs; P.fwd_smem = smem;
       }
     }
   }
+  if (ok && H % 64 == 0) {
+    CUtensorMap blocked;
+    if (make_tmap_blocks64(&blocked, ws, (uint64_t)H, rows, (uint64_t)H * 2, FB, (uint32_t)P.fwd_bb)) {
+      P.tm_h = blocked;
+      P.fwd_slab = true;
+    }
+  }
+  for (int pb = 0; pb < 2; ++pb)
+    ok = ok && make_tmap_2d(&P.tm_dz[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64,
+                            (uint32_t)BM);
+  ok = ok && make_tmap_2d(&P.tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
+  if (!ok) { P.rc = MEBPTT_ERR_UNSUPPORTED; return; }
+  // the clustered backward kernel, if the device can keep enough clusters resident
+  // (MEBPTT_BWD_CLUSTER = 0, 4 or 8 in the environment overrides the choice)
+  const char* force = getenv("MEBPTT_BWD_CLUSTER");
+  for (int cs : {8, 4}) {
+    if (force && atoi(force) != cs) continue;
+    if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
+    const int kbs = (G / 64) / cs;
+    const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * cs * BM * NU * 4 + 1024;
+    if (smem > 220 * 1024) continue;
+    const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
+    cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at1[1];
+    at1[0].id = cudaLaunchAttributeClusterDimension;
+    at1[0].val.clusterDim.x = cs; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
+    cfg.attrs = at1; cfg.numAttrs = 1;
+    int nclusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+    if (nclusters * cs < ncta) continue;
+    P.bwd_cs = cs; P.bwdc_smem = smem;
+    break;
+  }
+  if (P.bwd_cs) {
+    for (int pb = 0; pb < 2; ++pb)
+      ok = ok && make_tmap_2d(&P.tm_dz_b[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B,
+                              (uint64_t)G * 2, 64, 64);
+    ok = ok && make_tmap_2d(&P.tm_wt_c, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, (uint32_t)(NU * P.bwd_cs));
+    if (!ok) { P.rc = MEBPTT_ERR_UNSUPPORTED; return; }
+  }
+
+}
+
+// The set for (problem, plan, workspace, device): from the cache, or built and put there.  ws may
+// be null: then only the host part is made (what counting launches needs, or a machine without a GPU).
+std::shared_ptr<Prepared> prepare(const Layout& y, const Plan* p, bool want_dx, char* ws, bool allow_pinned) {
+  int dev = -1;
+  if (ws && cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); dev = -1; }
+  {
+    std::lock_guard<std::mutex> lock(g_prep_mu);
+    for (size_t i = 0; i < g_prep.size(); ++i) {
+      const Prepared& q = *g_prep[i];
+      if (q.plan_id == p->id && q.I == y.I && q.H == y.H && q.O == y.O && q.B == y.B && q.t == y.t &&
+          q.want_dx == want_dx && q.ws == ws && q.device == dev) {
+        std::shared_ptr<Prepared> hit = g_prep[i];
+        g_prep.erase(g_prep.begin() + (long)i);
+        g_prep.insert(g_prep.begin(), hit);
+        g_prep_stats[1]++;
+        return hit;
+      }
+    }
+  }
+  // built outside the lock (two threads may build the same set at the same time: both are valid)
+  std::shared_ptr<Prepared> P = std::make_shared<Prepared>();
+  P->plan_id = p->id; P->I = y.I; P->H = y.H; P->O = y.O; P->B = y.B; P->t = y.t;
+  P->want_dx = want_dx; P->ws = ws; P->device = dev;
+  build_host_part(*P, y, p, allow_pinned && ws != nullptr);
+  if (P->rc == MEBPTT_OK && ws) build_device_part(*P, y, ws);
+  g_prep_stats[0]++;
+  if (P->pinned) g_prep_stats[2]++;
+  if (P->rc == MEBPTT_OK) {
+    std::lock_guard<std::mutex> lock(g_prep_mu);
+    g_prep.insert(g_prep.begin(), P);
+    if (g_prep.size() > kPrepCapacity) g_prep.pop_back();
+  }
+  return P;
+}
+}  // namespace
+
+void forget_plan(uint64_t plan_id) {
+  std::lock_guard<std::mutex> lock(g_prep_mu);
+  for (size_t i = g_prep.size(); i-- > 0;)
+    if (g_prep[i]->plan_id == plan_id) g_prep.erase(g_prep.begin() + (long)i);
+}
+
+void prepare_stats(int64_t* out) {
+  for (int i = 0; i < 3; ++i) out[i] = g_prep_stats[i].load();
+  std::lock_guard<std::mutex> lock(g_prep_mu);
+  out[3] = (int64_t)g_prep.size();
+}
+
+int prepare_host(const Layout& y, const Plan* p, bool want_dx) { return prepare(y, p, want_dx, nullptr, false)->rc; }
+
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
+                 bool side_stream) {
+  const int B = y.B, H = y.H, I = y.I, O = y.O, S = y.S, G = 4 * H, K = I + H;
+  const int BM = 64;  // batch rows per MMA tile (B <= 64)
+  const int ncta = H / NU;
+  int64_t launches = 0;
+  char* ws = io.ws;
+  auto at = [&](size_t off) { return ws + off; };
+
+  // ---- the prepared set of this (problem, plan, workspace) --------------------------------------
+  const std::shared_ptr<Prepared> prep = prepare(y, p, want_dx, dry ? nullptr : ws, !io.pageable_tape);
+  if (prep->rc != MEBPTT_OK) return prep->rc;
+  const Prepared& P = *prep;
+  const size_t nops = p->tape.size();
+  const std::vector<WorkItem>& items = P.items;
   const DevOp* dops = reinterpret_cast<const DevOp*>(at(y.off_tape));
   uint32_t* sync = reinterpret_cast<uint32_t*>(at(y.off_sync));
   int* status = reinterpret_cast<int*>(at(y.off_status));
@@ -1464,96 +1799,13 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   const int KBh = (H + 63) / 64;
   const int KB0 = fwd_first_part_blocks(H);       // 64-wide blocks of the recurrent contraction in its first part
   const int fwd_groups = B > FB ? 2 : 1;          // groups of CTAs that each own FB batch rows
-  int fwd_ncg = (H + FU - 1) / FU;                // CTAs per group
-  const int fwd_parts = KB0 < KBh ? 2 : 1;
-  int fwd_smem = (KBh * FG + fwd_parts * KB0 * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
-  bool fwd_pair = false;                          // clusters of two CTAs that split the contraction
-  bool fwd_slab = false;                          // h_{k-1} by one copy per part instead of one per K tile
-  int fwd_bb = KB0;                               // K tiles per barrier
   const int bwd_smem = ((G + 63) / 64) * 1024 + NST * BM * 128 + 1024;
-  CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
-  int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
+  const CUtensorMap &tm_h = P.tm_h, &tm_w = P.tm_w, &tm_wt = P.tm_wt, &tm_wt_c = P.tm_wt_c;
+  const CUtensorMap* tm_dz = P.tm_dz;
+  const CUtensorMap* tm_dz_b = P.tm_dz_b;
+  const int bwd_cs = P.bwd_cs, bwdc_smem = P.bwdc_smem, fwd_ncg = P.fwd_ncg, fwd_smem = P.fwd_smem, fwd_bb = P.fwd_bb;
+  const bool fwd_pair = P.fwd_pair, fwd_slab = P.fwd_slab;
   if (!dry) {
-    static const bool attrs = [] {
-      const int big = 220 * 1024;  // the kernels also hold a few static barriers
-      cudaFuncSetAttribute(fwd_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-      cudaFuncSetAttribute(bwd_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-      return true;
-    }();
-    (void)attrs;
-    // the whole workspace as rows of H bfloat16: any h block starts at a whole row
-    const uint64_t rows = y.total / ((size_t)H * 2);
-    bool ok = make_tmap_2d(&tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, FB);
-    ok = ok && make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, FG);
-    if (ok && KB0 < KBh) {
-      // the paired forward kernel, if the device can keep its clusters resident and
-      // MEBPTT_FWD_PAIR=1 in the environment asks for it (measured slower so far: the hand-over of
-      // the partial tiles between the two CTAs costs more than the halved contraction saves)
-      const char* force = getenv("MEBPTT_FWD_PAIR");
-      const int pairs = (H + 2 * FU - 1) / (2 * FU);
-      const int grid = fwd_groups * 2 * pairs;
-      const int bb = KB0 >= 4 ? (KB0 + 1) / 2 : KB0;   // two barriers per step where a half is long enough
-      const int smem = (KB0 * 2 * FG + ((KB0 + bb - 1) / bb) * bb * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
-      if (force && atoi(force) == 1) {
-        const void* fn = (const void*)fwd_run_pair_kernel;
-        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
-        cudaLaunchAttribute at1[1];
-        at1[0].id = cudaLaunchAttributeClusterDimension;
-        at1[0].val.clusterDim.x = 2; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
-        cfg.attrs = at1; cfg.numAttrs = 1;
-        int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) cudaGetLastError();
-        else if (nclusters * 2 >= grid &&
-                 make_tmap_2d(&tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, 2 * FG)) {
-          fwd_pair = true; fwd_ncg = 2 * pairs; fwd_smem = smem; fwd_bb = bb;
-        }
-      }
-    }
-    if (ok && H % 64 == 0) {
-      CUtensorMap blocked;
-      if (make_tmap_blocks64(&blocked, ws, (uint64_t)H, rows, (uint64_t)H * 2, FB, (uint32_t)fwd_bb)) {
-        tm_h = blocked;
-        fwd_slab = true;
-      }
-    }
-    for (int pb = 0; pb < 2; ++pb)
-      ok = ok && make_tmap_2d(&tm_dz[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, 64,
-                              (uint32_t)BM);
-    ok = ok && make_tmap_2d(&tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
-    if (!ok) return MEBPTT_ERR_UNSUPPORTED;
-    // the clustered backward kernel, if the device can keep enough clusters resident
-    // (MEBPTT_BWD_CLUSTER = 0, 4 or 8 in the environment overrides the choice)
-    const char* force = getenv("MEBPTT_BWD_CLUSTER");
-    for (int cs : {8, 4}) {
-      if (force && atoi(force) != cs) continue;
-      if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
-      const int kbs = (G / 64) / cs;
-      const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * cs * BM * NU * 4 + 1024;
-      if (smem > 220 * 1024) continue;
-      const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
-      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(ncta); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
-      cudaLaunchAttribute at1[1];
-      at1[0].id = cudaLaunchAttributeClusterDimension;
-      at1[0].val.clusterDim.x = cs; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
-      cfg.attrs = at1; cfg.numAttrs = 1;
-      int nclusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
-      if (nclusters * cs < ncta) continue;
-      bwd_cs = cs; bwdc_smem = smem;
-      break;
-    }
-    if (bwd_cs) {
-      for (int pb = 0; pb < 2; ++pb)
-        ok = ok && make_tmap_2d(&tm_dz_b[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B,
-                                (uint64_t)G * 2, 64, 64);
-      ok = ok && make_tmap_2d(&tm_wt_c, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, (uint32_t)(NU * bwd_cs));
-      if (!ok) return MEBPTT_ERR_UNSUPPORTED;
-    }
-
     cudaMemsetAsync(dh, 0, (size_t)B * H * 4, s);
     cudaMemsetAsync(dc, 0, (size_t)B * H * 4, s);
     cudaMemsetAsync(io.dW, 0, (size_t)G * K * 4, s);
@@ -1563,7 +1815,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
     cudaMemsetAsync(sync, 0, y.n_sync * 4, s);
     cudaMemsetAsync(status, 0, 256, s);
-    cudaMemcpyAsync(at(y.off_tape), dev.data(), 2 * nops * sizeof(DevOp), cudaMemcpyHostToDevice, s);
+    // (from page-locked memory: an asynchronous copy proper; from pageable memory, which only the
+    // allocation-free entry point uses, the call may wait for the stream to reach the copy)
+    cudaMemcpyAsync(at(y.off_tape), P.tape, P.tape_entries * sizeof(DevOp), cudaMemcpyHostToDevice, s);
     launch_pdl(pack_weights, dim3(592), dim3(256), 0, s, reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
                reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh, wpT_ih, bias_p, woutT);
     // Peek of the initial state: the caller's (h0, c0) as a hidden block inside the workspace
@@ -1627,22 +1881,11 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       // a forward run: consecutive operations k, k+1, ... each starting from the state the
       // previous one wrote; at most S of them per launch
       const int n = wi.n;
-      // Input projections Zx of the S steps from the start of the run on, unless the buffer already
-      // holds them: recomputation sweeps keep returning to the same stored state, so one
-      // projection serves many short runs.  (The values do not depend on how steps are batched.)
+      // input projections Zx, unless the window in place holds those of this run
       const int k0 = first.k;
-      if (!(k0 >= zx_lo && k0 + n <= zx_hi)) {
+      if (P.zx_hi[item]) {
         zx_lo = k0;
-        // as far as the runs that will still find their steps in this window reach (the first
-        // forward run that does not fit in the S steps from k0 on replaces the window)
-        const int cap = (int)((int64_t)k0 + S <= y.t + 1 ? k0 + S : y.t + 1);
-        zx_hi = k0 + n;
-        for (size_t j = item + 1; j < items.size(); ++j) {
-          if (items[j].kind != WorkItem::FWD) continue;
-          const int kj = p->tape[items[j].i].k, ej = kj + items[j].n;
-          if (kj < k0 || ej > cap) break;
-          if (ej > zx_hi) zx_hi = ej;
-        }
+        zx_hi = P.zx_hi[item];
         const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
         need_x(zx_hi - 1);
         gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
@@ -1651,7 +1894,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (!dry && rc == MEBPTT_OK) {
         FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
                      io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0, off16(y.plane), off16(y.hsz)};
-        void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
+        FwdPairArgs pa{a, reinterpret_cast<__nv_bfloat16*>(at(y.off_xring))};
+        void* args_pair[] = {(void*)&tm_w, (void*)&pa};
+        void* args_one[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
+        void** args = fwd_pair ? args_pair : args_one;
         const void* fn = fwd_pair ? (const void*)fwd_run_pair_kernel : (const void*)fwd_run_kernel;
         const int span = span_begin(timer, 0, n, s);
         if (!cuda_ok(launch_coop(fn, fwd_groups * fwd_ncg, 192, fwd_smem, s, args, fwd_pair ? 2 : 1), "forward run launch"))

@@ -516,3 +516,47 @@ def test_launch_count_is_what_the_profiler_sees(H, base, kw, plans):
         seen = sum(1 for ev in prof.events()
                    if ev.device_type == torch.autograd.DeviceType.CUDA and not ev.name.startswith(("Memset", "Memcpy")))
         assert seen == B.mebptt_lstm_launch_count(dp.desc, plan), (base, mode, m, seen)
+
+
+def test_prepared_set_is_reused_per_workspace_and_the_enqueue_is_cheap(H):
+    """The per-step call looks its prepared set (tape, tensor maps, kernel variants) up instead of
+    rebuilding it: one set per (problem, plan, workspace), a new one when the workspace moves, the
+    bits of the first call on every later one, and -- at config 3 with the headline budget -- an
+    enqueue that takes the host under a quarter of what the step takes the device."""
+    import time
+    import torch
+    from paper_1606_03401_b200 import binding as B
+    cfg = synth.CONFIGS["c3"]
+    dp = H.DeviceProblem(cfg)
+    plan = dp.plan("msm", 100)
+    s0 = B.mebptt_lstm_prepare_stats()
+    first = dp.run(plan)
+    s1 = B.mebptt_lstm_prepare_stats()
+    assert s1["built"] == s0["built"] + 1 and s1["page_locked"] == s0["page_locked"] + 1
+    again = dp.run(plan)
+    s2 = B.mebptt_lstm_prepare_stats()
+    assert s2["built"] == s1["built"] and s2["reused"] == s1["reused"] + 1
+    assert_bit_identical(again, first)
+    # the workspace moves: the tensor maps are made anew, the results stay
+    keep = dp._ws
+    dp._ws = torch.empty(keep.numel() + 4096, dtype=torch.uint8, device=keep.device)[256:]
+    assert dp._ws.data_ptr() != keep.data_ptr()
+    moved = dp.run(plan)
+    assert B.mebptt_lstm_prepare_stats()["built"] == s2["built"] + 1
+    assert_bit_identical(moved, first)
+    # host time of an enqueue against device time of the step
+    torch.cuda.synchronize()
+    host, dev = [], []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        t0 = time.perf_counter()
+        dp.enqueue(plan)
+        host.append((time.perf_counter() - t0) * 1e3)
+        e1.record()
+        torch.cuda.synchronize()
+        dev.append(e0.elapsed_time(e1))
+    host_ms, dev_ms = sorted(host)[len(host) // 2], sorted(dev)[len(dev) // 2]
+    print(f"c3 msm m=100: host enqueue {host_ms:.2f} ms, device {dev_ms:.2f} ms")
+    assert host_ms < 0.25 * dev_ms, (host_ms, dev_ms)
