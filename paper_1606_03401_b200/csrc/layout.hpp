@@ -52,7 +52,7 @@ struct Layout {
   size_t off_a3 = 0, off_w3 = 0, off_wmn3 = 0, off_wout3 = 0, off_woutmn3 = 0;
   size_t off_z = 0, off_split = 0, off_st_dz = 0, off_st_in = 0, off_st_hp = 0, off_st_dy = 0, off_st_h = 0;
   size_t off_zx = 0, off_zleaf = 0, off_hprev = 0, off_hk = 0, off_y = 0;
-  size_t off_sync = 0, off_tape = 0, off_status = 0, off_split_dh = 0, off_xring = 0;
+  size_t off_sync = 0, off_tape = 0, off_status = 0, off_split_dh = 0;
   size_t off_a3_run = 0, off_zrun = 0, off_hrun = 0, off_dha_run = 0, off_dy_run = 0, split_floats = 0;
   size_t n_sync = 0, tape_bytes = 0;
   size_t total = 0;
@@ -295,7 +295,6 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_dy = take(2 * SB * y.O * 2);
     y.off_dha = take(SB * y.H * 4);
     y.off_zleaf = take(SB * G * 4);   // pre-activations of a batch of leaves
-    y.off_xring = take((size_t)4 * 64 * y.H * 2);   // exchange ring of the paired forward kernel: 4 slots of [64][H]
     y.off_loss_part = take((size_t)y.S * loss_parts_per_step(y.B, y.O) * 4);
     y.n_sync = 64 * (work_items(p, y.S).size() + 1);   // two 128-byte lines per persistent launch (one per group of CTAs)
     y.off_sync = take(y.n_sync * 4);

@@ -83,9 +83,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 // The same, restricted to global memory: what a thread needs between observing (acquire) data
 // that other CTAs wrote with ordinary stores and reading that data with TMA.
-// Restricted to this CTA's shared memory: what a thread needs between writing an MMA operand tile
-// with ordinary stores and handing it to the tensor core.
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -244,35 +241,6 @@ __device__ __forceinline__ void st_peer_f4(void* local_smem, uint32_t peer_rank,
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem)), "r"(peer_rank));
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
                : "memory");
-}
-// Address of `local_smem` in the shared memory of CTA `peer_rank` of this cluster (shared::cluster window).
-__device__ __forceinline__ uint32_t peer_smem_u32(const void* local_smem, uint32_t peer_rank) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem)), "r"(peer_rank));
-  return remote;
-}
-// Asynchronous 16-byte store into the shared memory of a CTA of this cluster (its own included);
-// on arrival the 16 bytes are counted on the mbarrier `remote_bar`, which must lie in the same CTA
-// as the destination.  A thread that waits for that barrier's phase sees the data.
-__device__ __forceinline__ void st_async_f4(uint32_t remote_addr, uint32_t remote_bar, float4 v) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
-               ::"r"(remote_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar)
-               : "memory");
-}
-// Arrival on named barrier `id` without waiting; `count` is the number of threads the barrier expects
-// in all (arrivers and waiters).  Memory accesses made before it are performed with respect to the
-// threads that bar.sync on the same barrier.
-__device__ __forceinline__ void named_barrier_arrive(uint32_t id, uint32_t count) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-// ---- words that other CTAs poll: strong (relaxed, gpu scope) accesses -----------------------------
-__device__ __forceinline__ void st_relaxed_u2(void* p, uint2 v) {
-  asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
-}
-__device__ __forceinline__ uint4 ld_relaxed_u4(const void* p) {
-  uint4 v;
-  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-  return v;
 }
 // Barrier among `count` threads (a multiple of 32) of this CTA; ids 1..15 (0 is __syncthreads).
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t count) {

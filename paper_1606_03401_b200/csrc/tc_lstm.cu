@@ -100,37 +100,51 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 // ------------------------------------------------------------------------------------------
 // forward run
 // ------------------------------------------------------------------------------------------
-// What bounds a step of the recurrence is the time h_{k-1} takes to reach every SM that holds a
-// part of W_hh (the bytes all SMs pull through the L2 together, and the bytes each takes in) and
-// the number of MMA instructions one thread must issue for a tile (one per 16 contraction
-// indices, whatever the tile's size).  Three things cut both:
+// A step of the recurrence is bound by latency, not by bytes or flops: h_{k-1} has to get from the
+// SMs that produce it to every SM that holds a part of W_hh (stores, release of a step counter, a
+// poll with acquire, the fetch), and one thread must then issue an MMA per 16 contraction indices.
+// What the kernel does about it:
 //
 //   * The batch rows of an LSTM never mix, so the grid is cut into groups of CTAs that each own
-//     FB = 32 batch rows: a CTA pulls only its group's rows of h_{k-1} and groups synchronise
-//     among themselves only (a step counter per group).
-//   * The product is taken transposed: gate rows of W_hh (resident in shared memory, rows permuted
-//     to 4 u + q) are the M side of the MMA and the 32 batch rows the N side, so that a tile of
-//     full height serves a batch slice of 32.
-//   * Two neighbouring CTAs (a cluster of two) share 32 hidden units and split the contraction
-//     index: CTA r keeps the block [128 gate rows][K half r] of W_hh, pulls only that half of the
-//     columns of h_{k-1}, and issues half the MMAs.  The partial tile [128][32] leaves TMEM one
-//     gate row per thread and goes, 64 rows each, to the CTA that owns those rows -- into its
-//     shared memory, its own or the neighbour's (distributed shared memory).
+//     FB = 32 batch rows: a CTA pulls only its group's rows of h_{k-1}, and groups synchronise
+//     among themselves only (a step counter per group, in a cache line of its own).  CTA c of a
+//     group owns hidden units 16 c .. 16 c + 15.
+//   * The product is taken transposed: the CTA's 64 gate rows of W_hh (resident in shared memory,
+//     rows permuted to 4 u + q) are the M side of the MMA and the 32 batch rows the N side, so that
+//     a tile of full height serves a batch slice of 32.
+//   * The TMA unit accepts one copy request at a time and takes ~100 ns for each, whatever its
+//     size: sixteen tile copies are a microsecond and a half before the last tile even starts.
+//     h_{k-1} is therefore fetched with two copies (one per half of the contraction index) over a
+//     3-D tensor map that sees a row as blocks of 64 columns, which land as consecutive swizzled
+//     tiles.
+//   * The contraction is summed in two parts (two TMEM accumulators; the MMAs of the first are
+//     issued while the second half of h_{k-1} is still arriving):  z = (Zx + part 0) + part 1, Zx
+//     being the batched input projection, bias included.  The batched GEMMs of a leaf batch
+//     accumulate in the same order, so both give the same bits.
+//   * The accumulators [64 gate rows][32 batch rows] leave TMEM one gate row per thread and are
+//     handed over through shared memory; each of the 128 epilogue threads then owns four hidden
+//     units of one batch row -- four threads side by side cover 32 bytes of a row, so a warp's
+//     store is 8 full sectors instead of 32 quarter sectors, and the stores are what the release
+//     that follows waits for.  The thread applies the gates and updates c_t, h_t (which stay in
+//     registers from step to step) and writes the state where the tape says (scratch, a slot of
+//     the arena, or a whole internal state).
 //
-// Each of the 128 epilogue threads then owns four hidden units of one batch row: it adds, in a
-// fixed order, z = (Zx + part 0) + part 1 -- Zx being the batched input projection, bias included
-// -- applies the gates and updates c_t, h_t (which stay in registers from step to step), and
-// writes the state where the tape says (scratch, a slot of the arena, or a whole internal state).
-// fwd_run_kernel is the same computation without clusters: one CTA per 16 hidden units takes both
-// halves of the contraction into two accumulators.  Both give the same bits, and so do the
-// batched GEMMs of a leaf batch, which accumulate Zx, the first and the second half in that order.
+// Measured and dropped (config 3, microseconds per forward operation against 4.47 for this
+// kernel): clusters of two CTAs that split the contraction index and exchange partial tiles
+// through distributed shared memory, by ordinary remote stores with a release/acquire barrier
+// (5.0) or by asynchronous stores that count on the receiver's barrier (exchange 0.66 of the
+// 4.5 us step); h_k as its own signal -- a ring of exchange slots whose words hold an impossible
+// bit pattern until h_k is written with strong stores, polled with strong 16-byte loads into
+// registers and staged into the swizzled tiles by the epilogue warps, the step counter kept off
+// the critical path for the reuse of slots only -- which removes the 1.5 us signalling round but
+// loses as much to the staging and to waiting for the slowest producer (5.3).
 //
 // Warps 0-3: epilogue; warp 4: TMA producer; warp 5: MMA issuer.  All of h_{k-1} a CTA needs is
 // resident in shared memory for the step (H <= 1024), so the producer never waits for a free slot.
 constexpr int FU = 16;          // hidden units per CTA
 constexpr int FG = 4 * FU;      // gate rows per CTA
 constexpr int FB = 32;          // batch rows per group of CTAs: the N of the MMA
-constexpr int PART_LD = FB + 4; // row stride of a partial tile in shared memory (floats)
+constexpr int PART_LD = FG + 4; // row stride of an accumulator handed over in shared memory, [batch row][gate row] (floats)
 constexpr int SYNC_STRIDE = 32; // words between the step counters of two groups (one 128-byte line each)
 
 struct FwdRunArgs {
@@ -148,12 +162,6 @@ struct FwdRunArgs {
   uint32_t plane16;      // distance between gate planes, in 16-byte units
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
 };
-
-// The exchange ring of the paired kernel (described there): value of an empty word, slots, rows per slot.
-constexpr uint32_t XR_EMPTY = 0xffffffffu;
-constexpr int XR_SLOTS = 4;
-constexpr int XR_ROWS = 2 * FB;
-__device__ __forceinline__ uint32_t xr_word(uint32_t w) { return w == XR_EMPTY ? 0x7fff7fffu : w; }
 
 // 64-wide blocks of the contraction index in the first part of the split (all of them if there is one)
 __host__ __device__ inline int fwd_first_part_blocks(int H) {
@@ -198,9 +206,7 @@ __device__ __forceinline__ void fwd_cell_gates(FwdCell& st, const float4 (&z)[4]
     st.c[u] = fmaf(fv[u], st.c[u], iv[u] * gv[u]);
     hv[u] = ov[u] * tanh_fast(st.c[u]);
   }
-  // (a pair of NaNs with every payload bit set is what an empty word of the exchange ring of the
-  // paired kernel holds: such a result is written as the canonical NaN pair by both kernels)
-  o.hnew = make_uint2(xr_word(pack_bf16x2(hv[0], hv[1])), xr_word(pack_bf16x2(hv[2], hv[3])));
+  o.hnew = make_uint2(pack_bf16x2(hv[0], hv[1]), pack_bf16x2(hv[2], hv[3]));
   o.gi = make_uint2(pack_bf16x2(iv[0], iv[1]), pack_bf16x2(iv[2], iv[3]));
   o.gf = make_uint2(pack_bf16x2(fv[0], fv[1]), pack_bf16x2(fv[2], fv[3]));
   o.gg = make_uint2(pack_bf16x2(gv[0], gv[1]), pack_bf16x2(gv[2], gv[3]));
@@ -232,17 +238,16 @@ __device__ __forceinline__ void fwd_cell_rest(FwdCell& st, const FwdRunArgs& a, 
     for (int v = 0; v < 4; ++v) st.zx[v] = zp[v];
   }
 }
-// z = (Zx + part 0) + part 1 for the 16 gate rows of this thread; a part is [64 gate rows][PART_LD]
-// with the batch row as the column.
-__device__ __forceinline__ void fwd_cell_sum(const FwdCell& st, const float* part0, const float* part1, int row0, int col,
-                                             float4 (&z)[4]) {
+// z = (Zx + part 0) + part 1 for the 16 gate rows of this thread: p0 / p1 point at its 16 floats
+// (gate rows 4 u + q of its four units) in the handed-over accumulators.
+__device__ __forceinline__ void fwd_cell_sum(const FwdCell& st, const float* p0, const float* p1, float4 (&z)[4]) {
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const float* p = part0 + (size_t)(row0 + 4 * u) * PART_LD + col;
-    z[u] = make_float4(st.zx[u].x + p[0], st.zx[u].y + p[PART_LD], st.zx[u].z + p[2 * PART_LD], st.zx[u].w + p[3 * PART_LD]);
-    if (part1) {
-      const float* q = part1 + (size_t)(row0 + 4 * u) * PART_LD + col;
-      z[u].x += q[0]; z[u].y += q[PART_LD]; z[u].z += q[2 * PART_LD]; z[u].w += q[3 * PART_LD];
+    const float4 x = *reinterpret_cast<const float4*>(p0 + 4 * u);
+    z[u] = make_float4(st.zx[u].x + x.x, st.zx[u].y + x.y, st.zx[u].z + x.z, st.zx[u].w + x.w);
+    if (p1) {
+      const float4 y = *reinterpret_cast<const float4*>(p1 + 4 * u);
+      z[u].x += y.x; z[u].y += y.y; z[u].z += y.z; z[u].w += y.w;
     }
   }
 }
@@ -264,7 +269,7 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   uint8_t* sW = sm;                    // KB tiles: this CTA's rows of W_hh
   uint8_t* tiles = sm + KB * W_TILE;   // KB tiles: the group's rows of h_{k-1}
   const int NQ = KB0 < KB ? 2 : 1;     // parts of the contraction: one barrier, one copy (slab mode), one accumulator each
-  float* part = reinterpret_cast<float*>(tiles + NQ * KB0 * H_TILE);   // [2][FG][PART_LD]
+  float* part = reinterpret_cast<float*>(tiles + NQ * KB0 * H_TILE);   // [2][FB][PART_LD]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int grp = blockIdx.x / a.ncg, cta = blockIdx.x % a.ncg;
@@ -361,10 +366,11 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
   } else {
     // ---- gates and state update ------------------------------------------------------------------
     // as a reader of TMEM: warp w, lanes 0 .. 15 hold accumulator rows (gate rows) 16 w .. 16 w + 15;
-    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of the CTA
+    // as an owner of state: batch row tid / 4 of the group, hidden units 4 (tid % 4) .. + 3 of the CTA
     const int zrow = 16 * warp + lane;
-    const int b = grp * FB + lane;                      // batch row
-    const int j0 = cta * FU + 4 * warp;                 // first hidden unit
+    const int bl = tid >> 2, u0 = 4 * (tid & 3);        // batch row inside the group, first unit inside the CTA
+    const int b = grp * FB + bl;                        // batch row
+    const int j0 = cta * FU + u0;                       // first hidden unit
     const bool owner = b < a.B && j0 < a.H;
     const size_t e0 = (size_t)b * a.H + j0;             // element index of (b, j0) in a [B][H] array
     const bool two = KB0 < KB;
@@ -379,11 +385,9 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
         tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)(h * FB), r);
         tmem_ld_wait();
         if (lane < 16) {
-          float4* dst = reinterpret_cast<float4*>(part + ((size_t)h * FG + zrow) * PART_LD);
+          float* dst = part + (size_t)h * FB * PART_LD + zrow;
 #pragma unroll
-          for (int v = 0; v < FB / 4; ++v)
-            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                                 __uint_as_float(r[4 * v + 3]));
+          for (int n = 0; n < FB; ++n) dst[n * PART_LD] = __uint_as_float(r[n]);
         }
       }
       tc_fence_before_sync();
@@ -391,7 +395,8 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
       FwdCellOut out;
       if (got && owner) {
         float4 z[4];
-        fwd_cell_sum(st, part, two ? part + FG * PART_LD : nullptr, 16 * warp, lane, z);
+        const float* p0 = part + (size_t)bl * PART_LD + 4 * u0;
+        fwd_cell_sum(st, p0, two ? p0 + FB * PART_LD : nullptr, z);
         fwd_cell_gates(st, z, out);
         // h_k first: it is what the other CTAs wait for
         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = out.hnew;
@@ -409,264 +414,6 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
     else if (blockIdx.x == 0) a.counters[0] += a.n;
   }
   if (warp == 4) tmem_dealloc(tmem, 64);
-}
-
-// Clusters of two CTAs per 32 hidden units and group, each taking one half of the contraction.
-//
-// How h_k travels.  A grid-wide counter (stores, release, poll with acquire, then a TMA fetch) puts
-// four dependent trips through the L2 on every step: measured 1.5 us for the signalling round of 128
-// CTAs alone.  Here h_k is its own signal.  Besides writing h_k where the tape says, every thread
-// writes it (strong, relaxed stores) into a ring of four exchange slots, [64 batch rows][H] each,
-// whose words hold an impossible value until then -- 0xffffffff, two bfloat16 NaNs with all payload
-// bits set; a value the arithmetic produces is rewritten if it collides.  The consumers read their
-// rows and columns of the slot with strong loads straight into registers, take every 16-byte piece
-// that holds no such word, put it into shared memory in the 128-byte swizzled tile layout, and ask
-// again only for what was not there yet.  One trip of the data through the L2 instead of four.
-//   Slot (i mod 4) is written at step i, read at step i + 1 and put back to the impossible value by
-// its writers at step i + 2, which is safe (who produces at step i + 2 has read all of h_{i+1}, so
-// everybody has finished reading h_i) and two steps ahead of the next writing.  That a reader of
-// step i + 5 cannot meet the words of step i any more is not left to the two steps in between: the
-// grid-wide counter is kept, off the critical path -- a spare warp signals (release) after the
-// stores of each step and acquires, for a step s, the signals of step s - 3 before the readers of
-// step s start.  Only the first exchange of a launch, which follows the initial clearing of the
-// ring, waits for the counter on the critical path.
-//
-// The partial tiles change hands between the two CTAs by asynchronous stores into (distributed)
-// shared memory that count their bytes on a barrier of the receiver.
-
-struct FwdPairArgs {
-  FwdRunArgs r;
-  __nv_bfloat16* xring;  // [XR_SLOTS][XR_ROWS][H]
-};
-
-__global__ void __launch_bounds__(192, 1) fwd_run_pair_kernel(const __grid_constant__ CUtensorMap tm_w,
-                                                              const FwdPairArgs pa) {
-  const FwdRunArgs& a = pa.r;
-  constexpr int PG = 2 * FG;              // gate rows of the pair: the M of the MMA
-  constexpr uint32_t W_TILE = PG * 128;   // [128 gate rows][64 contraction indices]
-  constexpr uint32_t H_TILE = FB * 128;   // [32 batch rows][64 contraction indices]
-  constexpr int MAXLD = 16;               // 16-byte pieces of h_{k-1} per thread and step: 8 rows x 2 (8 K tiles of 8 pieces / 32 lanes)
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t wfull, full[2], acc, pready;
-  __shared__ uint32_t tmem_slot;
-  __shared__ int failed;
-  __shared__ volatile int lag_ok;          // readers of local step s may start once lag_ok >= s
-
-  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int KB = (a.H + 63) / 64;          // 2 .. 16
-  const int KB0 = fwd_first_part_blocks(a.H);
-  const uint32_t rank = cluster_ctarank();
-  const int kb_lo = rank ? KB0 : 0;        // this CTA's blocks of the contraction index
-  const int nkb = rank ? KB - KB0 : KB0;   // 1 .. 8
-  const int nkb_a = (nkb + 1) / 2;         // K tiles behind the first of the two barriers
-  uint8_t* sW = sm;                        // KB0 tiles: the pair's gate rows, this CTA's K blocks
-  uint8_t* tiles = sm + KB0 * W_TILE;      // KB0 tiles: the group's rows of h_{k-1}, this CTA's K blocks
-  float* part = reinterpret_cast<float*>(tiles + KB0 * H_TILE);   // [2 senders][FG][PART_LD]
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int grp = blockIdx.x / a.ncg, pair = (blockIdx.x % a.ncg) >> 1;
-  uint32_t* const sync = a.sync + grp * SYNC_STRIDE;
-  const int rows_g = (a.B - grp * FB < FB) ? a.B - grp * FB : FB;   // batch rows of this group
-
-  if (tid == 0) {
-    mbar_init(&wfull, 1);
-    mbar_init(&full[0], 4);                // one arrival per epilogue warp
-    mbar_init(&full[1], 4);
-    mbar_init(&acc, 1);
-    mbar_init(&pready, 1);
-    failed = 0;
-    lag_ok = 0;
-    mbar_fence_init();
-    tma_prefetch_desc(&tm_w);
-  }
-  // rows past the batch and columns past H are never fetched: they stay zero
-  for (int e = tid; e < KB0 * (int)H_TILE / 16; e += 192) reinterpret_cast<uint4*>(tiles)[e] = make_uint4(0, 0, 0, 0);
-  if (warp == 4) tmem_alloc(&tmem_slot, 32);
-  fence_proxy_async();
-  tc_fence_before_sync();
-  cluster_sync();                          // the neighbour signals this CTA's barrier: it must be initialised
-  tc_fence_after_sync();
-  const uint32_t tmem = tmem_slot;
-  grid_dep_wait();
-
-  if (warp == 4) {
-    // ---- W_hh, then the counter: signal each step once its stores are out, and keep the readers'
-    // licence (lag_ok) ahead of them ---------------------------------------------------------------
-    if (lane == 0) {
-      mbar_arrive_expect_tx(&wfull, (uint32_t)nkb * W_TILE);
-      for (int kb = 0; kb < nkb; ++kb) tma_load_2d(sW + kb * W_TILE, &tm_w, (kb_lo + kb) * 64, pair * PG, &wfull);
-    }
-    for (int i = 0; i < a.n; ++i) {
-      named_barrier(2, 160);               // the epilogue threads' stores of step i (arrive) precede the release
-      if (lane == 0) {
-        red_release_add(sync, 1u);
-        if (i + 1 < a.n) {
-          // the readers of local step s want the signals of step max(0, s - 3): once those of step
-          // max(0, i - 1) are in, the readers of steps up to i + 2 may go -- long before they get there,
-          // except for the first exchange of the launch
-          const uint32_t need = (uint32_t)(i > 1 ? i : 1) * (uint32_t)a.ncg;
-          if (wait_counter(sync, need, &failed) && !failed)
-            asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32((const void*)&lag_ok)), "r"(i + 2) : "memory");
-        }
-        if (i + 2 == a.n || a.n == 1) grid_dep_launch();   // last step under way: the next kernel may set itself up
-      }
-      __syncwarp();
-    }
-    if (failed && lane == 0) (void)mbar_wait(&wfull, 0);
-  } else if (warp == 5) {
-    // ---- MMA issuer ----------------------------------------------------------------------------
-    constexpr uint32_t idesc = make_idesc(1, PG, FB, false, false);
-    bool ok = wait_or_fail(&wfull, 0, &failed);
-    const uint64_t w_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
-    const uint64_t h_desc0 = make_desc_sw128(smem_u32(tiles), 16, 1024);
-    for (int i = 0; i < a.n; ++i) {
-      uint64_t dw = w_desc0, dh = h_desc0;
-      for (int q = 0; q < 2 && ok; ++q) {
-        ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const int cnt = q ? nkb - nkb_a : nkb_a;
-        if (elect_one()) {
-          for (int kb = 0; kb < cnt; ++kb)
-            mma_f16_x4(tmem, dw + (uint64_t)(kb * (W_TILE >> 4)), dh + (uint64_t)(kb * (H_TILE >> 4)), idesc,
-                       (q > 0 || kb > 0) ? 1u : 0u);
-        }
-        __syncwarp();
-        dw += (uint64_t)nkb_a * (W_TILE >> 4);
-        dh += (uint64_t)nkb_a * (H_TILE >> 4);
-      }
-      if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
-      __syncwarp();
-    }
-  } else {
-    // ---- epilogue warps: fetch h_{k-1}, then gates and state update ------------------------------
-    // as a reader of TMEM: thread (w, lane) holds gate row 32 w + lane of the pair's partial tile; rows
-    // 0 .. 63 belong to the units of CTA 0 of the pair, rows 64 .. 127 to those of CTA 1;
-    // as an owner of state: batch row `lane` of the group, hidden units 4 w .. 4 w + 3 of this CTA;
-    // as a reader of h_{k-1}: batch rows 8 w .. 8 w + 7 of the group, 16-byte piece `lane` of every
-    // run of four K tiles (512 bytes of a row)
-    const int prow = 32 * warp + lane;
-    const uint32_t row_owner = (uint32_t)(prow >> 6);
-    const uint32_t send_addr = peer_smem_u32(part + ((size_t)rank * FG + (prow & 63)) * PART_LD, row_owner);
-    const uint32_t send_bar = peer_smem_u32(&pready, row_owner);
-    const int b = grp * FB + lane;
-    const int j0 = pair * 2 * FU + (int)rank * FU + 4 * warp;
-    const bool owner = b < a.B && j0 < a.H;
-    const size_t e0 = (size_t)b * a.H + j0;
-    const size_t xr_slot = (size_t)XR_ROWS * a.H;          // elements per exchange slot
-    FwdCell st;
-    fwd_cell_init(st, a, owner, b, j0, e0);
-    if (owner) {
-      // the ring starts empty (the first signal of every CTA, which the readers of step 1 wait for,
-      // comes after these stores)
-#pragma unroll
-      for (int sl = 0; sl < XR_SLOTS; ++sl) st_relaxed_u2(pa.xring + sl * xr_slot + e0, make_uint2(XR_EMPTY, XR_EMPTY));
-    }
-    // what this thread fetches: piece p (0 .. 8 lpr - 1) is row 8 w + p / lpr, K tile 4 (p % lpr) + lane / 8,
-    // 16-byte column lane % 8 of that tile; lpr = loads per row = 1 or 2 (up to 8 K tiles of 8 pieces
-    // for 32 lanes).  Which pieces exist, and which lie behind the first barrier, never changes.
-    const int ls = nkb > 4 ? 1 : 0;                          // log2(lpr)
-    const int c8 = lane & 7, kq = lane >> 3;
-    uint32_t pieces = 0, first_half = 0;
-    for (int p = 0; p < (8 << ls); ++p) {
-      const int row = 8 * warp + (p >> ls), kb = 4 * (p & ls) + kq;
-      if (row < rows_g && kb < nkb && (kb_lo + kb) * 64 + c8 * 8 < a.H) {
-        pieces |= 1u << p;
-        if (kb < nkb_a) first_half |= 1u << p;
-      }
-    }
-    const size_t g_off0 = (size_t)(grp * FB + 8 * warp) * a.H + (size_t)(kb_lo + kq) * 64 + c8 * 8;   // piece 0, in elements
-    for (int i = 0; i < a.n; ++i) {
-      const DevOp op = a.ops[i];
-      // ---- h_{k-1}: from where the tape says at the first step (written before this launch), from
-      // the ring afterwards -------------------------------------------------------------------------
-      {
-        const __nv_bfloat16* src = ((i == 0) ? reinterpret_cast<const __nv_bfloat16*>(a.ws + (size_t)op.h_src * 16)
-                                             : pa.xring + (size_t)((i - 1) % XR_SLOTS) * xr_slot) + g_off0;
-        if (i > 0) {
-          bool lic = false;
-          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-            int seen;
-            asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(seen) : "r"(smem_u32((const void*)&lag_ok)) : "memory");
-            if (seen >= i) { lic = true; break; }
-            if (spin > 64 && failed) break;
-          }
-          if (!lic) failed = 1;
-        }
-        for (int half = 0; half < 2; ++half) {
-          // first the pieces of the K tiles behind the first barrier, then the rest
-          uint32_t want = half ? (pieces & ~first_half) : first_half;
-          for (uint32_t round = 0; want != 0 && !failed; ++round) {
-            if (round >= (kSpinLimit >> 4)) { failed = 1; break; }
-            if (round > 0) __nanosleep(100);   // what was not there yet: ask again, but leave the L2 to the writers
-            uint4 v[MAXLD];
-#pragma unroll
-            for (int p = 0; p < MAXLD; ++p)
-              if (want >> p & 1u) v[p] = ld_relaxed_u4(src + (size_t)(p >> ls) * a.H + (p & ls) * 256);
-#pragma unroll
-            for (int p = 0; p < MAXLD; ++p) {
-              if (want >> p & 1u) {
-                const uint4 w = v[p];
-                if (i == 0 || (w.x != XR_EMPTY && w.y != XR_EMPTY && w.z != XR_EMPTY && w.w != XR_EMPTY)) {
-                  const int row = 8 * warp + (p >> ls), kb = 4 * (p & ls) + kq;
-                  *reinterpret_cast<uint4*>(tiles + kb * H_TILE + row * 128 + ((c8 ^ (row & 7)) << 4)) = w;
-                  want &= ~(1u << p);
-                }
-              }
-            }
-          }
-          fence_proxy_async_smem();        // the tiles are read by the tensor core through the async proxy
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&full[half]);
-        }
-      }
-      // ---- the pair's partial tile: every gate row to the CTA that owns its unit -------------------
-      const bool got = wait_or_fail(&acc, (uint32_t)i & 1, &failed);
-      tc_fence_after_sync();
-      if (tid == 0) mbar_arrive_expect_tx(&pready, 2u * FG * FB * 4u);   // 64 rows of 32 floats from each of the two CTAs
-      {
-        uint32_t r[32];
-        tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int v = 0; v < FB / 4; ++v)
-          st_async_f4(send_addr + 16u * v, send_bar,
-                      make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                                  __uint_as_float(r[4 * v + 3])));
-      }
-      tc_fence_before_sync();
-      bool all = false;
-      for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-        if (mbar_try_wait_cluster(&pready, (uint32_t)i & 1)) { all = true; break; }
-        if (spin > 256) {
-          if (failed) break;
-          __nanosleep(32);
-        }
-      }
-      if (!all) failed = 1;
-      FwdCellOut out;
-      const bool good = got && all && owner;
-      if (good) {
-        float4 z[4];
-        fwd_cell_sum(st, part, part + FG * PART_LD, 16 * warp, lane, z);
-        fwd_cell_gates(st, z, out);
-        // h_k into the ring first: it is what the other CTAs wait for
-        if (i + 1 < a.n) st_relaxed_u2(pa.xring + (size_t)(i % XR_SLOTS) * xr_slot + e0, out.hnew);
-        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.ws + (size_t)op.h_dst * 16) + e0) = out.hnew;
-        if (i + 2 < a.n) st_relaxed_u2(pa.xring + (size_t)((i + 2) % XR_SLOTS) * xr_slot + e0, make_uint2(XR_EMPTY, XR_EMPTY));
-        fwd_cell_rest(st, a, op, out, i, b, j0, e0);
-      }
-      named_barrier_arrive(2, 160);        // the spare warp signals once every epilogue thread is here
-    }
-  }
-
-  tc_fence_before_sync();
-  cluster_sync();   // no CTA leaves while its neighbour may still write into its shared memory or signal it
-  if (tid == 0) {
-    if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
-    else if (blockIdx.x == 0) a.counters[0] += a.n;
-  }
-  if (warp == 4) tmem_dealloc(tmem, 32);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1512,7 +1259,7 @@ struct Prepared {
   CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
   int fwd_ncg = 0, fwd_smem = 0, fwd_bb = 0;
-  bool fwd_pair = false, fwd_slab = false;
+  bool fwd_slab = false;
   int rc = MEBPTT_OK;
 
   Prepared() = default;
@@ -1625,8 +1372,7 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
   const int fwd_groups = B > FB ? 2 : 1;          // groups of CTAs that each own FB batch rows
   const int fwd_parts = KB0 < KBh ? 2 : 1;
   P.fwd_ncg = (H + FU - 1) / FU;                  // CTAs per group
-  P.fwd_smem = (KBh * FG + fwd_parts * KB0 * FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
-  P.fwd_pair = false;                             // clusters of two CTAs that split the contraction
+  P.fwd_smem = (KBh * FG + fwd_parts * KB0 * FB) * 128 + 2 * FB * PART_LD * 4 + 1024;
   P.fwd_slab = false;                             // h_{k-1} by one copy per part instead of one per K tile
   P.fwd_bb = KB0;                                 // K tiles per barrier
   P.bwd_cs = 0; P.bwdc_smem = 0;
@@ -1640,31 +1386,6 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
   const uint64_t rows = y.total / ((size_t)H * 2);
   bool ok = make_tmap_2d(&P.tm_h, ws, 2, (uint64_t)H, rows, (uint64_t)H * 2, 64, FB);
   ok = ok && make_tmap_2d(&P.tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, FG);
-  if (ok && KB0 < KBh) {
-    // the paired forward kernel, if the device can keep its clusters resident and
-    // MEBPTT_FWD_PAIR=1 in the environment asks for it (measured slower so far: the hand-over of
-    // the partial tiles between the two CTAs costs more than the halved contraction saves)
-    const char* force = getenv("MEBPTT_FWD_PAIR");
-    const int pairs = (H + 2 * FU - 1) / (2 * FU);
-    const int grid = fwd_groups * 2 * pairs;
-    const int smem = KB0 * (2 * FG + FB) * 128 + 2 * FG * PART_LD * 4 + 1024;
-    if (force && atoi(force) == 1) {
-      const void* fn = (const void*)fwd_run_pair_kernel;
-      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
-      cudaLaunchAttribute at1[1];
-      at1[0].id = cudaLaunchAttributeClusterDimension;
-      at1[0].val.clusterDim.x = 2; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
-      cfg.attrs = at1; cfg.numAttrs = 1;
-      int nclusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) cudaGetLastError();
-      else if (nclusters * 2 >= grid &&
-               make_tmap_2d(&P.tm_w, wp_hh, 2, (uint64_t)H, (uint64_t)G, (uint64_t)H * 2, 64, 2 * FG)) {
-        P.fwd_pair = true; P.fwd_ncg = 2 * pairs; P.fwd_smem = smem;
-      }
-    }
-  }
   if (ok && H % 64 == 0) {
     CUtensorMap blocked;
     if (make_tmap_blocks64(&blocked, ws, (uint64_t)H, rows, (uint64_t)H * 2, FB, (uint32_t)P.fwd_bb)) {
@@ -1804,7 +1525,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   const CUtensorMap* tm_dz = P.tm_dz;
   const CUtensorMap* tm_dz_b = P.tm_dz_b;
   const int bwd_cs = P.bwd_cs, bwdc_smem = P.bwdc_smem, fwd_ncg = P.fwd_ncg, fwd_smem = P.fwd_smem, fwd_bb = P.fwd_bb;
-  const bool fwd_pair = P.fwd_pair, fwd_slab = P.fwd_slab;
+  const bool fwd_slab = P.fwd_slab;
   if (!dry) {
     cudaMemsetAsync(dh, 0, (size_t)B * H * 4, s);
     cudaMemsetAsync(dc, 0, (size_t)B * H * 4, s);
@@ -1894,13 +1615,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (!dry && rc == MEBPTT_OK) {
         FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
                      io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0, off16(y.plane), off16(y.hsz)};
-        FwdPairArgs pa{a, reinterpret_cast<__nv_bfloat16*>(at(y.off_xring))};
-        void* args_pair[] = {(void*)&tm_w, (void*)&pa};
-        void* args_one[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
-        void** args = fwd_pair ? args_pair : args_one;
-        const void* fn = fwd_pair ? (const void*)fwd_run_pair_kernel : (const void*)fwd_run_kernel;
+        void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
+        const void* fn = (const void*)fwd_run_kernel;
         const int span = span_begin(timer, 0, n, s);
-        if (!cuda_ok(launch_coop(fn, fwd_groups * fwd_ncg, 192, fwd_smem, s, args, fwd_pair ? 2 : 1), "forward run launch"))
+        if (!cuda_ok(launch_coop(fn, fwd_groups * fwd_ncg, 192, fwd_smem, s, args, 1), "forward run launch"))
           rc = MEBPTT_ERR_CUDA;
         span_end(timer, span, s);
       }
