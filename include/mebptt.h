@@ -402,6 +402,20 @@ int mebptt_gemm_bf16(const void *A, int64_t lda, int a_major, const void *B, int
                      float *C, int64_t ldc, int accumulate, const float *bias,
                      int64_t M, int64_t N, int64_t K, int *status, void *stream);
 
+/*
+ * Testing aid for the bounded waits of the tensor-core kernels (no counterpart in the paper).
+ * Every wait of those kernels on a step counter or a barrier gives up after a bounded number of
+ * polls, reports MEBPTT_ERR_TIMEOUT through the status word (counters[3], or `status` of
+ * mebptt_gemm_bf16) and lets the kernel end in the ordinary way.  To see that path run without
+ * anything being wrong, a test sets a mask: bit 0 makes the forward run kernel's step counter wait
+ * for one CTA more than exist, bit 1 does the same to the backward run kernels, bit 2 makes the
+ * first pipeline stage of the batched contraction wait for 16 bytes more than its copies bring;
+ * the waits concerned then give up after a few thousand polls.  No memory is touched that an
+ * ordinary run would not touch.  mask = 0 restores normal behaviour; the setting is per process
+ * and meant for single-threaded tests only.  Returns MEBPTT_ERR_ARG for a mask outside 0..7.
+ */
+int mebptt_test_wait_fault(int mask);
+
 const char *mebptt_strerror(int status);
 
 #ifdef __cplusplus

@@ -86,6 +86,7 @@ _SIGS = {
     "mebptt_lstm_run_times": (_i32, [C.POINTER(C.c_double), C.POINTER(_i64), C.POINTER(_i64)]),
     "mebptt_lstm_prepare": (_i32, [_descp, _vp]),
     "mebptt_lstm_prepare_stats": (_i32, [C.POINTER(_i64)]),
+    "mebptt_test_wait_fault": (_i32, [_i32]),
     "mebptt_slot_copy": (_i32, [_vp, _vp, _sz, _vp]),
     "mebptt_gemm_bf16": (_i32, [_vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64, _i64, _i64, _vp, _vp]),
     "mebptt_strerror": (C.c_char_p, [_i32]),
@@ -292,6 +293,10 @@ def mebptt_lstm_prepare_stats() -> dict:
     out = (_i64 * 4)()
     _check(lib.mebptt_lstm_prepare_stats(out), "mebptt_lstm_prepare_stats")
     return {"built": out[0], "reused": out[1], "page_locked": out[2], "held": out[3]}
+
+
+def mebptt_test_wait_fault(mask: int) -> None:
+    _check(lib.mebptt_test_wait_fault(int(mask)), "mebptt_test_wait_fault")
 
 
 def mebptt_lstm_run_times() -> dict:

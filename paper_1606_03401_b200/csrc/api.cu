@@ -617,6 +617,12 @@ int mebptt_lstm_prepare(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan)
   return tc::prepare_host(y, p, desc->want_dx != 0);
 }
 
+int mebptt_test_wait_fault(int mask) {
+  if (mask < 0 || mask > 7) return MEBPTT_ERR_ARG;
+  tc::set_wait_fault_mask(mask);
+  return MEBPTT_OK;
+}
+
 int mebptt_lstm_prepare_stats(int64_t* out) {
   if (!out) return MEBPTT_ERR_ARG;
   tc::prepare_stats(out);

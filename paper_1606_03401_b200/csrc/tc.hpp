@@ -115,6 +115,15 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
                  bool side_stream);
 
 
+// Testing aid: which bounded waits are made to run out on purpose (0: none).  Bit 0: the step
+// counter of the forward run kernel is told to expect one CTA too many; bit 1: likewise for the
+// backward run kernels; bit 2: the first stage of a GEMM expects 16 bytes more than its copies
+// bring.  The waits then give up after `fault_poll_limit` polls instead of the usual limit, the
+// kernels leave through their ordinary exit path, and the status word receives MEBPTT_ERR_TIMEOUT.
+int wait_fault_mask();
+void set_wait_fault_mask(int mask);
+constexpr uint32_t fault_poll_limit = 1u << 14;
+
 // The prepared sets (work items, device tape, kernel variants, tensor maps) that run_step keeps per
 // (problem, plan, workspace, device).  forget_plan drops those of a plan that is being freed;
 // prepare_host makes (or finds) the host part only and returns its status; prepare_stats fills

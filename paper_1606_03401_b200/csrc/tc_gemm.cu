@@ -41,7 +41,7 @@ template <bool A_MN, bool B_MN, int BN = BN_WIDE>
 __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma,
                                                         const __grid_constant__ CUtensorMap tmb, GemmOut out,
                                                         int M, int N, int K, int STAGES, int* status,
-                                                        float* partial) {
+                                                        float* partial, int fault) {
   constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
   static_assert(BN == BN_WIDE || (!A_MN && !B_MN), "narrow tiles exist for K-major operands only");
   extern __shared__ uint8_t smem_raw[];
@@ -83,7 +83,9 @@ __global__ void __launch_bounds__(128) gemm_bf16_kernel(const __grid_constant__ 
       if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { failed = 1; break; }
       uint8_t* sA = ring + s * STAGE_BYTES;
       uint8_t* sB = sA + A_BYTES;
-      mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
+      // (fault: a testing aid -- the first stage is told to expect 16 bytes that never come, so the
+      // issuer's bounded wait runs out and the kernel leaves through its failure path)
+      mbar_arrive_expect_tx(&full[s], STAGE_BYTES + ((fault && kb == 0) ? 16u : 0u));
       ++armed;
       if (A_MN) {
         tma_load_2d(sA, &tma, m0, (kb_lo + kb) * BK, &full[s]);
@@ -430,7 +432,7 @@ int gemm_bf16(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
              : a_mn ? (b_mn ? gemm_bf16_kernel<true, true> : gemm_bf16_kernel<true, false>)
                     : (b_mn ? gemm_bf16_kernel<false, true> : gemm_bf16_kernel<false, false>);
   const cudaError_t e = launch_on(early, fn, grid, dim3(128), (size_t)GEMM_SMEM, s, ta, tb, out, M, N, K, stages, status,
-                                  splits > 1 ? split->partial : nullptr);
+                                  splits > 1 ? split->partial : nullptr, (wait_fault_mask() & 4) ? 1 : 0);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return MEBPTT_ERR_CUDA;

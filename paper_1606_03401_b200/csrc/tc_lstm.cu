@@ -86,8 +86,9 @@ __device__ __forceinline__ bool wait_or_fail(uint64_t* bar, uint32_t parity, vol
   *failed = 1;
   return false;
 }
-__device__ __forceinline__ bool wait_counter(const uint32_t* ctr, uint32_t target, volatile int* failed) {
-  for (uint32_t i = 0; i < (kSpinLimit >> 1); ++i) {
+__device__ __forceinline__ bool wait_counter(const uint32_t* ctr, uint32_t target, volatile int* failed,
+                                             uint32_t limit = kSpinLimit >> 1) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (ld_acquire(ctr) >= target) return true;
     if (i > 4096 && *failed) return false;
   }
@@ -159,6 +160,8 @@ struct FwdRunArgs {
   int ncg;               // CTAs per group
   int bb;                // K tiles (64 contraction indices each) per barrier and, in slab mode, per copy
   int slab;              // 1: tm_h is a blocked 3-D map and one copy brings bb tiles; 0: one 2-D copy per tile
+  uint32_t expect;       // signals a step is complete with: ncg (a testing aid may ask for one too many)
+  uint32_t poll_limit;   // polls of the step counter before the wait gives up
   uint32_t plane16;      // distance between gate planes, in 16-byte units
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
 };
@@ -308,7 +311,7 @@ __global__ void __launch_bounds__(192, 1) fwd_run_kernel(const __grid_constant__
       // only reach accumulator columns that no thread reads)
       const int32_t row = (int32_t)(((uint64_t)op.h_src * 16u) / row_bytes) + grp * FB;
       int go = 1;
-      if (lane == 0) go = (i == 0 || wait_counter(sync, (uint32_t)i * (uint32_t)a.ncg, &failed)) && !failed;
+      if (lane == 0) go = !failed && (i == 0 || wait_counter(sync, (uint32_t)i * a.expect, &failed, a.poll_limit)) && !failed;
       go = __shfl_sync(0xffffffffu, go, 0);
       if (!go) continue;
       // the acquire of lane 0 reaches the other lanes through the shuffle; the proxy fence then orders
@@ -436,6 +439,10 @@ struct BwdRunArgs {
   uint32_t plane16, hsz16;
   const float* zleaf;      // leaf batch: [S][B][4H] pre-activations z_k (gate columns permuted); NULL otherwise
   int loss_parts;          // partial sums of the loss per step
+  int tb;                  // clustered kernel: K tiles per barrier and, in slab mode, per copy
+  int slab;                // clustered kernel: 1: tm_dz is a blocked 3-D map and one copy brings tb tiles
+  uint32_t expect;         // signals a step is complete with: the grid size (a testing aid may ask for one too many)
+  uint32_t poll_limit;     // polls of the step counter before the wait gives up
 };
 
 // What the gate derivatives of one batch row and 8 hidden units read from memory at one step: the
@@ -631,7 +638,7 @@ __global__ void __launch_bounds__(128, 1) bwd_run_kernel(const __grid_constant__
 
     if (is_p) {
       // ---- producer: all of dz_k through the ring -----------------------------------------
-      bool ok = wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed);
+      bool ok = wait_counter(a.sync, (uint32_t)(i + 1) * a.expect, &failed, a.poll_limit);
       if (ok) {
         fence_proxy_async();
         const int32_t row = sidx * a.B;
@@ -721,11 +728,12 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int G = 4 * a.H;
   const int KBS = (G / 64) / CS;           // 64-wide K blocks in this CTA's slice (<= 16)
-  const int NQ = (KBS + 3) / 4;            // blocks of four K tiles, one barrier each
+  const int TB = a.tb;                     // K tiles per barrier
+  const int NQ = (KBS + TB - 1) / TB;      // <= 4
   uint8_t* sW = sm;                        // KBS tiles [NC rows][128 B]
   uint8_t* ring = sW + KBS * W_TILE;       // KBS tiles [64 rows][128 B], all of the slice at once
   // partial sums received from the cluster: [2 buffers][CS senders][64 rows][8 columns]
-  float* recv = reinterpret_cast<float*>(ring + KBS * A_TILE);
+  float* recv = reinterpret_cast<float*>(ring + NQ * TB * A_TILE);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
@@ -769,17 +777,24 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
         a.loss_t[a.ops[i].k - 1] = sum;
       }
       int go = 1;
-      if (lane == 0) go = wait_counter(a.sync, (uint32_t)(i + 1) * (uint32_t)ncta, &failed) && !failed;
+      if (lane == 0) go = !failed && wait_counter(a.sync, (uint32_t)(i + 1) * a.expect, &failed, a.poll_limit) && !failed;
       go = __shfl_sync(0xffffffffu, go, 0);
       if (!go) continue;
       if (lane < NQ) {
+        // (the TMA unit takes its copy requests one at a time, ~100 ns each: in slab mode one copy over
+        // a map that sees a row as blocks of 64 columns brings the TB tiles of a barrier)
         fence_proxy_async_global();
         const int32_t row = sidx * a.B;
         const int q = lane;
-        const int kb0 = 4 * q, kb1 = (kb0 + 4 < KBS) ? kb0 + 4 : KBS;
-        mbar_arrive_expect_tx(&full[q], (uint32_t)(kb1 - kb0) * A_TILE);
-        for (int kb = kb0; kb < kb1; ++kb)
-          tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
+        const int kb0 = TB * q, kb1 = (kb0 + TB < KBS) ? kb0 + TB : KBS;
+        if (a.slab) {
+          mbar_arrive_expect_tx(&full[q], (uint32_t)TB * A_TILE);   // a box counts in full
+          tma_load_3d(ring + kb0 * A_TILE, &tm_dz, 0, row, (int)rank * KBS + kb0, &full[q]);
+        } else {
+          mbar_arrive_expect_tx(&full[q], (uint32_t)(kb1 - kb0) * A_TILE);
+          for (int kb = kb0; kb < kb1; ++kb)
+            tma_load_2d(ring + kb * A_TILE, &tm_dz, ((int)rank * KBS + kb) * 64, row, &full[q]);
+        }
       }
       armed = i;
       if (i == a.n - 1 && lane == 0) grid_dep_launch();
@@ -802,15 +817,15 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
         ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
         if (!ok) break;
         tc_fence_after_sync();
-        const int nkb = (4 * q + 4 < KBS) ? 4 : KBS - 4 * q;
+        const int nkb = (TB * q + TB < KBS) ? TB : KBS - TB * q;
         if (elect_one()) {
           for (int kb = 0; kb < nkb; ++kb)
             mma_f16_x4(tmem, da + (uint64_t)(kb * (A_TILE >> 4)), db + (uint64_t)(kb * (W_TILE >> 4)), idesc,
                        (q > 0 || kb > 0) ? 1u : 0u);
         }
         __syncwarp();
-        da += 4 * (A_TILE >> 4);
-        db += 4 * (W_TILE >> 4);
+        da += (uint64_t)TB * (A_TILE >> 4);
+        db += (uint64_t)TB * (W_TILE >> 4);
       }
       if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
       __syncwarp();
@@ -1258,6 +1273,8 @@ struct Prepared {
   // device part
   CUtensorMap tm_h, tm_w, tm_dz[2], tm_wt, tm_dz_b[2], tm_wt_c;
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
+  int bwd_tb = 4;                  // its K tiles per barrier
+  bool bwd_slab = false;           // its slice of dz by one copy per barrier instead of one per K tile
   int fwd_ncg = 0, fwd_smem = 0, fwd_bb = 0;
   bool fwd_slab = false;
   int rc = MEBPTT_OK;
@@ -1405,7 +1422,8 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
     if (force && atoi(force) != cs) continue;
     if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
     const int kbs = (G / 64) / cs;
-    const int smem = kbs * (NU * cs * 128) + kbs * BM * 128 + 2 * cs * BM * NU * 4 + 1024;
+    const int tb = kbs > 8 ? 8 : 4;   // K tiles per barrier: at most four barriers, two where the slice is long
+    const int smem = kbs * (NU * cs * 128) + ((kbs + tb - 1) / tb) * tb * BM * 128 + 2 * cs * BM * NU * 4 + 1024;
     if (smem > 220 * 1024) continue;
     const void* fn = cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
     cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -1418,13 +1436,19 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
     int nclusters = 0;
     if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
     if (nclusters * cs < ncta) continue;
-    P.bwd_cs = cs; P.bwdc_smem = smem;
+    P.bwd_cs = cs; P.bwdc_smem = smem; P.bwd_tb = tb;
     break;
   }
   if (P.bwd_cs) {
+    // the staging chunk as [columns / 64][rows][64] if the driver takes such a map, else tile by tile
+    P.bwd_slab = true;
     for (int pb = 0; pb < 2; ++pb)
-      ok = ok && make_tmap_2d(&P.tm_dz_b[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B,
-                              (uint64_t)G * 2, 64, 64);
+      P.bwd_slab = P.bwd_slab && make_tmap_blocks64(&P.tm_dz_b[pb], dz + (size_t)pb * S * B * G, (uint64_t)G, (uint64_t)S * B,
+                                                   (uint64_t)G * 2, 64, (uint32_t)P.bwd_tb);
+    if (!P.bwd_slab)
+      for (int pb = 0; pb < 2; ++pb)
+        ok = ok && make_tmap_2d(&P.tm_dz_b[pb], dz + (size_t)pb * S * B * G, 2, (uint64_t)G, (uint64_t)S * B,
+                                (uint64_t)G * 2, 64, 64);
     ok = ok && make_tmap_2d(&P.tm_wt_c, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, (uint32_t)(NU * P.bwd_cs));
     if (!ok) { P.rc = MEBPTT_ERR_UNSUPPORTED; return; }
   }
@@ -1466,6 +1490,12 @@ std::shared_ptr<Prepared> prepare(const Layout& y, const Plan* p, bool want_dx, 
   return P;
 }
 }  // namespace
+
+namespace {
+std::atomic<int> g_wait_fault{0};
+}
+int wait_fault_mask() { return g_wait_fault.load(); }
+void set_wait_fault_mask(int mask) { g_wait_fault.store(mask); }
 
 void forget_plan(uint64_t plan_id) {
   std::lock_guard<std::mutex> lock(g_prep_mu);
@@ -1576,6 +1606,7 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
 
   int launch_id = 0;
   int rc = MEBPTT_OK;
+  const int fault = wait_fault_mask();   // testing aid, 0 outside the tests of the bounded waits
   if (!dry && !cuda_ok(cudaGetLastError(), "set-up (memsets, tape upload, weight packing)")) rc = MEBPTT_ERR_CUDA;
   auto gemm_on = [&](cudaStream_t st, const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn,
                      GemmOut out, int M, int N, int Kc) {
@@ -1614,7 +1645,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
         FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
-                     io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0, off16(y.plane), off16(y.hsz)};
+                     io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0,
+                     (uint32_t)fwd_ncg + ((fault & 1) ? 1u : 0u), (fault & 1) ? fault_poll_limit : (kSpinLimit >> 1),
+                     off16(y.plane), off16(y.hsz)};
         void* args[] = {(void*)&tm_h, (void*)&tm_w, (void*)&a};
         const void* fn = (const void*)fwd_run_kernel;
         const int span = span_begin(timer, 0, n, s);
@@ -1692,7 +1725,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
         BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
-                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts};
+                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts, P.bwd_tb, P.bwd_slab ? 1 : 0,
+                     (uint32_t)ncta + ((fault & 2) ? 1u : 0u), (fault & 2) ? fault_poll_limit : (kSpinLimit >> 1)};
         void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         const int span = span_begin(timer, 1, n, s);
         if (bwd_cs) {
