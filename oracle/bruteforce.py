@@ -116,14 +116,16 @@ def ism_unrestricted(t: int, m: int):
     return _zero_one_bfs(start, lambda u: u[0] == 0, moves)
 
 
-def msm_protocol(t: int, m: int, alpha: int, beta: int | None = None):
+def msm_protocol(t: int, m: int, alpha: int, beta: int | None = None, sigma: int = 1):
     """Cheapest divide-and-conquer tree of the mixed protocol, found by trying them all.
 
     A tree node handles a subsequence of length n whose start state is stored and chooses
     either a hidden-state push at 1 <= y < n (one unit) or an internal-state push at
     1 <= y <= n (alpha units; beta if y = 1 and the Section 3.4 variant is on; none if y = n,
     because then the state never leaves the working core).  Feasibility is decided by a
-    running count of the units in use against the budget m, not by any formula.
+    running count of the units in use against the budget m, not by any formula.  ``sigma`` is
+    the size of a hidden state in the unit of m (1 in Section 3.3): what a hidden-state push
+    takes, and what the start state of the whole sequence occupies from the beginning.
     """
     best = [INFEASIBLE]
 
@@ -141,10 +143,10 @@ def msm_protocol(t: int, m: int, alpha: int, beta: int | None = None):
             return
         # hidden-state push at y
         for y in range(1, n):
-            if in_use + 1 <= budget_here:
+            if in_use + sigma <= budget_here:
                 # right part: starts at the pushed state, may fill the rest of the budget;
                 # then the push is released and the left part follows with the full budget
-                search(n - y, in_use + 1, budget_here, spent + y,
+                search(n - y, in_use + sigma, budget_here, spent + y,
                        lambda sp, y=y: search(y, in_use, budget_here, sp, cont))
         # internal-state push at y
         for y in range(1, n + 1):
@@ -162,6 +164,6 @@ def msm_protocol(t: int, m: int, alpha: int, beta: int | None = None):
         if best[0] is INFEASIBLE or spent < best[0]:
             best[0] = spent
 
-    if m >= 1:
-        search(t, 1, m, 0, done)
+    if m >= sigma:
+        search(t, sigma, m, 0, done)
     return best[0]

@@ -87,16 +87,28 @@ def ism_tables(t_max: int, m_max: int):
 # --------------------------------------------------------------------------------------
 # Sections 3.3 and 3.4, Eqs. (6)-(10): mixed memorisation
 # --------------------------------------------------------------------------------------
-def msm_tables(t_max: int, m_max: int, alpha: int, beta: int | None = None):
+def msm_tables(t_max: int, m_max: int, alpha: int, beta: int | None = None, sigma: int = 1):
     """C, H, D1, D2 for BPTT-MSM; ``beta`` switches on the variant of Section 3.4.
 
-    Q1(t, m, y) = y + C(y, m) + C(t - y, m - 1),               1 <= y <  t
+    Q1(t, m, y) = y + C(y, m) + C(t - y, m - sigma),           1 <= y <  t
     Q2(t, m, y) = y + C(y - 1, m) + C(t - y, m - a(y)),        1 <= y <= t
     with a(y) = alpha, or (Section 3.4) beta when y = 1 and alpha when y > 1.
-    C(0, .) = 0 everywhere, C(t > 0, m <= 0) = INF.  H = 1 (hidden) wins ties.
+    C(0, .) = 0 everywhere, C(t > 0, m < sigma) = INF.  H = 1 (hidden) wins ties.
+
+    ``sigma`` is the size of a hidden state in the unit m is counted in.  Section 3.3 measures
+    memory "in the units of hidden states", i.e. sigma = 1, and an internal state then has to be
+    a whole number alpha of them.  Where it is not -- Section 3.3 calls alpha application-specific,
+    and Appendix C has slots of arbitrary sizes s_i -- the same recursion is written over a finer
+    unit (the greatest common divisor of the sizes): a hidden state takes sigma units, an internal
+    state alpha, one without its input hidden state beta, and the start state of a subsequence,
+    which Section 3.1 counts as one of the m hidden states, sigma of the m units.
     """
-    if alpha < 2:
+    if sigma < 1:
+        raise ValueError("sigma must be a positive integer")
+    if alpha < 2 and sigma == 1:
         raise ValueError("alpha must be an integer >= 2 (Section 3.3)")
+    if alpha < sigma:
+        raise ValueError("an internal state contains a hidden state: alpha >= sigma")
     if beta is not None and not (1 <= beta <= alpha):
         raise ValueError("need 1 <= beta <= alpha (Section 3.4)")
     C = np.full((t_max + 1, m_max + 1), INF, dtype=np.int64)
@@ -106,18 +118,18 @@ def msm_tables(t_max: int, m_max: int, alpha: int, beta: int | None = None):
     C[0, :] = 0
 
     def Cget(tt, mm):
-        """C with the conventions for m <= 0 (vectorised over tt)."""
+        """C with the conventions for budgets that cannot hold a start state (vectorised over tt)."""
         tt = np.asarray(tt, dtype=np.int64)
-        if mm <= 0:
+        if mm < sigma:
             return np.where(tt == 0, np.int64(0), INF)
         return C[tt, mm]
 
-    for m in range(1, m_max + 1):
+    for m in range(sigma, m_max + 1):
         for t in range(1, t_max + 1):
             c1 = INF
             if t >= 2:
                 y = np.arange(1, t, dtype=np.int64)
-                Q1 = _sat(y + C[y, m] + Cget(t - y, m - 1))
+                Q1 = _sat(y + C[y, m] + Cget(t - y, m - sigma))
                 k1 = int(np.argmin(Q1))
                 c1 = Q1[k1]
                 D1[t, m] = y[k1]
@@ -208,8 +220,8 @@ def saturation_budget(mode: int, t: int, alpha: int = 4) -> int:
     return max(1, t)
 
 
-def plan_tables(mode: int, t: int, m: int, alpha: int = 4, beta: int | None = None):
-    """Tables for one (mode, t, m) problem, in a dict."""
+def plan_tables(mode: int, t: int, m: int, alpha: int = 4, beta: int | None = None, sigma: int = 1):
+    """Tables for one (mode, t, m) problem, in a dict (sigma: size of a hidden state, MSM only)."""
     if mode == HSM:
         C, D = hsm_tables(t, m)
         return {"mode": HSM, "C": C, "D": D}
@@ -217,14 +229,14 @@ def plan_tables(mode: int, t: int, m: int, alpha: int = 4, beta: int | None = No
         C, D = ism_tables(t, m)
         return {"mode": ISM, "C": C, "D": D}
     if mode == MSM:
-        C, H, D1, D2 = msm_tables(t, m, alpha, beta)
-        return {"mode": MSM, "C": C, "H": H, "D1": D1, "D2": D2, "alpha": alpha, "beta": beta}
+        C, H, D1, D2 = msm_tables(t, m, alpha, beta, sigma)
+        return {"mode": MSM, "C": C, "H": H, "D1": D1, "D2": D2, "alpha": alpha, "beta": beta, "sigma": sigma}
     raise ValueError("unknown mode")
 
 
-def cost(mode: int, t: int, m: int, alpha: int = 4, beta: int | None = None) -> int:
+def cost(mode: int, t: int, m: int, alpha: int = 4, beta: int | None = None, sigma: int = 1) -> int:
     """C(t, m): the predicted number of forward operations."""
-    return int(plan_tables(mode, t, m, alpha, beta)["C"][t, m])
+    return int(plan_tables(mode, t, m, alpha, beta, sigma)["C"][t, m])
 
 
 # --------------------------------------------------------------------------------------
@@ -301,7 +313,7 @@ class _Machine:
         self.ops.append(("B", k, src))
 
 
-def simulate(mode: int, t: int, m: int, tables=None, alpha: int = 4, beta: int | None = None):
+def simulate(mode: int, t: int, m: int, tables=None, alpha: int = 4, beta: int | None = None, sigma: int = 1):
     """Run the execution protocol for (mode, t, m) and return its integer statistics.
 
     Returns a dict with ``forwards`` (executed forward operations), ``backwards``,
@@ -309,11 +321,12 @@ def simulate(mode: int, t: int, m: int, tables=None, alpha: int = 4, beta: int |
     if the budget is exceeded, or if backward steps do not come in the order t, t-1, ..., 1.
     """
     if tables is None:
-        tables = plan_tables(mode, t, m, alpha, beta)
+        tables = plan_tables(mode, t, m, alpha, beta, sigma)
+    sg = tables.get("sigma", 1) if mode == MSM else 1
     if mode == ISM:
         mach = _Machine(t, m, 0)
     else:
-        mach = _Machine(t, m, 1)  # the initial hidden state takes one unit
+        mach = _Machine(t, m, sg)  # the initial hidden state takes the units of one hidden state
 
     def sweep(s: int, n: int, last_save: str | None):
         """n consecutive forward operations from the stored state at s."""
@@ -367,8 +380,8 @@ def simulate(mode: int, t: int, m: int, tables=None, alpha: int = 4, beta: int |
             if int(Hh[t_, m_]) == 1:
                 y = int(D1[t_, m_])
                 sweep(s, y, None)
-                mach.push("hidden", s + y, 1)
-                exec_msm(t_ - y, m_ - 1, s + y)
+                mach.push("hidden", s + y, sg)
+                exec_msm(t_ - y, m_ - sg, s + y)
                 mach.pop()
                 t_ = y
             else:

@@ -247,3 +247,58 @@ def test_chen_schedules_against_closed_forms():
     assert P.chen_recursive(1000, 1, 4, 3)["units"] >= 10
     for t in (100, 1000):
         assert P.chen_recursive(t, 3, 4, 3)["forwards"] >= P.cost(P.MSM, t, P.chen_recursive(t, 3, 4, 3)["units"], 4, 3)
+
+
+# ---------------------------------------------------------------- sizes that are no whole hidden states
+@pytest.mark.parametrize("sigma,alpha,beta", [(3, 10, 7), (3, 10, None), (2, 5, 3), (2, 7, None), (1, 4, 3)])
+def test_sized_msm_matches_protocol_enumeration(sigma, alpha, beta):
+    """The mixed recursion over a finer unit (a hidden state of sigma units, an internal state of
+    alpha, beta without its input state -- e.g. 3 : 10 : 7 for bfloat16 h and gates with a float32
+    cell state) against the exhaustive enumeration of protocol trees with a unit counter."""
+    for t in range(1, 7):
+        mm = alpha * t + sigma
+        C = P.msm_tables(t, mm, alpha, beta, sigma)[0]
+        for m in range(1, mm + 1):
+            found = BF.msm_protocol(t, m, alpha, beta, sigma)
+            if found is BF.INFEASIBLE:
+                assert m < sigma and C[t, m] >= P.INF, (t, m)       # not even the start state fits
+            else:
+                assert found == C[t, m], (t, m)
+
+
+def test_sized_msm_closed_forms_and_scaling():
+    t_max = 40
+    # sigma = 1 is Section 3.3 itself
+    for alpha, beta in [(4, None), (4, 3), (5, None)]:
+        a = P.msm_tables(t_max, 60, alpha, beta)[0]
+        b = P.msm_tables(t_max, 60, alpha, beta, 1)[0]
+        assert np.array_equal(a, b)
+    # multiplying every size by k changes nothing but the unit: C(t, k m + r; k sigma, k alpha, k beta)
+    # = C(t, m; sigma, alpha, beta) for 0 <= r < k
+    base = P.msm_tables(t_max, 30, 4, 3)[0]
+    k = 3
+    scaled = P.msm_tables(t_max, 30 * k + k - 1, 4 * k, 3 * k, k)[0]
+    for m in range(1, 31):
+        for r in range(k):
+            assert np.array_equal(scaled[:, k * m + r], base[:, m]), (m, r)
+    assert np.all(scaled[1:, :k] >= P.INF)                 # no room for the start state
+    # boundaries of Section 3.3 in the finer unit: only the start state fits -> t (t + 1) / 2;
+    # every internal state fits -> t
+    C = P.msm_tables(t_max, 10 * t_max + 3, 10, 7, 3)[0]
+    for t in range(1, t_max + 1):
+        assert C[t, 3] == t * (t + 1) // 2 and C[t, 5] == t * (t + 1) // 2
+        assert C[t, 3 + 10 * (t - 1)] == t
+    # a finer unit never costs more than rounding the sizes up to whole hidden states: with
+    # sizes 3 : 10 : 7 a budget of 3 m units holds what m units hold at 1 : 4 : 3 (= 3 : 12 : 9)
+    fine = P.msm_tables(t_max, 3 * 30, 10, 7, 3)[0]
+    coarse = P.msm_tables(t_max, 30, 4, 3)[0]
+    for m in range(1, 31):
+        assert np.all(fine[:, 3 * m] <= coarse[:, m])
+    assert np.any(fine[:, 3 * 8] < coarse[:, 8])
+
+
+def test_sized_msm_protocol_runs_within_budget():
+    for t, m in [(30, 20), (57, 41), (100, 100), (100, 33)]:
+        tab = P.plan_tables(P.MSM, t, m, 10, 7, 3)
+        r = P.simulate(P.MSM, t, m, tab)
+        assert r["forwards"] == tab["C"][t, m] and r["peak_units"] <= m and r["backwards"] == t
