@@ -43,9 +43,13 @@ WORKLOADS = {
     # t = 1000 (alpha = 4, beta = 3), so MSM at m = 127 is the like-for-like DP policy
     # "chenrec": Chen's recursive schedule with k = 3 cuts per level (22 units at t = 1000), beside
     # MSM at the same 22 units
-    "c3": ("msm", 100, [("msm", 10), ("msm", 22), ("chenrec", 3), ("msm", 32), ("msm", 127), ("chen", 0), ("msm", 1000)]),
+    # "msmx": BPTT-MSM planned over the byte sizes of the layout's states (bf16: hidden : internal :
+    # without input state = 3 : 10 : 7) at the bytes of m hidden states, beside "msm3" = the same
+    # bytes with internal states rounded up to 4 (3 without input state) hidden states
+    "c3": ("msm", 100, [("msm", 10), ("msm", 22), ("chenrec", 3), ("msm", 32), ("msm3", 100), ("msmx", 100),
+                        ("msm", 127), ("chen", 0), ("msm", 1000)]),
     "c4": ("ism", 50, [("ism", 20), ("ism", 200), ("msm", 80), ("msm", 200), ("msm", 800)]),
-    "c5": ("msm", 341, [("msm", 1365), ("msm", 5461)]),
+    "c5": ("msm", 341, [("msm3", 341), ("msmx", 341), ("msm", 1365), ("msm", 5461)]),
     "p0": ("hsm", 100, [("hsm", 10), ("hsm", 50), ("hsm", 500), ("hsm", 1000)]),
 }
 
@@ -152,10 +156,22 @@ def kernel_breakdown(dp, plans):
             print(f"| {k} | {n} | {v:.1f} | {v / n:.2f} | {100 * v / tot:.1f}% |", file=sys.stderr)
 
 
-# DRAM traffic of the forward run kernel per forward operation, from the ncu capture summarised in
-# profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md (42.39 MB read, 0.29 MB written, per launch of
-# 32 operations).  Valid for config 3's layer sizes and the kernel as profiled there.
-FWD_RUN_DRAM_BYTES_PER_OP_C3 = (42.389248e6 + 0.290816e6) / 32
+def profiled_traffic(kernel_source: str, summary: str):
+    """DRAM bytes per forward operation from the committed ncu summary of the dominant kernel, or
+    None if the kernel's source has changed since the counters were taken (the summary records the
+    hash of the source file it was taken from)."""
+    import hashlib
+    import re
+    try:
+        text = open(os.path.join(ROOT, summary)).read()
+        sha = hashlib.sha256(open(os.path.join(ROOT, kernel_source), "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    m_sha = re.search(r"kernel source sha256\[:16\]:\s*([0-9a-f]{16})", text)
+    m_b = re.search(r"DRAM bytes per forward operation:\s*([0-9.eE+]+)", text)
+    if not m_sha or not m_b or m_sha.group(1) != sha:
+        return None
+    return float(m_b.group(1))
 
 
 def max_over_ranks(v: float, world: int, device) -> float:
@@ -295,6 +311,15 @@ def main():
     W = max(3, args.warmup)
     ms, clocks = timed(plan, args.steps, W, sample_clocks=True)
     ms = max_over(ms)
+    # host time of one enqueue (the call returns before the device has started on the step)
+    torch.cuda.synchronize()
+    host_ms = []
+    for _ in range(5):
+        t0 = time.perf_counter()
+        dp.enqueue(plan)
+        host_ms.append((time.perf_counter() - t0) * 1e3)
+        torch.cuda.synchronize()
+    host_enqueue_ms = statistics.median(host_ms)
     counters = dp.out["counters"].cpu().numpy()
     assert int(counters[0]) == plan.cost and int(counters[3]) == 0, counters
 
@@ -328,17 +353,22 @@ def main():
         f_ms, f_n, f_ops = runs["forward"]
         b_ms, b_n, b_ops = runs["backward"]
         flops_rec = 2 * cfg.batch * cfg.hidden * 4 * cfg.hidden      # the recurrent contraction of one operation
+        per_op_traffic = (profiled_traffic("paper_1606_03401_b200/csrc/tc_lstm.cu",
+                                           "profiles/ncu_full_fwd_run_kernel_c3_shapes_t64.md")
+                          if (cfg.name == "c3" and cfg.input == 1024) else None)
         achieved = f_ops * flops_rec / (f_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": achieved / peak_tf,
-                    "traffic": FWD_RUN_DRAM_BYTES_PER_OP_C3 * (f_ops / f_n) if (cfg.name == "c3" and cfg.input == 1024) else None,
+                    "traffic": (per_op_traffic * (f_ops / f_n)) if per_op_traffic else None,
                     "kernel": "fwd_run_kernel (a run of forward operations: recurrent gate contraction + cell update)",
                     "launches": f_n // 3, "ops_per_launch": f_ops / f_n, "us_per_launch": f_ms * 1e3 / f_n,
                     "us_per_op": f_ms * 1e3 / f_ops,
                     "share_of_step": (f_ms / 3) / ms,
                     "backward_runs": {"kernel": "bwd_run_cluster_kernel", "launches": b_n // 3,
                                       "us_per_op": b_ms * 1e3 / max(1, b_ops), "share_of_step": (b_ms / 3) / ms},
-                    "traffic_note": "DRAM bytes per launch = bytes per operation (ncu, 32-operation launch) x mean operations per launch",
+                    "traffic_note": ("DRAM bytes per launch = bytes per operation (ncu capture of a 32-operation launch, "
+                                     "config 3's layer sizes) x mean operations per launch; null when the kernel's "
+                                     "source has changed since the capture"),
                     "how": f"CUDA events around each launch, 3 steps; {flops_rec} flops per operation x operations per launch / mean "
                            f"launch duration; peak = bf16 sustained ({pk['source']})"}
     else:
@@ -354,20 +384,32 @@ def main():
                                "forward operation on the CUDA-core path (gate contraction + cell update in one launch per layer)"),
                     "how": "(T(m) - T(full memory)) / (C(t,m) - t) = duration of one forward operation; "
                            f"{flops_fwd_op} flops per operation; peak = bf16 sustained ({pk['source']})"
-                           + ("" if cfg.dtype == "bf16" else " x 0.5 (nominal tf32:bf16 ratio)")}
+                           + ("" if cfg.dtype == "bf16" else " / 2: float32 storage takes three bf16 MMAs per product, so the "
+                              "rate of useful float32-product flops is at most a third of the bf16 peak; half of it "
+                              "(the nominal tf32 : bf16 ratio) is the denominator used here")}
+
+    # the whole step against the tensor peak: forward operations executed, backward operations
+    # (dh and dW products, dx is not asked for here), readout with its two gradients
+    flops_step = plan.cost * flops_fwd_op + cfg.t * flops_fwd_op + cfg.t * (flops_fwd_op - 2 * cfg.batch * cfg.input * 4 * cfg.hidden) \
+        + cfg.t * 6 * cfg.batch * cfg.hidden * cfg.readout
+    roofline["step_frac"] = flops_step / (ms * 1e-3) / 1e12 / peak_tf
+    roofline["step_flops"] = flops_step
 
     budgets = []
     if not args.no_budgets and rank == 0 or (not args.no_budgets and world > 1):
         for omode, om in others:
+            unit_b = B.mebptt_lstm_unit_bytes(dp.desc)
             op = (B.mebptt_plan_chen_sqrt(cfg.t, 4, 3) if omode == "chen" else
-                  B.mebptt_plan_chen_recursive(cfg.t, om, 4, 3) if omode == "chenrec" else dp.plan(omode, om))
-            om = op.m
+                  B.mebptt_plan_chen_recursive(cfg.t, om, 4, 3) if omode == "chenrec" else
+                  B.mebptt_plan_bytes_exact(dp.desc, om * unit_b, True) if omode == "msmx" else
+                  dp.plan("msm", om, beta=3) if omode == "msm3" else dp.plan(omode, om))
+            om = op.m if omode != "msmx" else om
             oms, _ = timed(op, max(2, args.steps // 2), 1)
             oms = max_over(oms)
             budgets.append({"mode": omode, "m": om, "C": op.cost, "ms_per_step": oms,
                             "seq_steps_per_s": world * cfg.t / (oms * 1e-3),
                             "ratio_vs_full": oms / ms_full, "paper_model_ratio": (op.cost / cfg.t + 2) / 3,
-                            "arena_bytes": op.arena_units * B.mebptt_lstm_unit_bytes(dp.desc)})
+                            "arena_bytes": op.arena_units * unit_b // op.sigma})
 
     # end to end: host buffers in, host buffers out
     e2e = None
@@ -434,6 +476,7 @@ def main():
             "metric": "lstm_bptt_seq_steps_per_s", "value": job_value(world, cfg.t, ms), "unit": "seq-steps/s",
             "n_gpus": world, "steps": args.steps, "warmup": W, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "host_enqueue_ms": host_enqueue_ms,
             "config": {"workload": f"{cfg.name}: L{cfg.layers} I{cfg.input} H{cfg.hidden} B{cfg.batch} t{cfg.t} O{cfg.readout}",
                        "mode": mode, "m": plan.m, "alpha": plan.alpha, "C": plan.cost,
                        "train_steps_per_s": world / (ms * 1e-3),

@@ -277,6 +277,18 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc *desc, const mebptt_plan
  * Workspace: caller-owned, 256-byte aligned, >= mebptt_lstm_workspace_bytes(); contents on
  *   entry do not matter and are undefined on exit.
  * stream: a cudaStream_t (NULL = the default stream).
+ * Streams and events owned by the library: on the tensor-core path for one-layer bfloat16
+ *   problems, the first step on a device creates, and keeps until the process ends, two
+ *   non-blocking streams and 22 events without timing.  On the first (lowest priority) run the
+ *   weight-gradient contractions and bias sums of a finished chunk of time steps, inside the
+ *   caller's workspace and output buffers, while the caller's stream goes on with the next chunk;
+ *   events order them after the backward steps they read and before the reuse of their staging
+ *   buffers, and the caller's stream waits for them before the step's last kernel.  The second
+ *   carries the host-to-device copies of mebptt_lstm_train_step_host that overlap the forward
+ *   pass.  Everything the call enqueues is therefore complete when `stream` has reached the end
+ *   of the call's work; the caller needs no knowledge of the two streams, but must not use the
+ *   workspace or the outputs on other streams before that.  mebptt_lstm_train_step_static uses
+ *   neither stream.
  * Outputs (overwritten, not accumulated; all float32):
  *   loss [1]; dW like W; db like b; dW_out [O][H]; db_out [O]; dx [t][B][I] or NULL.
  *   counters: int64[8] -- [0] forward operations executed, [1] backward operations executed,
@@ -309,6 +321,32 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc *desc, const mebptt_plan_
                                 void *workspace, size_t workspace_bytes, void *stream,
                                 float *loss, float *dW, float *db, float *dW_out, float *db_out,
                                 float *dx, int64_t *counters);
+
+/*
+ * Mixed memorisation over the layout's real sizes.  Section 3.3 counts memory in hidden states and
+ * wants the internal state to be a whole number alpha of them; where it is not (bfloat16 h and
+ * gates with a float32 cell state: 20/6 of a hidden state, 14/6 without the input state) rounding
+ * up plans memory that is never used.  Section 3.3 calls alpha application-specific and Appendix C
+ * works with slots of arbitrary sizes; here the recursion of Eqs. (6)-(10) runs over a finer unit:
+ *
+ *   mebptt_plan_sized(t, m, sigma, alpha, beta)  BPTT-MSM where a hidden state takes sigma units of
+ *       m, an internal state alpha, one without its input hidden state beta (0: Section 3.4 off);
+ *       Q1 recurses on m - sigma, the start state occupies sigma units.  sigma = 1 is
+ *       mebptt_plan_ex(MEBPTT_MSM).  1 <= sigma <= 64, sigma <= alpha <= 64 sigma.  Tape locations,
+ *       peak and arena units of such a plan are in the same finer unit.
+ *   mebptt_plan_bytes_exact(desc, bytes, use_beta, include_working)  takes as the unit the
+ *       greatest common divisor of the byte sizes of the three kinds of state in desc's layout
+ *       (config 5: 1 MiB, sizes 3 : 10 : 7), converts the byte budget and plans as above; with
+ *       include_working the budget covers the whole device workspace, as in mebptt_plan_for_bytes.
+ *   mebptt_plan_sigma  the sigma of a plan (1 for every other constructor).
+ *
+ * A plan can be executed with a descriptor whose layout fits its sizes (checked; else
+ * MEBPTT_ERR_UNSUPPORTED).
+ */
+int mebptt_plan_sized(int64_t t, int64_t m, int sigma, int alpha, int beta, mebptt_plan_t **out);
+int mebptt_plan_bytes_exact(const mebptt_lstm_desc *desc, size_t budget_bytes, int use_beta,
+                            int include_working, mebptt_plan_t **out);
+int mebptt_plan_sigma(const mebptt_plan_t *plan);
 
 /*
  * What a training step derives from (descriptor, plan, workspace address, device) alone -- the

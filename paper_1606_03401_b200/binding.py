@@ -67,6 +67,9 @@ _SIGS = {
     "mebptt_plan_t_len": (_i64, [_vp]),
     "mebptt_plan_m": (_i64, [_vp]),
     "mebptt_plan_mode": (_i32, [_vp]),
+    "mebptt_plan_sized": (_i32, [_i64, _i64, _i32, _i32, _i32, C.POINTER(_vp)]),
+    "mebptt_plan_bytes_exact": (_i32, [_descp, _sz, _i32, _i32, C.POINTER(_vp)]),
+    "mebptt_plan_sigma": (_i32, [_vp]),
     "mebptt_plan_alpha": (_i32, [_vp]),
     "mebptt_plan_beta": (_i32, [_vp]),
     "mebptt_plan_tables": (_i32, [_vp, C.POINTER(C.POINTER(C.c_int64)), C.POINTER(C.POINTER(C.c_int32)),
@@ -133,6 +136,7 @@ class Plan:
     t = property(lambda self: lib.mebptt_plan_t_len(self._h))
     m = property(lambda self: lib.mebptt_plan_m(self._h))
     mode = property(lambda self: lib.mebptt_plan_mode(self._h))
+    sigma = property(lambda self: lib.mebptt_plan_sigma(self._h))
     alpha = property(lambda self: lib.mebptt_plan_alpha(self._h))
     beta = property(lambda self: lib.mebptt_plan_beta(self._h))
 
@@ -213,6 +217,19 @@ def mebptt_plan_for_bytes(desc, nbytes: int, mode: int, include_working: bool = 
     h = _vp()
     _check(lib.mebptt_plan_for_bytes(C.byref(desc), nbytes, mode, int(include_working), C.byref(h)),
            "mebptt_plan_for_bytes")
+    return Plan(h)
+
+
+def mebptt_plan_sized(t: int, m: int, sigma: int, alpha: int, beta: int = 0) -> Plan:
+    h = _vp()
+    _check(lib.mebptt_plan_sized(t, m, sigma, alpha, beta, C.byref(h)), "mebptt_plan_sized")
+    return Plan(h)
+
+
+def mebptt_plan_bytes_exact(desc, nbytes: int, use_beta: bool = True, include_working: bool = False) -> Plan:
+    h = _vp()
+    _check(lib.mebptt_plan_bytes_exact(C.byref(desc), nbytes, int(use_beta), int(include_working), C.byref(h)),
+           "mebptt_plan_bytes_exact")
     return Plan(h)
 
 

@@ -7,6 +7,7 @@
 #include <cstring>
 #include <vector>
 
+#include "env.hpp"
 #include "kernels.hpp"
 #include "layout.hpp"
 #include "mebptt.h"
@@ -25,7 +26,7 @@ inline char* loc_base(const Layout& y, char* ws, int32_t loc) {
     case MEBPTT_LOC_PING: return ws + y.off_ping;
     case MEBPTT_LOC_PONG: return ws + y.off_pong;
     case MEBPTT_LOC_CORE: return ws + y.off_core;
-    default: return ws + y.off_arena + (size_t)loc * y.unit;
+    default: return ws + y.off_arena + (size_t)loc * y.loc_bytes;
   }
 }
 
@@ -41,21 +42,68 @@ inline void hidden_at(const Layout& y, const StepIO& io, int32_t loc, int l, con
   }
 }
 
+// Where layer l of a forward operation finds its input state and puts its output state.
+struct FwdPtrs {
+  const void* h_prev; const float* c_prev;
+  void* h_out; float* c_out;
+  void* gates;                       // NULL: the destination holds a hidden state only
+  void* h_in_copy; float* c_in_copy; // NULL unless the destination is a whole internal state
+};
+inline FwdPtrs fwd_ptrs(const Layout& y, const StepIO& io, const mebptt_op& op, int l) {
+  FwdPtrs f{};
+  char* dst = loc_base(y, io.ws, op.dst);
+  hidden_at(y, io, op.src, l, &f.h_prev, &f.c_prev);
+  f.h_out = dst + y.h_off(l);
+  f.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
+  if (op.dst_fmt != MEBPTT_FMT_HIDDEN) f.gates = dst + y.rec_gates + (size_t)l * y.gsz;
+  if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+    f.h_in_copy = dst + y.rec_in + y.h_off(l);
+    f.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
+  }
+  return f;
+}
+// What layer l of a backward operation reads of its internal state, and the layer's input at that step.
+struct BwdPtrs {
+  const void* gates; const float* c_t;
+  const void* h_prev; const float* c_prev;
+  const void* in;
+};
+inline BwdPtrs bwd_ptrs(const Layout& y, const StepIO& io, const mebptt_op& op, int l) {
+  BwdPtrs b{};
+  char* rec = loc_base(y, io.ws, op.src);
+  b.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+  b.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
+  if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
+    b.h_prev = rec + y.rec_in + y.h_off(l);
+    b.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
+  } else {
+    hidden_at(y, io, op.aux, l, &b.h_prev, &b.c_prev);
+  }
+  b.in = (l == 0) ? (const void*)(io.x + (size_t)(op.k - 1) * y.B * y.I * y.esz) : (const void*)(rec + y.h_off(l - 1));
+  return b;
+}
+
 int check_common(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
   if (!valid_desc(desc) || !plan) return MEBPTT_ERR_ARG;
   const Plan* p = reinterpret_cast<const Plan*>(plan);
   if (p->t != desc->t) return MEBPTT_ERR_ARG;
-  // the LSTM's internal state needs 4 units (3 without its input hidden state)
-  if (p->mode != MEBPTT_HSM && p->alpha < 4) return MEBPTT_ERR_UNSUPPORTED;
-  if (p->mode == MEBPTT_MSM && p->beta != 0 && p->beta < 3) return MEBPTT_ERR_UNSUPPORTED;
+  // the plan's sizes must hold this layout's states: a hidden state is sigma units of the plan, and
+  // its internal states (alpha units; beta without the input hidden state) must fit theirs.  With
+  // sigma = 1 that is alpha >= 4 and beta >= 3 for every layout of this library.
+  Layout y;
+  state_layout(desc, y);
+  const size_t sg = (size_t)(p->sigma > 0 ? p->sigma : 1);
+  if (y.unit % sg != 0 || (y.unit / sg) % y.granule != 0) return MEBPTT_ERR_UNSUPPORTED;
+  const size_t loc_bytes = y.unit / sg;
+  if (p->mode != MEBPTT_HSM && (size_t)p->alpha * loc_bytes < y.rec) return MEBPTT_ERR_UNSUPPORTED;
+  if (p->mode == MEBPTT_MSM && p->beta != 0 && (size_t)p->beta * loc_bytes < y.rec_in) return MEBPTT_ERR_UNSUPPORTED;
   return MEBPTT_OK;
 }
 
 int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const StepIO& io, cudaStream_t s,
              bool side_stream = true) {
   if (y.tensor_path) {
-    static const bool no_overlap = getenv("MEBPTT_NO_OVERLAP") != nullptr;
-    return (int)tc::run_step(y, p, io, desc->want_dx != 0, s, false, side_stream && !no_overlap);
+    return (int)tc::run_step(y, p, io, desc->want_dx != 0, s, false, side_stream && !env::no_overlap());
   }
   const size_t bh = (size_t)y.B * y.H;
   const size_t plane_elems = y.plane / y.esz;
@@ -134,18 +182,13 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
       char* dst = loc_base(y, ws, op.dst);
       for (int l = 0; l < y.L; ++l) {
         generic::FwdArgs a{};
-        hidden_at(y, io, op.src, l, &a.h_prev, &a.c_prev);
+        const FwdPtrs f = fwd_ptrs(y, io, op, l);
+        a.h_prev = f.h_prev; a.c_prev = f.c_prev; a.h_out = f.h_out; a.c_out = f.c_out;
+        a.gates = f.gates; a.h_in_copy = f.h_in_copy; a.c_in_copy = f.c_in_copy;
         a.in = (l == 0) ? (const void*)x_k : (const void*)(dst + y.h_off(l - 1));
         a.I = (l == 0) ? y.I : y.H;
         a.W = io.W + y.w_layer_offset(l) * y.esz;
         a.bias = io.b + (size_t)l * 4 * y.H;
-        a.h_out = dst + y.h_off(l);
-        a.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
-        if (op.dst_fmt != MEBPTT_FMT_HIDDEN) a.gates = dst + y.rec_gates + (size_t)l * y.gsz;
-        if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-          a.h_in_copy = dst + y.rec_in + y.h_off(l);
-          a.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
-        }
         a.plane_elems = plane_elems;
         a.B = y.B; a.H = y.H;
         a.counters = (l == 0) ? io.counters : nullptr;
@@ -175,16 +218,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.dha = dha;
         a.dh_rec = dh_rec + (size_t)l * bh;
         a.dc_rec = dc_rec + (size_t)l * bh;
-        a.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+        const BwdPtrs q = bwd_ptrs(y, io, op, l);
+        a.gates = q.gates; a.c_t = q.c_t; a.h_prev = q.h_prev; a.c_prev = q.c_prev; a.in = q.in;
         a.plane_elems = plane_elems;
-        a.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
-        if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-          a.h_prev = rec + y.rec_in + y.h_off(l);
-          a.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
-        } else {
-          hidden_at(y, io, op.aux, l, &a.h_prev, &a.c_prev);
-        }
-        a.in = (l == 0) ? (const void*)x_k : (const void*)(rec + y.h_off(l - 1));
         a.I = (l == 0) ? y.I : y.H;
         a.W = io.W + y.w_layer_offset(l) * y.esz;
         a.dz = dz;
@@ -212,7 +248,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   // input products, the readout and the gradients handed down are then batched over the run);
   // everything else, and the leaves of the recursion, go operation by operation.  Both give the
   // same bits; MEBPTT_STEPWISE_PER_OP=1 keeps to single operations (the tests compare the two).
-  const bool per_op_only = getenv("MEBPTT_STEPWISE_PER_OP") != nullptr;
+  const bool per_op_only = env::stepwise_per_op();
   if (!(y.stepwise_tc || y.stepwise_x3) || per_op_only) {
     for (const mebptt_op& op : p->tape) {
       if (rc != MEBPTT_OK) break;
@@ -237,18 +273,11 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         const int64_t k0 = ops[0].k;
         for (int l = 0; l < y.L && rc == MEBPTT_OK; ++l) {
           for (int j = 0; j < n; ++j) {
-            const mebptt_op& op = ops[j];
-            char* dst = loc_base(y, ws, op.dst);
+            const FwdPtrs q = fwd_ptrs(y, io, ops[j], l);
             stepwise::FwdRunStep& f = fst[j];
             f = stepwise::FwdRunStep{};
-            hidden_at(y, io, op.src, l, &f.h_prev, &f.c_prev);
-            f.h_out = dst + y.h_off(l);
-            f.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
-            if (op.dst_fmt != MEBPTT_FMT_HIDDEN) f.gates = dst + y.rec_gates + (size_t)l * y.gsz;
-            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-              f.h_in_copy = dst + y.rec_in + y.h_off(l);
-              f.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
-            }
+            f.h_prev = q.h_prev; f.c_prev = q.c_prev; f.h_out = q.h_out; f.c_out = q.c_out;
+            f.gates = q.gates; f.h_in_copy = q.h_in_copy; f.c_in_copy = q.c_in_copy;
           }
           const int I_l = l == 0 ? y.I : y.H;
           const float* in = (l == 0) ? reinterpret_cast<const float*>(io.x) + (size_t)(k0 - 1) * y.B * y.I : x3.h_run;
@@ -274,16 +303,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
             b.dha = (l == y.L - 1) ? x3.dha_run + (size_t)a * bh : dha;
             b.dh_rec = dh_rec + (size_t)l * bh;
             b.dc_rec = dc_rec + (size_t)l * bh;
-            b.gates = rec + y.rec_gates + (size_t)l * y.gsz;
+            const BwdPtrs q = bwd_ptrs(y, io, op, l);
+            b.gates = q.gates; b.c_t = q.c_t; b.h_prev = q.h_prev; b.c_prev = q.c_prev; b.in = q.in;
             b.plane_elems = plane_elems;
-            b.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
-            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-              b.h_prev = rec + y.rec_in + y.h_off(l);
-              b.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
-            } else {
-              hidden_at(y, io, op.aux, l, &b.h_prev, &b.c_prev);
-            }
-            b.in = (l == 0) ? (const void*)x_k : (const void*)(rec + y.h_off(l - 1));
             b.I = (l == 0) ? y.I : y.H;
             b.W = io.W + y.w_layer_offset(l) * y.esz;
             b.dz = dz;
@@ -305,18 +327,11 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         const int64_t k0 = ops[0].k;
         for (int l = 0; l < y.L && rc == MEBPTT_OK; ++l) {
           for (int j = 0; j < n; ++j) {
-            const mebptt_op& op = ops[j];
-            char* dst = loc_base(y, ws, op.dst);
+            const FwdPtrs q = fwd_ptrs(y, io, ops[j], l);
             stepwise::FwdRunStep& f = fst[j];
             f = stepwise::FwdRunStep{};
-            hidden_at(y, io, op.src, l, &f.h_prev, &f.c_prev);
-            f.h_out = dst + y.h_off(l);
-            f.c_out = reinterpret_cast<float*>(dst + y.c_off(l));
-            if (op.dst_fmt != MEBPTT_FMT_HIDDEN) f.gates = dst + y.rec_gates + (size_t)l * y.gsz;
-            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-              f.h_in_copy = dst + y.rec_in + y.h_off(l);
-              f.c_in_copy = reinterpret_cast<float*>(dst + y.rec_in + y.c_off(l));
-            }
+            f.h_prev = q.h_prev; f.c_prev = q.c_prev; f.h_out = q.h_out; f.c_out = q.c_out;
+            f.gates = q.gates; f.h_in_copy = q.h_in_copy; f.c_in_copy = q.c_in_copy;
           }
           const void* in = (l == 0) ? (const void*)(io.x + (size_t)(k0 - 1) * y.B * y.I * y.esz) : (const void*)tcw.hrun;
           rc = stepwise::forward_run_layer(fst.data(), n, in, l == 0 ? y.I : y.H, io.W + y.w_layer_offset(l) * y.esz,
@@ -334,18 +349,9 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
                                    loss_t + (k_lo - 1), y.B, y.H, y.O, tcw, s);
         for (int l = y.L - 1; l >= 0 && rc == MEBPTT_OK; --l) {
           for (int a = 0; a < n; ++a) {
-            const mebptt_op& op = op_at(a);
-            char* rec = loc_base(y, ws, op.src);
+            const BwdPtrs q = bwd_ptrs(y, io, op_at(a), l);
             stepwise::BwdRunStep& b = bst[a];
-            b.gates = rec + y.rec_gates + (size_t)l * y.gsz;
-            b.c_t = reinterpret_cast<const float*>(rec + y.c_off(l));
-            if (op.dst_fmt == MEBPTT_FMT_INTERNAL) {
-              b.h_prev = rec + y.rec_in + y.h_off(l);
-              b.c_prev = reinterpret_cast<const float*>(rec + y.rec_in + y.c_off(l));
-            } else {
-              hidden_at(y, io, op.aux, l, &b.h_prev, &b.c_prev);
-            }
-            b.in = (l == 0) ? (const void*)(io.x + (size_t)(op.k - 1) * y.B * y.I * y.esz) : (const void*)(rec + y.h_off(l - 1));
+            b.gates = q.gates; b.c_t = q.c_t; b.h_prev = q.h_prev; b.c_prev = q.c_prev; b.in = q.in;
           }
           float* d_lo = (l > 0) ? tcw.dha_run : (desc->want_dx ? io.dx + (size_t)(k_lo - 1) * y.B * y.I : nullptr);
           rc = stepwise::backward_run_layer(bst.data(), n, s_lo, l, l == 0 ? y.I : y.H, io.W + y.w_layer_offset(l) * y.esz,
@@ -430,10 +436,41 @@ int mebptt_plan_for_bytes(const mebptt_lstm_desc* desc, size_t budget_bytes, int
   return MEBPTT_ERR_BUDGET;
 }
 
+int mebptt_plan_bytes_exact(const mebptt_lstm_desc* desc, size_t budget_bytes, int use_beta, int include_working,
+                            mebptt_plan_t** out) {
+  if (!out || !valid_desc(desc)) return MEBPTT_ERR_ARG;
+  *out = nullptr;
+  Layout y;
+  state_layout(desc, y);
+  // the finest unit in which a hidden state, an internal state and one without its input state are
+  // all whole: their greatest common divisor (a multiple of the layout's granule, as they are)
+  const size_t rec_short = y.rec_in;   // output hidden state + gate planes
+  const size_t f = gcd_sz(gcd_sz(y.unit, y.rec), rec_short);
+  const int sigma = (int)(y.unit / f), alpha = (int)(y.rec / f), beta = use_beta ? (int)(rec_short / f) : 0;
+  if (sigma > 64) return MEBPTT_ERR_UNSUPPORTED;
+  int64_t m = (int64_t)(budget_bytes / f);
+  for (int round = 0; round < 64 && m >= sigma; ++round) {
+    mebptt_plan_t* plan = nullptr;
+    const int rc = mebptt_plan_sized(desc->t, m, sigma, alpha, beta, &plan);
+    if (rc != MEBPTT_OK) return rc;
+    if (!include_working) { *out = plan; return MEBPTT_OK; }
+    const size_t need = mebptt_lstm_workspace_bytes(desc, plan);
+    if (need == 0) { mebptt_plan_free(plan); return MEBPTT_ERR_UNSUPPORTED; }
+    if (need <= budget_bytes) { *out = plan; return MEBPTT_OK; }
+    const int64_t m_used = mebptt_plan_m(plan);
+    mebptt_plan_free(plan);
+    const int64_t drop = (int64_t)((need - budget_bytes + f - 1) / f);
+    m = (m_used < m ? m_used : m) - (drop > 0 ? drop : 1);
+  }
+  return MEBPTT_ERR_BUDGET;
+}
+
 size_t mebptt_lstm_workspace_bytes(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan) {
   if (check_common(desc, plan) != MEBPTT_OK) return 0;
   Layout y;
   workspace_layout(desc, reinterpret_cast<const Plan*>(plan), y);
+  // the persistent kernels address the workspace in 16-byte units held in 32 bits
+  if (y.tensor_path && y.total >= ((size_t)1 << 36)) return 0;
   return y.total;
 }
 
@@ -517,6 +554,7 @@ int train_step_impl(const mebptt_lstm_desc* desc, const mebptt_plan_t* plan, con
   const Plan* p = reinterpret_cast<const Plan*>(plan);
   Layout y;
   workspace_layout(desc, p, y);
+  if (y.tensor_path && y.total >= ((size_t)1 << 36)) return MEBPTT_ERR_UNSUPPORTED;   // 16-byte offsets in 32 bits
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < y.total)
     return MEBPTT_ERR_WORKSPACE;
   StepIO io{(const char*)W, (const char*)W_out, (const char*)x, (const char*)h0,
@@ -575,8 +613,7 @@ int mebptt_lstm_train_step_host(const mebptt_lstm_desc* desc, const mebptt_plan_
   cudaMemcpyAsync(ws + g.c0, c0, g.nc0, cudaMemcpyHostToDevice, s);
   // x is read progressively by the forward pass and the targets not before the first backward
   // operation: the tensor-core path copies both beside the forward pass
-  static const bool no_overlap = getenv("MEBPTT_NO_OVERLAP") != nullptr;
-  const bool late_targets = y.tensor_path && !no_overlap;
+  const bool late_targets = y.tensor_path && !env::no_overlap();
   if (!late_targets) {
     cudaMemcpyAsync(ws + g.x, x, g.nx, cudaMemcpyHostToDevice, s);
     cudaMemcpyAsync(ws + g.targets, targets, g.ntargets, cudaMemcpyHostToDevice, s);

@@ -9,12 +9,11 @@
 #include <atomic>
 #include <cstdlib>
 
+#include "env.hpp"
+
 namespace mebptt {
 
-inline bool pdl_enabled() {
-  static const bool on = getenv("MEBPTT_NO_PDL") == nullptr;
-  return on;
-}
+inline bool pdl_enabled() { return !env::no_pdl(); }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_on(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

@@ -37,6 +37,7 @@ struct Layout {
   size_t gsz = 0;        // one layer's four gate planes
   size_t plane = 0;      // one gate plane
   size_t unit = 0;       // one hidden state of the stack
+  size_t loc_bytes = 0;  // what one unit of a tape location (and of the plan's budget m) is in bytes: unit / sigma
   size_t rec = 0;        // one internal state
   // record-relative offsets
   size_t rec_gates = 0;  // gates of layer 0
@@ -205,9 +206,10 @@ inline std::vector<WorkItem> work_items(const Plan* p, int S) {
 inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y) {
   state_layout(d, y);
   y.arena_units = p->arena_units;
+  y.loc_bytes = y.unit / (size_t)(p->sigma > 0 ? p->sigma : 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, y.granule); return r; };
-  y.off_arena = take((size_t)y.arena_units * y.unit);
+  y.off_arena = take((size_t)y.arena_units * y.loc_bytes);
   y.off_core = take(y.rec);
   y.off_ping = take(y.unit);
   y.off_pong = take(y.unit);

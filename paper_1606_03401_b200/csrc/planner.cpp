@@ -5,6 +5,7 @@
 // split point y walks one column forwards and one backwards), then transposed once into the
 // row-major layout the C interface documents.
 #include "plan.hpp"
+#include "env.hpp"
 
 #include <algorithm>
 #include <atomic>
@@ -102,11 +103,8 @@ struct ConvexPrefix {
   }
 };
 
-inline bool plan_scan_only() {
-  // verification aid: MEBPTT_PLAN_SCAN=1 keeps the plain scan everywhere (the tests compare the two)
-  const char* e = getenv("MEBPTT_PLAN_SCAN");
-  return e && e[0] == '1';
-}
+// verification aid: keeps the plain scan everywhere (the tests compare the two)
+inline bool plan_scan_only() { return env::plan_scan(); }
 
 template <class T>
 struct Inf;
@@ -204,11 +202,16 @@ void solve_ism(int64_t t_max, int64_t m_max, Cols<T>& C, Cols<int32_t>& D) {
 }
 
 template <class T>
-void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Cols<int32_t>& D1,
+void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, int sigma, Cols<T>& C, Cols<int32_t>& D1,
                Cols<int32_t>& D2, Cols<uint8_t>& H) {
   // Section 3.3 with the reading C(0, m) = 0 for every m (also m <= 0) and C(t > 0, m <= 0) = inf.
   // Q1 = y + C(y, m) + C(t - y, m - 1), 1 <= y < t;  Q2 = y + C(y - 1, m) + C(t - y, m - a(y)),
   // 1 <= y <= t, a(y) = alpha, or beta at y = 1 when the Section 3.4 variant is on.
+  // sigma generalises the unit: where an internal state is no whole number of hidden states
+  // (Section 3.3 calls alpha application-specific; Appendix C has slots of arbitrary sizes), m is
+  // counted in a finer unit in which a hidden state takes sigma, an internal state alpha and one
+  // without its input state beta: Q1 then recurses on m - sigma, and a budget below sigma cannot
+  // even hold the start state of a sequence.
   const T INF = Inf<T>::v;
   std::vector<T> nonpos((size_t)t_max + 1, INF);  // the column of any budget <= 0
   nonpos[0] = 0;
@@ -218,7 +221,7 @@ void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Co
     std::fill(D2.col(m), D2.col(m) + t_max + 1, 0);
     std::fill(H.col(m), H.col(m) + t_max + 1, (uint8_t)0);
   }
-  auto column = [&](int64_t m) -> const T* { return m <= 0 ? nonpos.data() : C.col(m); };
+  auto column = [&](int64_t m) -> const T* { return m < sigma ? nonpos.data() : C.col(m); };
   // The columns of this mode are not convex in t, so every cell is a scan; what is left to gain is
   // that cell (t, m) needs the columns m - 1, m - alpha, m - beta only up to row t - 1.  Several
   // threads therefore fill consecutive columns at once, each a few rows behind the columns it
@@ -226,24 +229,24 @@ void solve_msm(int64_t t_max, int64_t m_max, int alpha, int beta, Cols<T>& C, Co
   std::vector<std::atomic<int64_t>> rows((size_t)m_max + 1);
   for (auto& r : rows) r.store(0, std::memory_order_relaxed);
   auto wait_for = [&](int64_t m, int64_t upto) -> int64_t {   // until column m is filled up to row `upto`; how far it is
-    if (m <= 0) return t_max;
+    if (m < sigma) return t_max;
     int64_t got;
     while ((got = rows[(size_t)m].load(std::memory_order_acquire)) < upto) std::this_thread::yield();
     return got;
   };
-  std::atomic<int64_t> next_column{1};
+  std::atomic<int64_t> next_column{sigma};   // columns below sigma stay infinite (row 0 apart)
   auto worker = [&]() {
    for (;;) {
     const int64_t m = next_column.fetch_add(1, std::memory_order_relaxed);
     if (m > m_max) return;
     T* c = C.col(m);
-    const T* cm1 = column(m - 1);
+    const T* cm1 = column(m - sigma);
     const T* cma = column(m - alpha);
     const T* cmb = beta > 0 ? column(m - beta) : nullptr;
     int64_t sure = 0;   // rows of the columns read that are known to be there
     for (int64_t t = 1; t <= t_max; ++t) {
       if (sure < t - 1) {
-        sure = std::min(wait_for(m - 1, t - 1), wait_for(m - alpha, t - 1));
+        sure = std::min(wait_for(m - sigma, t - 1), wait_for(m - alpha, t - 1));
         if (cmb) sure = std::min(sure, wait_for(m - beta, t - 1));
       }
       T c1 = INF, c2 = INF;
@@ -319,7 +322,7 @@ void solve(Plan& p) {
   } else {
     Cols<int32_t> D2(t, m, 0);
     Cols<uint8_t> H(t, m, 0);
-    solve_msm<T>(t, m, p.alpha, p.beta, C, D, D2, H);
+    solve_msm<T>(t, m, p.alpha, p.beta, p.sigma, C, D, D2, H);
     transpose_into(D2, p.D2);
     transpose_into(H, p.H);
   }
@@ -334,7 +337,7 @@ struct Emitter {
   Plan& p;
   int64_t units;      // paper's accounting
   int64_t top = 0;    // physical arena top, hidden-state units
-  explicit Emitter(Plan& pl) : p(pl), units(pl.mode == MEBPTT_ISM ? 0 : 1) { p.peak_units = units; }
+  explicit Emitter(Plan& pl) : p(pl), units(pl.mode == MEBPTT_ISM ? 0 : pl.sigma) { p.peak_units = units; }
 
   int64_t Cat(int64_t t, int64_t m) const { return p.C[(size_t)t * (p.m + 1) + m]; }
   int32_t Dat(int64_t t, int64_t m) const { return p.D[(size_t)t * (p.m + 1) + m]; }
@@ -417,15 +420,15 @@ struct Emitter {
 
   // Section 3.3 (and 3.4 when beta > 0).
   void msm(int64_t t, int64_t m, int64_t s, int32_t loc) {
-    const int a = p.alpha, b = p.beta;
+    const int a = p.alpha, b = p.beta, sg = p.sigma;
     while (t > 0) {
       if (Hat(t, m) == 1) {
         const int64_t y = Dat(t, m);
         const int32_t slot = (int32_t)top;
-        grow(1, 1);
+        grow(sg, sg);
         sweep(s, y, loc, slot, MEBPTT_FMT_HIDDEN);
-        msm(t - y, m - 1, s + y, slot);
-        shrink(1, 1);
+        msm(t - y, m - sg, s + y, slot);
+        shrink(sg, sg);
         t = y;
       } else {
         const int64_t y = D2at(t, m);
@@ -602,21 +605,22 @@ int build_chen_recursive_plan(int64_t t, int k, int alpha, int beta, Plan** out)
   return MEBPTT_OK;
 }
 
-int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out) {
+int build_plan(int64_t t, int64_t m, int mode, int alpha, int beta, Plan** out, int sigma) {
   if (!out) return MEBPTT_ERR_ARG;
   *out = nullptr;
   if (t < 1 || t > (int64_t)1 << 24) return MEBPTT_ERR_ARG;
   if (mode != MEBPTT_HSM && mode != MEBPTT_ISM && mode != MEBPTT_MSM) return MEBPTT_ERR_ARG;
-  if (alpha < 2 || alpha > 64) return MEBPTT_ERR_ARG;
-  if (beta < 0 || beta > alpha) return MEBPTT_ERR_ARG;
+  if (sigma < 1 || sigma > 64 || (sigma > 1 && mode != MEBPTT_MSM)) return MEBPTT_ERR_ARG;
+  if (alpha < 2 || alpha < sigma || alpha > 64 * sigma) return MEBPTT_ERR_ARG;
+  if (beta < 0 || beta > alpha || (beta > 0 && beta < sigma)) return MEBPTT_ERR_ARG;
   if (m < 1) return MEBPTT_ERR_BUDGET;
   if (mode != MEBPTT_MSM) beta = 0;
   // beyond saturation more memory changes nothing
-  const int64_t sat = (mode == MEBPTT_MSM) ? std::max<int64_t>(1, (int64_t)alpha * (t - 1) + 1) : t;
+  const int64_t sat = (mode == MEBPTT_MSM) ? std::max<int64_t>(1, (int64_t)alpha * (t - 1) + sigma) : t;
   m = std::min(m, sat);
   Plan* p = new_plan();
   if (!p) return MEBPTT_ERR_OOM;
-  p->t = t; p->m = m; p->mode = mode; p->alpha = alpha; p->beta = beta;
+  p->t = t; p->m = m; p->mode = mode; p->alpha = alpha; p->beta = beta; p->sigma = sigma;
   try {
     if (t * (t + 1) / 2 + t < (int64_t)Inf<int32_t>::v) solve<int32_t>(*p);
     else solve<int64_t>(*p);
@@ -649,7 +653,7 @@ int validate_plan(const Plan& p) {
   int64_t next_bwd = p.t, forwards = 0, peak = 0;
   const int a = p.alpha, b = p.beta;
   auto rec_units = [&](int fmt) -> int64_t {
-    if (fmt == MEBPTT_FMT_HIDDEN) return 1;
+    if (fmt == MEBPTT_FMT_HIDDEN) return p.sigma;
     if (fmt == MEBPTT_FMT_INTERNAL) return a;
     return b;
   };
@@ -742,6 +746,10 @@ int64_t mebptt_plan_arena_units(const mebptt_plan_t* plan) { return plan ? P_(pl
 int64_t mebptt_plan_t_len(const mebptt_plan_t* plan) { return plan ? P_(plan)->t : -1; }
 int64_t mebptt_plan_m(const mebptt_plan_t* plan) { return plan ? P_(plan)->m : -1; }
 int mebptt_plan_mode(const mebptt_plan_t* plan) { return plan ? P_(plan)->mode : -1; }
+int mebptt_plan_sized(int64_t t, int64_t m, int sigma, int alpha, int beta, mebptt_plan_t** out) {
+  return mebptt::build_plan(t, m, MEBPTT_MSM, alpha, beta, reinterpret_cast<Plan**>(out), sigma);
+}
+int mebptt_plan_sigma(const mebptt_plan_t* plan) { return plan ? P_(plan)->sigma : -1; }
 int mebptt_plan_alpha(const mebptt_plan_t* plan) { return plan ? P_(plan)->alpha : -1; }
 int mebptt_plan_beta(const mebptt_plan_t* plan) { return plan ? P_(plan)->beta : -1; }
 

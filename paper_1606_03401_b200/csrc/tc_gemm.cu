@@ -362,8 +362,7 @@ __global__ void splitk_reduce(const float* partial, int splits, int M, int N, in
 // operands, each part at least 8 blocks of 64 long; a second kernel adds the parts.  Only where at
 // least four parts come out of it: below that the extra pass costs more than it saves.
 int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_floats) {
-  static const bool no_split = getenv("MEBPTT_NO_SPLITK") != nullptr;
-  if (no_split) return 1;
+  if (env::no_splitk()) return 1;
   const int wide_tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
   const bool narrow = !a_mn && !b_mn && wide_tiles <= 37 && N >= 2 * BN_NARROW;
   const int BN = narrow ? BN_NARROW : BN_WIDE;
@@ -377,8 +376,7 @@ int gemm_split_count(bool a_mn, bool b_mn, int M, int N, int K, size_t partial_f
 }
 
 int gemm_split_count_deferred(int M, int N, int K) {
-  static const bool no_split = getenv("MEBPTT_NO_SPLITK") != nullptr;
-  if (no_split) return 1;
+  if (env::no_splitk()) return 1;
   const int tiles = ((N + BN_WIDE - 1) / BN_WIDE) * ((M + BM - 1) / BM);
   const int nk = (K + BK - 1) / BK;
   int want = 148 / tiles;

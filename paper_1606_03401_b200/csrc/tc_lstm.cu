@@ -1089,8 +1089,7 @@ inline uint32_t off16(size_t byte_off) { return (uint32_t)(byte_off >> 4); }
 // With MEBPTT_DEBUG set in the environment, failed CUDA calls are named on stderr.
 inline bool cuda_ok(cudaError_t e, const char* what) {
   if (e == cudaSuccess) return true;
-  static const bool verbose = getenv("MEBPTT_DEBUG") != nullptr;
-  if (verbose) fprintf(stderr, "mebptt: %s failed: %s\n", what, cudaGetErrorString(e));
+  if (env::debug()) fprintf(stderr, "mebptt: %s failed: %s\n", what, cudaGetErrorString(e));
   return false;
 }
 
@@ -1301,7 +1300,7 @@ void build_host_part(Prepared& P, const Layout& y, const Plan* p, bool allow_pin
       case MEBPTT_LOC_PING: return y.off_ping;
       case MEBPTT_LOC_PONG: return y.off_pong;
       case MEBPTT_LOC_CORE: return y.off_core;
-      default: return y.off_arena + (size_t)loc * y.unit;
+      default: return y.off_arena + (size_t)loc * y.loc_bytes;
     }
   };
   const int S = y.S;
@@ -1416,10 +1415,10 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
   ok = ok && make_tmap_2d(&P.tm_wt, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, NU);
   if (!ok) { P.rc = MEBPTT_ERR_UNSUPPORTED; return; }
   // the clustered backward kernel, if the device can keep enough clusters resident
-  // (MEBPTT_BWD_CLUSTER = 0, 4 or 8 in the environment overrides the choice)
-  const char* force = getenv("MEBPTT_BWD_CLUSTER");
+  // (a switch in the environment can override the choice: env.hpp)
+  const int force = env::bwd_cluster();
   for (int cs : {8, 4}) {
-    if (force && atoi(force) != cs) continue;
+    if (force >= 0 && force != cs) continue;
     if (G % 64 != 0 || (G / 64) % cs != 0 || ncta % cs != 0 || (G / 64) / cs > 16) continue;
     const int kbs = (G / 64) / cs;
     const int tb = kbs > 8 ? 8 : 4;   // K tiles per barrier: at most four barriers, two where the slice is long

@@ -560,3 +560,34 @@ def test_prepared_set_is_reused_per_workspace_and_the_enqueue_is_cheap(H):
     host_ms, dev_ms = sorted(host)[len(host) // 2], sorted(dev)[len(dev) // 2]
     print(f"c3 msm m=100: host enqueue {host_ms:.2f} ms, device {dev_ms:.2f} ms")
     assert host_ms < 0.25 * dev_ms, (host_ms, dev_ms)
+
+
+@pytest.mark.parametrize("base,kw", [
+    ("c2", dict(input=128, hidden=256, batch=64, t=70, readout=128)),                  # persistent tensor path
+    ("c5", dict(layers=2, input=64, hidden=128, batch=32, t=45, readout=40)),           # step by step, bf16, two layers
+    ("c1", dict(t=24)),                                                                 # float32: sizes 1 : 4 : 3
+])
+def test_plans_over_the_layouts_byte_sizes_give_the_same_gradients(H, base, kw):
+    """BPTT-MSM planned over the real sizes of the layout's states (bfloat16: hidden : internal :
+    without input state = 3 : 10 : 7 units) instead of internal states rounded up to whole hidden
+    states: forward count equal to the oracle's cost for those sizes, peak within the budget, the
+    bits of the full-memory run, and never more forward operations than the rounded plan at the
+    same bytes."""
+    from paper_1606_03401_b200 import binding as B
+    cfg = _cfg(base, **kw)
+    dp = H.DeviceProblem(cfg, want_dx=True)
+    full = dp.run(dp.full_memory_plan())
+    unit = B.mebptt_lstm_unit_bytes(dp.desc)
+    for units in (3, 7, 12):
+        nbytes = units * unit
+        for use_beta in (False, True):
+            plan = B.mebptt_plan_bytes_exact(dp.desc, nbytes, use_beta)
+            assert plan.cost == P.cost(P.MSM, cfg.t, plan.m, plan.alpha, plan.beta or None, plan.sigma)
+            res = dp.run(plan)
+            assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+            assert res["counters"][2] == plan.peak_units <= plan.m
+            assert_bit_identical(res, full, want_dx=True)
+            rounded = dp.plan("msm", units, beta=3 if use_beta else 0)
+            assert plan.cost <= rounded.cost
+    if cfg.dtype == "bf16":
+        assert (plan.sigma, plan.alpha, plan.beta) == (3, 10, 7)

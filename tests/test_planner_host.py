@@ -279,3 +279,47 @@ def test_chen_recursive_schedule(beta):
     assert B.mebptt_plan_chen_recursive(20, 20, 4, 0).cost == 20
     with pytest.raises(B.MebpttError):
         B.mebptt_plan_chen_recursive(10, 0, 4, 3)
+
+
+@pytest.mark.parametrize("sigma,alpha,beta", [(3, 10, 7), (3, 10, 0), (2, 5, 3), (1, 4, 3), (5, 17, 12)])
+def test_sized_mixed_planner_matches_oracle_tables_and_replays(sigma, alpha, beta):
+    """mebptt_plan_sized (a hidden state of sigma units, internal states of alpha / beta) against
+    the oracle's recursion over the same sizes: every cost of the table, and a tape that replays
+    within the budget with exactly C(t, m) forward operations."""
+    from oracle import policy as P
+    t = 45
+    for m in [sigma, sigma + 1, alpha + sigma - 1, alpha + sigma, 3 * alpha, 7 * alpha + 2, alpha * t + sigma + 5]:
+        plan = B.mebptt_plan_sized(t, m, sigma, alpha, beta)
+        ref = P.msm_tables(t, plan.m, alpha, beta or None, sigma)[0]
+        C = plan.tables()["C"]
+        assert np.array_equal(np.minimum(C, P.INF), np.minimum(ref, P.INF)), (m,)
+        assert plan.cost == ref[t, plan.m] and plan.sigma == sigma
+        assert plan.peak_units <= plan.m and B.lib.mebptt_plan_validate(plan.handle) == 0
+        fwd = int((plan.tape()["kind"] == B.MEBPTT_OP_FWD).sum())
+        assert fwd == plan.cost
+    with pytest.raises(B.MebpttError):
+        B.mebptt_plan_sized(t, sigma - 1 if sigma > 1 else 0, sigma, alpha, beta)   # not even the start state fits
+
+
+def test_plan_bytes_exact_uses_the_layout_sizes():
+    """Config 5's layout (two layers, bfloat16 h and gates, float32 c): hidden : internal : without
+    input state = 3 : 10 : 7 units of 1 MiB.  At 1 GiB the exact sizes save forward operations
+    against internal states rounded up to 4 (3) hidden states, and never cost more."""
+    from oracle import policy as P
+    desc = B.make_desc(2, 1024, 2048, 1024, 128, 1000, "bf16")
+    exact = B.mebptt_plan_bytes_exact(desc, 1 << 30)
+    assert (exact.sigma, exact.alpha, exact.beta, exact.m) == (3, 10, 7, 1024)
+    assert exact.cost == P.cost(P.MSM, 1000, 1024, 10, 7, 3)
+    rounded = B.mebptt_plan_ex(1000, B.mebptt_budget_bytes_to_units(desc, 1 << 30), B.MEBPTT_MSM, 4, 3)
+    assert exact.cost < rounded.cost
+    assert B.mebptt_lstm_workspace_bytes(desc, exact) > 0
+    # a float32 layout is 1 : 4 : 3 already
+    d32 = B.make_desc(1, 32, 64, 32, 4, 64, "fp32")
+    p32 = B.mebptt_plan_bytes_exact(d32, 20 * B.mebptt_lstm_unit_bytes(d32))
+    assert (p32.sigma, p32.alpha, p32.beta, p32.m) == (1, 4, 3, 20)
+    # the whole workspace inside the budget
+    inside = B.mebptt_plan_bytes_exact(desc, 2 << 30, True, True)
+    assert B.mebptt_lstm_workspace_bytes(desc, inside) <= 2 << 30
+    # a plan over sizes the layout does not fit is refused at execution time (here: at sizing time)
+    tight = B.mebptt_plan_sized(1000, 300, 3, 9, 7)      # internal states one unit too small for this layout
+    assert B.mebptt_lstm_workspace_bytes(desc, tight) == 0
