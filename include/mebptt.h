@@ -230,6 +230,15 @@ enum { MEBPTT_FLAG_NO_TENSOR_CORES = 1 };
  * collected by mebptt_lstm_run_times.  Each pair costs a few microseconds of stream time, so a
  * step that is timed as a whole should not set it.  Ignored by the CUDA-core path. */
 enum { MEBPTT_FLAG_TIME_RUNS = 2 };
+/* The recurrent core is a GRU instead of an LSTM (Section 1: the method does not depend on the
+ * architecture of the core; plans, tape, budgets and every entry point are the same):
+ *     r = sigmoid(W_r [x_t ; h_{t-1}] + b_r),   z = sigmoid(W_z [x_t ; h_{t-1}] + b_z),
+ *     q = W_hn h_{t-1},   n = tanh(W_xn x_t + b_n + r q),   h_t = (1 - z) n + z h_{t-1}.
+ * W is then [3H][I_l + H] per layer (row blocks r, z, n), b [3H], and so are dW, db.  The hidden
+ * state is h alone: c0 is not read, and the cell-state part of a memory slot stays unused, so the
+ * sizes of slots and the units of m are those of the LSTM layout (alpha = 4: h_t, the planes r, z,
+ * n, q, and h_{t-1}).  Runs on the CUDA-core kernels in every precision (MEBPTT_TF32 = MEBPTT_FP32). */
+enum { MEBPTT_FLAG_GRU = 4 };
 
 /* Bytes of one hidden-state unit (all layers) for this descriptor; 0 on a bad descriptor. */
 size_t mebptt_lstm_unit_bytes(const mebptt_lstm_desc *desc);

@@ -185,6 +185,7 @@ def mebptt_plan_ex(t: int, m: int, mode: int, alpha: int = 4, beta: int = 0) -> 
 
 MEBPTT_FLAG_NO_TENSOR_CORES = 1
 MEBPTT_FLAG_TIME_RUNS = 2
+MEBPTT_FLAG_GRU = 4
 
 
 def mebptt_plan_chen_sqrt(t: int, alpha: int = 4, beta: int = 3) -> Plan:

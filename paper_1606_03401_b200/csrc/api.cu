@@ -167,7 +167,7 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
   cudaMemsetAsync(dh_rec, 0, (size_t)y.L * bh * 4, s);
   cudaMemsetAsync(dc_rec, 0, (size_t)y.L * bh * 4, s);
   cudaMemsetAsync(io.dW, 0, y.w_total_elems() * 4, s);
-  cudaMemsetAsync(io.db, 0, (size_t)y.L * 4 * y.H * 4, s);
+  cudaMemsetAsync(io.db, 0, (size_t)y.L * y.NG * y.H * 4, s);
   cudaMemsetAsync(io.dW_out, 0, (size_t)y.O * y.H * 4, s);
   cudaMemsetAsync(io.db_out, 0, (size_t)y.O * 4, s);
   cudaMemsetAsync(io.counters, 0, 8 * sizeof(int64_t), s);
@@ -188,12 +188,13 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.in = (l == 0) ? (const void*)x_k : (const void*)(dst + y.h_off(l - 1));
         a.I = (l == 0) ? y.I : y.H;
         a.W = io.W + y.w_layer_offset(l) * y.esz;
-        a.bias = io.b + (size_t)l * 4 * y.H;
+        a.bias = io.b + (size_t)l * y.NG * y.H;
         a.plane_elems = plane_elems;
         a.B = y.B; a.H = y.H;
         a.counters = (l == 0) ? io.counters : nullptr;
         if (y.stepwise_x3) rc = stepwise3::forward_step(a, x3, l, w_off[l], s);
         else if (y.stepwise_tc) rc = stepwise::forward_step(a, tcw, s);
+        else if (y.gru) generic::gru_forward_step(y.dtype, a, s);
         else generic::forward_step(y.dtype, a, s);
         if (rc != MEBPTT_OK) break;
       }
@@ -225,12 +226,13 @@ int run_step(const mebptt_lstm_desc* desc, const Plan* p, const Layout& y, const
         a.W = io.W + y.w_layer_offset(l) * y.esz;
         a.dz = dz;
         a.dW = io.dW + y.w_layer_offset(l);
-        a.db = io.db + (size_t)l * 4 * y.H;
+        a.db = io.db + (size_t)l * y.NG * y.H;
         a.d_lo = (l > 0) ? dha : (desc->want_dx ? io.dx + (size_t)(k - 1) * y.B * y.I : nullptr);
         a.B = y.B; a.H = y.H;
         a.counters = (l == y.L - 1) ? io.counters : nullptr;
         if (y.stepwise_x3) rc = stepwise3::backward_layer(a, x3, l, w_off[l], sidx, s);
         else if (y.stepwise_tc) rc = stepwise::backward_layer(a, tcw, l, sidx, s);
+        else if (y.gru) generic::gru_backward_layer(y.dtype, a, s);
         else generic::backward_layer(y.dtype, a, s);
         if (rc != MEBPTT_OK) break;
       }
@@ -380,7 +382,7 @@ void staging_layout(const Layout& y, bool want_dx, size_t base, Staging& g) {
   size_t o = base;
   auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
   const size_t bh = (size_t)y.B * y.H;
-  g.nW = y.w_total_elems() * y.esz; g.nb = (size_t)y.L * 4 * y.H * 4;
+  g.nW = y.w_total_elems() * y.esz; g.nb = (size_t)y.L * y.NG * y.H * 4;
   g.nW_out = (size_t)y.O * y.H * y.esz; g.nb_out = (size_t)y.O * 4;
   g.nx = (size_t)y.t * y.B * y.I * y.esz; g.ntargets = (size_t)y.t * y.B * y.O * 4;
   g.nh0 = (size_t)y.L * bh * y.esz; g.nc0 = (size_t)y.L * bh * 4;
@@ -536,7 +538,8 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc* desc, const mebptt_plan
     }
     return 2 * L + 2 + forwards + readouts + p->t * bwd + chunks * (3 * (2 * L + 1) + L + 1) + 1;
   }
-  return p->cost * L + p->t * (5 + 4 * L) + 1;
+  // (a GRU layer's backward operation takes two launches more: its weight gradient comes in three blocks)
+  return p->cost * L + p->t * (5 + (y.gru ? 6 : 4) * L) + 1;
 }
 
 }  // extern "C"

@@ -1,4 +1,5 @@
-// Shape-agnostic LSTM kernels: float32 FMA arithmetic on CUDA cores.
+// Shape-agnostic kernels of the recurrent cores (LSTM, and the GRU further down): float32 FMA
+// arithmetic on CUDA cores.
 //
 // This is the path of MEBPTT_FP32 (exact float32 products, which tensor cores do not offer) and
 // of every shape the tensor-core kernels do not cover.  Operands are float32 or bfloat16 in
@@ -297,6 +298,155 @@ __global__ void finalize(const float* loss_t, int64_t t, float* loss, int64_t* c
 
 inline dim3 tiles(int M, int N) { return dim3((N + TN - 1) / TN, (M + TM - 1) / TM); }
 
+// ------------------------------------------------------------------ the GRU core
+// r = sigmoid(W_r [x ; h] + b_r), z = sigmoid(W_z [x ; h] + b_z), q = W_hn h,
+// n = tanh(W_xn x + b_n + r q), h' = (1 - z) n + z h.  The forward contraction keeps the layout of
+// the LSTM one -- four adjacent columns per hidden unit -- with the columns r, z, the input part of
+// n and its recurrent part q; the four planes of an internal state hold r, z, n, q.  The hidden
+// state is h alone (the cell-state part of a slot stays unused).
+template <class T>
+struct GruFwdB {  // column 4 j + c: c = 0, 1 -> weight rows c H + j; c = 2 -> row 2H + j over the input columns, c = 3 over the recurrent ones
+  const T* W; int H, K, I;
+  __device__ float operator()(int k, int n) const {
+    const int j = n >> 2, c = n & 3;
+    if (c < 2) return ldf(W, (size_t)(c * H + j) * K + k);
+    return ((c == 2) == (k < I)) ? ldf(W, (size_t)(2 * H + j) * K + k) : 0.f;
+  }
+};
+template <class T>
+struct GruFwdEpi {
+  const float* bias; const T* h_prev; T* h_out; T* gates; T* h_in_copy;
+  int B, H; size_t plane;
+  int64_t* counters;
+  __device__ float operator()(float (&acc)[4][4], int b0, int n0, int M, int N) const {
+    const int j = n0 >> 2;
+    if (j < H) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int b = b0 + r;
+        if (b >= B) break;
+        const size_t e = (size_t)b * H + j;
+        const float gr = sigmoidf_(acc[r][0] + bias[0 * H + j]);
+        const float gz = sigmoidf_(acc[r][1] + bias[1 * H + j]);
+        const float q = acc[r][3];
+        const float gn = tanhf(fmaf(gr, q, acc[r][2] + bias[2 * H + j]));
+        const float hp = ldf(h_prev, e);
+        stf(h_out, e, fmaf(gz, hp - gn, gn));   // (1 - z) n + z h
+        if (gates) {
+          stf(gates, 0 * plane + e, gr);
+          stf(gates, 1 * plane + e, gz);
+          stf(gates, 2 * plane + e, gn);
+          stf(gates, 3 * plane + e, q);
+        }
+        if (h_in_copy) h_in_copy[e] = h_prev[e];
+      }
+    }
+    if (counters && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) counters[0] += 1;
+    return 0.f;
+  }
+  __device__ void block_result(float, int) const {}
+};
+// Gate derivatives.  dz4 [B][4H], column blocks: d r_pre, d z_pre, d n_pre, d q; dhz = dh z is the
+// part of the gradient that reaches h_{k-1} past the gates.
+template <class T>
+__global__ void gru_gate_bwd(const float* dha, const float* dh_rec, float* dhz, const T* gates, size_t plane,
+                             const T* h_prev, float* dz4, int B, int H, int64_t* counters) {
+  const size_t n = (size_t)B * H;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+    const int b = (int)(e / H), j = (int)(e % H);
+    const float gr = ldf(gates, 0 * plane + e), gz = ldf(gates, 1 * plane + e);
+    const float gn = ldf(gates, 2 * plane + e), q = ldf(gates, 3 * plane + e);
+    const float dh = dha[e] + dh_rec[e];
+    const float dn_pre = dh * (1.f - gz) * (1.f - gn * gn);
+    const float dz_pre = dh * (ldf(h_prev, e) - gn) * gz * (1.f - gz);
+    float* row = dz4 + (size_t)b * 4 * H;
+    row[0 * H + j] = dn_pre * q * gr * (1.f - gr);
+    row[1 * H + j] = dz_pre;
+    row[2 * H + j] = dn_pre;
+    row[3 * H + j] = dn_pre * gr;
+    dhz[e] = dh * gz;
+  }
+  if (counters && blockIdx.x == 0 && threadIdx.x == 0) counters[1] += 1;
+}
+// the [4H][K] matrix dz4 is contracted against: rows c H + j of W for c = 0, 1; row 2H + j over the
+// input columns for c = 2 and over the recurrent columns for c = 3.  col0: first column asked for.
+template <class T>
+struct GruWB {
+  const T* W; int H, K, I, col0;
+  __device__ float operator()(int g, int c) const {
+    const int blk = g / H, j = g - blk * H, col = c + col0;
+    if (blk < 2) return ldf(W, (size_t)(blk * H + j) * K + col);
+    return ((blk == 2) == (col < I)) ? ldf(W, (size_t)(2 * H + j) * K + col) : 0.f;
+  }
+};
+// like DinEpi, plus the part of dh that bypasses the gates
+struct GruDinEpi {
+  float* lo; int I; float* dh; int H; const float* dhz;
+  __device__ float operator()(float (&acc)[4][4], int b0, int c0, int M, int N) const {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int b = b0 + r, col = c0 + c;
+        if (b < M && col < N) {
+          if (col < I) { if (lo) lo[(size_t)b * I + col] = acc[r][c]; }
+          else dh[(size_t)b * H + (col - I)] = acc[r][c] + dhz[(size_t)b * H + (col - I)];
+        }
+      }
+    return 0.f;
+  }
+  __device__ void block_result(float, int) const {}
+};
+// out[n] += sum_b v[b][n] over the first N columns of rows that are `ld` apart, b ascending
+__global__ void colsum_accum_ld(const float* v, int B, int N, int ld, float* out) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += v[(size_t)b * ld + n];
+  out[n] += s;
+}
+
+template <class T>
+void gru_forward_step_t(const FwdArgs& a, cudaStream_t s) {
+  const int K = a.I + a.H;
+  FwdA<T> fa{(const T*)a.in, (const T*)a.h_prev, a.I, a.H};
+  GruFwdB<T> fb{(const T*)a.W, a.H, K, a.I};
+  GruFwdEpi<T> epi{a.bias, (const T*)a.h_prev, (T*)a.h_out, (T*)a.gates, (T*)a.h_in_copy, a.B, a.H, a.plane_elems,
+                   a.counters};
+  gemm_tiled<true, true, false><<<tiles(a.B, 4 * a.H), 256, 0, s>>>(a.B, 4 * a.H, K, fa, fb, epi);
+}
+
+template <class T>
+void gru_backward_layer_t(const BwdArgs& a, cudaStream_t s) {
+  const int K = a.I + a.H, H = a.H, G4 = 4 * a.H;
+  const size_t n = (size_t)a.B * a.H;
+  const int blocks = (int)((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256);
+  float* dhz = a.dc_rec;   // a GRU carries no cell-state gradient: the buffer holds dh z for this step
+  gru_gate_bwd<T><<<blocks, 256, 0, s>>>(a.dha, a.dh_rec, dhz, (const T*)a.gates, a.plane_elems, (const T*)a.h_prev,
+                                          a.dz, a.B, a.H, a.counters);
+  // dW: the rows of r and z against [in ; h_prev]; the rows of n against in (d n_pre) and h_prev (d q)
+  gemm_tiled<false, false, false><<<tiles(2 * H, K), 256, 0, s>>>(2 * H, K, a.B, DzTA{a.dz, G4},
+                                                                   InB<T>{(const T*)a.in, (const T*)a.h_prev, a.I, a.H},
+                                                                   AccumEpi{a.dW, K});
+  gemm_tiled<false, false, false><<<tiles(H, a.I), 256, 0, s>>>(H, a.I, a.B, DzTA{a.dz + 2 * H, G4},
+                                                                 HB<T>{(const T*)a.in, a.I},
+                                                                 AccumEpi{a.dW + (size_t)2 * H * K, K});
+  gemm_tiled<false, false, false><<<tiles(H, H), 256, 0, s>>>(H, H, a.B, DzTA{a.dz + 3 * H, G4},
+                                                               HB<T>{(const T*)a.h_prev, a.H},
+                                                               AccumEpi{a.dW + (size_t)2 * H * K + a.I, K});
+  colsum_accum_ld<<<(3 * H + 127) / 128, 128, 0, s>>>(a.dz, a.B, 3 * H, G4, a.db);
+  // d_in = dz4 against the expanded weights, plus dh z on the recurrent columns
+  if (a.d_lo) {
+    gemm_tiled<true, false, false><<<tiles(a.B, K), 256, 0, s>>>(a.B, K, G4, DzA{a.dz, G4},
+                                                                  GruWB<T>{(const T*)a.W, H, K, a.I, 0},
+                                                                  GruDinEpi{a.d_lo, a.I, a.dh_rec, a.H, dhz});
+  } else {
+    gemm_tiled<true, false, false><<<tiles(a.B, H), 256, 0, s>>>(a.B, H, G4, DzA{a.dz, G4},
+                                                                  GruWB<T>{(const T*)a.W, H, K, a.I, a.I},
+                                                                  GruDinEpi{nullptr, 0, a.dh_rec, a.H, dhz});
+  }
+}
+
 template <class T>
 void forward_step_t(const FwdArgs& a, cudaStream_t s) {
   const int K = a.I + a.H;
@@ -362,6 +512,14 @@ void readout(int dtype, const ReadoutArgs& a, cudaStream_t s) {
 void backward_layer(int dtype, const BwdArgs& a, cudaStream_t s) {
   if (dtype == MEBPTT_BF16) backward_layer_t<__nv_bfloat16>(a, s);
   else backward_layer_t<float>(a, s);
+}
+void gru_forward_step(int dtype, const FwdArgs& a, cudaStream_t s) {
+  if (dtype == MEBPTT_BF16) gru_forward_step_t<__nv_bfloat16>(a, s);
+  else gru_forward_step_t<float>(a, s);
+}
+void gru_backward_layer(int dtype, const BwdArgs& a, cudaStream_t s) {
+  if (dtype == MEBPTT_BF16) gru_backward_layer_t<__nv_bfloat16>(a, s);
+  else gru_backward_layer_t<float>(a, s);
 }
 void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
                    const int* status, cudaStream_t s) {

@@ -69,6 +69,11 @@ struct BwdArgs {
 void forward_step(int dtype, const FwdArgs& a, cudaStream_t s);
 void readout(int dtype, const ReadoutArgs& a, cudaStream_t s);
 void backward_layer(int dtype, const BwdArgs& a, cudaStream_t s);
+// The same two operations for the GRU core (W is [3H][I + H], gate blocks r, z, n; bias [3H]; the four
+// planes of an internal state hold r, z, n and q = W_hn h; c_prev / c_out / c_t are not used and dc_rec
+// serves as scratch).
+void gru_forward_step(int dtype, const FwdArgs& a, cudaStream_t s);
+void gru_backward_layer(int dtype, const BwdArgs& a, cudaStream_t s);
 // status: device word whose value goes to counters[3]
 void finalize_step(const float* loss_t, int64_t t, float* loss, int64_t* counters, int64_t peak_units,
                    const int* status, cudaStream_t s);

@@ -30,6 +30,8 @@ struct Layout {
   bool tensor_path = false;
   bool stepwise_tc = false;   // step-by-step operations with their contractions on the tensor cores
   bool stepwise_x3 = false;   // likewise for float32 storage, operands split into bfloat16 halves
+  bool gru = false;           // the core is a GRU (CUDA-core kernels)
+  int NG = 4;                 // row blocks of H rows in a layer's weight matrix and bias: 4 (LSTM) or 3 (GRU)
   size_t esz = 0;        // bytes of one operand element
   size_t granule = 0;
   size_t hsz = 0;        // one layer's h
@@ -60,7 +62,7 @@ struct Layout {
   int64_t arena_units = 0;
   int n_loss_part = 0;
 
-  size_t w_layer_elems(int l) const { return (size_t)4 * H * ((l == 0 ? I : H) + H); }
+  size_t w_layer_elems(int l) const { return (size_t)NG * H * ((l == 0 ? I : H) + H); }
   size_t w_layer_offset(int l) const {  // elements before layer l
     size_t o = 0;
     for (int i = 0; i < l; ++i) o += w_layer_elems(i);
@@ -79,7 +81,7 @@ inline bool valid_desc(const mebptt_lstm_desc* d) {
   if (d->input > (1 << 16) || d->hidden > (1 << 16) || d->readout > (1 << 16) || d->batch > (1 << 16)) return false;
   if (d->dtype != MEBPTT_FP32 && d->dtype != MEBPTT_TF32 && d->dtype != MEBPTT_BF16) return false;
   if (d->want_dx != 0 && d->want_dx != 1) return false;
-  if (d->flags & ~(MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_TIME_RUNS)) return false;
+  if (d->flags & ~(MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_TIME_RUNS | MEBPTT_FLAG_GRU)) return false;
   return true;
 }
 
@@ -87,7 +89,7 @@ inline bool valid_desc(const mebptt_lstm_desc* d) {
 // tile, sizes that keep every TMA stride a multiple of 16 bytes, and a recurrent weight slice per
 // CTA (8 hidden units x 4 gates x H) that fits in shared memory with one CTA per SM.
 inline bool tensor_path_supported(const mebptt_lstm_desc* d) {
-  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && d->dtype == MEBPTT_BF16 && d->layers == 1 && d->batch <= 64 && d->hidden % 8 == 0 &&
+  return !(d->flags & (MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_GRU)) && d->dtype == MEBPTT_BF16 && d->layers == 1 && d->batch <= 64 && d->hidden % 8 == 0 &&
          d->input % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
          d->hidden <= 1024;
 }
@@ -102,7 +104,7 @@ inline int loss_parts_per_step(int B, int O) { return loss_fused(B, O) ? (B / 32
 // their contractions to the tensor-core GEMM: bfloat16 storage, TMA-friendly strides, and whole
 // 32-row groups per step for the loss epilogue.
 inline bool stepwise_tc_supported(const mebptt_lstm_desc* d) {
-  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && !tensor_path_supported(d) && d->dtype == MEBPTT_BF16 &&
+  return !(d->flags & (MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_GRU)) && !tensor_path_supported(d) && d->dtype == MEBPTT_BF16 &&
          d->batch % 32 == 0 && d->input % 8 == 0 && d->hidden % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
          (d->batch / 32) * ((d->readout + 31) / 32) <= 4096;
 }
@@ -110,7 +112,7 @@ inline bool stepwise_tc_supported(const mebptt_lstm_desc* d) {
 // Float32 storage with tensor-core contractions (MEBPTT_TF32): the same step-by-step scheme over
 // operands split into bfloat16 halves.
 inline bool stepwise_x3_supported(const mebptt_lstm_desc* d) {
-  return !(d->flags & MEBPTT_FLAG_NO_TENSOR_CORES) && d->dtype == MEBPTT_TF32 && d->batch % 32 == 0 &&
+  return !(d->flags & (MEBPTT_FLAG_NO_TENSOR_CORES | MEBPTT_FLAG_GRU)) && d->dtype == MEBPTT_TF32 && d->batch % 32 == 0 &&
          d->input % 8 == 0 && d->hidden % 8 == 0 && d->readout % 8 == 0 && d->hidden >= 64 &&
          (d->batch / 32) * ((d->readout + 31) / 32) <= 4096;
 }
@@ -118,6 +120,8 @@ inline bool stepwise_x3_supported(const mebptt_lstm_desc* d) {
 inline void state_layout(const mebptt_lstm_desc* d, Layout& y) {
   y.L = d->layers; y.I = d->input; y.H = d->hidden; y.O = d->readout; y.B = d->batch;
   y.dtype = d->dtype; y.t = d->t;
+  y.gru = (d->flags & MEBPTT_FLAG_GRU) != 0;
+  y.NG = y.gru ? 3 : 4;
   y.tensor_path = tensor_path_supported(d);
   y.stepwise_tc = stepwise_tc_supported(d);
   y.stepwise_x3 = stepwise_x3_supported(d);

@@ -33,6 +33,8 @@ class DeviceProblem:
         self.prob = prob if prob is not None else synth.make_problem(cfg)
         self.host = synth.to_device_arrays(cfg, self.prob)
         self.want_dx = bool(want_dx)
+        if getattr(cfg, "cell", "lstm") == "gru":
+            flags |= B.MEBPTT_FLAG_GRU
         self.desc = B.make_desc(cfg.layers, cfg.input, cfg.hidden, cfg.readout, cfg.batch, cfg.t,
                                 cfg.dtype, want_dx=int(self.want_dx), flags=flags)
         self.dev = {k: _upload(v, self.device) for k, v in self.host.items()}
@@ -86,8 +88,9 @@ class DeviceProblem:
         c, out, off = self.cfg, [], 0
         for l in range(c.layers):
             K = (c.input if l == 0 else c.hidden) + c.hidden
-            n = 4 * c.hidden * K
-            out.append(flat[off:off + n].reshape(4 * c.hidden, K))
+            ng = 3 if getattr(c, "cell", "lstm") == "gru" else 4
+            n = ng * c.hidden * K
+            out.append(flat[off:off + n].reshape(ng * c.hidden, K))
             off += n
         return out
 

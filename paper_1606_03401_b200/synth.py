@@ -38,6 +38,7 @@ class LstmConfig:
     readout: int
     dtype: str          # "fp32" | "tf32" | "bf16"
     seed: int
+    cell: str = "lstm"  # "lstm" | "gru": the recurrent core (a GRU has three gate blocks and no cell state)
 
     def asdict(self):
         return asdict(self)
@@ -91,9 +92,11 @@ def make_problem(cfg: LstmConfig, general: bool = False) -> dict:
     W, b = [], []
     for l in range(L):
         I_l = I if l == 0 else H
-        W.append(opnd(rng.uniform(-lim, lim, size=(4 * H, I_l + H))))
-        bias = np.zeros(4 * H)
-        bias[H:2 * H] = 1.0            # forget gate
+        ng = 3 if cfg.cell == "gru" else 4
+        W.append(opnd(rng.uniform(-lim, lim, size=(ng * H, I_l + H))))
+        bias = np.zeros(ng * H)
+        if cfg.cell != "gru":
+            bias[H:2 * H] = 1.0        # forget gate
         b.append(bias)
     W_out = opnd(rng.uniform(-lim, lim, size=(O, H)))
     b_out = np.zeros(O)
@@ -102,7 +105,7 @@ def make_problem(cfg: LstmConfig, general: bool = False) -> dict:
     h0 = np.zeros((L, B, H))
     c0 = np.zeros((L, B, H))
     if general:
-        b = [round_to_fp32(v + rng.uniform(-0.3, 0.3, size=4 * H)) for v in b]
+        b = [round_to_fp32(v + rng.uniform(-0.3, 0.3, size=v.size)) for v in b]
         b_out = round_to_fp32(rng.uniform(-0.3, 0.3, size=O))
         h0 = opnd(0.5 * rng.standard_normal(size=(L, B, H)))
         c0 = round_to_fp32(0.5 * rng.standard_normal(size=(L, B, H)))

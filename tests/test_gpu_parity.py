@@ -495,6 +495,7 @@ def test_c5_shape_across_chunks_against_oracle_with_byte_budget(H):
 
 @pytest.mark.parametrize("base,kw,plans", [
     ("c1", dict(t=20), [("hsm", 4), ("msm", 9)]),                                                   # CUDA-core path
+    ("c1", dict(t=20, layers=2, cell="gru"), [("msm", 9)]),                                          # CUDA-core path, GRU core
     ("c2", dict(input=128, hidden=256, batch=64, t=70, readout=128), [("hsm", 5), ("msm", 13), ("ism", 70)]),  # persistent tensor path
     ("c5", dict(layers=2, input=64, hidden=72, batch=32, t=45, readout=40), [("msm", 11), ("ism", 45)]),      # step by step, bf16
     ("c4", dict(layers=1, input=64, hidden=128, batch=32, t=45, readout=40), [("msm", 11), ("ism", 45)]),     # step by step, float32 storage
@@ -591,3 +592,30 @@ def test_plans_over_the_layouts_byte_sizes_give_the_same_gradients(H, base, kw):
             assert plan.cost <= rounded.cost
     if cfg.dtype == "bf16":
         assert (plan.sigma, plan.alpha, plan.beta) == (3, 10, 7)
+
+
+@pytest.mark.parametrize("dtype,shape", [("fp32", dict(layers=1, input=32, hidden=64, batch=4, t=40, readout=32)),
+                                         ("fp32", dict(layers=2, input=24, hidden=40, batch=6, t=20, readout=10)),
+                                         ("bf16", dict(layers=2, input=24, hidden=40, batch=6, t=20, readout=10)),
+                                         ("tf32", dict(layers=1, input=70, hidden=65, batch=67, t=9, readout=66))])
+def test_gru_core_matches_oracle_and_is_plan_independent(H, dtype, shape):
+    """A second recurrent core behind the same plans and tape (Section 1: the method does not depend
+    on the architecture of the core): a GRU, with general biases and initial state, against its own
+    fp64 oracle per tensor and per block, bit-identical under every kind of plan, forward count equal
+    to C(t, m)."""
+    cfg = _cfg("c1", dtype=dtype, cell="gru", **shape)
+    prob = synth.make_problem(cfg, general=True)
+    assert prob["W"][0].shape[0] == 3 * cfg.hidden
+    dp = H.DeviceProblem(cfg, prob, want_dx=True)
+    ref = oracle_run(prob)
+    full = dp.run(dp.full_memory_plan())
+    assert full["counters"][0] == cfg.t and full["counters"][1] == cfg.t and full["counters"][3] == 0
+    assert_close_to_oracle(full, ref, dtype, want_dx=True)
+    for mode, m, beta in [("hsm", 1, 0), ("hsm", 4, 0), ("ism", 2, 0), ("msm", 9, 0), ("msm", 13, 3)]:
+        plan = dp.plan(mode, m, beta=beta)
+        res = dp.run(plan)
+        assert res["counters"][0] == plan.cost and res["counters"][1] == cfg.t and res["counters"][3] == 0
+        assert_bit_identical(res, full, want_dx=True)
+    # without dx the first layer skips its input-gradient columns; nothing else may change
+    nodx = H.DeviceProblem(cfg, prob, want_dx=False)
+    assert_bit_identical(nodx.run(nodx.plan("msm", 9)), full)

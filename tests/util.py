@@ -1,12 +1,15 @@
 """Helpers shared by the GPU parity tests."""
 import numpy as np
 
+from oracle import gru_bptt as OG
 from oracle import lstm_bptt as O
 
 TOL = {"fp32": 1e-4, "tf32": 1e-4, "bf16": 2e-2}   # relative L2 error against the fp64 oracle
 
 
 def oracle_run(prob):
+    if prob["W"][0].shape[0] % 3 == 0 and prob["W"][0].shape[0] // 3 == prob["h0"].shape[-1]:   # three gate blocks: a GRU
+        return OG.gru_bptt(prob["W"], prob["b"], prob["W_out"], prob["b_out"], prob["x"], prob["targets"], prob["h0"])
     return O.lstm_bptt(prob["W"], prob["b"], prob["W_out"], prob["b_out"], prob["x"], prob["targets"],
                        prob["h0"], prob["c0"])
 
@@ -32,15 +35,16 @@ def rel_l2(a, b):
 BLOCK_FACTOR = 4.0   # a block may be this many times further off than the whole tensor is allowed to be
 
 
-def _blocks(name, arr):
+def _blocks(name, arr, gates=4):
     """(label, index) pairs cutting an oracle array into the blocks a kernel mistake would hit:
     gate blocks and 128 x 128 tiles of a weight gradient, 32 entries of a bias gradient, one
     time step of dx."""
-    if name == "dW":          # [4H, K]
+    if name == "dW":          # [4H, K] (LSTM) or [3H, K] (GRU): K - I = H columns are recurrent
         G, K = arr.shape
-        H = G // 4
-        for q in range(4):
-            yield f"gate {'ifgo'[q]}", (slice(q * H, (q + 1) * H), slice(None))
+        ng = 4 if gates == 4 else 3
+        H = G // ng
+        for q in range(ng):
+            yield f"gate block {q}", (slice(q * H, (q + 1) * H), slice(None))
         for r in range(0, G, 128):
             for c in range(0, K, 128):
                 yield f"tile ({r},{c})", (slice(r, r + 128), slice(c, c + 128))
@@ -57,13 +61,13 @@ def _blocks(name, arr):
             yield f"step {k + 1}", (k,)
 
 
-def _assert_blocks_close(name, got, ref, tol):
+def _assert_blocks_close(name, got, ref, tol, gates=4):
     """Relative L2 per block.  The denominator is the block's own norm, floored at a tenth of
     what an average block of the tensor carries, so that a block that happens to be near zero is
     held to the tensor's scale instead of its own."""
     got = np.asarray(got, np.float64).reshape(ref.shape)
     labels, num, den = [], [], []
-    for label, idx in _blocks(name, ref):
+    for label, idx in _blocks(name, ref, gates):
         labels.append(label)
         num.append(np.linalg.norm(got[idx] - ref[idx]))
         den.append(np.linalg.norm(ref[idx]))
@@ -90,8 +94,9 @@ def assert_close_to_oracle(res, ref, dtype, want_dx=False):
     for k, e in errs.items():
         assert e <= tol, (k, e, errs)
     off_w = off_b = 0
+    H = ref["dW_out"].shape[1]
     for l, (w, v) in enumerate(zip(ref["dW"], ref["db"])):
-        errs[f"dW[{l}] worst block"] = _assert_blocks_close("dW", res["dW"][off_w:off_w + w.size], w, tol)
+        errs[f"dW[{l}] worst block"] = _assert_blocks_close("dW", res["dW"][off_w:off_w + w.size], w, tol, w.shape[0] // H)
         errs[f"db[{l}] worst block"] = _assert_blocks_close("db", res["db"][off_b:off_b + v.size], v, tol)
         off_w += w.size
         off_b += v.size
