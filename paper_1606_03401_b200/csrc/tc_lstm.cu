@@ -166,10 +166,12 @@ struct FwdRunArgs {
   uint32_t hsz16;        // distance from h to c inside a hidden block, in 16-byte units
 };
 
-// 64-wide blocks of the contraction index in the first part of the split (all of them if there is one)
+// 64-wide blocks of the contraction index in the first part of the split (all of them if there is
+// one part only: below 640 columns the second accumulator and its hand-over cost more than starting
+// the MMAs half a fetch earlier saves)
 __host__ __device__ inline int fwd_first_part_blocks(int H) {
   const int KB = (H + 63) / 64;
-  return KB >= 2 ? (KB + 1) / 2 : KB;
+  return KB >= 10 ? (KB + 1) / 2 : KB;
 }
 
 // State update of one thread: batch row b, hidden units j0 .. j0 + 3.  z[u] holds the four
