@@ -5,8 +5,13 @@
 //   MEBPTT_NO_PDL=1           launch without programmatic stream serialization
 //   MEBPTT_NO_OVERLAP=1       weight-gradient GEMMs on the caller's stream instead of the side stream;
 //                             host-buffer inputs copied in front of the step instead of beside it
+//   MEBPTT_NO_PRIORITY=1      the step on the caller's stream itself instead of the library's stream of
+//                             the most urgent priority
+//   MEBPTT_NO_ZX_AHEAD=1      input projections in the step's stream, when a run needs them, instead of a
+//                             window ahead on a stream of their own
 //   MEBPTT_BWD_CLUSTER=0|4|8  backward run kernel: unclustered (what a profiler that cannot launch
 //                             clustered cooperative grids can capture), or the cluster size
+//   MEBPTT_NO_BWD_GROUPS=1    backward run kernel without groups of batch rows (same bits)
 //   MEBPTT_NO_SPLITK=1        no contraction is split along K (other rounding on the step-by-step paths)
 //   MEBPTT_STEPWISE_PER_OP=1  step-by-step paths operation by operation instead of in runs (same bits)
 //   MEBPTT_PLAN_SCAN=1        the planner scans every split point instead of walking convex columns
@@ -31,7 +36,10 @@ inline int integer(const char* name) {
 
 inline bool no_pdl() { static const bool v = flag("MEBPTT_NO_PDL"); return v; }
 inline bool no_overlap() { static const bool v = flag("MEBPTT_NO_OVERLAP"); return v; }
+inline bool no_priority() { static const bool v = flag("MEBPTT_NO_PRIORITY"); return v; }
+inline bool no_zx_ahead() { static const bool v = flag("MEBPTT_NO_ZX_AHEAD"); return v; }
 inline int bwd_cluster() { static const int v = integer("MEBPTT_BWD_CLUSTER"); return v; }
+inline bool no_bwd_groups() { static const bool v = flag("MEBPTT_NO_BWD_GROUPS"); return v; }
 inline bool no_splitk() { static const bool v = flag("MEBPTT_NO_SPLITK"); return v; }
 inline bool stepwise_per_op() { return flag("MEBPTT_STEPWISE_PER_OP"); }   // read per call: tests switch it
 inline bool plan_scan() { return flag("MEBPTT_PLAN_SCAN"); }               // likewise

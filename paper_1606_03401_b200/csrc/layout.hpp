@@ -291,7 +291,8 @@ inline void workspace_layout(const mebptt_lstm_desc* d, const Plan* p, Layout& y
     y.off_wpT_ih = take(d->want_dx ? G * y.I * 2 : 0);
     y.off_bias_p = take(G * 4);
     y.off_woutT = take((size_t)y.O * y.H * 2);
-    y.off_zx = take(SB * G * 4);
+    // two copies: the projections of the next window are computed while the runs read this one's
+    y.off_zx = take(2 * SB * G * 4);
     // two copies of what the weight-gradient GEMMs read: they may still be running (on the
     // library's side stream) while the backward pass fills the stages of the next chunk
     y.off_dz = take(2 * SB * G * 2);

@@ -936,6 +936,298 @@ __global__ void __launch_bounds__(192, 1) bwd_run_cluster_kernel(const __grid_co
 }
 
 // ------------------------------------------------------------------------------------------
+// backward run, clusters inside groups of batch rows
+// ------------------------------------------------------------------------------------------
+// The same split along K as above (clusters of four CTAs, partial tiles reduced in rank order), with
+// what the forward kernel does about latency: the grid is cut into groups of CTAs that each own
+// FB = 32 batch rows and have a step counter of their own, so that a CTA pulls half the bytes of
+// dz_k and a step is signalled by half the CTAs; the product is taken transposed (the cluster's 64
+// columns of dh, as rows of W_hh^T resident in shared memory, are the M side of the MMA, the 32
+// batch rows the N side); and all 128 epilogue threads take part in the gate derivatives, each with
+// four hidden units of one batch row.  CTA c of a group owns hidden units 16 c .. 16 c + 15; the
+// partial sums of a column are added in the order of the ranks as above, so both kernels give the
+// same bits.
+struct GateInputs4 {
+  uint2 qi, qf, qg, qo;
+  float4 t, p, d;
+};
+__device__ __forceinline__ GateInputs4 load_gate_inputs4(const BwdRunArgs& a, const DevOp& op, int sidx, int b, int j0,
+                                                         size_t e0, size_t pl) {
+  GateInputs4 in;
+  const char* ws = a.ws;
+  in.d = *reinterpret_cast<const float4*>(a.dha + ((size_t)sidx * a.B) * a.H + e0);
+  in.p = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(ws + (size_t)op.c_src * 16) + e0);
+  if (a.zleaf) {
+    // a leaf of the recursion: its forward operation redone from the pre-activations, with the
+    // arithmetic of the forward kernel
+    const float4* zp = reinterpret_cast<const float4*>(a.zleaf + ((size_t)sidx * a.B + b) * 4 * a.H + (size_t)4 * j0);
+    const float cp[4] = {in.p.x, in.p.y, in.p.z, in.p.w};
+    float ct[4], iv[4], fv[4], gv[4], ov[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float4 z = zp[u];
+      iv[u] = sigmoid_fast(z.x);
+      fv[u] = sigmoid_fast(z.y);
+      gv[u] = tanh_fast(z.z);
+      ov[u] = sigmoid_fast(z.w);
+      ct[u] = fmaf(fv[u], cp[u], iv[u] * gv[u]);
+    }
+    in.qi = make_uint2(pack_bf16x2(iv[0], iv[1]), pack_bf16x2(iv[2], iv[3]));
+    in.qf = make_uint2(pack_bf16x2(fv[0], fv[1]), pack_bf16x2(fv[2], fv[3]));
+    in.qg = make_uint2(pack_bf16x2(gv[0], gv[1]), pack_bf16x2(gv[2], gv[3]));
+    in.qo = make_uint2(pack_bf16x2(ov[0], ov[1]), pack_bf16x2(ov[2], ov[3]));
+    in.t = make_float4(ct[0], ct[1], ct[2], ct[3]);
+    return in;
+  }
+  const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(ws + (size_t)op.gates * 16) + e0;
+  in.qi = *reinterpret_cast<const uint2*>(g);
+  in.qf = *reinterpret_cast<const uint2*>(g + pl);
+  in.qg = *reinterpret_cast<const uint2*>(g + 2 * pl);
+  in.qo = *reinterpret_cast<const uint2*>(g + 3 * pl);
+  in.t = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(ws + (size_t)op.c_dst * 16) + e0);
+  return in;
+}
+
+// The arithmetic of compute_gates for four hidden units.
+__device__ __forceinline__ void compute_gates4(const BwdRunArgs& a, const GateInputs4& in, int sidx, int b, int j0,
+                                               const float (&dh)[4], float (&dc)[4]) {
+  const int G = 4 * a.H;
+  const float dhav[4] = {in.d.x, in.d.y, in.d.z, in.d.w};
+  const uint32_t wi[2] = {in.qi.x, in.qi.y}, wf[2] = {in.qf.x, in.qf.y}, wg[2] = {in.qg.x, in.qg.y}, wo[2] = {in.qo.x, in.qo.y};
+  const float ct[4] = {in.t.x, in.t.y, in.t.z, in.t.w};
+  const float cp[4] = {in.p.x, in.p.y, in.p.z, in.p.w};
+  uint32_t out[8];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int w = u >> 1;
+    const bool hi = (u & 1) != 0;
+    const float gi = hi ? bf16_hi(wi[w]) : bf16_lo(wi[w]);
+    const float gf = hi ? bf16_hi(wf[w]) : bf16_lo(wf[w]);
+    const float gg = hi ? bf16_hi(wg[w]) : bf16_lo(wg[w]);
+    const float go = hi ? bf16_hi(wo[w]) : bf16_lo(wo[w]);
+    const float dht = dhav[u] + dh[u];
+    const float th = tanh_fast(ct[u]);
+    const float d_o = dht * th;
+    const float dct = fmaf(dht * go, 1.f - th * th, dc[u]);
+    const float zi = dct * gg * gi * (1.f - gi);
+    const float zf = dct * cp[u] * gf * (1.f - gf);
+    const float zg = dct * gi * (1.f - gg * gg);
+    const float zo = d_o * go * (1.f - go);
+    dc[u] = dct * gf;
+    out[2 * u] = pack_bf16x2(zi, zf);
+    out[2 * u + 1] = pack_bf16x2(zg, zo);
+  }
+  uint4* dzp = reinterpret_cast<uint4*>(a.dz + ((size_t)sidx * a.B + b) * G + (size_t)4 * j0);
+  dzp[0] = make_uint4(out[0], out[1], out[2], out[3]);
+  dzp[1] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
+constexpr int GCS = 4;           // CTAs per cluster
+constexpr int RECV_LD = FB + 4;  // row stride of a received partial tile, [dh column][batch row] (floats)
+
+__global__ void __launch_bounds__(192, 1) bwd_run_group_kernel(const __grid_constant__ CUtensorMap tm_dz,
+                                                               const __grid_constant__ CUtensorMap tm_wt,
+                                                               const BwdRunArgs a) {
+  constexpr int NC = FU * GCS;             // columns of dh the cluster produces: the M of the MMA
+  constexpr uint32_t W_TILE = NC * 128;    // [64 columns of dh][64 contraction indices]
+  constexpr uint32_t A_TILE = FB * 128;    // [32 batch rows][64 contraction indices]
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t wfull, full[4], acc, pready[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int failed;
+
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int G = 4 * a.H;
+  const int KBS = (G / 64) / GCS;          // 64-wide K blocks in this CTA's slice (<= 16)
+  const int TB = a.tb;                     // K tiles per barrier and per copy
+  const int NQ = (KBS + TB - 1) / TB;      // <= 4
+  uint8_t* sW = sm;                        // KBS tiles of W_hh^T
+  uint8_t* ring = sW + KBS * W_TILE;       // KBS tiles of dz_k, all of the slice at once
+  // partial sums received from the cluster: [2 buffers][GCS senders][16 columns][RECV_LD]
+  float* recv = reinterpret_cast<float*>(ring + NQ * TB * A_TILE);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ncg = (int)gridDim.x / ((a.B > FB) ? 2 : 1);   // CTAs per group
+  const int grp = blockIdx.x / ncg, cta = blockIdx.x % ncg;
+  const uint32_t rank = cluster_ctarank();
+  const int cl = cta / GCS;
+  uint32_t* const sync = a.sync + grp * SYNC_STRIDE;
+
+  if (tid == 0) {
+    mbar_init(&wfull, 1);
+    for (int s = 0; s < 4; ++s) mbar_init(&full[s], 1);
+    mbar_init(&acc, 1);
+    mbar_init(&pready[0], GCS);
+    mbar_init(&pready[1], GCS);
+    failed = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_dz);
+    tma_prefetch_desc(&tm_wt);
+  }
+  if (warp == 4) tmem_alloc(&tmem_slot, 32);
+  tc_fence_before_sync();
+  cluster_sync();                          // peers arrive on each other's barriers: all must be initialised
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  grid_dep_wait();
+
+  if (warp == 4) {
+    // ---- producer: this CTA's K-slice of the group's rows of dz_k; lane 0 watches the group's step
+    // counter, lanes 0 .. NQ-1 each request one block of TB tiles -------------------------------------
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&wfull, (uint32_t)KBS * W_TILE);
+      for (int kb = 0; kb < KBS; ++kb)
+        tma_load_2d(sW + kb * W_TILE, &tm_wt, ((int)rank * KBS + kb) * 64, cl * NC, &wfull);
+    }
+    int armed = -1;
+    for (int i = 0; i < a.n; ++i) {
+      const int sidx = (a.ops[i].k - 1) % a.S;
+      if (blockIdx.x == 0 && lane == 31) {
+        // loss term of this step: its partial sums in a fixed order (on a lane that is off the
+        // critical path of the recurrence)
+        float sum = 0.f;
+        for (int p = 0; p < a.loss_parts; ++p) sum += a.loss_part[sidx * a.loss_parts + p];
+        a.loss_t[a.ops[i].k - 1] = sum;
+      }
+      int go = 1;
+      if (lane == 0) go = !failed && wait_counter(sync, (uint32_t)(i + 1) * a.expect, &failed, a.poll_limit) && !failed;
+      go = __shfl_sync(0xffffffffu, go, 0);
+      if (!go) continue;
+      if (lane < NQ) {
+        fence_proxy_async_global();
+        // rows past the batch are never used: they only reach accumulator columns that no thread reads
+        const int32_t row = sidx * a.B + grp * FB;
+        mbar_arrive_expect_tx(&full[lane], (uint32_t)TB * A_TILE);   // a box counts in full
+        tma_load_3d(ring + TB * lane * A_TILE, &tm_dz, 0, row, (int)rank * KBS + TB * lane, &full[lane]);
+      }
+      armed = i;
+      if (i == a.n - 1 && lane == 0) grid_dep_launch();
+      __syncwarp();
+    }
+    if (failed && lane == 0) {
+      (void)mbar_wait(&wfull, 0);
+      if (armed >= 0)
+        for (int q = 0; q < NQ; ++q) (void)mbar_wait(&full[q], (uint32_t)armed & 1);
+    }
+  } else if (warp == 5) {
+    // ---- MMA issuer: the whole warp walks the loop, one elected lane issues --------------------
+    constexpr uint32_t idesc = make_idesc(1, NC, FB, false, false);
+    bool ok = wait_or_fail(&wfull, 0, &failed);
+    const uint64_t w_desc0 = make_desc_sw128(smem_u32(sW), 16, 1024);
+    const uint64_t z_desc0 = make_desc_sw128(smem_u32(ring), 16, 1024);
+    for (int i = 0; i < a.n; ++i) {
+      uint64_t dw = w_desc0, dzd = z_desc0;
+      for (int q = 0; q < NQ && ok; ++q) {
+        ok = wait_or_fail(&full[q], (uint32_t)i & 1, &failed);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int nkb = (TB * q + TB < KBS) ? TB : KBS - TB * q;
+        if (elect_one()) {
+          for (int kb = 0; kb < nkb; ++kb)
+            mma_f16_x4(tmem, dw + (uint64_t)(kb * (W_TILE >> 4)), dzd + (uint64_t)(kb * (A_TILE >> 4)), idesc,
+                       (q > 0 || kb > 0) ? 1u : 0u);
+        }
+        __syncwarp();
+        dw += (uint64_t)TB * (W_TILE >> 4);
+        dzd += (uint64_t)TB * (A_TILE >> 4);
+      }
+      if (elect_one()) mma_commit(&acc);   // always: the epilogue counts on one arrival per step
+      __syncwarp();
+    }
+  } else {
+    // ---- gate derivatives -------------------------------------------------------------------------
+    // as a reader of TMEM: warp w, lanes 0 .. 15 hold accumulator rows 16 w .. 16 w + 15, the columns
+    // of dh that CTA w of the cluster owns; as an owner of state: batch row tid / 4 of the group,
+    // hidden units 4 (tid % 4) .. + 3 of the CTA
+    const int bl = tid >> 2, u0 = 4 * (tid & 3);
+    const int b = grp * FB + bl;
+    const int j0 = cta * FU + u0;
+    const bool owner = b < a.B;
+    const size_t e0 = (size_t)b * a.H + j0;
+    const size_t pl = (size_t)a.plane16 * 8;
+    float dh[4], dc[4];
+    if (owner) {
+      const float4 a0 = *reinterpret_cast<const float4*>(a.dh + e0), c0 = *reinterpret_cast<const float4*>(a.dc + e0);
+      dh[0] = a0.x; dh[1] = a0.y; dh[2] = a0.z; dh[3] = a0.w;
+      dc[0] = c0.x; dc[1] = c0.y; dc[2] = c0.z; dc[3] = c0.w;
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { dh[u] = 0.f; dc[u] = 0.f; }
+    }
+
+    // Reduces the partial tiles of product number `it` into this thread's dh: each row thread reads
+    // its row of this CTA's partial tile from TMEM (one column of dh, 32 batch rows) and sends it
+    // into the shared memory of the CTA that owns the column; once all senders have signalled, an
+    // owner adds the partial values of its columns in the order of the ranks.
+    auto reduce_partials = [&](int it) {
+      float* buf = recv + (size_t)(it & 1) * GCS * FU * RECV_LD;
+      const bool got = wait_or_fail(&acc, (uint32_t)it & 1, &failed);
+      tc_fence_after_sync();
+      uint32_t r[32];
+      tmem_ld_32x32(tmem + ((uint32_t)(32 * warp) << 16), r);
+      tmem_ld_wait();
+      if (lane < 16) {
+        float* dst = buf + ((size_t)rank * FU + lane) * RECV_LD;      // slot of sender `rank`, column `lane` of CTA `warp`
+#pragma unroll
+        for (int v = 0; v < FB / 4; ++v)
+          st_peer_f4(dst + 4 * v, (uint32_t)warp, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                              __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+      }
+      tc_fence_before_sync();
+      named_barrier(1, 128);
+      if (tid < GCS) mbar_arrive_peer(&pready[it & 1], (uint32_t)tid);   // release: the stores above are visible
+      bool all = false;
+      for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait_cluster(&pready[it & 1], (uint32_t)(it >> 1) & 1)) { all = true; break; }
+        if (spin > 256) {
+          if (failed) break;
+          __nanosleep(64);
+        }
+      }
+      if (!all) failed = 1;
+      if (got && all && owner) {
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int p = 0; p < GCS; ++p) {
+          const float* src = buf + ((size_t)p * FU + u0) * RECV_LD + bl;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) sum[u] += src[u * RECV_LD];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) dh[u] = sum[u];
+      }
+    };
+
+    GateInputs4 gin;
+    if (owner) gin = load_gate_inputs4(a, a.ops[0], (a.ops[0].k - 1) % a.S, b, j0, e0, pl);
+    for (int i = 0; i < a.n; ++i) {
+      const DevOp op = a.ops[i];
+      const int sidx = (op.k - 1) % a.S;
+      if (i > 0) reduce_partials(i - 1);
+      if (owner && !failed) compute_gates4(a, gin, sidx, b, j0, dh, dc);
+      named_barrier(1, 128);   // all of this CTA's dz stores precede the release below
+      if (tid == 0) red_release_add(sync, 1u);
+      // the inputs of the next (earlier) step do not depend on the recurrence: fetch them while the
+      // exchange of this step is in flight
+      if (owner && i + 1 < a.n) gin = load_gate_inputs4(a, a.ops[i + 1], (a.ops[i + 1].k - 1) % a.S, b, j0, e0, pl);
+    }
+    reduce_partials(a.n - 1);
+    if (owner && !failed) {
+      *reinterpret_cast<float4*>(a.dh + e0) = make_float4(dh[0], dh[1], dh[2], dh[3]);
+      *reinterpret_cast<float4*>(a.dc + e0) = make_float4(dc[0], dc[1], dc[2], dc[3]);
+    }
+  }
+
+  tc_fence_before_sync();
+  cluster_sync();   // no CTA leaves while a peer may still read its partial tiles or signal it
+  if (tid == 0) {
+    if (failed) *a.status = MEBPTT_ERR_TIMEOUT;
+    else if (blockIdx.x == 0) a.counters[1] += a.n;
+  }
+  if (warp == 4) tmem_dealloc(tmem, 32);
+}
+
+// ------------------------------------------------------------------------------------------
 // small kernels off the recurrence
 // ------------------------------------------------------------------------------------------
 // Packs the weights once per training step: gate rows permuted to 4 u + q (the four gates of
@@ -1044,23 +1336,48 @@ __global__ void loss_dy(const DevOp* ops, const float* y, const float* targets, 
 }
 
 // out[map(n)] += sum_r v[r][n]; perm_h > 0 maps column 4 u + q to q perm_h + u.  A block of
-// 32 x 8 threads sums 32 columns: thread (x, g) takes rows g, g + 8, ... in ascending order, then
-// the eight partial sums are added in the order g = 0 .. 7.
-__global__ void colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out, int perm_h) {
-  __shared__ float part[8][33];
+// 32 x 32 threads sums 64 columns: thread (x, g) takes the rows g, g + 32, ... of columns 2 x and
+// 2 x + 1 into four running sums (row g + 32 i goes to sum i mod 4, so that four loads are in
+// flight), adds them as (0 + 1) + (2 + 3), and the 32 partial sums of a column are added in the
+// order g = 0 .. 31: fixed, whatever the plan.
+__global__ void __launch_bounds__(1024) colsum_bf16(const __nv_bfloat16* v, int rows, int N, float* out, int perm_h) {
+  __shared__ float2 part[32][33];
   grid_dep_wait();
   grid_dep_launch();
-  const int n = blockIdx.x * 32 + threadIdx.x, g = threadIdx.y;
-  float s = 0.f;
-  if (n < N)
-    for (int r = g; r < rows; r += 8) s += __bfloat162float(v[(size_t)r * N + n]);
-  part[g][threadIdx.x] = s;
+  const int n = (blockIdx.x * 32 + threadIdx.x) * 2, g = threadIdx.y;
+  float2 acc[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) acc[j] = make_float2(0.f, 0.f);
+  if (n < N) {
+    const bool pair = (N & 1) == 0;   // then column n + 1 exists and the two lie in one aligned word
+    auto load = [&](int r) {
+      const __nv_bfloat16* q = v + (size_t)r * N + n;
+      if (pair) return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(q));
+      return make_float2(__bfloat162float(q[0]), n + 1 < N ? __bfloat162float(q[1]) : 0.f);
+    };
+    int r = g;
+    for (; r + 96 < rows; r += 128) {
+      float2 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = load(r + 32 * j);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { acc[j].x += x[j].x; acc[j].y += x[j].y; }
+    }
+#pragma unroll
+    for (int j = 0; j < 3; ++j)   // at most three rows are left
+      if (r + 32 * j < rows) {
+        const float2 x = load(r + 32 * j);
+        acc[j].x += x.x; acc[j].y += x.y;
+      }
+  }
+  part[g][threadIdx.x] = make_float2((acc[0].x + acc[1].x) + (acc[2].x + acc[3].x), (acc[0].y + acc[1].y) + (acc[2].y + acc[3].y));
   __syncthreads();
-  if (g == 0 && n < N) {
+  if (g < 2 && n + g < N) {
     float tot = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) tot += part[i][threadIdx.x];
-    const int o = perm_h ? ((n & 3) * perm_h + (n >> 2)) : n;
+    for (int i = 0; i < 32; ++i) tot += g ? part[i][threadIdx.x].y : part[i][threadIdx.x].x;
+    const int c = n + g;
+    const int o = perm_h ? ((c & 3) * perm_h + (c >> 2)) : c;
     out[o] += tot;
   }
 }
@@ -1106,6 +1423,11 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
 constexpr int X_PIECES = 8;
 struct SideStream {
   cudaStream_t stream = nullptr;
+  cudaStream_t main = nullptr;                 // the step itself, at the most urgent priority
+  cudaEvent_t fork = nullptr, join = nullptr;  // the caller's stream -> main, main -> the caller's stream
+  cudaStream_t zx = nullptr;                   // input projections of the window after the one in use
+  cudaEvent_t zx_free[2] = {nullptr, nullptr};   // copy b of the window buffer has no reader left (recorded on the step's stream)
+  cudaEvent_t zx_ready[2] = {nullptr, nullptr};  // copy b holds its window (recorded on the zx stream)
   cudaEvent_t ready[2] = {nullptr, nullptr};   // stages of parity p are complete (recorded on the caller's stream)
   cudaEvent_t done[2] = {nullptr, nullptr};    // GEMMs reading parity p have finished (recorded on the side stream)
   cudaStream_t copy = nullptr;                 // host-to-device copies that overlap the forward pass
@@ -1126,7 +1448,15 @@ SideStream* side_stream_for_current_device() {
     tried[dev] = true;
     int lo = 0, hi = 0;
     cudaDeviceGetStreamPriorityRange(&lo, &hi);   // lo = numerically largest = least urgent
-    bool ok = cudaStreamCreateWithPriority(&t.stream, cudaStreamNonBlocking, lo) == cudaSuccess;
+    bool ok = cudaStreamCreateWithPriority(&t.stream, cudaStreamNonBlocking, lo) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&t.main, cudaStreamNonBlocking, hi) == cudaSuccess &&
+              cudaEventCreateWithFlags(&t.fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&t.join, cudaEventDisableTiming) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&t.zx, cudaStreamNonBlocking, (lo + hi) / 2) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i) {
+      ok = cudaEventCreateWithFlags(&t.zx_free[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&t.zx_ready[i], cudaEventDisableTiming) == cudaSuccess;
+    }
     for (int i = 0; i < 2 && ok; ++i) {
       ok = cudaEventCreateWithFlags(&t.ready[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&t.done[i], cudaEventDisableTiming) == cudaSuccess;
@@ -1267,6 +1597,7 @@ struct Prepared {
   int device = -1;
   // host part
   std::vector<WorkItem> items;
+  std::vector<int> zx_next;  // per item that opens a window: the item that opens the next one (-1: none)
   std::vector<int> zx_hi;  // per item: a forward run that projects its inputs anew does so up to this step (exclusive); 0: the window in place serves it
   DevOp* tape = nullptr;   // [2 nops]: the tape, then the compacted leaves of leaf batches
   size_t tape_entries = 0;
@@ -1276,6 +1607,9 @@ struct Prepared {
   int bwd_cs = 0, bwdc_smem = 0;   // cluster size of the backward kernel (0: one CTA per 8 columns, unclustered)
   int bwd_tb = 4;                  // its K tiles per barrier
   bool bwd_slab = false;           // its slice of dz by one copy per barrier instead of one per K tile
+  bool bwd_grp = false;            // the backward kernel with groups of batch rows (then bwd_cs is its cluster size)
+  int bwdg_smem = 0, bwdg_tb = 8, bwdg_ncg = 0;
+  CUtensorMap tm_dz_g[2], tm_wt_g;
   int fwd_ncg = 0, fwd_smem = 0, fwd_bb = 0;
   bool fwd_slab = false;
   int rc = MEBPTT_OK;
@@ -1331,6 +1665,9 @@ void build_host_part(Prepared& P, const Layout& y, const Plan* p, bool allow_pin
     }
     P.zx_hi[item] = zx_hi;
   }
+  P.zx_next.assign(P.items.size(), -1);
+  for (int item = (int)P.items.size() - 1, next = -1; item >= 0; --item)
+    if (P.zx_hi[item]) { P.zx_next[item] = next; next = item; }
   // the tape as the kernels read it
   P.tape_entries = 2 * nops;
   const size_t bytes = (P.tape_entries ? P.tape_entries : 1) * sizeof(DevOp);
@@ -1440,6 +1777,35 @@ void build_device_part(Prepared& P, const Layout& y, char* ws) {
     P.bwd_cs = cs; P.bwdc_smem = smem; P.bwd_tb = tb;
     break;
   }
+  // the kernel with groups of batch rows, where the batch fills two groups and the driver takes a
+  // map that sees the staging chunk as [columns / 64][rows][64]
+  if (P.bwd_cs && force < 0 && !env::no_bwd_groups() && B > FB && B <= 2 * FB && H % (FU * GCS) == 0 &&
+      (G / 64) % GCS == 0 && (G / 64) / GCS <= 16) {
+    const int kbs = (G / 64) / GCS;
+    const int tb = kbs > 8 ? 8 : 4;
+    const int nq = (kbs + tb - 1) / tb;
+    const int smem = kbs * (FU * GCS * 128) + nq * tb * FB * 128 + 2 * GCS * FU * RECV_LD * 4 + 1024;
+    const int ncg = H / FU;
+    bool g_ok = smem <= 220 * 1024;
+    const void* fn = (const void*)bwd_run_group_kernel;
+    if (g_ok) {
+      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * ncg); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem;
+      cudaLaunchAttribute at1[1];
+      at1[0].id = cudaLaunchAttributeClusterDimension;
+      at1[0].val.clusterDim.x = GCS; at1[0].val.clusterDim.y = 1; at1[0].val.clusterDim.z = 1;
+      cfg.attrs = at1; cfg.numAttrs = 1;
+      int nclusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess) { cudaGetLastError(); g_ok = false; }
+      else g_ok = nclusters * GCS >= 2 * ncg;
+    }
+    for (int pb = 0; pb < 2 && g_ok; ++pb)
+      g_ok = make_tmap_blocks64(&P.tm_dz_g[pb], dz + (size_t)pb * S * B * G, (uint64_t)G, (uint64_t)S * B, (uint64_t)G * 2, FB,
+                                (uint32_t)tb);
+    g_ok = g_ok && make_tmap_2d(&P.tm_wt_g, wpT_hh, 2, (uint64_t)G, (uint64_t)H, (uint64_t)G * 2, 64, FU * GCS);
+    if (g_ok) { P.bwd_grp = true; P.bwdg_smem = smem; P.bwdg_tb = tb; P.bwdg_ncg = ncg; }
+  }
   if (P.bwd_cs) {
     // the staging chunk as [columns / 64][rows][64] if the driver takes such a map, else tile by tile
     P.bwd_slab = true;
@@ -1512,7 +1878,7 @@ void prepare_stats(int64_t* out) {
 
 int prepare_host(const Layout& y, const Plan* p, bool want_dx) { return prepare(y, p, want_dx, nullptr, false)->rc; }
 
-int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t s, bool dry,
+int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_dx, cudaStream_t caller, bool dry,
                  bool side_stream) {
   const int B = y.B, H = y.H, I = y.I, O = y.O, S = y.S, G = 4 * H, K = I + H;
   const int BM = 64;  // batch rows per MMA tile (B <= 64)
@@ -1557,6 +1923,18 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   const CUtensorMap* tm_dz_b = P.tm_dz_b;
   const int bwd_cs = P.bwd_cs, bwdc_smem = P.bwdc_smem, fwd_ncg = P.fwd_ncg, fwd_smem = P.fwd_smem, fwd_bb = P.fwd_bb;
   const bool fwd_slab = P.fwd_slab;
+  // With streams of its own the library runs the step on one of the most urgent priority, ordered
+  // after what the caller's stream holds and joined to it at the end.  The caller's stream is of the
+  // least urgent priority as a rule, the same as the stream of the weight-gradient GEMMs: a grid of
+  // theirs that becomes eligible together with a kernel of the recurrence would otherwise take the
+  // SMs first as often as not, and every CTA of it runs for tens of microseconds.
+  SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
+  cudaStream_t s = caller;
+  if (side && !env::no_priority()) {
+    cudaEventRecord(side->fork, caller);
+    cudaStreamWaitEvent(side->main, side->fork, 0);
+    s = side->main;
+  }
   if (!dry) {
     cudaMemsetAsync(dh, 0, (size_t)B * H * 4, s);
     cudaMemsetAsync(dc, 0, (size_t)B * H * 4, s);
@@ -1589,11 +1967,12 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     if (io.targets_host && !late.targets)
       cudaMemcpyAsync(const_cast<float*>(io.targets), io.targets_host, io.targets_bytes, cudaMemcpyHostToDevice, s);
   }
-  int x_waited = 0;   // pieces of x the caller's stream has already waited for
-  auto need_x = [&](int64_t steps) {   // time steps [0, steps) of x are about to be read on `s`
-    while (x_waited < late.x_pieces && (int64_t)x_waited * late.steps_per_piece < steps)
-      cudaStreamWaitEvent(s, late.side->x_ready[x_waited++], 0);
+  int x_waited = 0, x_waited_zx = 0;   // pieces of x the step's stream (the zx stream) has already waited for
+  auto need_x_on = [&](cudaStream_t st, int& waited, int64_t steps) {   // time steps [0, steps) of x are about to be read on `st`
+    while (waited < late.x_pieces && (int64_t)waited * late.steps_per_piece < steps)
+      cudaStreamWaitEvent(st, late.side->x_ready[waited++], 0);
   };
+  auto need_x = [&](int64_t steps) { need_x_on(s, x_waited, steps); };
 
   int t_waited = 0;   // pieces of the targets, counted from the last, the caller's stream has waited for
   auto need_targets = [&](int64_t k_lo) {   // the targets of time steps k_lo .. t are about to be read on `s`
@@ -1619,13 +1998,25 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   };
   auto gemm = [&](const void* A, int64_t lda, bool amn, const void* Bm, int64_t ldb, bool bmn, GemmOut out, int M,
                   int N, int Kc) { gemm_on(s, A, lda, amn, Bm, ldb, bmn, out, M, N, Kc); };
-  SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
   bool side_busy[2] = {false, false};   // GEMMs reading the stages of this parity were put on the side stream
 
   RunTimer* timer = (!dry && io.time_runs) ? run_timer_for_current_device() : nullptr;
   bool targets_waited = false;
   int zx_lo = 0, zx_hi = 0;   // time steps [zx_lo, zx_hi) whose input projections the Zx buffer holds
   float* zleaf = reinterpret_cast<float*>(at(y.off_zleaf));
+  const bool zx_ahead = side && !env::no_zx_ahead();
+  int zx_w = -1;          // windows opened so far, less one
+  float* zx_cur = zx;     // the copy of the buffer that holds the window in use
+  auto project_window = [&](size_t it, int w) {
+    const int k0 = p->tape[items[it].i].k, hi = P.zx_hi[it];
+    cudaEventRecord(side->zx_free[w & 1], s);
+    cudaStreamWaitEvent(side->zx, side->zx_free[w & 1], 0);
+    need_x_on(side->zx, x_waited_zx, hi - 1);
+    const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
+    gemm_on(side->zx, xk, I, false, wp_ih, I, false,
+            GemmOut{GemmOut::STORE_F32, zx + (size_t)(w & 1) * S * B * G, G, bias_p, 0}, (hi - k0) * B, G, I);
+    cudaEventRecord(side->zx_ready[w & 1], side->zx);
+  };
   for (size_t item = 0; item < items.size() && rc == MEBPTT_OK; ++item) {
     const WorkItem& wi = items[item];
     const size_t i = wi.i;
@@ -1639,13 +2030,26 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       if (P.zx_hi[item]) {
         zx_lo = k0;
         zx_hi = P.zx_hi[item];
-        const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
-        need_x(zx_hi - 1);
-        gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
+        if (!zx_ahead) {
+          const __nv_bfloat16* xk = reinterpret_cast<const __nv_bfloat16*>(io.x) + (size_t)(k0 - 1) * B * I;
+          need_x(zx_hi - 1);
+          gemm(xk, I, false, wp_ih, I, false, GemmOut{GemmOut::STORE_F32, zx, G, bias_p, 0}, (zx_hi - zx_lo) * B, G, I);
+        } else {
+          // Windows alternate between the two copies of the buffer.  The projections of a window
+          // depend on x alone: those of the next window are put on a stream of their own as soon
+          // as its copy has no reader left (every run of the window before this one is in the
+          // step's stream by now), so that they run beside this window's runs and what follows
+          // them, on the SMs the persistent kernels leave free.
+          ++zx_w;
+          if (zx_w == 0) project_window(item, 0);
+          cudaStreamWaitEvent(s, side->zx_ready[zx_w & 1], 0);
+          if (P.zx_next[item] >= 0) project_window((size_t)P.zx_next[item], zx_w + 1);
+          zx_cur = zx + (size_t)(zx_w & 1) * S * B * G;
+        }
       }
       ++launches;
       if (!dry && rc == MEBPTT_OK) {
-        FwdRunArgs a{dops + i, n, ws, zx + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
+        FwdRunArgs a{dops + i, n, ws, zx_cur + (size_t)(k0 - zx_lo) * B * G, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
                      io.counters, B, H, fwd_ncg, fwd_bb, fwd_slab ? 1 : 0,
                      (uint32_t)fwd_ncg + ((fault & 1) ? 1u : 0u), (fault & 1) ? fault_poll_limit : (kSpinLimit >> 1),
                      off16(y.plane), off16(y.hsz)};
@@ -1725,12 +2129,20 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
       gemm(dy_c + (size_t)s_lo * B * O, O, false, woutT, O, false,
            GemmOut{GemmOut::STORE_F32, dha + (size_t)s_lo * B * H, H, nullptr, 0}, n * B, H, O);
       if (!dry && rc == MEBPTT_OK) {
+        const bool grouped = P.bwd_grp;
         BwdRunArgs a{bops, n, ws, dha, dz_c, dh, dc, loss_part, loss_t, sync + (size_t)launch_id * 2 * SYNC_STRIDE, status,
-                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts, P.bwd_tb, P.bwd_slab ? 1 : 0,
-                     (uint32_t)ncta + ((fault & 2) ? 1u : 0u), (fault & 2) ? fault_poll_limit : (kSpinLimit >> 1)};
-        void* args[] = {(void*)(bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]), (void*)(bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
+                     io.counters, B, H, S, off16(y.plane), off16(y.hsz), leaf ? zleaf : nullptr, parts,
+                     grouped ? P.bwdg_tb : P.bwd_tb, (grouped || P.bwd_slab) ? 1 : 0,
+                     (uint32_t)(grouped ? P.bwdg_ncg : ncta) + ((fault & 2) ? 1u : 0u),
+                     (fault & 2) ? fault_poll_limit : (kSpinLimit >> 1)};
+        void* args[] = {(void*)(grouped ? &P.tm_dz_g[pb] : bwd_cs ? &tm_dz_b[pb] : &tm_dz[pb]),
+                        (void*)(grouped ? &P.tm_wt_g : bwd_cs ? &tm_wt_c : &tm_wt), (void*)&a};
         const int span = span_begin(timer, 1, n, s);
-        if (bwd_cs) {
+        if (grouped) {
+          if (!cuda_ok(launch_coop((const void*)bwd_run_group_kernel, 2 * P.bwdg_ncg, 192, P.bwdg_smem, s, args, GCS, false),
+                       "backward run launch (groups of batch rows)"))
+            rc = MEBPTT_ERR_CUDA;
+        } else if (bwd_cs) {
           const void* fn = bwd_cs == 8 ? (const void*)bwd_run_cluster_kernel<8> : (const void*)bwd_run_cluster_kernel<4>;
           // launched in plain stream order: early residency of a clustered grid measured no gain
           if (!cuda_ok(launch_coop(fn, ncta, 192, bwdc_smem, s, args, bwd_cs, false), "backward run launch (clusters)"))
@@ -1760,8 +2172,8 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
         gemm_on(gs, dy_c, O, true, hk_c, H, true, GemmOut{GemmOut::ACCUM_F32, io.dW_out, H, nullptr, 0}, O, H, R);
         launches += 2;
         if (!dry && rc == MEBPTT_OK) {
-          launch_on(gs == s, colsum_bf16, dim3((G + 31) / 32), dim3(32, 8), 0, gs, dz_c, R, G, io.db, H);
-          launch_on(gs == s, colsum_bf16, dim3((O + 31) / 32), dim3(32, 8), 0, gs, dy_c, R, O, io.db_out, 0);
+          launch_on(gs == s, colsum_bf16, dim3((G + 63) / 64), dim3(32, 32), 0, gs, dz_c, R, G, io.db, H);
+          launch_on(gs == s, colsum_bf16, dim3((O + 63) / 64), dim3(32, 32), 0, gs, dy_c, R, O, io.db_out, 0);
         }
         if (want_dx)
           gemm_on(gs, dz_c, G, false, wpT_ih, G, false,
@@ -1781,6 +2193,10 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   if (!dry && rc == MEBPTT_OK) {
     launch_pdl(finalize_tc, dim3(1), dim3(32), 0, s, loss_t, (int64_t)y.t, io.loss, io.counters, (int64_t)p->peak_units, status);
     if (!cuda_ok(cudaGetLastError(), "training step (last error)")) rc = MEBPTT_ERR_CUDA;
+  }
+  if (s != caller) {
+    cudaEventRecord(side->join, s);
+    cudaStreamWaitEvent(caller, side->join, 0);
   }
   if (dry) return launches;
   return rc;
