@@ -5,8 +5,8 @@
 //   MEBPTT_NO_PDL=1           launch without programmatic stream serialization
 //   MEBPTT_NO_OVERLAP=1       weight-gradient GEMMs on the caller's stream instead of the side stream;
 //                             host-buffer inputs copied in front of the step instead of beside it
-//   MEBPTT_NO_PRIORITY=1      the step on the caller's stream itself instead of the library's stream of
-//                             the most urgent priority
+//   MEBPTT_PRIORITY=1         the step on a stream of the library's, of the most urgent priority, instead
+//                             of the caller's stream itself
 //   MEBPTT_NO_ZX_AHEAD=1      input projections in the step's stream, when a run needs them, instead of a
 //                             window ahead on a stream of their own
 //   MEBPTT_BWD_CLUSTER=0|4|8  backward run kernel: unclustered (what a profiler that cannot launch
@@ -36,7 +36,7 @@ inline int integer(const char* name) {
 
 inline bool no_pdl() { static const bool v = flag("MEBPTT_NO_PDL"); return v; }
 inline bool no_overlap() { static const bool v = flag("MEBPTT_NO_OVERLAP"); return v; }
-inline bool no_priority() { static const bool v = flag("MEBPTT_NO_PRIORITY"); return v; }
+inline bool priority() { static const bool v = flag("MEBPTT_PRIORITY"); return v; }
 inline bool no_zx_ahead() { static const bool v = flag("MEBPTT_NO_ZX_AHEAD"); return v; }
 inline int bwd_cluster() { static const int v = integer("MEBPTT_BWD_CLUSTER"); return v; }
 inline bool no_bwd_groups() { static const bool v = flag("MEBPTT_NO_BWD_GROUPS"); return v; }

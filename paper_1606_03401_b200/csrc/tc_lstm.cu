@@ -1923,14 +1923,15 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
   const CUtensorMap* tm_dz_b = P.tm_dz_b;
   const int bwd_cs = P.bwd_cs, bwdc_smem = P.bwdc_smem, fwd_ncg = P.fwd_ncg, fwd_smem = P.fwd_smem, fwd_bb = P.fwd_bb;
   const bool fwd_slab = P.fwd_slab;
-  // With streams of its own the library runs the step on one of the most urgent priority, ordered
-  // after what the caller's stream holds and joined to it at the end.  The caller's stream is of the
-  // least urgent priority as a rule, the same as the stream of the weight-gradient GEMMs: a grid of
-  // theirs that becomes eligible together with a kernel of the recurrence would otherwise take the
-  // SMs first as often as not, and every CTA of it runs for tens of microseconds.
+  // On request (a switch in the environment) the step runs on a stream of the library's, of the most
+  // urgent priority, ordered after what the caller's stream holds and joined to it at the end: the
+  // caller's stream is of the least urgent priority as a rule, like the stream of the weight-gradient
+  // GEMMs, whose grids then take free SMs as readily as the kernels of the recurrence do.  Measured
+  // at config 3: 0.46 ms faster at MSM m = 100, 0.4 to 0.7 ms slower at m = 10, m = 32 and with full
+  // memory (the gradient GEMMs fall behind and the step ends waiting for them).  Off by default.
   SideStream* side = (!dry && side_stream) ? side_stream_for_current_device() : nullptr;
   cudaStream_t s = caller;
-  if (side && !env::no_priority()) {
+  if (side && env::priority()) {
     cudaEventRecord(side->fork, caller);
     cudaStreamWaitEvent(side->main, side->fork, 0);
     s = side->main;
