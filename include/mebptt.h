@@ -287,17 +287,22 @@ int64_t mebptt_lstm_launch_count(const mebptt_lstm_desc *desc, const mebptt_plan
  *   entry do not matter and are undefined on exit.
  * stream: a cudaStream_t (NULL = the default stream).
  * Streams and events owned by the library: on the tensor-core path for one-layer bfloat16
- *   problems, the first step on a device creates, and keeps until the process ends, two
- *   non-blocking streams and 22 events without timing.  On the first (lowest priority) run the
+ *   problems, the first step on a device creates, and keeps until the process ends, four
+ *   non-blocking streams and 28 events without timing.  On the first (lowest priority) run the
  *   weight-gradient contractions and bias sums of a finished chunk of time steps, inside the
  *   caller's workspace and output buffers, while the caller's stream goes on with the next chunk;
  *   events order them after the backward steps they read and before the reuse of their staging
  *   buffers, and the caller's stream waits for them before the step's last kernel.  The second
- *   carries the host-to-device copies of mebptt_lstm_train_step_host that overlap the forward
- *   pass.  Everything the call enqueues is therefore complete when `stream` has reached the end
- *   of the call's work; the caller needs no knowledge of the two streams, but must not use the
- *   workspace or the outputs on other streams before that.  mebptt_lstm_train_step_static uses
- *   neither stream.
+ *   (middle priority) computes the input projections of the window of time steps after the one
+ *   the forward runs are reading, into the other of two copies of the window buffer inside the
+ *   workspace; every forward run that opens a window waits for its projections first, so nothing
+ *   of it is left when the step ends.  The third carries the host-to-device copies of
+ *   mebptt_lstm_train_step_host that overlap the forward pass.  The fourth (most urgent
+ *   priority) is used only on request (MEBPTT_PRIORITY=1 in the environment): the step then runs
+ *   there, ordered after what `stream` holds and joined to `stream` at its end.  Everything the
+ *   call enqueues is therefore complete when `stream` has reached the end of the call's work; the
+ *   caller needs no knowledge of these streams, but must not use the workspace or the outputs on
+ *   other streams before that.  mebptt_lstm_train_step_static uses none of them.
  * Outputs (overwritten, not accumulated; all float32):
  *   loss [1]; dW like W; db like b; dW_out [O][H]; db_out [O]; dx [t][B][I] or NULL.
  *   counters: int64[8] -- [0] forward operations executed, [1] backward operations executed,
