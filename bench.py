@@ -364,7 +364,7 @@ def main():
                     "launches": f_n // 3, "ops_per_launch": f_ops / f_n, "us_per_launch": f_ms * 1e3 / f_n,
                     "us_per_op": f_ms * 1e3 / f_ops,
                     "share_of_step": (f_ms / 3) / ms,
-                    "backward_runs": {"kernel": "bwd_run_cluster_kernel", "launches": b_n // 3,
+                    "backward_runs": {"kernel": "bwd_run_group_kernel (bwd_run_cluster_kernel where B <= 32)", "launches": b_n // 3,
                                       "us_per_op": b_ms * 1e3 / max(1, b_ops), "share_of_step": (b_ms / 3) / ms},
                     "traffic_note": ("DRAM bytes per launch = bytes per operation (ncu capture of a 32-operation launch, "
                                      "config 3's layer sizes) x mean operations per launch; null when the kernel's "
