@@ -173,7 +173,11 @@ def test_slot_copy(H, nbytes):
 
 @pytest.mark.parametrize("shape", [dict(input=64, hidden=64, batch=64, t=40, readout=64),
                                    dict(input=72, hidden=200, batch=24, t=37, readout=40),
-                                   dict(input=256, hidden=256, batch=64, t=50, readout=256)])
+                                   dict(input=256, hidden=256, batch=64, t=50, readout=256),
+                                   # two groups of batch rows, the second one ragged; a K-slice per CTA
+                                   # of the backward cluster that is shorter than one copy's box
+                                   dict(input=64, hidden=192, batch=40, t=40, readout=48),
+                                   dict(input=128, hidden=768, batch=56, t=36, readout=64)])
 def test_tensor_core_path_matches_oracle_and_cuda_core_path(H, shape):
     """bf16 shapes the tcgen05 kernels cover: oracle parity, bit identity across plans, and
     agreement with the CUDA-core kernels (same roundings of stored values, other sum order)."""
