@@ -1232,10 +1232,11 @@ __global__ void __launch_bounds__(192, 1) bwd_run_group_kernel(const __grid_cons
 // ------------------------------------------------------------------------------------------
 // Packs the weights once per training step: gate rows permuted to 4 u + q (the four gates of
 // hidden unit u adjacent), W_ih and W_hh split, their transposes for the backward products, the
-// transposed readout matrix, and the permuted bias.
-__global__ void pack_weights(const __nv_bfloat16* W, const float* bias, const __nv_bfloat16* W_out, int I, int H,
-                             int O, __nv_bfloat16* wp_ih, __nv_bfloat16* wp_hh, __nv_bfloat16* wpT_hh,
-                             __nv_bfloat16* wpT_ih, float* bias_p, __nv_bfloat16* woutT) {
+// transposed readout matrix, and the permuted bias.  Element by element: for widths that are not
+// multiples of 8 (the tiled kernel below serves the rest).
+__global__ void pack_weights_scalar(const __nv_bfloat16* W, const float* bias, const __nv_bfloat16* W_out, int I, int H,
+                                    int O, __nv_bfloat16* wp_ih, __nv_bfloat16* wp_hh, __nv_bfloat16* wpT_hh,
+                                    __nv_bfloat16* wpT_ih, float* bias_p, __nv_bfloat16* woutT) {
   grid_dep_wait();
   grid_dep_launch();
   const int G = 4 * H, K = I + H;
@@ -1260,6 +1261,77 @@ __global__ void pack_weights(const __nv_bfloat16* W, const float* bias, const __
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < (size_t)O * H; e += stride) {
     const int o = (int)(e / H), j = (int)(e % H);
     woutT[(size_t)j * O + o] = W_out[e];
+  }
+}
+
+// The same in tiles of 64 x 64 through shared memory, 16 bytes per access on both sides of a
+// transpose (I, H, O multiples of 8).  A block of 256 threads takes tiles in turn: first those of
+// W (tile row = 64 permuted gate rows, i.e. 16 hidden units), then those of W_out.
+__global__ void __launch_bounds__(256) pack_weights(const __nv_bfloat16* W, const float* bias, const __nv_bfloat16* W_out, int I,
+                                                    int H, int O, __nv_bfloat16* wp_ih, __nv_bfloat16* wp_hh,
+                                                    __nv_bfloat16* wpT_hh, __nv_bfloat16* wpT_ih, float* bias_p,
+                                                    __nv_bfloat16* woutT) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // 144-byte rows: 16-byte accesses stay aligned
+  grid_dep_wait();
+  grid_dep_launch();
+  const int G = 4 * H, K = I + H;
+  const int tid = threadIdx.x;
+  const int r = tid >> 2, seg = (tid & 3) * 16;   // this thread's row of a tile and its 16 columns
+  const int tc_w = (K + 63) / 64, tr_w = (G + 63) / 64;
+  const int tc_o = (H + 63) / 64, tr_o = (O + 63) / 64;
+  const int n_w = tc_w * tr_w, n_o = tc_o * tr_o;
+  for (int t = blockIdx.x; t < n_w + n_o; t += gridDim.x) {
+    const bool is_w = t < n_w;
+    const int tt = is_w ? t : t - n_w;
+    const int r0 = (tt / (is_w ? tc_w : tc_o)) * 64, c0 = (tt % (is_w ? tc_w : tc_o)) * 64;
+    const int rows = is_w ? G : O, cols = is_w ? K : H;
+    // ---- in: row r0 + r of the (permuted) source, columns c0 + seg .. + 15
+    const int pr = r0 + r;   // permuted gate row, or row of W_out
+    uint4 v[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+    if (pr < rows) {
+      const size_t src_row = is_w ? (size_t)((pr & 3) * H + (pr >> 2)) : (size_t)pr;
+      const __nv_bfloat16* src = (is_w ? W : W_out) + src_row * cols;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int c = c0 + seg + 8 * h;
+        if (c < cols) v[h] = *reinterpret_cast<const uint4*>(src + c);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) *reinterpret_cast<uint4*>(&tile[r][seg + 8 * h]) = v[h];
+    if (is_w && pr < rows) {
+      // the row-major copies, split at column I (a multiple of 8, so no 16-byte piece straddles it)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int c = c0 + seg + 8 * h;
+        if (c >= cols) continue;
+        if (c < I) *reinterpret_cast<uint4*>(wp_ih + (size_t)pr * I + c) = v[h];
+        else *reinterpret_cast<uint4*>(wp_hh + (size_t)pr * H + (c - I)) = v[h];
+      }
+    }
+    __syncthreads();
+    // ---- out, transposed: column c0 + r of the tile, rows r0 + seg .. + 15
+    const int c = c0 + r;
+    if (c < cols) {
+      __nv_bfloat16* dst = is_w ? (c < I ? (wpT_ih ? wpT_ih + (size_t)c * G : nullptr) : wpT_hh + (size_t)(c - I) * G)
+                                : woutT + (size_t)c * O;
+      if (dst) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int rr = seg + 8 * h;
+          if (r0 + rr >= rows) continue;   // rows is a multiple of 8
+          __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) o[j] = tile[rr + j][r];
+          *reinterpret_cast<uint4*>(dst + r0 + rr) = *reinterpret_cast<const uint4*>(o);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + tid; e < (size_t)G; e += (size_t)gridDim.x * blockDim.x) {
+    const int q = (int)e / H, u = (int)e % H;
+    bias_p[4 * u + q] = bias[e];
   }
 }
 
@@ -1949,8 +2021,9 @@ int64_t run_step(const Layout& y, const Plan* p, const StepPtrs& io, bool want_d
     // (from page-locked memory: an asynchronous copy proper; from pageable memory, which only the
     // allocation-free entry point uses, the call may wait for the stream to reach the copy)
     cudaMemcpyAsync(at(y.off_tape), P.tape, P.tape_entries * sizeof(DevOp), cudaMemcpyHostToDevice, s);
-    launch_pdl(pack_weights, dim3(592), dim3(256), 0, s, reinterpret_cast<const __nv_bfloat16*>(io.W), io.b,
-               reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O, wp_ih, wp_hh, wpT_hh, wpT_ih, bias_p, woutT);
+    launch_pdl((I % 8 == 0 && H % 8 == 0 && O % 8 == 0) ? pack_weights : pack_weights_scalar, dim3(592), dim3(256), 0, s,
+               reinterpret_cast<const __nv_bfloat16*>(io.W), io.b, reinterpret_cast<const __nv_bfloat16*>(io.W_out), I, H, O,
+               wp_ih, wp_hh, wpT_hh, wpT_ih, bias_p, woutT);
     // Peek of the initial state: the caller's (h0, c0) as a hidden block inside the workspace
     launch_pdl(copy16_tc, dim3(64), dim3(256), 0, s, reinterpret_cast<uint4*>(at(y.off_init)),
                reinterpret_cast<const uint4*>(io.h0), (size_t)B * H * 2 / 16);
